@@ -1,0 +1,146 @@
+/*
+ * NOVAK per-parameter optimizer step -- CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the definition the CUDA library is
+ * checked against.  It is plain scalar C in double precision, one element at a
+ * time, in the order the paper gives its phases (Section 5.1: Nesterov
+ * approximation -> moments -> bias correction -> rectification -> direction
+ * -> decoupled decay and update -> lookahead).  It shares no code, header,
+ * table or constant with the CUDA library and is never called by it; only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg load it.
+ *
+ * Readings taken where the paper is ambiguous (each is also listed in the
+ * design notes of the repository):
+ *   - The first-moment bias correction is applied once: the parameter change
+ *     is  -alpha * r_t * m_hat / (sqrt(v_hat) + eps)  (Eq. 24 with Eq. 24a).
+ *     bias1_power = 2 reproduces the literal pairing of Eq. 8 with Eq. 24
+ *     (1/(1-beta1^t) applied twice).                      [parity unpinned]
+ *   - Eq. 13's g~ replaces g in BOTH moment updates (Table 2 lists it under
+ *     gradient processing; the proof of Thm 6.1 writes g_t <- g_t + ...).
+ *   - Eq. 16 is taken literally: beta1*m_hat + (1-beta1)*u.   [parity unpinned]
+ *   - The branch of Eq. 8 is "rho_t >= 5"; the other branch keeps the
+ *     adaptive denominator and sets r_t = 1.
+ *   - Lookahead has two modes.  LAST: slow += alpha_LA*(fast - slow) on steps
+ *     with t mod k == 0.  TRAJ_MEAN: the rule in the proof of Thm 6.2,
+ *     slow += alpha_LA*(mean of the k fast iterates of the window - slow).
+ *     Which of the two is "the" method is a reading.          [parity unpinned]
+ *   - Moments are not touched by a synchronisation.
+ *
+ * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
+ * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
+ */
+#include <math.h>
+#include <stdint.h>
+
+typedef struct {
+    double lr;               /* alpha  > 0                                  */
+    double beta1;            /* [0,1)                                       */
+    double beta2;            /* [0,1)                                       */
+    double eps;              /* > 0                                         */
+    double weight_decay;     /* lambda >= 0                                 */
+    double nesterov_beta;    /* beta_N in [0,1)                             */
+    double lookahead_alpha;  /* alpha_LA in (0,1), used when lookahead_k>0  */
+    int32_t nesterov_variant;/* 0 none, 1 approximation (Eq.13), 2 classical (Eq.16) */
+    int32_t lookahead_k;     /* 0 = lookahead off                           */
+    int32_t lookahead_mode;  /* 0 LAST, 1 TRAJ_MEAN                         */
+    int32_t rectified;       /* 1: Eq. 8-9, 0: r_t = 1 on every step        */
+    int32_t bias1_power;     /* 1 (default reading) or 2                    */
+} novak_oracle_hparams;
+
+typedef struct {
+    double bc1;       /* 1 - beta1^t                        (Eq. 5) */
+    double bc2;       /* 1 - beta2^t                        (Eq. 5) */
+    double rho_inf;   /* Eq. 6 */
+    double rho_t;     /* Eq. 7 */
+    double r_t;       /* Eq. 9, or 1 on the un-rectified branch     */
+    double step_size; /* alpha * r_t / bc1^(bias1_power-1)          */
+    double decay;     /* 1 - alpha*lambda                   (Eq. 18) */
+    int32_t rect_branch; /* 1 when Eq. 8's first case was taken      */
+    int32_t is_sync;     /* 1 when lookahead_k>0 and t mod k == 0    */
+} novak_oracle_scalars;
+
+/* Per-step scalars for the 1-based step index t (Eq. 5-9, 18). */
+void novak_oracle_scalars_at(const novak_oracle_hparams *h, int64_t t,
+                             novak_oracle_scalars *s)
+{
+    long double b1t = powl((long double)h->beta1, (long double)t);
+    long double b2t = powl((long double)h->beta2, (long double)t);
+    s->bc1 = (double)(1.0L - b1t);
+    s->bc2 = (double)(1.0L - b2t);
+    s->rho_inf = 2.0 / (1.0 - h->beta2) - 1.0;
+    s->rho_t = (double)((long double)s->rho_inf
+                        - 2.0L * (long double)t * b2t / (1.0L - b2t));
+    s->rect_branch = 0;
+    s->r_t = 1.0;
+    if (h->rectified && s->rho_t >= 5.0) {
+        double num = (s->rho_t - 4.0) * (s->rho_t - 2.0) * s->rho_inf;
+        double den = (s->rho_inf - 4.0) * (s->rho_inf - 2.0) * s->rho_t;
+        s->r_t = sqrt(num / den);
+        s->rect_branch = 1;
+    }
+    s->step_size = h->lr * s->r_t;
+    if (h->bias1_power == 2)
+        s->step_size /= s->bc1;
+    s->decay = 1.0 - h->lr * h->weight_decay;
+    s->is_sync = (h->lookahead_k > 0 && (t % h->lookahead_k) == 0) ? 1 : 0;
+}
+
+/*
+ * One step (index t, 1-based, i.e. after the counter was incremented) over n
+ * independent elements.  theta, m, v are updated in place; g is read only.
+ * slow is used when lookahead_k > 0 (caller sets slow = theta_0 before the
+ * first step, Eq. 28); acc when lookahead_mode == 1 (caller zeroes it).
+ */
+void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
+                       double *theta, const double *g, double *m, double *v,
+                       double *slow, double *acc)
+{
+    novak_oracle_scalars s;
+    novak_oracle_scalars_at(h, t, &s);
+    const int k = h->lookahead_k;
+
+    for (int64_t i = 0; i < n; ++i) {
+        /* Phase 2: Nesterov approximation, Eq. 13 (m[i] is m_{t-1}). */
+        double gt = g[i];
+        if (h->nesterov_variant == 1)
+            gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
+
+        /* Phase 4: Eq. 1-2. */
+        m[i] = h->beta1 * m[i] + (1.0 - h->beta1) * gt;
+        v[i] = h->beta2 * v[i] + (1.0 - h->beta2) * gt * gt;
+
+        /* Phase 5: Eq. 5. */
+        double m_hat = m[i] / s.bc1;
+        double v_hat = v[i] / s.bc2;
+
+        /* Phase 8: Eq. 17, then Eq. 16 for the classical variant. */
+        double u = m_hat / (sqrt(v_hat) + h->eps);
+        if (h->nesterov_variant == 2)
+            u = h->beta1 * m_hat + (1.0 - h->beta1) * u;
+
+        /* Phase 9: Eq. 18 then Eq. 24 (decay with the base rate alpha). */
+        double theta_fast = theta[i] * s.decay - s.step_size * u;
+
+        /* Phase 10: lookahead. */
+        if (k <= 0) {
+            theta[i] = theta_fast;
+        } else if (h->lookahead_mode == 0) {
+            if (s.is_sync) {
+                theta[i] = slow[i] + h->lookahead_alpha * (theta_fast - slow[i]);
+                slow[i] = theta[i];
+            } else {
+                theta[i] = theta_fast;
+            }
+        } else {
+            acc[i] += theta_fast;
+            if (s.is_sync) {
+                theta[i] = slow[i]
+                         + h->lookahead_alpha * (acc[i] / (double)k - slow[i]);
+                slow[i] = theta[i];
+                acc[i] = 0.0;
+            } else {
+                theta[i] = theta_fast;
+            }
+        }
+    }
+}

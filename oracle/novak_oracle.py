@@ -1,0 +1,192 @@
+"""ctypes front end of the CPU oracle (``novak_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this module, and this module imports nothing from them.
+
+The arithmetic lives in the C file; this module only compiles it (gcc, no
+fast-math), keeps the double-precision state arrays, counts steps and records
+on which steps a lookahead synchronisation happened.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from concurrent.futures import ThreadPoolExecutor
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "novak_oracle.c")
+_LIB = os.path.join(_HERE, "libnovak_oracle.so")
+
+NESTEROV_NONE, NESTEROV_APPROX, NESTEROV_CLASSICAL = 0, 1, 2
+LOOKAHEAD_LAST, LOOKAHEAD_TRAJ_MEAN = 0, 1
+
+
+class HParams(ctypes.Structure):
+    _fields_ = [
+        ("lr", ctypes.c_double),
+        ("beta1", ctypes.c_double),
+        ("beta2", ctypes.c_double),
+        ("eps", ctypes.c_double),
+        ("weight_decay", ctypes.c_double),
+        ("nesterov_beta", ctypes.c_double),
+        ("lookahead_alpha", ctypes.c_double),
+        ("nesterov_variant", ctypes.c_int32),
+        ("lookahead_k", ctypes.c_int32),
+        ("lookahead_mode", ctypes.c_int32),
+        ("rectified", ctypes.c_int32),
+        ("bias1_power", ctypes.c_int32),
+    ]
+
+
+class Scalars(ctypes.Structure):
+    _fields_ = [
+        ("bc1", ctypes.c_double),
+        ("bc2", ctypes.c_double),
+        ("rho_inf", ctypes.c_double),
+        ("rho_t", ctypes.c_double),
+        ("r_t", ctypes.c_double),
+        ("step_size", ctypes.c_double),
+        ("decay", ctypes.c_double),
+        ("rect_branch", ctypes.c_int32),
+        ("is_sync", ctypes.c_int32),
+    ]
+
+
+def compile_oracle(src: str = _SRC, out: str = _LIB, force: bool = False) -> str:
+    """Compile the C oracle into a shared object (skipped when up to date)."""
+    if (not force and os.path.exists(out)
+            and os.path.getmtime(out) >= os.path.getmtime(src)):
+        return out
+    tmp = f"{out}.{os.getpid()}.tmp"
+    subprocess.run(
+        ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fno-fast-math",
+         "-ffp-contract=off", "-o", tmp, src, "-lm"],
+        check=True)
+    os.replace(tmp, out)
+    return out
+
+
+def load_library(path: str | None = None) -> ctypes.CDLL:
+    lib = ctypes.CDLL(path or compile_oracle())
+    lib.novak_oracle_scalars_at.argtypes = [
+        ctypes.POINTER(HParams), ctypes.c_int64, ctypes.POINTER(Scalars)]
+    lib.novak_oracle_scalars_at.restype = None
+    dp = ctypes.POINTER(ctypes.c_double)
+    lib.novak_oracle_step.argtypes = [
+        ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64,
+        dp, dp, dp, dp, dp, dp]
+    lib.novak_oracle_step.restype = None
+    return lib
+
+
+_lib_lock = threading.Lock()
+_default_lib: ctypes.CDLL | None = None
+
+
+def default_library() -> ctypes.CDLL:
+    global _default_lib
+    with _lib_lock:
+        if _default_lib is None:
+            _default_lib = load_library()
+        return _default_lib
+
+
+@dataclass
+class Config:
+    """Hyperparameters in the paper's notation (Algorithm 1, Input)."""
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 1e-2
+    nesterov_variant: int = NESTEROV_APPROX
+    lookahead_k: int = 5
+    lookahead_alpha: float = 0.5
+    nesterov_beta: float | None = None   # None -> beta1
+    lookahead_mode: int = LOOKAHEAD_LAST
+    rectified: bool = True
+    bias1_power: int = 1
+
+    def to_c(self) -> HParams:
+        nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
+        return HParams(self.lr, self.beta1, self.beta2, self.eps,
+                       self.weight_decay, nb, self.lookahead_alpha,
+                       self.nesterov_variant, self.lookahead_k,
+                       self.lookahead_mode, int(self.rectified),
+                       self.bias1_power)
+
+
+def _dptr(a: np.ndarray, offset: int = 0):
+    assert a.dtype == np.float64 and a.flags.c_contiguous
+    return ctypes.cast(a.ctypes.data + 8 * offset,
+                       ctypes.POINTER(ctypes.c_double))
+
+
+class Oracle:
+    """The optimizer over a list of tensors, state held in float64.
+
+    ``params`` are the initial values (any float dtype; widened exactly).
+    ``step(grads)`` advances every tensor by one NOVAK step.
+    """
+
+    def __init__(self, cfg: Config, params, lib: ctypes.CDLL | None = None):
+        self.cfg = cfg
+        self.h = cfg.to_c()
+        self.lib = lib or default_library()
+        self.theta = [np.ascontiguousarray(np.asarray(p, dtype=np.float64)).reshape(-1).copy()
+                      for p in params]
+        self.m = [np.zeros_like(p) for p in self.theta]
+        self.v = [np.zeros_like(p) for p in self.theta]
+        self.slow = [p.copy() for p in self.theta] if cfg.lookahead_k > 0 else None
+        self.acc = ([np.zeros_like(p) for p in self.theta]
+                    if cfg.lookahead_k > 0 and cfg.lookahead_mode == LOOKAHEAD_TRAJ_MEAN
+                    else None)
+        self.t = 0
+        self.sync_steps: list[int] = []
+        self.rect_flags: list[int] = []
+
+    def scalars(self, t: int) -> Scalars:
+        s = Scalars()
+        self.lib.novak_oracle_scalars_at(ctypes.byref(self.h), t, ctypes.byref(s))
+        return s
+
+    def _run(self, i: int, g: np.ndarray, lo: int, hi: int):
+        null = ctypes.POINTER(ctypes.c_double)()
+        self.lib.novak_oracle_step(
+            ctypes.byref(self.h), self.t, hi - lo,
+            _dptr(self.theta[i], lo), _dptr(g, lo),
+            _dptr(self.m[i], lo), _dptr(self.v[i], lo),
+            _dptr(self.slow[i], lo) if self.slow is not None else null,
+            _dptr(self.acc[i], lo) if self.acc is not None else null)
+
+    def step(self, grads, threads: int = 1):
+        """One step.  ``threads`` > 1 splits each tensor into disjoint element
+        ranges handled by separate host threads (elements are independent)."""
+        assert len(grads) == len(self.theta)
+        self.t += 1
+        s = self.scalars(self.t)
+        self.rect_flags.append(int(s.rect_branch))
+        if s.is_sync:
+            self.sync_steps.append(self.t)
+        gs = [np.ascontiguousarray(np.asarray(g, dtype=np.float64)).reshape(-1)
+              for g in grads]
+        for i, g in enumerate(gs):
+            assert g.size == self.theta[i].size
+        if threads <= 1:
+            for i, g in enumerate(gs):
+                self._run(i, g, 0, g.size)
+            return
+        jobs = []
+        for i, g in enumerate(gs):
+            n = g.size
+            parts = min(threads, max(1, n // 65536))
+            bounds = [n * j // parts for j in range(parts + 1)]
+            jobs += [(i, g, bounds[j], bounds[j + 1]) for j in range(parts)]
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(lambda a: self._run(*a), jobs))

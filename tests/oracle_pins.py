@@ -1,0 +1,439 @@
+"""Pins for the CPU oracle: facts fixed by the paper and by mathematics.
+
+Every pin is a function ``pin_xxx(lib)`` that raises AssertionError when the
+oracle library ``lib`` (a ctypes handle of the compiled C file) violates it.
+They are collected in ``ALL_PINS`` so that ``test_oracle_pins.py`` can run
+them on the real oracle and ``test_oracle_mutants.py`` on deliberately broken
+copies of it (each planted mistake has to trip at least one pin).
+
+None of the pins re-types the oracle's recurrences: they use closed forms
+(geometric series), explicit unrolled sums, library optimizers
+(torch.optim.AdamW / RAdam in float64) and invariants (Prop. 6.3-6.5).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+import torch
+
+from oracle import novak_oracle as O
+
+
+def _mk(lib, params, **kw):
+    return O.Oracle(O.Config(**kw), params, lib=lib)
+
+
+def _close(a, b, rtol=1e-12, atol=1e-15, what=""):
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    err = np.abs(a - b)
+    tol = atol + rtol * np.abs(b)
+    assert np.all(err <= tol), f"{what}: max err {err.max():.3e} (tol {tol.min():.3e})"
+
+
+_C = np.array([0.3, -0.02, 1e-4, -7.0, 0.0, 2.5e-3])
+_TH0 = np.array([0.05, -0.4, 1.0, 0.0, 0.7, -1e-3])
+
+
+# --------------------------------------------------------------------------
+# Moments and update under a constant gradient (Eq. 1-2, 5, 17, 18, 24)
+# --------------------------------------------------------------------------
+def pin_constant_grad_none(lib):
+    """g == c for all t  =>  m_T = c(1-b1^T), v_T = c^2(1-b2^T), so m_hat = c,
+    v_hat = c^2, u = c/(|c|+eps) and, with r_t = 1,
+    theta_T = theta_0 d^T - alpha u (1-d^T)/(1-d),  d = 1-alpha*lambda."""
+    b1, b2, lr, wd, eps, T = 0.9, 0.999, 1e-3, 1e-2, 1e-8, 37
+    o = _mk(lib, [_TH0], lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd,
+            nesterov_variant=O.NESTEROV_NONE, lookahead_k=0, rectified=False)
+    for _ in range(T):
+        o.step([_C])
+    _close(o.m[0], _C * (1 - b1 ** T), what="m_T")
+    _close(o.v[0], _C ** 2 * (1 - b2 ** T), what="v_T")
+    d = 1 - lr * wd
+    u = _C / (np.abs(_C) + eps)
+    geo = (1 - d ** T) / (1 - d)
+    _close(o.theta[0], _TH0 * d ** T - lr * u * geo, rtol=1e-11, what="theta_T")
+
+
+def pin_constant_grad_approx(lib):
+    """Eq. 13 feeding both moments.  With b = b1 - (1-b1) bN:
+    m_t = c (1 - b^t),  g~_t = c (1 + bN b^(t-1)),
+    v_T = (1-b2) sum_i b2^(T-i) g~_i^2   (explicit sum, no recurrence)."""
+    b1, b2, bN, T = 0.9, 0.999, 0.7, 23
+    o = _mk(lib, [_TH0], beta1=b1, beta2=b2, nesterov_variant=O.NESTEROV_APPROX,
+            nesterov_beta=bN, lookahead_k=0, rectified=False)
+    for _ in range(T):
+        o.step([_C])
+    b = b1 - (1 - b1) * bN
+    _close(o.m[0], _C * (1 - b ** T), what="m_T approx")
+    gt = [_C * (1 + bN * b ** (i - 1)) for i in range(1, T + 1)]
+    v = sum((1 - b2) * b2 ** (T - i) * gt[i - 1] ** 2 for i in range(1, T + 1))
+    _close(o.v[0], v, what="v_T approx")
+
+
+def pin_constant_grad_classical(lib):
+    """Eq. 16 literal under constant c: u = b1 c + (1-b1) c/(|c|+eps)."""
+    b1, lr, wd, eps, T = 0.8, 2e-3, 0.05, 1e-8, 11
+    o = _mk(lib, [_TH0], lr=lr, beta1=b1, eps=eps, weight_decay=wd,
+            nesterov_variant=O.NESTEROV_CLASSICAL, lookahead_k=0, rectified=False)
+    for _ in range(T):
+        o.step([_C])
+    d = 1 - lr * wd
+    u = b1 * _C + (1 - b1) * _C / (np.abs(_C) + eps)
+    _close(o.theta[0], _TH0 * d ** T - lr * u * (1 - d ** T) / (1 - d),
+           rtol=1e-11, what="theta_T classical")
+
+
+# --------------------------------------------------------------------------
+# Unrolled-sum brute force with random gradients (no recurrence anywhere)
+# --------------------------------------------------------------------------
+def _unrolled(th0, G, lr, b1, b2, eps, wd, variant, bN, r):
+    """theta_T from explicit sums.  G: (T, n) gradients; r: (T,) step factors."""
+    T = G.shape[0]
+    if variant == O.NESTEROV_APPROX:
+        b = b1 - (1 - b1) * bN
+        w = (1 - b1) * (1 + bN)
+        M = [sum(w * b ** (t - i) * G[i - 1] for i in range(1, t + 1))
+             for t in range(0, T + 1)]                      # M[t] = m_t, M[0] = 0
+        Gt = [(1 + bN) * G[t - 1] - bN * M[t - 1] for t in range(1, T + 1)]
+    else:
+        M = [sum((1 - b1) * b1 ** (t - i) * G[i - 1] for i in range(1, t + 1))
+             for t in range(0, T + 1)]
+        Gt = [G[t - 1] for t in range(1, T + 1)]
+    d = 1 - lr * wd
+    total = th0 * d ** T
+    us = []
+    for t in range(1, T + 1):
+        v = sum((1 - b2) * b2 ** (t - i) * Gt[i - 1] ** 2 for i in range(1, t + 1))
+        mh = M[t] / (1 - b1 ** t)
+        vh = v / (1 - b2 ** t)
+        u = mh / (np.sqrt(vh) + eps)
+        if variant == O.NESTEROV_CLASSICAL:
+            u = b1 * mh + (1 - b1) * u
+        us.append(u)
+        total = total - d ** (T - t) * lr * r[t - 1] * u
+    return total, M[T], us
+
+
+def pin_unrolled_random(lib):
+    rng = np.random.default_rng(7)
+    T, n = 14, 9
+    G = rng.normal(0, 1e-2, size=(T, n))
+    G[3, 2] = 0.0
+    th0 = rng.normal(0, 0.05, size=n)
+    lr, b1, b2, eps, wd, bN = 3e-3, 0.85, 0.98, 1e-8, 0.02, 0.6
+    for variant in (O.NESTEROV_NONE, O.NESTEROV_APPROX, O.NESTEROV_CLASSICAL):
+        o = _mk(lib, [th0], lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd,
+                nesterov_variant=variant, nesterov_beta=bN, lookahead_k=0,
+                rectified=False)
+        for t in range(T):
+            o.step([G[t]])
+        th, mT, _ = _unrolled(th0, G, lr, b1, b2, eps, wd, variant, bN, np.ones(T))
+        _close(o.m[0], mT, rtol=1e-11, atol=1e-16, what=f"m unrolled v{variant}")
+        _close(o.theta[0], th, rtol=1e-10, atol=1e-14, what=f"theta unrolled v{variant}")
+
+
+# --------------------------------------------------------------------------
+# Library special cases
+# --------------------------------------------------------------------------
+def pin_adamw_library(lib):
+    """rectified off, Nesterov none, no lookahead == torch.optim.AdamW (fp64),
+    step for step (same eps placement: sqrt(v_hat)+eps)."""
+    g = torch.Generator().manual_seed(11)
+    T, n = 25, 33
+    th0 = torch.randn(n, generator=g, dtype=torch.float64) * 0.05
+    G = torch.randn(T, n, generator=g, dtype=torch.float64) * 1e-2
+    lr, b1, b2, eps, wd = 1e-3, 0.9, 0.999, 1e-8, 1e-2
+    p = th0.clone().requires_grad_(True)
+    opt = torch.optim.AdamW([p], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd,
+                            foreach=False)
+    o = _mk(lib, [th0.numpy()], lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd,
+            nesterov_variant=O.NESTEROV_NONE, lookahead_k=0, rectified=False)
+    for t in range(T):
+        p.grad = G[t].clone()
+        opt.step()
+        o.step([G[t].numpy()])
+        _close(o.theta[0], p.detach().numpy(), rtol=1e-12, atol=1e-16,
+               what=f"AdamW step {t + 1}")
+
+
+def pin_radam_library(lib):
+    """On rectified steps the per-step change theta_t - d*theta_{t-1} equals
+    torch.optim.RAdam's (decoupled decay, fp64) when eps is negligible; this
+    fixes r_t (Eq. 6-9), both bias corrections and the decay factor.  The
+    earlier steps differ by design (the paper keeps the denominator there)."""
+    g = torch.Generator().manual_seed(5)
+    T, n = 40, 17
+    th0 = torch.randn(n, generator=g, dtype=torch.float64) * 0.05
+    G = torch.randn(T, n, generator=g, dtype=torch.float64) * 1e-2
+    lr, wd, eps = 1e-3, 1e-2, 1e-30
+    for b1, b2 in ((0.9, 0.999), (0.8, 0.99)):
+        p = th0.clone().requires_grad_(True)
+        opt = torch.optim.RAdam([p], lr=lr, betas=(b1, b2), eps=eps, weight_decay=wd,
+                                decoupled_weight_decay=True, foreach=False)
+        o = _mk(lib, [th0.numpy()], lr=lr, beta1=b1, beta2=b2, eps=eps,
+                weight_decay=wd, nesterov_variant=O.NESTEROV_NONE, lookahead_k=0,
+                rectified=True)
+        d = 1 - lr * wd
+        n_rect = 0
+        for t in range(1, T + 1):
+            p_prev = p.detach().clone().numpy()
+            o_prev = o.theta[0].copy()
+            p.grad = G[t - 1].clone()
+            opt.step()
+            o.step([G[t - 1].numpy()])
+            if o.rect_flags[-1]:
+                n_rect += 1
+                _close(o.theta[0] - d * o_prev, p.detach().numpy() - d * p_prev,
+                       rtol=1e-9, atol=1e-18, what=f"RAdam delta t={t} b2={b2}")
+        assert n_rect >= T - 6
+
+
+# --------------------------------------------------------------------------
+# Host scalars (Eq. 5-9)
+# --------------------------------------------------------------------------
+def _scalars(lib, t, **kw):
+    o = _mk(lib, [np.zeros(1)], **kw)
+    return o.scalars(t)
+
+
+def pin_scalars(lib):
+    # rho_1 == 1 for every beta2: rho_inf - 2 b/(1-b) = (1+b)/(1-b) - 2b/(1-b).
+    for b2 in (0.5, 0.9, 0.99, 0.999, 0.9999):
+        s = _scalars(lib, 1, beta2=b2)
+        assert abs(s.rho_t - 1.0) < 1e-9 * s.rho_inf, (b2, s.rho_t)
+        assert abs(s.rho_inf - (1 + b2) / (1 - b2)) < 1e-9 * s.rho_inf
+    # beta2 = 0.999: rho_inf = 1999; first rectified step is t = 6.
+    flags = [_scalars(lib, t, beta2=0.999).rect_branch for t in range(1, 12)]
+    assert flags == [0] * 5 + [1] * 6, flags
+    assert abs(_scalars(lib, 1, beta2=0.999).rho_inf - 1999.0) < 1e-9
+    # rho_t increases towards rho_inf; r_t in (0,1] and -> 1 (Prop. 6.4).
+    prev_rho, prev_r = -1.0, 0.0
+    for t in (1, 2, 5, 6, 7, 20, 100, 1000, 10 ** 4, 10 ** 5, 10 ** 6):
+        s = _scalars(lib, t, beta2=0.999)
+        # strictly increasing until beta2^t underflows against rho_inf
+        assert s.rho_t <= s.rho_inf
+        assert s.rho_t > prev_rho or (t >= 10 ** 5 and s.rho_t == prev_rho)
+        prev_rho = s.rho_t
+        if s.rect_branch:
+            assert 0.0 < s.r_t <= 1.0
+            assert s.r_t > prev_r or (t >= 10 ** 5 and s.r_t == prev_r)
+            prev_r = s.r_t
+        else:
+            assert s.r_t == 1.0
+    assert _scalars(lib, 10 ** 6, beta2=0.999).r_t > 0.9999
+    # r_t at the threshold rho_t = 5 in closed form: with rho_t -> 5 exactly,
+    # r^2 = 3*rho_inf / (5 (rho_inf-4)(rho_inf-2)); r_6 must sit just above it.
+    s6 = _scalars(lib, 6, beta2=0.999)
+    r5 = math.sqrt(3 * 1999.0 / (5 * 1995.0 * 1997.0))
+    assert r5 < s6.r_t < 2 * r5, (s6.r_t, r5)
+    # bias corrections against the log form 1 - exp(t log beta) (Section 5.8).
+    for t in (1, 3, 10, 1000, 123456):
+        s = _scalars(lib, t, beta1=0.9, beta2=0.999)
+        assert abs(s.bc1 + math.expm1(t * math.log(0.9))) < 1e-15
+        assert abs(s.bc2 + math.expm1(t * math.log(0.999))) < 1e-15
+    # rectified = False never takes the first case of Eq. 8.
+    assert _scalars(lib, 50, beta2=0.999, rectified=False).rect_branch == 0
+    # rho_inf <= 5 (beta2 <= 2/3): never rectified, nothing undefined.
+    for t in (1, 10, 1000):
+        s = _scalars(lib, t, beta2=0.6)
+        assert s.rect_branch == 0 and s.r_t == 1.0
+    # decay uses the base rate alpha (Eq. 18), sync flags follow t mod k.
+    s = _scalars(lib, 10, lr=0.25, weight_decay=0.5, lookahead_k=5)
+    assert s.decay == 1 - 0.125 and s.is_sync == 1
+    assert _scalars(lib, 11, lookahead_k=5).is_sync == 0
+    assert _scalars(lib, 10, lookahead_k=0).is_sync == 0
+
+
+def pin_rectified_step_scaling(lib):
+    """On a rectified step the change is r_t times the un-rectified one, and
+    r_t is the same number the scalar routine reports (Eq. 8 first case)."""
+    rng = np.random.default_rng(3)
+    th0, G = rng.normal(0, 0.05, 5), rng.normal(0, 1e-2, (9, 5))
+    a = _mk(lib, [th0], weight_decay=0.0, lookahead_k=0, rectified=True,
+            nesterov_variant=O.NESTEROV_NONE)
+    b = _mk(lib, [th0], weight_decay=0.0, lookahead_k=0, rectified=False,
+            nesterov_variant=O.NESTEROV_NONE)
+    for t in range(1, 10):
+        pa, pb = a.theta[0].copy(), b.theta[0].copy()
+        a.step([G[t - 1]])
+        b.step([G[t - 1]])
+        r = a.scalars(t).r_t
+        _close(a.theta[0] - pa, r * (b.theta[0] - pb), rtol=1e-9, atol=1e-18,
+               what=f"r_t scaling t={t}")
+        if t <= 5:
+            assert r == 1.0
+        else:
+            assert r < 0.1
+
+
+# --------------------------------------------------------------------------
+# Decoupled decay (Prop. 6.5) and lookahead (Eq. 28-31, Thm 6.2)
+# --------------------------------------------------------------------------
+def pin_pure_decay(lib):
+    """g == 0: m = v = 0, u = 0/(0+eps) = 0, theta_t = theta_0 (1-alpha*lambda)^t
+    for every variant; with LAST lookahead each window maps S to
+    S (1 + a (d^k - 1))."""
+    lr, wd, T = 0.05, 0.3, 17
+    d = 1 - lr * wd
+    z = np.zeros_like(_TH0)
+    for variant in (0, 1, 2):
+        o = _mk(lib, [_TH0], lr=lr, weight_decay=wd, nesterov_variant=variant,
+                lookahead_k=0)
+        for _ in range(T):
+            o.step([z])
+        _close(o.theta[0], _TH0 * d ** T, what=f"pure decay v{variant}")
+        assert not o.m[0].any() and not o.v[0].any()
+    k, a = 5, 0.5
+    o = _mk(lib, [_TH0], lr=lr, weight_decay=wd, lookahead_k=k, lookahead_alpha=a)
+    for _ in range(T):
+        o.step([z])
+    w = (1 + a * (d ** k - 1)) ** (T // k)
+    _close(o.theta[0], _TH0 * w * d ** (T % k), what="decay with LAST lookahead")
+    _close(o.slow[0], _TH0 * w, what="slow after decay windows")
+    assert o.sync_steps == [5, 10, 15]
+
+
+def pin_lookahead_last(lib):
+    """After k steps slow <- slow + a (fast - slow), where fast is what k plain
+    steps (no lookahead) produce from the same start; moments are untouched;
+    the second window starts from the synchronised point."""
+    rng = np.random.default_rng(2)
+    k, a, n = 4, 0.3, 7
+    th0, G = rng.normal(0, 0.05, n), rng.normal(0, 1e-2, (2 * k, n))
+    la = _mk(lib, [th0], lookahead_k=k, lookahead_alpha=a)
+    pl = _mk(lib, [th0], lookahead_k=0)
+    for t in range(k):
+        la.step([G[t]])
+        pl.step([G[t]])
+        if t < k - 1:
+            _close(la.theta[0], pl.theta[0], what="fast weights before sync")
+            _close(la.slow[0], th0, what="slow untouched before sync")
+    want = th0 + a * (pl.theta[0] - th0)
+    _close(la.theta[0], want, what="theta at sync")
+    _close(la.slow[0], want, what="slow at sync")
+    _close(la.m[0], pl.m[0], what="m untouched by sync")
+    _close(la.v[0], pl.v[0], what="v untouched by sync")
+    # Second window: continue the plain run from the synchronised point.
+    pl.theta[0][:] = want
+    for t in range(k, 2 * k):
+        la.step([G[t]])
+        pl.step([G[t]])
+    _close(la.theta[0], want + a * (pl.theta[0] - want), what="second sync")
+    assert la.sync_steps == [k, 2 * k] and la.t == 2 * k
+
+
+def pin_lookahead_traj_mean(lib):
+    """TRAJ_MEAN: slow <- slow + a (mean of the window's k fast iterates - slow)
+    (proof of Thm 6.2); k = 1 coincides with LAST; a constant displacement d per
+    step gives slow + a d (k+1)/2."""
+    rng = np.random.default_rng(4)
+    k, a, n = 5, 0.6, 6
+    th0, G = rng.normal(0, 0.05, n), rng.normal(0, 1e-2, (2 * k, n))
+    tm = _mk(lib, [th0], lookahead_k=k, lookahead_alpha=a,
+             lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN)
+    pl = _mk(lib, [th0], lookahead_k=0)
+    start = th0.copy()
+    for w in range(2):
+        its = []
+        for t in range(w * k, (w + 1) * k):
+            tm.step([G[t]])
+            pl.step([G[t]])
+            its.append(pl.theta[0].copy())
+        want = start + a * (np.mean(its, axis=0) - start)
+        _close(tm.theta[0], want, what=f"traj-mean sync {w}")
+        _close(tm.slow[0], want, what=f"traj-mean slow {w}")
+        assert not tm.acc[0].any()
+        pl.theta[0][:] = want
+        start = want
+    # k = 1
+    x = _mk(lib, [th0], lookahead_k=1, lookahead_alpha=a,
+            lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN)
+    y = _mk(lib, [th0], lookahead_k=1, lookahead_alpha=a)
+    for t in range(4):
+        x.step([G[t]])
+        y.step([G[t]])
+    _close(x.theta[0], y.theta[0], what="traj-mean k=1 == last")
+    # constant displacement: constant g, no decay, r=1 -> each step moves by
+    # dlt = -lr * c/(|c|+eps);  mean of iterates = S + dlt (k+1)/2.
+    lr, eps = 1e-2, 1e-8
+    o = _mk(lib, [_TH0], lr=lr, eps=eps, weight_decay=0.0, rectified=False,
+            nesterov_variant=O.NESTEROV_NONE, lookahead_k=k, lookahead_alpha=a,
+            lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN)
+    for _ in range(k):
+        o.step([_C])
+    dlt = -lr * _C / (np.abs(_C) + eps)
+    _close(o.theta[0], _TH0 + a * dlt * (k + 1) / 2, rtol=1e-11, what="const displacement")
+
+
+def pin_bias1_power(lib):
+    """bias1_power = 2 divides the step by (1 - beta1^t) once more (Eq. 8 used
+    together with Eq. 24); nothing else changes."""
+    rng = np.random.default_rng(9)
+    th0, G = rng.normal(0, 0.05, 4), rng.normal(0, 1e-2, (8, 4))
+    a = _mk(lib, [th0], weight_decay=0.0, lookahead_k=0, bias1_power=1)
+    b = _mk(lib, [th0], weight_decay=0.0, lookahead_k=0, bias1_power=2)
+    for t in range(1, 9):
+        pa, pb = a.theta[0].copy(), b.theta[0].copy()
+        a.step([G[t - 1]])
+        b.step([G[t - 1]])
+        _close((b.theta[0] - pb) * (1 - 0.9 ** t), a.theta[0] - pa, rtol=1e-9,
+               atol=1e-18, what=f"bias1_power t={t}")
+        _close(a.m[0], b.m[0])
+
+
+# --------------------------------------------------------------------------
+# Invariants (Prop. 6.3) and structure
+# --------------------------------------------------------------------------
+def pin_moment_bounds(lib):
+    """|m_t| <= max_i |g~_i| and v_t <= max_i g~_i^2 element-wise (Prop. 6.3),
+    v_t >= 0; g~ = g for variants none/classical."""
+    rng = np.random.default_rng(1)
+    T, n = 60, 50
+    G = rng.normal(0, 1e-2, (T, n)) * rng.integers(0, 2, (T, n))
+    for variant in (O.NESTEROV_NONE, O.NESTEROV_CLASSICAL):
+        o = _mk(lib, [rng.normal(0, 0.05, n)], nesterov_variant=variant)
+        for t in range(T):
+            o.step([G[t]])
+            gmax = np.abs(G[: t + 1]).max(axis=0)
+            assert np.all(np.abs(o.m[0]) <= gmax + 1e-18)
+            assert np.all(o.v[0] <= gmax ** 2 + 1e-24) and np.all(o.v[0] >= 0)
+
+
+def pin_elements_independent(lib):
+    """Splitting a tensor, permuting tensors or threading the element ranges
+    does not change any element (the step has no cross-element term)."""
+    rng = np.random.default_rng(8)
+    n, T = 200_000, 7
+    th0 = rng.normal(0, 0.05, n)
+    G = rng.normal(0, 1e-2, (T, n))
+    whole = _mk(lib, [th0], lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN, lookahead_k=3)
+    parts = _mk(lib, [th0[:77], th0[77:1000], th0[1000:]],
+                lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN, lookahead_k=3)
+    thr = _mk(lib, [th0], lookahead_mode=O.LOOKAHEAD_TRAJ_MEAN, lookahead_k=3)
+    for t in range(T):
+        whole.step([G[t]])
+        parts.step([G[t][:77], G[t][77:1000], G[t][1000:]])
+        thr.step([G[t]], threads=3)
+    assert np.array_equal(np.concatenate(parts.theta), whole.theta[0])
+    assert np.array_equal(thr.theta[0], whole.theta[0])
+    assert np.array_equal(np.concatenate(parts.slow), whole.slow[0])
+
+
+ALL_PINS = [
+    pin_constant_grad_none,
+    pin_constant_grad_approx,
+    pin_constant_grad_classical,
+    pin_unrolled_random,
+    pin_adamw_library,
+    pin_radam_library,
+    pin_scalars,
+    pin_rectified_step_scaling,
+    pin_pure_decay,
+    pin_lookahead_last,
+    pin_lookahead_traj_mean,
+    pin_bias1_power,
+    pin_moment_bounds,
+    pin_elements_independent,
+]

@@ -1,0 +1,65 @@
+"""Each plausible mistake planted in the oracle must trip at least one pin.
+
+The mistake is planted in a copy of the oracle's C source (text replacement),
+compiled on the CPU into a temporary library and run through the same pins as
+the real oracle.  A mutant that passes every pin would mean the pins cannot
+tell the oracle from a wrong one.
+"""
+import os
+
+import pytest
+
+from oracle import novak_oracle as O
+from oracle_pins import ALL_PINS
+
+SRC = os.path.join(os.path.dirname(O.__file__), "novak_oracle.c")
+
+# (name, text in the oracle, replacement)
+MUTANTS = [
+    ("m_sign", "(1.0 - h->beta1) * gt;", "(1.0 + h->beta1) * gt;"),
+    ("v_not_squared", "(1.0 - h->beta2) * gt * gt;", "(1.0 - h->beta2) * gt;"),
+    ("v_uses_beta1", "h->beta2 * v[i]", "h->beta1 * v[i]"),
+    ("approx_sign", "h->nesterov_beta * (g[i] - m[i]);", "h->nesterov_beta * (m[i] - g[i]);"),
+    ("approx_uses_new_m_only_first_moment",
+     "(1.0 - h->beta2) * gt * gt;", "(1.0 - h->beta2) * g[i] * g[i];"),
+    ("vhat_uses_bc1", "double v_hat = v[i] / s.bc2;", "double v_hat = v[i] / s.bc1;"),
+    ("mhat_uses_bc2", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i] / s.bc2;"),
+    ("mhat_uncorrected", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i];"),
+    ("eps_inside_root", "(sqrt(v_hat) + h->eps)", "sqrt(v_hat + h->eps)"),
+    ("update_sign", "theta[i] * s.decay - s.step_size * u;", "theta[i] * s.decay + s.step_size * u;"),
+    ("decay_without_lr", "1.0 - h->lr * h->weight_decay;", "1.0 - h->weight_decay;"),
+    ("decay_with_rectified_rate", "1.0 - h->lr * h->weight_decay;",
+     "1.0 - h->lr * s->r_t * h->weight_decay;"),
+    ("classical_swapped", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
+     "u = (1.0 - h->beta1) * m_hat + h->beta1 * u;"),
+    ("last_sync_sign", "h->lookahead_alpha * (theta_fast - slow[i]);",
+     "h->lookahead_alpha * (slow[i] - theta_fast);"),
+    ("sync_off_by_one", "(t % h->lookahead_k) == 0", "(t % h->lookahead_k) == 1"),
+    ("rho_drops_t", "2.0L * (long double)t * b2t", "2.0L * b2t"),
+    ("rho_uses_beta1", "- 2.0L * (long double)t * b2t / (1.0L - b2t)",
+     "- 2.0L * (long double)t * b1t / (1.0L - b1t)"),
+    ("threshold_textbook", "s->rho_t >= 5.0", "s->rho_t > 4.0"),
+    ("r_inverted", "sqrt(num / den)", "sqrt(den / num)"),
+    ("r_not_rooted", "sqrt(num / den)", "(num / den)"),
+    ("traj_mean_not_divided", "acc[i] / (double)k", "acc[i]"),
+    ("traj_acc_not_reset", "acc[i] = 0.0;", ";"),
+    ("bias1_power_ignored", "if (h->bias1_power == 2)", "if (0)"),
+    ("rectified_flag_ignored", "if (h->rectified && s->rho_t >= 5.0)", "if (s->rho_t >= 5.0)"),
+]
+
+
+@pytest.mark.parametrize("name,old,new", MUTANTS, ids=[m[0] for m in MUTANTS])
+def test_mutant_is_caught(name, old, new, tmp_path):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, f"mutation site for {name} not found in the oracle"
+    src = tmp_path / "mutant.c"
+    src.write_text(text.replace(old, new))
+    lib = O.load_library(O.compile_oracle(str(src), str(tmp_path / "mutant.so"), force=True))
+    caught = []
+    for pin in ALL_PINS:
+        try:
+            pin(lib)
+        except AssertionError:
+            caught.append(pin.__name__)
+            break
+    assert caught, f"mutant {name} passed every pin"
