@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the NOVAK per-parameter optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
+
+One "step" = one novak_step (one fused kernel launch) over a whole synthetic
+parameter set.  Prints ONE JSON line (rank 0).  Default workload: the
+ResNet-50-shaped set (161 tensors, 25,557,032 fp32 parameters), the
+configuration the headline metric is quoted on.
+
+  value     parameter updates/s with everything resident in HBM (CUDA events
+            around exactly K steps, max over ranks).
+  roofline  algorithmic bytes per launch / average launch duration against the
+            measured HBM copy rate of this machine (MEASURED_PEAKS.json).
+  e2e       the same metric through novak_step_host: gradients start in pinned
+            host memory, updated parameters are copied back, inside the timed
+            region.
+  cpu_baseline  the CPU oracle, as it stands, on the host cores (reported
+            baseline, not a target).
+
+With N > 1 (torchrun) every rank steps its own replica of the workload on its
+own GPU: the step has no cross-element term, hence no collective on the data
+path; only the barrier and the MAX of the timings use the process group.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "parameter updates/sec per novak_step"
+UNIT = "param-updates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per element and launch from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of the step kernel,
+# averaged over the sync schedule); None until a capture exists for the workload.
+NCU_DRAM_BYTES_PER_ELEM = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="workload index 0..4")
+    ap.add_argument("--lookahead-mode", default="last", choices=["last", "traj_mean"])
+    ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
+    ap.add_argument("--chunk-elems", type=int, default=None)
+    ap.add_argument("--ctas-per-sm", type=int, default=None)
+    ap.add_argument("--serpentine", type=int, default=None)
+    ap.add_argument("--lib", default=None, help="alternative libnovak.so (tuning builds)")
+    ap.add_argument("--e2e-steps", type=int, default=30)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    return ap.parse_args()
+
+
+def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int) -> int:
+    """Bytes the method itself has to move for one element on step t: theta, g, m, v
+    read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
+    arrays on the steps that touch them."""
+    b = 12 + grad_bytes + 12
+    if k <= 0:
+        return b
+    sync = t % k == 0
+    if mode == "last" or k == 1:
+        if t == 1:
+            b += 4                       # slow <- theta_0
+        if sync:
+            b += 4 if t == 1 else 8      # slow read (not at t=1) + written
+        return b
+    first = (t - 1) % k == 0
+    if t == 1:
+        b += 4
+    if not first:
+        b += 4                           # running sum read
+    if sync:
+        b += 8                           # slow read + written
+    else:
+        b += 4                           # running sum written
+    return b
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, device_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception as exc:  # pragma: no cover
+            self.error = str(exc)
+
+    _NAMES = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+        0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+        0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self._NAMES.items():
+                    if mask & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [],
+                    "note": "no NVML samples"}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def run_reference(args, rank):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    from oracle import novak_oracle as O
+    from paper_2601_07876_b200 import workloads as W
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from harness import oracle_config
+
+    wl = W.get_workload(args.config)
+    hyper = dict(wl.hyper, lookahead_mode=args.lookahead_mode)
+    cores = len(os.sched_getaffinity(0))
+    rng = np.random.default_rng(W.MASTER_SEED)
+
+    def make(n):
+        o = O.Oracle(oracle_config(hyper), [rng.normal(0, 0.05, n)])
+        g = rng.normal(0, 1e-3, n).astype(np.float32).astype(np.float64)
+        return o, g
+
+    # size the per-step sample so that steps+warmup finish in about two minutes
+    probe_n = min(wl.total, 1 << 21)
+    o, g = make(probe_n)
+    o.step([g], threads=cores)
+    t0 = time.perf_counter()
+    for _ in range(3):
+        o.step([g], threads=cores)
+    rate = 3 * probe_n / (time.perf_counter() - t0)
+    n = int(min(wl.total, max(4096, rate * 120.0 / (args.steps + args.warmup))))
+    o, g = make(n)
+    for _ in range(args.warmup):
+        o.step([g], threads=cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.step([g], threads=cores)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = (f"first {n} of {wl.total} elements of {wl.name} as one tensor, "
+              f"{args.steps} oracle steps, {cores} threads over disjoint ranges")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
+                   "lookahead_mode": args.lookahead_mode},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def cpu_baseline(wl, hyper, seconds):
+    """Oracle on the host cores for about `seconds` of work on a bounded sample."""
+    import numpy as np
+    from oracle import novak_oracle as O
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from harness import oracle_config
+    cores = len(os.sched_getaffinity(0))
+    n = min(wl.total, 1 << 24)
+    rng = np.random.default_rng(1)
+    o = O.Oracle(oracle_config(hyper), [rng.normal(0, 0.05, n)])
+    g = rng.normal(0, 1e-3, n).astype(np.float32).astype(np.float64)
+    o.step([g], threads=cores)
+    steps, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < seconds and steps < 5000:
+        o.step([g], threads=cores)
+        steps += 1
+    dt = time.perf_counter() - t0
+    return {"value": n * steps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} elements of {wl.name} as one tensor x {steps} steps "
+                      f"({dt:.1f} s), threads over disjoint element ranges"}
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2601_07876_b200 import binding as B
+    from paper_2601_07876_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the NOVAK step has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    lib = B.load_library(args.lib) if args.lib else None
+    wl = W.get_workload(args.config)
+    hyper = dict(wl.hyper, lookahead_mode=args.lookahead_mode)
+    k = hyper["lookahead_k"]
+    gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
+
+    flat_p = W.alloc_flat(wl, torch.float32, dev)
+    W.init_params(wl, flat_p)
+    params = W.views(flat_p, wl)
+    pool_n = max(1, min(args.pool, int(8e9 // (wl.total * gbytes)) or 1))
+    src = W.GradSource(wl, dev, seed_offset=rank)
+    scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
+    pool_flat = [W.alloc_flat(wl, wl.grad_dtype, dev) for _ in range(pool_n)]
+    for gf in pool_flat:
+        src.fill(gf, scratch)
+    del scratch
+    opt = B.NovakOptimizer(params, **hyper, chunk_elems=args.chunk_elems,
+                           ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine, lib=lib)
+    pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- resident timing: exactly K steps between two events
+    for i in range(max(3, args.warmup)):
+        opt.step(pool[i % pool_n])
+    t_first = opt.info()["t"] + 1
+    launches0 = opt.info()["launches"]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for i in range(args.steps):
+            opt.step(pool[i % pool_n])
+        ev1.record()
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = opt.info()["launches"] - launches0
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * wl.total * args.steps / (ms * 1e-3)
+    alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t)
+              for t in range(t_first, t_first + args.steps)) / args.steps
+    bytes_per_launch = alg * wl.total
+    achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
+    peak, peak_src = measured_peak()
+    per_elem = NCU_DRAM_BYTES_PER_ELEM.get((wl.name, args.lookahead_mode))
+
+    # ---------------- per-step distribution (separate short pass, event per step)
+    per = {}
+    if rank == 0:
+        n_ps = min(args.steps, 300)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_ps + 1)]
+        t_ps = opt.info()["t"] + 1
+        evs[0].record()
+        for i in range(n_ps):
+            opt.step(pool[i % pool_n])
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        times = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_ps)]
+        sync = sorted(x for i, x in enumerate(times) if k > 0 and (t_ps + i) % k == 0)
+        plain = sorted(x for i, x in enumerate(times) if not (k > 0 and (t_ps + i) % k == 0))
+        q = lambda s, f: s[min(len(s) - 1, int(f * len(s)))] if s else None
+        per = {"non_sync_ms": {"p10": q(plain, .1), "p50": q(plain, .5), "p90": q(plain, .9)},
+               "sync_ms": {"p10": q(sync, .1), "p50": q(sync, .5), "p90": q(sync, .9)},
+               "steps": n_ps}
+
+    # ---------------- end to end through novak_step_host (pinned host buffers)
+    e2e = None
+    if not args.no_e2e:
+        h_g = W.alloc_flat(wl, wl.grad_dtype, dev, pin=True)
+        h_p = W.alloc_flat(wl, torch.float32, dev, pin=True)
+        h_g.copy_(pool_flat[0])
+        d_g = pool_flat[0]
+        offs, _ = W.element_offsets(wl)
+        hp = B.ptr_array([h_p.data_ptr() + 4 * o for o in offs])
+        hg = B.ptr_array([h_g.data_ptr() + gbytes * o for o in offs])
+        dg = B.ptr_array([d_g.data_ptr() + gbytes * o for o in offs])
+        stream = torch.cuda.current_stream().cuda_stream
+        gdt = B.NOVAK_GRAD_BF16 if gbytes == 2 else B.NOVAK_GRAD_F32
+
+        def host_step():
+            opt.handle.step_host(hp, hg, opt._params_arr, dg, opt._numel_arr, opt.n, gdt, stream)
+
+        for _ in range(3):
+            host_step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(args.e2e_steps):
+            host_step()
+        e1.record()
+        barrier()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"value": world * wl.total * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": wl.total * gbytes, "d2h_bytes_per_step": wl.total * 4,
+               "ms_per_step": ems / args.e2e_steps, "steps": args.e2e_steps,
+               "api": "novak_step_host (pinned host gradients in, parameters out)"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(wl, hyper, args.cpu_seconds)
+
+    if rank == 0:
+        info = opt.info()
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
+                "grad_dtype": "bf16" if gbytes == 2 else "f32",
+                "lookahead_k": k, "lookahead_mode": args.lookahead_mode,
+                "grad_pool": pool_n,
+                "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
+                      "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),
+                "chunk_elems": int(opt.handle.get_option(B.NOVAK_OPT_CHUNK_ELEMS)),
+                "ctas_per_sm": int(opt.handle.get_option(B.NOVAK_OPT_CTAS_PER_SM)),
+                "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
+                "grid": info["grid"], "block": info["block"], "n_chunks": info["n_chunks"],
+                "replicas": "each rank steps its own replica; no data-path collective",
+            },
+            "hbm_gbs": achieved,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_source": peak_src,
+                         "algorithmic_bytes_per_elem": alg,
+                         "traffic": per_elem * wl.total if per_elem else None,
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "per_step": per,
+            "e2e": e2e,
+            "cpu_baseline": cpu,
+            "gpu_launches": launches,
+            "clocks": clocks.summary(),
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

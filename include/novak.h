@@ -1,0 +1,241 @@
+/*
+ * novak.h -- C ABI of the B200 (sm_100a) NOVAK per-parameter optimizer step.
+ *
+ * One handle (novak_opt) = one hyperparameter set = one "parameter group".
+ * The caller owns every device buffer (parameters, gradients, the state
+ * buffer); the library owns the handle and a small device-side work table
+ * (tensor records + chunk table) that lets ONE kernel launch cover every
+ * tensor of the group.
+ *
+ * What a step computes, per element, in fp32 (the paper's phases 2, 4-10;
+ * Section 5.1, Table 2):
+ *     g~ = g                         (variants none, classical)
+ *     g~ = g + beta_N (g - m)        (approximation, Eq. 13)
+ *     m  = beta1 m + (1-beta1) g~    (Eq. 1)
+ *     v  = beta2 v + (1-beta2) g~^2  (Eq. 2)
+ *     m^ = m/(1-beta1^t), v^ = v/(1-beta2^t)              (Eq. 5)
+ *     u  = m^/(sqrt(v^)+eps)                               (Eq. 17)
+ *     u  = beta1 m^ + (1-beta1) u    (classical only, Eq. 16)
+ *     theta_fast = theta (1 - alpha lambda) - alpha r_t u  (Eq. 18, 24, 24a)
+ *     lookahead on steps with t mod k == 0                 (Eq. 28-31)
+ * The per-step scalars (1-beta^t, rho_t, the branch of Eq. 8, r_t, the decay
+ * factor, the sync flag) are computed once per step on the host in double
+ * precision and passed to the kernel by value.
+ *
+ * Threading: a handle is not thread safe; use one handle per host thread.
+ * Streams: all work of a handle must be issued on one stream (or on streams
+ * the caller orders itself): the device work table is updated in stream order.
+ * No call synchronises the device.  Pointers named d_* are device pointers,
+ * h_* host pointers; "host array of device pointers" means the array lives in
+ * host memory and its entries point to device memory.
+ */
+#ifndef NOVAK_H
+#define NOVAK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct novak_opt novak_opt;
+
+/* Status codes returned by every int-valued call. */
+enum {
+    NOVAK_OK = 0,
+    NOVAK_EINVAL = 1,  /* bad argument; nothing was changed or enqueued      */
+    NOVAK_ESTATE = 2,  /* call not valid in the handle's current state       */
+    NOVAK_ECUDA = 3,   /* a CUDA runtime call failed; see novak_last_error() */
+    NOVAK_ENOMEM = 4   /* host or device allocation failed                   */
+};
+
+/* nesterov_variant (Section 4.4). TRUE needs a closure that re-evaluates the
+ * gradient, which this path does not have: it is accepted and downgraded to
+ * APPROX with NOVAK_WARN_TRUE_DOWNGRADED set (Section 7.3's downgrade rule). */
+enum {
+    NOVAK_NESTEROV_NONE = 0,
+    NOVAK_NESTEROV_APPROX = 1,
+    NOVAK_NESTEROV_CLASSICAL = 2,
+    NOVAK_NESTEROV_TRUE = 3
+};
+
+enum { NOVAK_GRAD_F32 = 0, NOVAK_GRAD_BF16 = 1 };
+
+/* Lookahead rule applied on steps with t mod k == 0 (Section 4.7).
+ * LAST:      slow += alpha_LA (theta_fast - slow); theta = slow.
+ *            The slow weights are read and written on those steps only.
+ * TRAJ_MEAN: slow += alpha_LA (mean of the window's k fast iterates - slow),
+ *            the rule in the proof of Thm 6.2; keeps a running sum (one more
+ *            state array, touched every step). */
+enum { NOVAK_LOOKAHEAD_LAST = 0, NOVAK_LOOKAHEAD_TRAJ_MEAN = 1 };
+
+/* Keys of novak_set_option / novak_get_option. */
+enum {
+    NOVAK_OPT_NESTEROV_BETA = 1,  /* beta_N in [0,1); default beta1 (Eq. 13)          */
+    NOVAK_OPT_LOOKAHEAD_MODE = 2, /* NOVAK_LOOKAHEAD_*; only before attach             */
+    NOVAK_OPT_RECTIFIED = 3,      /* 1 (default): Eq. 8-9; 0: r_t = 1 on every step    */
+    NOVAK_OPT_LR = 4,             /* alpha > 0; may change between steps               */
+    NOVAK_OPT_BIAS1_POWER = 5,    /* 1 (default) or 2: divide the step by (1-beta1^t)
+                                     once more (Eq. 8 taken together with Eq. 24)      */
+    NOVAK_OPT_CHUNK_ELEMS = 6,    /* elements per chunk-table entry (multiple of 1024);
+                                     only before the first step                        */
+    NOVAK_OPT_CTAS_PER_SM = 7,    /* persistent grid = SMs x this; 0: one CTA per chunk */
+    NOVAK_OPT_SERPENTINE = 8,     /* 1: walk the chunk table backwards on even steps so
+                                     the tail of one step is still in L2 for the next  */
+    NOVAK_OPT_WEIGHT_DECAY = 9    /* lambda >= 0; may change between steps             */
+};
+
+/* Warning bits (novak_info.warnings). */
+enum {
+    NOVAK_WARN_TRUE_DOWNGRADED = 1u, /* nesterov_variant TRUE ran as APPROX           */
+    NOVAK_WARN_SCALAR_PATH = 2u      /* some tensor's pointers do not share 16-byte
+                                        alignment; it runs on 4-byte accesses          */
+};
+
+/* Read-only view of the handle after the last successful step. */
+typedef struct novak_info {
+    int64_t t;              /* steps taken (1-based index of the last step)        */
+    int64_t n_syncs;        /* lookahead synchronisations so far                   */
+    int64_t last_sync_step; /* t of the most recent one, 0 if none                 */
+    int64_t total_numel;
+    int64_t launches;       /* kernels launched by this handle since creation      */
+    double bc1, bc2;        /* 1-beta1^t, 1-beta2^t of the last step       (Eq. 5) */
+    double rho_inf, rho_t;  /*                                          (Eq. 6-7)  */
+    double r_t;             /* Eq. 9, or 1 on the un-rectified branch              */
+    double step_size;       /* alpha r_t (divided by bc1 when BIAS1_POWER = 2)     */
+    double decay;           /* 1 - alpha lambda                           (Eq. 18) */
+    int32_t rect_branch;    /* 1: first case of Eq. 8 (rho_t >= 5) was taken       */
+    int32_t is_sync;        /* 1: the last step synchronised                       */
+    int32_t nesterov_variant; /* effective variant (after the downgrade)           */
+    int32_t lookahead_mode;
+    int32_t lookahead_k;
+    int32_t n_tensors;
+    int32_t n_chunks;
+    int32_t grid, block;    /* launch shape of the last step                       */
+    uint32_t warnings;
+} novak_info;
+
+/* Counters and hyperparameters for checkpoint / resume (Table 3: t and the
+ * quantities derived from it).  The state arrays themselves are read and
+ * written through novak_state_ptrs. */
+typedef struct novak_meta {
+    uint64_t magic;
+    int64_t t, n_syncs, last_sync_step;
+    int64_t total_numel;
+    double lr, beta1, beta2, eps, weight_decay, nesterov_beta, lookahead_alpha;
+    int32_t nesterov_variant, lookahead_k, lookahead_mode, rectified, bias1_power;
+    int32_t n_tensors;
+    uint32_t warnings;
+    uint32_t reserved;
+} novak_meta;
+
+/* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
+ * Creates a handle.  lr > 0; beta1, beta2 in [0,1) and beta2 < 1 - 1e-8;
+ * eps > 0; weight_decay >= 0; nesterov_variant one of NOVAK_NESTEROV_*;
+ * lookahead_k >= 0 (0 = lookahead off); lookahead_alpha in (0,1) when k > 0.
+ * NaN fails every test.  Returns NOVAK_EINVAL (and *out = NULL) otherwise.
+ * Does no CUDA work.  The library owns *out; release with novak_destroy. */
+int novak_create(novak_opt **out, double lr, double beta1, double beta2,
+                 double eps, double weight_decay, int nesterov_variant,
+                 int lookahead_k, double lookahead_alpha);
+
+/* Frees the handle and its device work table.  Never touches caller buffers.
+ * NULL is allowed. */
+void novak_destroy(novak_opt *opt);
+
+/* Options not in novak_create's list (Algorithm 1, Hyperparameters).  Values
+ * are validated like novak_create's (NOVAK_EINVAL); keys that change the
+ * state layout or the chunk table return NOVAK_ESTATE once state is attached
+ * (LOOKAHEAD_MODE) or a step was taken (CHUNK_ELEMS). */
+int novak_set_option(novak_opt *opt, int key, double value);
+int novak_get_option(const novak_opt *opt, int key, double *value);
+
+/* Table 3: bytes of optimizer state for n tensors of numel[i] fp32 elements:
+ * m and v always, the slow weights when lookahead_k > 0, the running sum in
+ * TRAJ_MEAN mode.  Includes per-tensor padding (each tensor's slice may start
+ * up to 31 elements into a 128-byte aligned slot so that it shares the
+ * parameter's alignment).  Returns 0 on bad arguments. */
+size_t novak_state_bytes(const novak_opt *opt, const int64_t *numel, int n);
+
+/* Algorithm 1, Initialize: m_0 = v_0 = 0, t = 0.
+ * d_state: caller-allocated device buffer, 256-byte aligned, at least
+ * novak_state_bytes() long; the caller keeps ownership and must keep it alive
+ * while the handle uses it.  d_params (host array of n device pointers, may be
+ * NULL) fixes each slice's alignment phase so that state and parameter share
+ * 16-byte alignment; with NULL, slices start at their slot's base.  The whole
+ * buffer is zero-filled asynchronously on `stream` (a cudaStream_t); the slow
+ * weights are set to theta_0 by the first step's kernel (Eq. 28).
+ * Errors: NOVAK_EINVAL (NULL, n <= 0, numel[i] <= 0, misaligned or short
+ * buffer, parameter pointer not 4-byte aligned), NOVAK_ECUDA. */
+int novak_attach_state(novak_opt *opt, void *d_state, size_t bytes,
+                       void *const *d_params, const int64_t *numel, int n,
+                       void *stream);
+
+/* One optimizer step over every tensor of the group: ONE kernel launch on
+ * `stream`, no synchronisation, no allocation after the first call.
+ * d_params: host array of n device pointers to contiguous fp32 tensors,
+ *           updated in place (4-byte aligned at least).
+ * d_grads:  host array of n device pointers to contiguous gradients of
+ *           grad_dtype (fp32, or bf16 widened exactly), read only.
+ * numel:    must equal the attached layout (NOVAK_ESTATE otherwise).
+ * Pointers may change between steps (the device tensor records are refreshed
+ * in stream order when they do).  Tensors whose parameter, gradient and state
+ * addresses are congruent modulo 16 bytes run on 128-bit accesses; others on
+ * 4-byte accesses (NOVAK_WARN_SCALAR_PATH).
+ * Errors: NOVAK_EINVAL (NULL, n mismatch, bad dtype, misaligned pointer),
+ * NOVAK_ESTATE (no state attached), NOVAK_ENOMEM, NOVAK_ECUDA.  On any error
+ * nothing is enqueued and t is unchanged. */
+int novak_step(novak_opt *opt, void *const *d_params,
+               const void *const *d_grads, const int64_t *numel, int n,
+               int grad_dtype, void *stream);
+
+/* The same step for a caller whose gradients arrive in, and whose updated
+ * parameters return to, HOST memory (pinned memory for asynchronous copies):
+ * copies h_grads[i] -> d_grads[i], runs novak_step, copies d_params[i] ->
+ * h_params[i], all enqueued on `stream` in that order.  Runs of tensors that
+ * are adjacent in both host and device memory are merged into one copy.
+ * The device tensors remain the master copy; the state stays on the device.
+ * Same errors as novak_step. */
+int novak_step_host(novak_opt *opt, void *const *h_params,
+                    const void *const *h_grads, void *const *d_params,
+                    void *const *d_grads, const int64_t *numel, int n,
+                    int grad_dtype, void *stream);
+
+/* Counters and the last step's scalars (bit-exact step and sync indices). */
+int novak_get_info(const novak_opt *opt, novak_info *out);
+
+/* The host-side scalar plan for an arbitrary 1-based step index t, without
+ * touching the handle's counters or the device (Eq. 5-9, 18).  Fills bc1, bc2,
+ * rho_inf, rho_t, r_t, step_size, decay, rect_branch, is_sync of *out; the
+ * other fields are copied from the handle. */
+int novak_plan(const novak_opt *opt, int64_t t, novak_info *out);
+
+/* Device pointers of tensor i's state slices (NULL for arrays the mode does
+ * not keep).  For checkpointing and for tests; valid after attach. */
+int novak_state_ptrs(const novak_opt *opt, int tensor, void **d_m, void **d_v,
+                     void **d_slow, void **d_acc);
+
+/* Checkpoint / resume of everything that is not a device array.  Import
+ * requires an attached state of the same tensor list and the same
+ * layout-relevant hyperparameters (NOVAK_ESTATE otherwise). */
+int novak_export_meta(const novak_opt *opt, novak_meta *out);
+int novak_import_meta(novak_opt *opt, const novak_meta *in);
+
+/* Host-only helper exposing the chunk-table builder: splits n tensors of
+ * numel[i] elements whose first element sits phase[i] (0..31, may be NULL)
+ * elements past a 128-byte boundary into entries (tensor, offset, len) with
+ * len <= chunk_elems, every entry after a tensor's first starting on a
+ * 128-byte boundary.  Writes up to cap entries and returns the number the
+ * table needs (negative on bad arguments). */
+int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
+                           int64_t chunk_elems, int32_t *tensor, int64_t *offset,
+                           int32_t *len, int64_t cap);
+
+/* Text of the last error on this handle ("" if none).  Owned by the handle. */
+const char *novak_last_error(const novak_opt *opt);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NOVAK_H */

@@ -1,0 +1,361 @@
+"""Python binding of the NOVAK step library (``libnovak.so``, see include/novak.h).
+
+Argument marshalling only: every function here has the name of the C entry
+point it calls and passes plain pointers and sizes through ``ctypes``.  No
+arithmetic of the method runs in Python and there is no fallback: if the
+library cannot be loaded (or built with nvcc) the import of this module's
+users fails with the reason.
+
+PyTorch appears only as the owner of device memory and streams:
+``NovakOptimizer`` takes ``torch`` tensors, hands their ``data_ptr()`` to the
+library and keeps the state buffer alive.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import (POINTER, Structure, byref, c_char_p, c_double, c_int, c_int32,
+                    c_int64, c_size_t, c_uint32, c_uint64, c_void_p)
+
+from . import build as _build
+
+# ---- constants of include/novak.h ------------------------------------------
+NOVAK_OK, NOVAK_EINVAL, NOVAK_ESTATE, NOVAK_ECUDA, NOVAK_ENOMEM = range(5)
+NOVAK_NESTEROV_NONE, NOVAK_NESTEROV_APPROX, NOVAK_NESTEROV_CLASSICAL, NOVAK_NESTEROV_TRUE = range(4)
+NOVAK_GRAD_F32, NOVAK_GRAD_BF16 = 0, 1
+NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
+(NOVAK_OPT_NESTEROV_BETA, NOVAK_OPT_LOOKAHEAD_MODE, NOVAK_OPT_RECTIFIED, NOVAK_OPT_LR,
+ NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
+ NOVAK_OPT_WEIGHT_DECAY) = range(1, 10)
+NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
+
+_STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
+
+
+class novak_info(Structure):
+    _fields_ = [
+        ("t", c_int64), ("n_syncs", c_int64), ("last_sync_step", c_int64),
+        ("total_numel", c_int64), ("launches", c_int64),
+        ("bc1", c_double), ("bc2", c_double), ("rho_inf", c_double), ("rho_t", c_double),
+        ("r_t", c_double), ("step_size", c_double), ("decay", c_double),
+        ("rect_branch", c_int32), ("is_sync", c_int32), ("nesterov_variant", c_int32),
+        ("lookahead_mode", c_int32), ("lookahead_k", c_int32), ("n_tensors", c_int32),
+        ("n_chunks", c_int32), ("grid", c_int32), ("block", c_int32), ("warnings", c_uint32),
+    ]
+
+    def as_dict(self) -> dict:
+        return {name: getattr(self, name) for name, _ in self._fields_}
+
+
+class novak_meta(Structure):
+    _fields_ = [
+        ("magic", c_uint64), ("t", c_int64), ("n_syncs", c_int64), ("last_sync_step", c_int64),
+        ("total_numel", c_int64),
+        ("lr", c_double), ("beta1", c_double), ("beta2", c_double), ("eps", c_double),
+        ("weight_decay", c_double), ("nesterov_beta", c_double), ("lookahead_alpha", c_double),
+        ("nesterov_variant", c_int32), ("lookahead_k", c_int32), ("lookahead_mode", c_int32),
+        ("rectified", c_int32), ("bias1_power", c_int32), ("n_tensors", c_int32),
+        ("warnings", c_uint32), ("reserved", c_uint32),
+    ]
+
+
+class NovakError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        msg = f"{where}: {_STATUS.get(status, status)}"
+        super().__init__(f"{msg} ({detail})" if detail else msg)
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> ctypes.CDLL:
+    """Loads ``libnovak.so``; builds it first when it is missing or stale and
+    nvcc is present.  Raises when neither works: there is no other path."""
+    global _lib
+    if path is None and _lib is not None:
+        return _lib
+    if path is None:
+        path = _build.LIB
+        if not _build.up_to_date():
+            try:
+                _build.build()
+            except Exception as exc:  # a stale but loadable library is still refused
+                if not os.path.exists(path):
+                    raise RuntimeError(
+                        f"libnovak.so is missing and could not be built: {exc}") from exc
+                raise
+    lib = ctypes.CDLL(path)
+    vp, i64p = c_void_p, POINTER(c_int64)
+    vpp = POINTER(c_void_p)
+    sigs = {
+        "novak_create": (c_int, [POINTER(vp), c_double, c_double, c_double, c_double, c_double,
+                                 c_int, c_int, c_double]),
+        "novak_destroy": (None, [vp]),
+        "novak_set_option": (c_int, [vp, c_int, c_double]),
+        "novak_get_option": (c_int, [vp, c_int, POINTER(c_double)]),
+        "novak_state_bytes": (c_size_t, [vp, i64p, c_int]),
+        "novak_attach_state": (c_int, [vp, vp, c_size_t, vpp, i64p, c_int, vp]),
+        "novak_step": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
+        "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
+        "novak_state_ptrs": (c_int, [vp, c_int, vpp, vpp, vpp, vpp]),
+        "novak_export_meta": (c_int, [vp, POINTER(novak_meta)]),
+        "novak_import_meta": (c_int, [vp, POINTER(novak_meta)]),
+        "novak_build_chunks": (c_int64, [i64p, POINTER(c_int32), c_int, c_int64,
+                                         POINTER(c_int32), i64p, POINTER(c_int32), c_int64]),
+        "novak_last_error": (c_char_p, [vp]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    if path == _build.LIB:
+        _lib = lib
+    return lib
+
+
+def _check(lib, handle, status: int, where: str):
+    if status != NOVAK_OK:
+        detail = lib.novak_last_error(handle).decode() if handle else ""
+        raise NovakError(status, where, detail)
+
+
+def ptr_array(ptrs):
+    """Host array of pointers (``void* const*``) from Python ints."""
+    return (c_void_p * len(ptrs))(*ptrs)
+
+
+def i64_array(vals):
+    return (c_int64 * len(vals))(*vals)
+
+
+def novak_build_chunks(numel, phase=None, chunk_elems=8192, lib=None):
+    """Host-only chunk-table builder; returns (tensor, offset, len) lists."""
+    lib = lib or load_library()
+    n = len(numel)
+    num = i64_array(numel)
+    ph = (c_int32 * n)(*phase) if phase is not None else None
+    need = lib.novak_build_chunks(num, ph, n, chunk_elems, None, None, None, 0)
+    if need < 0:
+        raise NovakError(NOVAK_EINVAL, "novak_build_chunks")
+    t, o, ln = (c_int32 * need)(), (c_int64 * need)(), (c_int32 * need)()
+    lib.novak_build_chunks(num, ph, n, chunk_elems, t, o, ln, need)
+    return list(t), list(o), list(ln)
+
+
+_NESTEROV = {"none": NOVAK_NESTEROV_NONE, "approximation": NOVAK_NESTEROV_APPROX,
+             "approx": NOVAK_NESTEROV_APPROX, "classical": NOVAK_NESTEROV_CLASSICAL,
+             "true": NOVAK_NESTEROV_TRUE}
+_LA_MODE = {"last": NOVAK_LOOKAHEAD_LAST, "traj_mean": NOVAK_LOOKAHEAD_TRAJ_MEAN}
+
+
+class Handle:
+    """A ``novak_opt*`` with the C calls as methods of the same names (minus
+    the prefix).  No torch here: pointers are Python ints."""
+
+    def __init__(self, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2,
+                 nesterov_variant=NOVAK_NESTEROV_APPROX, lookahead_k=5, lookahead_alpha=0.5,
+                 lib=None):
+        self.lib = lib or load_library()
+        h = c_void_p()
+        st = self.lib.novak_create(byref(h), lr, beta1, beta2, eps, weight_decay,
+                                   nesterov_variant, lookahead_k, lookahead_alpha)
+        if st != NOVAK_OK:
+            raise NovakError(st, "novak_create", "hyperparameter validation failed")
+        self.h = h
+
+    def destroy(self):
+        if getattr(self, "h", None):
+            self.lib.novak_destroy(self.h)
+            self.h = None
+
+    __del__ = destroy
+
+    def set_option(self, key: int, value: float):
+        _check(self.lib, self.h, self.lib.novak_set_option(self.h, key, float(value)),
+               "novak_set_option")
+
+    def get_option(self, key: int) -> float:
+        v = c_double()
+        _check(self.lib, self.h, self.lib.novak_get_option(self.h, key, byref(v)),
+               "novak_get_option")
+        return v.value
+
+    def state_bytes(self, numel) -> int:
+        return self.lib.novak_state_bytes(self.h, i64_array(numel), len(numel))
+
+    def attach_state(self, d_state: int, nbytes: int, d_params, numel, stream: int = 0):
+        pa = ptr_array(d_params) if d_params is not None else None
+        _check(self.lib, self.h,
+               self.lib.novak_attach_state(self.h, d_state, nbytes, pa, i64_array(numel),
+                                           len(numel), stream),
+               "novak_attach_state")
+
+    def step(self, params_arr, grads_arr, numel_arr, n: int, grad_dtype: int, stream: int = 0):
+        """``*_arr`` are ctypes arrays made with ptr_array / i64_array."""
+        st = self.lib.novak_step(self.h, params_arr, grads_arr, numel_arr, n, grad_dtype, stream)
+        if st != NOVAK_OK:
+            _check(self.lib, self.h, st, "novak_step")
+
+    def step_host(self, h_params_arr, h_grads_arr, d_params_arr, d_grads_arr, numel_arr, n,
+                  grad_dtype: int, stream: int = 0):
+        st = self.lib.novak_step_host(self.h, h_params_arr, h_grads_arr, d_params_arr,
+                                      d_grads_arr, numel_arr, n, grad_dtype, stream)
+        if st != NOVAK_OK:
+            _check(self.lib, self.h, st, "novak_step_host")
+
+    def get_info(self) -> novak_info:
+        out = novak_info()
+        _check(self.lib, self.h, self.lib.novak_get_info(self.h, byref(out)), "novak_get_info")
+        return out
+
+    def plan(self, t: int) -> novak_info:
+        out = novak_info()
+        _check(self.lib, self.h, self.lib.novak_plan(self.h, t, byref(out)), "novak_plan")
+        return out
+
+    def state_ptrs(self, tensor: int):
+        m, v, s, a = c_void_p(), c_void_p(), c_void_p(), c_void_p()
+        _check(self.lib, self.h,
+               self.lib.novak_state_ptrs(self.h, tensor, byref(m), byref(v), byref(s), byref(a)),
+               "novak_state_ptrs")
+        return m.value, v.value, s.value, a.value
+
+    def export_meta(self) -> novak_meta:
+        out = novak_meta()
+        _check(self.lib, self.h, self.lib.novak_export_meta(self.h, byref(out)),
+               "novak_export_meta")
+        return out
+
+    def import_meta(self, meta: novak_meta):
+        _check(self.lib, self.h, self.lib.novak_import_meta(self.h, byref(meta)),
+               "novak_import_meta")
+
+    def last_error(self) -> str:
+        return self.lib.novak_last_error(self.h).decode()
+
+
+class GradList:
+    """Marshalled gradient list (pointer array + dtype), reusable across steps."""
+
+    def __init__(self, grads):
+        import torch
+        dts = {g.dtype for g in grads}
+        if dts == {torch.float32}:
+            self.dtype = NOVAK_GRAD_F32
+        elif dts == {torch.bfloat16}:
+            self.dtype = NOVAK_GRAD_BF16
+        else:
+            raise TypeError(f"gradients must be all float32 or all bfloat16, got {dts}")
+        for g in grads:
+            if not g.is_contiguous() or not g.is_cuda:
+                raise ValueError("gradients must be contiguous CUDA tensors")
+        self.tensors = list(grads)           # keeps the memory alive
+        self.numel = [g.numel() for g in grads]
+        self.arr = ptr_array([g.data_ptr() for g in grads])
+
+
+class NovakOptimizer:
+    """NOVAK over a list of fp32 CUDA tensors (one parameter group).
+
+    ``step(grads)`` enqueues one fused kernel on the current torch stream.  The
+    tensors are updated in place; optimizer state lives in one torch-owned
+    byte buffer carved by the library.
+    """
+
+    def __init__(self, params, lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
+                 nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
+                 nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
+                 chunk_elems=None, ctas_per_sm=None, serpentine=None, lib=None):
+        import torch
+        self.params = list(params)
+        if not self.params:
+            raise ValueError("empty parameter list")
+        for p in self.params:
+            if p.dtype != torch.float32 or not p.is_cuda or not p.is_contiguous():
+                raise ValueError("parameters must be contiguous float32 CUDA tensors")
+        self.device = self.params[0].device
+        variant = _NESTEROV[nesterov] if isinstance(nesterov, str) else int(nesterov)
+        self.handle = Handle(lr, betas[0], betas[1], eps, weight_decay, variant, lookahead_k,
+                             lookahead_alpha, lib=lib)
+        h = self.handle
+        if nesterov_beta is not None:
+            h.set_option(NOVAK_OPT_NESTEROV_BETA, nesterov_beta)
+        mode = _LA_MODE[lookahead_mode] if isinstance(lookahead_mode, str) else int(lookahead_mode)
+        h.set_option(NOVAK_OPT_LOOKAHEAD_MODE, mode)
+        h.set_option(NOVAK_OPT_RECTIFIED, 1 if rectified else 0)
+        h.set_option(NOVAK_OPT_BIAS1_POWER, bias1_power)
+        if chunk_elems is not None:
+            h.set_option(NOVAK_OPT_CHUNK_ELEMS, chunk_elems)
+        if ctas_per_sm is not None:
+            h.set_option(NOVAK_OPT_CTAS_PER_SM, ctas_per_sm)
+        if serpentine is not None:
+            h.set_option(NOVAK_OPT_SERPENTINE, 1 if serpentine else 0)
+        self.numel = [p.numel() for p in self.params]
+        self.n = len(self.params)
+        self._numel_arr = i64_array(self.numel)
+        self._param_ptrs = [p.data_ptr() for p in self.params]
+        self._params_arr = ptr_array(self._param_ptrs)
+        nbytes = h.state_bytes(self.numel)
+        if nbytes == 0:
+            raise ValueError("every parameter tensor needs at least one element")
+        with torch.cuda.device(self.device):
+            self.state_buffer = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+            h.attach_state(self.state_buffer.data_ptr(), nbytes, self._param_ptrs, self.numel,
+                           self._stream())
+        self._last_grads = None
+
+    def _stream(self) -> int:
+        import torch
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def prepare(self, grads) -> GradList:
+        gl = GradList(grads)
+        if gl.numel != self.numel:
+            raise ValueError("gradient shapes do not match the parameters")
+        return gl
+
+    def step(self, grads):
+        """One step.  ``grads``: list of tensors, or a ``GradList`` from prepare()."""
+        gl = grads if isinstance(grads, GradList) else self.prepare(grads)
+        self.handle.step(self._params_arr, gl.arr, self._numel_arr, self.n, gl.dtype,
+                         self._stream())
+        self._last_grads = gl
+
+    def info(self) -> dict:
+        return self.handle.get_info().as_dict()
+
+    def plan(self, t: int) -> dict:
+        return self.handle.plan(t).as_dict()
+
+    def _view(self, ptr, numel):
+        if not ptr:
+            return None
+        off = ptr - self.state_buffer.data_ptr()
+        return self.state_buffer[off: off + 4 * numel].view(self.params[0].dtype)
+
+    def state(self, i: int) -> dict:
+        """Views (no copies) of tensor i's state slices inside the state buffer."""
+        m, v, s, a = self.handle.state_ptrs(i)
+        n = self.numel[i]
+        return {"m": self._view(m, n), "v": self._view(v, n), "slow": self._view(s, n),
+                "acc": self._view(a, n)}
+
+    def state_dict(self) -> dict:
+        """Layout-independent checkpoint: counters + per-tensor copies of the state."""
+        meta = self.handle.export_meta()
+        tensors = []
+        for i in range(self.n):
+            tensors.append({k: (t.clone() if t is not None else None)
+                            for k, t in self.state(i).items()})
+        return {"meta": bytes(meta), "tensors": tensors}
+
+    def load_state_dict(self, sd: dict):
+        meta = novak_meta.from_buffer_copy(sd["meta"])
+        self.handle.import_meta(meta)
+        for i, saved in enumerate(sd["tensors"]):
+            for k, dst in self.state(i).items():
+                if dst is not None:
+                    dst.copy_(saved[k])

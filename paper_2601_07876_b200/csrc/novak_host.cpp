@@ -1,0 +1,688 @@
+// Host side of the NOVAK step library: the C ABI, hyperparameter validation,
+// the per-step scalar plan (double precision), the state layout, the
+// multi-tensor chunk table and the launch.  Declarations and argument
+// contracts are in include/novak.h.
+#include "novak.h"
+#include "novak_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using novak::Chunk;
+using novak::StepScalars;
+using novak::TensorRec;
+
+namespace {
+
+constexpr int kRing = 4;                       // pinned staging slots for tensor records
+constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763031ull;  // "NOVAKv01"
+constexpr int64_t kDefaultChunkElems = 8192;
+constexpr int kDefaultCtasPerSm = 0;
+
+struct Hyper {
+    double lr, beta1, beta2, eps, wd, beta_n, la_alpha;
+    int nesterov, la_k, la_mode, rectified, bias1_power;
+};
+
+struct Plan {
+    double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay;
+    int rect_branch, is_sync;
+};
+
+// Eq. 5-9 and 18 for the 1-based step index t.  1 - beta^t is evaluated as
+// -expm1(t log beta) for every t (Section 5.8 gives the log form for large t).
+Plan make_plan(const Hyper &h, int64_t t)
+{
+    Plan p;
+    const double td = static_cast<double>(t);
+    const double l1 = h.beta1 > 0.0 ? td * std::log(h.beta1) : -INFINITY;
+    const double l2 = h.beta2 > 0.0 ? td * std::log(h.beta2) : -INFINITY;
+    p.bc1 = -std::expm1(l1);
+    p.bc2 = -std::expm1(l2);
+    const double b2t = std::exp(l2);
+    p.rho_inf = 2.0 / (1.0 - h.beta2) - 1.0;
+    p.rho_t = p.rho_inf - 2.0 * td * b2t / p.bc2;
+    p.rect_branch = (h.rectified && p.rho_t >= 5.0) ? 1 : 0;
+    p.r_t = 1.0;
+    if (p.rect_branch) {
+        const double a = (p.rho_t - 4.0) / (p.rho_inf - 4.0);
+        const double b = (p.rho_t - 2.0) / (p.rho_inf - 2.0);
+        p.r_t = std::sqrt(a * b * (p.rho_inf / p.rho_t));
+    }
+    p.step_size = h.lr * p.r_t;
+    if (h.bias1_power == 2) p.step_size /= p.bc1;
+    p.decay = 1.0 - h.lr * h.wd;
+    p.is_sync = (h.la_k > 0 && t % h.la_k == 0) ? 1 : 0;
+    return p;
+}
+
+int lookahead_action(const Hyper &h, int64_t t)
+{
+    using namespace novak;
+    if (h.la_k <= 0) return LA_NONE;
+    const bool first_step = (t == 1);
+    const bool sync = (t % h.la_k == 0);
+    const bool first_of_window = ((t - 1) % h.la_k == 0);
+    const bool traj = (h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN && h.la_k > 1);
+    int la = 0;
+    if (first_step) la |= LA_S_INIT | LA_S_WRITE;
+    if (sync) {
+        la |= LA_SYNC | LA_S_WRITE;
+        if (!first_step) la |= LA_S_READ;
+    }
+    if (traj) {
+        if (!first_of_window) la |= LA_A_READ;
+        if (sync) la |= LA_TRAJ; else la |= LA_A_WRITE;
+    }
+    return la;
+}
+
+int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// Splits tensors into chunk-table entries; see novak_build_chunks in novak.h.
+void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chunk_elems,
+                  std::vector<Chunk> &out)
+{
+    out.clear();
+    for (int i = 0; i < n; ++i) {
+        int64_t off = 0;
+        const int32_t ph = phase ? phase[i] : 0;
+        if (ph != 0) {
+            const int64_t head = std::min<int64_t>(numel[i], kSlotAlign - ph);
+            out.push_back(Chunk{i, static_cast<int32_t>(head), 0});
+            off = head;
+        }
+        while (off < numel[i]) {
+            const int64_t len = std::min<int64_t>(chunk_elems, numel[i] - off);
+            out.push_back(Chunk{i, static_cast<int32_t>(len), off});
+            off += len;
+        }
+    }
+}
+
+}  // namespace
+
+struct novak_opt {
+    Hyper h{};
+    uint32_t warnings = 0;
+    int64_t chunk_elems = kDefaultChunkElems;
+    int ctas_per_sm = kDefaultCtasPerSm;
+    int serpentine = 0;
+
+    // state layout (fixed by novak_attach_state)
+    bool attached = false;
+    char *d_state = nullptr;
+    int n = 0;
+    int n_arrays = 0;
+    int64_t region_elems = 0;
+    int64_t total_numel = 0;
+    std::vector<int64_t> numel, slot_off;
+    std::vector<int32_t> phase;
+
+    // counters
+    int64_t t = 0, n_syncs = 0, last_sync = 0, launches = 0;
+    Plan last_plan{};
+    int last_grid = 0;
+
+    // device work table
+    Chunk *d_chunks = nullptr;
+    int n_chunks = 0;
+    TensorRec *d_recs = nullptr;
+    TensorRec *h_recs[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ring_ev[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    int ring_pos = 0;
+    std::vector<void *> cur_p;
+    std::vector<const void *> cur_g;
+    int cur_gdtype = -1;
+    int sms = 0;
+
+    std::string err;
+};
+
+namespace {
+
+int fail(novak_opt *o, int code, const char *fmt, ...)
+{
+    if (o) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        o->err = buf;
+    }
+    return code;
+}
+
+int fail_cuda(novak_opt *o, cudaError_t e, const char *what)
+{
+    return fail(o, NOVAK_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool in_unit(double x) { return x >= 0.0 && x < 1.0; }  // false for NaN
+
+int n_state_arrays(const Hyper &h)
+{
+    int a = 2;
+    if (h.la_k > 0) a += 1;
+    if (h.la_k > 0 && h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN) a += 1;
+    return a;
+}
+
+float *slice(const novak_opt *o, int array, int i)
+{
+    return reinterpret_cast<float *>(o->d_state) + array * o->region_elems + o->slot_off[i] +
+           o->phase[i];
+}
+
+void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
+{
+    std::memset(out, 0, sizeof *out);
+    out->t = o->t;
+    out->n_syncs = o->n_syncs;
+    out->last_sync_step = o->last_sync;
+    out->total_numel = o->total_numel;
+    out->launches = o->launches;
+    out->bc1 = p.bc1; out->bc2 = p.bc2;
+    out->rho_inf = p.rho_inf; out->rho_t = p.rho_t;
+    out->r_t = p.r_t; out->step_size = p.step_size; out->decay = p.decay;
+    out->rect_branch = p.rect_branch; out->is_sync = p.is_sync;
+    out->nesterov_variant = o->h.nesterov;
+    out->lookahead_mode = o->h.la_mode;
+    out->lookahead_k = o->h.la_k;
+    out->n_tensors = o->n;
+    out->n_chunks = o->n_chunks;
+    out->grid = o->last_grid;
+    out->block = novak::step_block_threads();
+    out->warnings = o->warnings;
+}
+
+void release_device(novak_opt *o)
+{
+    if (o->d_chunks) cudaFree(o->d_chunks);
+    if (o->d_recs) cudaFree(o->d_recs);
+    for (int i = 0; i < kRing; ++i) {
+        if (o->h_recs[i]) cudaFreeHost(o->h_recs[i]);
+        if (o->ring_ev[i]) cudaEventDestroy(o->ring_ev[i]);
+        o->h_recs[i] = nullptr;
+        o->ring_ev[i] = nullptr;
+    }
+    o->d_chunks = nullptr;
+    o->d_recs = nullptr;
+    o->n_chunks = 0;
+    o->cur_p.clear();
+    o->cur_g.clear();
+    o->cur_gdtype = -1;
+}
+
+// First step: chunk table and record buffers on the device.
+int prepare_device(novak_opt *o, cudaStream_t stream)
+{
+    cudaError_t e;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(o, e, "cudaGetDevice");
+    if ((e = cudaDeviceGetAttribute(&o->sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaDeviceGetAttribute");
+
+    std::vector<Chunk> chunks;
+    build_chunks(o->numel.data(), o->phase.data(), o->n, o->chunk_elems, chunks);
+    if (o->ctas_per_sm > 0) {
+        // A persistent grid takes chunks round-robin: longest first keeps the
+        // CTAs' totals within one chunk of each other.
+        std::stable_sort(chunks.begin(), chunks.end(),
+                         [](const Chunk &a, const Chunk &b) { return a.len > b.len; });
+    }
+    if (chunks.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
+
+    const size_t cbytes = chunks.size() * sizeof(Chunk);
+    const size_t rbytes = static_cast<size_t>(o->n) * sizeof(TensorRec);
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_chunks), cbytes)) != cudaSuccess) {
+        release_device(o);
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(chunk table, %zu B): %s", cbytes, cudaGetErrorString(e));
+    }
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_recs), rbytes)) != cudaSuccess) {
+        release_device(o);
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(tensor records, %zu B): %s", rbytes, cudaGetErrorString(e));
+    }
+    for (int i = 0; i < kRing; ++i) {
+        if ((e = cudaHostAlloc(reinterpret_cast<void **>(&o->h_recs[i]), rbytes, cudaHostAllocDefault)) != cudaSuccess ||
+            (e = cudaEventCreateWithFlags(&o->ring_ev[i], cudaEventDisableTiming)) != cudaSuccess) {
+            release_device(o);
+            return fail(o, NOVAK_ENOMEM, "pinned record ring: %s", cudaGetErrorString(e));
+        }
+    }
+    // The table is built once: a blocking copy keeps the host vector's
+    // lifetime trivial.  Ordered before the first launch by the stream sync.
+    if ((e = cudaMemcpyAsync(o->d_chunks, chunks.data(), cbytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess) {
+        release_device(o);
+        return fail_cuda(o, e, "chunk table upload");
+    }
+    o->n_chunks = static_cast<int>(chunks.size());
+    return NOVAK_OK;
+}
+
+// Refreshes the device tensor records when the caller's pointers changed.
+int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
+                    int grad_dtype, cudaStream_t stream)
+{
+    const int n = o->n;
+    const bool same = o->cur_gdtype == grad_dtype && !o->cur_p.empty() &&
+                      std::memcmp(o->cur_p.data(), d_params, n * sizeof(void *)) == 0 &&
+                      std::memcmp(o->cur_g.data(), d_grads, n * sizeof(void *)) == 0;
+    if (same) return NOVAK_OK;
+
+    const uintptr_t gmask = grad_dtype == NOVAK_GRAD_BF16 ? 1u : 3u;
+    const uintptr_t gvec = grad_dtype == NOVAK_GRAD_BF16 ? 8u : 16u;
+    bool scalar_path = false;
+    for (int i = 0; i < n; ++i) {
+        const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
+        const uintptr_t g = reinterpret_cast<uintptr_t>(d_grads[i]);
+        if (!p || !g) return fail(o, NOVAK_EINVAL, "tensor %d: NULL pointer", i);
+        if ((p & 3u) || (g & gmask)) return fail(o, NOVAK_EINVAL, "tensor %d: pointer not aligned to its element size", i);
+        // 128-bit path needs parameter, state and gradient congruent mod 16 B.
+        const uintptr_t m = reinterpret_cast<uintptr_t>(slice(o, 0, i));
+        if (((p ^ m) & 15u) || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
+            scalar_path = true;
+    }
+    const int slot = o->ring_pos;
+    cudaError_t e;
+    if ((e = cudaEventSynchronize(o->ring_ev[slot])) != cudaSuccess)
+        return fail_cuda(o, e, "cudaEventSynchronize(record ring)");
+    TensorRec *h = o->h_recs[slot];
+    const bool la = o->h.la_k > 0;
+    const bool traj = la && o->h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN;
+    for (int i = 0; i < n; ++i) {
+        h[i].p = static_cast<float *>(d_params[i]);
+        h[i].g = d_grads[i];
+        h[i].m = slice(o, 0, i);
+        h[i].v = slice(o, 1, i);
+        h[i].slow = la ? slice(o, 2, i) : nullptr;
+        h[i].acc = traj ? slice(o, 3, i) : nullptr;
+    }
+    if ((e = cudaMemcpyAsync(o->d_recs, h, n * sizeof(TensorRec), cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "tensor record upload");
+    if ((e = cudaEventRecord(o->ring_ev[slot], stream)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaEventRecord(record ring)");
+    o->ring_pos = (slot + 1) % kRing;
+    o->cur_p.assign(d_params, d_params + n);
+    o->cur_g.assign(d_grads, d_grads + n);
+    o->cur_gdtype = grad_dtype;
+    if (scalar_path) o->warnings |= NOVAK_WARN_SCALAR_PATH;
+    return NOVAK_OK;
+}
+
+int check_hyper(const Hyper &h, const char **why)
+{
+    *why = "";
+    if (!(h.lr > 0.0) || !std::isfinite(h.lr)) { *why = "lr must be > 0"; return 0; }
+    if (!in_unit(h.beta1)) { *why = "beta1 must be in [0,1)"; return 0; }
+    if (!in_unit(h.beta2)) { *why = "beta2 must be in [0,1)"; return 0; }
+    if (!(h.beta2 < 1.0 - 1e-8)) { *why = "beta2 must be < 1 - 1e-8 (rho_inf)"; return 0; }
+    if (!(h.eps > 0.0) || !std::isfinite(h.eps)) { *why = "eps must be > 0"; return 0; }
+    if (!(h.wd >= 0.0) || !std::isfinite(h.wd)) { *why = "weight_decay must be >= 0"; return 0; }
+    if (!in_unit(h.beta_n)) { *why = "nesterov beta must be in [0,1)"; return 0; }
+    if (h.nesterov < NOVAK_NESTEROV_NONE || h.nesterov > NOVAK_NESTEROV_CLASSICAL) { *why = "unknown nesterov_variant"; return 0; }
+    if (h.la_k < 0) { *why = "lookahead_k must be >= 0"; return 0; }
+    if (h.la_k > 0 && !(h.la_alpha > 0.0 && h.la_alpha < 1.0)) { *why = "lookahead_alpha must be in (0,1)"; return 0; }
+    if (h.la_mode != NOVAK_LOOKAHEAD_LAST && h.la_mode != NOVAK_LOOKAHEAD_TRAJ_MEAN) { *why = "unknown lookahead mode"; return 0; }
+    if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
+    return 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+int novak_create(novak_opt **out, double lr, double beta1, double beta2, double eps,
+                 double weight_decay, int nesterov_variant, int lookahead_k,
+                 double lookahead_alpha)
+{
+    if (!out) return NOVAK_EINVAL;
+    *out = nullptr;
+    Hyper h{};
+    h.lr = lr; h.beta1 = beta1; h.beta2 = beta2; h.eps = eps; h.wd = weight_decay;
+    h.beta_n = beta1;
+    h.la_alpha = lookahead_alpha;
+    h.la_k = lookahead_k;
+    h.la_mode = NOVAK_LOOKAHEAD_LAST;
+    h.rectified = 1;
+    h.bias1_power = 1;
+    uint32_t warn = 0;
+    h.nesterov = nesterov_variant;
+    if (nesterov_variant == NOVAK_NESTEROV_TRUE) {
+        h.nesterov = NOVAK_NESTEROV_APPROX;  // no closure on this path: downgrade, warn
+        warn |= NOVAK_WARN_TRUE_DOWNGRADED;
+    }
+    const char *why;
+    if (!check_hyper(h, &why)) return NOVAK_EINVAL;
+    novak_opt *o = new (std::nothrow) novak_opt();
+    if (!o) return NOVAK_ENOMEM;
+    o->h = h;
+    o->warnings = warn;
+    o->last_plan = make_plan(h, 1);
+    *out = o;
+    return NOVAK_OK;
+}
+
+void novak_destroy(novak_opt *opt)
+{
+    if (!opt) return;
+    release_device(opt);
+    delete opt;
+}
+
+int novak_set_option(novak_opt *o, int key, double value)
+{
+    if (!o) return NOVAK_EINVAL;
+    Hyper h = o->h;
+    const char *why = "";
+    switch (key) {
+    case NOVAK_OPT_NESTEROV_BETA: h.beta_n = value; break;
+    case NOVAK_OPT_LOOKAHEAD_MODE:
+        if (o->attached) return fail(o, NOVAK_ESTATE, "lookahead mode changes the state layout: set it before attach");
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "unknown lookahead mode");
+        h.la_mode = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_RECTIFIED:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "rectified must be 0 or 1");
+        h.rectified = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_LR: h.lr = value; break;
+    case NOVAK_OPT_WEIGHT_DECAY: h.wd = value; break;
+    case NOVAK_OPT_BIAS1_POWER:
+        if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
+        h.bias1_power = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_CHUNK_ELEMS: {
+        if (o->d_chunks) return fail(o, NOVAK_ESTATE, "chunk size is fixed once a step was taken");
+        const int64_t c = static_cast<int64_t>(value);
+        if (!(value >= 1024.0 && value <= 16777216.0) || c % 1024 != 0 || static_cast<double>(c) != value)
+            return fail(o, NOVAK_EINVAL, "chunk_elems must be a multiple of 1024 in [1024, 2^24]");
+        o->chunk_elems = c;
+        return NOVAK_OK;
+    }
+    case NOVAK_OPT_CTAS_PER_SM:
+        if (o->d_chunks) return fail(o, NOVAK_ESTATE, "grid policy is fixed once a step was taken");
+        if (!(value >= 0.0 && value <= 32.0) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "ctas_per_sm must be an integer in [0, 32]");
+        o->ctas_per_sm = static_cast<int>(value);
+        return NOVAK_OK;
+    case NOVAK_OPT_SERPENTINE:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "serpentine must be 0 or 1");
+        o->serpentine = static_cast<int>(value);
+        return NOVAK_OK;
+    default:
+        return fail(o, NOVAK_EINVAL, "unknown option key %d", key);
+    }
+    if (!check_hyper(h, &why)) return fail(o, NOVAK_EINVAL, "%s", why);
+    o->h = h;
+    return NOVAK_OK;
+}
+
+int novak_get_option(const novak_opt *o, int key, double *value)
+{
+    if (!o || !value) return NOVAK_EINVAL;
+    switch (key) {
+    case NOVAK_OPT_NESTEROV_BETA: *value = o->h.beta_n; break;
+    case NOVAK_OPT_LOOKAHEAD_MODE: *value = o->h.la_mode; break;
+    case NOVAK_OPT_RECTIFIED: *value = o->h.rectified; break;
+    case NOVAK_OPT_LR: *value = o->h.lr; break;
+    case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
+    case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
+    case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
+    case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
+    case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
+    default: return NOVAK_EINVAL;
+    }
+    return NOVAK_OK;
+}
+
+size_t novak_state_bytes(const novak_opt *o, const int64_t *numel, int n)
+{
+    if (!o || !numel || n <= 0) return 0;
+    int64_t region = 0;
+    for (int i = 0; i < n; ++i) {
+        if (numel[i] <= 0) return 0;
+        region += round_up(numel[i] + kSlotAlign - 1, kSlotAlign);
+    }
+    return static_cast<size_t>(region) * sizeof(float) * n_state_arrays(o->h);
+}
+
+int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d_params,
+                       const int64_t *numel, int n, void *stream)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!d_state || !numel || n <= 0) return fail(o, NOVAK_EINVAL, "attach: NULL buffer or empty tensor list");
+    if (reinterpret_cast<uintptr_t>(d_state) & 255u) return fail(o, NOVAK_EINVAL, "attach: state buffer must be 256-byte aligned");
+    const size_t need = novak_state_bytes(o, numel, n);
+    if (need == 0) return fail(o, NOVAK_EINVAL, "attach: every numel must be > 0");
+    if (bytes < need) return fail(o, NOVAK_EINVAL, "attach: state buffer has %zu B, needs %zu B", bytes, need);
+    std::vector<int32_t> phase(n, 0);
+    if (d_params) {
+        for (int i = 0; i < n; ++i) {
+            const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
+            if (!p || (p & 3u)) return fail(o, NOVAK_EINVAL, "attach: parameter %d is NULL or not 4-byte aligned", i);
+            phase[i] = static_cast<int32_t>((p % (kSlotAlign * 4)) / 4);
+        }
+    }
+    cudaError_t e = cudaMemsetAsync(d_state, 0, need, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail_cuda(o, e, "cudaMemsetAsync(state)");
+
+    release_device(o);
+    o->d_state = static_cast<char *>(d_state);
+    o->n = n;
+    o->n_arrays = n_state_arrays(o->h);
+    o->numel.assign(numel, numel + n);
+    o->phase = phase;
+    o->slot_off.resize(n);
+    int64_t off = 0, total = 0;
+    for (int i = 0; i < n; ++i) {
+        o->slot_off[i] = off;
+        off += round_up(numel[i] + kSlotAlign - 1, kSlotAlign);
+        total += numel[i];
+    }
+    o->region_elems = off;
+    o->total_numel = total;
+    o->t = 0; o->n_syncs = 0; o->last_sync = 0;
+    o->attached = true;
+    o->err.clear();
+    return NOVAK_OK;
+}
+
+int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
+               const int64_t *numel, int n, int grad_dtype, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "step: no state attached");
+    if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step: NULL argument");
+    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16) return fail(o, NOVAK_EINVAL, "step: unknown grad_dtype %d", grad_dtype);
+    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
+        return fail(o, NOVAK_ESTATE, "step: tensor list differs from the attached layout");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    int rc;
+    if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
+    if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
+
+    const int64_t t = o->t + 1;
+    const Plan p = make_plan(o->h, t);
+    const int la = lookahead_action(o->h, t);
+    StepScalars s;
+    s.beta1 = static_cast<float>(o->h.beta1);
+    s.omb1 = static_cast<float>(1.0 - o->h.beta1);
+    s.beta2 = static_cast<float>(o->h.beta2);
+    s.omb2 = static_cast<float>(1.0 - o->h.beta2);
+    s.beta_n = static_cast<float>(o->h.beta_n);
+    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
+    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
+    s.eps = static_cast<float>(o->h.eps);
+    s.decay = static_cast<float>(p.decay);
+    s.step = static_cast<float>(p.step_size);
+    s.la_alpha = static_cast<float>(o->h.la_alpha);
+    s.k = static_cast<float>(o->h.la_k > 0 ? o->h.la_k : 1);
+
+    novak::LaunchCfg cfg;
+    cfg.grid = o->n_chunks;
+    if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
+    cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
+    cudaError_t e = novak::launch_step(o->d_chunks, o->n_chunks, o->d_recs, s, o->h.nesterov,
+                                       grad_dtype, la, cfg, stream);
+    if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
+
+    o->t = t;
+    o->launches += 1;
+    o->last_plan = p;
+    o->last_grid = cfg.grid;
+    if (p.is_sync) { o->n_syncs += 1; o->last_sync = t; }
+    return NOVAK_OK;
+}
+
+int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_grads,
+                    void *const *d_params, void *const *d_grads, const int64_t *numel, int n,
+                    int grad_dtype, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "step_host: no state attached");
+    if (!h_params || !h_grads || !d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step_host: NULL argument");
+    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16) return fail(o, NOVAK_EINVAL, "step_host: unknown grad_dtype %d", grad_dtype);
+    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
+        return fail(o, NOVAK_ESTATE, "step_host: tensor list differs from the attached layout");
+    for (int i = 0; i < n; ++i)
+        if (!h_params[i] || !h_grads[i] || !d_params[i] || !d_grads[i])
+            return fail(o, NOVAK_EINVAL, "step_host: tensor %d has a NULL pointer", i);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t gsz = grad_dtype == NOVAK_GRAD_BF16 ? 2 : 4;
+    cudaError_t e;
+
+    // gradients host -> device, merging runs adjacent on both sides
+    for (int i = 0; i < n;) {
+        const char *hs = static_cast<const char *>(h_grads[i]);
+        char *ds = static_cast<char *>(d_grads[i]);
+        size_t bytes = static_cast<size_t>(numel[i]) * gsz;
+        int j = i + 1;
+        while (j < n && static_cast<const char *>(h_grads[j]) == hs + bytes &&
+               static_cast<char *>(d_grads[j]) == ds + bytes) {
+            bytes += static_cast<size_t>(numel[j]) * gsz;
+            ++j;
+        }
+        if ((e = cudaMemcpyAsync(ds, hs, bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "gradient upload");
+        i = j;
+    }
+    const int rc = novak_step(o, d_params, const_cast<const void *const *>(d_grads), numel, n, grad_dtype, stream_);
+    if (rc != NOVAK_OK) return rc;
+    // parameters device -> host
+    for (int i = 0; i < n;) {
+        char *hs = static_cast<char *>(h_params[i]);
+        const char *ds = static_cast<const char *>(d_params[i]);
+        size_t bytes = static_cast<size_t>(numel[i]) * 4;
+        int j = i + 1;
+        while (j < n && static_cast<char *>(h_params[j]) == hs + bytes &&
+               static_cast<const char *>(d_params[j]) == ds + bytes) {
+            bytes += static_cast<size_t>(numel[j]) * 4;
+            ++j;
+        }
+        if ((e = cudaMemcpyAsync(hs, ds, bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "parameter download");
+        i = j;
+    }
+    return NOVAK_OK;
+}
+
+int novak_get_info(const novak_opt *o, novak_info *out)
+{
+    if (!o || !out) return NOVAK_EINVAL;
+    fill_info(o, o->last_plan, out);
+    return NOVAK_OK;
+}
+
+int novak_plan(const novak_opt *o, int64_t t, novak_info *out)
+{
+    if (!o || !out || t < 1) return NOVAK_EINVAL;
+    fill_info(o, make_plan(o->h, t), out);
+    return NOVAK_OK;
+}
+
+int novak_state_ptrs(const novak_opt *o, int tensor, void **d_m, void **d_v, void **d_slow,
+                     void **d_acc)
+{
+    if (!o || !o->attached || tensor < 0 || tensor >= o->n) return NOVAK_EINVAL;
+    if (d_m) *d_m = slice(o, 0, tensor);
+    if (d_v) *d_v = slice(o, 1, tensor);
+    if (d_slow) *d_slow = o->n_arrays > 2 ? slice(o, 2, tensor) : nullptr;
+    if (d_acc) *d_acc = o->n_arrays > 3 ? slice(o, 3, tensor) : nullptr;
+    return NOVAK_OK;
+}
+
+int novak_export_meta(const novak_opt *o, novak_meta *out)
+{
+    if (!o || !out) return NOVAK_EINVAL;
+    std::memset(out, 0, sizeof *out);
+    out->magic = kMetaMagic;
+    out->t = o->t; out->n_syncs = o->n_syncs; out->last_sync_step = o->last_sync;
+    out->total_numel = o->total_numel;
+    out->lr = o->h.lr; out->beta1 = o->h.beta1; out->beta2 = o->h.beta2; out->eps = o->h.eps;
+    out->weight_decay = o->h.wd; out->nesterov_beta = o->h.beta_n;
+    out->lookahead_alpha = o->h.la_alpha;
+    out->nesterov_variant = o->h.nesterov; out->lookahead_k = o->h.la_k;
+    out->lookahead_mode = o->h.la_mode; out->rectified = o->h.rectified;
+    out->bias1_power = o->h.bias1_power;
+    out->n_tensors = o->n;
+    out->warnings = o->warnings;
+    return NOVAK_OK;
+}
+
+int novak_import_meta(novak_opt *o, const novak_meta *in)
+{
+    if (!o || !in) return NOVAK_EINVAL;
+    if (in->magic != kMetaMagic) return fail(o, NOVAK_EINVAL, "import: not a NOVAK meta record");
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "import: attach the state first");
+    if (in->n_tensors != o->n || in->total_numel != o->total_numel ||
+        in->lookahead_k != o->h.la_k || in->lookahead_mode != o->h.la_mode)
+        return fail(o, NOVAK_ESTATE, "import: tensor list or lookahead layout differs");
+    if (in->t < 0 || in->n_syncs < 0) return fail(o, NOVAK_EINVAL, "import: negative counter");
+    Hyper h = o->h;
+    h.lr = in->lr; h.beta1 = in->beta1; h.beta2 = in->beta2; h.eps = in->eps;
+    h.wd = in->weight_decay; h.beta_n = in->nesterov_beta; h.la_alpha = in->lookahead_alpha;
+    h.nesterov = in->nesterov_variant; h.rectified = in->rectified;
+    h.bias1_power = in->bias1_power;
+    const char *why;
+    if (!check_hyper(h, &why)) return fail(o, NOVAK_EINVAL, "import: %s", why);
+    o->h = h;
+    o->t = in->t; o->n_syncs = in->n_syncs; o->last_sync = in->last_sync_step;
+    o->warnings |= in->warnings;
+    o->last_plan = make_plan(h, in->t > 0 ? in->t : 1);
+    return NOVAK_OK;
+}
+
+int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
+                           int64_t chunk_elems, int32_t *tensor, int64_t *offset,
+                           int32_t *len, int64_t cap)
+{
+    if (!numel || n <= 0 || chunk_elems < kSlotAlign || chunk_elems % kSlotAlign != 0 ||
+        chunk_elems > INT32_MAX || cap < 0)
+        return -1;
+    for (int i = 0; i < n; ++i)
+        if (numel[i] <= 0 || (phase && (phase[i] < 0 || phase[i] >= kSlotAlign))) return -1;
+    std::vector<Chunk> chunks;
+    build_chunks(numel, phase, n, chunk_elems, chunks);
+    const int64_t count = static_cast<int64_t>(chunks.size());
+    for (int64_t i = 0; i < count && i < cap; ++i) {
+        if (tensor) tensor[i] = chunks[i].tensor;
+        if (offset) offset[i] = chunks[i].offset;
+        if (len) len[i] = chunks[i].len;
+    }
+    return count;
+}
+
+const char *novak_last_error(const novak_opt *o) { return o ? o->err.c_str() : ""; }
+
+}  // extern "C"

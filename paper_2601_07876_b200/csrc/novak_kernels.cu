@@ -1,0 +1,301 @@
+// Fused multi-tensor NOVAK step kernel for sm_100a.
+//
+// One launch covers every tensor of a parameter group.  A CTA walks the chunk
+// table (grid-stride); for each chunk it reads theta, g, m, v (and the
+// lookahead arrays on the steps that need them) exactly once with 128-bit
+// coalesced accesses, does the paper's phases 2 and 4-10 in registers (fp32,
+// IEEE sqrt and division, no fast-math) and writes theta, m, v (and the
+// lookahead arrays) exactly once.  There is no shared memory, no atomic, no
+// barrier and no wait of any kind, so a launch does a bounded amount of work
+// per CTA and cannot hang.
+//
+// The step is HBM bound: 28 B per element against ~45 fp32 instructions, so
+// the design goal is bytes in flight per SM, not arithmetic: each thread
+// issues NOVAK_UNROLL independent 16-byte loads per stream before the first
+// use.
+#include "novak_internal.h"
+
+#include "novak.h"
+
+#ifndef NOVAK_BLOCK
+#define NOVAK_BLOCK 256
+#endif
+#ifndef NOVAK_UNROLL
+#define NOVAK_UNROLL 2
+#endif
+#ifndef NOVAK_MIN_CTAS
+#define NOVAK_MIN_CTAS 4
+#endif
+
+namespace novak {
+namespace {
+
+constexpr int kBlock = NOVAK_BLOCK;
+constexpr int kUnroll = NOVAK_UNROLL;
+
+template <int N>
+struct Vec {
+    float a[N];
+};
+
+// ---- global memory access: streaming hints, each address touched once per step
+template <int N>
+__device__ __forceinline__ Vec<N> load_f32(const float *base, int idx);
+
+template <>
+__device__ __forceinline__ Vec<4> load_f32<4>(const float *base, int idx)
+{
+    const float4 t = __ldcs(reinterpret_cast<const float4 *>(base) + idx);
+    Vec<4> r;
+    r.a[0] = t.x; r.a[1] = t.y; r.a[2] = t.z; r.a[3] = t.w;
+    return r;
+}
+
+template <>
+__device__ __forceinline__ Vec<1> load_f32<1>(const float *base, int idx)
+{
+    Vec<1> r;
+    r.a[0] = __ldcs(base + idx);
+    return r;
+}
+
+template <int N>
+__device__ __forceinline__ void store_f32(float *base, int idx, const Vec<N> &x);
+
+template <>
+__device__ __forceinline__ void store_f32<4>(float *base, int idx, const Vec<4> &x)
+{
+    __stcs(reinterpret_cast<float4 *>(base) + idx,
+           make_float4(x.a[0], x.a[1], x.a[2], x.a[3]));
+}
+
+template <>
+__device__ __forceinline__ void store_f32<1>(float *base, int idx, const Vec<1> &x)
+{
+    __stcs(base + idx, x.a[0]);
+}
+
+// bf16 -> fp32 is exact: the 16 bits are the upper half of the fp32 pattern.
+template <int N, int GT>
+__device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
+{
+    if constexpr (GT == NOVAK_GRAD_F32) {
+        return load_f32<N>(static_cast<const float *>(base), idx);
+    } else if constexpr (N == 4) {
+        const uint2 t = __ldcs(static_cast<const uint2 *>(base) + idx);
+        Vec<4> r;
+        r.a[0] = __uint_as_float(t.x << 16);
+        r.a[1] = __uint_as_float(t.x & 0xffff0000u);
+        r.a[2] = __uint_as_float(t.y << 16);
+        r.a[3] = __uint_as_float(t.y & 0xffff0000u);
+        return r;
+    } else {
+        const unsigned short t = __ldcs(static_cast<const unsigned short *>(base) + idx);
+        Vec<1> r;
+        r.a[0] = __uint_as_float(static_cast<unsigned>(t) << 16);
+        return r;
+    }
+}
+
+// ---- the per-element update, phases 2 and 4-10 (Section 5.1)
+template <int NEST, int LA>
+__device__ __forceinline__ void update_element(float &p, float g, float &m, float &v,
+                                               float &slow, float &acc,
+                                               const StepScalars &s)
+{
+    // Phase 2, Eq. 13: g~ = g + beta_N (g - m_{t-1})
+    if constexpr (NEST == NOVAK_NESTEROV_APPROX)
+        g = fmaf(s.beta_n, g - m, g);
+    // Phase 4, Eq. 1-2
+    m = fmaf(s.beta1, m, s.omb1 * g);
+    v = fmaf(s.beta2, v, s.omb2 * (g * g));
+    // Phase 5, Eq. 5
+    const float m_hat = m * s.inv_bc1;
+    const float v_hat = v * s.inv_bc2;
+    // Phase 8, Eq. 17 (IEEE sqrt and division), Eq. 16 for the classical blend
+#ifdef NOVAK_APPROX_MATH
+    float rt, u;
+    asm("sqrt.approx.f32 %0, %1;" : "=f"(rt) : "f"(v_hat));
+    asm("div.full.f32 %0, %1, %2;" : "=f"(u) : "f"(m_hat), "f"(rt + s.eps));
+#else
+    float u = m_hat / (sqrtf(v_hat) + s.eps);
+#endif
+    if constexpr (NEST == NOVAK_NESTEROV_CLASSICAL)
+        u = fmaf(s.beta1, m_hat, s.omb1 * u);
+    // Phase 9, Eq. 18 + 24: decay with the base rate, step with alpha r_t
+    const float theta_in = p;
+    const float theta_fast = fmaf(theta_in, s.decay, -(s.step * u));
+    // Phase 10, Eq. 28-31
+    float out = theta_fast;
+    float sum = theta_fast;
+    if constexpr ((LA & LA_A_READ) != 0)
+        sum = acc + theta_fast;
+    if constexpr ((LA & LA_A_WRITE) != 0)
+        acc = sum;
+    if constexpr ((LA & LA_SYNC) != 0) {
+        const float slow_in = (LA & LA_S_INIT) ? theta_in : slow;
+        const float target = (LA & LA_TRAJ) ? __fdiv_rn(sum, s.k) : theta_fast;
+        out = fmaf(s.la_alpha, target - slow_in, slow_in);
+        slow = out;
+    } else if constexpr ((LA & LA_S_INIT) != 0) {
+        slow = theta_in;
+    }
+    p = out;
+}
+
+// One full tile: U vectors per thread and per stream, every load issued
+// before the first use so that U x (4..6) 16-byte requests are in flight.
+template <int N, int U, int NEST, int GT, int LA>
+__device__ __forceinline__ void run_tile(float *p, const void *g, float *m, float *v,
+                                         float *slow, float *acc, int first,
+                                         const StepScalars &s)
+{
+    constexpr bool kReadS = (LA & LA_S_READ) != 0;
+    constexpr bool kWriteS = (LA & LA_S_WRITE) != 0;
+    constexpr bool kReadA = (LA & LA_A_READ) != 0;
+    constexpr bool kWriteA = (LA & LA_A_WRITE) != 0;
+    Vec<N> P[U], G[U], M[U], V[U], S[U], A[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+        P[j] = load_f32<N>(p, idx);
+        G[j] = load_grad<N, GT>(g, idx);
+        M[j] = load_f32<N>(m, idx);
+        V[j] = load_f32<N>(v, idx);
+        if constexpr (kReadS) S[j] = load_f32<N>(slow, idx);
+        if constexpr (kReadA) A[j] = load_f32<N>(acc, idx);
+    }
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+#pragma unroll
+        for (int e = 0; e < N; ++e)
+            update_element<NEST, LA>(P[j].a[e], G[j].a[e], M[j].a[e], V[j].a[e],
+                                     S[j].a[e], A[j].a[e], s);
+        store_f32<N>(p, idx, P[j]);
+        store_f32<N>(m, idx, M[j]);
+        store_f32<N>(v, idx, V[j]);
+        if constexpr (kWriteS) store_f32<N>(slow, idx, S[j]);
+        if constexpr (kWriteA) store_f32<N>(acc, idx, A[j]);
+    }
+}
+
+// nvec vectors of N elements: full tiles of U vectors per thread, then the
+// remainder one vector per thread at a time.
+template <int N, int U, int NEST, int GT, int LA>
+__device__ __forceinline__ void run_span(float *p, const void *g, float *m, float *v,
+                                         float *slow, float *acc, int nvec,
+                                         const StepScalars &s)
+{
+    constexpr int kTile = kBlock * U;
+    int base = 0;
+#pragma unroll 1
+    for (; base + kTile <= nvec; base += kTile)
+        run_tile<N, U, NEST, GT, LA>(p, g, m, v, slow, acc, base + threadIdx.x, s);
+#pragma unroll 1
+    for (int idx = base + threadIdx.x; idx < nvec; idx += kBlock)
+        run_tile<N, 1, NEST, GT, LA>(p, g, m, v, slow, acc, idx, s);
+}
+
+template <int NEST, int GT, int LA>
+__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS)
+novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
+                  const TensorRec *__restrict__ recs, const StepScalars s, int reverse)
+{
+    constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
+    constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
+
+#pragma unroll 1
+    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+        const Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
+        const TensorRec r = recs[ch.tensor];
+        float *p = r.p + ch.offset;
+        float *m = r.m + ch.offset;
+        float *v = r.v + ch.offset;
+        float *slow = kUseS ? r.slow + ch.offset : nullptr;
+        float *acc = kUseA ? r.acc + ch.offset : nullptr;
+        const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
+
+        uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(m) |
+                         reinterpret_cast<uintptr_t>(v);
+        if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
+        if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
+        const bool aligned = (bits & 15u) == 0 &&
+                             (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
+        if (aligned) {
+            const int nvec = ch.len >> 2;
+            run_span<4, kUnroll, NEST, GT, LA>(p, g, m, v, slow, acc, nvec, s);
+            // ragged tail of a tensor: at most 3 elements
+            const int idx = (nvec << 2) + threadIdx.x;
+            if (idx < ch.len)
+                run_tile<1, 1, NEST, GT, LA>(p, g, m, v, slow, acc, idx, s);
+        } else {
+            // parameter, gradient and state do not share 16-byte alignment
+            run_span<1, 4, NEST, GT, LA>(p, g, m, v, slow, acc, ch.len, s);
+        }
+    }
+}
+
+using KernelFn = void (*)(const Chunk *, int, const TensorRec *, StepScalars, int);
+
+template <int NEST, int GT>
+KernelFn pick_la(int la)
+{
+    switch (la) {
+#define NOVAK_LA_CASE(X) case (X): return novak_step_kernel<NEST, GT, (X)>;
+        NOVAK_LA_CASE(LA_NONE)
+        NOVAK_LA_CASE(LA_S_INIT | LA_S_WRITE)
+        NOVAK_LA_CASE(LA_S_INIT | LA_S_WRITE | LA_SYNC)
+        NOVAK_LA_CASE(LA_S_READ | LA_S_WRITE | LA_SYNC)
+        NOVAK_LA_CASE(LA_A_WRITE)
+        NOVAK_LA_CASE(LA_A_WRITE | LA_S_INIT | LA_S_WRITE)
+        NOVAK_LA_CASE(LA_A_READ | LA_A_WRITE)
+        NOVAK_LA_CASE(LA_A_READ | LA_S_READ | LA_S_WRITE | LA_SYNC | LA_TRAJ)
+#undef NOVAK_LA_CASE
+    default: return nullptr;
+    }
+}
+
+template <int NEST>
+KernelFn pick_gt(int grad_dtype, int la)
+{
+    switch (grad_dtype) {
+    case NOVAK_GRAD_F32: return pick_la<NEST, NOVAK_GRAD_F32>(la);
+    case NOVAK_GRAD_BF16: return pick_la<NEST, NOVAK_GRAD_BF16>(la);
+    default: return nullptr;
+    }
+}
+
+KernelFn pick_kernel(int nesterov, int grad_dtype, int la)
+{
+    switch (nesterov) {
+    case NOVAK_NESTEROV_NONE: return pick_gt<NOVAK_NESTEROV_NONE>(grad_dtype, la);
+    case NOVAK_NESTEROV_APPROX: return pick_gt<NOVAK_NESTEROV_APPROX>(grad_dtype, la);
+    case NOVAK_NESTEROV_CLASSICAL: return pick_gt<NOVAK_NESTEROV_CLASSICAL>(grad_dtype, la);
+    default: return nullptr;
+    }
+}
+
+}  // namespace
+
+int step_block_threads() { return kBlock; }
+
+cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int *ctas_per_sm)
+{
+    KernelFn fn = pick_kernel(nesterov, grad_dtype, la);
+    if (!fn) return cudaErrorInvalidValue;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, fn, kBlock, 0);
+}
+
+cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
+                        const StepScalars &s, int nesterov, int grad_dtype, int la,
+                        const LaunchCfg &cfg, cudaStream_t stream)
+{
+    KernelFn fn = pick_kernel(nesterov, grad_dtype, la);
+    if (!fn || n_chunks <= 0 || cfg.grid <= 0) return cudaErrorInvalidValue;
+    fn<<<cfg.grid, kBlock, 0, stream>>>(d_chunks, n_chunks, d_recs, s, cfg.reverse);
+    return cudaGetLastError();
+}
+
+}  // namespace novak

@@ -1,0 +1,173 @@
+"""Shared helpers of the GPU parity tests: run the CUDA library and the CPU
+oracle on the same seeded inputs and compare element by element."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import novak_oracle as O
+from paper_2601_07876_b200 import binding as B
+from paper_2601_07876_b200 import workloads as W
+
+# Tolerance of the fp32 CUDA path against the fp64 oracle after N steps:
+# |gpu - oracle| <= ATOL + RTOL * |oracle| for theta, m, v, slow, acc.
+RTOL, ATOL = 1e-5, 1e-7
+
+_NEST = {"none": O.NESTEROV_NONE, "approximation": O.NESTEROV_APPROX,
+         "classical": O.NESTEROV_CLASSICAL, "true": O.NESTEROV_APPROX}
+_MODE = {"last": O.LOOKAHEAD_LAST, "traj_mean": O.LOOKAHEAD_TRAJ_MEAN}
+
+
+def oracle_config(hyper: dict) -> O.Config:
+    h = dict(hyper)
+    b1, b2 = h.pop("betas", (0.9, 0.999))
+    return O.Config(
+        lr=h.pop("lr", 1e-3), beta1=b1, beta2=b2, eps=h.pop("eps", 1e-8),
+        weight_decay=h.pop("weight_decay", 1e-2),
+        nesterov_variant=_NEST[h.pop("nesterov", "approximation")],
+        lookahead_k=h.pop("lookahead_k", 5), lookahead_alpha=h.pop("lookahead_alpha", 0.5),
+        nesterov_beta=h.pop("nesterov_beta", None),
+        lookahead_mode=_MODE[h.pop("lookahead_mode", "last")],
+        rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1))
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
+
+
+def assert_close(gpu, ref: np.ndarray, what: str):
+    got = to_f64(gpu) if isinstance(gpu, torch.Tensor) else np.asarray(gpu, np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    err = np.abs(got - ref)
+    tol = ATOL + RTOL * np.abs(ref)
+    bad = err > tol
+    if bad.any():
+        i = int(np.argmax(err - tol))
+        raise AssertionError(
+            f"{what}: {int(bad.sum())}/{bad.size} elements out of tolerance; worst at {i}: "
+            f"gpu={got.flat[i]!r} oracle={ref.flat[i]!r} err={err.flat[i]:.3e} tol={tol.flat[i]:.3e}")
+    assert np.isfinite(got).all(), f"{what}: non-finite values"
+
+
+class Pair:
+    """CUDA optimizer and oracle over the same tensors (every element)."""
+
+    def __init__(self, params, hyper: dict, opt_kwargs: dict | None = None, lib=None):
+        self.params = params
+        self.hyper = hyper
+        self.oracle = O.Oracle(oracle_config(hyper), [to_f64(p) for p in params])
+        self.opt = B.NovakOptimizer(params, **hyper, **(opt_kwargs or {}), lib=lib)
+        self.sync_steps = []
+        self.rect_flags = []
+
+    def step(self, grads, threads=1):
+        self.opt.step(grads)
+        info = self.opt.info()
+        if info["is_sync"]:
+            self.sync_steps.append(info["t"])
+        self.rect_flags.append(info["rect_branch"])
+        self.oracle.step([to_f64(g) for g in grads], threads=threads)
+
+    def check(self, what=""):
+        torch.cuda.synchronize()
+        o, info = self.oracle, self.opt.info()
+        assert info["t"] == o.t
+        assert self.sync_steps == o.sync_steps
+        assert info["n_syncs"] == len(o.sync_steps)
+        assert info["last_sync_step"] == (o.sync_steps[-1] if o.sync_steps else 0)
+        assert self.rect_flags == o.rect_flags
+        for i, p in enumerate(self.params):
+            st = self.opt.state(i)
+            assert_close(p, o.theta[i], f"{what} theta[{i}]")
+            assert_close(st["m"], o.m[i], f"{what} m[{i}]")
+            assert_close(st["v"], o.v[i], f"{what} v[{i}]")
+            if o.slow is not None:
+                assert_close(st["slow"], o.slow[i], f"{what} slow[{i}]")
+            else:
+                assert st["slow"] is None
+            if o.acc is not None and (o.cfg.lookahead_k > 1):
+                # between syncs the running sum is defined; right after a sync the
+                # oracle holds 0 and the kernel leaves the old sum (never read again)
+                if o.t % o.cfg.lookahead_k != 0:
+                    assert_close(st["acc"], o.acc[i], f"{what} acc[{i}]")
+
+
+def make_tensors(numels, device, offsets=None, dtype=torch.float32, fill=None):
+    """Views of one flat buffer; offsets[i] extra elements of misalignment
+    (relative to a 256-byte boundary) per tensor.  Gaps hold `fill`."""
+    offsets = offsets or [0] * len(numels)
+    starts, cur = [], 64
+    for n, o in zip(numels, offsets):
+        cur = (cur + 63) // 64 * 64 + o
+        starts.append(cur)
+        cur += n
+    total = (cur + 63) // 64 * 64 + 64
+    flat = torch.zeros(total, dtype=dtype, device=device)
+    if fill is not None:
+        flat.fill_(fill)
+    return flat, [flat[s:s + n] for s, n in zip(starts, numels)], starts
+
+
+def gaps_mask(total, starts, numels, device):
+    m = torch.ones(total, dtype=torch.bool, device=device)
+    for s, n in zip(starts, numels):
+        m[s:s + n] = False
+    return m
+
+
+class SampledPair:
+    """Full-size workload on the GPU, oracle on a fixed sample of elements
+    (exact for them: the step has no cross-element term)."""
+
+    def __init__(self, wl: W.Workload, device, hyper_override: dict | None = None,
+                 opt_kwargs: dict | None = None):
+        self.wl = wl
+        self.hyper = dict(wl.hyper, **(hyper_override or {}))
+        self.flat_p = W.alloc_flat(wl, torch.float32, device)
+        W.init_params(wl, self.flat_p)
+        self.flat_g = W.alloc_flat(wl, wl.grad_dtype, device)
+        self.scratch = (W.alloc_flat(wl, torch.float32, device)
+                        if wl.grad_dtype != torch.float32 else None)
+        self.params = W.views(self.flat_p, wl)
+        self.grads = W.views(self.flat_g, wl)
+        idx, tid, local = W.sample_indices(wl)
+        self.idx = idx.to(device)
+        self.tid, self.local = tid, local
+        self.src = W.GradSource(wl, device)
+        self.oracle = O.Oracle(oracle_config(self.hyper), [to_f64(self.flat_p[self.idx])])
+        self.opt = B.NovakOptimizer(self.params, **self.hyper, **(opt_kwargs or {}))
+        self.glist = self.opt.prepare(self.grads)
+        self.sync_steps, self.rect_flags = [], []
+
+    def step(self, threads=1):
+        self.src.fill(self.flat_g, self.scratch)
+        self.opt.step(self.glist)
+        info = self.opt.info()
+        if info["is_sync"]:
+            self.sync_steps.append(info["t"])
+        self.rect_flags.append(info["rect_branch"])
+        self.oracle.step([to_f64(self.flat_g[self.idx])], threads=threads)
+
+    def _gather_state(self, key):
+        out = torch.empty(self.idx.numel(), dtype=torch.float32, device=self.idx.device)
+        bounds = torch.searchsorted(self.tid, torch.arange(len(self.wl.numel) + 1))
+        for i in range(len(self.wl.numel)):
+            lo, hi = int(bounds[i]), int(bounds[i + 1])
+            if hi > lo:
+                out[lo:hi] = self.opt.state(i)[key][self.local[lo:hi].to(out.device)]
+        return out
+
+    def check(self):
+        torch.cuda.synchronize()
+        o, info = self.oracle, self.opt.info()
+        assert info["t"] == o.t and self.sync_steps == o.sync_steps
+        assert self.rect_flags == o.rect_flags
+        assert info["n_syncs"] == len(o.sync_steps)
+        name = self.wl.name
+        assert_close(self.flat_p[self.idx], o.theta[0], f"{name} theta")
+        assert_close(self._gather_state("m"), o.m[0], f"{name} m")
+        assert_close(self._gather_state("v"), o.v[0], f"{name} v")
+        if o.slow is not None:
+            assert_close(self._gather_state("slow"), o.slow[0], f"{name} slow")
+        if o.acc is not None and o.cfg.lookahead_k > 1 and o.t % o.cfg.lookahead_k != 0:
+            assert_close(self._gather_state("acc"), o.acc[0], f"{name} acc")

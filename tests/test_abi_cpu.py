@@ -1,0 +1,165 @@
+"""Host-side checks of the C-ABI library that need no GPU: exported symbols,
+hyperparameter validation, the downgrade rule, the scalar planner against the
+oracle's independently computed scalars, the chunk-table builder."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import novak_oracle as O
+from paper_2601_07876_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    return B.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "novak.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    names = set(re.findall(r"\b(novak_[a-z_]+)\s*\(", header))
+    assert {"novak_create", "novak_step", "novak_destroy"} <= names
+    for name in sorted(names):
+        assert hasattr(lib, name), f"{name} declared in novak.h but not exported"
+    # and the binding declares a signature for each of them
+    src = open(os.path.join(ROOT, "paper_2601_07876_b200", "binding.py")).read()
+    for name in sorted(names):
+        assert f'"{name}"' in src, f"binding has no signature for {name}"
+
+
+def test_struct_sizes_match_header(lib):
+    # The C structs end on 8-byte boundaries; a drifted field would shift these.
+    assert ctypes.sizeof(B.novak_info) == 5 * 8 + 7 * 8 + 10 * 4
+    assert ctypes.sizeof(B.novak_meta) == 8 + 4 * 8 + 7 * 8 + 8 * 4
+
+
+GOOD = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2,
+            nesterov_variant=1, lookahead_k=5, lookahead_alpha=0.5)
+
+
+@pytest.mark.parametrize("bad", [
+    dict(lr=0.0), dict(lr=-1.0), dict(lr=float("nan")), dict(lr=float("inf")),
+    dict(beta1=1.0), dict(beta1=-0.1), dict(beta2=1.0), dict(beta2=1 - 1e-9),
+    dict(beta2=float("nan")), dict(eps=0.0), dict(eps=-1e-8), dict(weight_decay=-1e-3),
+    dict(nesterov_variant=4), dict(nesterov_variant=-1), dict(lookahead_k=-1),
+    dict(lookahead_alpha=0.0), dict(lookahead_alpha=1.0), dict(lookahead_alpha=float("nan")),
+])
+def test_create_rejects_invalid_hyperparameters(bad):
+    """Section 5.8, hyperparameter validation."""
+    with pytest.raises(B.NovakError) as e:
+        B.Handle(**{**GOOD, **bad})
+    assert e.value.status == B.NOVAK_EINVAL
+
+
+def test_create_accepts_boundaries():
+    B.Handle(**{**GOOD, "beta1": 0.0, "beta2": 0.0, "weight_decay": 0.0}).destroy()
+    # lookahead off: alpha is not looked at
+    B.Handle(**{**GOOD, "lookahead_k": 0, "lookahead_alpha": 7.0}).destroy()
+
+
+def test_true_nesterov_is_downgraded_with_warning():
+    """Section 7.3: the fast path runs 'true' as 'approximation' and warns."""
+    h = B.Handle(**{**GOOD, "nesterov_variant": B.NOVAK_NESTEROV_TRUE})
+    info = h.get_info()
+    assert info.nesterov_variant == B.NOVAK_NESTEROV_APPROX
+    assert info.warnings & B.NOVAK_WARN_TRUE_DOWNGRADED
+    h2 = B.Handle(**GOOD)
+    assert h2.get_info().warnings == 0
+
+
+def test_options_validate_and_roundtrip():
+    h = B.Handle(**GOOD)
+    assert h.get_option(B.NOVAK_OPT_NESTEROV_BETA) == 0.9   # default beta_N = beta1
+    h.set_option(B.NOVAK_OPT_NESTEROV_BETA, 0.5)
+    assert h.get_option(B.NOVAK_OPT_NESTEROV_BETA) == 0.5
+    for key, bad in ((B.NOVAK_OPT_NESTEROV_BETA, 1.0), (B.NOVAK_OPT_LOOKAHEAD_MODE, 2),
+                     (B.NOVAK_OPT_RECTIFIED, 3), (B.NOVAK_OPT_LR, 0.0),
+                     (B.NOVAK_OPT_BIAS1_POWER, 3), (B.NOVAK_OPT_CHUNK_ELEMS, 1000),
+                     (B.NOVAK_OPT_CTAS_PER_SM, -1), (B.NOVAK_OPT_WEIGHT_DECAY, -1.0),
+                     (99, 1.0)):
+        with pytest.raises(B.NovakError) as e:
+            h.set_option(key, bad)
+        assert e.value.status == B.NOVAK_EINVAL
+        assert h.last_error()
+    h.set_option(B.NOVAK_OPT_LR, 5e-4)
+    assert h.get_option(B.NOVAK_OPT_LR) == 5e-4
+
+
+def test_step_without_state_is_estate():
+    h = B.Handle(**GOOD)
+    arr = B.ptr_array([16])
+    with pytest.raises(B.NovakError) as e:
+        h.step(arr, arr, B.i64_array([4]), 1, B.NOVAK_GRAD_F32)
+    assert e.value.status == B.NOVAK_ESTATE
+    assert h.get_info().t == 0
+
+
+def test_state_bytes():
+    h = B.Handle(**GOOD)                       # lookahead LAST: m, v, slow
+    # each tensor gets a slot of round_up(numel + 31, 32) elements
+    assert h.state_bytes([1]) == 3 * 32 * 4
+    assert h.state_bytes([32, 33]) == 3 * (64 + 64) * 4
+    assert h.state_bytes([0]) == 0 and h.state_bytes([5, -1]) == 0
+    h.set_option(B.NOVAK_OPT_LOOKAHEAD_MODE, B.NOVAK_LOOKAHEAD_TRAJ_MEAN)
+    assert h.state_bytes([1]) == 4 * 32 * 4
+    h0 = B.Handle(**{**GOOD, "lookahead_k": 0})
+    assert h0.state_bytes([1]) == 2 * 32 * 4
+
+
+@pytest.mark.parametrize("kw", [
+    dict(), dict(beta1=0.8, beta2=0.99), dict(beta2=0.6), dict(beta1=0.0, beta2=0.5),
+    dict(beta2=0.9999, lr=3e-2, weight_decay=0.3), dict(lookahead_k=1), dict(lookahead_k=7),
+])
+def test_planner_agrees_with_oracle_scalars(kw):
+    """The library's scalar plan (-expm1(t log beta), double) against the
+    oracle's (powl, long double): Eq. 5-9, 18 and the sync schedule."""
+    g = {**GOOD, **kw}
+    h = B.Handle(**g)
+    o = O.Oracle(O.Config(lr=g["lr"], beta1=g["beta1"], beta2=g["beta2"], eps=g["eps"],
+                          weight_decay=g["weight_decay"], lookahead_k=g["lookahead_k"],
+                          lookahead_alpha=g["lookahead_alpha"]), [np.zeros(1)])
+    for t in list(range(1, 40)) + [100, 999, 1000, 1001, 12345, 10 ** 6, 10 ** 8]:
+        a, b = h.plan(t), o.scalars(t)
+        assert a.rect_branch == b.rect_branch and a.is_sync == b.is_sync, t
+        for name in ("bc1", "bc2", "rho_inf", "r_t", "step_size", "decay"):
+            x, y = getattr(a, name), getattr(b, name)
+            assert abs(x - y) <= 1e-12 * abs(y), (t, name, x, y)
+        assert abs(a.rho_t - b.rho_t) <= 1e-9 * max(1.0, b.rho_inf), (t, a.rho_t, b.rho_t)
+
+
+def test_planner_options():
+    h = B.Handle(**GOOD)
+    h.set_option(B.NOVAK_OPT_RECTIFIED, 0)
+    assert h.plan(50).rect_branch == 0 and h.plan(50).r_t == 1.0
+    h.set_option(B.NOVAK_OPT_RECTIFIED, 1)
+    p1 = h.plan(7)
+    h.set_option(B.NOVAK_OPT_BIAS1_POWER, 2)
+    p2 = h.plan(7)
+    assert abs(p2.step_size * p2.bc1 - p1.step_size) < 1e-18
+
+
+def test_chunk_builder_covers_every_element_once():
+    numel = [1, 31, 32, 33, 8192, 8193, 100_000, 5]
+    phase = [0, 3, 31, 0, 7, 0, 16, 30]
+    for C in (1024, 8192):
+        t, o, ln = B.novak_build_chunks(numel, phase, C)
+        seen = [np.zeros(n, dtype=np.int32) for n in numel]
+        for ti, oi, li in zip(t, o, ln):
+            assert 0 < li <= C
+            seen[ti][oi:oi + li] += 1
+            # every entry after a tensor's head starts on a 128-byte boundary
+            if oi > 0:
+                assert (phase[ti] + oi) % 32 == 0
+        assert all((s == 1).all() for s in seen)
+        # a tensor with phase 0 has no head entry
+        assert [li for ti, li in zip(t, ln) if ti == 3] == [33]
+        assert [li for ti, li in zip(t, ln) if ti == 1] == [29, 2]
+    with pytest.raises(B.NovakError):
+        B.novak_build_chunks([0], None, 1024)
+    with pytest.raises(B.NovakError):
+        B.novak_build_chunks([5], [32], 1024)
