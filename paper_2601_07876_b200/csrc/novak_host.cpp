@@ -23,7 +23,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
 constexpr uint64_t kMetaMagic = 0x4e4f56414b763031ull;  // "NOVAKv01"
-constexpr int64_t kDefaultChunkElems = 8192;
+constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 
 struct Hyper {
