@@ -202,6 +202,40 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
                     void *const *d_grads, const int64_t *numel, int n,
                     int grad_dtype, void *stream);
 
+/* The paper has no counterpart of this call; it exists for callers that must
+ * not allocate device memory.
+ *
+ * novak_step with its device work table (tensor records + chunk table) kept in
+ * an array that is part of the library image itself instead of memory obtained
+ * from cudaMalloc.  It is meant for processes in which a framework's pool owns
+ * all device memory up front and a later cudaMalloc would fail or fragment it,
+ * and for call sites (real-time loops, callbacks of an allocator) where an
+ * allocation may not happen at all.  The call itself, on every invocation, makes
+ * no cudaMalloc / cudaFree / cudaHostAlloc / event creation; parameters,
+ * gradients and the state buffer are the caller's as in novak_step.
+ *
+ * Limits: at most 4096 tensors and 131072 chunk-table entries (= 268 M
+ * elements at the default 2048 elements per entry; raise
+ * NOVAK_OPT_CHUNK_ELEMS before the first step for larger groups).  Beyond that
+ * the call returns NOVAK_EINVAL with the limit in novak_last_error() and does
+ * nothing.  The array costs 2.2 MiB on every GPU that loads the library, until
+ * the process exits.
+ *
+ * The array is ONE per GPU and shared by every handle and every call.  It keeps
+ * what the last call wrote; each call rewrites, in stream order, the part it
+ * reads whenever another handle used the table in between or this handle's
+ * pointers changed (nothing in it needs to start from zero).  Two calls that
+ * may overlap on the GPU (different streams, no ordering between them) race on
+ * the table: order them yourself.
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.
+ * Arguments, results and errors otherwise as novak_step; both calls may be
+ * mixed on one handle and advance the same step counter. */
+int novak_step_noalloc(novak_opt *opt, void *const *d_params,
+                       const void *const *d_grads, const int64_t *numel, int n,
+                       int grad_dtype, void *stream);
+
 /* Counters and the last step's scalars (bit-exact step and sync indices). */
 int novak_get_info(const novak_opt *opt, novak_info *out);
 

@@ -97,6 +97,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_state_bytes": (c_size_t, [vp, i64p, c_int]),
         "novak_attach_state": (c_int, [vp, vp, c_size_t, vpp, i64p, c_int, vp]),
         "novak_step": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_step_noalloc": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
         "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
@@ -198,6 +199,15 @@ class Handle:
         st = self.lib.novak_step(self.h, params_arr, grads_arr, numel_arr, n, grad_dtype, stream)
         if st != NOVAK_OK:
             _check(self.lib, self.h, st, "novak_step")
+
+    def step_noalloc(self, params_arr, grads_arr, numel_arr, n: int, grad_dtype: int,
+                     stream: int = 0):
+        """novak_step for callers that must not allocate device memory: the work
+        table lives in an array inside the library (see novak.h for its limits)."""
+        st = self.lib.novak_step_noalloc(self.h, params_arr, grads_arr, numel_arr, n,
+                                         grad_dtype, stream)
+        if st != NOVAK_OK:
+            _check(self.lib, self.h, st, "novak_step_noalloc")
 
     def step_host(self, h_params_arr, h_grads_arr, d_params_arr, d_grads_arr, numel_arr, n,
                   grad_dtype: int, stream: int = 0):

@@ -143,6 +143,14 @@ struct novak_opt {
     int cur_gdtype = -1;
     int sms = 0;
 
+    // host copies of the work table for novak_step_noalloc (no device memory of ours)
+    std::vector<Chunk> na_chunks;
+    std::vector<TensorRec> na_recs;
+    std::vector<void *> na_p;
+    std::vector<const void *> na_g;
+    int na_gdtype = -1;
+    uint64_t na_token = 0;       // identifies this handle's upload in the shared table
+
     std::string err;
 };
 
@@ -402,7 +410,8 @@ int novak_set_option(novak_opt *o, int key, double value)
         h.bias1_power = static_cast<int>(value);
         break;
     case NOVAK_OPT_CHUNK_ELEMS: {
-        if (o->d_chunks) return fail(o, NOVAK_ESTATE, "chunk size is fixed once a step was taken");
+        if (o->d_chunks || !o->na_chunks.empty())
+            return fail(o, NOVAK_ESTATE, "chunk size is fixed once a step was taken");
         const int64_t c = static_cast<int64_t>(value);
         if (!(value >= 1024.0 && value <= 16777216.0) || c % 1024 != 0 || static_cast<double>(c) != value)
             return fail(o, NOVAK_EINVAL, "chunk_elems must be a multiple of 1024 in [1024, 2^24]");
@@ -477,6 +486,9 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     if (e != cudaSuccess) return fail_cuda(o, e, "cudaMemsetAsync(state)");
 
     release_device(o);
+    o->na_chunks.clear();
+    o->na_p.clear();
+    o->na_token = 0;
     o->d_state = static_cast<char *>(d_state);
     o->n = n;
     o->n_arrays = n_state_arrays(o->h);
@@ -594,6 +606,129 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
             return fail_cuda(o, e, "parameter download");
         i = j;
     }
+    return NOVAK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// novak_step_noalloc: the same step with its work table in the library's
+// statically allocated device array instead of cudaMalloc'ed memory.
+// ---------------------------------------------------------------------------
+namespace {
+// Which upload the shared table of each device currently holds (0 = none).
+uint64_t g_noalloc_owner[64] = {};
+uint64_t g_noalloc_next_token = 1;
+}  // namespace
+
+int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d_grads,
+                       const int64_t *numel, int n, int grad_dtype, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "step_noalloc: no state attached");
+    if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step_noalloc: NULL argument");
+    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16)
+        return fail(o, NOVAK_EINVAL, "step_noalloc: unknown grad_dtype %d", grad_dtype);
+    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
+        return fail(o, NOVAK_ESTATE, "step_noalloc: tensor list differs from the attached layout");
+    if (n > novak::kNoAllocMaxTensors)
+        return fail(o, NOVAK_EINVAL, "step_noalloc: %d tensors exceed the static table's %d; "
+                    "split the group or use novak_step", n, novak::kNoAllocMaxTensors);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    if (o->na_chunks.empty())
+        build_chunks(o->numel.data(), o->phase.data(), o->n, o->chunk_elems, o->na_chunks);
+    if (o->na_chunks.size() > static_cast<size_t>(novak::kNoAllocMaxChunks)) {
+        const size_t need = o->na_chunks.size();
+        o->na_chunks.clear();
+        return fail(o, NOVAK_EINVAL, "step_noalloc: %zu chunk-table entries exceed the static "
+                    "table's %d; raise NOVAK_OPT_CHUNK_ELEMS (now %lld) or use novak_step",
+                    need, novak::kNoAllocMaxChunks, static_cast<long long>(o->chunk_elems));
+    }
+
+    // tensor records: rebuilt on the host when the caller's pointers changed
+    bool changed = o->na_gdtype != grad_dtype || o->na_p.empty() ||
+                   std::memcmp(o->na_p.data(), d_params, n * sizeof(void *)) != 0 ||
+                   std::memcmp(o->na_g.data(), d_grads, n * sizeof(void *)) != 0;
+    if (changed) {
+        const uintptr_t gmask = grad_dtype == NOVAK_GRAD_BF16 ? 1u : 3u;
+        for (int i = 0; i < n; ++i) {
+            const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
+            const uintptr_t g = reinterpret_cast<uintptr_t>(d_grads[i]);
+            if (!p || !g) return fail(o, NOVAK_EINVAL, "tensor %d: NULL pointer", i);
+            if ((p & 3u) || (g & gmask))
+                return fail(o, NOVAK_EINVAL, "tensor %d: pointer not aligned to its element size", i);
+        }
+        const bool la = o->h.la_k > 0;
+        const bool traj = la && o->h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN;
+        o->na_recs.resize(n);
+        for (int i = 0; i < n; ++i) {
+            TensorRec &r = o->na_recs[i];
+            r.p = static_cast<float *>(d_params[i]);
+            r.g = d_grads[i];
+            r.m = slice(o, 0, i);
+            r.v = slice(o, 1, i);
+            r.slow = la ? slice(o, 2, i) : nullptr;
+            r.acc = traj ? slice(o, 3, i) : nullptr;
+        }
+        o->na_p.assign(d_params, d_params + n);
+        o->na_g.assign(d_grads, d_grads + n);
+        o->na_gdtype = grad_dtype;
+        o->na_token = 0;  // forces an upload below
+    }
+
+    // The static table of the current device (first call on a device resolves
+    // its address; nothing is allocated).
+    TensorRec *d_recs = nullptr;
+    Chunk *d_chunks = nullptr;
+    int dev = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(o, e, "cudaGetDevice");
+    if ((e = novak::noalloc_table(&d_recs, &d_chunks)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaGetSymbolAddress(static work table)");
+    if (o->na_token == 0 || g_noalloc_owner[dev] != o->na_token) {
+        // Every handle shares the table: (re)write the part this step reads.
+        // Copies from pageable memory are staged by the driver before the call
+        // returns, so the host vectors may change afterwards.
+        if ((e = cudaMemcpyAsync(d_recs, o->na_recs.data(), n * sizeof(TensorRec),
+                                 cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+            (e = cudaMemcpyAsync(d_chunks, o->na_chunks.data(), o->na_chunks.size() * sizeof(Chunk),
+                                 cudaMemcpyHostToDevice, stream)) != cudaSuccess) {
+            g_noalloc_owner[dev] = 0;
+            return fail_cuda(o, e, "static work table upload");
+        }
+        o->na_token = g_noalloc_next_token++;
+        g_noalloc_owner[dev] = o->na_token;
+    }
+
+    const int64_t t = o->t + 1;
+    const Plan p = make_plan(o->h, t);
+    const int la_action = lookahead_action(o->h, t);
+    StepScalars s;
+    s.beta1 = static_cast<float>(o->h.beta1);
+    s.omb1 = static_cast<float>(1.0 - o->h.beta1);
+    s.beta2 = static_cast<float>(o->h.beta2);
+    s.omb2 = static_cast<float>(1.0 - o->h.beta2);
+    s.beta_n = static_cast<float>(o->h.beta_n);
+    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
+    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
+    s.eps = static_cast<float>(o->h.eps);
+    s.decay = static_cast<float>(p.decay);
+    s.step = static_cast<float>(p.step_size);
+    s.la_alpha = static_cast<float>(o->h.la_alpha);
+    s.k = static_cast<float>(o->h.la_k > 0 ? o->h.la_k : 1);
+
+    const int n_chunks = static_cast<int>(o->na_chunks.size());
+    novak::LaunchCfg cfg;
+    cfg.grid = n_chunks;
+    cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
+    e = novak::launch_step(d_chunks, n_chunks, d_recs, s, o->h.nesterov, grad_dtype, la_action,
+                           cfg, stream);
+    if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
+
+    o->t = t;
+    o->launches += 1;
+    o->last_plan = p;
+    o->last_grid = cfg.grid;
+    if (p.is_sync) { o->n_syncs += 1; o->last_sync = t; }
     return NOVAK_OK;
 }
 

@@ -67,4 +67,13 @@ cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_
                         const StepScalars &s, int nesterov, int grad_dtype, int la,
                         const LaunchCfg &cfg, cudaStream_t stream);
 
+// ---- work table for callers that cannot allocate device memory --------------
+// Capacity of the statically allocated table behind novak_step_noalloc.
+constexpr int kNoAllocMaxTensors = 4096;
+constexpr int kNoAllocMaxChunks = 131072;
+
+// Device addresses of the static table on the CURRENT device (resolved once per
+// device with cudaGetSymbolAddress).  No allocation.
+cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks);
+
 }  // namespace novak

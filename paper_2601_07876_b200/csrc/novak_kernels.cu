@@ -279,6 +279,36 @@ KernelFn pick_kernel(int nesterov, int grad_dtype, int la)
 
 }  // namespace
 
+// Work table of novak_step_noalloc: tensor records followed by the chunk table,
+// resident in every GPU that loads this library until the process exits
+// (192 KiB + 2 MiB).  In host code this name is only a handle for
+// cudaGetSymbolAddress, never a device address.
+struct NoAllocTable {
+    TensorRec recs[kNoAllocMaxTensors];
+    Chunk chunks[kNoAllocMaxChunks];
+};
+static __device__ __align__(256) unsigned char g_noalloc_table[sizeof(NoAllocTable)];
+
+cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks)
+{
+    constexpr int kMaxDevices = 64;
+    static void *resolved[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!resolved[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_noalloc_table);  // address on the current device
+        if (e != cudaSuccess) return e;
+        resolved[dev] = ptr;
+    }
+    NoAllocTable *t = static_cast<NoAllocTable *>(resolved[dev]);
+    *d_recs = t->recs;
+    *d_chunks = t->chunks;
+    return cudaSuccess;
+}
+
 int step_block_threads() { return kBlock; }
 
 cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int *ctas_per_sm)
