@@ -57,6 +57,7 @@ def parse_args():
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
     ap.add_argument("--serpentine", type=int, default=None)
+    ap.add_argument("--dependent-launch", type=int, default=None)
     ap.add_argument("--lib", default=None, help="alternative libnovak.so (tuning builds)")
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-e2e", action="store_true")
@@ -274,7 +275,8 @@ def main():
         src.fill(gf, scratch)
     del scratch
     opt = B.NovakOptimizer(params, **hyper, chunk_elems=args.chunk_elems,
-                           ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine, lib=lib)
+                           ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
+                           dependent_launch=args.dependent_launch, lib=lib)
     pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
 
     def barrier():
@@ -287,6 +289,7 @@ def main():
         opt.step(pool[i % pool_n])
     t_first = opt.info()["t"] + 1
     launches0 = opt.info()["launches"]
+    uploads0 = opt.info()["record_uploads"]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with ClockSampler(local) as clocks:
@@ -297,6 +300,7 @@ def main():
         barrier()
     ms = ev0.elapsed_time(ev1)
     launches = opt.info()["launches"] - launches0
+    uploads = opt.info()["record_uploads"] - uploads0
     if world > 1:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -385,6 +389,8 @@ def main():
                 "chunk_elems": int(opt.handle.get_option(B.NOVAK_OPT_CHUNK_ELEMS)),
                 "ctas_per_sm": int(opt.handle.get_option(B.NOVAK_OPT_CTAS_PER_SM)),
                 "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
+                "dependent_launch": int(opt.handle.get_option(B.NOVAK_OPT_DEPENDENT_LAUNCH)),
+                "record_uploads_in_timed_region": uploads,
                 "grid": info["grid"], "block": info["block"], "n_chunks": info["n_chunks"],
                 "replicas": "each rank steps its own replica; no data-path collective",
             },

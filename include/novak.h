@@ -83,7 +83,13 @@ enum {
     NOVAK_OPT_CTAS_PER_SM = 7,    /* persistent grid = SMs x this; 0: one CTA per chunk */
     NOVAK_OPT_SERPENTINE = 8,     /* 1: walk the chunk table backwards on even steps so
                                      the tail of one step is still in L2 for the next  */
-    NOVAK_OPT_WEIGHT_DECAY = 9    /* lambda >= 0; may change between steps             */
+    NOVAK_OPT_WEIGHT_DECAY = 9,   /* lambda >= 0; may change between steps             */
+    NOVAK_OPT_DEPENDENT_LAUNCH = 10 /* 1 (default): launch the step kernel with
+                                     programmatic stream serialization, so its CTAs
+                                     become resident and fetch their work-table
+                                     entries while the previous kernel on the stream
+                                     drains; they touch no tensor before that kernel
+                                     has completed.  0: plain launch               */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -100,6 +106,8 @@ typedef struct novak_info {
     int64_t last_sync_step; /* t of the most recent one, 0 if none                 */
     int64_t total_numel;
     int64_t launches;       /* kernels launched by this handle since creation      */
+    int64_t record_uploads; /* times novak_step had to copy the tensor records to
+                               the device (a pointer list it did not hold yet)     */
     double bc1, bc2;        /* 1-beta1^t, 1-beta2^t of the last step       (Eq. 5) */
     double rho_inf, rho_t;  /*                                          (Eq. 6-7)  */
     double r_t;             /* Eq. 9, or 1 on the un-rectified branch              */
@@ -179,8 +187,10 @@ int novak_attach_state(novak_opt *opt, void *d_state, size_t bytes,
  * d_grads:  host array of n device pointers to contiguous gradients of
  *           grad_dtype (fp32, or bf16 widened exactly), read only.
  * numel:    must equal the attached layout (NOVAK_ESTATE otherwise).
- * Pointers may change between steps (the device tensor records are refreshed
- * in stream order when they do).  Tensors whose parameter, gradient and state
+ * Pointers may change between steps: the handle keeps the device tensor records
+ * of the 8 most recently used (params, grads) pointer lists, so a caller that
+ * cycles through a few gradient buffers enqueues nothing but the kernel; a list
+ * it does not hold is uploaded in stream order (novak_info.record_uploads).  Tensors whose parameter, gradient and state
  * addresses are congruent modulo 16 bytes run on 128-bit accesses; others on
  * 4-byte accesses (NOVAK_WARN_SCALAR_PATH).
  * Errors: NOVAK_EINVAL (NULL, n mismatch, bad dtype, misaligned pointer),

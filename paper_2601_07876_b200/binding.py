@@ -26,7 +26,7 @@ NOVAK_GRAD_F32, NOVAK_GRAD_BF16 = 0, 1
 NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
 (NOVAK_OPT_NESTEROV_BETA, NOVAK_OPT_LOOKAHEAD_MODE, NOVAK_OPT_RECTIFIED, NOVAK_OPT_LR,
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
- NOVAK_OPT_WEIGHT_DECAY) = range(1, 10)
+ NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH) = range(1, 11)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -35,7 +35,7 @@ _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA"
 class novak_info(Structure):
     _fields_ = [
         ("t", c_int64), ("n_syncs", c_int64), ("last_sync_step", c_int64),
-        ("total_numel", c_int64), ("launches", c_int64),
+        ("total_numel", c_int64), ("launches", c_int64), ("record_uploads", c_int64),
         ("bc1", c_double), ("bc2", c_double), ("rho_inf", c_double), ("rho_t", c_double),
         ("r_t", c_double), ("step_size", c_double), ("decay", c_double),
         ("rect_branch", c_int32), ("is_sync", c_int32), ("nesterov_variant", c_int32),
@@ -278,7 +278,8 @@ class NovakOptimizer:
     def __init__(self, params, lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
-                 chunk_elems=None, ctas_per_sm=None, serpentine=None, lib=None):
+                 chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
+                 lib=None):
         import torch
         self.params = list(params)
         if not self.params:
@@ -303,6 +304,8 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_CTAS_PER_SM, ctas_per_sm)
         if serpentine is not None:
             h.set_option(NOVAK_OPT_SERPENTINE, 1 if serpentine else 0)
+        if dependent_launch is not None:
+            h.set_option(NOVAK_OPT_DEPENDENT_LAUNCH, 1 if dependent_launch else 0)
         self.numel = [p.numel() for p in self.params]
         self.n = len(self.params)
         self._numel_arr = i64_array(self.numel)

@@ -21,6 +21,7 @@ using novak::TensorRec;
 namespace {
 
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
+constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
 constexpr uint64_t kMetaMagic = 0x4e4f56414b763031ull;  // "NOVAKv01"
 constexpr int64_t kDefaultChunkElems = 2048;
@@ -115,6 +116,7 @@ struct novak_opt {
     int64_t chunk_elems = kDefaultChunkElems;
     int ctas_per_sm = kDefaultCtasPerSm;
     int serpentine = 0;
+    int pdl = 1;
 
     // state layout (fixed by novak_attach_state)
     bool attached = false;
@@ -134,13 +136,24 @@ struct novak_opt {
     // device work table
     Chunk *d_chunks = nullptr;
     int n_chunks = 0;
-    TensorRec *d_recs = nullptr;
+    TensorRec *d_recs = nullptr;       // kRecTables tables of n records each
     TensorRec *h_recs[kRing] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ring_ev[kRing] = {nullptr, nullptr, nullptr, nullptr};
     int ring_pos = 0;
-    std::vector<void *> cur_p;
-    std::vector<const void *> cur_g;
-    int cur_gdtype = -1;
+    // Which (parameter, gradient) pointer lists the device tables hold.  A
+    // caller that rotates through a few gradient buffers finds its table
+    // already resident and the step enqueues nothing but the kernel.
+    struct RecTable {
+        std::vector<void *> p;
+        std::vector<const void *> g;
+        int gdtype = -1;
+        uint64_t hash = 0;
+        int64_t last_use = 0;
+    };
+    RecTable tables[kRecTables];
+    int cur_table = -1;
+    int64_t table_clock = 0;
+    int64_t record_uploads = 0;
     int sms = 0;
 
     // host copies of the work table for novak_step_noalloc (no device memory of ours)
@@ -198,6 +211,7 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->last_sync_step = o->last_sync;
     out->total_numel = o->total_numel;
     out->launches = o->launches;
+    out->record_uploads = o->record_uploads;
     out->bc1 = p.bc1; out->bc2 = p.bc2;
     out->rho_inf = p.rho_inf; out->rho_t = p.rho_t;
     out->r_t = p.r_t; out->step_size = p.step_size; out->decay = p.decay;
@@ -225,9 +239,13 @@ void release_device(novak_opt *o)
     o->d_chunks = nullptr;
     o->d_recs = nullptr;
     o->n_chunks = 0;
-    o->cur_p.clear();
-    o->cur_g.clear();
-    o->cur_gdtype = -1;
+    for (auto &tb : o->tables) {
+        tb.p.clear();
+        tb.g.clear();
+        tb.gdtype = -1;
+        tb.last_use = 0;
+    }
+    o->cur_table = -1;
 }
 
 // First step: chunk table and record buffers on the device.
@@ -255,9 +273,9 @@ int prepare_device(novak_opt *o, cudaStream_t stream)
         release_device(o);
         return fail(o, NOVAK_ENOMEM, "cudaMalloc(chunk table, %zu B): %s", cbytes, cudaGetErrorString(e));
     }
-    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_recs), rbytes)) != cudaSuccess) {
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_recs), rbytes * kRecTables)) != cudaSuccess) {
         release_device(o);
-        return fail(o, NOVAK_ENOMEM, "cudaMalloc(tensor records, %zu B): %s", rbytes, cudaGetErrorString(e));
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(tensor records, %zu B): %s", rbytes * kRecTables, cudaGetErrorString(e));
     }
     for (int i = 0; i < kRing; ++i) {
         if ((e = cudaHostAlloc(reinterpret_cast<void **>(&o->h_recs[i]), rbytes, cudaHostAllocDefault)) != cudaSuccess ||
@@ -277,15 +295,36 @@ int prepare_device(novak_opt *o, cudaStream_t stream)
     return NOVAK_OK;
 }
 
-// Refreshes the device tensor records when the caller's pointers changed.
+uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype)
+{
+    uint64_t h = 0xcbf29ce484222325ull ^ static_cast<uint64_t>(grad_dtype);
+    for (int i = 0; i < n; ++i) {
+        h = (h ^ reinterpret_cast<uintptr_t>(d_params[i])) * 0x100000001b3ull;
+        h = (h ^ reinterpret_cast<uintptr_t>(d_grads[i])) * 0x100000001b3ull;
+    }
+    return h;
+}
+
+// Selects the device record table that holds the caller's pointer lists,
+// uploading them (in stream order, into the least recently used table) when
+// none does.
 int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
                     int grad_dtype, cudaStream_t stream)
 {
     const int n = o->n;
-    const bool same = o->cur_gdtype == grad_dtype && !o->cur_p.empty() &&
-                      std::memcmp(o->cur_p.data(), d_params, n * sizeof(void *)) == 0 &&
-                      std::memcmp(o->cur_g.data(), d_grads, n * sizeof(void *)) == 0;
-    if (same) return NOVAK_OK;
+    const uint64_t hash = hash_pointers(d_params, d_grads, n, grad_dtype);
+    int lru = 0;
+    for (int k = 0; k < kRecTables; ++k) {
+        novak_opt::RecTable &tb = o->tables[k];
+        if (tb.gdtype == grad_dtype && tb.hash == hash && !tb.p.empty() &&
+            std::memcmp(tb.p.data(), d_params, n * sizeof(void *)) == 0 &&
+            std::memcmp(tb.g.data(), d_grads, n * sizeof(void *)) == 0) {
+            tb.last_use = ++o->table_clock;
+            o->cur_table = k;
+            return NOVAK_OK;
+        }
+        if (tb.last_use < o->tables[lru].last_use) lru = k;
+    }
 
     const uintptr_t gmask = grad_dtype == NOVAK_GRAD_BF16 ? 1u : 3u;
     const uintptr_t gvec = grad_dtype == NOVAK_GRAD_BF16 ? 8u : 16u;
@@ -315,14 +354,23 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         h[i].slow = la ? slice(o, 2, i) : nullptr;
         h[i].acc = traj ? slice(o, 3, i) : nullptr;
     }
-    if ((e = cudaMemcpyAsync(o->d_recs, h, n * sizeof(TensorRec), cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    // Stream order puts this copy behind every earlier launch that read the
+    // table being replaced.
+    novak_opt::RecTable &tb = o->tables[lru];
+    tb.p.clear();
+    if ((e = cudaMemcpyAsync(o->d_recs + static_cast<size_t>(lru) * n, h, n * sizeof(TensorRec),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return fail_cuda(o, e, "tensor record upload");
     if ((e = cudaEventRecord(o->ring_ev[slot], stream)) != cudaSuccess)
         return fail_cuda(o, e, "cudaEventRecord(record ring)");
     o->ring_pos = (slot + 1) % kRing;
-    o->cur_p.assign(d_params, d_params + n);
-    o->cur_g.assign(d_grads, d_grads + n);
-    o->cur_gdtype = grad_dtype;
+    tb.p.assign(d_params, d_params + n);
+    tb.g.assign(d_grads, d_grads + n);
+    tb.gdtype = grad_dtype;
+    tb.hash = hash;
+    tb.last_use = ++o->table_clock;
+    o->cur_table = lru;
+    o->record_uploads += 1;
     if (scalar_path) o->warnings |= NOVAK_WARN_SCALAR_PATH;
     return NOVAK_OK;
 }
@@ -428,6 +476,10 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "serpentine must be 0 or 1");
         o->serpentine = static_cast<int>(value);
         return NOVAK_OK;
+    case NOVAK_OPT_DEPENDENT_LAUNCH:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "dependent_launch must be 0 or 1");
+        o->pdl = static_cast<int>(value);
+        return NOVAK_OK;
     default:
         return fail(o, NOVAK_EINVAL, "unknown option key %d", key);
     }
@@ -449,6 +501,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
+    case NOVAK_OPT_DEPENDENT_LAUNCH: *value = o->pdl; break;
     default: return NOVAK_EINVAL;
     }
     return NOVAK_OK;
@@ -545,7 +598,9 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     cfg.grid = o->n_chunks;
     if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
-    cudaError_t e = novak::launch_step(o->d_chunks, o->n_chunks, o->d_recs, s, o->h.nesterov,
+    cfg.pdl = o->pdl;
+    const TensorRec *d_recs = o->d_recs + static_cast<size_t>(o->cur_table) * o->n;
+    cudaError_t e = novak::launch_step(o->d_chunks, o->n_chunks, d_recs, s, o->h.nesterov,
                                        grad_dtype, la, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
 
@@ -720,6 +775,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     novak::LaunchCfg cfg;
     cfg.grid = n_chunks;
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
+    cfg.pdl = o->pdl;
     e = novak::launch_step(d_chunks, n_chunks, d_recs, s, o->h.nesterov, grad_dtype, la_action,
                            cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");

@@ -53,6 +53,7 @@ enum : int {
 struct LaunchCfg {
     int grid;
     int reverse;     // walk the chunk table from the end
+    int pdl;         // launch with programmatic stream serialization
 };
 
 // Threads per CTA of the step kernel (fixed at compile time).

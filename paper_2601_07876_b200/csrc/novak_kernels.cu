@@ -197,6 +197,19 @@ __device__ __forceinline__ void run_span(float *p, const void *g, float *m, floa
         run_tile<N, 1, NEST, GT, LA>(p, g, m, v, slow, acc, idx, s);
 }
 
+// Programmatic dependent launch (PTX griddepcontrol).  launch_dependents lets
+// the next kernel on the stream become resident once every CTA of this grid
+// has started; wait blocks until the previous grid on the stream has completed
+// and its writes are visible.  Both are no-ops in a plain launch.
+__device__ __forceinline__ void grid_dependency_release()
+{
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 template <int NEST, int GT, int LA>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS)
 novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
@@ -206,10 +219,17 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
     constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
 
+    grid_dependency_release();
+    int c = blockIdx.x;
+    if (c >= n_chunks) return;
+    // The work table is written by copies only, never by a kernel, so it may be
+    // read before the previous kernel on the stream has finished.
+    Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
+    TensorRec r = recs[ch.tensor];
+    grid_dependency_wait();
+
 #pragma unroll 1
-    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-        const Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
-        const TensorRec r = recs[ch.tensor];
+    for (;;) {
         float *p = r.p + ch.offset;
         float *m = r.m + ch.offset;
         float *v = r.v + ch.offset;
@@ -234,6 +254,10 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
             // parameter, gradient and state do not share 16-byte alignment
             run_span<1, 4, NEST, GT, LA>(p, g, m, v, slow, acc, ch.len, s);
         }
+        c += gridDim.x;
+        if (c >= n_chunks) break;
+        ch = chunks[reverse ? n_chunks - 1 - c : c];
+        r = recs[ch.tensor];
     }
 }
 
@@ -324,8 +348,17 @@ cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_
 {
     KernelFn fn = pick_kernel(nesterov, grad_dtype, la);
     if (!fn || n_chunks <= 0 || cfg.grid <= 0) return cudaErrorInvalidValue;
-    fn<<<cfg.grid, kBlock, 0, stream>>>(d_chunks, n_chunks, d_recs, s, cfg.reverse);
-    return cudaGetLastError();
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(cfg.grid));
+    lc.blockDim = dim3(kBlock);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = cfg.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, s, cfg.reverse);
 }
 
 }  // namespace novak

@@ -32,10 +32,32 @@ def test_every_declared_symbol_is_exported(lib):
         assert f'"{name}"' in src, f"binding has no signature for {name}"
 
 
-def test_struct_sizes_match_header(lib):
-    # The C structs end on 8-byte boundaries; a drifted field would shift these.
-    assert ctypes.sizeof(B.novak_info) == 5 * 8 + 7 * 8 + 10 * 4
-    assert ctypes.sizeof(B.novak_meta) == 8 + 4 * 8 + 7 * 8 + 8 * 4
+def test_struct_layouts_match_header(lib, tmp_path):
+    """gcc compiles include/novak.h and prints sizeof / offsetof of every field;
+    the ctypes mirrors must agree (a drifted or missing field shifts an offset)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("gcc not found")
+    lines = ["#include <stdio.h>", "#include <stddef.h>", '#include "novak.h"', "int main(void){"]
+    for cls in (B.novak_info, B.novak_meta):
+        name = cls.__name__
+        lines.append(f'printf("{name} %zu\\n", sizeof({name}));')
+        for field, _ in cls._fields_:
+            lines.append(f'printf("{name}.{field} %zu\\n", offsetof({name}, {field}));')
+    lines.append("return 0;}")
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([gcc, "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    got = dict(l.split() for l in subprocess.run([str(exe)], capture_output=True, text=True,
+                                                 check=True).stdout.splitlines())
+    for cls in (B.novak_info, B.novak_meta):
+        name = cls.__name__
+        assert int(got[name]) == ctypes.sizeof(cls)
+        for field, _ in cls._fields_:
+            assert int(got[f"{name}.{field}"]) == getattr(cls, field).offset, field
 
 
 GOOD = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2,

@@ -165,7 +165,8 @@ def test_bit_identical_reruns_and_launch_options():
     numels = [70001, 12, 8192, 30000]
     results = []
     for kw in (dict(), dict(), dict(ctas_per_sm=2), dict(chunk_elems=1024),
-               dict(serpentine=True), dict(ctas_per_sm=1, serpentine=True, chunk_elems=2048)):
+               dict(serpentine=True), dict(ctas_per_sm=1, serpentine=True, chunk_elems=2048),
+               dict(dependent_launch=False), dict(dependent_launch=False, ctas_per_sm=1)):
         _, params, _ = _fresh(numels, seed=4)
         opt = B.NovakOptimizer(params, **BASE, **kw)
         gen = _gen(6)
@@ -244,6 +245,29 @@ def test_gradient_pointers_may_change_every_step():
     for t in range(9):
         pair.step(pool[t % 3])
     pair.check("rotating pool")
+
+
+def test_record_tables_are_reused_and_evicted_least_recently_used_first():
+    """A pointer list seen before costs no upload; the handle keeps 8 lists and
+    replaces the least recently used one.  Results match the oracle either way."""
+    numels = [9000, 100, 2049]
+    _, params, _ = _fresh(numels, seed=43)
+    pair = Pair(params, dict(BASE))
+    gen = _gen(44)
+    pool = [_grads(numels, gen) for _ in range(10)]
+    for t in range(12):                      # lists 0..3 in rotation: 4 uploads
+        pair.step(pool[t % 4])
+    assert pair.opt.info()["record_uploads"] == 4
+    for i in range(4, 10):                   # 6 more lists: 10 > 8, lists 0 and 1 evicted
+        pair.step(pool[i])
+    assert pair.opt.info()["record_uploads"] == 10
+    pair.step(pool[3])                       # still resident
+    pair.step(pool[9])
+    assert pair.opt.info()["record_uploads"] == 10
+    pair.step(pool[0])                       # was evicted: uploaded again
+    assert pair.opt.info()["record_uploads"] == 11
+    pair.check("record tables")
+    assert pair.opt.info()["launches"] == 21
 
 
 def test_error_paths_leave_the_handle_unchanged():
