@@ -39,10 +39,35 @@ METRIC = "parameter updates/sec per novak_step"
 UNIT = "param-updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per element and launch from the ncu captures summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum of the step kernel,
-# averaged over the sync schedule); None until a capture exists for the workload.
-NCU_DRAM_BYTES_PER_ELEM = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the step kernel from the
+# ncu captures summarised under profiles/: bytes of a non-sync and of a sync launch, and
+# the hashes of the kernel sources at capture time.  A capture stops counting (traffic
+# = null) as soon as the kernel sources differ from what was profiled.
+NCU_TRAFFIC = {
+    ("resnet50", "last"): {
+        "plain": 660.13e6, "sync": 868.75e6,
+        "sources": {"novak_kernels.cu": "492306a98c33b577", "novak_internal.h": "01bf4cebf2ed19b2"},
+        "summary": "profiles/novak_step_kernel_resnet50.md",
+    },
+}
+
+
+def ncu_traffic(workload: str, mode: str, sync_fraction: float):
+    """Per-launch DRAM traffic from the committed ncu capture, averaged over the sync
+    schedule of the timed steps, or None when no capture matches the built kernel."""
+    import hashlib
+    rec = NCU_TRAFFIC.get((workload, mode))
+    if rec is None:
+        return None
+    for name, want in rec["sources"].items():
+        path = os.path.join(ROOT, "paper_2601_07876_b200", "csrc", name)
+        try:
+            with open(path, "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest()[:16] != want:
+                    return None
+        except OSError:
+            return None
+    return (1.0 - sync_fraction) * rec["plain"] + sync_fraction * rec["sync"]
 
 
 def parse_args():
@@ -60,6 +85,8 @@ def parse_args():
     ap.add_argument("--dependent-launch", type=int, default=None)
     ap.add_argument("--lib", default=None, help="alternative libnovak.so (tuning builds)")
     ap.add_argument("--e2e-steps", type=int, default=30)
+    ap.add_argument("--host-segment-elems", type=int, default=None,
+                    help="run length of novak_step_host's pipeline (0: no pipelining)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -312,7 +339,8 @@ def main():
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
-    per_elem = NCU_DRAM_BYTES_PER_ELEM.get((wl.name, args.lookahead_mode))
+    n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
+    traffic = ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -347,6 +375,10 @@ def main():
         stream = torch.cuda.current_stream().cuda_stream
         gdt = B.NOVAK_GRAD_BF16 if gbytes == 2 else B.NOVAK_GRAD_F32
 
+        if args.host_segment_elems is not None:
+            opt.handle.set_option(B.NOVAK_OPT_HOST_SEGMENT_ELEMS, args.host_segment_elems)
+        launches_e2e = opt.info()["launches"]
+
         def host_step():
             opt.handle.step_host(hp, hg, opt._params_arr, dg, opt._numel_arr, opt.n, gdt, stream)
 
@@ -367,7 +399,10 @@ def main():
         e2e = {"value": world * wl.total * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": wl.total * gbytes, "d2h_bytes_per_step": wl.total * 4,
                "ms_per_step": ems / args.e2e_steps, "steps": args.e2e_steps,
-               "api": "novak_step_host (pinned host gradients in, parameters out)"}
+               "launches_per_step": (opt.info()["launches"] - launches_e2e) // (args.e2e_steps + 3),
+               "host_segment_elems": int(opt.handle.get_option(B.NOVAK_OPT_HOST_SEGMENT_ELEMS)),
+               "api": "novak_step_host (pinned host gradients in, parameters out; upload, "
+                      "kernel and download pipelined in runs of the chunk table)"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -398,7 +433,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_source": peak_src,
                          "algorithmic_bytes_per_elem": alg,
-                         "traffic": per_elem * wl.total if per_elem else None,
+                         "traffic": traffic,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "per_step": per,
             "e2e": e2e,

@@ -84,12 +84,15 @@ enum {
     NOVAK_OPT_SERPENTINE = 8,     /* 1: walk the chunk table backwards on even steps so
                                      the tail of one step is still in L2 for the next  */
     NOVAK_OPT_WEIGHT_DECAY = 9,   /* lambda >= 0; may change between steps             */
-    NOVAK_OPT_DEPENDENT_LAUNCH = 10 /* 1 (default): launch the step kernel with
+    NOVAK_OPT_DEPENDENT_LAUNCH = 10, /* 1 (default): launch the step kernel with
                                      programmatic stream serialization, so its CTAs
                                      become resident and fetch their work-table
                                      entries while the previous kernel on the stream
                                      drains; they touch no tensor before that kernel
                                      has completed.  0: plain launch               */
+    NOVAK_OPT_HOST_SEGMENT_ELEMS = 11 /* novak_step_host pipelines the step in runs of
+                                     about this many elements (default 4 Mi; at most
+                                     32 runs per step; 0: one run, nothing overlaps)   */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -201,12 +204,19 @@ int novak_step(novak_opt *opt, void *const *d_params,
                int grad_dtype, void *stream);
 
 /* The same step for a caller whose gradients arrive in, and whose updated
- * parameters return to, HOST memory (pinned memory for asynchronous copies):
- * copies h_grads[i] -> d_grads[i], runs novak_step, copies d_params[i] ->
- * h_params[i], all enqueued on `stream` in that order.  Runs of tensors that
- * are adjacent in both host and device memory are merged into one copy.
- * The device tensors remain the master copy; the state stays on the device.
- * Same errors as novak_step. */
+ * parameters return to, HOST memory (pinned memory, or the copies do not
+ * overlap anything).  The chunk table is cut into runs of about
+ * NOVAK_OPT_HOST_SEGMENT_ELEMS elements; for each run the gradients go
+ * h_grads -> d_grads on an upload stream of the handle, the step kernel runs
+ * over that run on `stream` once they have arrived, and the updated
+ * parameters go d_params -> h_params on a download stream, so that upload,
+ * kernel and download of different runs overlap (one kernel launch per run).
+ * Everything is ordered behind the work already on `stream`, and work enqueued
+ * on `stream` afterwards sees all copies finished.  The first call creates the
+ * two streams and their events.  The device tensors remain the master copy;
+ * the state stays on the device.  Ranges adjacent in both host and device
+ * memory are merged into one copy.  Errors as novak_step, except that after
+ * NOVAK_ECUDA part of the step may already have been enqueued. */
 int novak_step_host(novak_opt *opt, void *const *h_params,
                     const void *const *h_grads, void *const *d_params,
                     void *const *d_grads, const int64_t *numel, int n,

@@ -26,7 +26,7 @@ NOVAK_GRAD_F32, NOVAK_GRAD_BF16 = 0, 1
 NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
 (NOVAK_OPT_NESTEROV_BETA, NOVAK_OPT_LOOKAHEAD_MODE, NOVAK_OPT_RECTIFIED, NOVAK_OPT_LR,
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
- NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH) = range(1, 11)
+ NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS) = range(1, 12)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}

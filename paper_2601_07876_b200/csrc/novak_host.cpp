@@ -26,6 +26,8 @@ constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
 constexpr uint64_t kMetaMagic = 0x4e4f56414b763031ull;  // "NOVAKv01"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
+constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
+constexpr int kMaxHostSegments = 32;
 
 struct Hyper {
     double lr, beta1, beta2, eps, wd, beta_n, la_alpha;
@@ -117,6 +119,7 @@ struct novak_opt {
     int ctas_per_sm = kDefaultCtasPerSm;
     int serpentine = 0;
     int pdl = 1;
+    int64_t host_segment_elems = kDefaultHostSegmentElems;
 
     // state layout (fixed by novak_attach_state)
     bool attached = false;
@@ -135,6 +138,7 @@ struct novak_opt {
 
     // device work table
     Chunk *d_chunks = nullptr;
+    std::vector<Chunk> h_chunks;       // host copy of the device chunk table
     int n_chunks = 0;
     TensorRec *d_recs = nullptr;       // kRecTables tables of n records each
     TensorRec *h_recs[kRing] = {nullptr, nullptr, nullptr, nullptr};
@@ -155,6 +159,15 @@ struct novak_opt {
     int64_t table_clock = 0;
     int64_t record_uploads = 0;
     int sms = 0;
+
+    // novak_step_host: the chunk table cut into segments, each with the element
+    // ranges it covers, two copy streams and the events that order them.
+    struct Range { int tensor; int64_t off, len; };
+    struct Segment { int c0, c1; std::vector<Range> ranges; };
+    std::vector<Segment> segments;
+    int64_t segments_for = -1;          // host_segment_elems the segments were cut for
+    cudaStream_t up_stream = nullptr, down_stream = nullptr;
+    std::vector<cudaEvent_t> host_ev;   // [0] start, [1] end, then (uploaded, stepped) per segment
 
     // host copies of the work table for novak_step_noalloc (no device memory of ours)
     std::vector<Chunk> na_chunks;
@@ -236,6 +249,14 @@ void release_device(novak_opt *o)
         o->h_recs[i] = nullptr;
         o->ring_ev[i] = nullptr;
     }
+    for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
+    o->host_ev.clear();
+    if (o->up_stream) cudaStreamDestroy(o->up_stream);
+    if (o->down_stream) cudaStreamDestroy(o->down_stream);
+    o->up_stream = o->down_stream = nullptr;
+    o->segments.clear();
+    o->segments_for = -1;
+    o->h_chunks.clear();
     o->d_chunks = nullptr;
     o->d_recs = nullptr;
     o->n_chunks = 0;
@@ -292,6 +313,7 @@ int prepare_device(novak_opt *o, cudaStream_t stream)
         return fail_cuda(o, e, "chunk table upload");
     }
     o->n_chunks = static_cast<int>(chunks.size());
+    o->h_chunks.swap(chunks);
     return NOVAK_OK;
 }
 
@@ -480,6 +502,11 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "dependent_launch must be 0 or 1");
         o->pdl = static_cast<int>(value);
         return NOVAK_OK;
+    case NOVAK_OPT_HOST_SEGMENT_ELEMS:
+        if (!(value >= 0.0 && value <= 4294967296.0) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "host_segment_elems must be an integer in [0, 2^32]");
+        o->host_segment_elems = static_cast<int64_t>(value);
+        return NOVAK_OK;
     default:
         return fail(o, NOVAK_EINVAL, "unknown option key %d", key);
     }
@@ -502,6 +529,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
     case NOVAK_OPT_DEPENDENT_LAUNCH: *value = o->pdl; break;
+    case NOVAK_OPT_HOST_SEGMENT_ELEMS: *value = static_cast<double>(o->host_segment_elems); break;
     default: return NOVAK_EINVAL;
     }
     return NOVAK_OK;
@@ -562,53 +590,185 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     return NOVAK_OK;
 }
 
+}  // extern "C"
+
+namespace {
+
+StepScalars make_scalars(const Hyper &h, const Plan &p)
+{
+    StepScalars s;
+    s.beta1 = static_cast<float>(h.beta1);
+    s.omb1 = static_cast<float>(1.0 - h.beta1);
+    s.beta2 = static_cast<float>(h.beta2);
+    s.omb2 = static_cast<float>(1.0 - h.beta2);
+    s.beta_n = static_cast<float>(h.beta_n);
+    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
+    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
+    s.eps = static_cast<float>(h.eps);
+    s.decay = static_cast<float>(p.decay);
+    s.step = static_cast<float>(p.step_size);
+    s.la_alpha = static_cast<float>(h.la_alpha);
+    s.k = static_cast<float>(h.la_k > 0 ? h.la_k : 1);
+    return s;
+}
+
+// Everything one step needs, fixed before anything is enqueued.
+struct StepCtx {
+    int64_t t;
+    Plan plan;
+    int la;
+    int grad_dtype;
+    StepScalars s;
+    const TensorRec *d_recs;
+    int reverse;
+};
+
+int check_step_args(novak_opt *o, const char *who, void *const *d_params,
+                    const void *const *d_grads, const int64_t *numel, int n, int grad_dtype)
+{
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "%s: no state attached", who);
+    if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "%s: NULL argument", who);
+    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16)
+        return fail(o, NOVAK_EINVAL, "%s: unknown grad_dtype %d", who, grad_dtype);
+    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
+        return fail(o, NOVAK_ESTATE, "%s: tensor list differs from the attached layout", who);
+    return NOVAK_OK;
+}
+
+// Work table on the device, records for these pointers, the scalar plan of step t+1.
+int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, int grad_dtype,
+               cudaStream_t stream, StepCtx *ctx)
+{
+    int rc;
+    if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
+    if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
+    ctx->t = o->t + 1;
+    ctx->plan = make_plan(o->h, ctx->t);
+    ctx->la = lookahead_action(o->h, ctx->t);
+    ctx->grad_dtype = grad_dtype;
+    ctx->s = make_scalars(o->h, ctx->plan);
+    ctx->d_recs = o->d_recs + static_cast<size_t>(o->cur_table) * o->n;
+    ctx->reverse = (o->serpentine && (ctx->t % 2 == 0)) ? 1 : 0;
+    return NOVAK_OK;
+}
+
+// One launch over chunk-table entries [c0, c1).
+cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaStream_t stream)
+{
+    novak::LaunchCfg cfg;
+    const int count = c1 - c0;
+    cfg.grid = count;
+    if (o->ctas_per_sm > 0) cfg.grid = std::min(count, o->sms * o->ctas_per_sm);
+    cfg.reverse = ctx.reverse;
+    cfg.pdl = o->pdl;
+    o->last_grid = cfg.grid;
+    return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, ctx.s, o->h.nesterov,
+                              ctx.grad_dtype, ctx.la, cfg, stream);
+}
+
+void commit_step(novak_opt *o, const StepCtx &ctx, int launches)
+{
+    o->t = ctx.t;
+    o->launches += launches;
+    o->last_plan = ctx.plan;
+    if (ctx.plan.is_sync) { o->n_syncs += 1; o->last_sync = ctx.t; }
+}
+
+// Cuts the chunk table into runs of about host_segment_elems elements and lists,
+// per run, the element ranges of the tensors it covers.
+void build_segments(novak_opt *o)
+{
+    o->segments.clear();
+    o->segments_for = o->host_segment_elems;
+    const bool in_tensor_order = (o->ctas_per_sm == 0);
+    int64_t want = o->host_segment_elems;
+    if (want <= 0 || !in_tensor_order) want = INT64_MAX;
+    else want = std::max<int64_t>(want, (o->total_numel + kMaxHostSegments - 1) / kMaxHostSegments);
+    novak_opt::Segment seg{0, 0, {}};
+    int64_t have = 0;
+    auto add = [&](const Chunk &c) {
+        if (in_tensor_order && !seg.ranges.empty() && seg.ranges.back().tensor == c.tensor &&
+            seg.ranges.back().off + seg.ranges.back().len == c.offset)
+            seg.ranges.back().len += c.len;
+        else
+            seg.ranges.push_back({c.tensor, c.offset, c.len});
+    };
+    for (int c = 0; c < o->n_chunks; ++c) {
+        add(o->h_chunks[c]);
+        have += o->h_chunks[c].len;
+        seg.c1 = c + 1;
+        if (have >= want && c + 1 < o->n_chunks) {
+            o->segments.push_back(seg);
+            seg = novak_opt::Segment{c + 1, c + 1, {}};
+            have = 0;
+        }
+    }
+    o->segments.push_back(seg);
+}
+
+int prepare_host_pipeline(novak_opt *o)
+{
+    cudaError_t e;
+    if (!o->up_stream &&
+        (e = cudaStreamCreateWithFlags(&o->up_stream, cudaStreamNonBlocking)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaStreamCreate(upload)");
+    if (!o->down_stream &&
+        (e = cudaStreamCreateWithFlags(&o->down_stream, cudaStreamNonBlocking)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaStreamCreate(download)");
+    const size_t need = 2 + 2 * o->segments.size();
+    while (o->host_ev.size() < need) {
+        cudaEvent_t ev;
+        if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess)
+            return fail_cuda(o, e, "cudaEventCreate(host pipeline)");
+        o->host_ev.push_back(ev);
+    }
+    return NOVAK_OK;
+}
+
+// Copies the ranges of one segment between host and device tensors, merging
+// ranges that are adjacent on both sides into one copy.
+cudaError_t copy_ranges(const novak_opt::Segment &seg, void *const *dst, const void *const *src,
+                        size_t elem_bytes, cudaMemcpyKind kind, cudaStream_t stream)
+{
+    size_t i = 0;
+    const size_t n = seg.ranges.size();
+    while (i < n) {
+        const novak_opt::Range &r = seg.ranges[i];
+        char *d = static_cast<char *>(dst[r.tensor]) + r.off * elem_bytes;
+        const char *sr = static_cast<const char *>(src[r.tensor]) + r.off * elem_bytes;
+        size_t bytes = static_cast<size_t>(r.len) * elem_bytes;
+        size_t j = i + 1;
+        while (j < n) {
+            const novak_opt::Range &q = seg.ranges[j];
+            if (static_cast<char *>(dst[q.tensor]) + q.off * elem_bytes != d + bytes ||
+                static_cast<const char *>(src[q.tensor]) + q.off * elem_bytes != sr + bytes)
+                break;
+            bytes += static_cast<size_t>(q.len) * elem_bytes;
+            ++j;
+        }
+        const cudaError_t e = cudaMemcpyAsync(d, sr, bytes, kind, stream);
+        if (e != cudaSuccess) return e;
+        i = j;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
 int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
                const int64_t *numel, int n, int grad_dtype, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
-    if (!o->attached) return fail(o, NOVAK_ESTATE, "step: no state attached");
-    if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step: NULL argument");
-    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16) return fail(o, NOVAK_EINVAL, "step: unknown grad_dtype %d", grad_dtype);
-    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
-        return fail(o, NOVAK_ESTATE, "step: tensor list differs from the attached layout");
+    int rc = check_step_args(o, "step", d_params, d_grads, numel, n, grad_dtype);
+    if (rc != NOVAK_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-
-    int rc;
-    if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
-    if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
-
-    const int64_t t = o->t + 1;
-    const Plan p = make_plan(o->h, t);
-    const int la = lookahead_action(o->h, t);
-    StepScalars s;
-    s.beta1 = static_cast<float>(o->h.beta1);
-    s.omb1 = static_cast<float>(1.0 - o->h.beta1);
-    s.beta2 = static_cast<float>(o->h.beta2);
-    s.omb2 = static_cast<float>(1.0 - o->h.beta2);
-    s.beta_n = static_cast<float>(o->h.beta_n);
-    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
-    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
-    s.eps = static_cast<float>(o->h.eps);
-    s.decay = static_cast<float>(p.decay);
-    s.step = static_cast<float>(p.step_size);
-    s.la_alpha = static_cast<float>(o->h.la_alpha);
-    s.k = static_cast<float>(o->h.la_k > 0 ? o->h.la_k : 1);
-
-    novak::LaunchCfg cfg;
-    cfg.grid = o->n_chunks;
-    if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
-    cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
-    cfg.pdl = o->pdl;
-    const TensorRec *d_recs = o->d_recs + static_cast<size_t>(o->cur_table) * o->n;
-    cudaError_t e = novak::launch_step(o->d_chunks, o->n_chunks, d_recs, s, o->h.nesterov,
-                                       grad_dtype, la, cfg, stream);
+    StepCtx ctx;
+    if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
+    const cudaError_t e = launch_range(o, ctx, 0, o->n_chunks, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
-
-    o->t = t;
-    o->launches += 1;
-    o->last_plan = p;
-    o->last_grid = cfg.grid;
-    if (p.is_sync) { o->n_syncs += 1; o->last_sync = t; }
+    commit_step(o, ctx, 1);
     return NOVAK_OK;
 }
 
@@ -617,50 +777,66 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
                     int grad_dtype, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
-    if (!o->attached) return fail(o, NOVAK_ESTATE, "step_host: no state attached");
-    if (!h_params || !h_grads || !d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step_host: NULL argument");
-    if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16) return fail(o, NOVAK_EINVAL, "step_host: unknown grad_dtype %d", grad_dtype);
-    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
-        return fail(o, NOVAK_ESTATE, "step_host: tensor list differs from the attached layout");
+    if (!h_params || !h_grads) return fail(o, NOVAK_EINVAL, "step_host: NULL argument");
+    int rc = check_step_args(o, "step_host", d_params, const_cast<const void *const *>(d_grads),
+                             numel, n, grad_dtype);
+    if (rc != NOVAK_OK) return rc;
     for (int i = 0; i < n; ++i)
         if (!h_params[i] || !h_grads[i] || !d_params[i] || !d_grads[i])
             return fail(o, NOVAK_EINVAL, "step_host: tensor %d has a NULL pointer", i);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const size_t gsz = grad_dtype == NOVAK_GRAD_BF16 ? 2 : 4;
-    cudaError_t e;
 
-    // gradients host -> device, merging runs adjacent on both sides
-    for (int i = 0; i < n;) {
-        const char *hs = static_cast<const char *>(h_grads[i]);
-        char *ds = static_cast<char *>(d_grads[i]);
-        size_t bytes = static_cast<size_t>(numel[i]) * gsz;
-        int j = i + 1;
-        while (j < n && static_cast<const char *>(h_grads[j]) == hs + bytes &&
-               static_cast<char *>(d_grads[j]) == ds + bytes) {
-            bytes += static_cast<size_t>(numel[j]) * gsz;
-            ++j;
+    StepCtx ctx;
+    if ((rc = begin_step(o, d_params, const_cast<const void *const *>(d_grads), grad_dtype, stream,
+                         &ctx)) != NOVAK_OK)
+        return rc;
+    if (o->segments.empty() || o->segments_for != o->host_segment_elems) build_segments(o);
+    if ((rc = prepare_host_pipeline(o)) != NOVAK_OK) return rc;
+
+    // upload stream: gradients of segment i; caller's stream: kernel over segment
+    // i once they have arrived; download stream: its parameters once the kernel
+    // has run.  Both copy streams start behind the caller's earlier work and the
+    // caller's stream ends behind the last download.
+    const int n_seg = static_cast<int>(o->segments.size());
+    cudaEvent_t ev_start = o->host_ev[0], ev_end = o->host_ev[1];
+    cudaError_t e;
+    const char *what = "host pipeline";
+    int launched = 0;
+    bool forked = false;
+    do {
+        what = "cudaEventRecord(start)";
+        if ((e = cudaEventRecord(ev_start, stream)) != cudaSuccess) break;
+        if ((e = cudaStreamWaitEvent(o->up_stream, ev_start, 0)) != cudaSuccess) break;
+        if ((e = cudaStreamWaitEvent(o->down_stream, ev_start, 0)) != cudaSuccess) break;
+        forked = true;
+        for (int i = 0; i < n_seg && e == cudaSuccess; ++i) {
+            const novak_opt::Segment &seg = o->segments[i];
+            cudaEvent_t ev_up = o->host_ev[2 + 2 * i], ev_step = o->host_ev[3 + 2 * i];
+            what = "gradient upload";
+            if ((e = copy_ranges(seg, d_grads, h_grads, gsz, cudaMemcpyHostToDevice, o->up_stream)) != cudaSuccess) break;
+            if ((e = cudaEventRecord(ev_up, o->up_stream)) != cudaSuccess) break;
+            if ((e = cudaStreamWaitEvent(stream, ev_up, 0)) != cudaSuccess) break;
+            what = "step kernel launch";
+            if ((e = launch_range(o, ctx, seg.c0, seg.c1, stream)) != cudaSuccess) break;
+            ++launched;
+            if ((e = cudaEventRecord(ev_step, stream)) != cudaSuccess) break;
+            if ((e = cudaStreamWaitEvent(o->down_stream, ev_step, 0)) != cudaSuccess) break;
+            what = "parameter download";
+            if ((e = copy_ranges(seg, h_params, const_cast<const void *const *>(d_params), 4,
+                                 cudaMemcpyDeviceToHost, o->down_stream)) != cudaSuccess) break;
         }
-        if ((e = cudaMemcpyAsync(ds, hs, bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-            return fail_cuda(o, e, "gradient upload");
-        i = j;
+    } while (false);
+    if (forked) {
+        // join even after a failure so that the caller's stream stays ordered
+        // behind whatever the copy streams were given
+        cudaError_t j;
+        if ((j = cudaEventRecord(ev_end, o->down_stream)) == cudaSuccess)
+            j = cudaStreamWaitEvent(stream, ev_end, 0);
+        if (e == cudaSuccess && j != cudaSuccess) { e = j; what = "join of the copy streams"; }
     }
-    const int rc = novak_step(o, d_params, const_cast<const void *const *>(d_grads), numel, n, grad_dtype, stream_);
-    if (rc != NOVAK_OK) return rc;
-    // parameters device -> host
-    for (int i = 0; i < n;) {
-        char *hs = static_cast<char *>(h_params[i]);
-        const char *ds = static_cast<const char *>(d_params[i]);
-        size_t bytes = static_cast<size_t>(numel[i]) * 4;
-        int j = i + 1;
-        while (j < n && static_cast<char *>(h_params[j]) == hs + bytes &&
-               static_cast<const char *>(d_params[j]) == ds + bytes) {
-            bytes += static_cast<size_t>(numel[j]) * 4;
-            ++j;
-        }
-        if ((e = cudaMemcpyAsync(hs, ds, bytes, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
-            return fail_cuda(o, e, "parameter download");
-        i = j;
-    }
+    if (launched == n_seg) commit_step(o, ctx, launched);
+    if (e != cudaSuccess) return fail_cuda(o, e, what);
     return NOVAK_OK;
 }
 

@@ -314,32 +314,54 @@ def test_error_paths_leave_the_handle_unchanged():
     assert opt.info()["t"] == 2
 
 
-def test_step_host_matches_step_and_returns_parameters():
-    """novak_step_host = upload gradients, the same step, download parameters."""
-    numels = [6000, 31, 8192]
+@pytest.mark.parametrize("segment_elems,gdtype", [(None, torch.float32), (2048, torch.float32),
+                                                  (4096, torch.bfloat16), (0, torch.float32)])
+def test_step_host_matches_step_and_returns_parameters(segment_elems, gdtype):
+    """novak_step_host = upload gradients, the same step, download parameters, pipelined
+    in runs of the chunk table: bit-identical to novak_step whatever the run length."""
+    numels = [6000, 31, 8192, 20000, 3]
     hyper = dict(BASE, lookahead_k=2)
     _, pa, _ = _fresh(numels, seed=61)
     pflat_b, pb, _ = _fresh(numels, seed=61)
     a = B.NovakOptimizer(pa, **hyper)
     b = B.NovakOptimizer(pb, **hyper)
+    if segment_elems is not None:
+        b.handle.set_option(B.NOVAK_OPT_HOST_SEGMENT_ELEMS, segment_elems)
     gen = _gen(62)
     total = sum(numels)
-    h_g = torch.empty(total, dtype=torch.float32).pin_memory()
+    esz = 2 if gdtype == torch.bfloat16 else 4
+    gdt = B.NOVAK_GRAD_BF16 if gdtype == torch.bfloat16 else B.NOVAK_GRAD_F32
+    h_g = torch.empty(total, dtype=gdtype).pin_memory()
     h_p = torch.empty(total, dtype=torch.float32).pin_memory()
-    d_g = torch.empty(total, dtype=torch.float32, device=DEV)
+    d_g = torch.empty(total, dtype=gdtype, device=DEV)
     offs = np.concatenate([[0], np.cumsum(numels)])[:-1]
-    hg_arr = B.ptr_array([h_g.data_ptr() + 4 * int(o) for o in offs])
+    hg_arr = B.ptr_array([h_g.data_ptr() + esz * int(o) for o in offs])
     hp_arr = B.ptr_array([h_p.data_ptr() + 4 * int(o) for o in offs])
-    dg_arr = B.ptr_array([d_g.data_ptr() + 4 * int(o) for o in offs])
+    dg_arr = B.ptr_array([d_g.data_ptr() + esz * int(o) for o in offs])
     stream = torch.cuda.current_stream().cuda_stream
+    launches = 0
     for _ in range(4):
-        grads = _grads(numels, gen)
+        grads = _grads(numels, gen, dtype=gdtype)
         a.step(grads)
         h_g.copy_(torch.cat([g.reshape(-1) for g in grads]).cpu())
+        h_p.fill_(float("nan"))
+        before = b.info()["launches"]
         b.handle.step_host(hp_arr, hg_arr, b._params_arr, dg_arr, b._numel_arr, len(numels),
-                           B.NOVAK_GRAD_F32, stream)
+                           gdt, stream)
+        # work enqueued on the caller's stream afterwards sees the step finished
+        seen = torch.cat([p.reshape(-1) for p in pb]).clone()
         torch.cuda.synchronize()
-        assert torch.equal(h_p, torch.cat([p.reshape(-1) for p in pa]).cpu())
+        launches = b.info()["launches"] - before
+        expect = torch.cat([p.reshape(-1) for p in pa])
+        assert torch.equal(seen, expect)
+        assert torch.equal(h_p, expect.cpu())
     for x, y in zip(pa, pb):
         assert torch.equal(x, y)
-    assert b.info()["t"] == 4 and b.info()["launches"] == 4
+    for i in range(len(numels)):
+        for key in ("m", "v", "slow"):
+            assert torch.equal(a.state(i)[key], b.state(i)[key])
+    assert b.info()["t"] == 4 and b.info()["n_syncs"] == 2
+    if segment_elems in (None, 0):
+        assert launches == 1
+    else:
+        assert 2 <= launches <= 32
