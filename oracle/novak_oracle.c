@@ -25,6 +25,13 @@
  *     slow += alpha_LA*(mean of the k fast iterates of the window - slow).
  *     Which of the two is "the" method is a reading.          [parity unpinned]
  *   - Moments are not touched by a synchronisation.
+ *   - Phase 2 (gradient processing) runs clipping first, on the norm of the
+ *     raw gradient (Section 7.3: before any other processing), then
+ *     centralization, then the Nesterov approximation.  Table 2 lists
+ *     centralization above clipping; the two steps are linear and commute, so
+ *     the only difference is which norm is compared with c_clip.
+ *     Clipping scales by c_clip/||g|| when ||g|| > c_clip (Table 2's activation
+ *     condition), with no epsilon in the denominator.
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
@@ -142,5 +149,54 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
                 theta[i] = theta_fast;
             }
         }
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * Phase 2, gradient processing (Section 5.1; Table 2; Section 5.8).
+ * ---------------------------------------------------------------------- */
+
+/* Global L2 norm of the gradient: every element of every tensor of the group
+ * (Section 5.8: the threshold applies to the global gradient norm). */
+double novak_oracle_global_norm(int32_t n_tensors, const int64_t *numel,
+                                const double *const *g)
+{
+    double sum = 0.0;
+    for (int32_t k = 0; k < n_tensors; ++k)
+        for (int64_t i = 0; i < numel[k]; ++i)
+            sum += g[k][i] * g[k][i];
+    return sqrt(sum);
+}
+
+/* Gradient clipping (Table 2: active when ||g_t|| > c_clip; norm computation
+ * and scaling): the factor that brings the norm down to c_clip, else 1. */
+double novak_oracle_clip_factor(double norm, double c_clip)
+{
+    if (norm > c_clip)
+        return c_clip / norm;
+    return 1.0;
+}
+
+/* g <- factor * g */
+void novak_oracle_scale(int64_t n, double factor, double *g)
+{
+    for (int64_t i = 0; i < n; ++i)
+        g[i] = factor * g[i];
+}
+
+/* Gradient centralization, Eq. 26, for a tensor of dimension > 1 stored
+ * contiguously as rows x row_len (row = one index of dimension 0, row_len =
+ * the product of dimensions 1..d): subtract from every element the mean over
+ * dimensions 1..d of its row. */
+void novak_oracle_centralize(int64_t rows, int64_t row_len, double *g)
+{
+    for (int64_t r = 0; r < rows; ++r) {
+        double *row = g + r * row_len;
+        double sum = 0.0;
+        for (int64_t j = 0; j < row_len; ++j)
+            sum += row[j];
+        const double mean = sum / (double)row_len;
+        for (int64_t j = 0; j < row_len; ++j)
+            row[j] = row[j] - mean;
     }
 }

@@ -82,6 +82,15 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64,
         dp, dp, dp, dp, dp, dp]
     lib.novak_oracle_step.restype = None
+    lib.novak_oracle_global_norm.argtypes = [
+        ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(dp)]
+    lib.novak_oracle_global_norm.restype = ctypes.c_double
+    lib.novak_oracle_clip_factor.argtypes = [ctypes.c_double, ctypes.c_double]
+    lib.novak_oracle_clip_factor.restype = ctypes.c_double
+    lib.novak_oracle_scale.argtypes = [ctypes.c_int64, ctypes.c_double, dp]
+    lib.novak_oracle_scale.restype = None
+    lib.novak_oracle_centralize.argtypes = [ctypes.c_int64, ctypes.c_int64, dp]
+    lib.novak_oracle_centralize.restype = None
     return lib
 
 
@@ -112,6 +121,8 @@ class Config:
     lookahead_mode: int = LOOKAHEAD_LAST
     rectified: bool = True
     bias1_power: int = 1
+    clip_threshold: float = 0.0          # c_clip; 0 = clipping off
+    centralize: bool = False             # Eq. 26 on tensors given with rows > 0
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -135,8 +146,13 @@ class Oracle:
     ``step(grads)`` advances every tensor by one NOVAK step.
     """
 
-    def __init__(self, cfg: Config, params, lib: ctypes.CDLL | None = None):
+    def __init__(self, cfg: Config, params, lib: ctypes.CDLL | None = None, rows=None):
+        """``rows[i]``: size of dimension 0 of tensor i when it has more than
+        one dimension (it is then centralized when cfg.centralize), else 0."""
         self.cfg = cfg
+        self.rows = list(rows) if rows is not None else None
+        self.grad_norms: list[float] = []
+        self.clip_factors: list[float] = []
         self.h = cfg.to_c()
         self.lib = lib or default_library()
         self.theta = [np.ascontiguousarray(np.asarray(p, dtype=np.float64)).reshape(-1).copy()
@@ -165,6 +181,31 @@ class Oracle:
             _dptr(self.slow[i], lo) if self.slow is not None else null,
             _dptr(self.acc[i], lo) if self.acc is not None else null)
 
+    def process_gradients(self, gs):
+        """Phase 2 before the Nesterov approximation: clipping on the global norm
+        of the raw gradient, then centralization (both in the C file)."""
+        cfg = self.cfg
+        if cfg.clip_threshold <= 0 and not cfg.centralize:
+            return gs
+        gs = [g.copy() for g in gs]
+        if cfg.clip_threshold > 0:
+            n = len(gs)
+            numel = (ctypes.c_int64 * n)(*[g.size for g in gs])
+            ptrs = (ctypes.POINTER(ctypes.c_double) * n)(*[_dptr(g) for g in gs])
+            norm = self.lib.novak_oracle_global_norm(n, numel, ptrs)
+            factor = self.lib.novak_oracle_clip_factor(norm, cfg.clip_threshold)
+            self.grad_norms.append(norm)
+            self.clip_factors.append(factor)
+            for g in gs:
+                self.lib.novak_oracle_scale(g.size, factor, _dptr(g))
+        if cfg.centralize:
+            assert self.rows is not None and len(self.rows) == len(gs)
+            for g, r in zip(gs, self.rows):
+                if r > 0:
+                    assert g.size % r == 0
+                    self.lib.novak_oracle_centralize(r, g.size // r, _dptr(g))
+        return gs
+
     def step(self, grads, threads: int = 1):
         """One step.  ``threads`` > 1 splits each tensor into disjoint element
         ranges handled by separate host threads (elements are independent)."""
@@ -178,6 +219,7 @@ class Oracle:
               for g in grads]
         for i, g in enumerate(gs):
             assert g.size == self.theta[i].size
+        gs = self.process_gradients(gs)
         if threads <= 1:
             for i, g in enumerate(gs):
                 self._run(i, g, 0, g.size)

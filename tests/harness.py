@@ -35,11 +35,18 @@ def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to(torch.float32).cpu().numpy().astype(np.float64)
 
 
+# Worst error seen per quantity since the last reset, as a fraction of the
+# tolerance (printed by the full-size tests so that the margin is on record).
+MARGINS: dict = {}
+
+
 def assert_close(gpu, ref: np.ndarray, what: str):
     got = to_f64(gpu) if isinstance(gpu, torch.Tensor) else np.asarray(gpu, np.float64)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
     err = np.abs(got - ref)
     tol = ATOL + RTOL * np.abs(ref)
+    if err.size:
+        MARGINS[what] = max(MARGINS.get(what, 0.0), float((err / tol).max()))
     bad = err > tol
     if bad.any():
         i = int(np.argmax(err - tol))

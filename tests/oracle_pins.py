@@ -7,8 +7,9 @@ them on the real oracle and ``test_oracle_mutants.py`` on deliberately broken
 copies of it (each planted mistake has to trip at least one pin).
 
 None of the pins re-types the oracle's recurrences: they use closed forms
-(geometric series), explicit unrolled sums, library optimizers
-(torch.optim.AdamW / RAdam in float64) and invariants (Prop. 6.3-6.5).
+(geometric series), explicit unrolled sums, library routines
+(torch.optim.AdamW / RAdam, torch.nn.utils.clip_grad_norm_, tensor.mean, all
+in float64), worked examples and invariants (Prop. 6.3-6.5).
 """
 from __future__ import annotations
 
@@ -421,6 +422,121 @@ def pin_elements_independent(lib):
     assert np.array_equal(np.concatenate(parts.slow), whole.slow[0])
 
 
+# --------------------------------------------------------------------------
+# Phase 2: global-norm clipping (Table 2, Section 5.8) and centralization (Eq. 26)
+# --------------------------------------------------------------------------
+def _prep(lib, grads, rows=None, **kw):
+    o = O.Oracle(O.Config(lookahead_k=0, **kw), [np.zeros(g.size) for g in grads], lib=lib,
+                 rows=rows)
+    out = o.process_gradients([np.asarray(g, np.float64).reshape(-1).copy() for g in grads])
+    return o, out
+
+
+def pin_clip_closed_forms(lib):
+    """3-4-5 and constant-vector norms; a clipped gradient has norm exactly c_clip and
+    keeps its direction; a gradient inside the ball is returned bit for bit."""
+    g = [np.array([3.0, 0.0]), np.array([0.0, -4.0, 0.0])]
+    o, out = _prep(lib, g, clip_threshold=1.0)
+    _close(o.grad_norms[0], 5.0, what="3-4-5 norm")
+    _close(o.clip_factors[0], 0.2, what="3-4-5 factor")
+    _close(np.concatenate(out), [0.6, 0.0, 0.0, -0.8, 0.0], what="3-4-5 clipped")
+    # n equal entries a: ||g|| = |a| sqrt(n), spread over tensors of different sizes
+    a, sizes = -0.37, [7, 1, 92]
+    o, out = _prep(lib, [np.full(n, a) for n in sizes], clip_threshold=0.5)
+    _close(o.grad_norms[0], abs(a) * math.sqrt(sum(sizes)), what="constant-vector norm")
+    flat = np.concatenate(out)
+    _close(math.sqrt(math.fsum(flat * flat)), 0.5, what="norm after clipping")
+    _close(flat, np.full(sum(sizes), -0.5 / math.sqrt(sum(sizes))), what="direction kept")
+    # inside the ball, and exactly on it: untouched
+    rng = np.random.default_rng(3)
+    g = [rng.normal(0, 1e-3, 50), rng.normal(0, 1e-3, 9)]
+    o, out = _prep(lib, g, clip_threshold=1.0)
+    assert o.clip_factors[0] == 1.0
+    assert all(np.array_equal(x, y) for x, y in zip(out, g))
+    o, out = _prep(lib, [np.array([0.6, 0.8])], clip_threshold=1.0)
+    assert o.clip_factors[0] == 1.0 or abs(o.clip_factors[0] - 1.0) < 1e-15
+
+
+def pin_clip_library(lib):
+    """torch.nn.utils.clip_grad_norm_ (whose factor is c/(norm + 1e-6), clamped to 1)
+    on random multi-tensor gradients: norm identical, gradients equal to ~1e-6."""
+    rng = np.random.default_rng(11)
+    shapes = [(5, 3), (17,), (2, 3, 2, 2), (1,)]
+    g = [rng.normal(0, 2.0, s) for s in shapes]
+    ps = [torch.zeros(s, dtype=torch.float64, requires_grad=True) for s in shapes]
+    for p, x in zip(ps, g):
+        p.grad = torch.tensor(x)
+    total = torch.nn.utils.clip_grad_norm_(ps, max_norm=1.5)
+    o, out = _prep(lib, g, clip_threshold=1.5)
+    _close(o.grad_norms[0], float(total), rtol=1e-13, what="norm vs torch")
+    for x, p in zip(out, ps):
+        _close(x, p.grad.numpy().reshape(-1), rtol=2e-6, what="clipped vs torch")
+
+
+def pin_centralize_library_and_invariants(lib):
+    """Eq. 26 against torch's g - g.mean(dim=(1..d)); rows sum to zero; applying it
+    twice changes nothing; tensors given with rows = 0 (one dimension) are untouched;
+    a row of equal entries becomes zero."""
+    rng = np.random.default_rng(5)
+    shapes = [(4, 3, 2, 2), (6, 5), (7,), (3, 1)]
+    g = [rng.normal(0.3, 1.0, s) for s in shapes]
+    rows = [4, 6, 0, 3]
+    _, out = _prep(lib, g, rows=rows, centralize=True)
+    for x, y, s in zip(out, g, shapes):
+        t = torch.tensor(y)
+        if len(s) > 1:
+            want = t - t.mean(dim=tuple(range(1, len(s))), keepdim=True)
+        else:
+            want = t
+        _close(x, want.numpy().reshape(-1), rtol=1e-12, atol=1e-15, what=f"GC {s}")
+        if len(s) > 1:
+            _close(x.reshape(s[0], -1).sum(axis=1), 0.0, atol=1e-14, what="row sums")
+    assert np.array_equal(out[2], g[2].reshape(-1))
+    _close(out[3], 0.0, atol=0.0, what="rows of one element")
+    _, twice = _prep(lib, out, rows=rows, centralize=True)
+    for x, y in zip(twice, out):
+        _close(x, y, atol=1e-15, what="idempotent")
+    # not the mean over dimension 0 (columns) and not the tensor's overall mean
+    gm = np.array([[1.0, 2.0, 6.0], [10.0, 20.0, 30.0]])
+    _, out = _prep(lib, [gm], rows=[2], centralize=True)
+    _close(out[0], [-2.0, -1.0, 3.0, -10.0, 0.0, 10.0], what="worked 2x3 example")
+
+
+def pin_clip_then_centralize_then_step(lib):
+    """Order inside phase 2 and its hand-over to the moments.  The clip factor comes
+    from the RAW norm (a gradient whose centralized norm is below c_clip but whose raw
+    norm is above is still scaled); the processed gradient is what Eq. 1-2 see: one
+    step from m = v = 0 with no Nesterov term gives m_1 = (1-b1) g', v_1 = (1-b2) g'^2."""
+    g = np.array([[10.0, 10.2], [-10.0, -9.8]])          # raw norm ~20, centralized ~0.2
+    b1, b2 = 0.9, 0.99
+    o = O.Oracle(O.Config(beta1=b1, beta2=b2, nesterov_variant=O.NESTEROV_NONE, lookahead_k=0,
+                          clip_threshold=1.0, centralize=True), [np.zeros(4)], lib=lib, rows=[2])
+    o.step([g.reshape(-1)])
+    raw = math.sqrt(10.0 ** 2 + 10.2 ** 2 + 10.0 ** 2 + 9.8 ** 2)
+    gp = (g - g.mean(axis=1, keepdims=True)).reshape(-1) / raw
+    _close(o.grad_norms[0], raw, what="raw norm")
+    _close(o.m[0], (1 - b1) * gp, rtol=1e-10, what="m_1 from processed gradient")
+    _close(o.v[0], (1 - b2) * gp ** 2, rtol=1e-10, what="v_1 from processed gradient")
+    # and with the library: clip + centralize by hand, then torch.optim.AdamW
+    rng = np.random.default_rng(21)
+    th0 = rng.normal(0, 0.1, (3, 4))
+    G = rng.normal(0, 1.0, (6, 3, 4))
+    p = torch.tensor(th0.copy(), requires_grad=True)
+    opt = torch.optim.AdamW([p], lr=1e-2, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.1)
+    o = O.Oracle(O.Config(lr=1e-2, weight_decay=0.1, nesterov_variant=O.NESTEROV_NONE,
+                          lookahead_k=0, rectified=False, clip_threshold=0.7, centralize=True),
+                 [th0], lib=lib, rows=[3])
+    for t in range(6):
+        gt = torch.tensor(G[t])
+        n = float(gt.norm())
+        gt = gt * (0.7 / n if n > 0.7 else 1.0)
+        p.grad = gt - gt.mean(dim=1, keepdim=True)
+        opt.step()
+        o.step([G[t]])
+    # torch's AdamW puts eps before the bias scaling of the root: agree to ~1e-7 relative
+    _close(o.theta[0], p.detach().numpy().reshape(-1), rtol=1e-6, what="AdamW after clip + GC")
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -436,4 +552,8 @@ ALL_PINS = [
     pin_bias1_power,
     pin_moment_bounds,
     pin_elements_independent,
+    pin_clip_closed_forms,
+    pin_clip_library,
+    pin_centralize_library_and_invariants,
+    pin_clip_then_centralize_then_step,
 ]

@@ -5,6 +5,7 @@ elements because the step has no cross-element term."""
 import pytest
 import torch
 
+import harness
 from harness import SampledPair
 from paper_2601_07876_b200 import workloads as W
 
@@ -21,10 +22,13 @@ def test_fullsize_workload(index, mode):
     need = wl.total * 4 * 8
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of device memory")
+    harness.MARGINS.clear()
     pair = SampledPair(wl, DEV, dict(lookahead_mode=mode))
     for _ in range(wl.steps):
         pair.step(threads=8)
     pair.check()
+    print(f"\nPARITY {wl.name} {mode} steps={wl.steps} sampled={pair.idx.numel()} worst |err|/tol: "
+          + ", ".join(f"{k.split()[-1]} {v:.3f}" for k, v in harness.MARGINS.items()))
     k = pair.hyper["lookahead_k"]
     assert pair.sync_steps == list(range(k, wl.steps + 1, k))
     assert pair.rect_flags == [0] * 5 + [1] * (wl.steps - 5)

@@ -45,6 +45,19 @@ MUTANTS = [
     ("traj_acc_not_reset", "acc[i] = 0.0;", ";"),
     ("bias1_power_ignored", "if (h->bias1_power == 2)", "if (0)"),
     ("rectified_flag_ignored", "if (h->rectified && s->rho_t >= 5.0)", "if (s->rho_t >= 5.0)"),
+    # phase 2: clipping and centralization
+    ("norm_not_rooted", "return sqrt(sum);", "return sum;"),
+    ("norm_l1", "sum += g[k][i] * g[k][i];", "sum += fabs(g[k][i]);"),
+    ("norm_first_tensor_only", "for (int32_t k = 0; k < n_tensors; ++k)", "for (int32_t k = 0; k < 1; ++k)"),
+    ("clip_inverted", "return c_clip / norm;", "return norm / c_clip;"),
+    ("clip_always", "if (norm > c_clip)", "if (1)"),
+    ("clip_when_small", "if (norm > c_clip)", "if (norm < c_clip)"),
+    ("scale_dropped", "g[i] = factor * g[i];", "g[i] = g[i];"),
+    ("gc_mean_over_rows", "const double mean = sum / (double)row_len;", "const double mean = sum / (double)rows;"),
+    ("gc_added", "row[j] = row[j] - mean;", "row[j] = row[j] + mean;"),
+    ("gc_sum_of_first_entries", "sum += row[j];", "sum += row[0];"),
+    ("gc_mean_of_previous_row", "row[j] = row[j] - mean;", "row[j] = row[j] - (r ? prev : mean);\n        prev = mean;"),
+    ("gc_first_row_only", "for (int64_t r = 0; r < rows; ++r) {", "for (int64_t r = 0; r < 1; ++r) {"),
 ]
 
 
@@ -53,7 +66,7 @@ def test_mutant_is_caught(name, old, new, tmp_path):
     text = open(SRC).read()
     assert text.count(old) >= 1, f"mutation site for {name} not found in the oracle"
     src = tmp_path / "mutant.c"
-    src.write_text(text.replace(old, new))
+    src.write_text("static double prev;\n" + text.replace(old, new))
     lib = O.load_library(O.compile_oracle(str(src), str(tmp_path / "mutant.so"), force=True))
     caught = []
     for pin in ALL_PINS:
