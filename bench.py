@@ -78,6 +78,10 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="workload index 0..4")
     ap.add_argument("--lookahead-mode", default="last", choices=["last", "traj_mean"])
+    ap.add_argument("--clip", type=float, default=0.0,
+                    help="c_clip of the global-norm clipping (0: off, the headline path)")
+    ap.add_argument("--centralize", action="store_true",
+                    help="gradient centralization on tensors with more than one dimension")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -93,11 +97,13 @@ def parse_args():
     return ap.parse_args()
 
 
-def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int) -> int:
+def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
+                               phase2: bool = False) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
-    arrays on the steps that touch them."""
-    b = 12 + grad_bytes + 12
+    arrays on the steps that touch them, plus one more read of g when clipping or
+    centralization is on (the norm and the row means are needed before the update)."""
+    b = 12 + grad_bytes + 12 + (grad_bytes if phase2 else 0)
     if k <= 0:
         return b
     sync = t % k == 0
@@ -293,7 +299,8 @@ def main():
 
     flat_p = W.alloc_flat(wl, torch.float32, dev)
     W.init_params(wl, flat_p)
-    params = W.views(flat_p, wl)
+    params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
+    phase2 = args.clip > 0 or args.centralize
     pool_n = max(1, min(args.pool, int(8e9 // (wl.total * gbytes)) or 1))
     src = W.GradSource(wl, dev, seed_offset=rank)
     scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
@@ -301,7 +308,8 @@ def main():
     for gf in pool_flat:
         src.fill(gf, scratch)
     del scratch
-    opt = B.NovakOptimizer(params, **hyper, chunk_elems=args.chunk_elems,
+    opt = B.NovakOptimizer(params, **hyper, clip_threshold=args.clip, centralize=args.centralize,
+                           chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
     pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
@@ -334,13 +342,13 @@ def main():
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * wl.total * args.steps / (ms * 1e-3)
-    alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t)
+    alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    traffic = None if phase2 else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -418,6 +426,7 @@ def main():
                 "workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
                 "grad_dtype": "bf16" if gbytes == 2 else "f32",
                 "lookahead_k": k, "lookahead_mode": args.lookahead_mode,
+                "clip_threshold": args.clip, "centralize": bool(args.centralize),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
                       "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),

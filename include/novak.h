@@ -90,9 +90,14 @@ enum {
                                      entries while the previous kernel on the stream
                                      drains; they touch no tensor before that kernel
                                      has completed.  0: plain launch               */
-    NOVAK_OPT_HOST_SEGMENT_ELEMS = 11 /* novak_step_host pipelines the step in runs of
+    NOVAK_OPT_HOST_SEGMENT_ELEMS = 11, /* novak_step_host pipelines the step in runs of
                                      about this many elements (default 4 Mi; at most
                                      32 runs per step; 0: one run, nothing overlaps)   */
+    NOVAK_OPT_CLIP_THRESHOLD = 12, /* c_clip >= 0 of the global-norm gradient clipping
+                                     (Section 5.8; the paper's default is 1.0), 0
+                                     (default here): off.  May change between steps  */
+    NOVAK_OPT_CENTRALIZE = 13     /* 1: gradient centralization (Eq. 26) on the tensors
+                                     that novak_set_tensor_rows gave rows; 0 (default)  */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -125,6 +130,9 @@ typedef struct novak_info {
     int32_t n_chunks;
     int32_t grid, block;    /* launch shape of the last step                       */
     uint32_t warnings;
+    int32_t grad_processing; /* phase 2 as configured: 0 none, 1 clipping,
+                                2 centralization (with or without clipping)        */
+    int32_t reserved;
 } novak_info;
 
 /* Counters and hyperparameters for checkpoint / resume (Table 3: t and the
@@ -138,7 +146,8 @@ typedef struct novak_meta {
     int32_t nesterov_variant, lookahead_k, lookahead_mode, rectified, bias1_power;
     int32_t n_tensors;
     uint32_t warnings;
-    uint32_t reserved;
+    int32_t centralize;
+    double clip_threshold;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
@@ -234,11 +243,14 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
  * no cudaMalloc / cudaFree / cudaHostAlloc / event creation; parameters,
  * gradients and the state buffer are the caller's as in novak_step.
  *
+ * Gradient clipping and centralization need scratch memory that the library
+ * allocates, so this call returns NOVAK_ESTATE while either is switched on.
+ *
  * Limits: at most 4096 tensors and 131072 chunk-table entries (= 268 M
  * elements at the default 2048 elements per entry; raise
  * NOVAK_OPT_CHUNK_ELEMS before the first step for larger groups).  Beyond that
  * the call returns NOVAK_EINVAL with the limit in novak_last_error() and does
- * nothing.  The array costs 2.2 MiB on every GPU that loads the library, until
+ * nothing.  The array costs 2.25 MiB on every GPU that loads the library, until
  * the process exits.
  *
  * The array is ONE per GPU and shared by every handle and every call.  It keeps
@@ -255,6 +267,37 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
 int novak_step_noalloc(novak_opt *opt, void *const *d_params,
                        const void *const *d_grads, const int64_t *numel, int n,
                        int grad_dtype, void *stream);
+
+/* Phase 2, gradient centralization (Eq. 26; Table 2: "use_gc = true, dim > 1").
+ * rows[i] (host array, n entries) is the size of dimension 0 of tensor i when
+ * the tensor has more than one dimension, else 0.  With NOVAK_OPT_CENTRALIZE on,
+ * a tensor with rows[i] > 0 is treated as rows[i] x (numel[i]/rows[i]) and the
+ * mean of each row (all of dimensions 1..d) is subtracted from the row's
+ * gradient before the Nesterov approximation; tensors with rows[i] = 0 are left
+ * as they are.  Call after novak_attach_state; may be called again between steps.
+ * Errors: NOVAK_ESTATE (nothing attached), NOVAK_EINVAL (NULL, n mismatch,
+ * negative rows, numel not a multiple of rows, a tensor with rows of 2^31 or more
+ * elements).
+ *
+ * Phase 2 as a whole (Section 5.1, Table 2, Section 5.8), when clipping or
+ * centralization is on: novak_step first runs a statistics pass (two kernels)
+ * that reads the gradient once and leaves in device memory (a) the global L2
+ * norm of the raw gradient over every tensor of the group and the clip factor
+ * c_clip/||g|| (1 when ||g|| <= c_clip), (b) the row means; the step kernel
+ * then uses g' = factor * (g - row mean).  Clipping acts on the norm of the raw
+ * gradient, before any other processing (Section 7.3).  Three launches per
+ * step, no host synchronisation, no floating-point atomics (results are
+ * bit-identical from run to run); the scratch (24 B per chunk-table entry +
+ * 8 B per row) is allocated by the first such step.  Centralization needs
+ * chunk-table entries of at most 2048 elements (the default).
+ * novak_step_noalloc refuses to run in this mode (NOVAK_ESTATE). */
+int novak_set_tensor_rows(novak_opt *opt, const int64_t *rows, int n);
+
+/* Convergence monitoring (Section 5.8 tracks ||g_t||): the global gradient norm
+ * and the clip factor of the last step that ran phase 2.  Copies 16 bytes from
+ * the device and SYNCHRONISES `stream`.  Either output may be NULL.
+ * NOVAK_ESTATE when no such step has run. */
+int novak_get_grad_stats(novak_opt *opt, double *norm, double *factor, void *stream);
 
 /* Counters and the last step's scalars (bit-exact step and sync indices). */
 int novak_get_info(const novak_opt *opt, novak_info *out);

@@ -26,7 +26,8 @@ NOVAK_GRAD_F32, NOVAK_GRAD_BF16 = 0, 1
 NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
 (NOVAK_OPT_NESTEROV_BETA, NOVAK_OPT_LOOKAHEAD_MODE, NOVAK_OPT_RECTIFIED, NOVAK_OPT_LR,
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
- NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS) = range(1, 12)
+ NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
+ NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE) = range(1, 14)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -41,6 +42,7 @@ class novak_info(Structure):
         ("rect_branch", c_int32), ("is_sync", c_int32), ("nesterov_variant", c_int32),
         ("lookahead_mode", c_int32), ("lookahead_k", c_int32), ("n_tensors", c_int32),
         ("n_chunks", c_int32), ("grid", c_int32), ("block", c_int32), ("warnings", c_uint32),
+        ("grad_processing", c_int32), ("reserved", c_int32),
     ]
 
     def as_dict(self) -> dict:
@@ -55,7 +57,7 @@ class novak_meta(Structure):
         ("weight_decay", c_double), ("nesterov_beta", c_double), ("lookahead_alpha", c_double),
         ("nesterov_variant", c_int32), ("lookahead_k", c_int32), ("lookahead_mode", c_int32),
         ("rectified", c_int32), ("bias1_power", c_int32), ("n_tensors", c_int32),
-        ("warnings", c_uint32), ("reserved", c_uint32),
+        ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
     ]
 
 
@@ -99,6 +101,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_step": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_step_noalloc": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_set_tensor_rows": (c_int, [vp, i64p, c_int]),
+        "novak_get_grad_stats": (c_int, [vp, POINTER(c_double), POINTER(c_double), vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
         "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
         "novak_state_ptrs": (c_int, [vp, c_int, vpp, vpp, vpp, vpp]),
@@ -216,6 +220,19 @@ class Handle:
         if st != NOVAK_OK:
             _check(self.lib, self.h, st, "novak_step_host")
 
+    def set_tensor_rows(self, rows):
+        _check(self.lib, self.h,
+               self.lib.novak_set_tensor_rows(self.h, i64_array(rows), len(rows)),
+               "novak_set_tensor_rows")
+
+    def get_grad_stats(self, stream: int = 0):
+        """(global gradient norm, clip factor) of the last step; synchronises the stream."""
+        norm, factor = c_double(), c_double()
+        _check(self.lib, self.h,
+               self.lib.novak_get_grad_stats(self.h, byref(norm), byref(factor), stream),
+               "novak_get_grad_stats")
+        return norm.value, factor.value
+
     def get_info(self) -> novak_info:
         out = novak_info()
         _check(self.lib, self.h, self.lib.novak_get_info(self.h, byref(out)), "novak_get_info")
@@ -278,6 +295,7 @@ class NovakOptimizer:
     def __init__(self, params, lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
+                 clip_threshold=0.0, centralize=False,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -305,7 +323,9 @@ class NovakOptimizer:
         if serpentine is not None:
             h.set_option(NOVAK_OPT_SERPENTINE, 1 if serpentine else 0)
         if dependent_launch is not None:
-            h.set_option(NOVAK_OPT_DEPENDENT_LAUNCH, 1 if dependent_launch else 0)
+            h.set_option(NOVAK_OPT_DEPENDENT_LAUNCH,
+                         (7 if dependent_launch else 0) if isinstance(dependent_launch, bool)
+                         else int(dependent_launch))
         self.numel = [p.numel() for p in self.params]
         self.n = len(self.params)
         self._numel_arr = i64_array(self.numel)
@@ -319,6 +339,15 @@ class NovakOptimizer:
             h.attach_state(self.state_buffer.data_ptr(), nbytes, self._param_ptrs, self.numel,
                            self._stream())
         self._last_grads = None
+        if clip_threshold:
+            h.set_option(NOVAK_OPT_CLIP_THRESHOLD, clip_threshold)
+        if centralize:
+            # Eq. 26 applies to tensors with more than one dimension
+            h.set_tensor_rows([p.shape[0] if p.dim() > 1 else 0 for p in self.params])
+            h.set_option(NOVAK_OPT_CENTRALIZE, 1)
+
+    def grad_stats(self):
+        return self.handle.get_grad_stats(self._stream())
 
     def _stream(self) -> int:
         import torch

@@ -1,17 +1,24 @@
-"""Builds ``libnovak.so`` (the C-ABI library) in-tree with nvcc for sm_100a."""
+"""Builds ``libnovak.so`` (the C-ABI library) in-tree with nvcc for sm_100a.
+
+Every source is compiled to an object on its own, in parallel, then linked."""
 from __future__ import annotations
 
 import os
 import shutil
 import subprocess
 import sys
+import tempfile
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libnovak.so")
-SOURCES = [os.path.join(CSRC, "novak_host.cpp"), os.path.join(CSRC, "novak_kernels.cu")]
-HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(ROOT, "include", "novak.h")]
+SOURCES = [os.path.join(CSRC, f) for f in (
+    "novak_host.cpp", "novak_launch.cu", "novak_grad_stats.cu",
+    "novak_step_pre0.cu", "novak_step_pre1.cu", "novak_step_pre2.cu")]
+HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(CSRC, "novak_step_kernel.cuh"),
+           os.path.join(ROOT, "include", "novak.h")]
 
 
 def nvcc_path() -> str:
@@ -21,15 +28,20 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found: the NOVAK library cannot be built")
 
 
-def nvcc_command(out: str = LIB, extra: list[str] | None = None) -> list[str]:
+def compile_command(src: str, obj: str, extra: list[str] | None = None) -> list[str]:
     return [
         nvcc_path(), "-O3", "-std=c++17",
         "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-        "-Xcompiler", "-fPIC,-Wall,-Wextra", "-shared",
+        "-Xcompiler", "-fPIC,-Wall,-Wextra",
         "-I", os.path.join(ROOT, "include"), "-I", CSRC,
         *(extra or []),
-        "-o", out, *SOURCES,
+        "-x", "cu", "-c", "-o", obj, src,
     ]
+
+
+def link_command(objs: list[str], out: str) -> list[str]:
+    return [nvcc_path(), "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
+            "-o", out, *objs]
 
 
 def up_to_date(out: str = LIB) -> bool:
@@ -39,21 +51,36 @@ def up_to_date(out: str = LIB) -> bool:
     return all(os.path.getmtime(f) <= t for f in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None) -> str:
+def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None,
+          out: str = LIB) -> str:
     """Compiles the library if a source is newer than the built file."""
-    if not force and not extra and up_to_date():
+    if not force and not extra and out == LIB and up_to_date():
         return LIB
-    tmp = f"{LIB}.{os.getpid()}.tmp"
-    cmd = nvcc_command(tmp, (["-Xptxas", "-v"] if verbose else []) + (extra or []))
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
-        if os.path.exists(tmp):
-            os.remove(tmp)
-        raise RuntimeError("nvcc failed building libnovak.so")
-    os.replace(tmp, LIB)
-    return LIB
+    flags = (["-Xptxas", "-v"] if verbose else []) + (extra or [])
+    with tempfile.TemporaryDirectory(prefix="novak_build_") as tmpdir:
+        objs = [os.path.join(tmpdir, os.path.basename(s) + ".o") for s in SOURCES]
+
+        def one(pair):
+            return subprocess.run(compile_command(pair[0], pair[1], flags),
+                                  capture_output=True, text=True)
+
+        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
+            results = list(pool.map(one, zip(SOURCES, objs)))
+        failed = [r for r in results if r.returncode != 0]
+        if verbose or failed:
+            for r in results:
+                sys.stderr.write(r.stdout + r.stderr)
+        if failed:
+            raise RuntimeError("nvcc failed building libnovak.so")
+        tmp = f"{out}.{os.getpid()}.tmp"
+        res = subprocess.run(link_command(objs, tmp), capture_output=True, text=True)
+        if res.returncode != 0:
+            sys.stderr.write(res.stdout + res.stderr)
+            if os.path.exists(tmp):
+                os.remove(tmp)
+            raise RuntimeError("nvcc failed linking libnovak.so")
+        os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

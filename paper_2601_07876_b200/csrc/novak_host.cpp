@@ -15,6 +15,7 @@
 #include <vector>
 
 using novak::Chunk;
+using novak::PrepOut;
 using novak::StepScalars;
 using novak::TensorRec;
 
@@ -23,7 +24,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763031ull;  // "NOVAKv01"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763032ull;  // "NOVAKv02"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -31,7 +32,9 @@ constexpr int kMaxHostSegments = 32;
 
 struct Hyper {
     double lr, beta1, beta2, eps, wd, beta_n, la_alpha;
+    double clip;            // c_clip of the global-norm clipping, 0: off
     int nesterov, la_k, la_mode, rectified, bias1_power;
+    int centralize;         // Eq. 26 on tensors that were given rows
 };
 
 struct Plan {
@@ -118,7 +121,7 @@ struct novak_opt {
     int64_t chunk_elems = kDefaultChunkElems;
     int ctas_per_sm = kDefaultCtasPerSm;
     int serpentine = 0;
-    int pdl = 1;
+    int pdl = 7;                       // bit 0: step kernel, 1: statistics, 2: its second kernel
     int64_t host_segment_elems = kDefaultHostSegmentElems;
 
     // state layout (fixed by novak_attach_state)
@@ -130,6 +133,8 @@ struct novak_opt {
     int64_t total_numel = 0;
     std::vector<int64_t> numel, slot_off;
     std::vector<int32_t> phase;
+    std::vector<int64_t> rows, row_off;   // dimension 0 of each tensor (0: none), prefix sums
+    int64_t total_rows = 0;
 
     // counters
     int64_t t = 0, n_syncs = 0, last_sync = 0, launches = 0;
@@ -159,6 +164,14 @@ struct novak_opt {
     int64_t table_clock = 0;
     int64_t record_uploads = 0;
     int sms = 0;
+
+    // Scratch of the gradient statistics pass (one allocation): its result, one
+    // sum of squares and two row-piece sums per chunk-table entry, the row means.
+    char *d_prep = nullptr;
+    int64_t prep_rows = -1;             // total_rows the scratch was sized for
+    PrepOut *prep_out = nullptr;
+    double *chunk_sq = nullptr, *seg_first = nullptr, *seg_last = nullptr, *cta_sq = nullptr;
+    float2 *row_mean = nullptr;
 
     // novak_step_host: the chunk table cut into segments, each with the element
     // ranges it covers, two copy streams and the events that order them.
@@ -216,6 +229,13 @@ float *slice(const novak_opt *o, int array, int i)
            o->phase[i];
 }
 
+int pre_mode(const novak_opt *o)
+{
+    if (o->h.centralize && o->total_rows > 0) return novak::PRE_CENTER;
+    if (o->h.clip > 0.0) return novak::PRE_SCALE;
+    return novak::PRE_NONE;
+}
+
 void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
 {
     std::memset(out, 0, sizeof *out);
@@ -237,6 +257,7 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->grid = o->last_grid;
     out->block = novak::step_block_threads();
     out->warnings = o->warnings;
+    out->grad_processing = pre_mode(o);
 }
 
 void release_device(novak_opt *o)
@@ -249,6 +270,12 @@ void release_device(novak_opt *o)
         o->h_recs[i] = nullptr;
         o->ring_ev[i] = nullptr;
     }
+    if (o->d_prep) cudaFree(o->d_prep);
+    o->d_prep = nullptr;
+    o->prep_rows = -1;
+    o->prep_out = nullptr;
+    o->chunk_sq = o->seg_first = o->seg_last = o->cta_sq = nullptr;
+    o->row_mean = nullptr;
     for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
     o->host_ev.clear();
     if (o->up_stream) cudaStreamDestroy(o->up_stream);
@@ -280,12 +307,6 @@ int prepare_device(novak_opt *o, cudaStream_t stream)
 
     std::vector<Chunk> chunks;
     build_chunks(o->numel.data(), o->phase.data(), o->n, o->chunk_elems, chunks);
-    if (o->ctas_per_sm > 0) {
-        // A persistent grid takes chunks round-robin: longest first keeps the
-        // CTAs' totals within one chunk of each other.
-        std::stable_sort(chunks.begin(), chunks.end(),
-                         [](const Chunk &a, const Chunk &b) { return a.len > b.len; });
-    }
     if (chunks.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
 
     const size_t cbytes = chunks.size() * sizeof(Chunk);
@@ -314,6 +335,53 @@ int prepare_device(novak_opt *o, cudaStream_t stream)
     }
     o->n_chunks = static_cast<int>(chunks.size());
     o->h_chunks.swap(chunks);
+    return NOVAK_OK;
+}
+
+// Forget which pointer lists the device record tables hold (their contents
+// depend on the centralization settings as well as on the pointers).
+void invalidate_tables(novak_opt *o)
+{
+    for (auto &tb : o->tables) {
+        tb.p.clear();
+        tb.g.clear();
+        tb.gdtype = -1;
+        tb.last_use = 0;
+    }
+    o->cur_table = -1;
+}
+
+// Scratch of the statistics pass, allocated when a step first needs it.
+int prepare_prep(novak_opt *o, cudaStream_t stream)
+{
+    if (o->d_prep && o->prep_rows == o->total_rows) return NOVAK_OK;
+    cudaError_t e;
+    if (o->d_prep) {
+        cudaFree(o->d_prep);           // waits for the device; sizes changed
+        o->d_prep = nullptr;
+        invalidate_tables(o);
+    }
+    const size_t nc = static_cast<size_t>(o->n_chunks);
+    const size_t off_sq = 256;
+    const size_t off_first = off_sq + nc * sizeof(double);
+    const size_t off_last = off_first + nc * sizeof(double);
+    const size_t off_cta = off_last + nc * sizeof(double);
+    const size_t off_mean = off_cta + static_cast<size_t>(novak::grad_stats_ctas(o->n_chunks)) * sizeof(double);
+    const size_t bytes = off_mean + static_cast<size_t>(o->total_rows) * sizeof(float2) + 16;
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
+        o->d_prep = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(gradient statistics, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    if ((e = cudaMemsetAsync(o->d_prep, 0, bytes, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaMemsetAsync(gradient statistics)");
+    o->prep_out = reinterpret_cast<PrepOut *>(o->d_prep);
+    o->chunk_sq = reinterpret_cast<double *>(o->d_prep + off_sq);
+    o->seg_first = reinterpret_cast<double *>(o->d_prep + off_first);
+    o->seg_last = reinterpret_cast<double *>(o->d_prep + off_last);
+    o->cta_sq = reinterpret_cast<double *>(o->d_prep + off_cta);
+    o->row_mean = reinterpret_cast<float2 *>(o->d_prep + off_mean);
+    o->prep_rows = o->total_rows;
+    invalidate_tables(o);              // records carry pointers into this scratch
     return NOVAK_OK;
 }
 
@@ -375,6 +443,10 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         h[i].v = slice(o, 1, i);
         h[i].slow = la ? slice(o, 2, i) : nullptr;
         h[i].acc = traj ? slice(o, 3, i) : nullptr;
+        const bool rows = o->h.centralize && o->row_mean && !o->rows.empty() && o->rows[i] > 0;
+        h[i].mean = rows ? o->row_mean + o->row_off[i] : nullptr;
+        h[i].row_len = rows ? static_cast<uint32_t>(o->numel[i] / o->rows[i]) : 0u;
+        h[i].reserved = 0;
     }
     // Stream order puts this copy behind every earlier launch that read the
     // table being replaced.
@@ -412,6 +484,8 @@ int check_hyper(const Hyper &h, const char **why)
     if (h.la_k > 0 && !(h.la_alpha > 0.0 && h.la_alpha < 1.0)) { *why = "lookahead_alpha must be in (0,1)"; return 0; }
     if (h.la_mode != NOVAK_LOOKAHEAD_LAST && h.la_mode != NOVAK_LOOKAHEAD_TRAJ_MEAN) { *why = "unknown lookahead mode"; return 0; }
     if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
+    if (!(h.clip >= 0.0) || !std::isfinite(h.clip)) { *why = "clip threshold must be >= 0"; return 0; }
+    if (h.centralize != 0 && h.centralize != 1) { *why = "centralize must be 0 or 1"; return 0; }
     return 1;
 }
 
@@ -433,6 +507,8 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.la_mode = NOVAK_LOOKAHEAD_LAST;
     h.rectified = 1;
     h.bias1_power = 1;
+    h.clip = 0.0;
+    h.centralize = 0;
     uint32_t warn = 0;
     h.nesterov = nesterov_variant;
     if (nesterov_variant == NOVAK_NESTEROV_TRUE) {
@@ -479,6 +555,12 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
         h.bias1_power = static_cast<int>(value);
         break;
+    case NOVAK_OPT_CLIP_THRESHOLD: h.clip = value; break;
+    case NOVAK_OPT_CENTRALIZE:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "centralize must be 0 or 1");
+        if (h.centralize != static_cast<int>(value)) invalidate_tables(o);
+        h.centralize = static_cast<int>(value);
+        break;
     case NOVAK_OPT_CHUNK_ELEMS: {
         if (o->d_chunks || !o->na_chunks.empty())
             return fail(o, NOVAK_ESTATE, "chunk size is fixed once a step was taken");
@@ -499,7 +581,8 @@ int novak_set_option(novak_opt *o, int key, double value)
         o->serpentine = static_cast<int>(value);
         return NOVAK_OK;
     case NOVAK_OPT_DEPENDENT_LAUNCH:
-        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "dependent_launch must be 0 or 1");
+        if (!(value >= 0.0 && value <= 7.0) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "dependent_launch must be an integer in [0, 7]");
         o->pdl = static_cast<int>(value);
         return NOVAK_OK;
     case NOVAK_OPT_HOST_SEGMENT_ELEMS:
@@ -525,6 +608,8 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_LR: *value = o->h.lr; break;
     case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
     case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
+    case NOVAK_OPT_CLIP_THRESHOLD: *value = o->h.clip; break;
+    case NOVAK_OPT_CENTRALIZE: *value = o->h.centralize; break;
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
@@ -584,6 +669,9 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     }
     o->region_elems = off;
     o->total_numel = total;
+    o->rows.assign(n, 0);
+    o->row_off.assign(n, 0);
+    o->total_rows = 0;
     o->t = 0; o->n_syncs = 0; o->last_sync = 0;
     o->attached = true;
     o->err.clear();
@@ -621,6 +709,7 @@ struct StepCtx {
     StepScalars s;
     const TensorRec *d_recs;
     int reverse;
+    int pre;                 // novak::PRE_*
 };
 
 int check_step_args(novak_opt *o, const char *who, void *const *d_params,
@@ -641,6 +730,11 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
 {
     int rc;
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
+    ctx->pre = pre_mode(o);
+    if (ctx->pre == novak::PRE_CENTER && o->chunk_elems > 2048)
+        return fail(o, NOVAK_ESTATE, "centralization needs chunk-table entries of at most 2048 "
+                    "elements (NOVAK_OPT_CHUNK_ELEMS is %lld)", static_cast<long long>(o->chunk_elems));
+    if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
     if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
     ctx->t = o->t + 1;
     ctx->plan = make_plan(o->h, ctx->t);
@@ -649,7 +743,18 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     ctx->s = make_scalars(o->h, ctx->plan);
     ctx->d_recs = o->d_recs + static_cast<size_t>(o->cur_table) * o->n;
     ctx->reverse = (o->serpentine && (ctx->t % 2 == 0)) ? 1 : 0;
+    // After a statistics pass the END of the gradient is what L2 still holds:
+    // the step kernel then walks the table from the end.
+    if (ctx->pre != novak::PRE_NONE) ctx->reverse = 1;
     return NOVAK_OK;
+}
+
+// Phase 2's statistics pass over the whole group: global norm, clip factor, row means.
+cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream)
+{
+    return novak::launch_grad_stats(o->d_chunks, o->n_chunks, ctx.d_recs, ctx.grad_dtype,
+                                    o->h.clip, o->chunk_sq, o->seg_first, o->seg_last,
+                                    o->cta_sq, o->prep_out, ctx.pre == novak::PRE_CENTER, o->pdl, stream);
 }
 
 // One launch over chunk-table entries [c0, c1).
@@ -661,9 +766,10 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     if (o->ctas_per_sm > 0) cfg.grid = std::min(count, o->sms * o->ctas_per_sm);
     cfg.reverse = ctx.reverse;
     cfg.pdl = o->pdl;
+    cfg.pre = ctx.pre;
     o->last_grid = cfg.grid;
-    return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, ctx.s, o->h.nesterov,
-                              ctx.grad_dtype, ctx.la, cfg, stream);
+    return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.s,
+                              o->h.nesterov, ctx.grad_dtype, ctx.la, cfg, stream);
 }
 
 void commit_step(novak_opt *o, const StepCtx &ctx, int launches)
@@ -680,14 +786,13 @@ void build_segments(novak_opt *o)
 {
     o->segments.clear();
     o->segments_for = o->host_segment_elems;
-    const bool in_tensor_order = (o->ctas_per_sm == 0);
     int64_t want = o->host_segment_elems;
-    if (want <= 0 || !in_tensor_order) want = INT64_MAX;
+    if (want <= 0) want = INT64_MAX;
     else want = std::max<int64_t>(want, (o->total_numel + kMaxHostSegments - 1) / kMaxHostSegments);
     novak_opt::Segment seg{0, 0, {}};
     int64_t have = 0;
     auto add = [&](const Chunk &c) {
-        if (in_tensor_order && !seg.ranges.empty() && seg.ranges.back().tensor == c.tensor &&
+        if (!seg.ranges.empty() && seg.ranges.back().tensor == c.tensor &&
             seg.ranges.back().off + seg.ranges.back().len == c.offset)
             seg.ranges.back().len += c.len;
         else
@@ -766,9 +871,16 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     StepCtx ctx;
     if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
-    const cudaError_t e = launch_range(o, ctx, 0, o->n_chunks, stream);
-    if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
-    commit_step(o, ctx, 1);
+    cudaError_t e;
+    int launches = 1;
+    if (ctx.pre != novak::PRE_NONE) {
+        if ((e = launch_stats(o, ctx, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "gradient statistics kernel launch");
+        launches += 2;
+    }
+    if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "step kernel launch");
+    commit_step(o, ctx, launches);
     return NOVAK_OK;
 }
 
@@ -802,7 +914,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
     cudaEvent_t ev_start = o->host_ev[0], ev_end = o->host_ev[1];
     cudaError_t e;
     const char *what = "host pipeline";
-    int launched = 0;
+    int launched = 0, extra_launches = 0;
     bool forked = false;
     do {
         what = "cudaEventRecord(start)";
@@ -810,13 +922,30 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
         if ((e = cudaStreamWaitEvent(o->up_stream, ev_start, 0)) != cudaSuccess) break;
         if ((e = cudaStreamWaitEvent(o->down_stream, ev_start, 0)) != cudaSuccess) break;
         forked = true;
+        const bool stats = ctx.pre != novak::PRE_NONE;
+        if (stats) {
+            // The norm and the row means need the whole gradient: every run is
+            // uploaded before the statistics kernel, and only kernels and
+            // downloads of different runs overlap.
+            what = "gradient upload";
+            for (int i = 0; i < n_seg && e == cudaSuccess; ++i)
+                e = copy_ranges(o->segments[i], d_grads, h_grads, gsz, cudaMemcpyHostToDevice, o->up_stream);
+            if (e != cudaSuccess) break;
+            if ((e = cudaEventRecord(o->host_ev[2], o->up_stream)) != cudaSuccess) break;
+            if ((e = cudaStreamWaitEvent(stream, o->host_ev[2], 0)) != cudaSuccess) break;
+            what = "gradient statistics kernel launch";
+            if ((e = launch_stats(o, ctx, stream)) != cudaSuccess) break;
+            extra_launches += 2;
+        }
         for (int i = 0; i < n_seg && e == cudaSuccess; ++i) {
             const novak_opt::Segment &seg = o->segments[i];
             cudaEvent_t ev_up = o->host_ev[2 + 2 * i], ev_step = o->host_ev[3 + 2 * i];
-            what = "gradient upload";
-            if ((e = copy_ranges(seg, d_grads, h_grads, gsz, cudaMemcpyHostToDevice, o->up_stream)) != cudaSuccess) break;
-            if ((e = cudaEventRecord(ev_up, o->up_stream)) != cudaSuccess) break;
-            if ((e = cudaStreamWaitEvent(stream, ev_up, 0)) != cudaSuccess) break;
+            if (!stats) {
+                what = "gradient upload";
+                if ((e = copy_ranges(seg, d_grads, h_grads, gsz, cudaMemcpyHostToDevice, o->up_stream)) != cudaSuccess) break;
+                if ((e = cudaEventRecord(ev_up, o->up_stream)) != cudaSuccess) break;
+                if ((e = cudaStreamWaitEvent(stream, ev_up, 0)) != cudaSuccess) break;
+            }
             what = "step kernel launch";
             if ((e = launch_range(o, ctx, seg.c0, seg.c1, stream)) != cudaSuccess) break;
             ++launched;
@@ -835,7 +964,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
             j = cudaStreamWaitEvent(stream, ev_end, 0);
         if (e == cudaSuccess && j != cudaSuccess) { e = j; what = "join of the copy streams"; }
     }
-    if (launched == n_seg) commit_step(o, ctx, launched);
+    if (launched == n_seg) commit_step(o, ctx, launched + extra_launches);
     if (e != cudaSuccess) return fail_cuda(o, e, what);
     return NOVAK_OK;
 }
@@ -860,6 +989,9 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
         return fail(o, NOVAK_EINVAL, "step_noalloc: unknown grad_dtype %d", grad_dtype);
     if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
         return fail(o, NOVAK_ESTATE, "step_noalloc: tensor list differs from the attached layout");
+    if (pre_mode(o) != novak::PRE_NONE)
+        return fail(o, NOVAK_ESTATE, "step_noalloc: clipping and centralization keep scratch in "
+                    "allocated device memory; use novak_step, or switch them off");
     if (n > novak::kNoAllocMaxTensors)
         return fail(o, NOVAK_EINVAL, "step_noalloc: %d tensors exceed the static table's %d; "
                     "split the group or use novak_step", n, novak::kNoAllocMaxTensors);
@@ -899,6 +1031,9 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
             r.v = slice(o, 1, i);
             r.slow = la ? slice(o, 2, i) : nullptr;
             r.acc = traj ? slice(o, 3, i) : nullptr;
+            r.mean = nullptr;
+            r.row_len = 0;
+            r.reserved = 0;
         }
         o->na_p.assign(d_params, d_params + n);
         o->na_g.assign(d_grads, d_grads + n);
@@ -952,8 +1087,9 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     cfg.grid = n_chunks;
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
-    e = novak::launch_step(d_chunks, n_chunks, d_recs, s, o->h.nesterov, grad_dtype, la_action,
-                           cfg, stream);
+    cfg.pre = novak::PRE_NONE;
+    e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, s, o->h.nesterov, grad_dtype,
+                           la_action, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
 
     o->t = t;
@@ -961,6 +1097,45 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     o->last_plan = p;
     o->last_grid = cfg.grid;
     if (p.is_sync) { o->n_syncs += 1; o->last_sync = t; }
+    return NOVAK_OK;
+}
+
+int novak_set_tensor_rows(novak_opt *o, const int64_t *rows, int n)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "set_tensor_rows: attach the state first");
+    if (!rows || n != o->n) return fail(o, NOVAK_EINVAL, "set_tensor_rows: NULL or wrong tensor count");
+    int64_t total = 0;
+    for (int i = 0; i < n; ++i) {
+        if (rows[i] < 0) return fail(o, NOVAK_EINVAL, "set_tensor_rows: tensor %d has negative rows", i);
+        if (rows[i] == 0) continue;
+        if (o->numel[i] % rows[i] != 0)
+            return fail(o, NOVAK_EINVAL, "set_tensor_rows: tensor %d: %lld elements are not a multiple of %lld rows",
+                        i, static_cast<long long>(o->numel[i]), static_cast<long long>(rows[i]));
+        if (o->numel[i] >= (int64_t(1) << 31))
+            return fail(o, NOVAK_EINVAL, "set_tensor_rows: tensor %d has 2^31 or more elements", i);
+        total += rows[i];
+    }
+    o->rows.assign(rows, rows + n);
+    int64_t off = 0;
+    for (int i = 0; i < n; ++i) { o->row_off[i] = off; off += o->rows[i]; }
+    o->total_rows = total;
+    invalidate_tables(o);
+    return NOVAK_OK;
+}
+
+int novak_get_grad_stats(novak_opt *o, double *norm, double *factor, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->prep_out) return fail(o, NOVAK_ESTATE, "get_grad_stats: no step with clipping or centralization yet");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    PrepOut h;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(&h, o->prep_out, sizeof h, cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "get_grad_stats");
+    if (norm) *norm = h.norm;
+    if (factor) *factor = static_cast<double>(h.factor);
     return NOVAK_OK;
 }
 
@@ -1002,6 +1177,8 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->nesterov_variant = o->h.nesterov; out->lookahead_k = o->h.la_k;
     out->lookahead_mode = o->h.la_mode; out->rectified = o->h.rectified;
     out->bias1_power = o->h.bias1_power;
+    out->clip_threshold = o->h.clip;
+    out->centralize = o->h.centralize;
     out->n_tensors = o->n;
     out->warnings = o->warnings;
     return NOVAK_OK;
@@ -1021,6 +1198,9 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.wd = in->weight_decay; h.beta_n = in->nesterov_beta; h.la_alpha = in->lookahead_alpha;
     h.nesterov = in->nesterov_variant; h.rectified = in->rectified;
     h.bias1_power = in->bias1_power;
+    h.clip = in->clip_threshold;
+    if (h.centralize != in->centralize) invalidate_tables(o);
+    h.centralize = in->centralize;
     const char *why;
     if (!check_hyper(h, &why)) return fail(o, NOVAK_EINVAL, "import: %s", why);
     o->h = h;

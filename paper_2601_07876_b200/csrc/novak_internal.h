@@ -1,5 +1,5 @@
 // Internal types shared by the host planner (novak_host.cpp) and the device
-// code (novak_kernels.cu) of the NOVAK step library.  Not part of the C ABI.
+// code (novak_*.cu) of the NOVAK step library.  Not part of the C ABI.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -8,13 +8,16 @@
 namespace novak {
 
 // Per-tensor record in device memory: where the tensor's streams start.
-struct TensorRec {
-    float *p;        // parameters theta, fp32, updated in place
-    const void *g;   // gradient, fp32 or bf16, read only
-    float *m;        // first moment   (Eq. 1)
-    float *v;        // second moment  (Eq. 2)
-    float *slow;     // slow weights   (Eq. 28), NULL when lookahead is off
-    float *acc;      // running sum of the window's fast iterates (TRAJ_MEAN)
+struct __align__(16) TensorRec {
+    float *p;          // parameters theta, fp32, updated in place
+    const void *g;     // gradient, fp32 or bf16, read only
+    float *m;          // first moment   (Eq. 1)
+    float *v;          // second moment  (Eq. 2)
+    float *slow;       // slow weights   (Eq. 28), NULL when lookahead is off
+    float *acc;        // running sum of the window's fast iterates (TRAJ_MEAN)
+    float2 *mean;      // row means of the raw gradient (Eq. 26) as hi + lo, NULL: not centralized
+    uint32_t row_len;  // elements per row (product of dimensions 1..d), 0: not centralized
+    uint32_t reserved;
 };
 
 // One unit of work: `len` consecutive elements of one tensor.
@@ -50,23 +53,52 @@ enum : int {
     LA_TRAJ = 64     // target = running sum / k (else theta_fast)
 };
 
+// Gradient processing before the Nesterov approximation (phase 2; template
+// parameter of the step kernel).
+enum : int {
+    PRE_NONE = 0,    // g as given
+    PRE_SCALE = 1,   // g <- factor g, the clip factor read from device memory
+    PRE_CENTER = 2   // g <- factor (g - row mean) for tensors that have rows (Eq. 26)
+};
+
+// Result of the gradient statistics pass, in device memory; the step kernel
+// reads `factor` from here, so the host never waits for it.
+struct __align__(16) PrepOut {
+    double norm;       // global L2 norm of the raw gradient
+    float factor;      // clip factor: c_clip/norm when norm > c_clip, else 1
+    unsigned ticket;   // CTAs of the statistics kernel that have finished
+};
+
 struct LaunchCfg {
     int grid;
     int reverse;     // walk the chunk table from the end
-    int pdl;         // launch with programmatic stream serialization
+    int pdl;         // launch with programmatic stream serialization (bit 0)
+    int pre;         // PRE_*
 };
 
 // Threads per CTA of the step kernel (fixed at compile time).
 int step_block_threads();
 
 // Resident CTAs per SM of the step kernel instantiation for these modes.
-cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int *ctas_per_sm);
+cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int pre, int *ctas_per_sm);
 
 // Launches the fused step kernel.  Returns cudaErrorInvalidValue for a mode
-// combination that has no instantiation.
+// combination that has no instantiation.  `prep` may be NULL when cfg.pre is
+// PRE_NONE.
 cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                        const StepScalars &s, int nesterov, int grad_dtype, int la,
-                        const LaunchCfg &cfg, cudaStream_t stream);
+                        const PrepOut *prep, const StepScalars &s, int nesterov,
+                        int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream);
+
+// Launches the gradient statistics pass over the whole chunk table (two
+// kernels): the global norm of the raw gradient and the clip factor into *prep,
+// and, where a tensor record has rows, the row means of Eq. 26.  Scratch:
+// chunk_sq, seg_first, seg_last of n_chunks doubles each (seg_* may be NULL
+// when no tensor has rows) and cta_sq of grad_stats_ctas(n_chunks) doubles.
+int grad_stats_ctas(int n_chunks);
+cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
+                              int grad_dtype, double c_clip, double *chunk_sq,
+                              double *seg_first, double *seg_last, double *cta_sq,
+                              PrepOut *prep, bool any_rows, int pdl, cudaStream_t stream);
 
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.

@@ -1,18 +1,21 @@
-// Fused multi-tensor NOVAK step kernel for sm_100a.
+// Fused multi-tensor NOVAK step kernel for sm_100a (template; instantiated by
+// novak_step_pre*.cu, one translation unit per gradient pre-processing mode).
 //
-// One launch covers every tensor of a parameter group.  A CTA walks the chunk
-// table (grid-stride); for each chunk it reads theta, g, m, v (and the
-// lookahead arrays on the steps that need them) exactly once with 128-bit
-// coalesced accesses, does the paper's phases 2 and 4-10 in registers (fp32,
-// IEEE sqrt and division, no fast-math) and writes theta, m, v (and the
-// lookahead arrays) exactly once.  There is no shared memory, no atomic, no
-// barrier and no wait of any kind, so a launch does a bounded amount of work
-// per CTA and cannot hang.
+// One launch covers every tensor of a parameter group.  A CTA takes entries of
+// the chunk table; for each it reads theta, g, m, v (and the lookahead arrays
+// on the steps that need them) exactly once with 128-bit coalesced accesses,
+// does the paper's phases 2 and 4-10 in registers (fp32, IEEE sqrt and
+// division, no fast-math) and writes theta, m, v (and the lookahead arrays)
+// exactly once.  There is no shared memory, no atomic, no barrier and no spin
+// of any kind, so a launch does a bounded amount of work per CTA and cannot
+// hang.
 //
 // The step is HBM bound: 28 B per element against ~45 fp32 instructions, so
 // the design goal is bytes in flight per SM, not arithmetic: each thread
 // issues NOVAK_UNROLL independent 16-byte loads per stream before the first
 // use.
+#pragma once
+
 #include "novak_internal.h"
 
 #include "novak.h"
@@ -97,6 +100,46 @@ __device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
     }
 }
 
+// ---- phase 2 before the Nesterov approximation: clip factor and centralization
+struct PreArgs {
+    float factor;        // clip factor (1 when clipping is off or inactive)
+    const float2 *mean;  // row means of the raw gradient (hi + lo), NULL: tensor not centralized
+    uint32_t row_len;
+    uint32_t elem0;      // index within the tensor of the span's first element
+};
+
+// g <- factor (g - mean of its row), Eq. 26 with the clip factor applied after
+// the (linear) centring.  `e` is the tensor index of G's first element.  A
+// vector usually lies inside one row; the row mean is re-read only where it
+// crosses into the next one.  The mean comes as hi + lo: where g and the mean
+// nearly cancel, g - hi is exact and lo supplies the mean's remaining bits, so
+// the centred gradient carries a relative rounding error only.
+template <int N, int PRE>
+__device__ __forceinline__ void preprocess(Vec<N> &G, uint32_t e, const PreArgs &a)
+{
+    if constexpr (PRE == PRE_CENTER) {
+        if (a.mean != nullptr) {
+            uint32_t row = e / a.row_len;
+            uint32_t rem = e - row * a.row_len;
+            float2 mu = __ldg(a.mean + row);
+#pragma unroll
+            for (int j = 0; j < N; ++j) {
+                if (rem == a.row_len) {     // stepped over the end of the row
+                    rem = 0;
+                    ++row;
+                    mu = __ldg(a.mean + row);
+                }
+                G.a[j] = (G.a[j] - mu.x) - mu.y;
+                ++rem;
+            }
+        }
+    }
+    if constexpr (PRE != PRE_NONE) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) G.a[j] *= a.factor;
+    }
+}
+
 // ---- the per-element update, phases 2 and 4-10 (Section 5.1)
 template <int NEST, int LA>
 __device__ __forceinline__ void update_element(float &p, float g, float &m, float &v,
@@ -145,10 +188,10 @@ __device__ __forceinline__ void update_element(float &p, float g, float &m, floa
 
 // One full tile: U vectors per thread and per stream, every load issued
 // before the first use so that U x (4..6) 16-byte requests are in flight.
-template <int N, int U, int NEST, int GT, int LA>
+template <int N, int U, int NEST, int GT, int LA, int PRE>
 __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, float *v,
                                          float *slow, float *acc, int first,
-                                         const StepScalars &s)
+                                         const StepScalars &s, const PreArgs &pre)
 {
     constexpr bool kReadS = (LA & LA_S_READ) != 0;
     constexpr bool kWriteS = (LA & LA_S_WRITE) != 0;
@@ -168,6 +211,7 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const int idx = first + j * kBlock;
+        preprocess<N, PRE>(G[j], pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
 #pragma unroll
         for (int e = 0; e < N; ++e)
             update_element<NEST, LA>(P[j].a[e], G[j].a[e], M[j].a[e], V[j].a[e],
@@ -182,19 +226,19 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
 
 // nvec vectors of N elements: full tiles of U vectors per thread, then the
 // remainder one vector per thread at a time.
-template <int N, int U, int NEST, int GT, int LA>
+template <int N, int U, int NEST, int GT, int LA, int PRE>
 __device__ __forceinline__ void run_span(float *p, const void *g, float *m, float *v,
                                          float *slow, float *acc, int nvec,
-                                         const StepScalars &s)
+                                         const StepScalars &s, const PreArgs &pre)
 {
     constexpr int kTile = kBlock * U;
     int base = 0;
 #pragma unroll 1
     for (; base + kTile <= nvec; base += kTile)
-        run_tile<N, U, NEST, GT, LA>(p, g, m, v, slow, acc, base + threadIdx.x, s);
+        run_tile<N, U, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, base + threadIdx.x, s, pre);
 #pragma unroll 1
     for (int idx = base + threadIdx.x; idx < nvec; idx += kBlock)
-        run_tile<N, 1, NEST, GT, LA>(p, g, m, v, slow, acc, idx, s);
+        run_tile<N, 1, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, idx, s, pre);
 }
 
 // Programmatic dependent launch (PTX griddepcontrol).  launch_dependents lets
@@ -210,10 +254,11 @@ __device__ __forceinline__ void grid_dependency_wait()
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-template <int NEST, int GT, int LA>
+template <int NEST, int GT, int LA, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS)
 novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                  const TensorRec *__restrict__ recs, const StepScalars s, int reverse)
+                  const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
+                  const StepScalars s, int reverse)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
@@ -228,8 +273,16 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     TensorRec r = recs[ch.tensor];
     grid_dependency_wait();
 
+    // The clip factor is the statistics kernel's output: read it only now.
+    PreArgs pre;
+    pre.factor = 1.0f;
+    if constexpr (PRE != PRE_NONE) pre.factor = prep->factor;
+
 #pragma unroll 1
     for (;;) {
+        pre.mean = (PRE == PRE_CENTER) ? r.mean : nullptr;
+        pre.row_len = r.row_len;
+        pre.elem0 = static_cast<uint32_t>(ch.offset);
         float *p = r.p + ch.offset;
         float *m = r.m + ch.offset;
         float *v = r.v + ch.offset;
@@ -245,14 +298,14 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                              (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
         if (aligned) {
             const int nvec = ch.len >> 2;
-            run_span<4, kUnroll, NEST, GT, LA>(p, g, m, v, slow, acc, nvec, s);
+            run_span<4, kUnroll, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, nvec, s, pre);
             // ragged tail of a tensor: at most 3 elements
             const int idx = (nvec << 2) + threadIdx.x;
             if (idx < ch.len)
-                run_tile<1, 1, NEST, GT, LA>(p, g, m, v, slow, acc, idx, s);
+                run_tile<1, 1, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, idx, s, pre);
         } else {
             // parameter, gradient and state do not share 16-byte alignment
-            run_span<1, 4, NEST, GT, LA>(p, g, m, v, slow, acc, ch.len, s);
+            run_span<1, 4, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, ch.len, s, pre);
         }
         c += gridDim.x;
         if (c >= n_chunks) break;
@@ -261,13 +314,14 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
 }
 
-using KernelFn = void (*)(const Chunk *, int, const TensorRec *, StepScalars, int);
+using StepKernelFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *,
+                              StepScalars, int);
 
-template <int NEST, int GT>
-KernelFn pick_la(int la)
+template <int NEST, int GT, int PRE>
+StepKernelFn pick_la(int la)
 {
     switch (la) {
-#define NOVAK_LA_CASE(X) case (X): return novak_step_kernel<NEST, GT, (X)>;
+#define NOVAK_LA_CASE(X) case (X): return novak_step_kernel<NEST, GT, (X), PRE>;
         NOVAK_LA_CASE(LA_NONE)
         NOVAK_LA_CASE(LA_S_INIT | LA_S_WRITE)
         NOVAK_LA_CASE(LA_S_INIT | LA_S_WRITE | LA_SYNC)
@@ -281,84 +335,28 @@ KernelFn pick_la(int la)
     }
 }
 
-template <int NEST>
-KernelFn pick_gt(int grad_dtype, int la)
+template <int NEST, int PRE>
+StepKernelFn pick_gt(int grad_dtype, int la)
 {
     switch (grad_dtype) {
-    case NOVAK_GRAD_F32: return pick_la<NEST, NOVAK_GRAD_F32>(la);
-    case NOVAK_GRAD_BF16: return pick_la<NEST, NOVAK_GRAD_BF16>(la);
+    case NOVAK_GRAD_F32: return pick_la<NEST, NOVAK_GRAD_F32, PRE>(la);
+    case NOVAK_GRAD_BF16: return pick_la<NEST, NOVAK_GRAD_BF16, PRE>(la);
     default: return nullptr;
     }
 }
 
-KernelFn pick_kernel(int nesterov, int grad_dtype, int la)
+// Every instantiation for one pre-processing mode (3 variants x 2 gradient
+// types x 8 lookahead actions).
+template <int PRE>
+StepKernelFn pick_step_kernel(int nesterov, int grad_dtype, int la)
 {
     switch (nesterov) {
-    case NOVAK_NESTEROV_NONE: return pick_gt<NOVAK_NESTEROV_NONE>(grad_dtype, la);
-    case NOVAK_NESTEROV_APPROX: return pick_gt<NOVAK_NESTEROV_APPROX>(grad_dtype, la);
-    case NOVAK_NESTEROV_CLASSICAL: return pick_gt<NOVAK_NESTEROV_CLASSICAL>(grad_dtype, la);
+    case NOVAK_NESTEROV_NONE: return pick_gt<NOVAK_NESTEROV_NONE, PRE>(grad_dtype, la);
+    case NOVAK_NESTEROV_APPROX: return pick_gt<NOVAK_NESTEROV_APPROX, PRE>(grad_dtype, la);
+    case NOVAK_NESTEROV_CLASSICAL: return pick_gt<NOVAK_NESTEROV_CLASSICAL, PRE>(grad_dtype, la);
     default: return nullptr;
     }
 }
 
 }  // namespace
-
-// Work table of novak_step_noalloc: tensor records followed by the chunk table,
-// resident in every GPU that loads this library until the process exits
-// (192 KiB + 2 MiB).  In host code this name is only a handle for
-// cudaGetSymbolAddress, never a device address.
-struct NoAllocTable {
-    TensorRec recs[kNoAllocMaxTensors];
-    Chunk chunks[kNoAllocMaxChunks];
-};
-static __device__ __align__(256) unsigned char g_noalloc_table[sizeof(NoAllocTable)];
-
-cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks)
-{
-    constexpr int kMaxDevices = 64;
-    static void *resolved[kMaxDevices] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!resolved[dev]) {
-        void *ptr = nullptr;
-        e = cudaGetSymbolAddress(&ptr, g_noalloc_table);  // address on the current device
-        if (e != cudaSuccess) return e;
-        resolved[dev] = ptr;
-    }
-    NoAllocTable *t = static_cast<NoAllocTable *>(resolved[dev]);
-    *d_recs = t->recs;
-    *d_chunks = t->chunks;
-    return cudaSuccess;
-}
-
-int step_block_threads() { return kBlock; }
-
-cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int *ctas_per_sm)
-{
-    KernelFn fn = pick_kernel(nesterov, grad_dtype, la);
-    if (!fn) return cudaErrorInvalidValue;
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, fn, kBlock, 0);
-}
-
-cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                        const StepScalars &s, int nesterov, int grad_dtype, int la,
-                        const LaunchCfg &cfg, cudaStream_t stream)
-{
-    KernelFn fn = pick_kernel(nesterov, grad_dtype, la);
-    if (!fn || n_chunks <= 0 || cfg.grid <= 0) return cudaErrorInvalidValue;
-    cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(static_cast<unsigned>(cfg.grid));
-    lc.blockDim = dim3(kBlock);
-    lc.dynamicSmemBytes = 0;
-    lc.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = cfg.pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, s, cfg.reverse);
-}
-
 }  // namespace novak

@@ -28,7 +28,14 @@ def oracle_config(hyper: dict) -> O.Config:
         lookahead_k=h.pop("lookahead_k", 5), lookahead_alpha=h.pop("lookahead_alpha", 0.5),
         nesterov_beta=h.pop("nesterov_beta", None),
         lookahead_mode=_MODE[h.pop("lookahead_mode", "last")],
-        rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1))
+        rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1),
+        clip_threshold=h.pop("clip_threshold", 0.0), centralize=h.pop("centralize", False))
+
+
+def tensor_rows(tensors):
+    """Dimension 0 of every tensor with more than one dimension, else 0 (Eq. 26
+    applies to tensors of dimension > 1)."""
+    return [int(t.shape[0]) if t.dim() > 1 else 0 for t in tensors]
 
 
 def to_f64(t: torch.Tensor) -> np.ndarray:
@@ -42,6 +49,7 @@ MARGINS: dict = {}
 
 def assert_close(gpu, ref: np.ndarray, what: str):
     got = to_f64(gpu) if isinstance(gpu, torch.Tensor) else np.asarray(gpu, np.float64)
+    got, ref = got.reshape(-1), np.asarray(ref).reshape(-1)
     assert got.shape == ref.shape, (what, got.shape, ref.shape)
     err = np.abs(got - ref)
     tol = ATOL + RTOL * np.abs(ref)
@@ -62,10 +70,18 @@ class Pair:
     def __init__(self, params, hyper: dict, opt_kwargs: dict | None = None, lib=None):
         self.params = params
         self.hyper = hyper
-        self.oracle = O.Oracle(oracle_config(hyper), [to_f64(p) for p in params])
+        self.oracle = O.Oracle(oracle_config(hyper), [to_f64(p) for p in params],
+                               rows=tensor_rows(params))
         self.opt = B.NovakOptimizer(params, **hyper, **(opt_kwargs or {}), lib=lib)
         self.sync_steps = []
         self.rect_flags = []
+        self.grad_norms, self.clip_factors = [], []
+
+    def record_grad_stats(self):
+        """Reads the step's gradient norm and clip factor back (synchronises)."""
+        norm, factor = self.opt.grad_stats()
+        self.grad_norms.append(norm)
+        self.clip_factors.append(factor)
 
     def step(self, grads, threads=1):
         self.opt.step(grads)
@@ -83,6 +99,11 @@ class Pair:
         assert info["n_syncs"] == len(o.sync_steps)
         assert info["last_sync_step"] == (o.sync_steps[-1] if o.sync_steps else 0)
         assert self.rect_flags == o.rect_flags
+        if self.grad_norms:
+            # four squares at a time are added in fp32, the rest in double; the factor
+            # is rounded to fp32
+            np.testing.assert_allclose(self.grad_norms, o.grad_norms, rtol=1e-7)
+            np.testing.assert_allclose(self.clip_factors, o.clip_factors, rtol=1e-6)
         for i, p in enumerate(self.params):
             st = self.opt.state(i)
             assert_close(p, o.theta[i], f"{what} theta[{i}]")

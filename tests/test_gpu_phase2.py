@@ -1,0 +1,211 @@
+"""Phase 2 on the GPU (global-norm clipping, gradient centralization) against
+the CPU oracle, element by element, through the C ABI.  Same tolerance as the
+other parity tests; the gradient norm itself to 1e-7."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import harness
+from harness import Pair, make_tensors, to_f64
+from paper_2601_07876_b200 import binding as B
+from paper_2601_07876_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+BASE = dict(lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
+            nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5)
+
+# rows shorter, equal to and longer than a chunk-table entry (2048 elements), odd row
+# lengths (rows cross 128-bit vectors and entry boundaries), rows of 1 and 2 elements,
+# a single row, one-dimensional tensors in between, and some misaligned starts
+SHAPES = [(8, 3, 3, 3), (33,), (10, 257), (3, 5000), (4097, 2), (1, 7), (5, 1), (2048,),
+          (6, 2048), (7, 1000, 3), (2, 3, 4100)]
+OFFSETS = [0, 1, 0, 3, 0, 2, 0, 0, 0, 0, 1]
+
+
+def _gen(seed):
+    return torch.Generator(device=DEV).manual_seed(seed)
+
+
+def _shaped(shapes, offsets, dtype=torch.float32):
+    numels = [math.prod(s) for s in shapes]
+    flat, views, _ = make_tensors(numels, DEV, offsets, dtype=dtype)
+    return flat, [v.view(s) for v, s in zip(views, shapes)]
+
+
+def _fill_grads(grads, gen, std, mean=0.0):
+    for g in grads:
+        g.copy_(torch.empty(g.shape, dtype=torch.float32, device=DEV)
+                .normal_(mean, std, generator=gen))
+
+
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("phase2", [dict(clip_threshold=0.05), dict(clip_threshold=1e3),
+                                    dict(centralize=True),
+                                    dict(clip_threshold=0.05, centralize=True)])
+@pytest.mark.parametrize("variant", [("approximation", "last"), ("classical", "traj_mean"),
+                                     ("none", "last")])
+def test_clip_and_centralize_every_element(gdtype, phase2, variant):
+    nesterov, mode = variant
+    _, params = _shaped(SHAPES, OFFSETS)
+    gen = _gen(5)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    hyper = dict(BASE, nesterov=nesterov, lookahead_mode=mode, **phase2)
+    pair = Pair(params, hyper)
+    _, grads = _shaped(SHAPES, OFFSETS, dtype=gdtype)
+    for t in range(7):
+        # a non-zero mean makes the row means matter; the norm is ~0.3: clipped at 0.05
+        _fill_grads(grads, gen, std=1e-3, mean=5e-4 * (1 + t % 3))
+        pair.step(grads)
+        if "clip_threshold" in phase2:
+            pair.record_grad_stats()
+    pair.check(f"phase2 {phase2}")
+    info = pair.opt.info()
+    assert info["grad_processing"] == (2 if phase2.get("centralize") else 1)
+    assert info["launches"] == 3 * 7          # two statistics kernels + the step kernel
+    if phase2.get("clip_threshold") == 0.05:
+        assert all(f < 1.0 for f in pair.clip_factors)
+    if phase2.get("clip_threshold") == 1e3:
+        assert all(f == 1.0 for f in pair.clip_factors)
+
+
+def test_phase2_is_bit_identical_from_run_to_run_and_across_launch_options():
+    results = []
+    for kw in (dict(), dict(), dict(dependent_launch=False), dict(chunk_elems=1024)):
+        _, params = _shaped(SHAPES, OFFSETS)
+        gen = _gen(9)
+        for p in params:
+            p.normal_(0.0, 0.05, generator=gen)
+        opt = B.NovakOptimizer(params, **BASE, clip_threshold=0.05, centralize=True, **kw)
+        _, grads = _shaped(SHAPES, OFFSETS)
+        norms = []
+        for _ in range(6):
+            _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+            opt.step(grads)
+            norms.append(opt.grad_stats()[0])
+        torch.cuda.synchronize()
+        results.append((norms, [p.clone() for p in params]))
+    for norms, params in results[1:3]:      # same chunking: bit-identical, norm included
+        assert norms == results[0][0]
+        for a, b in zip(params, results[0][1]):
+            assert torch.equal(a, b)
+    # another chunk length adds the squares in another order: equal to rounding
+    np.testing.assert_allclose(results[3][0], results[0][0], rtol=1e-12)
+
+
+def test_options_can_change_between_steps_and_rows_can_be_reset():
+    shapes = [(12, 300), (50,), (4, 2, 9)]
+    _, params = _shaped(shapes, [0, 0, 0])
+    gen = _gen(17)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    opt = B.NovakOptimizer(params, **BASE)
+    oracle = harness.O.Oracle(harness.oracle_config(dict(BASE)), [to_f64(p) for p in params],
+                              rows=harness.tensor_rows(params))
+    _, grads = _shaped(shapes, [0, 0, 0])
+    plan = [dict(), dict(clip=0.02), dict(clip=0.02, gc=True), dict(gc=True), dict(),
+            dict(clip=0.5, gc=True)]
+    for cfg in plan:
+        _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+        opt.handle.set_option(B.NOVAK_OPT_CLIP_THRESHOLD, cfg.get("clip", 0.0))
+        if cfg.get("gc"):
+            opt.handle.set_tensor_rows(harness.tensor_rows(params))
+        opt.handle.set_option(B.NOVAK_OPT_CENTRALIZE, 1 if cfg.get("gc") else 0)
+        oracle.cfg.clip_threshold = cfg.get("clip", 0.0)
+        oracle.cfg.centralize = bool(cfg.get("gc"))
+        opt.step(grads)
+        oracle.step([to_f64(g) for g in grads])
+    torch.cuda.synchronize()
+    for i, p in enumerate(params):
+        harness.assert_close(p, oracle.theta[i], f"theta[{i}]")
+        harness.assert_close(opt.state(i)["m"], oracle.m[i], f"m[{i}]")
+        harness.assert_close(opt.state(i)["v"], oracle.v[i], f"v[{i}]")
+
+
+def test_set_tensor_rows_rejects_bad_input_and_noalloc_refuses_phase2():
+    shapes = [(6, 10), (8,)]
+    _, params = _shaped(shapes, [0, 0])
+    opt = B.NovakOptimizer(params, **BASE)
+    h = opt.handle
+    for bad in ([7, 0], [-1, 0], [6], [6, 0, 0]):
+        with pytest.raises(B.NovakError) as e:
+            h.set_tensor_rows(bad)
+        assert e.value.status == B.NOVAK_EINVAL
+    with pytest.raises(B.NovakError):
+        h.set_option(B.NOVAK_OPT_CLIP_THRESHOLD, -1.0)
+    with pytest.raises(B.NovakError) as e:
+        h.get_grad_stats()
+    assert e.value.status == B.NOVAK_ESTATE
+    h.set_option(B.NOVAK_OPT_CLIP_THRESHOLD, 1.0)
+    _, grads = _shaped(shapes, [0, 0])
+    gl = opt.prepare(grads)
+    with pytest.raises(B.NovakError) as e:
+        h.step_noalloc(opt._params_arr, gl.arr, opt._numel_arr, opt.n, gl.dtype, opt._stream())
+    assert e.value.status == B.NOVAK_ESTATE
+    assert opt.info()["t"] == 0
+
+
+def test_step_host_with_phase2_matches_step():
+    shapes = [(20, 300), (31,), (9, 1000), (3,)]
+    numels = [math.prod(s) for s in shapes]
+    hyper = dict(BASE, lookahead_k=2, clip_threshold=0.02, centralize=True)
+    gen = _gen(23)
+    _, pa = _shaped(shapes, [0] * 4)
+    for p in pa:
+        p.normal_(0.0, 0.05, generator=gen)
+    _, pb = _shaped(shapes, [0] * 4)
+    for x, y in zip(pa, pb):
+        y.copy_(x)
+    a = B.NovakOptimizer(pa, **hyper)
+    b = B.NovakOptimizer(pb, **hyper)
+    b.handle.set_option(B.NOVAK_OPT_HOST_SEGMENT_ELEMS, 4096)
+    total = sum(numels)
+    h_g = torch.empty(total, dtype=torch.float32).pin_memory()
+    h_p = torch.empty(total, dtype=torch.float32).pin_memory()
+    d_g = torch.empty(total, dtype=torch.float32, device=DEV)
+    offs = np.concatenate([[0], np.cumsum(numels)])[:-1]
+    hg = B.ptr_array([h_g.data_ptr() + 4 * int(o) for o in offs])
+    hp = B.ptr_array([h_p.data_ptr() + 4 * int(o) for o in offs])
+    dg = B.ptr_array([d_g.data_ptr() + 4 * int(o) for o in offs])
+    stream = torch.cuda.current_stream().cuda_stream
+    _, grads = _shaped(shapes, [0] * 4)
+    for _ in range(4):
+        _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+        a.step(grads)
+        h_g.copy_(torch.cat([g.reshape(-1) for g in grads]).cpu())
+        b.handle.step_host(hp, hg, b._params_arr, dg, b._numel_arr, len(numels),
+                           B.NOVAK_GRAD_F32, stream)
+        torch.cuda.synchronize()
+        assert torch.equal(h_p, torch.cat([p.reshape(-1) for p in pa]).cpu())
+    assert a.grad_stats() == b.grad_stats()
+
+
+def test_fullsize_resnet50_with_clipping_and_centralization():
+    """The benchmark's ResNet-50-shaped set with its real tensor shapes (53 conv / fc
+    weights with rows, 108 one-dimensional tensors), every element against the oracle."""
+    wl = W.get_workload(1)
+    flat_p = W.alloc_flat(wl, torch.float32, DEV)
+    W.init_params(wl, flat_p)
+    params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
+    flat_g = W.alloc_flat(wl, torch.float32, DEV)
+    grads = [v.view(s) for v, s in zip(W.views(flat_g, wl), wl.shapes)]
+    src = W.GradSource(wl, DEV)
+    harness.MARGINS.clear()
+    pair = Pair(params, dict(wl.hyper, clip_threshold=1.0, centralize=True))
+    for _ in range(12):
+        src.fill(flat_g)
+        pair.step(grads, threads=8)
+        pair.record_grad_stats()
+    pair.check("resnet50 phase2")
+    assert all(f < 1.0 for f in pair.clip_factors)     # norm ~ 5: the clipping is active
+    top = sorted(harness.MARGINS.items(), key=lambda kv: -kv[1])[:4]
+    print("\nworst tensors:", [(k, round(v, 3), wl.shapes[int(k.split("[")[1][:-1])]) for k, v in top])
+    worst = {}
+    for k, v in harness.MARGINS.items():
+        worst[k.split()[-1].split("[")[0]] = max(worst.get(k.split()[-1].split("[")[0], 0.0), v)
+    print("\nPARITY resnet50 clip+centralize steps=12 every element worst |err|/tol: "
+          + ", ".join(f"{k} {v:.3f}" for k, v in worst.items()))
