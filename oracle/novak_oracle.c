@@ -32,6 +32,11 @@
  *     the only difference is which norm is compared with c_clip.
  *     Clipping scales by c_clip/||g|| when ||g|| > c_clip (Table 2's activation
  *     condition), with no epsilon in the denominator.
+ *   - Adaptive beta (Eq. 3-4): beta1(t), beta2(t) replace beta1, beta2 in the
+ *     moment updates (Eq. 1-2) only.  The bias corrections (Eq. 5), rho_inf
+ *     (set once at initialisation in Algorithm 1), rho_t, r_t and the classical
+ *     blend (Eq. 16) keep the base values, as those equations are written.
+ *                                                              [parity unpinned]
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
@@ -52,6 +57,9 @@ typedef struct {
     int32_t lookahead_mode;  /* 0 LAST, 1 TRAJ_MEAN                         */
     int32_t rectified;       /* 1: Eq. 8-9, 0: r_t = 1 on every step        */
     int32_t bias1_power;     /* 1 (default reading) or 2                    */
+    int32_t adaptive_beta;   /* 1: Eq. 3-4 warm-up of beta1, beta2 in Eq. 1-2 */
+    double tau1;             /* warm-up time scale of beta1 (paper: 1000)   */
+    double tau2;             /* warm-up time scale of beta2 (paper: 5000)   */
 } novak_oracle_hparams;
 
 typedef struct {
@@ -64,6 +72,8 @@ typedef struct {
     double decay;     /* 1 - alpha*lambda                   (Eq. 18) */
     int32_t rect_branch; /* 1 when Eq. 8's first case was taken      */
     int32_t is_sync;     /* 1 when lookahead_k>0 and t mod k == 0    */
+    double beta1_t;   /* coefficient of Eq. 1 at this step: beta1, or Eq. 3 */
+    double beta2_t;   /* coefficient of Eq. 2 at this step: beta2, or Eq. 4 */
 } novak_oracle_scalars;
 
 /* Per-step scalars for the 1-based step index t (Eq. 5-9, 18). */
@@ -90,6 +100,13 @@ void novak_oracle_scalars_at(const novak_oracle_hparams *h, int64_t t,
         s->step_size /= s->bc1;
     s->decay = 1.0 - h->lr * h->weight_decay;
     s->is_sync = (h->lookahead_k > 0 && (t % h->lookahead_k) == 0) ? 1 : 0;
+    /* Phase 3, Eq. 3-4: momentum coefficients warmed up over tau1, tau2 steps. */
+    s->beta1_t = h->beta1;
+    s->beta2_t = h->beta2;
+    if (h->adaptive_beta) {
+        s->beta1_t = h->beta1 * (1.0 - exp(-(double)t / h->tau1));
+        s->beta2_t = h->beta2 * (1.0 - exp(-(double)t / h->tau2));
+    }
 }
 
 /*
@@ -112,9 +129,9 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
         if (h->nesterov_variant == 1)
             gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
 
-        /* Phase 4: Eq. 1-2. */
-        m[i] = h->beta1 * m[i] + (1.0 - h->beta1) * gt;
-        v[i] = h->beta2 * v[i] + (1.0 - h->beta2) * gt * gt;
+        /* Phase 4: Eq. 1-2 (with the coefficients of Eq. 3-4 when warmed up). */
+        m[i] = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
+        v[i] = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
 
         /* Phase 5: Eq. 5. */
         double m_hat = m[i] / s.bc1;

@@ -41,6 +41,9 @@ class HParams(ctypes.Structure):
         ("lookahead_mode", ctypes.c_int32),
         ("rectified", ctypes.c_int32),
         ("bias1_power", ctypes.c_int32),
+        ("adaptive_beta", ctypes.c_int32),
+        ("tau1", ctypes.c_double),
+        ("tau2", ctypes.c_double),
     ]
 
 
@@ -55,6 +58,8 @@ class Scalars(ctypes.Structure):
         ("decay", ctypes.c_double),
         ("rect_branch", ctypes.c_int32),
         ("is_sync", ctypes.c_int32),
+        ("beta1_t", ctypes.c_double),
+        ("beta2_t", ctypes.c_double),
     ]
 
 
@@ -123,6 +128,9 @@ class Config:
     bias1_power: int = 1
     clip_threshold: float = 0.0          # c_clip; 0 = clipping off
     centralize: bool = False             # Eq. 26 on tensors given with rows > 0
+    adaptive_beta: bool = False          # Eq. 3-4
+    tau1: float = 1000.0
+    tau2: float = 5000.0
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -130,7 +138,7 @@ class Config:
                        self.weight_decay, nb, self.lookahead_alpha,
                        self.nesterov_variant, self.lookahead_k,
                        self.lookahead_mode, int(self.rectified),
-                       self.bias1_power)
+                       self.bias1_power, int(self.adaptive_beta), self.tau1, self.tau2)
 
 
 def _dptr(a: np.ndarray, offset: int = 0):

@@ -537,6 +537,57 @@ def pin_clip_then_centralize_then_step(lib):
     _close(o.theta[0], p.detach().numpy().reshape(-1), rtol=1e-6, what="AdamW after clip + GC")
 
 
+# --------------------------------------------------------------------------
+# Phase 3: adaptive beta (Eq. 3-4)
+# --------------------------------------------------------------------------
+def pin_adaptive_beta(lib):
+    """beta(t) = beta (1 - exp(-t/tau)) in Eq. 1-2 only.  Moments as explicit sums of
+    products (no recurrence); the schedule's own values; bias corrections, rho_t, r_t
+    and the classical blend unchanged; a vanishing tau gives the constant-beta run."""
+    b1, b2, t1, t2, T = 0.9, 0.999, 7.0, 20.0, 25
+    rng = np.random.default_rng(13)
+    G = rng.normal(0, 1.0, (T, 5))
+    th0 = rng.normal(0, 0.1, 5)
+    kw = dict(beta1=b1, beta2=b2, lookahead_k=0, nesterov_variant=O.NESTEROV_NONE)
+    o = _mk(lib, [th0], adaptive_beta=True, tau1=t1, tau2=t2, **kw)
+    ref = _mk(lib, [th0], **kw)
+    B1 = [b1 * (1 - math.exp(-t / t1)) for t in range(1, T + 1)]
+    B2 = [b2 * (1 - math.exp(-t / t2)) for t in range(1, T + 1)]
+    assert B1[0] < 0.15 * b1 and abs(B1[-1] - b1) < 0.03 * b1     # warms up from near 0 to beta
+    for t in range(1, T + 1):
+        o.step([G[t - 1]])
+        ref.step([G[t - 1]])
+        s, sr = o.scalars(t), ref.scalars(t)
+        _close(s.beta1_t, B1[t - 1], what="beta1(t)")
+        _close(s.beta2_t, B2[t - 1], what="beta2(t)")
+        for name in ("bc1", "bc2", "rho_inf", "rho_t", "r_t", "step_size", "decay"):
+            assert getattr(s, name) == getattr(sr, name), name      # base betas everywhere else
+        assert s.rect_branch == sr.rect_branch
+    m = sum((1 - B1[i]) * math.prod(B1[i + 1:]) * G[i] for i in range(T))
+    v = sum((1 - B2[i]) * math.prod(B2[i + 1:]) * G[i] ** 2 for i in range(T))
+    _close(o.m[0], m, rtol=1e-11, what="m_T under Eq. 3")
+    _close(o.v[0], v, rtol=1e-11, what="v_T under Eq. 4")
+    # half way: beta(tau ln 2) = beta / 2
+    h = _mk(lib, [th0], adaptive_beta=True, tau1=10 / math.log(2), tau2=10 / math.log(2), **kw)
+    _close(h.scalars(10).beta1_t, b1 / 2, what="beta1 at tau ln 2")
+    _close(h.scalars(10).beta2_t, b2 / 2, what="beta2 at tau ln 2")
+    # tau -> 0: the schedule is at its limit from the first step on
+    z = _mk(lib, [th0], adaptive_beta=True, tau1=1e-3, tau2=1e-3, **kw)
+    for t in range(T):
+        z.step([G[t]])
+    _close(z.theta[0], ref.theta[0], rtol=1e-14, what="tau -> 0 equals constant beta")
+    assert not np.allclose(o.theta[0], ref.theta[0], rtol=1e-6)    # and the warm-up matters
+    # the classical blend keeps the base beta1: one step from m = v = 0
+    c = _mk(lib, [np.zeros(1)], lr=1.0, weight_decay=0.0, eps=1e-8, beta1=b1, beta2=b2,
+            lookahead_k=0, nesterov_variant=O.NESTEROV_CLASSICAL, rectified=False,
+            adaptive_beta=True, tau1=t1, tau2=t2)
+    c.step([np.array([2.0])])
+    mh = (1 - B1[0]) * 2.0 / (1 - b1)
+    vh = (1 - B2[0]) * 4.0 / (1 - b2)
+    _close(c.theta[0], -(b1 * mh + (1 - b1) * mh / (math.sqrt(vh) + 1e-8)), rtol=1e-12,
+           what="classical blend with base beta1")
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -556,4 +607,5 @@ ALL_PINS = [
     pin_clip_library,
     pin_centralize_library_and_invariants,
     pin_clip_then_centralize_then_step,
+    pin_adaptive_beta,
 ]

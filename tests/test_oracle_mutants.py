@@ -16,12 +16,12 @@ SRC = os.path.join(os.path.dirname(O.__file__), "novak_oracle.c")
 
 # (name, text in the oracle, replacement)
 MUTANTS = [
-    ("m_sign", "(1.0 - h->beta1) * gt;", "(1.0 + h->beta1) * gt;"),
-    ("v_not_squared", "(1.0 - h->beta2) * gt * gt;", "(1.0 - h->beta2) * gt;"),
-    ("v_uses_beta1", "h->beta2 * v[i]", "h->beta1 * v[i]"),
+    ("m_sign", "(1.0 - s.beta1_t) * gt;", "(1.0 + s.beta1_t) * gt;"),
+    ("v_not_squared", "(1.0 - s.beta2_t) * gt * gt;", "(1.0 - s.beta2_t) * gt;"),
+    ("v_uses_beta1", "s.beta2_t * v[i]", "s.beta1_t * v[i]"),
     ("approx_sign", "h->nesterov_beta * (g[i] - m[i]);", "h->nesterov_beta * (m[i] - g[i]);"),
     ("approx_uses_new_m_only_first_moment",
-     "(1.0 - h->beta2) * gt * gt;", "(1.0 - h->beta2) * g[i] * g[i];"),
+     "(1.0 - s.beta2_t) * gt * gt;", "(1.0 - s.beta2_t) * g[i] * g[i];"),
     ("vhat_uses_bc1", "double v_hat = v[i] / s.bc2;", "double v_hat = v[i] / s.bc1;"),
     ("mhat_uses_bc2", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i] / s.bc2;"),
     ("mhat_uncorrected", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i];"),
@@ -45,6 +45,16 @@ MUTANTS = [
     ("traj_acc_not_reset", "acc[i] = 0.0;", ";"),
     ("bias1_power_ignored", "if (h->bias1_power == 2)", "if (0)"),
     ("rectified_flag_ignored", "if (h->rectified && s->rho_t >= 5.0)", "if (s->rho_t >= 5.0)"),
+    # phase 3: adaptive beta
+    ("warmup_sign", "exp(-(double)t / h->tau1)", "exp((double)t / h->tau1)"),
+    ("warmup_beta2_uses_tau1", "exp(-(double)t / h->tau2)", "exp(-(double)t / h->tau1)"),
+    ("warmup_not_complemented", "h->beta2 * (1.0 - exp(-(double)t / h->tau2));",
+     "h->beta2 * exp(-(double)t / h->tau2);"),
+    ("warmup_in_bias_correction", "s->bc1 = (double)(1.0L - b1t);",
+     "s->bc1 = (double)(1.0L - b1t); if (h->adaptive_beta) s->bc1 = 1.0 - pow(h->beta1 * (1.0 - exp(-(double)t / h->tau1)), (double)t);"),
+    ("warmup_in_classical_blend", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
+     "u = s.beta1_t * m_hat + (1.0 - s.beta1_t) * u;"),
+    ("warmup_flag_ignored", "if (h->adaptive_beta) {", "if (1) {"),
     # phase 2: clipping and centralization
     ("norm_not_rooted", "return sqrt(sum);", "return sum;"),
     ("norm_l1", "sum += g[k][i] * g[k][i];", "sum += fabs(g[k][i]);"),
