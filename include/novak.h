@@ -96,8 +96,14 @@ enum {
     NOVAK_OPT_CLIP_THRESHOLD = 12, /* c_clip >= 0 of the global-norm gradient clipping
                                      (Section 5.8; the paper's default is 1.0), 0
                                      (default here): off.  May change between steps  */
-    NOVAK_OPT_CENTRALIZE = 13     /* 1: gradient centralization (Eq. 26) on the tensors
+    NOVAK_OPT_CENTRALIZE = 13,    /* 1: gradient centralization (Eq. 26) on the tensors
                                      that novak_set_tensor_rows gave rows; 0 (default)  */
+    NOVAK_OPT_ADAPTIVE_BETA = 14, /* 1: momentum scheduling (Section 4.2): the moment
+                                     updates (Eq. 1-2) use beta1(t), beta2(t) of Eq. 3-4;
+                                     bias corrections, rho_t, r_t and the classical
+                                     blend keep the base values.  0 (default)          */
+    NOVAK_OPT_BETA1_TAU = 15,     /* tau_1 > 0 of Eq. 3 (default 1000)                 */
+    NOVAK_OPT_BETA2_TAU = 16      /* tau_2 > 0 of Eq. 4 (default 5000)                 */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -133,6 +139,8 @@ typedef struct novak_info {
     int32_t grad_processing; /* phase 2 as configured: 0 none, 1 clipping,
                                 2 centralization (with or without clipping)        */
     int32_t reserved;
+    double beta1_t, beta2_t; /* coefficients the last step's Eq. 1-2 used: the base
+                                values, or Eq. 3-4 with NOVAK_OPT_ADAPTIVE_BETA     */
 } novak_info;
 
 /* Counters and hyperparameters for checkpoint / resume (Table 3: t and the
@@ -148,6 +156,9 @@ typedef struct novak_meta {
     uint32_t warnings;
     int32_t centralize;
     double clip_threshold;
+    double beta1_tau, beta2_tau;
+    int32_t adaptive_beta;
+    int32_t reserved;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".

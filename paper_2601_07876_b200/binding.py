@@ -27,7 +27,8 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
 (NOVAK_OPT_NESTEROV_BETA, NOVAK_OPT_LOOKAHEAD_MODE, NOVAK_OPT_RECTIFIED, NOVAK_OPT_LR,
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
- NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE) = range(1, 14)
+ NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
+ NOVAK_OPT_BETA2_TAU) = range(1, 17)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -43,6 +44,7 @@ class novak_info(Structure):
         ("lookahead_mode", c_int32), ("lookahead_k", c_int32), ("n_tensors", c_int32),
         ("n_chunks", c_int32), ("grid", c_int32), ("block", c_int32), ("warnings", c_uint32),
         ("grad_processing", c_int32), ("reserved", c_int32),
+        ("beta1_t", c_double), ("beta2_t", c_double),
     ]
 
     def as_dict(self) -> dict:
@@ -58,6 +60,8 @@ class novak_meta(Structure):
         ("nesterov_variant", c_int32), ("lookahead_k", c_int32), ("lookahead_mode", c_int32),
         ("rectified", c_int32), ("bias1_power", c_int32), ("n_tensors", c_int32),
         ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
+        ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
+        ("reserved", c_int32),
     ]
 
 
@@ -295,7 +299,7 @@ class NovakOptimizer:
     def __init__(self, params, lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
-                 clip_threshold=0.0, centralize=False,
+                 clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -339,6 +343,12 @@ class NovakOptimizer:
             h.attach_state(self.state_buffer.data_ptr(), nbytes, self._param_ptrs, self.numel,
                            self._stream())
         self._last_grads = None
+        if tau1 is not None:
+            h.set_option(NOVAK_OPT_BETA1_TAU, tau1)
+        if tau2 is not None:
+            h.set_option(NOVAK_OPT_BETA2_TAU, tau2)
+        if adaptive_beta:
+            h.set_option(NOVAK_OPT_ADAPTIVE_BETA, 1)
         if clip_threshold:
             h.set_option(NOVAK_OPT_CLIP_THRESHOLD, clip_threshold)
         if centralize:

@@ -24,7 +24,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763032ull;  // "NOVAKv02"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763033ull;  // "NOVAKv03"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -35,10 +35,13 @@ struct Hyper {
     double clip;            // c_clip of the global-norm clipping, 0: off
     int nesterov, la_k, la_mode, rectified, bias1_power;
     int centralize;         // Eq. 26 on tensors that were given rows
+    int adaptive_beta;      // Eq. 3-4
+    double tau1, tau2;      // warm-up time scales of beta1, beta2
 };
 
 struct Plan {
     double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay;
+    double beta1_t, beta2_t;   // coefficients of Eq. 1-2 at this step (Eq. 3-4 when warmed up)
     int rect_branch, is_sync;
 };
 
@@ -66,6 +69,13 @@ Plan make_plan(const Hyper &h, int64_t t)
     if (h.bias1_power == 2) p.step_size /= p.bc1;
     p.decay = 1.0 - h.lr * h.wd;
     p.is_sync = (h.la_k > 0 && t % h.la_k == 0) ? 1 : 0;
+    // Phase 3, Eq. 3-4: only the moment updates see the warmed-up coefficients.
+    p.beta1_t = h.beta1;
+    p.beta2_t = h.beta2;
+    if (h.adaptive_beta) {
+        p.beta1_t = h.beta1 * -std::expm1(-td / h.tau1);
+        p.beta2_t = h.beta2 * -std::expm1(-td / h.tau2);
+    }
     return p;
 }
 
@@ -258,6 +268,8 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->block = novak::step_block_threads();
     out->warnings = o->warnings;
     out->grad_processing = pre_mode(o);
+    out->beta1_t = p.beta1_t;
+    out->beta2_t = p.beta2_t;
 }
 
 void release_device(novak_opt *o)
@@ -486,6 +498,8 @@ int check_hyper(const Hyper &h, const char **why)
     if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
     if (!(h.clip >= 0.0) || !std::isfinite(h.clip)) { *why = "clip threshold must be >= 0"; return 0; }
     if (h.centralize != 0 && h.centralize != 1) { *why = "centralize must be 0 or 1"; return 0; }
+    if (h.adaptive_beta != 0 && h.adaptive_beta != 1) { *why = "adaptive_beta must be 0 or 1"; return 0; }
+    if (!(h.tau1 > 0.0) || !std::isfinite(h.tau1) || !(h.tau2 > 0.0) || !std::isfinite(h.tau2)) { *why = "warm-up time scales must be > 0"; return 0; }
     return 1;
 }
 
@@ -509,6 +523,9 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.bias1_power = 1;
     h.clip = 0.0;
     h.centralize = 0;
+    h.adaptive_beta = 0;
+    h.tau1 = 1000.0;       // Section 4.2's values
+    h.tau2 = 5000.0;
     uint32_t warn = 0;
     h.nesterov = nesterov_variant;
     if (nesterov_variant == NOVAK_NESTEROV_TRUE) {
@@ -555,6 +572,12 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
         h.bias1_power = static_cast<int>(value);
         break;
+    case NOVAK_OPT_ADAPTIVE_BETA:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "adaptive_beta must be 0 or 1");
+        h.adaptive_beta = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_BETA1_TAU: h.tau1 = value; break;
+    case NOVAK_OPT_BETA2_TAU: h.tau2 = value; break;
     case NOVAK_OPT_CLIP_THRESHOLD: h.clip = value; break;
     case NOVAK_OPT_CENTRALIZE:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "centralize must be 0 or 1");
@@ -608,6 +631,9 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_LR: *value = o->h.lr; break;
     case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
     case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
+    case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
+    case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
+    case NOVAK_OPT_BETA2_TAU: *value = o->h.tau2; break;
     case NOVAK_OPT_CLIP_THRESHOLD: *value = o->h.clip; break;
     case NOVAK_OPT_CENTRALIZE: *value = o->h.centralize; break;
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
@@ -685,10 +711,12 @@ namespace {
 StepScalars make_scalars(const Hyper &h, const Plan &p)
 {
     StepScalars s;
-    s.beta1 = static_cast<float>(h.beta1);
-    s.omb1 = static_cast<float>(1.0 - h.beta1);
-    s.beta2 = static_cast<float>(h.beta2);
-    s.omb2 = static_cast<float>(1.0 - h.beta2);
+    s.beta1 = static_cast<float>(p.beta1_t);
+    s.omb1 = static_cast<float>(1.0 - p.beta1_t);
+    s.beta2 = static_cast<float>(p.beta2_t);
+    s.omb2 = static_cast<float>(1.0 - p.beta2_t);
+    s.blend_b1 = static_cast<float>(h.beta1);
+    s.blend_omb1 = static_cast<float>(1.0 - h.beta1);
     s.beta_n = static_cast<float>(h.beta_n);
     s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
     s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
@@ -1068,19 +1096,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     const int64_t t = o->t + 1;
     const Plan p = make_plan(o->h, t);
     const int la_action = lookahead_action(o->h, t);
-    StepScalars s;
-    s.beta1 = static_cast<float>(o->h.beta1);
-    s.omb1 = static_cast<float>(1.0 - o->h.beta1);
-    s.beta2 = static_cast<float>(o->h.beta2);
-    s.omb2 = static_cast<float>(1.0 - o->h.beta2);
-    s.beta_n = static_cast<float>(o->h.beta_n);
-    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
-    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
-    s.eps = static_cast<float>(o->h.eps);
-    s.decay = static_cast<float>(p.decay);
-    s.step = static_cast<float>(p.step_size);
-    s.la_alpha = static_cast<float>(o->h.la_alpha);
-    s.k = static_cast<float>(o->h.la_k > 0 ? o->h.la_k : 1);
+    const StepScalars s = make_scalars(o->h, p);
 
     const int n_chunks = static_cast<int>(o->na_chunks.size());
     novak::LaunchCfg cfg;
@@ -1179,6 +1195,9 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->bias1_power = o->h.bias1_power;
     out->clip_threshold = o->h.clip;
     out->centralize = o->h.centralize;
+    out->adaptive_beta = o->h.adaptive_beta;
+    out->beta1_tau = o->h.tau1;
+    out->beta2_tau = o->h.tau2;
     out->n_tensors = o->n;
     out->warnings = o->warnings;
     return NOVAK_OK;
@@ -1199,6 +1218,9 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.nesterov = in->nesterov_variant; h.rectified = in->rectified;
     h.bias1_power = in->bias1_power;
     h.clip = in->clip_threshold;
+    h.adaptive_beta = in->adaptive_beta;
+    h.tau1 = in->beta1_tau;
+    h.tau2 = in->beta2_tau;
     if (h.centralize != in->centralize) invalidate_tables(o);
     h.centralize = in->centralize;
     const char *why;

@@ -30,8 +30,9 @@ struct __align__(16) Chunk {
 // Per-step scalars, computed in double on the host and rounded once
 // (Section 8.1: computed once per step and broadcast to every thread).
 struct StepScalars {
-    float beta1, omb1;     // beta1, 1-beta1
-    float beta2, omb2;     // beta2, 1-beta2
+    float beta1, omb1;     // coefficient of Eq. 1 at this step (Eq. 3 when warmed up), 1 - it
+    float beta2, omb2;     // coefficient of Eq. 2 at this step (Eq. 4 when warmed up), 1 - it
+    float blend_b1, blend_omb1;  // base beta1, 1-beta1 of the classical blend (Eq. 16)
     float beta_n;          // Eq. 13
     float inv_bc1, inv_bc2;// 1/(1-beta1^t), 1/(1-beta2^t)   (Eq. 5)
     float eps;

@@ -164,7 +164,7 @@ __device__ __forceinline__ void update_element(float &p, float g, float &m, floa
     float u = m_hat / (sqrtf(v_hat) + s.eps);
 #endif
     if constexpr (NEST == NOVAK_NESTEROV_CLASSICAL)
-        u = fmaf(s.beta1, m_hat, s.omb1 * u);
+        u = fmaf(s.blend_b1, m_hat, s.blend_omb1 * u);
     // Phase 9, Eq. 18 + 24: decay with the base rate, step with alpha r_t
     const float theta_in = p;
     const float theta_fast = fmaf(theta_in, s.decay, -(s.step * u));

@@ -165,6 +165,33 @@ def test_planner_options():
     assert abs(p2.step_size * p2.bc1 - p1.step_size) < 1e-18
 
 
+def test_planner_adaptive_beta_agrees_with_oracle():
+    """Eq. 3-4 in the library's plan (-expm1(-t/tau)) against the oracle's (1 - exp)."""
+    h = B.Handle(**GOOD)
+    for name in ("beta1_t", "beta2_t"):
+        assert getattr(h.plan(3), name) == GOOD[name[:5]]        # off: the base values
+    h.set_option(B.NOVAK_OPT_ADAPTIVE_BETA, 1)
+    assert h.get_option(B.NOVAK_OPT_BETA1_TAU) == 1000.0
+    assert h.get_option(B.NOVAK_OPT_BETA2_TAU) == 5000.0
+    for taus in ((1000.0, 5000.0), (7.0, 20.0), (500.0, 2500.0)):
+        h.set_option(B.NOVAK_OPT_BETA1_TAU, taus[0])
+        h.set_option(B.NOVAK_OPT_BETA2_TAU, taus[1])
+        o = O.Oracle(O.Config(adaptive_beta=True, tau1=taus[0], tau2=taus[1]), [np.zeros(1)])
+        ref = B.Handle(**GOOD)
+        for t in [1, 2, 5, 6, 100, 1000, 5000, 10 ** 5, 10 ** 7]:
+            a, b, r = h.plan(t), o.scalars(t), ref.plan(t)
+            assert abs(a.beta1_t - b.beta1_t) <= 1e-13 * b.beta1_t, (t, a.beta1_t, b.beta1_t)
+            assert abs(a.beta2_t - b.beta2_t) <= 1e-13 * b.beta2_t, (t, a.beta2_t, b.beta2_t)
+            # nothing else of the plan moves (Eq. 5-9 keep the base coefficients)
+            for name in ("bc1", "bc2", "rho_t", "r_t", "step_size", "rect_branch"):
+                assert getattr(a, name) == getattr(r, name), name
+    for bad in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(B.NovakError):
+            h.set_option(B.NOVAK_OPT_BETA1_TAU, bad)
+    with pytest.raises(B.NovakError):
+        h.set_option(B.NOVAK_OPT_ADAPTIVE_BETA, 2)
+
+
 def test_chunk_builder_covers_every_element_once():
     numel = [1, 31, 32, 33, 8192, 8193, 100_000, 5]
     phase = [0, 3, 31, 0, 7, 0, 16, 30]

@@ -236,6 +236,24 @@ def test_options_rectified_off_and_bias1_power_and_beta_n():
         pair.check(str(extra))
 
 
+@pytest.mark.parametrize("nesterov", ["approximation", "classical"])
+def test_adaptive_beta_warm_up(nesterov):
+    """Eq. 3-4 with short time scales so that 30 steps cross most of the warm-up."""
+    numels = [9000, 33, 2049]
+    _, params, _ = _fresh(numels, seed=51)
+    pair = Pair(params, dict(BASE, nesterov=nesterov, adaptive_beta=True, tau1=6.0, tau2=25.0))
+    gen = _gen(52)
+    for t in range(1, 31):
+        pair.step(_grads(numels, gen))
+        info, s = pair.opt.info(), pair.oracle.scalars(t)
+        assert abs(info["beta1_t"] - s.beta1_t) < 1e-13 and abs(info["beta2_t"] - s.beta2_t) < 1e-13
+    assert 0.89 < pair.opt.info()["beta1_t"] < 0.9
+    pair.check("adaptive beta")
+    # the paper's time scales as the default
+    opt = B.NovakOptimizer(_fresh([100], seed=1)[1], **BASE, adaptive_beta=True)
+    assert opt.plan(1000)["beta1_t"] == pytest.approx(0.9 * (1 - np.exp(-1.0)), rel=1e-12)
+
+
 def test_gradient_pointers_may_change_every_step():
     numels = [9000, 100]
     _, params, _ = _fresh(numels, seed=41)
