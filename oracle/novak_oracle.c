@@ -37,6 +37,11 @@
  *     (set once at initialisation in Algorithm 1), rho_t, r_t and the classical
  *     blend (Eq. 16) keep the base values, as those equations are written.
  *                                                              [parity unpinned]
+ *   - Layer-wise adaptation (Eq. 19, 25): one trust ratio per tensor,
+ *     clip(||theta_t||_2 / ||u_t||_2, 0.1, 10), theta_t the parameters before
+ *     the step, u_t the base direction of Eq. 17 (before the classical blend),
+ *     multiplying the step size of Eq. 24a; where ||u_t|| = 0 the ratio is
+ *     undefined and taken as 1 (the update is zero there anyway).
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
@@ -110,14 +115,46 @@ void novak_oracle_scalars_at(const novak_oracle_hparams *h, int64_t t,
 }
 
 /*
+ * Layer-wise adaptation, Eq. 19 / 25, for ONE tensor of n elements at step t:
+ * clip(||theta_t||_2 / ||u_t||_2, 0.1, 10), where u_t is the base direction of
+ * Eq. 17 that this step's gradient produces (the moments are advanced in local
+ * variables only; nothing is written).  1 when ||u_t|| = 0.
+ */
+double novak_oracle_trust_ratio(const novak_oracle_hparams *h, int64_t t, int64_t n,
+                                const double *theta, const double *g,
+                                const double *m, const double *v)
+{
+    novak_oracle_scalars s;
+    novak_oracle_scalars_at(h, t, &s);
+    double sum_theta = 0.0, sum_u = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double gt = g[i];
+        if (h->nesterov_variant == 1)
+            gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
+        const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
+        const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
+        const double u = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);   /* Eq. 5, 17 */
+        sum_theta += theta[i] * theta[i];
+        sum_u += u * u;
+    }
+    if (sum_u == 0.0)
+        return 1.0;
+    double eta = sqrt(sum_theta) / sqrt(sum_u);
+    if (eta < 0.1) eta = 0.1;
+    if (eta > 10.0) eta = 10.0;
+    return eta;
+}
+
+/*
  * One step (index t, 1-based, i.e. after the counter was incremented) over n
  * independent elements.  theta, m, v are updated in place; g is read only.
  * slow is used when lookahead_k > 0 (caller sets slow = theta_0 before the
  * first step, Eq. 28); acc when lookahead_mode == 1 (caller zeroes it).
+ * trust is the tensor's lambda_trust of Eq. 24a (1 without layer adaptation).
  */
 void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
                        double *theta, const double *g, double *m, double *v,
-                       double *slow, double *acc)
+                       double *slow, double *acc, double trust)
 {
     novak_oracle_scalars s;
     novak_oracle_scalars_at(h, t, &s);
@@ -143,7 +180,7 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
             u = h->beta1 * m_hat + (1.0 - h->beta1) * u;
 
         /* Phase 9: Eq. 18 then Eq. 24 (decay with the base rate alpha). */
-        double theta_fast = theta[i] * s.decay - s.step_size * u;
+        double theta_fast = theta[i] * s.decay - s.step_size * trust * u;
 
         /* Phase 10: lookahead. */
         if (k <= 0) {

@@ -85,8 +85,11 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     dp = ctypes.POINTER(ctypes.c_double)
     lib.novak_oracle_step.argtypes = [
         ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64,
-        dp, dp, dp, dp, dp, dp]
+        dp, dp, dp, dp, dp, dp, ctypes.c_double]
     lib.novak_oracle_step.restype = None
+    lib.novak_oracle_trust_ratio.argtypes = [
+        ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64, dp, dp, dp, dp]
+    lib.novak_oracle_trust_ratio.restype = ctypes.c_double
     lib.novak_oracle_global_norm.argtypes = [
         ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(dp)]
     lib.novak_oracle_global_norm.restype = ctypes.c_double
@@ -128,6 +131,7 @@ class Config:
     bias1_power: int = 1
     clip_threshold: float = 0.0          # c_clip; 0 = clipping off
     centralize: bool = False             # Eq. 26 on tensors given with rows > 0
+    layer_adaptation: bool = False       # Eq. 19 / 25, one trust ratio per tensor
     adaptive_beta: bool = False          # Eq. 3-4
     tau1: float = 1000.0
     tau2: float = 5000.0
@@ -159,6 +163,7 @@ class Oracle:
         one dimension (it is then centralized when cfg.centralize), else 0."""
         self.cfg = cfg
         self.rows = list(rows) if rows is not None else None
+        self.trust: list[list[float]] = []   # per step, per tensor (layer adaptation)
         self.grad_norms: list[float] = []
         self.clip_factors: list[float] = []
         self.h = cfg.to_c()
@@ -180,14 +185,14 @@ class Oracle:
         self.lib.novak_oracle_scalars_at(ctypes.byref(self.h), t, ctypes.byref(s))
         return s
 
-    def _run(self, i: int, g: np.ndarray, lo: int, hi: int):
+    def _run(self, i: int, g: np.ndarray, lo: int, hi: int, trust: float = 1.0):
         null = ctypes.POINTER(ctypes.c_double)()
         self.lib.novak_oracle_step(
             ctypes.byref(self.h), self.t, hi - lo,
             _dptr(self.theta[i], lo), _dptr(g, lo),
             _dptr(self.m[i], lo), _dptr(self.v[i], lo),
             _dptr(self.slow[i], lo) if self.slow is not None else null,
-            _dptr(self.acc[i], lo) if self.acc is not None else null)
+            _dptr(self.acc[i], lo) if self.acc is not None else null, trust)
 
     def process_gradients(self, gs):
         """Phase 2 before the Nesterov approximation: clipping on the global norm
@@ -228,15 +233,21 @@ class Oracle:
         for i, g in enumerate(gs):
             assert g.size == self.theta[i].size
         gs = self.process_gradients(gs)
+        trust = [1.0] * len(gs)
+        if self.cfg.layer_adaptation:
+            trust = [self.lib.novak_oracle_trust_ratio(
+                ctypes.byref(self.h), self.t, g.size, _dptr(self.theta[i]), _dptr(g),
+                _dptr(self.m[i]), _dptr(self.v[i])) for i, g in enumerate(gs)]
+            self.trust.append(trust)
         if threads <= 1:
             for i, g in enumerate(gs):
-                self._run(i, g, 0, g.size)
+                self._run(i, g, 0, g.size, trust[i])
             return
         jobs = []
         for i, g in enumerate(gs):
             n = g.size
             parts = min(threads, max(1, n // 65536))
             bounds = [n * j // parts for j in range(parts + 1)]
-            jobs += [(i, g, bounds[j], bounds[j + 1]) for j in range(parts)]
+            jobs += [(i, g, bounds[j], bounds[j + 1], trust[i]) for j in range(parts)]
         with ThreadPoolExecutor(max_workers=threads) as pool:
             list(pool.map(lambda a: self._run(*a), jobs))

@@ -588,6 +588,74 @@ def pin_adaptive_beta(lib):
            what="classical blend with base beta1")
 
 
+# --------------------------------------------------------------------------
+# Phase 7: layer-wise adaptation (Eq. 19 / 25)
+# --------------------------------------------------------------------------
+def pin_trust_ratio(lib):
+    """lambda_trust = clip(||theta_t|| / ||u_t||, 0.1, 10) per tensor, multiplying the
+    gradient part of the step only.  u_t is recovered from a run WITHOUT layer adaptation
+    (whose step is pinned by the closed forms and library optimizers above), the norms are
+    numpy's: the adapted step must be the plain one stretched by that ratio."""
+    rng = np.random.default_rng(31)
+    lr, wd = 1e-2, 0.1
+    kw = dict(lr=lr, weight_decay=wd, lookahead_k=0, nesterov_variant=O.NESTEROV_APPROX)
+    th = [rng.normal(0, 0.3, 40), rng.normal(0, 3.0, 7), rng.normal(0, 0.02, 300)]
+    d = 1 - lr * wd
+    plain = _mk(lib, th, **kw)
+    adapt = _mk(lib, th, layer_adaptation=True, **kw)
+    for t in range(1, 9):
+        G = [rng.normal(0, 1.0, x.size) for x in th]
+        # both runs start the step from the adapted run's state
+        for i in range(3):
+            plain.theta[i][:] = adapt.theta[i]
+            plain.m[i][:] = adapt.m[i]
+            plain.v[i][:] = adapt.v[i]
+        before = [x.copy() for x in adapt.theta]
+        plain.t = adapt.t
+        plain.step(G)
+        adapt.step(G)
+        step = plain.scalars(t).step_size
+        for i in range(3):
+            u = -(plain.theta[i] - before[i] * d) / step              # Eq. 24 solved for u_t
+            want = np.linalg.norm(before[i]) / np.linalg.norm(u)
+            want = min(max(want, 0.1), 10.0)
+            _close(adapt.trust[-1][i], want, rtol=1e-9, what=f"lambda_trust t={t} tensor {i}")
+            _close(adapt.theta[i] - before[i] * d, want * (plain.theta[i] - before[i] * d),
+                   rtol=1e-9, atol=1e-15, what="only the gradient part is stretched")
+            _close(adapt.m[i], plain.m[i], rtol=0, atol=0, what="moments untouched")
+    ratios = np.array(adapt.trust)
+    assert ratios[:, 0].max() < 10 and ratios[:, 0].min() > 0.1      # tensor 0 unclipped ...
+    assert len({round(float(x), 6) for x in ratios[0]}) == 3          # ... and one ratio per tensor
+    # closed form at t = 1 (variant none): u = g/(|g|+eps), so ||u|| = sqrt(n) |g|/(|g|+eps)
+    n, g0, eps = 16, 0.25, 1e-8
+    o = _mk(lib, [np.full(n, 0.5)], layer_adaptation=True, lr=lr, weight_decay=wd, eps=eps,
+            lookahead_k=0, nesterov_variant=O.NESTEROV_NONE)
+    o.step([np.full(n, -g0)])
+    lam = (0.5 * math.sqrt(n)) / (math.sqrt(n) * g0 / (g0 + eps))
+    _close(o.trust[0][0], lam, what="closed form lambda")
+    _close(o.theta[0], 0.5 * d + lr * lam * g0 / (g0 + eps), what="closed form step")
+    # the clip bounds, and theta -> a theta scales the ratio by a inside them
+    for scale, want in ((1e-4, 0.1), (1e4, 10.0)):
+        o = _mk(lib, [np.full(n, 0.5 * scale)], layer_adaptation=True, lookahead_k=0, **{})
+        o.step([np.full(n, g0)])
+        assert o.trust[0][0] == want
+    a = _mk(lib, [th[0]], layer_adaptation=True, **kw)
+    b = _mk(lib, [3.0 * th[0]], layer_adaptation=True, **kw)
+    G = rng.normal(0, 1.0, 40)
+    a.step([G]); b.step([G])
+    _close(b.trust[0][0], 3.0 * a.trust[0][0], what="scale equivariance")
+    # the ratio uses the base direction of Eq. 17, not the blended one of Eq. 16
+    c = _mk(lib, [th[0]], layer_adaptation=True, **dict(kw, nesterov_variant=O.NESTEROV_CLASSICAL))
+    e = _mk(lib, [th[0]], layer_adaptation=True, **dict(kw, nesterov_variant=O.NESTEROV_NONE))
+    c.step([G]); e.step([G])
+    _close(c.trust[0][0], e.trust[0][0], what="base direction in the ratio")
+    # zero gradient from zero moments: u = 0, ratio taken as 1, pure decay
+    z = _mk(lib, [th[1]], layer_adaptation=True, **kw)
+    z.step([np.zeros(7)])
+    assert z.trust[0][0] == 1.0
+    _close(z.theta[0], th[1] * d, what="pure decay with u = 0")
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -608,4 +676,5 @@ ALL_PINS = [
     pin_centralize_library_and_invariants,
     pin_clip_then_centralize_then_step,
     pin_adaptive_beta,
+    pin_trust_ratio,
 ]

@@ -26,7 +26,7 @@ MUTANTS = [
     ("mhat_uses_bc2", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i] / s.bc2;"),
     ("mhat_uncorrected", "double m_hat = m[i] / s.bc1;", "double m_hat = m[i];"),
     ("eps_inside_root", "(sqrt(v_hat) + h->eps)", "sqrt(v_hat + h->eps)"),
-    ("update_sign", "theta[i] * s.decay - s.step_size * u;", "theta[i] * s.decay + s.step_size * u;"),
+    ("update_sign", "theta[i] * s.decay - s.step_size * trust * u;", "theta[i] * s.decay + s.step_size * trust * u;"),
     ("decay_without_lr", "1.0 - h->lr * h->weight_decay;", "1.0 - h->weight_decay;"),
     ("decay_with_rectified_rate", "1.0 - h->lr * h->weight_decay;",
      "1.0 - h->lr * s->r_t * h->weight_decay;"),
@@ -55,6 +55,20 @@ MUTANTS = [
     ("warmup_in_classical_blend", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
      "u = s.beta1_t * m_hat + (1.0 - s.beta1_t) * u;"),
     ("warmup_flag_ignored", "if (h->adaptive_beta) {", "if (1) {"),
+    # phase 7: layer-wise adaptation
+    ("trust_inverted", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sqrt(sum_u) / sqrt(sum_theta);"),
+    ("trust_of_squared_norms", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sum_theta / sum_u;"),
+    ("trust_l1", "sum_u += u * u;", "sum_u += fabs(u);"),
+    ("trust_lower_clip_missing", "if (eta < 0.1) eta = 0.1;", ";"),
+    ("trust_upper_clip_missing", "if (eta > 10.0) eta = 10.0;", ";"),
+    ("trust_old_moments", "const double u = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);",
+     "const double u = (m[i] / s.bc1) / (sqrt(v[i] / s.bc2) + h->eps);"),
+    ("trust_without_nesterov_term", "gt = g[i] + h->nesterov_beta * (g[i] - m[i]);\n        const double m_new",
+     "gt = g[i];\n        const double m_new"),
+    ("trust_on_decay_too", "theta[i] * s.decay - s.step_size * trust * u;",
+     "trust * (theta[i] * s.decay - s.step_size * u);"),
+    ("trust_dropped", "s.step_size * trust * u;", "s.step_size * u;"),
+    ("trust_zero_direction", "if (sum_u == 0.0)\n        return 1.0;", "if (sum_u == 0.0)\n        return 10.0;"),
     # phase 2: clipping and centralization
     ("norm_not_rooted", "return sqrt(sum);", "return sum;"),
     ("norm_l1", "sum += g[k][i] * g[k][i];", "sum += fabs(g[k][i]);"),
