@@ -83,6 +83,9 @@ def parse_args():
                     help="c_clip of the global-norm clipping (0: off, the headline path)")
     ap.add_argument("--centralize", action="store_true",
                     help="gradient centralization on tensors with more than one dimension")
+    ap.add_argument("--layer-adaptation", action="store_true",
+                    help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
+    ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -99,12 +102,14 @@ def parse_args():
 
 
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
-                               phase2: bool = False) -> int:
+                               phase2: bool = False, trust: bool = False) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
     arrays on the steps that touch them, plus one more read of g when clipping or
     centralization is on (the norm and the row means are needed before the update)."""
     b = 12 + grad_bytes + 12 + (grad_bytes if phase2 else 0)
+    if trust:
+        b += 12 + grad_bytes             # theta, g, m, v read once more for the norms of Eq. 19
     if k <= 0:
         return b
     sync = t % k == 0
@@ -310,6 +315,7 @@ def main():
         src.fill(gf, scratch)
     del scratch
     opt = B.NovakOptimizer(params, **hyper, clip_threshold=args.clip, centralize=args.centralize,
+                           layer_adaptation=args.layer_adaptation, adaptive_beta=args.adaptive_beta,
                            chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
@@ -343,13 +349,14 @@ def main():
         ms = float(t.item())
     ms_per_step = ms / args.steps
     value = world * wl.total * args.steps / (ms * 1e-3)
-    alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2)
+    alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
+                                         args.layer_adaptation)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = None if phase2 else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    traffic = None if (phase2 or args.layer_adaptation) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -428,6 +435,8 @@ def main():
                 "grad_dtype": "bf16" if gbytes == 2 else "f32",
                 "lookahead_k": k, "lookahead_mode": args.lookahead_mode,
                 "clip_threshold": args.clip, "centralize": bool(args.centralize),
+                "layer_adaptation": bool(args.layer_adaptation),
+                "adaptive_beta": bool(args.adaptive_beta),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
                       "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),

@@ -103,7 +103,12 @@ enum {
                                      bias corrections, rho_t, r_t and the classical
                                      blend keep the base values.  0 (default)          */
     NOVAK_OPT_BETA1_TAU = 15,     /* tau_1 > 0 of Eq. 3 (default 1000)                 */
-    NOVAK_OPT_BETA2_TAU = 16      /* tau_2 > 0 of Eq. 4 (default 5000)                 */
+    NOVAK_OPT_BETA2_TAU = 16,     /* tau_2 > 0 of Eq. 4 (default 5000)                 */
+    NOVAK_OPT_LAYER_ADAPTATION = 17 /* 1: layer-wise adaptation (Eq. 19 / 25): each
+                                     tensor's step is stretched by its trust ratio
+                                     clip(||theta_t|| / ||u_t||, 0.1, 10).  Two more
+                                     kernels per step read theta, g, m, v once more
+                                     (+16 B per element).  0 (default)               */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -141,6 +146,8 @@ typedef struct novak_info {
     int32_t reserved;
     double beta1_t, beta2_t; /* coefficients the last step's Eq. 1-2 used: the base
                                 values, or Eq. 3-4 with NOVAK_OPT_ADAPTIVE_BETA     */
+    int32_t layer_adaptation;
+    int32_t reserved2;
 } novak_info;
 
 /* Counters and hyperparameters for checkpoint / resume (Table 3: t and the
@@ -158,7 +165,7 @@ typedef struct novak_meta {
     double clip_threshold;
     double beta1_tau, beta2_tau;
     int32_t adaptive_beta;
-    int32_t reserved;
+    int32_t layer_adaptation;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
@@ -254,8 +261,9 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
  * no cudaMalloc / cudaFree / cudaHostAlloc / event creation; parameters,
  * gradients and the state buffer are the caller's as in novak_step.
  *
- * Gradient clipping and centralization need scratch memory that the library
- * allocates, so this call returns NOVAK_ESTATE while either is switched on.
+ * Gradient clipping, centralization and layer adaptation need scratch memory
+ * that the library allocates, so this call returns NOVAK_ESTATE while any of
+ * them is switched on.
  *
  * Limits: at most 4096 tensors and 131072 chunk-table entries (= 268 M
  * elements at the default 2048 elements per entry; raise
@@ -309,6 +317,14 @@ int novak_set_tensor_rows(novak_opt *opt, const int64_t *rows, int n);
  * the device and SYNCHRONISES `stream`.  Either output may be NULL.
  * NOVAK_ESTATE when no such step has run. */
 int novak_get_grad_stats(novak_opt *opt, double *norm, double *factor, void *stream);
+
+/* Layer-wise adaptation (Eq. 19 / 25, NOVAK_OPT_LAYER_ADAPTATION): the trust
+ * ratio of every tensor as the last step used it, h_out[i] for tensor i (host
+ * array of n floats).  The ratio is ||theta_t||_2 / ||u_t||_2 clipped to
+ * [0.1, 10], theta_t the parameters before the step, u_t the step's base
+ * direction (Eq. 17); 1 where ||u_t|| = 0.  Copies n floats from the device and
+ * SYNCHRONISES `stream`.  NOVAK_ESTATE when no such step has run. */
+int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
 
 /* Counters and the last step's scalars (bit-exact step and sync indices). */
 int novak_get_info(const novak_opt *opt, novak_info *out);

@@ -28,7 +28,7 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
- NOVAK_OPT_BETA2_TAU) = range(1, 17)
+ NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION) = range(1, 18)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -45,6 +45,7 @@ class novak_info(Structure):
         ("n_chunks", c_int32), ("grid", c_int32), ("block", c_int32), ("warnings", c_uint32),
         ("grad_processing", c_int32), ("reserved", c_int32),
         ("beta1_t", c_double), ("beta2_t", c_double),
+        ("layer_adaptation", c_int32), ("reserved2", c_int32),
     ]
 
     def as_dict(self) -> dict:
@@ -61,7 +62,7 @@ class novak_meta(Structure):
         ("rectified", c_int32), ("bias1_power", c_int32), ("n_tensors", c_int32),
         ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
         ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
-        ("reserved", c_int32),
+        ("layer_adaptation", c_int32),
     ]
 
 
@@ -107,6 +108,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_set_tensor_rows": (c_int, [vp, i64p, c_int]),
         "novak_get_grad_stats": (c_int, [vp, POINTER(c_double), POINTER(c_double), vp]),
+        "novak_get_trust_ratios": (c_int, [vp, POINTER(ctypes.c_float), c_int, vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
         "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
         "novak_state_ptrs": (c_int, [vp, c_int, vpp, vpp, vpp, vpp]),
@@ -237,6 +239,13 @@ class Handle:
                "novak_get_grad_stats")
         return norm.value, factor.value
 
+    def get_trust_ratios(self, n: int, stream: int = 0):
+        """Per-tensor trust ratios of the last step; synchronises the stream."""
+        out = (ctypes.c_float * n)()
+        _check(self.lib, self.h, self.lib.novak_get_trust_ratios(self.h, out, n, stream),
+               "novak_get_trust_ratios")
+        return list(out)
+
     def get_info(self) -> novak_info:
         out = novak_info()
         _check(self.lib, self.h, self.lib.novak_get_info(self.h, byref(out)), "novak_get_info")
@@ -300,6 +309,7 @@ class NovakOptimizer:
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
+                 layer_adaptation=False,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -349,12 +359,17 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_BETA2_TAU, tau2)
         if adaptive_beta:
             h.set_option(NOVAK_OPT_ADAPTIVE_BETA, 1)
+        if layer_adaptation:
+            h.set_option(NOVAK_OPT_LAYER_ADAPTATION, 1)
         if clip_threshold:
             h.set_option(NOVAK_OPT_CLIP_THRESHOLD, clip_threshold)
         if centralize:
             # Eq. 26 applies to tensors with more than one dimension
             h.set_tensor_rows([p.shape[0] if p.dim() > 1 else 0 for p in self.params])
             h.set_option(NOVAK_OPT_CENTRALIZE, 1)
+
+    def trust_ratios(self):
+        return self.handle.get_trust_ratios(self.n, self._stream())
 
     def grad_stats(self):
         return self.handle.get_grad_stats(self._stream())

@@ -24,7 +24,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763033ull;  // "NOVAKv03"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763034ull;  // "NOVAKv04"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -35,6 +35,7 @@ struct Hyper {
     double clip;            // c_clip of the global-norm clipping, 0: off
     int nesterov, la_k, la_mode, rectified, bias1_power;
     int centralize;         // Eq. 26 on tensors that were given rows
+    int layer_adapt;        // Eq. 19 / 25: one trust ratio per tensor
     int adaptive_beta;      // Eq. 3-4
     double tau1, tau2;      // warm-up time scales of beta1, beta2
 };
@@ -183,6 +184,14 @@ struct novak_opt {
     double *chunk_sq = nullptr, *seg_first = nullptr, *seg_last = nullptr, *cta_sq = nullptr;
     float2 *row_mean = nullptr;
 
+    // Scratch of layer adaptation (one allocation): two sums of squares per
+    // chunk-table entry, where each tensor's entries start, the trust ratios.
+    char *d_trust = nullptr;
+    double *chunk_u2 = nullptr, *chunk_p2 = nullptr;
+    int *tensor_first = nullptr;
+    float *trust = nullptr;
+    std::vector<int> h_tensor_first;
+
     // novak_step_host: the chunk table cut into segments, each with the element
     // ranges it covers, two copy streams and the events that order them.
     struct Range { int tensor; int64_t off, len; };
@@ -268,6 +277,7 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->block = novak::step_block_threads();
     out->warnings = o->warnings;
     out->grad_processing = pre_mode(o);
+    out->layer_adaptation = o->h.layer_adapt;
     out->beta1_t = p.beta1_t;
     out->beta2_t = p.beta2_t;
 }
@@ -282,6 +292,11 @@ void release_device(novak_opt *o)
         o->h_recs[i] = nullptr;
         o->ring_ev[i] = nullptr;
     }
+    if (o->d_trust) cudaFree(o->d_trust);
+    o->d_trust = nullptr;
+    o->chunk_u2 = o->chunk_p2 = nullptr;
+    o->tensor_first = nullptr;
+    o->trust = nullptr;
     if (o->d_prep) cudaFree(o->d_prep);
     o->d_prep = nullptr;
     o->prep_rows = -1;
@@ -397,6 +412,34 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
     return NOVAK_OK;
 }
 
+// Scratch of layer adaptation, allocated when a step first needs it.
+int prepare_trust(novak_opt *o, cudaStream_t stream)
+{
+    if (o->d_trust) return NOVAK_OK;
+    const size_t nc = static_cast<size_t>(o->n_chunks), n = static_cast<size_t>(o->n);
+    const size_t off_p2 = nc * sizeof(double);
+    const size_t off_first = 2 * nc * sizeof(double);
+    const size_t off_trust = off_first + (n + 1) * sizeof(int);
+    const size_t bytes = off_trust + n * sizeof(float) + 16;
+    cudaError_t e;
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_trust), bytes)) != cudaSuccess) {
+        o->d_trust = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(layer adaptation, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    o->chunk_u2 = reinterpret_cast<double *>(o->d_trust);
+    o->chunk_p2 = reinterpret_cast<double *>(o->d_trust + off_p2);
+    o->tensor_first = reinterpret_cast<int *>(o->d_trust + off_first);
+    o->trust = reinterpret_cast<float *>(o->d_trust + off_trust);
+    // the table lists a tensor's entries consecutively, tensors in order
+    o->h_tensor_first.assign(n + 1, o->n_chunks);
+    for (int c = o->n_chunks - 1; c >= 0; --c) o->h_tensor_first[o->h_chunks[c].tensor] = c;
+    if ((e = cudaMemcpyAsync(o->tensor_first, o->h_tensor_first.data(), (n + 1) * sizeof(int),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "layer adaptation table upload");
+    return NOVAK_OK;
+}
+
 uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype)
 {
     uint64_t h = 0xcbf29ce484222325ull ^ static_cast<uint64_t>(grad_dtype);
@@ -498,6 +541,7 @@ int check_hyper(const Hyper &h, const char **why)
     if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
     if (!(h.clip >= 0.0) || !std::isfinite(h.clip)) { *why = "clip threshold must be >= 0"; return 0; }
     if (h.centralize != 0 && h.centralize != 1) { *why = "centralize must be 0 or 1"; return 0; }
+    if (h.layer_adapt != 0 && h.layer_adapt != 1) { *why = "layer_adaptation must be 0 or 1"; return 0; }
     if (h.adaptive_beta != 0 && h.adaptive_beta != 1) { *why = "adaptive_beta must be 0 or 1"; return 0; }
     if (!(h.tau1 > 0.0) || !std::isfinite(h.tau1) || !(h.tau2 > 0.0) || !std::isfinite(h.tau2)) { *why = "warm-up time scales must be > 0"; return 0; }
     return 1;
@@ -523,6 +567,7 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.bias1_power = 1;
     h.clip = 0.0;
     h.centralize = 0;
+    h.layer_adapt = 0;
     h.adaptive_beta = 0;
     h.tau1 = 1000.0;       // Section 4.2's values
     h.tau2 = 5000.0;
@@ -571,6 +616,10 @@ int novak_set_option(novak_opt *o, int key, double value)
     case NOVAK_OPT_BIAS1_POWER:
         if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
         h.bias1_power = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_LAYER_ADAPTATION:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "layer_adaptation must be 0 or 1");
+        h.layer_adapt = static_cast<int>(value);
         break;
     case NOVAK_OPT_ADAPTIVE_BETA:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "adaptive_beta must be 0 or 1");
@@ -631,6 +680,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_LR: *value = o->h.lr; break;
     case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
     case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
+    case NOVAK_OPT_LAYER_ADAPTATION: *value = o->h.layer_adapt; break;
     case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
     case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
     case NOVAK_OPT_BETA2_TAU: *value = o->h.tau2; break;
@@ -738,6 +788,7 @@ struct StepCtx {
     const TensorRec *d_recs;
     int reverse;
     int pre;                 // novak::PRE_*
+    const float *trust;      // per-tensor factors of Eq. 25, NULL without layer adaptation
 };
 
 int check_step_args(novak_opt *o, const char *who, void *const *d_params,
@@ -763,6 +814,8 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
         return fail(o, NOVAK_ESTATE, "centralization needs chunk-table entries of at most 2048 "
                     "elements (NOVAK_OPT_CHUNK_ELEMS is %lld)", static_cast<long long>(o->chunk_elems));
     if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
+    if (o->h.layer_adapt && (rc = prepare_trust(o, stream)) != NOVAK_OK) return rc;
+    ctx->trust = o->h.layer_adapt ? o->trust : nullptr;
     if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
     ctx->t = o->t + 1;
     ctx->plan = make_plan(o->h, ctx->t);
@@ -773,8 +826,32 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     ctx->reverse = (o->serpentine && (ctx->t % 2 == 0)) ? 1 : 0;
     // After a statistics pass the END of the gradient is what L2 still holds:
     // the step kernel then walks the table from the end.
-    if (ctx->pre != novak::PRE_NONE) ctx->reverse = 1;
+    if (ctx->pre != novak::PRE_NONE || ctx->trust) ctx->reverse = 1;
     return NOVAK_OK;
+}
+
+// Everything that has to see the whole group before the first element is
+// updated: phase 2's statistics, then phase 7's trust ratios.  Returns the
+// number of kernels launched through *launches.
+cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream);
+cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, int *launches,
+                             const char **what)
+{
+    cudaError_t e;
+    if (ctx.pre != novak::PRE_NONE) {
+        *what = "gradient statistics kernel launch";
+        if ((e = launch_stats(o, ctx, stream)) != cudaSuccess) return e;
+        *launches += 2;
+    }
+    if (ctx.trust) {
+        *what = "layer adaptation kernel launch";
+        e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
+                                      o->prep_out, ctx.s, o->h.nesterov, ctx.grad_dtype, ctx.pre,
+                                      o->chunk_u2, o->chunk_p2, o->trust, o->pdl, stream);
+        if (e != cudaSuccess) return e;
+        *launches += 2;
+    }
+    return cudaSuccess;
 }
 
 // Phase 2's statistics pass over the whole group: global norm, clip factor, row means.
@@ -796,7 +873,7 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     cfg.pdl = o->pdl;
     cfg.pre = ctx.pre;
     o->last_grid = cfg.grid;
-    return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.s,
+    return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.trust, ctx.s,
                               o->h.nesterov, ctx.grad_dtype, ctx.la, cfg, stream);
 }
 
@@ -901,11 +978,9 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
     cudaError_t e;
     int launches = 1;
-    if (ctx.pre != novak::PRE_NONE) {
-        if ((e = launch_stats(o, ctx, stream)) != cudaSuccess)
-            return fail_cuda(o, e, "gradient statistics kernel launch");
-        launches += 2;
-    }
+    const char *what = "";
+    if ((e = launch_prepasses(o, ctx, stream, &launches, &what)) != cudaSuccess)
+        return fail_cuda(o, e, what);
     if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess)
         return fail_cuda(o, e, "step kernel launch");
     commit_step(o, ctx, launches);
@@ -950,7 +1025,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
         if ((e = cudaStreamWaitEvent(o->up_stream, ev_start, 0)) != cudaSuccess) break;
         if ((e = cudaStreamWaitEvent(o->down_stream, ev_start, 0)) != cudaSuccess) break;
         forked = true;
-        const bool stats = ctx.pre != novak::PRE_NONE;
+        const bool stats = ctx.pre != novak::PRE_NONE || ctx.trust != nullptr;
         if (stats) {
             // The norm and the row means need the whole gradient: every run is
             // uploaded before the statistics kernel, and only kernels and
@@ -961,9 +1036,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
             if (e != cudaSuccess) break;
             if ((e = cudaEventRecord(o->host_ev[2], o->up_stream)) != cudaSuccess) break;
             if ((e = cudaStreamWaitEvent(stream, o->host_ev[2], 0)) != cudaSuccess) break;
-            what = "gradient statistics kernel launch";
-            if ((e = launch_stats(o, ctx, stream)) != cudaSuccess) break;
-            extra_launches += 2;
+            if ((e = launch_prepasses(o, ctx, stream, &extra_launches, &what)) != cudaSuccess) break;
         }
         for (int i = 0; i < n_seg && e == cudaSuccess; ++i) {
             const novak_opt::Segment &seg = o->segments[i];
@@ -1017,9 +1090,9 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
         return fail(o, NOVAK_EINVAL, "step_noalloc: unknown grad_dtype %d", grad_dtype);
     if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
         return fail(o, NOVAK_ESTATE, "step_noalloc: tensor list differs from the attached layout");
-    if (pre_mode(o) != novak::PRE_NONE)
-        return fail(o, NOVAK_ESTATE, "step_noalloc: clipping and centralization keep scratch in "
-                    "allocated device memory; use novak_step, or switch them off");
+    if (pre_mode(o) != novak::PRE_NONE || o->h.layer_adapt)
+        return fail(o, NOVAK_ESTATE, "step_noalloc: clipping, centralization and layer adaptation keep "
+                    "scratch in allocated device memory; use novak_step, or switch them off");
     if (n > novak::kNoAllocMaxTensors)
         return fail(o, NOVAK_EINVAL, "step_noalloc: %d tensors exceed the static table's %d; "
                     "split the group or use novak_step", n, novak::kNoAllocMaxTensors);
@@ -1104,7 +1177,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
     cfg.pre = novak::PRE_NONE;
-    e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, s, o->h.nesterov, grad_dtype,
+    e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, nullptr, s, o->h.nesterov, grad_dtype,
                            la_action, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
 
@@ -1155,6 +1228,19 @@ int novak_get_grad_stats(novak_opt *o, double *norm, double *factor, void *strea
     return NOVAK_OK;
 }
 
+int novak_get_trust_ratios(novak_opt *o, float *h_out, int n, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!h_out || n != o->n) return fail(o, NOVAK_EINVAL, "get_trust_ratios: NULL or wrong tensor count");
+    if (!o->trust || o->t == 0) return fail(o, NOVAK_ESTATE, "get_trust_ratios: no step with layer adaptation yet");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(h_out, o->trust, n * sizeof(float), cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "get_trust_ratios");
+    return NOVAK_OK;
+}
+
 int novak_get_info(const novak_opt *o, novak_info *out)
 {
     if (!o || !out) return NOVAK_EINVAL;
@@ -1196,6 +1282,7 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->clip_threshold = o->h.clip;
     out->centralize = o->h.centralize;
     out->adaptive_beta = o->h.adaptive_beta;
+    out->layer_adaptation = o->h.layer_adapt;
     out->beta1_tau = o->h.tau1;
     out->beta2_tau = o->h.tau2;
     out->n_tensors = o->n;
@@ -1219,6 +1306,7 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.bias1_power = in->bias1_power;
     h.clip = in->clip_threshold;
     h.adaptive_beta = in->adaptive_beta;
+    h.layer_adapt = in->layer_adaptation;
     h.tau1 = in->beta1_tau;
     h.tau2 = in->beta2_tau;
     if (h.centralize != in->centralize) invalidate_tables(o);

@@ -85,10 +85,24 @@ cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int pre, int *c
 
 // Launches the fused step kernel.  Returns cudaErrorInvalidValue for a mode
 // combination that has no instantiation.  `prep` may be NULL when cfg.pre is
-// PRE_NONE.
+// PRE_NONE; `trust` (one factor per tensor, Eq. 25) is NULL without layer
+// adaptation.  The chunk entries' tensor indices address recs and trust, so
+// d_chunks may point into the middle of the table.
 cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                        const PrepOut *prep, const StepScalars &s, int nesterov,
+                        const PrepOut *prep, const float *trust, const StepScalars &s, int nesterov,
                         int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream);
+
+// Layer-wise adaptation (Eq. 19 / 25), two kernels over the whole chunk table:
+// per entry the sums of squares of theta_t and of this step's base direction
+// u_t (moments advanced in registers, nothing stored) into chunk_p2 / chunk_u2
+// (n_chunks doubles each), then one CTA per tensor adds its entries
+// [tensor_first[i], tensor_first[i+1]) in order and writes
+// trust[i] = clip(||theta|| / ||u||, 0.1, 10), 1 where ||u|| = 0.
+cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
+                               int n_tensors, const int *tensor_first, const PrepOut *prep,
+                               const StepScalars &s, int nesterov, int grad_dtype, int pre,
+                               double *chunk_u2, double *chunk_p2, float *trust, int pdl,
+                               cudaStream_t stream);
 
 // Launches the gradient statistics pass over the whole chunk table (two
 // kernels): the global norm of the raw gradient and the clip factor into *prep,

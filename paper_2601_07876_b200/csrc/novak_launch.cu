@@ -21,7 +21,7 @@ namespace {
 constexpr int kBlock = NOVAK_BLOCK;
 
 using StepKernelFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *,
-                              StepScalars, int);
+                              const float *, StepScalars, int);
 
 StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
 {
@@ -77,7 +77,7 @@ cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int pre, int *c
 }
 
 cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                        const PrepOut *prep, const StepScalars &s, int nesterov,
+                        const PrepOut *prep, const float *trust, const StepScalars &s, int nesterov,
                         int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream)
 {
     StepKernelFn fn = pick_kernel(nesterov, grad_dtype, la, cfg.pre);
@@ -93,7 +93,7 @@ cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
-    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, s, cfg.reverse);
+    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, trust, s, cfg.reverse);
 }
 
 }  // namespace novak

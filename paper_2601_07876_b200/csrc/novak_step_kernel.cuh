@@ -102,6 +102,7 @@ __device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
 
 // ---- phase 2 before the Nesterov approximation: clip factor and centralization
 struct PreArgs {
+    float step;          // alpha r_t, times the tensor's trust ratio under layer adaptation
     float factor;        // clip factor (1 when clipping is off or inactive)
     const float2 *mean;  // row means of the raw gradient (hi + lo), NULL: tensor not centralized
     uint32_t row_len;
@@ -140,11 +141,11 @@ __device__ __forceinline__ void preprocess(Vec<N> &G, uint32_t e, const PreArgs 
     }
 }
 
-// ---- the per-element update, phases 2 and 4-10 (Section 5.1)
-template <int NEST, int LA>
-__device__ __forceinline__ void update_element(float &p, float g, float &m, float &v,
-                                               float &slow, float &acc,
-                                               const StepScalars &s)
+// ---- phases 2 (Nesterov approximation), 4, 5 and 8 up to the base direction:
+// advances m and v with the processed gradient g and returns u of Eq. 17.
+template <int NEST>
+__device__ __forceinline__ float base_direction(float g, float &m, float &v, float &m_hat,
+                                                const StepScalars &s)
 {
     // Phase 2, Eq. 13: g~ = g + beta_N (g - m_{t-1})
     if constexpr (NEST == NOVAK_NESTEROV_APPROX)
@@ -153,21 +154,33 @@ __device__ __forceinline__ void update_element(float &p, float g, float &m, floa
     m = fmaf(s.beta1, m, s.omb1 * g);
     v = fmaf(s.beta2, v, s.omb2 * (g * g));
     // Phase 5, Eq. 5
-    const float m_hat = m * s.inv_bc1;
+    m_hat = m * s.inv_bc1;
     const float v_hat = v * s.inv_bc2;
-    // Phase 8, Eq. 17 (IEEE sqrt and division), Eq. 16 for the classical blend
+    // Phase 8, Eq. 17 (IEEE sqrt and division)
 #ifdef NOVAK_APPROX_MATH
     float rt, u;
     asm("sqrt.approx.f32 %0, %1;" : "=f"(rt) : "f"(v_hat));
     asm("div.full.f32 %0, %1, %2;" : "=f"(u) : "f"(m_hat), "f"(rt + s.eps));
+    return u;
 #else
-    float u = m_hat / (sqrtf(v_hat) + s.eps);
+    return m_hat / (sqrtf(v_hat) + s.eps);
 #endif
+}
+
+// ---- the per-element update, phases 2 and 4-10 (Section 5.1)
+template <int NEST, int LA>
+__device__ __forceinline__ void update_element(float &p, float g, float &m, float &v,
+                                               float &slow, float &acc,
+                                               const StepScalars &s, float step)
+{
+    float m_hat;
+    float u = base_direction<NEST>(g, m, v, m_hat, s);
+    // Eq. 16 for the classical blend
     if constexpr (NEST == NOVAK_NESTEROV_CLASSICAL)
         u = fmaf(s.blend_b1, m_hat, s.blend_omb1 * u);
     // Phase 9, Eq. 18 + 24: decay with the base rate, step with alpha r_t
     const float theta_in = p;
-    const float theta_fast = fmaf(theta_in, s.decay, -(s.step * u));
+    const float theta_fast = fmaf(theta_in, s.decay, -(step * u));
     // Phase 10, Eq. 28-31
     float out = theta_fast;
     float sum = theta_fast;
@@ -215,7 +228,7 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
 #pragma unroll
         for (int e = 0; e < N; ++e)
             update_element<NEST, LA>(P[j].a[e], G[j].a[e], M[j].a[e], V[j].a[e],
-                                     S[j].a[e], A[j].a[e], s);
+                                     S[j].a[e], A[j].a[e], s, pre.step);
         store_f32<N>(p, idx, P[j]);
         store_f32<N>(m, idx, M[j]);
         store_f32<N>(v, idx, V[j]);
@@ -258,7 +271,7 @@ template <int NEST, int GT, int LA, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS)
 novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                   const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                  const StepScalars s, int reverse)
+                  const float *__restrict__ trust, const StepScalars s, int reverse)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
@@ -280,6 +293,8 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 
 #pragma unroll 1
     for (;;) {
+        // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
+        pre.step = trust != nullptr ? s.step * __ldg(trust + ch.tensor) : s.step;
         pre.mean = (PRE == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
@@ -315,7 +330,7 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 }
 
 using StepKernelFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *,
-                              StepScalars, int);
+                              const float *, StepScalars, int);
 
 template <int NEST, int GT, int PRE>
 StepKernelFn pick_la(int la)

@@ -209,3 +209,82 @@ def test_fullsize_resnet50_with_clipping_and_centralization():
         worst[k.split()[-1].split("[")[0]] = max(worst.get(k.split()[-1].split("[")[0], 0.0), v)
     print("\nPARITY resnet50 clip+centralize steps=12 every element worst |err|/tol: "
           + ", ".join(f"{k} {v:.3f}" for k, v in worst.items()))
+
+
+# ---------------------------------------------------------------------------
+# Phase 7: layer-wise adaptation (Eq. 19 / 25)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("extra", [dict(), dict(clip_threshold=0.05, centralize=True),
+                                   dict(adaptive_beta=True, tau1=5.0, tau2=20.0)])
+@pytest.mark.parametrize("variant", [("approximation", "last"), ("classical", "traj_mean"),
+                                     ("none", "last")])
+def test_layer_adaptation_every_element(gdtype, extra, variant):
+    nesterov, mode = variant
+    _, params = _shaped(SHAPES, OFFSETS)
+    gen = _gen(71)
+    # parameter scales from 1e-4 to 30: ratios below, inside and above the clip range
+    for i, p in enumerate(params):
+        p.normal_(0.0, 10.0 ** (-4 + 5.5 * i / (len(params) - 1)), generator=gen)
+    pair = Pair(params, dict(BASE, nesterov=nesterov, lookahead_mode=mode,
+                             layer_adaptation=True, **extra))
+    _, grads = _shaped(SHAPES, OFFSETS, dtype=gdtype)
+    for t in range(7):
+        _fill_grads(grads, gen, std=1e-3, mean=5e-4)
+        pair.step(grads)
+        got = pair.opt.trust_ratios()
+        np.testing.assert_allclose(got, pair.oracle.trust[-1], rtol=2e-6)
+    pair.check(f"layer adaptation {extra}")
+    seen = np.array(pair.oracle.trust)
+    assert (seen == 0.1).any() and (seen == 10.0).any() and ((seen > 0.1) & (seen < 10.0)).any()
+    n_pre = 2 if extra.get("centralize") or extra.get("clip_threshold") else 0
+    assert pair.opt.info()["launches"] == 7 * (3 + n_pre)
+    assert pair.opt.info()["layer_adaptation"] == 1
+
+
+def test_layer_adaptation_zero_gradient_and_reruns():
+    """A tensor whose direction is zero gets ratio 1 (and only decays); reruns agree bit for bit."""
+    shapes = [(5, 300), (4000,), (7,)]
+    outs = []
+    for _ in range(2):
+        _, params = _shaped(shapes, [0, 0, 0])
+        gen = _gen(3)
+        for p in params:
+            p.normal_(0.0, 0.1, generator=gen)
+        before = params[2].clone()
+        opt = B.NovakOptimizer(params, **BASE, layer_adaptation=True)
+        _, grads = _shaped(shapes, [0, 0, 0])
+        ratios = []
+        for _ in range(3):
+            _fill_grads(grads[:2], gen, std=1e-2)
+            grads[2].zero_()
+            opt.step(grads)
+            ratios.append(opt.trust_ratios())
+        torch.cuda.synchronize()
+        assert all(r[2] == 1.0 for r in ratios)
+        d = np.float32(1 - 1e-3 * 1e-2)
+        expect = before * d * d * d
+        assert torch.allclose(params[2], expect, rtol=1e-6, atol=0)
+        outs.append((ratios, [p.clone() for p in params]))
+    assert outs[0][0] == outs[1][0]
+    for a, b in zip(outs[0][1], outs[1][1]):
+        assert torch.equal(a, b)
+
+
+def test_fullsize_resnet50_with_layer_adaptation():
+    wl = W.get_workload(1)
+    flat_p = W.alloc_flat(wl, torch.float32, DEV)
+    W.init_params(wl, flat_p)
+    params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
+    flat_g = W.alloc_flat(wl, torch.float32, DEV)
+    grads = [v.view(s) for v, s in zip(W.views(flat_g, wl), wl.shapes)]
+    src = W.GradSource(wl, DEV)
+    harness.MARGINS.clear()
+    pair = Pair(params, dict(wl.hyper, layer_adaptation=True))
+    for _ in range(12):
+        src.fill(flat_g)
+        pair.step(grads, threads=8)
+        np.testing.assert_allclose(pair.opt.trust_ratios(), pair.oracle.trust[-1], rtol=2e-6)
+    pair.check("resnet50 layer adaptation")
+    worst = max(harness.MARGINS.values())
+    print(f"\nPARITY resnet50 layer adaptation steps=12 every element worst |err|/tol: {worst:.3f}")
