@@ -42,6 +42,10 @@
  *     the step, u_t the base direction of Eq. 17 (before the classical blend),
  *     multiplying the step size of Eq. 24a; where ||u_t|| = 0 the ratio is
  *     undefined and taken as 1 (the update is zero there anyway).
+ *   - Sparse updates (Eq. 27): u <- u * 1{|u| > tau} on the base direction of
+ *     Eq. 17, before the classical blend (the order of Table 2, phase 8); the
+ *     trust ratio (phase 7) sees the unmasked direction.  tau = 0 switches the
+ *     mask off (Table 2: active when sparse_threshold > 0).
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
@@ -65,6 +69,7 @@ typedef struct {
     int32_t adaptive_beta;   /* 1: Eq. 3-4 warm-up of beta1, beta2 in Eq. 1-2 */
     double tau1;             /* warm-up time scale of beta1 (paper: 1000)   */
     double tau2;             /* warm-up time scale of beta2 (paper: 5000)   */
+    double sparse_threshold; /* tau of Eq. 27; 0 = no mask                  */
 } novak_oracle_hparams;
 
 typedef struct {
@@ -174,8 +179,10 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
         double m_hat = m[i] / s.bc1;
         double v_hat = v[i] / s.bc2;
 
-        /* Phase 8: Eq. 17, then Eq. 16 for the classical variant. */
+        /* Phase 8: Eq. 17, the mask of Eq. 27, then Eq. 16 for the classical variant. */
         double u = m_hat / (sqrt(v_hat) + h->eps);
+        if (h->sparse_threshold > 0.0 && !(fabs(u) > h->sparse_threshold))
+            u = 0.0;
         if (h->nesterov_variant == 2)
             u = h->beta1 * m_hat + (1.0 - h->beta1) * u;
 
@@ -252,5 +259,24 @@ void novak_oracle_centralize(int64_t rows, int64_t row_len, double *g)
         const double mean = sum / (double)row_len;
         for (int64_t j = 0; j < row_len; ++j)
             row[j] = row[j] - mean;
+    }
+}
+
+/* The base direction u_t of Eq. 17 that step t would produce for each of n
+ * elements (moments advanced in local variables; nothing is written).  Lets a
+ * test see how close |u| comes to the threshold of Eq. 27. */
+void novak_oracle_direction(const novak_oracle_hparams *h, int64_t t, int64_t n,
+                            const double *g, const double *m, const double *v,
+                            double *u_out)
+{
+    novak_oracle_scalars s;
+    novak_oracle_scalars_at(h, t, &s);
+    for (int64_t i = 0; i < n; ++i) {
+        double gt = g[i];
+        if (h->nesterov_variant == 1)
+            gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
+        const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
+        const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
+        u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);
     }
 }

@@ -44,6 +44,7 @@ class HParams(ctypes.Structure):
         ("adaptive_beta", ctypes.c_int32),
         ("tau1", ctypes.c_double),
         ("tau2", ctypes.c_double),
+        ("sparse_threshold", ctypes.c_double),
     ]
 
 
@@ -90,6 +91,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.novak_oracle_trust_ratio.argtypes = [
         ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64, dp, dp, dp, dp]
     lib.novak_oracle_trust_ratio.restype = ctypes.c_double
+    lib.novak_oracle_direction.argtypes = [
+        ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64, dp, dp, dp, dp]
+    lib.novak_oracle_direction.restype = None
     lib.novak_oracle_global_norm.argtypes = [
         ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(dp)]
     lib.novak_oracle_global_norm.restype = ctypes.c_double
@@ -135,6 +139,7 @@ class Config:
     adaptive_beta: bool = False          # Eq. 3-4
     tau1: float = 1000.0
     tau2: float = 5000.0
+    sparse_threshold: float = 0.0        # tau of Eq. 27; 0 = off
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -142,7 +147,8 @@ class Config:
                        self.weight_decay, nb, self.lookahead_alpha,
                        self.nesterov_variant, self.lookahead_k,
                        self.lookahead_mode, int(self.rectified),
-                       self.bias1_power, int(self.adaptive_beta), self.tau1, self.tau2)
+                       self.bias1_power, int(self.adaptive_beta), self.tau1, self.tau2,
+                       self.sparse_threshold)
 
 
 def _dptr(a: np.ndarray, offset: int = 0):
@@ -177,6 +183,8 @@ class Oracle:
                     if cfg.lookahead_k > 0 and cfg.lookahead_mode == LOOKAHEAD_TRAJ_MEAN
                     else None)
         self.t = 0
+        self.track_threshold_margin = False
+        self.threshold_margin = [np.full(p.size, np.inf) for p in self.theta]
         self.sync_steps: list[int] = []
         self.rect_flags: list[int] = []
 
@@ -233,6 +241,15 @@ class Oracle:
         for i, g in enumerate(gs):
             assert g.size == self.theta[i].size
         gs = self.process_gradients(gs)
+        if self.cfg.sparse_threshold > 0 and self.track_threshold_margin:
+            # how close |u| comes to tau, per element, over the whole run (for tests: a
+            # lower-precision implementation may decide Eq. 27 differently right at tau)
+            for i, g in enumerate(gs):
+                u = np.empty_like(g)
+                self.lib.novak_oracle_direction(ctypes.byref(self.h), self.t, g.size, _dptr(g),
+                                                _dptr(self.m[i]), _dptr(self.v[i]), _dptr(u))
+                rel = np.abs(np.abs(u) / self.cfg.sparse_threshold - 1.0)
+                self.threshold_margin[i] = np.minimum(self.threshold_margin[i], rel)
         trust = [1.0] * len(gs)
         if self.cfg.layer_adaptation:
             trust = [self.lib.novak_oracle_trust_ratio(

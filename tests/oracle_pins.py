@@ -656,6 +656,51 @@ def pin_trust_ratio(lib):
     _close(z.theta[0], th[1] * d, what="pure decay with u = 0")
 
 
+# --------------------------------------------------------------------------
+# Phase 8: sparse updates (Eq. 27)
+# --------------------------------------------------------------------------
+def pin_sparse_mask(lib):
+    """u <- u 1{|u| > tau}.  At t = 1 from zero moments (variant none) u = g/(|g|+eps), so
+    whether an element moves is known in closed form; masked elements only decay; the
+    classical blend still adds beta1 m_hat to a masked u; tau = 0 is the plain run."""
+    lr, wd, eps, tau = 1e-2, 0.1, 0.5, 0.4
+    g = np.array([1.0, 0.5, 0.35, -0.2, -2.0, 1e-3, 0.0])        # u = g/(|g|+0.5)
+    u = g / (np.abs(g) + eps)                                    # .667 .5 .412 -.286 -.8 .002 0
+    th = np.linspace(-1, 1, g.size)
+    d = 1 - lr * wd
+    kw = dict(lr=lr, weight_decay=wd, eps=eps, lookahead_k=0, rectified=False)
+    o = _mk(lib, [th], sparse_threshold=tau, nesterov_variant=O.NESTEROV_NONE, **kw)
+    o.step([g])
+    keep = np.abs(u) > tau
+    assert keep.tolist() == [True, True, True, False, True, False, False]   # |g| = .35 < tau < |u|
+    _close(o.theta[0], th * d - lr * np.where(keep, u, 0.0), what="masked step")
+    _close(o.m[0], 0.1 * g, what="moments ignore the mask")
+    # |u| == tau exactly is NOT kept (strict inequality): g = 2 eps/3... use tau = 0.5, g = 0.5
+    e = _mk(lib, [np.zeros(1)], sparse_threshold=0.5, nesterov_variant=O.NESTEROV_NONE, **kw)
+    e.step([np.array([0.5])])
+    assert e.theta[0][0] == 0.0
+    # classical: Eq. 16 blends the masked u with m_hat
+    b1 = 0.9
+    c = _mk(lib, [th], sparse_threshold=tau, nesterov_variant=O.NESTEROV_CLASSICAL, **kw)
+    c.step([g])
+    _close(c.theta[0], th * d - lr * (b1 * g + (1 - b1) * np.where(keep, u, 0.0)),
+           what="blend after the mask")
+    # tau = 0: off, identical to a run that never heard of the mask
+    rng = np.random.default_rng(2)
+    a = _mk(lib, [th], sparse_threshold=0.0, **kw)
+    b = _mk(lib, [th], **kw)
+    for _ in range(5):
+        G = rng.normal(0, 1, g.size)
+        a.step([G]); b.step([G])
+    assert np.array_equal(a.theta[0], b.theta[0])
+    # the trust ratio (phase 7) sees the unmasked direction
+    t1 = _mk(lib, [th], sparse_threshold=tau, layer_adaptation=True,
+             nesterov_variant=O.NESTEROV_NONE, **kw)
+    t0 = _mk(lib, [th], layer_adaptation=True, nesterov_variant=O.NESTEROV_NONE, **kw)
+    t1.step([g]); t0.step([g])
+    assert t1.trust[0][0] == t0.trust[0][0]
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -677,4 +722,5 @@ ALL_PINS = [
     pin_clip_then_centralize_then_step,
     pin_adaptive_beta,
     pin_trust_ratio,
+    pin_sparse_mask,
 ]

@@ -55,6 +55,13 @@ MUTANTS = [
     ("warmup_in_classical_blend", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
      "u = s.beta1_t * m_hat + (1.0 - s.beta1_t) * u;"),
     ("warmup_flag_ignored", "if (h->adaptive_beta) {", "if (1) {"),
+    # phase 8: sparse updates
+    ("mask_inverted", "!(fabs(u) > h->sparse_threshold))", "(fabs(u) > h->sparse_threshold))"),
+    ("mask_signed", "!(fabs(u) > h->sparse_threshold))", "!(u > h->sparse_threshold))"),
+    ("mask_not_strict", "!(fabs(u) > h->sparse_threshold))", "!(fabs(u) >= h->sparse_threshold))"),
+    ("mask_after_blend", "if (h->sparse_threshold > 0.0 && !(fabs(u) > h->sparse_threshold))\n            u = 0.0;\n        if (h->nesterov_variant == 2)\n            u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
+     "if (h->nesterov_variant == 2)\n            u = h->beta1 * m_hat + (1.0 - h->beta1) * u;\n        if (h->sparse_threshold > 0.0 && !(fabs(u) > h->sparse_threshold))\n            u = 0.0;"),
+    ("mask_on_gradient", "!(fabs(u) > h->sparse_threshold))", "!(fabs(gt) > h->sparse_threshold))"),
     # phase 7: layer-wise adaptation
     ("trust_inverted", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sqrt(sum_u) / sqrt(sum_theta);"),
     ("trust_of_squared_norms", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sum_theta / sum_u;"),
