@@ -104,11 +104,15 @@ enum {
                                      blend keep the base values.  0 (default)          */
     NOVAK_OPT_BETA1_TAU = 15,     /* tau_1 > 0 of Eq. 3 (default 1000)                 */
     NOVAK_OPT_BETA2_TAU = 16,     /* tau_2 > 0 of Eq. 4 (default 5000)                 */
-    NOVAK_OPT_LAYER_ADAPTATION = 17 /* 1: layer-wise adaptation (Eq. 19 / 25): each
+    NOVAK_OPT_LAYER_ADAPTATION = 17, /* 1: layer-wise adaptation (Eq. 19 / 25): each
                                      tensor's step is stretched by its trust ratio
                                      clip(||theta_t|| / ||u_t||, 0.1, 10).  Two more
                                      kernels per step read theta, g, m, v once more
                                      (+16 B per element).  0 (default)               */
+    NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base
+                                     directions with |u| <= tau are set to zero before
+                                     the classical blend; 0 (default): no mask.  The
+                                     comparison is made in fp32 on the kernel's u     */
 };
 
 /* Warning bits (novak_info.warnings). */
@@ -166,6 +170,7 @@ typedef struct novak_meta {
     double beta1_tau, beta2_tau;
     int32_t adaptive_beta;
     int32_t layer_adaptation;
+    double sparse_threshold;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".

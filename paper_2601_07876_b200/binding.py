@@ -28,7 +28,7 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
- NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION) = range(1, 18)
+ NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD) = range(1, 19)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -62,7 +62,7 @@ class novak_meta(Structure):
         ("rectified", c_int32), ("bias1_power", c_int32), ("n_tensors", c_int32),
         ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
         ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
-        ("layer_adaptation", c_int32),
+        ("layer_adaptation", c_int32), ("sparse_threshold", c_double),
     ]
 
 
@@ -309,7 +309,7 @@ class NovakOptimizer:
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
-                 layer_adaptation=False,
+                 layer_adaptation=False, sparse_threshold=0.0,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -361,6 +361,8 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_ADAPTIVE_BETA, 1)
         if layer_adaptation:
             h.set_option(NOVAK_OPT_LAYER_ADAPTATION, 1)
+        if sparse_threshold:
+            h.set_option(NOVAK_OPT_SPARSE_THRESHOLD, sparse_threshold)
         if clip_threshold:
             h.set_option(NOVAK_OPT_CLIP_THRESHOLD, clip_threshold)
         if centralize:

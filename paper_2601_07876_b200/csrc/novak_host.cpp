@@ -24,7 +24,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763034ull;  // "NOVAKv04"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763035ull;  // "NOVAKv05"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -38,6 +38,7 @@ struct Hyper {
     int layer_adapt;        // Eq. 19 / 25: one trust ratio per tensor
     int adaptive_beta;      // Eq. 3-4
     double tau1, tau2;      // warm-up time scales of beta1, beta2
+    double sparse_tau;      // tau of Eq. 27, 0: no mask
 };
 
 struct Plan {
@@ -541,6 +542,7 @@ int check_hyper(const Hyper &h, const char **why)
     if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
     if (!(h.clip >= 0.0) || !std::isfinite(h.clip)) { *why = "clip threshold must be >= 0"; return 0; }
     if (h.centralize != 0 && h.centralize != 1) { *why = "centralize must be 0 or 1"; return 0; }
+    if (!(h.sparse_tau >= 0.0) || !std::isfinite(h.sparse_tau)) { *why = "sparse threshold must be >= 0"; return 0; }
     if (h.layer_adapt != 0 && h.layer_adapt != 1) { *why = "layer_adaptation must be 0 or 1"; return 0; }
     if (h.adaptive_beta != 0 && h.adaptive_beta != 1) { *why = "adaptive_beta must be 0 or 1"; return 0; }
     if (!(h.tau1 > 0.0) || !std::isfinite(h.tau1) || !(h.tau2 > 0.0) || !std::isfinite(h.tau2)) { *why = "warm-up time scales must be > 0"; return 0; }
@@ -568,6 +570,7 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.clip = 0.0;
     h.centralize = 0;
     h.layer_adapt = 0;
+    h.sparse_tau = 0.0;
     h.adaptive_beta = 0;
     h.tau1 = 1000.0;       // Section 4.2's values
     h.tau2 = 5000.0;
@@ -617,6 +620,7 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
         h.bias1_power = static_cast<int>(value);
         break;
+    case NOVAK_OPT_SPARSE_THRESHOLD: h.sparse_tau = value; break;
     case NOVAK_OPT_LAYER_ADAPTATION:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "layer_adaptation must be 0 or 1");
         h.layer_adapt = static_cast<int>(value);
@@ -680,6 +684,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_LR: *value = o->h.lr; break;
     case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
     case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
+    case NOVAK_OPT_SPARSE_THRESHOLD: *value = o->h.sparse_tau; break;
     case NOVAK_OPT_LAYER_ADAPTATION: *value = o->h.layer_adapt; break;
     case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
     case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
@@ -775,6 +780,7 @@ StepScalars make_scalars(const Hyper &h, const Plan &p)
     s.step = static_cast<float>(p.step_size);
     s.la_alpha = static_cast<float>(h.la_alpha);
     s.k = static_cast<float>(h.la_k > 0 ? h.la_k : 1);
+    s.sparse_tau = h.sparse_tau > 0.0 ? static_cast<float>(h.sparse_tau) : -1.0f;
     return s;
 }
 
@@ -1283,6 +1289,7 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->centralize = o->h.centralize;
     out->adaptive_beta = o->h.adaptive_beta;
     out->layer_adaptation = o->h.layer_adapt;
+    out->sparse_threshold = o->h.sparse_tau;
     out->beta1_tau = o->h.tau1;
     out->beta2_tau = o->h.tau2;
     out->n_tensors = o->n;
@@ -1307,6 +1314,7 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.clip = in->clip_threshold;
     h.adaptive_beta = in->adaptive_beta;
     h.layer_adapt = in->layer_adaptation;
+    h.sparse_tau = in->sparse_threshold;
     h.tau1 = in->beta1_tau;
     h.tau2 = in->beta2_tau;
     if (h.centralize != in->centralize) invalidate_tables(o);

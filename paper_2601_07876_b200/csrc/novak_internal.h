@@ -40,6 +40,7 @@ struct StepScalars {
     float step;            // alpha r_t                     (Eq. 8-9, 24a)
     float la_alpha;        // alpha_LA                      (Eq. 30)
     float k;               // lookahead period as a float (divisor of the running sum)
+    float sparse_tau;      // Eq. 27: directions with |u| <= tau are dropped; -1 when off
 };
 
 // What the lookahead phase does on this step (bit mask; template parameter).

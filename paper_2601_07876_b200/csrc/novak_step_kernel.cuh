@@ -175,6 +175,9 @@ __device__ __forceinline__ void update_element(float &p, float g, float &m, floa
 {
     float m_hat;
     float u = base_direction<NEST>(g, m, v, m_hat, s);
+    // Eq. 27: u 1{|u| > tau}.  With the mask off tau is -1 and nothing, NaN
+    // included, compares below it.
+    u = (fabsf(u) <= s.sparse_tau) ? 0.0f : u;
     // Eq. 16 for the classical blend
     if constexpr (NEST == NOVAK_NESTEROV_CLASSICAL)
         u = fmaf(s.blend_b1, m_hat, s.blend_omb1 * u);

@@ -31,6 +31,7 @@ def oracle_config(hyper: dict) -> O.Config:
         rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1),
         clip_threshold=h.pop("clip_threshold", 0.0), centralize=h.pop("centralize", False),
         layer_adaptation=h.pop("layer_adaptation", False),
+        sparse_threshold=h.pop("sparse_threshold", 0.0),
         adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
         tau2=h.pop("tau2", None) or 5000.0)
 

@@ -288,3 +288,51 @@ def test_fullsize_resnet50_with_layer_adaptation():
     pair.check("resnet50 layer adaptation")
     worst = max(harness.MARGINS.values())
     print(f"\nPARITY resnet50 layer adaptation steps=12 every element worst |err|/tol: {worst:.3f}")
+
+
+# ---------------------------------------------------------------------------
+# Phase 8: sparse updates (Eq. 27)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("nesterov", ["approximation", "classical"])
+def test_sparse_mask(nesterov):
+    """u 1{|u| > tau} is a yes/no decision taken on an fp32 u here and on an fp64 u in
+    the oracle: an element whose |u| came within 1e-4 (relative) of tau at any step may
+    legitimately differ and is left out; every other element has to match as usual."""
+    numels = [70001, 33, 8192]
+    tau = 0.3
+    flat, views, _ = make_tensors(numels, DEV)
+    gen = _gen(81)
+    for p in views:
+        p.normal_(0.0, 0.05, generator=gen)
+    pair = Pair(views, dict(BASE, nesterov=nesterov, sparse_threshold=tau, lookahead_k=3))
+    pair.oracle.track_threshold_margin = True
+    _, grads, _ = make_tensors(numels, DEV)
+    for _ in range(9):
+        _fill_grads(grads, gen, std=1e-2)
+        pair.step(grads)
+    torch.cuda.synchronize()
+    o = pair.oracle
+    total = kept = 0
+    for i, p in enumerate(views):
+        sure = o.threshold_margin[i] > 1e-4
+        total += sure.size
+        kept += int(sure.sum())
+        st = pair.opt.state(i)
+        harness.assert_close(to_f64(p)[sure], o.theta[i][sure], f"sparse theta[{i}]")
+        harness.assert_close(to_f64(st["slow"])[sure], o.slow[i][sure], f"sparse slow[{i}]")
+        harness.assert_close(st["m"], o.m[i], f"sparse m[{i}]")      # moments ignore the mask
+        harness.assert_close(st["v"], o.v[i], f"sparse v[{i}]")
+    assert kept > 0.995 * total                      # only a handful of elements sit at tau
+    # the mask does bite: compare with the same run without it
+    flat2, views2, _ = make_tensors(numels, DEV)
+    gen = _gen(81)
+    for p in views2:
+        p.normal_(0.0, 0.05, generator=gen)
+    plain = B.NovakOptimizer(views2, **dict(BASE, nesterov=nesterov, lookahead_k=3))
+    for _ in range(9):
+        _fill_grads(grads, gen, std=1e-2)
+        plain.step(grads)
+    torch.cuda.synchronize()
+    assert not torch.allclose(views[0], views2[0], rtol=1e-4, atol=1e-7)
+    with pytest.raises(B.NovakError):
+        pair.opt.handle.set_option(B.NOVAK_OPT_SPARSE_THRESHOLD, -0.1)
