@@ -86,6 +86,8 @@ def parse_args():
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
+    ap.add_argument("--bf16-copy", action="store_true",
+                    help="the step also writes a bf16 copy of the parameters (+2 B per element)")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -102,7 +104,8 @@ def parse_args():
 
 
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
-                               phase2: bool = False, trust: bool = False) -> int:
+                               phase2: bool = False, trust: bool = False,
+                               copy16: bool = False) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
     arrays on the steps that touch them, plus one more read of g when clipping or
@@ -110,6 +113,8 @@ def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
     b = 12 + grad_bytes + 12 + (grad_bytes if phase2 else 0)
     if trust:
         b += 12 + grad_bytes             # theta, g, m, v read once more for the norms of Eq. 19
+    if copy16:
+        b += 2
     if k <= 0:
         return b
     sync = t % k == 0
@@ -320,6 +325,9 @@ def main():
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
     pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
+    if args.bf16_copy:
+        copy_flat = W.alloc_flat(wl, torch.bfloat16, dev)
+        opt.set_param_copies(W.views(copy_flat, wl))
 
     def barrier():
         if world > 1:
@@ -350,13 +358,13 @@ def main():
     ms_per_step = ms / args.steps
     value = world * wl.total * args.steps / (ms * 1e-3)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
-                                         args.layer_adaptation)
+                                         args.layer_adaptation, args.bf16_copy)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = None if (phase2 or args.layer_adaptation) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -436,7 +444,7 @@ def main():
                 "lookahead_k": k, "lookahead_mode": args.lookahead_mode,
                 "clip_threshold": args.clip, "centralize": bool(args.centralize),
                 "layer_adaptation": bool(args.layer_adaptation),
-                "adaptive_beta": bool(args.adaptive_beta),
+                "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
                       "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),

@@ -274,7 +274,7 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
  * elements at the default 2048 elements per entry; raise
  * NOVAK_OPT_CHUNK_ELEMS before the first step for larger groups).  Beyond that
  * the call returns NOVAK_EINVAL with the limit in novak_last_error() and does
- * nothing.  The array costs 2.25 MiB on every GPU that loads the library, until
+ * nothing.  The array costs 2.31 MiB on every GPU that loads the library, until
  * the process exits.
  *
  * The array is ONE per GPU and shared by every handle and every call.  It keeps
@@ -316,6 +316,21 @@ int novak_step_noalloc(novak_opt *opt, void *const *d_params,
  * chunk-table entries of at most 2048 elements (the default).
  * novak_step_noalloc refuses to run in this mode (NOVAK_ESTATE). */
 int novak_set_tensor_rows(novak_opt *opt, const int64_t *rows, int n);
+
+/* Mixed-precision training keeps fp32 master parameters in the optimizer and a
+ * bf16 copy for the forward and backward passes (the paper names reduced
+ * precision as future work, Section 10.3, without fixing a rule; this is the
+ * part of it that has an exact definition).  d_copies: host array of n device
+ * pointers to contiguous bf16 tensors of numel[i] elements, 2-byte aligned,
+ * caller-owned.  Every later step (novak_step, novak_step_host,
+ * novak_step_noalloc) stores, beside each updated fp32 parameter, its value
+ * rounded to nearest even in bf16 (+2 B per element written; no separate cast
+ * kernel).  Nothing reads the copies.  A copy whose address is not congruent to
+ * half its parameter's address modulo 8 puts the tensor on 4-byte accesses
+ * (NOVAK_WARN_SCALAR_PATH).  NULL switches the copies off.
+ * Errors: NOVAK_ESTATE (nothing attached), NOVAK_EINVAL (n mismatch, NULL or
+ * odd pointer). */
+int novak_set_param_copies(novak_opt *opt, void *const *d_copies, int n);
 
 /* Convergence monitoring (Section 5.8 tracks ||g_t||): the global gradient norm
  * and the clip factor of the last step that ran phase 2.  Copies 16 bytes from

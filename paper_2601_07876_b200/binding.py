@@ -107,6 +107,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_step_noalloc": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_set_tensor_rows": (c_int, [vp, i64p, c_int]),
+        "novak_set_param_copies": (c_int, [vp, vpp, c_int]),
         "novak_get_grad_stats": (c_int, [vp, POINTER(c_double), POINTER(c_double), vp]),
         "novak_get_trust_ratios": (c_int, [vp, POINTER(ctypes.c_float), c_int, vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
@@ -231,6 +232,12 @@ class Handle:
                self.lib.novak_set_tensor_rows(self.h, i64_array(rows), len(rows)),
                "novak_set_tensor_rows")
 
+    def set_param_copies(self, d_copies):
+        arr = ptr_array(d_copies) if d_copies is not None else None
+        n = len(d_copies) if d_copies is not None else 0
+        _check(self.lib, self.h, self.lib.novak_set_param_copies(self.h, arr, n),
+               "novak_set_param_copies")
+
     def get_grad_stats(self, stream: int = 0):
         """(global gradient norm, clip factor) of the last step; synchronises the stream."""
         norm, factor = c_double(), c_double()
@@ -309,7 +316,7 @@ class NovakOptimizer:
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
-                 layer_adaptation=False, sparse_threshold=0.0,
+                 layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -369,6 +376,28 @@ class NovakOptimizer:
             # Eq. 26 applies to tensors with more than one dimension
             h.set_tensor_rows([p.shape[0] if p.dim() > 1 else 0 for p in self.params])
             h.set_option(NOVAK_OPT_CENTRALIZE, 1)
+        self.param_copies = None
+        if param_copies is not None:
+            self.set_param_copies(param_copies)
+
+    def set_param_copies(self, copies):
+        """bf16 tensors (one per parameter) that every step fills with the updated
+        parameters rounded to nearest even; None switches them off."""
+        import torch
+        if copies is None:
+            self.handle.set_param_copies(None)
+            self.param_copies = None
+            return
+        copies = list(copies)
+        if len(copies) != self.n:
+            raise ValueError("one copy per parameter tensor")
+        for c, p in zip(copies, self.params):
+            if (c.dtype != torch.bfloat16 or not c.is_cuda or not c.is_contiguous()
+                    or c.numel() != p.numel()):
+                raise ValueError("copies must be contiguous bfloat16 CUDA tensors of the "
+                                 "parameters' sizes")
+        self.handle.set_param_copies([c.data_ptr() for c in copies])
+        self.param_copies = copies              # keeps the memory alive
 
     def trust_ratios(self):
         return self.handle.get_trust_ratios(self.n, self._stream())

@@ -147,6 +147,7 @@ struct novak_opt {
     std::vector<int32_t> phase;
     std::vector<int64_t> rows, row_off;   // dimension 0 of each tensor (0: none), prefix sums
     int64_t total_rows = 0;
+    std::vector<void *> copies;           // bf16 copies of the parameters the step also writes
 
     // counters
     int64_t t = 0, n_syncs = 0, last_sync = 0, launches = 0;
@@ -484,6 +485,10 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         const uintptr_t m = reinterpret_cast<uintptr_t>(slice(o, 0, i));
         if (((p ^ m) & 15u) || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
             scalar_path = true;
+        // the bf16 copy is stored 4 elements (8 bytes) at a time beside 16-byte parameters
+        if (!o->copies.empty() &&
+            ((p & 15u) >> 1) != (reinterpret_cast<uintptr_t>(o->copies[i]) & 7u))
+            scalar_path = true;
     }
     const int slot = o->ring_pos;
     cudaError_t e;
@@ -502,6 +507,7 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         const bool rows = o->h.centralize && o->row_mean && !o->rows.empty() && o->rows[i] > 0;
         h[i].mean = rows ? o->row_mean + o->row_off[i] : nullptr;
         h[i].row_len = rows ? static_cast<uint32_t>(o->numel[i] / o->rows[i]) : 0u;
+        h[i].p16 = o->copies.empty() ? nullptr : static_cast<__nv_bfloat16 *>(o->copies[i]);
         h[i].reserved = 0;
     }
     // Stream order puts this copy behind every earlier launch that read the
@@ -753,6 +759,7 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     o->rows.assign(n, 0);
     o->row_off.assign(n, 0);
     o->total_rows = 0;
+    o->copies.clear();
     o->t = 0; o->n_syncs = 0; o->last_sync = 0;
     o->attached = true;
     o->err.clear();
@@ -877,7 +884,7 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     if (o->ctas_per_sm > 0) cfg.grid = std::min(count, o->sms * o->ctas_per_sm);
     cfg.reverse = ctx.reverse;
     cfg.pdl = o->pdl;
-    cfg.pre = ctx.pre;
+    cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16);
     o->last_grid = cfg.grid;
     return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.trust, ctx.s,
                               o->h.nesterov, ctx.grad_dtype, ctx.la, cfg, stream);
@@ -1139,6 +1146,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
             r.slow = la ? slice(o, 2, i) : nullptr;
             r.acc = traj ? slice(o, 3, i) : nullptr;
             r.mean = nullptr;
+            r.p16 = o->copies.empty() ? nullptr : static_cast<__nv_bfloat16 *>(o->copies[i]);
             r.row_len = 0;
             r.reserved = 0;
         }
@@ -1182,7 +1190,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     cfg.grid = n_chunks;
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
-    cfg.pre = novak::PRE_NONE;
+    cfg.pre = novak::PRE_NONE | (o->copies.empty() ? 0 : novak::PRE_COPY16);
     e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, nullptr, s, o->h.nesterov, grad_dtype,
                            la_action, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
@@ -1216,6 +1224,26 @@ int novak_set_tensor_rows(novak_opt *o, const int64_t *rows, int n)
     for (int i = 0; i < n; ++i) { o->row_off[i] = off; off += o->rows[i]; }
     o->total_rows = total;
     invalidate_tables(o);
+    return NOVAK_OK;
+}
+
+int novak_set_param_copies(novak_opt *o, void *const *d_copies, int n)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "set_param_copies: attach the state first");
+    if (d_copies == nullptr) {
+        o->copies.clear();
+    } else {
+        if (n != o->n) return fail(o, NOVAK_EINVAL, "set_param_copies: wrong tensor count");
+        for (int i = 0; i < n; ++i) {
+            const uintptr_t c = reinterpret_cast<uintptr_t>(d_copies[i]);
+            if (!c || (c & 1u))
+                return fail(o, NOVAK_EINVAL, "set_param_copies: copy %d is NULL or not 2-byte aligned", i);
+        }
+        o->copies.assign(d_copies, d_copies + n);
+    }
+    invalidate_tables(o);
+    o->na_p.clear();              // the no-allocation path rebuilds its records too
     return NOVAK_OK;
 }
 

@@ -2,6 +2,7 @@
 // code (novak_*.cu) of the NOVAK step library.  Not part of the C ABI.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -16,6 +17,7 @@ struct __align__(16) TensorRec {
     float *slow;       // slow weights   (Eq. 28), NULL when lookahead is off
     float *acc;        // running sum of the window's fast iterates (TRAJ_MEAN)
     float2 *mean;      // row means of the raw gradient (Eq. 26) as hi + lo, NULL: not centralized
+    __nv_bfloat16 *p16; // bf16 copy of theta written by the step, NULL: none
     uint32_t row_len;  // elements per row (product of dimensions 1..d), 0: not centralized
     uint32_t reserved;
 };
@@ -60,7 +62,10 @@ enum : int {
 enum : int {
     PRE_NONE = 0,    // g as given
     PRE_SCALE = 1,   // g <- factor g, the clip factor read from device memory
-    PRE_CENTER = 2   // g <- factor (g - row mean) for tensors that have rows (Eq. 26)
+    PRE_CENTER = 2,  // g <- factor (g - row mean) for tensors that have rows (Eq. 26)
+    PRE_MASK = 3,
+    // OR-ed onto the above: the step also stores a bf16 copy of the new parameters
+    PRE_COPY16 = 4
 };
 
 // Result of the gradient statistics pass, in device memory; the step kernel
@@ -75,7 +80,7 @@ struct LaunchCfg {
     int grid;
     int reverse;     // walk the chunk table from the end
     int pdl;         // launch with programmatic stream serialization (bit 0)
-    int pre;         // PRE_*
+    int pre;         // PRE_* (with PRE_COPY16 where a bf16 copy is written)
 };
 
 // Threads per CTA of the step kernel (fixed at compile time).

@@ -15,6 +15,9 @@ namespace novak {
 void *step_kernel_pre0(int nesterov, int grad_dtype, int la);
 void *step_kernel_pre1(int nesterov, int grad_dtype, int la);
 void *step_kernel_pre2(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre0_copy(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre1_copy(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre2_copy(int nesterov, int grad_dtype, int la);
 
 namespace {
 
@@ -30,6 +33,9 @@ StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
     case PRE_NONE: fn = step_kernel_pre0(nesterov, grad_dtype, la); break;
     case PRE_SCALE: fn = step_kernel_pre1(nesterov, grad_dtype, la); break;
     case PRE_CENTER: fn = step_kernel_pre2(nesterov, grad_dtype, la); break;
+    case PRE_NONE | PRE_COPY16: fn = step_kernel_pre0_copy(nesterov, grad_dtype, la); break;
+    case PRE_SCALE | PRE_COPY16: fn = step_kernel_pre1_copy(nesterov, grad_dtype, la); break;
+    case PRE_CENTER | PRE_COPY16: fn = step_kernel_pre2_copy(nesterov, grad_dtype, la); break;
     default: break;
     }
     return reinterpret_cast<StepKernelFn>(fn);
@@ -39,7 +45,7 @@ StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
 
 // Work table of novak_step_noalloc: tensor records followed by the chunk table,
 // resident in every GPU that loads this library until the process exits
-// (256 KiB + 2 MiB).  In host code this name is only a handle for
+// (320 KiB + 2 MiB).  In host code this name is only a handle for
 // cudaGetSymbolAddress, never a device address.
 struct NoAllocTable {
     TensorRec recs[kNoAllocMaxTensors];
@@ -82,7 +88,7 @@ cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_
 {
     StepKernelFn fn = pick_kernel(nesterov, grad_dtype, la, cfg.pre);
     if (!fn || n_chunks <= 0 || cfg.grid <= 0) return cudaErrorInvalidValue;
-    if (cfg.pre != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
+    if ((cfg.pre & PRE_MASK) != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(cfg.grid));
     lc.blockDim = dim3(kBlock);

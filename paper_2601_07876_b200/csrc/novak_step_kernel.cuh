@@ -20,6 +20,8 @@
 
 #include "novak.h"
 
+#include <cuda_bf16.h>
+
 #ifndef NOVAK_BLOCK
 #define NOVAK_BLOCK 256
 #endif
@@ -78,6 +80,22 @@ __device__ __forceinline__ void store_f32<1>(float *base, int idx, const Vec<1> 
     __stcs(base + idx, x.a[0]);
 }
 
+// fp32 -> bf16, round to nearest even: the model copy of the updated parameters.
+template <int N>
+__device__ __forceinline__ void store_bf16(__nv_bfloat16 *base, int idx, const Vec<N> &x)
+{
+    if constexpr (N == 4) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(x.a[0], x.a[1]);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(x.a[2], x.a[3]);
+        uint2 t;
+        t.x = *reinterpret_cast<const unsigned *>(&lo);
+        t.y = *reinterpret_cast<const unsigned *>(&hi);
+        __stcs(reinterpret_cast<uint2 *>(base) + idx, t);
+    } else {
+        base[idx] = __float2bfloat16_rn(x.a[0]);
+    }
+}
+
 // bf16 -> fp32 is exact: the 16 bits are the upper half of the fp32 pattern.
 template <int N, int GT>
 __device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
@@ -102,6 +120,7 @@ __device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
 
 // ---- phase 2 before the Nesterov approximation: clip factor and centralization
 struct PreArgs {
+    __nv_bfloat16 *copy; // bf16 copy of the chunk's parameters (PRE_COPY16), else unused
     float step;          // alpha r_t, times the tensor's trust ratio under layer adaptation
     float factor;        // clip factor (1 when clipping is off or inactive)
     const float2 *mean;  // row means of the raw gradient (hi + lo), NULL: tensor not centralized
@@ -118,7 +137,7 @@ struct PreArgs {
 template <int N, int PRE>
 __device__ __forceinline__ void preprocess(Vec<N> &G, uint32_t e, const PreArgs &a)
 {
-    if constexpr (PRE == PRE_CENTER) {
+    if constexpr ((PRE & PRE_MASK) == PRE_CENTER) {
         if (a.mean != nullptr) {
             uint32_t row = e / a.row_len;
             uint32_t rem = e - row * a.row_len;
@@ -135,7 +154,7 @@ __device__ __forceinline__ void preprocess(Vec<N> &G, uint32_t e, const PreArgs 
             }
         }
     }
-    if constexpr (PRE != PRE_NONE) {
+    if constexpr ((PRE & PRE_MASK) != PRE_NONE) {
 #pragma unroll
         for (int j = 0; j < N; ++j) G.a[j] *= a.factor;
     }
@@ -233,6 +252,7 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
             update_element<NEST, LA>(P[j].a[e], G[j].a[e], M[j].a[e], V[j].a[e],
                                      S[j].a[e], A[j].a[e], s, pre.step);
         store_f32<N>(p, idx, P[j]);
+        if constexpr ((PRE & PRE_COPY16) != 0) store_bf16<N>(pre.copy, idx, P[j]);
         store_f32<N>(m, idx, M[j]);
         store_f32<N>(v, idx, V[j]);
         if constexpr (kWriteS) store_f32<N>(slow, idx, S[j]);
@@ -292,15 +312,16 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     // The clip factor is the statistics kernel's output: read it only now.
     PreArgs pre;
     pre.factor = 1.0f;
-    if constexpr (PRE != PRE_NONE) pre.factor = prep->factor;
+    if constexpr ((PRE & PRE_MASK) != PRE_NONE) pre.factor = prep->factor;
 
 #pragma unroll 1
     for (;;) {
         // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
         pre.step = trust != nullptr ? s.step * __ldg(trust + ch.tensor) : s.step;
-        pre.mean = (PRE == PRE_CENTER) ? r.mean : nullptr;
+        pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
+        pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
         float *p = r.p + ch.offset;
         float *m = r.m + ch.offset;
         float *v = r.v + ch.offset;
@@ -312,6 +333,8 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                          reinterpret_cast<uintptr_t>(v);
         if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
         if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
+        // the 64-bit stores of the bf16 copy need half the parameters' alignment
+        if ((PRE & PRE_COPY16) != 0) bits |= reinterpret_cast<uintptr_t>(pre.copy) << 1;
         const bool aligned = (bits & 15u) == 0 &&
                              (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
         if (aligned) {

@@ -1,0 +1,12 @@
+// Step kernel instantiations for centralized and scaled gradients, storing a bf16 copy of the
+// updated parameters beside the fp32 ones.
+#include "novak_step_kernel.cuh"
+
+namespace novak {
+
+void *step_kernel_pre2_copy(int nesterov, int grad_dtype, int la)
+{
+    return reinterpret_cast<void *>(pick_step_kernel<PRE_CENTER | PRE_COPY16>(nesterov, grad_dtype, la));
+}
+
+}  // namespace novak

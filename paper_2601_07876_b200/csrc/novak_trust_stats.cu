@@ -82,6 +82,7 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     grid_dependency_wait();              // parameters, moments, clip factor, row means
 
     PreArgs pre;
+    pre.copy = nullptr;
     pre.step = 0.0f;
     pre.factor = 1.0f;
     if constexpr (PRE != PRE_NONE) pre.factor = prep->factor;

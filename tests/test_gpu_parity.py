@@ -254,6 +254,46 @@ def test_adaptive_beta_warm_up(nesterov):
     assert opt.plan(1000)["beta1_t"] == pytest.approx(0.9 * (1 - np.exp(-1.0)), rel=1e-12)
 
 
+@pytest.mark.parametrize("copy_offsets", [None, [0, 1, 0, 2, 0, 3, 0, 0, 0, 0, 0, 0]])
+def test_bf16_parameter_copies_are_the_rounded_master(copy_offsets):
+    """The step also writes a bf16 copy of every updated parameter: the fp32 master matches
+    the oracle as always, the copy equals the master rounded to nearest even bit for bit
+    (torch's conversion as the independent check), and nothing is written beside it."""
+    offsets = [0, 1, 2, 3, 0, 0, 1, 0, 3, 0, 0, 2]
+    _, params, _ = _fresh(RAGGED, offsets=offsets, seed=91)
+    # copies share the parameters' alignment phase, or deliberately do not
+    cflat, copies, cstarts = make_tensors(RAGGED, DEV, copy_offsets or offsets,
+                                          dtype=torch.bfloat16, fill=7.0)
+    pair = Pair(params, dict(BASE, lookahead_k=2), opt_kwargs=dict(param_copies=copies))
+    gen = _gen(92)
+    for _ in range(5):
+        pair.step(_grads(RAGGED, gen, offsets=offsets))
+    pair.check("bf16 copies")
+    for p, c in zip(params, copies):
+        assert torch.equal(c, p.to(torch.bfloat16))
+    gaps = gaps_mask(cflat.numel(), cstarts, RAGGED, DEV)
+    assert bool((cflat[gaps] == 7.0).all())
+    scalar = bool(pair.opt.info()["warnings"] & B.NOVAK_WARN_SCALAR_PATH)
+    assert scalar == (copy_offsets is not None)
+    # the no-allocation entry point writes them too; NULL switches them off again
+    gl = pair.opt.prepare(_grads(RAGGED, gen, offsets=offsets))
+    pair.opt.handle.step_noalloc(pair.opt._params_arr, gl.arr, pair.opt._numel_arr, pair.opt.n,
+                                 gl.dtype, pair.opt._stream())
+    torch.cuda.synchronize()
+    for p, c in zip(params, copies):
+        assert torch.equal(c, p.to(torch.bfloat16))
+    pair.opt.set_param_copies(None)
+    before = [c.clone() for c in copies]
+    pair.opt.step(_grads(RAGGED, gen, offsets=offsets))
+    torch.cuda.synchronize()
+    for b, c in zip(before, copies):
+        assert torch.equal(b, c)
+    with pytest.raises(B.NovakError):
+        pair.opt.handle.set_param_copies([c.data_ptr() for c in copies[:-1]])
+    with pytest.raises(B.NovakError):
+        pair.opt.handle.set_param_copies([c.data_ptr() + 1 for c in copies])
+
+
 def test_gradient_pointers_may_change_every_step():
     numels = [9000, 100]
     _, params, _ = _fresh(numels, seed=41)
