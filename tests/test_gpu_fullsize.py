@@ -38,3 +38,47 @@ def test_fullsize_workload(index, mode):
     assert not misaligned, "every tensor should run on 128-bit accesses"
     del pair
     torch.cuda.empty_cache()
+
+
+def test_one_tensor_beyond_2_to_the_31_elements():
+    """Maximum sizes: element offsets past 2^31 (and chunk counts past 2^20) in one
+    tensor, with clipping on so that the statistics kernels cross the boundary too.
+    The oracle follows a sample: both ends, a window around element 2^31 and a comb."""
+    n = (1 << 31) + 4099                       # ragged: not a multiple of 4
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * (1 << 30):
+        pytest.skip("needs about 45 GiB of device memory")
+    from oracle import novak_oracle as O
+    from paper_2601_07876_b200 import binding as B
+    gen = torch.Generator(device=DEV).manual_seed(5)
+    p = torch.empty(n, dtype=torch.float32, device=DEV)
+    g = torch.empty(n, dtype=torch.float32, device=DEV)
+    blk = 1 << 28
+    for lo in range(0, n, blk):
+        p[lo:lo + blk].normal_(0.0, 0.05, generator=gen)
+    edge = 4096
+    idx = torch.cat([torch.arange(edge), torch.arange((1 << 31) - edge, (1 << 31) + edge),
+                     torch.arange(edge, n - edge, 1000003), torch.arange(n - edge, n)]).to(DEV)
+    hyper = dict(lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
+                 nesterov="approximation", lookahead_k=0, clip_threshold=1.0)
+    opt = B.NovakOptimizer([p], **hyper)
+    oracle = O.Oracle(harness.oracle_config(dict(hyper, clip_threshold=0.0)),
+                      [harness.to_f64(p[idx])])
+    for _ in range(3):
+        for lo in range(0, n, blk):
+            g[lo:lo + blk].normal_(0.0, 1e-3, generator=gen)
+        opt.step([g])
+        norm, factor = opt.grad_stats()
+        # the sample cannot know the global norm: take it from a plain float64 torch sum
+        want = float(sum(g[lo:lo + blk].double().square().sum() for lo in range(0, n, blk)) ** 0.5)
+        assert abs(norm - want) <= 1e-7 * want and want > 1.0
+        assert abs(factor - 1.0 / want) <= 1e-6 / want
+        oracle.step([harness.to_f64(g[idx]) * (1.0 / want)])
+    torch.cuda.synchronize()
+    info = opt.info()
+    assert info["total_numel"] == n and info["n_chunks"] == (n + 2047) // 2048
+    harness.assert_close(p[idx], oracle.theta[0], "2^31 theta")
+    harness.assert_close(opt.state(0)["m"][idx], oracle.m[0], "2^31 m")
+    harness.assert_close(opt.state(0)["v"][idx], oracle.v[0], "2^31 v")
+    del opt, p, g
+    torch.cuda.empty_cache()
