@@ -46,6 +46,14 @@
  *     Eq. 17, before the classical blend (the order of Table 2, phase 8); the
  *     trust ratio (phase 7) sees the unmasked direction.  tau = 0 switches the
  *     mask off (Table 2: active when sparse_threshold > 0).
+ *   - Automatic learning-rate scaling: Eq. 20-22 (two moving averages of the
+ *     global norms of gradient and parameters, gamma = 0.1, ratio clipped to
+ *     [0.1, 2]), the form Tables 2 and 3 describe (two norm computations, two
+ *     scalars of state).  Eq. 23, which Eq. 24a cites, is a different and
+ *     incompatible definition (one average, a pole at EMA = 1/e) and is not
+ *     used.  ||g_t|| is the norm of the gradient as given (the norm clipping
+ *     uses), ||theta_t|| that of the parameters before the step, both over
+ *     every tensor of the group; the averages start at 0.   [parity unpinned]
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
@@ -279,4 +287,24 @@ void novak_oracle_direction(const novak_oracle_hparams *h, int64_t t, int64_t n,
         const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
         u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);
     }
+}
+
+/* ------------------------------------------------------------------------
+ * Phase 7, automatic learning-rate scaling (Eq. 20-22).
+ * ---------------------------------------------------------------------- */
+
+/* Advances the two moving averages (Eq. 20, 21) with this step's global norms
+ * and returns alpha_auto = clip(g_bar / theta_bar, 0.1, 2) (Eq. 22).  The ratio
+ * of two zero averages is undefined and taken as 1. */
+double novak_oracle_auto_lr(double gamma, double grad_norm, double param_norm,
+                            double *g_bar, double *theta_bar)
+{
+    *g_bar = gamma * grad_norm + (1.0 - gamma) * *g_bar;
+    *theta_bar = gamma * param_norm + (1.0 - gamma) * *theta_bar;
+    if (*g_bar == 0.0 && *theta_bar == 0.0)
+        return 1.0;
+    double a = *g_bar / *theta_bar;
+    if (a < 0.1) a = 0.1;
+    if (a > 2.0) a = 2.0;
+    return a;
 }

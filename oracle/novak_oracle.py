@@ -94,6 +94,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.novak_oracle_direction.argtypes = [
         ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64, dp, dp, dp, dp]
     lib.novak_oracle_direction.restype = None
+    lib.novak_oracle_auto_lr.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                         dp, dp]
+    lib.novak_oracle_auto_lr.restype = ctypes.c_double
     lib.novak_oracle_global_norm.argtypes = [
         ctypes.c_int32, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(dp)]
     lib.novak_oracle_global_norm.restype = ctypes.c_double
@@ -140,6 +143,8 @@ class Config:
     tau1: float = 1000.0
     tau2: float = 5000.0
     sparse_threshold: float = 0.0        # tau of Eq. 27; 0 = off
+    auto_lr: bool = False                # Eq. 20-22
+    auto_lr_gamma: float = 0.1
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -170,6 +175,9 @@ class Oracle:
         self.cfg = cfg
         self.rows = list(rows) if rows is not None else None
         self.trust: list[list[float]] = []   # per step, per tensor (layer adaptation)
+        self.g_bar = ctypes.c_double(0.0)    # Eq. 20
+        self.theta_bar = ctypes.c_double(0.0)  # Eq. 21
+        self.auto_scales: list[float] = []
         self.grad_norms: list[float] = []
         self.clip_factors: list[float] = []
         self.h = cfg.to_c()
@@ -201,6 +209,12 @@ class Oracle:
             _dptr(self.m[i], lo), _dptr(self.v[i], lo),
             _dptr(self.slow[i], lo) if self.slow is not None else null,
             _dptr(self.acc[i], lo) if self.acc is not None else null, trust)
+
+    def _global_norm(self, arrays) -> float:
+        n = len(arrays)
+        numel = (ctypes.c_int64 * n)(*[a.size for a in arrays])
+        ptrs = (ctypes.POINTER(ctypes.c_double) * n)(*[_dptr(a) for a in arrays])
+        return self.lib.novak_oracle_global_norm(n, numel, ptrs)
 
     def process_gradients(self, gs):
         """Phase 2 before the Nesterov approximation: clipping on the global norm
@@ -240,6 +254,12 @@ class Oracle:
               for g in grads]
         for i, g in enumerate(gs):
             assert g.size == self.theta[i].size
+        auto = 1.0
+        if self.cfg.auto_lr:
+            auto = self.lib.novak_oracle_auto_lr(
+                self.cfg.auto_lr_gamma, self._global_norm(gs), self._global_norm(self.theta),
+                ctypes.byref(self.g_bar), ctypes.byref(self.theta_bar))
+            self.auto_scales.append(auto)
         gs = self.process_gradients(gs)
         if self.cfg.sparse_threshold > 0 and self.track_threshold_margin:
             # how close |u| comes to tau, per element, over the whole run (for tests: a
@@ -256,6 +276,7 @@ class Oracle:
                 ctypes.byref(self.h), self.t, g.size, _dptr(self.theta[i]), _dptr(g),
                 _dptr(self.m[i]), _dptr(self.v[i])) for i, g in enumerate(gs)]
             self.trust.append(trust)
+        trust = [x * auto for x in trust]    # Eq. 24a: both multiply the step size
         if threads <= 1:
             for i, g in enumerate(gs):
                 self._run(i, g, 0, g.size, trust[i])

@@ -701,6 +701,60 @@ def pin_sparse_mask(lib):
     assert t1.trust[0][0] == t0.trust[0][0]
 
 
+# --------------------------------------------------------------------------
+# Phase 7: automatic learning-rate scaling (Eq. 20-22)
+# --------------------------------------------------------------------------
+def pin_auto_lr(lib):
+    """The averages as explicit sums of numpy norms, the clipped ratio, and the adapted
+    step as the plain (pinned) step stretched by it; raw-gradient norm even when the
+    gradient is clipped afterwards; both clip bounds; one scale for every tensor."""
+    rng = np.random.default_rng(41)
+    lr, wd, gam = 1e-2, 0.1, 0.1
+    kw = dict(lr=lr, weight_decay=wd, lookahead_k=0, nesterov_variant=O.NESTEROV_APPROX)
+    th = [rng.normal(0, 0.3, 40), rng.normal(0, 0.5, 7)]
+    d = 1 - lr * wd
+    plain = _mk(lib, th, **kw)
+    auto = _mk(lib, th, auto_lr=True, clip_threshold=0.5, **kw)
+    plain.cfg.clip_threshold = 0.5
+    gn, pn = [], []
+    for t in range(1, 8):
+        G = [rng.normal(0, 0.1 * t, x.size) for x in th]
+        for i in range(2):
+            plain.theta[i][:] = auto.theta[i]
+            plain.m[i][:] = auto.m[i]
+            plain.v[i][:] = auto.v[i]
+        before = [x.copy() for x in auto.theta]
+        plain.t = auto.t
+        gn.append(np.linalg.norm(np.concatenate(G)))
+        pn.append(np.linalg.norm(np.concatenate(before)))
+        plain.step(G)
+        auto.step(G)
+        g_bar = sum(gam * (1 - gam) ** (t - i) * gn[i - 1] for i in range(1, t + 1))
+        p_bar = sum(gam * (1 - gam) ** (t - i) * pn[i - 1] for i in range(1, t + 1))
+        want = min(max(g_bar / p_bar, 0.1), 2.0)
+        _close(auto.g_bar.value, g_bar, what="Eq. 20")
+        _close(auto.theta_bar.value, p_bar, what="Eq. 21")
+        _close(auto.auto_scales[-1], want, what="Eq. 22")
+        for i in range(2):
+            _close(auto.theta[i] - before[i] * d, want * (plain.theta[i] - before[i] * d),
+                   rtol=1e-9, atol=1e-15, what="step stretched by alpha_auto")
+    seen = np.array(auto.auto_scales)
+    assert seen.min() > 0.1 and seen.max() < 2.0 and seen.max() > 1.5 * seen.min()
+    assert max(gn) > 0.5                       # the clipping was active: raw norm in Eq. 20
+    for scale, want in ((1e-3, 0.1), (1e3, 2.0)):
+        o = _mk(lib, [np.ones(10)], auto_lr=True, **kw)
+        o.step([np.full(10, scale)])
+        assert o.auto_scales[0] == want
+    # with layer adaptation both factors multiply the step (Eq. 24a)
+    both = _mk(lib, th, auto_lr=True, layer_adaptation=True, **kw)
+    only = _mk(lib, th, layer_adaptation=True, **kw)
+    G = [rng.normal(0, 0.3, x.size) for x in th]
+    both.step(G); only.step(G)
+    for i in range(2):
+        _close(both.theta[i] - th[i] * d, both.auto_scales[0] * (only.theta[i] - th[i] * d),
+               rtol=1e-9, atol=1e-15, what="alpha_auto times lambda_trust")
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -723,4 +777,5 @@ ALL_PINS = [
     pin_adaptive_beta,
     pin_trust_ratio,
     pin_sparse_mask,
+    pin_auto_lr,
 ]

@@ -55,6 +55,14 @@ MUTANTS = [
     ("warmup_in_classical_blend", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
      "u = s.beta1_t * m_hat + (1.0 - s.beta1_t) * u;"),
     ("warmup_flag_ignored", "if (h->adaptive_beta) {", "if (1) {"),
+    # phase 7: automatic learning-rate scaling
+    ("auto_inverted", "double a = *g_bar / *theta_bar;", "double a = *theta_bar / *g_bar;"),
+    ("auto_gamma_swapped", "*g_bar = gamma * grad_norm + (1.0 - gamma) * *g_bar;",
+     "*g_bar = (1.0 - gamma) * grad_norm + gamma * *g_bar;"),
+    ("auto_theta_not_averaged", "*theta_bar = gamma * param_norm + (1.0 - gamma) * *theta_bar;",
+     "*theta_bar = param_norm;"),
+    ("auto_upper_bound_10", "if (a > 2.0) a = 2.0;", "if (a > 10.0) a = 10.0;"),
+    ("auto_lower_clip_missing", "if (a < 0.1) a = 0.1;", ";"),
     # phase 8: sparse updates
     ("mask_inverted", "!(fabs(u) > h->sparse_threshold))", "(fabs(u) > h->sparse_threshold))"),
     ("mask_signed", "!(fabs(u) > h->sparse_threshold))", "!(u > h->sparse_threshold))"),
