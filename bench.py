@@ -86,6 +86,8 @@ def parse_args():
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
+    ap.add_argument("--auto-lr", action="store_true",
+                    help="Eq. 20-22: statistics pass plus one more read of the parameters")
     ap.add_argument("--bf16-copy", action="store_true",
                     help="the step also writes a bf16 copy of the parameters (+2 B per element)")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
@@ -105,7 +107,7 @@ def parse_args():
 
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
                                phase2: bool = False, trust: bool = False,
-                               copy16: bool = False) -> int:
+                               copy16: bool = False, auto: bool = False) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
     arrays on the steps that touch them, plus one more read of g when clipping or
@@ -115,6 +117,8 @@ def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
         b += 12 + grad_bytes             # theta, g, m, v read once more for the norms of Eq. 19
     if copy16:
         b += 2
+    if auto:
+        b += 4                           # ||theta_t|| of Eq. 21
     if k <= 0:
         return b
     sync = t % k == 0
@@ -311,7 +315,7 @@ def main():
     flat_p = W.alloc_flat(wl, torch.float32, dev)
     W.init_params(wl, flat_p)
     params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
-    phase2 = args.clip > 0 or args.centralize
+    phase2 = args.clip > 0 or args.centralize or args.auto_lr
     pool_n = max(1, min(args.pool, int(8e9 // (wl.total * gbytes)) or 1))
     src = W.GradSource(wl, dev, seed_offset=rank)
     scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
@@ -321,6 +325,7 @@ def main():
     del scratch
     opt = B.NovakOptimizer(params, **hyper, clip_threshold=args.clip, centralize=args.centralize,
                            layer_adaptation=args.layer_adaptation, adaptive_beta=args.adaptive_beta,
+                           auto_lr=args.auto_lr,
                            chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
@@ -358,7 +363,7 @@ def main():
     ms_per_step = ms / args.steps
     value = world * wl.total * args.steps / (ms * 1e-3)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
-                                         args.layer_adaptation, args.bf16_copy)
+                                         args.layer_adaptation, args.bf16_copy, args.auto_lr)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
@@ -445,6 +450,7 @@ def main():
                 "clip_threshold": args.clip, "centralize": bool(args.centralize),
                 "layer_adaptation": bool(args.layer_adaptation),
                 "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
+                "auto_lr": bool(args.auto_lr),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
                       "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),

@@ -109,6 +109,14 @@ enum {
                                      clip(||theta_t|| / ||u_t||, 0.1, 10).  Two more
                                      kernels per step read theta, g, m, v once more
                                      (+16 B per element).  0 (default)               */
+    NOVAK_OPT_AUTO_LR = 19,       /* 1: automatic learning-rate scaling (Eq. 20-22): the
+                                     step is stretched by clip(g_bar / theta_bar, 0.1,
+                                     2), moving averages of the global norms of the
+                                     gradient as given and of the parameters before
+                                     the step.  Runs the statistics pass and reads
+                                     the parameters once more (+4 B per element on top
+                                     of clipping's +4).  0 (default)                  */
+    NOVAK_OPT_AUTO_LR_GAMMA = 20, /* gamma in (0, 1] of Eq. 20-21 (default 0.1)        */
     NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base
                                      directions with |u| <= tau are set to zero before
                                      the classical blend; 0 (default): no mask.  The
@@ -171,6 +179,9 @@ typedef struct novak_meta {
     int32_t adaptive_beta;
     int32_t layer_adaptation;
     double sparse_threshold;
+    double auto_lr_gamma;
+    int32_t auto_lr;
+    int32_t reserved;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
@@ -345,6 +356,17 @@ int novak_get_grad_stats(novak_opt *opt, double *norm, double *factor, void *str
  * direction (Eq. 17); 1 where ||u_t|| = 0.  Copies n floats from the device and
  * SYNCHRONISES `stream`.  NOVAK_ESTATE when no such step has run. */
 int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
+
+/* Automatic learning-rate scaling (Eq. 20-22, NOVAK_OPT_AUTO_LR).  Its two
+ * moving averages live in device memory.  get: copies them and the last step's
+ * factor (Eq. 22) to the host and SYNCHRONISES `stream` (before the first such
+ * step: the initial zeros, or what set put in; any output may be NULL).  set:
+ * for resuming from a checkpoint; the values are written to the device in
+ * stream order at the next step.  NOVAK_EINVAL for negative or non-finite
+ * values. */
+int novak_get_auto_lr_state(novak_opt *opt, double *g_bar, double *theta_bar, double *scale,
+                            void *stream);
+int novak_set_auto_lr_state(novak_opt *opt, double g_bar, double theta_bar);
 
 /* Counters and the last step's scalars (bit-exact step and sync indices). */
 int novak_get_info(const novak_opt *opt, novak_info *out);

@@ -28,7 +28,8 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_BIAS1_POWER, NOVAK_OPT_CHUNK_ELEMS, NOVAK_OPT_CTAS_PER_SM, NOVAK_OPT_SERPENTINE,
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
- NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD) = range(1, 19)
+ NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
+ NOVAK_OPT_AUTO_LR_GAMMA) = range(1, 21)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -63,6 +64,7 @@ class novak_meta(Structure):
         ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
         ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
         ("layer_adaptation", c_int32), ("sparse_threshold", c_double),
+        ("auto_lr_gamma", c_double), ("auto_lr", c_int32), ("reserved", c_int32),
     ]
 
 
@@ -109,6 +111,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_set_tensor_rows": (c_int, [vp, i64p, c_int]),
         "novak_set_param_copies": (c_int, [vp, vpp, c_int]),
         "novak_get_grad_stats": (c_int, [vp, POINTER(c_double), POINTER(c_double), vp]),
+        "novak_get_auto_lr_state": (c_int, [vp, POINTER(c_double), POINTER(c_double),
+                                            POINTER(c_double), vp]),
+        "novak_set_auto_lr_state": (c_int, [vp, c_double, c_double]),
         "novak_get_trust_ratios": (c_int, [vp, POINTER(ctypes.c_float), c_int, vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
         "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
@@ -246,6 +251,18 @@ class Handle:
                "novak_get_grad_stats")
         return norm.value, factor.value
 
+    def get_auto_lr_state(self, stream: int = 0):
+        """(g_bar, theta_bar, last factor) of Eq. 20-22; synchronises the stream."""
+        a, b, c = c_double(), c_double(), c_double()
+        _check(self.lib, self.h,
+               self.lib.novak_get_auto_lr_state(self.h, byref(a), byref(b), byref(c), stream),
+               "novak_get_auto_lr_state")
+        return a.value, b.value, c.value
+
+    def set_auto_lr_state(self, g_bar: float, theta_bar: float):
+        _check(self.lib, self.h, self.lib.novak_set_auto_lr_state(self.h, g_bar, theta_bar),
+               "novak_set_auto_lr_state")
+
     def get_trust_ratios(self, n: int, stream: int = 0):
         """Per-tensor trust ratios of the last step; synchronises the stream."""
         out = (ctypes.c_float * n)()
@@ -317,6 +334,7 @@ class NovakOptimizer:
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
+                 auto_lr=False, auto_lr_gamma=None,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -370,6 +388,10 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_LAYER_ADAPTATION, 1)
         if sparse_threshold:
             h.set_option(NOVAK_OPT_SPARSE_THRESHOLD, sparse_threshold)
+        if auto_lr_gamma is not None:
+            h.set_option(NOVAK_OPT_AUTO_LR_GAMMA, auto_lr_gamma)
+        if auto_lr:
+            h.set_option(NOVAK_OPT_AUTO_LR, 1)
         if clip_threshold:
             h.set_option(NOVAK_OPT_CLIP_THRESHOLD, clip_threshold)
         if centralize:
@@ -442,17 +464,21 @@ class NovakOptimizer:
                 "acc": self._view(a, n)}
 
     def state_dict(self) -> dict:
-        """Layout-independent checkpoint: counters + per-tensor copies of the state."""
+        """Layout-independent checkpoint: counters + per-tensor copies of the state
+        (+ the two averages of the automatic learning-rate scaling)."""
         meta = self.handle.export_meta()
         tensors = []
         for i in range(self.n):
             tensors.append({k: (t.clone() if t is not None else None)
                             for k, t in self.state(i).items()})
-        return {"meta": bytes(meta), "tensors": tensors}
+        g_bar, theta_bar, _ = self.handle.get_auto_lr_state(self._stream())
+        return {"meta": bytes(meta), "tensors": tensors, "auto_lr": (g_bar, theta_bar)}
 
     def load_state_dict(self, sd: dict):
         meta = novak_meta.from_buffer_copy(sd["meta"])
         self.handle.import_meta(meta)
+        if "auto_lr" in sd:
+            self.handle.set_auto_lr_state(*sd["auto_lr"])
         for i, saved in enumerate(sd["tensors"]):
             for k, dst in self.state(i).items():
                 if dst is not None:

@@ -313,6 +313,47 @@ novak_grad_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
 }
 
+// Sum of squares of the parameters (for ||theta_t|| of Eq. 21): one CTA per 4
+// chunk-table entries, one sum per CTA filed under its first entry.  Launched
+// only when the automatic learning-rate scaling is on.
+__global__ void __launch_bounds__(kStatsBlock)
+novak_param_sumsq_kernel(const Chunk *__restrict__ chunks, int n_chunks,
+                         const TensorRec *__restrict__ recs, double *__restrict__ chunk_psq)
+{
+    __shared__ double sh[kStatsWarps];
+    constexpr int K = kStatsEntries;
+    grid_dependency_release();
+    const int c0 = blockIdx.x * K;
+    Chunk ch[K];
+    const float *p[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) ch[k] = chunks[min(c0 + k, n_chunks - 1)];
+#pragma unroll
+    for (int k = 0; k < K; ++k) p[k] = recs[ch[k].tensor].p + ch[k].offset;
+    grid_dependency_wait();          // the parameters come from the previous step
+    double sq = 0.0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (c0 + k >= n_chunks) break;
+        const uint32_t len = static_cast<uint32_t>(ch[k].len);
+        const bool aligned = (reinterpret_cast<uintptr_t>(p[k]) & 15u) == 0;
+        const uint32_t nvec = (len + 3u) >> 2;
+        for (uint32_t v = threadIdx.x; v < nvec; v += kStatsBlock) {
+            float x[4];
+            const uint32_t i = v << 2;
+            load_quad<NOVAK_GRAD_F32>(p[k], aligned, i, len - i < 4u ? len - i : 4u, x);
+            sq = sum_squares(x, sq);
+        }
+    }
+    const double total = block_sum(sq, sh);
+    if (threadIdx.x == 0) {
+        chunk_psq[c0] = total;
+#pragma unroll
+        for (int k = 1; k < K; ++k)
+            if (c0 + k < n_chunks) chunk_psq[c0 + k] = 0.0;
+    }
+}
+
 // Second kernel of the pass, one THREAD per chunk-table entry: puts together the
 // rows that entry boundaries cut (the thread of the entry in which such a row
 // BEGINS adds the pieces in entry order; the table lists a tensor's entries
@@ -323,7 +364,8 @@ template <bool ROWS>
 __global__ void __launch_bounds__(kStatsBlock)
 novak_grad_stats_finish_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                                const TensorRec *__restrict__ recs, double c_clip,
-                               const double *__restrict__ chunk_sq,
+                               double auto_gamma, const double *__restrict__ chunk_sq,
+                               const double *__restrict__ chunk_psq,
                                const double *__restrict__ seg_first,
                                const double *__restrict__ seg_last,
                                double *__restrict__ cta_sq, PrepOut *__restrict__ out)
@@ -334,9 +376,10 @@ novak_grad_stats_finish_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     grid_dependency_release();
     grid_dependency_wait();          // everything below is the first kernel's output
     const int i = blockIdx.x * kStatsBlock + threadIdx.x;
-    double sq = 0.0;
+    double sq = 0.0, psq = 0.0;
     if (i < n_chunks) {
         sq = chunk_sq[i];
+        if (chunk_psq != nullptr) psq = chunk_psq[i];
         if constexpr (ROWS) {
             const Chunk ci = chunks[i];
             const TensorRec ri = recs[ci.tensor];
@@ -362,9 +405,11 @@ novak_grad_stats_finish_kernel(const Chunk *__restrict__ chunks, int n_chunks,
         }
     }
     const double total = block_sum(sq, sh);
+    const double ptotal = chunk_psq != nullptr ? block_sum(psq, sh) : 0.0;
     if (threadIdx.x == 0) {
         cta_sq[blockIdx.x] = total;
-        __threadfence();             // this CTA's sum before its ticket
+        if (chunk_psq != nullptr) cta_sq[gridDim.x + blockIdx.x] = ptotal;
+        __threadfence();             // this CTA's sums before its ticket
         // wraps to 0 after the last CTA, ready for the next launch
         const unsigned ticket = atomicInc(&out->ticket, static_cast<unsigned>(gridDim.x) - 1u);
         sh_last = (ticket == static_cast<unsigned>(gridDim.x) - 1u) ? 1u : 0u;
@@ -374,15 +419,36 @@ novak_grad_stats_finish_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 
     // ---- the CTA that finished last: every CTA's sum is complete
     __threadfence();
-    double t = 0.0;
-    for (unsigned b = threadIdx.x; b < gridDim.x; b += kStatsBlock) t += __ldcg(cta_sq + b);
+    double t = 0.0, tp = 0.0;
+    for (unsigned b = threadIdx.x; b < gridDim.x; b += kStatsBlock) {
+        t += __ldcg(cta_sq + b);
+        if (chunk_psq != nullptr) tp += __ldcg(cta_sq + gridDim.x + b);
+    }
     const double sumsq = block_sum(t, sh);
+    const double psumsq = chunk_psq != nullptr ? block_sum(tp, sh) : 0.0;
     if (threadIdx.x == 0) {
         const double norm = sqrt(sumsq);
         // Table 2: clipping is active when ||g|| > c_clip
         const double factor = (c_clip > 0.0 && norm > c_clip) ? c_clip / norm : 1.0;
         out->norm = norm;
         out->factor = static_cast<float>(factor);
+        float scale = 1.0f;
+        if (chunk_psq != nullptr && auto_gamma > 0.0) {
+            // Eq. 20-22 on the norm of the gradient as given and of theta_t
+            const double pnorm = sqrt(psumsq);
+            const double g_bar = auto_gamma * norm + (1.0 - auto_gamma) * out->g_bar;
+            const double theta_bar = auto_gamma * pnorm + (1.0 - auto_gamma) * out->theta_bar;
+            double a = 1.0;              // 0/0: undefined, taken as 1
+            if (!(g_bar == 0.0 && theta_bar == 0.0)) {
+                a = g_bar / theta_bar;
+                a = a < 0.1 ? 0.1 : (a > 2.0 ? 2.0 : a);
+            }
+            out->pnorm = pnorm;
+            out->g_bar = g_bar;
+            out->theta_bar = theta_bar;
+            scale = static_cast<float>(a);
+        }
+        out->auto_scale = scale;
     }
 }
 
@@ -410,10 +476,12 @@ cudaError_t launch_pdl(const void *fn, unsigned grid, void **args, bool pdl, cud
 int grad_stats_ctas(int n_chunks) { return (n_chunks + kStatsBlock - 1) / kStatsBlock; }
 
 cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                              int grad_dtype, double c_clip, double *chunk_sq,
-                              double *seg_first, double *seg_last, double *cta_sq,
-                              PrepOut *prep, bool any_rows, int pdl, cudaStream_t stream)
+                              int grad_dtype, double c_clip, double auto_gamma, double *chunk_sq,
+                              double *chunk_psq, double *seg_first, double *seg_last,
+                              double *cta_sq, PrepOut *prep, bool any_rows, int pdl,
+                              cudaStream_t stream)
 {
+    if (auto_gamma > 0.0 && !chunk_psq) return cudaErrorInvalidValue;
     if (n_chunks <= 0 || !d_chunks || !d_recs || !chunk_sq || !cta_sq || !prep)
         return cudaErrorInvalidValue;
     if (any_rows && (!seg_first || !seg_last)) return cudaErrorInvalidValue;
@@ -436,8 +504,18 @@ cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorR
     const unsigned grid1 = static_cast<unsigned>((n_chunks + per_cta - 1) / per_cta);
     cudaError_t e = launch_pdl(first, grid1, args1, (pdl & 2) != 0, stream);
     if (e != cudaSuccess) return e;
+    const double *c_psq = nullptr;
+    if (auto_gamma > 0.0) {
+        void *args_p[] = {&d_chunks, &n_chunks, &d_recs, &chunk_psq};
+        const unsigned grid_p = static_cast<unsigned>((n_chunks + kStatsEntries - 1) / kStatsEntries);
+        e = launch_pdl(reinterpret_cast<const void *>(novak_param_sumsq_kernel), grid_p, args_p,
+                       (pdl & 2) != 0, stream);
+        if (e != cudaSuccess) return e;
+        c_psq = chunk_psq;
+    }
     const double *c_sq = chunk_sq, *c_first = seg_first, *c_last = seg_last;
-    void *args2[] = {&d_chunks, &n_chunks, &d_recs, &c_clip, &c_sq, &c_first, &c_last, &cta_sq, &prep};
+    void *args2[] = {&d_chunks, &n_chunks, &d_recs, &c_clip, &auto_gamma, &c_sq, &c_psq,
+                     &c_first, &c_last, &cta_sq, &prep};
     return launch_pdl(second, static_cast<unsigned>(grad_stats_ctas(n_chunks)), args2, (pdl & 4) != 0, stream);
 }
 

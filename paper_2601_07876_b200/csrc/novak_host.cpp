@@ -24,7 +24,7 @@ namespace {
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763035ull;  // "NOVAKv05"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763036ull;  // "NOVAKv06"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -39,6 +39,8 @@ struct Hyper {
     int adaptive_beta;      // Eq. 3-4
     double tau1, tau2;      // warm-up time scales of beta1, beta2
     double sparse_tau;      // tau of Eq. 27, 0: no mask
+    int auto_lr;            // Eq. 20-22
+    double auto_gamma;      // gamma of Eq. 20-21
 };
 
 struct Plan {
@@ -184,6 +186,10 @@ struct novak_opt {
     int64_t prep_rows = -1;             // total_rows the scratch was sized for
     PrepOut *prep_out = nullptr;
     double *chunk_sq = nullptr, *seg_first = nullptr, *seg_last = nullptr, *cta_sq = nullptr;
+    double *chunk_psq = nullptr;
+    // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
+    bool ema_pending = false;
+    double pending_g_bar = 0.0, pending_theta_bar = 0.0;
     float2 *row_mean = nullptr;
 
     // Scratch of layer adaptation (one allocation): two sums of squares per
@@ -253,7 +259,7 @@ float *slice(const novak_opt *o, int array, int i)
 int pre_mode(const novak_opt *o)
 {
     if (o->h.centralize && o->total_rows > 0) return novak::PRE_CENTER;
-    if (o->h.clip > 0.0) return novak::PRE_SCALE;
+    if (o->h.clip > 0.0 || o->h.auto_lr) return novak::PRE_SCALE;
     return novak::PRE_NONE;
 }
 
@@ -303,7 +309,7 @@ void release_device(novak_opt *o)
     o->d_prep = nullptr;
     o->prep_rows = -1;
     o->prep_out = nullptr;
-    o->chunk_sq = o->seg_first = o->seg_last = o->cta_sq = nullptr;
+    o->chunk_sq = o->seg_first = o->seg_last = o->cta_sq = o->chunk_psq = nullptr;
     o->row_mean = nullptr;
     for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
     o->host_ev.clear();
@@ -386,16 +392,26 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
     if (o->d_prep && o->prep_rows == o->total_rows) return NOVAK_OK;
     cudaError_t e;
     if (o->d_prep) {
-        cudaFree(o->d_prep);           // waits for the device; sizes changed
+        // sizes changed: keep the averages of Eq. 20-21 (the copy waits for the device)
+        if (!o->ema_pending) {
+            PrepOut old;
+            if ((e = cudaMemcpy(&old, o->prep_out, sizeof old, cudaMemcpyDeviceToHost)) != cudaSuccess)
+                return fail_cuda(o, e, "cudaMemcpy(gradient statistics)");
+            o->pending_g_bar = old.g_bar;
+            o->pending_theta_bar = old.theta_bar;
+            o->ema_pending = true;
+        }
+        cudaFree(o->d_prep);
         o->d_prep = nullptr;
         invalidate_tables(o);
     }
     const size_t nc = static_cast<size_t>(o->n_chunks);
     const size_t off_sq = 256;
-    const size_t off_first = off_sq + nc * sizeof(double);
+    const size_t off_psq = off_sq + nc * sizeof(double);
+    const size_t off_first = off_psq + nc * sizeof(double);
     const size_t off_last = off_first + nc * sizeof(double);
     const size_t off_cta = off_last + nc * sizeof(double);
-    const size_t off_mean = off_cta + static_cast<size_t>(novak::grad_stats_ctas(o->n_chunks)) * sizeof(double);
+    const size_t off_mean = off_cta + 2 * static_cast<size_t>(novak::grad_stats_ctas(o->n_chunks)) * sizeof(double);
     const size_t bytes = off_mean + static_cast<size_t>(o->total_rows) * sizeof(float2) + 16;
     if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
         o->d_prep = nullptr;
@@ -405,6 +421,7 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
         return fail_cuda(o, e, "cudaMemsetAsync(gradient statistics)");
     o->prep_out = reinterpret_cast<PrepOut *>(o->d_prep);
     o->chunk_sq = reinterpret_cast<double *>(o->d_prep + off_sq);
+    o->chunk_psq = reinterpret_cast<double *>(o->d_prep + off_psq);
     o->seg_first = reinterpret_cast<double *>(o->d_prep + off_first);
     o->seg_last = reinterpret_cast<double *>(o->d_prep + off_last);
     o->cta_sq = reinterpret_cast<double *>(o->d_prep + off_cta);
@@ -548,6 +565,8 @@ int check_hyper(const Hyper &h, const char **why)
     if (h.bias1_power != 1 && h.bias1_power != 2) { *why = "bias1_power must be 1 or 2"; return 0; }
     if (!(h.clip >= 0.0) || !std::isfinite(h.clip)) { *why = "clip threshold must be >= 0"; return 0; }
     if (h.centralize != 0 && h.centralize != 1) { *why = "centralize must be 0 or 1"; return 0; }
+    if (h.auto_lr != 0 && h.auto_lr != 1) { *why = "auto_lr must be 0 or 1"; return 0; }
+    if (!(h.auto_gamma > 0.0 && h.auto_gamma <= 1.0)) { *why = "auto_lr gamma must be in (0, 1]"; return 0; }
     if (!(h.sparse_tau >= 0.0) || !std::isfinite(h.sparse_tau)) { *why = "sparse threshold must be >= 0"; return 0; }
     if (h.layer_adapt != 0 && h.layer_adapt != 1) { *why = "layer_adaptation must be 0 or 1"; return 0; }
     if (h.adaptive_beta != 0 && h.adaptive_beta != 1) { *why = "adaptive_beta must be 0 or 1"; return 0; }
@@ -577,6 +596,8 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.centralize = 0;
     h.layer_adapt = 0;
     h.sparse_tau = 0.0;
+    h.auto_lr = 0;
+    h.auto_gamma = 0.1;    // Section 4.6
     h.adaptive_beta = 0;
     h.tau1 = 1000.0;       // Section 4.2's values
     h.tau2 = 5000.0;
@@ -627,6 +648,11 @@ int novak_set_option(novak_opt *o, int key, double value)
         h.bias1_power = static_cast<int>(value);
         break;
     case NOVAK_OPT_SPARSE_THRESHOLD: h.sparse_tau = value; break;
+    case NOVAK_OPT_AUTO_LR:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "auto_lr must be 0 or 1");
+        h.auto_lr = static_cast<int>(value);
+        break;
+    case NOVAK_OPT_AUTO_LR_GAMMA: h.auto_gamma = value; break;
     case NOVAK_OPT_LAYER_ADAPTATION:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "layer_adaptation must be 0 or 1");
         h.layer_adapt = static_cast<int>(value);
@@ -691,6 +717,8 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_WEIGHT_DECAY: *value = o->h.wd; break;
     case NOVAK_OPT_BIAS1_POWER: *value = o->h.bias1_power; break;
     case NOVAK_OPT_SPARSE_THRESHOLD: *value = o->h.sparse_tau; break;
+    case NOVAK_OPT_AUTO_LR: *value = o->h.auto_lr; break;
+    case NOVAK_OPT_AUTO_LR_GAMMA: *value = o->h.auto_gamma; break;
     case NOVAK_OPT_LAYER_ADAPTATION: *value = o->h.layer_adapt; break;
     case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
     case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
@@ -760,6 +788,7 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     o->row_off.assign(n, 0);
     o->total_rows = 0;
     o->copies.clear();
+    o->ema_pending = false;
     o->t = 0; o->n_syncs = 0; o->last_sync = 0;
     o->attached = true;
     o->err.clear();
@@ -827,6 +856,13 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
         return fail(o, NOVAK_ESTATE, "centralization needs chunk-table entries of at most 2048 "
                     "elements (NOVAK_OPT_CHUNK_ELEMS is %lld)", static_cast<long long>(o->chunk_elems));
     if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
+    if (o->ema_pending && o->prep_out) {
+        // averages set by the caller (or saved over a reallocation) go into the scratch
+        const double ema[2] = {o->pending_g_bar, o->pending_theta_bar};
+        cudaError_t e = cudaMemcpyAsync(&o->prep_out->g_bar, ema, sizeof ema, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return fail_cuda(o, e, "upload of the auto-LR averages");
+        o->ema_pending = false;
+    }
     if (o->h.layer_adapt && (rc = prepare_trust(o, stream)) != NOVAK_OK) return rc;
     ctx->trust = o->h.layer_adapt ? o->trust : nullptr;
     if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
@@ -854,7 +890,7 @@ cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stre
     if (ctx.pre != novak::PRE_NONE) {
         *what = "gradient statistics kernel launch";
         if ((e = launch_stats(o, ctx, stream)) != cudaSuccess) return e;
-        *launches += 2;
+        *launches += o->h.auto_lr ? 3 : 2;
     }
     if (ctx.trust) {
         *what = "layer adaptation kernel launch";
@@ -871,7 +907,8 @@ cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stre
 cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream)
 {
     return novak::launch_grad_stats(o->d_chunks, o->n_chunks, ctx.d_recs, ctx.grad_dtype,
-                                    o->h.clip, o->chunk_sq, o->seg_first, o->seg_last,
+                                    o->h.clip, o->h.auto_lr ? o->h.auto_gamma : 0.0, o->chunk_sq,
+                                    o->chunk_psq, o->seg_first, o->seg_last,
                                     o->cta_sq, o->prep_out, ctx.pre == novak::PRE_CENTER, o->pdl, stream);
 }
 
@@ -1262,6 +1299,40 @@ int novak_get_grad_stats(novak_opt *o, double *norm, double *factor, void *strea
     return NOVAK_OK;
 }
 
+int novak_get_auto_lr_state(novak_opt *o, double *g_bar, double *theta_bar, double *scale,
+                            void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (o->ema_pending || !o->prep_out) {
+        // nothing on the device yet: what a resume put in, or the initial zeros
+        if (g_bar) *g_bar = o->ema_pending ? o->pending_g_bar : 0.0;
+        if (theta_bar) *theta_bar = o->ema_pending ? o->pending_theta_bar : 0.0;
+        if (scale) *scale = 1.0;
+        return NOVAK_OK;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    PrepOut h;
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(&h, o->prep_out, sizeof h, cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "get_auto_lr_state");
+    if (g_bar) *g_bar = h.g_bar;
+    if (theta_bar) *theta_bar = h.theta_bar;
+    if (scale) *scale = static_cast<double>(h.auto_scale);
+    return NOVAK_OK;
+}
+
+int novak_set_auto_lr_state(novak_opt *o, double g_bar, double theta_bar)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!(g_bar >= 0.0) || !(theta_bar >= 0.0) || !std::isfinite(g_bar) || !std::isfinite(theta_bar))
+        return fail(o, NOVAK_EINVAL, "set_auto_lr_state: averages of norms are finite and >= 0");
+    o->pending_g_bar = g_bar;
+    o->pending_theta_bar = theta_bar;
+    o->ema_pending = true;
+    return NOVAK_OK;
+}
+
 int novak_get_trust_ratios(novak_opt *o, float *h_out, int n, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
@@ -1318,6 +1389,8 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->adaptive_beta = o->h.adaptive_beta;
     out->layer_adaptation = o->h.layer_adapt;
     out->sparse_threshold = o->h.sparse_tau;
+    out->auto_lr = o->h.auto_lr;
+    out->auto_lr_gamma = o->h.auto_gamma;
     out->beta1_tau = o->h.tau1;
     out->beta2_tau = o->h.tau2;
     out->n_tensors = o->n;
@@ -1343,6 +1416,8 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.adaptive_beta = in->adaptive_beta;
     h.layer_adapt = in->layer_adaptation;
     h.sparse_tau = in->sparse_threshold;
+    h.auto_lr = in->auto_lr;
+    h.auto_gamma = in->auto_lr_gamma;
     h.tau1 = in->beta1_tau;
     h.tau2 = in->beta2_tau;
     if (h.centralize != in->centralize) invalidate_tables(o);

@@ -74,6 +74,12 @@ struct __align__(16) PrepOut {
     double norm;       // global L2 norm of the raw gradient
     float factor;      // clip factor: c_clip/norm when norm > c_clip, else 1
     unsigned ticket;   // CTAs of the statistics kernel that have finished
+    // automatic learning-rate scaling (Eq. 20-22); the two averages persist from step to step
+    double pnorm;      // global L2 norm of the parameters before the step
+    double g_bar;      // Eq. 20
+    double theta_bar;  // Eq. 21
+    float auto_scale;  // Eq. 22, 1 when the scaling is off
+    float reserved;
 };
 
 struct LaunchCfg {
@@ -115,11 +121,16 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
 // and, where a tensor record has rows, the row means of Eq. 26.  Scratch:
 // chunk_sq, seg_first, seg_last of n_chunks doubles each (seg_* may be NULL
 // when no tensor has rows) and cta_sq of grad_stats_ctas(n_chunks) doubles.
+// With auto_gamma > 0 a third kernel sums the squares of the parameters into
+// chunk_psq (n_chunks doubles; cta_sq then holds 2 x grad_stats_ctas doubles)
+// and the pass also advances the averages of Eq. 20-21 in *prep and writes
+// Eq. 22's factor there; with auto_gamma = 0 that factor is written as 1.
 int grad_stats_ctas(int n_chunks);
 cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                              int grad_dtype, double c_clip, double *chunk_sq,
-                              double *seg_first, double *seg_last, double *cta_sq,
-                              PrepOut *prep, bool any_rows, int pdl, cudaStream_t stream);
+                              int grad_dtype, double c_clip, double auto_gamma, double *chunk_sq,
+                              double *chunk_psq, double *seg_first, double *seg_last,
+                              double *cta_sq, PrepOut *prep, bool any_rows, int pdl,
+                              cudaStream_t stream);
 
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.

@@ -312,12 +312,16 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     // The clip factor is the statistics kernel's output: read it only now.
     PreArgs pre;
     pre.factor = 1.0f;
-    if constexpr ((PRE & PRE_MASK) != PRE_NONE) pre.factor = prep->factor;
+    float step = s.step;
+    if constexpr ((PRE & PRE_MASK) != PRE_NONE) {
+        pre.factor = prep->factor;
+        step *= prep->auto_scale;        // Eq. 22 (1 when the scaling is off), Eq. 24a
+    }
 
 #pragma unroll 1
     for (;;) {
         // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
-        pre.step = trust != nullptr ? s.step * __ldg(trust + ch.tensor) : s.step;
+        pre.step = trust != nullptr ? step * __ldg(trust + ch.tensor) : step;
         pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);

@@ -32,6 +32,7 @@ def oracle_config(hyper: dict) -> O.Config:
         clip_threshold=h.pop("clip_threshold", 0.0), centralize=h.pop("centralize", False),
         layer_adaptation=h.pop("layer_adaptation", False),
         sparse_threshold=h.pop("sparse_threshold", 0.0),
+        auto_lr=h.pop("auto_lr", False), auto_lr_gamma=h.pop("auto_lr_gamma", None) or 0.1,
         adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
         tau2=h.pop("tau2", None) or 5000.0)
 

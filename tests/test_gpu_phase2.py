@@ -336,3 +336,83 @@ def test_sparse_mask(nesterov):
     assert not torch.allclose(views[0], views2[0], rtol=1e-4, atol=1e-7)
     with pytest.raises(B.NovakError):
         pair.opt.handle.set_option(B.NOVAK_OPT_SPARSE_THRESHOLD, -0.1)
+
+
+# ---------------------------------------------------------------------------
+# Phase 7: automatic learning-rate scaling (Eq. 20-22)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("extra", [dict(), dict(clip_threshold=0.05, centralize=True,
+                                                layer_adaptation=True, adaptive_beta=True,
+                                                tau1=5.0, tau2=20.0)])
+def test_auto_lr_every_element(gdtype, extra):
+    _, params = _shaped(SHAPES, OFFSETS)
+    gen = _gen(101)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    pair = Pair(params, dict(BASE, auto_lr=True, **extra))
+    _, grads = _shaped(SHAPES, OFFSETS, dtype=gdtype)
+    for t in range(8):
+        # the gradient scale sweeps the ratio through its clip range
+        _fill_grads(grads, gen, std=10.0 ** (-4 + 0.7 * t), mean=1e-4)
+        pair.step(grads)
+        g_bar, theta_bar, scale = pair.opt.handle.get_auto_lr_state(pair.opt._stream())
+        o = pair.oracle
+        assert abs(g_bar - o.g_bar.value) <= 1e-7 * o.g_bar.value
+        assert abs(theta_bar - o.theta_bar.value) <= 1e-6 * o.theta_bar.value
+        assert abs(scale - o.auto_scales[-1]) <= 2e-6 * o.auto_scales[-1]
+    pair.check(f"auto lr {extra}")
+    seen = pair.oracle.auto_scales
+    assert min(seen) == 0.1 and max(seen) == 2.0 and any(0.1 < s < 2.0 for s in seen)
+    per_step = 1 + 3 + (2 if extra.get("layer_adaptation") else 0)
+    assert pair.opt.info()["launches"] == 8 * per_step
+
+
+def test_auto_lr_state_survives_a_checkpoint_and_a_change_of_rows():
+    shapes = [(12, 300), (50,), (4, 2, 9)]
+
+    def fresh():
+        _, params = _shaped(shapes, [0, 0, 0])
+        g = _gen(7)
+        for p in params:
+            p.normal_(0.0, 0.05, generator=g)
+        return params
+
+    def grads_for(step):
+        _, grads = _shaped(shapes, [0, 0, 0])
+        _fill_grads(grads, _gen(1000 + step), std=1e-2 * (1 + step))
+        return grads
+
+    a_params = fresh()
+    a = B.NovakOptimizer(a_params, **BASE, auto_lr=True, clip_threshold=0.5)
+    for s in range(6):
+        if s == 4:      # centralization switched on mid-run re-sizes the scratch: averages kept
+            a.handle.set_tensor_rows(harness.tensor_rows(a_params))
+            a.handle.set_option(B.NOVAK_OPT_CENTRALIZE, 1)
+        a.step(grads_for(s))
+    b_params = fresh()
+    b = B.NovakOptimizer(b_params, **BASE, auto_lr=True, clip_threshold=0.5)
+    for s in range(3):
+        b.step(grads_for(s))
+    sd = b.state_dict()
+    saved = [p.clone() for p in b_params]
+    assert sd["auto_lr"][0] > 0 and sd["auto_lr"][1] > 0
+    c_params = fresh()
+    for p, q in zip(c_params, saved):
+        p.copy_(q)
+    c = B.NovakOptimizer(c_params, **BASE, auto_lr=True, clip_threshold=0.5)
+    c.load_state_dict(sd)
+    assert c.handle.get_auto_lr_state()[:2] == sd["auto_lr"]
+    for s in range(3, 6):
+        if s == 4:
+            c.handle.set_tensor_rows(harness.tensor_rows(c_params))
+            c.handle.set_option(B.NOVAK_OPT_CENTRALIZE, 1)
+        c.step(grads_for(s))
+    torch.cuda.synchronize()
+    for x, y in zip(a_params, c_params):
+        assert torch.equal(x, y)
+    assert a.handle.get_auto_lr_state() == c.handle.get_auto_lr_state()
+    with pytest.raises(B.NovakError):
+        c.handle.set_auto_lr_state(-1.0, 0.0)
+    with pytest.raises(B.NovakError):
+        c.handle.set_option(B.NOVAK_OPT_AUTO_LR_GAMMA, 0.0)
