@@ -86,6 +86,9 @@ def parse_args():
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
+    ap.add_argument("--zero1", action="store_true",
+                    help="one group sharded over the ranks (reduce-scatter, step on the owned "
+                         "range, all-gather) instead of one replica per rank: strong scaling")
     ap.add_argument("--auto-lr", action="store_true",
                     help="Eq. 20-22: statistics pass plus one more read of the parameters")
     ap.add_argument("--bf16-copy", action="store_true",
@@ -285,6 +288,72 @@ def cpu_baseline(wl, hyper, seconds):
                       f"({dt:.1f} s), threads over disjoint element ranges"}
 
 
+def run_zero1(args, rank, world, local):
+    """ZeRO-1: the group's optimizer state is split over the ranks; every step
+    reduce-scatters the gradients, steps the owned range and all-gathers the
+    parameters (NCCL).  Total work is fixed as N grows."""
+    import torch
+    import torch.distributed as dist
+    from paper_2601_07876_b200 import workloads as W
+    from paper_2601_07876_b200 import zero1
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    wl = W.get_workload(args.config)
+    if wl.grad_dtype != torch.float32:
+        raise SystemExit("--zero1 reduces fp32 gradients: pick an fp32 workload")
+    n = zero1.padded_numel(wl.total, world)
+    gen = torch.Generator(device=dev).manual_seed(W.MASTER_SEED)      # same parameters everywhere
+    flat_p = torch.zeros(n, device=dev)
+    flat_p[:wl.total].normal_(0.0, 0.05, generator=gen)
+    gen_g = torch.Generator(device=dev).manual_seed(W.MASTER_SEED + 1 + rank)
+    pool = []
+    for _ in range(max(1, min(args.pool, int(8e9 // (4 * n)) or 1))):
+        g = torch.zeros(n, device=dev)
+        g[:wl.total].normal_(0.0, 1e-2, generator=gen_g)
+        pool.append(g)
+    opt = zero1.ShardedNovak(flat_p, wl.numel, **wl.hyper)
+    scratch = torch.empty_like(pool[0])
+
+    def one(i):
+        scratch.copy_(pool[i % len(pool)])        # the reduce-scatter may overwrite its input
+        opt.step(scratch)
+
+    for i in range(max(3, args.warmup)):
+        one(i)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        ev0.record()
+        for i in range(args.steps):
+            one(i)
+        ev1.record()
+        dist.barrier()
+        torch.cuda.synchronize()
+    t = torch.tensor([ev0.elapsed_time(ev1)], device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    if rank == 0:
+        info = opt.local.info() if opt.local is not None else {}
+        print(json.dumps({
+            "metric": METRIC, "value": wl.total * args.steps / (ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
+                       "parallelism": f"zero1 x{world}: reduce-scatter(grad, avg) -> novak_step on "
+                                      f"the owned 1/{world} -> all-gather(params); the timed step "
+                                      "includes one device copy of the gradient buffer",
+                       "owned_elements_rank0": opt.hi - opt.lo},
+            "gpu_launches": info.get("launches"), "clocks": clocks.summary(),
+        }))
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -292,6 +361,9 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.zero1:
+        run_zero1(args, rank, world, local)
         return
 
     import torch

@@ -1,0 +1,110 @@
+"""ZeRO-1 style sharding of one parameter group over the ranks of a process group.
+
+Every rank holds the whole flat parameter buffer (for forward / backward) but
+only 1/world of the optimizer state.  One step:
+
+    reduce-scatter(gradients, average)  ->  NOVAK step on the owned range
+                                        ->  all-gather(parameters)
+
+The NOVAK step has no cross-element term, so the owned range may cut tensors
+anywhere; nothing is exchanged inside the step itself, and the ranks only have
+to take the same number of steps for their lookahead synchronisations to
+coincide.  Options that need a statistic of the WHOLE group (clipping,
+centralization, layer adaptation, automatic learning-rate scaling) would need
+an extra all-reduce between their statistics pass and the step; that is not
+built, and this class refuses them.
+
+Only argument marshalling and collectives live here: the local step is
+whatever ``make_local`` returns (the CUDA optimizer on a GPU; the tests plug in
+the CPU oracle to exercise the collectives under gloo).
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+from . import sharding
+
+ALIGN = 64      # elements: 256 bytes of fp32, so every rank's range starts 16-byte aligned
+
+
+def padded_numel(total: int, world: int) -> int:
+    """Length of the flat buffers: the next multiple of world x ALIGN elements."""
+    unit = world * ALIGN
+    return -(-total // unit) * unit
+
+
+class ShardedNovak:
+    """``flat_params``: one contiguous fp32 buffer of ``padded_numel(sum(numel), world)``
+    elements holding the group's tensors back to back (tensor i at the sum of the
+    earlier ``numel``); identical on every rank.  ``make_local(pieces)`` builds the
+    local optimizer over this rank's pieces (views into ``flat_params``) and must
+    return an object with ``step(list_of_gradient_views)``."""
+
+    def __init__(self, flat_params: torch.Tensor, numel, make_local=None, group=None,
+                 **hyper):
+        self.group = group
+        self.world = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+        self.numel = [int(n) for n in numel]
+        self.total = sum(self.numel)
+        if flat_params.dim() != 1 or flat_params.numel() != padded_numel(self.total, self.world):
+            raise ValueError("flat_params must be a 1-d buffer of padded_numel(total, world) elements")
+        for key in ("clip_threshold", "centralize", "layer_adaptation", "auto_lr"):
+            if hyper.get(key):
+                raise ValueError(f"{key} needs a statistic of the whole group: not available sharded")
+        self.flat_params = flat_params
+        self.shard = flat_params.numel() // self.world
+        lo = self.rank * self.shard
+        self.lo, self.hi = lo, min(lo + self.shard, self.total)   # owned elements (padding excluded)
+        self.slices = self._owned_slices()
+        self.param_shard = flat_params[lo:lo + self.shard]
+        self.grad_shard = torch.zeros_like(self.param_shard)
+        pieces = [self.param_shard[a - lo:b - lo] for a, b in self._flat_ranges()]
+        if make_local is None:
+            from .binding import NovakOptimizer
+            make_local = lambda ps: NovakOptimizer(ps, **hyper) if ps else None
+        self.local = make_local(pieces)
+        self.steps = 0
+
+    def _flat_ranges(self):
+        """Owned ranges of the flat space, one per tensor piece."""
+        out, base = [], 0
+        for n in self.numel:
+            a, b = max(base, self.lo), min(base + n, self.hi)
+            if a < b:
+                out.append((a, b))
+            base += n
+        return out
+
+    def _owned_slices(self):
+        """(tensor, start, stop) of every owned piece, as sharding.partition_flat gives them."""
+        out, base = [], 0
+        for t, n in enumerate(self.numel):
+            a, b = max(base, self.lo), min(base + n, self.hi)
+            if a < b:
+                out.append((t, a - base, b - base))
+            base += n
+        return out
+
+    def step(self, flat_grads: torch.Tensor):
+        """``flat_grads``: this rank's gradient of the whole group, laid out like
+        ``flat_params`` (padding ignored).  After the call ``flat_params`` holds the
+        updated parameters of the whole group on every rank."""
+        if flat_grads.shape != self.flat_params.shape:
+            raise ValueError("flat_grads must have the layout of flat_params")
+        backend = dist.get_backend(self.group)
+        if backend == "gloo":
+            # gloo has no reduce-scatter: all-reduce, then keep the owned range
+            dist.all_reduce(flat_grads, op=dist.ReduceOp.SUM, group=self.group)
+            self.grad_shard.copy_(flat_grads[self.rank * self.shard:(self.rank + 1) * self.shard])
+            self.grad_shard.div_(self.world)
+        else:
+            dist.reduce_scatter_tensor(self.grad_shard, flat_grads, op=dist.ReduceOp.AVG,
+                                       group=self.group)
+        if self.local is not None:
+            lo = self.lo
+            self.local.step([self.grad_shard[a - lo:b - lo] for a, b in self._flat_ranges()])
+        self.steps += 1
+        # every rank's updated range lands in every rank's own buffer
+        dist.all_gather_into_tensor(self.flat_params, self.param_shard, group=self.group)

@@ -423,3 +423,42 @@ def test_step_host_matches_step_and_returns_parameters(segment_elems, gdtype):
         assert launches == 1
     else:
         assert 2 <= launches <= 32
+
+
+def test_zero1_wrapper_drives_the_cuda_step_world_1():
+    """One rank over NCCL: reduce-scatter and all-gather degenerate to copies, the local
+    CUDA step runs on views of the flat buffer and matches the oracle; options that need
+    a statistic of the whole group are refused."""
+    import os
+    import socket
+    import torch.distributed as dist
+    from harness import oracle_config
+    from oracle import novak_oracle as O
+    from paper_2601_07876_b200 import zero1
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(DEV))
+    try:
+        numel = [5000, 33, 9000, 64]
+        total = sum(numel)
+        n = zero1.padded_numel(total, 1)
+        gen = _gen(111)
+        flat_p = torch.zeros(n, device=DEV)
+        flat_p[:total].normal_(0.0, 0.05, generator=gen)
+        oracle = O.Oracle(oracle_config(dict(BASE)), [to_f64(flat_p[:total])])
+        opt = zero1.ShardedNovak(flat_p, numel, **BASE)
+        for _ in range(6):
+            flat_g = torch.zeros(n, device=DEV)
+            flat_g[:total].normal_(0.0, 1e-2, generator=gen)
+            oracle.step([to_f64(flat_g[:total])])
+            opt.step(flat_g)
+        torch.cuda.synchronize()
+        assert_close(flat_p[:total], oracle.theta[0], "zero1 theta")
+        assert bool((flat_p[total:] == 0).all())
+        assert opt.local.info()["t"] == 6 and opt.local.info()["n_syncs"] == 1
+        with pytest.raises(ValueError):
+            zero1.ShardedNovak(flat_p, numel, clip_threshold=1.0, **BASE)
+    finally:
+        dist.destroy_process_group()
