@@ -23,12 +23,15 @@ def test_fullsize_workload(index, mode):
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of device memory")
     harness.MARGINS.clear()
+    harness.SCALED.clear()
     pair = SampledPair(wl, DEV, dict(lookahead_mode=mode))
     for _ in range(wl.steps):
         pair.step(threads=8)
     pair.check()
     print(f"\nPARITY {wl.name} {mode} steps={wl.steps} sampled={pair.idx.numel()} worst |err|/tol: "
-          + ", ".join(f"{k.split()[-1]} {v:.3f}" for k, v in harness.MARGINS.items()))
+          + ", ".join(f"{k.split()[-1]} {v:.3f}" for k, v in harness.MARGINS.items())
+          + "; moments relative to their rms: "
+          + ", ".join(f"{k.split()[-1]} {v:.2e}" for k, v in harness.SCALED.items()))
     k = pair.hyper["lookahead_k"]
     assert pair.sync_steps == list(range(k, wl.steps + 1, k))
     assert pair.rect_flags == [0] * 5 + [1] * (wl.steps - 5)
