@@ -322,9 +322,9 @@ int novak_step_noalloc(novak_opt *opt, void *const *d_params,
  * then uses g' = factor * (g - row mean).  Clipping acts on the norm of the raw
  * gradient, before any other processing (Section 7.3).  Three launches per
  * step, no host synchronisation, no floating-point atomics (results are
- * bit-identical from run to run); the scratch (24 B per chunk-table entry +
- * 8 B per row) is allocated by the first such step.  Centralization needs
- * chunk-table entries of at most 2048 elements (the default).
+ * bit-identical from run to run); the scratch (about 16 B per chunk-table entry
+ * + 8 B per row + 48 B per 8192 elements of tensors with rows) is allocated by
+ * the first such step and again when the rows change.
  * novak_step_noalloc refuses to run in this mode (NOVAK_ESTATE). */
 int novak_set_tensor_rows(novak_opt *opt, const int64_t *rows, int n);
 
@@ -397,6 +397,16 @@ int novak_import_meta(novak_opt *opt, const novak_meta *in);
 int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
                            int64_t chunk_elems, int32_t *tensor, int64_t *offset,
                            int32_t *len, int64_t cap);
+
+/* Host-only helper exposing how the statistics pass of the centralization cuts
+ * tensors with rows into units: groups of whole rows of up to 1024 elements,
+ * about 8192 elements per group (part_len = 0), or, for longer rows, slices
+ * [part_off, part_off + part_len) of at most 8192 elements of one row
+ * (n_rows = 1), consecutive in the table.  rows[i] as in novak_set_tensor_rows.  Writes up to cap entries and
+ * returns the number the table needs (negative on bad arguments). */
+int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
+                              int64_t *row0, int64_t *n_rows, int64_t *part_off,
+                              int64_t *part_len, int64_t cap);
 
 /* Text of the last error on this handle ("" if none).  Owned by the handle. */
 const char *novak_last_error(const novak_opt *opt);

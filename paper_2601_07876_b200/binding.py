@@ -122,6 +122,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_import_meta": (c_int, [vp, POINTER(novak_meta)]),
         "novak_build_chunks": (c_int64, [i64p, POINTER(c_int32), c_int, c_int64,
                                          POINTER(c_int32), i64p, POINTER(c_int32), c_int64]),
+        "novak_build_row_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, i64p,
+                                            i64p, c_int64]),
         "novak_last_error": (c_char_p, [vp]),
     }
     for name, (res, args) in sigs.items():
@@ -160,6 +162,21 @@ def novak_build_chunks(numel, phase=None, chunk_elems=8192, lib=None):
     t, o, ln = (c_int32 * need)(), (c_int64 * need)(), (c_int32 * need)()
     lib.novak_build_chunks(num, ph, n, chunk_elems, t, o, ln, need)
     return list(t), list(o), list(ln)
+
+
+def novak_build_row_units(numel, rows, lib=None):
+    """Host-only: the statistics pass's units for tensors with rows, as a list of
+    (tensor, row0, n_rows, part_off, part_len)."""
+    lib = lib or load_library()
+    n = len(numel)
+    num, rw = i64_array(numel), i64_array(rows)
+    need = lib.novak_build_row_units(num, rw, n, None, None, None, None, None, 0)
+    if need < 0:
+        raise NovakError(NOVAK_EINVAL, "novak_build_row_units")
+    t = (c_int32 * need)()
+    cols = [(c_int64 * need)() for _ in range(4)]
+    lib.novak_build_row_units(num, rw, n, t, *cols, need)
+    return list(zip(list(t), *[list(c) for c in cols]))
 
 
 _NESTEROV = {"none": NOVAK_NESTEROV_NONE, "approximation": NOVAK_NESTEROV_APPROX,

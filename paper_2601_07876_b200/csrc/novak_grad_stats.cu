@@ -7,18 +7,21 @@
 // Both stay in device memory; the step kernel that follows on the stream reads
 // them there, so the host never waits for a reduction.
 //
-// Decomposition: one CTA per 4 consecutive chunk-table entries (the table of the
-// step kernel); per entry when row means are wanted.
-// All sums are carried in double precision and combined in a fixed order (warp
-// shuffle tree, then warps in index order, then chunks in index order), so the
+// Decomposition.  Tensors without rows: one CTA per 4 consecutive chunk-table
+// entries (the table of the step kernel), sum of squares only.  Tensors with
+// rows: a table of row units built on the host, aligned to ROWS, not to the
+// chunk table: a unit is a group of whole rows of up to 1024 elements (a warp
+// streams each row, or a thread for rows shorter than 128 elements), or a
+// slice of at most 8192 elements of a longer row (the whole CTA; usually the
+// whole row).  No shared-memory
+// staging, no per-vector row arithmetic: a lane only ever adds along one row.
+// All sums are carried in double precision and combined in a fixed order (per
+// lane, warp shuffle tree, warps in index order, CTAs in index order), so the
 // result is bit-identical from run to run; there are no floating-point atomics.
-// A row that spans several entries leaves one partial sum per entry; a second,
-// small kernel (one thread per entry) adds those up in entry order and reduces
-// the per-entry sums of squares; its last CTA (an integer ticket counter)
-// writes the norm and the clip factor.  Nothing spins: every CTA does a bounded
-// amount of work and returns.
-//
-// Row means need chunk-table entries of at most 2048 elements (the host checks).
+// A second, small kernel adds the slices of long rows in order and reduces the
+// CTAs' sums of squares; its last CTA (an integer ticket counter) writes the
+// norm and the clip factor.  Nothing spins: every CTA does a bounded amount of
+// work and returns.
 #include "novak_internal.h"
 
 #include "novak.h"
@@ -76,14 +79,8 @@ __device__ __forceinline__ double block_sum(double x, double *sh)
     return t;
 }
 
-// Largest chunk-table entry the row-mean path handles: one shared-memory slot
-// per 4-element vector, two vectors per thread.
-constexpr int kStatsMaxChunk = 2048;
-constexpr int kStatsMaxVec = kStatsMaxChunk / 4;
-
-// Up to 4 consecutive gradient elements starting at element `i` of `g` (which
-// points at the entry's first element), as fp32; n < 4 at a tensor's end (the
-// rest reads as 0), n = 0 loads nothing.
+// Up to 4 consecutive gradient elements starting at element `i` of `g`, as
+// fp32; n < 4 at a ragged end (the rest reads as 0), n = 0 loads nothing.
 template <int GT>
 __device__ __forceinline__ void load_quad(const void *g, bool aligned, uint32_t i, uint32_t n,
                                           float (&x)[4])
@@ -118,23 +115,13 @@ __device__ __forceinline__ double sum_squares(const float (&x)[4], double sq)
     return sq + double(s);
 }
 
-// Splits a vector's sum at the end of the row of its first element, which sits
-// `rem` elements into a row of length L >= 4 (a vector touches at most two
-// rows).  Row sums are carried in double from the first addition on: an
-// absolute error in a row mean becomes an absolute error in every centred
-// gradient of the row, and the update direction m^/(sqrt(v^)+eps) amplifies
-// such an error by up to 1/eps where the centred gradient is below eps.
-__device__ __forceinline__ void split_at_row_end(const float (&x)[4], uint32_t rem, uint32_t L,
-                                                 double *lo, double *hi)
+// Row sums are carried in double from the first addition on: an absolute error
+// in a row mean becomes an absolute error in every centred gradient of the row,
+// and the update direction m^/(sqrt(v^)+eps) amplifies such an error by up to
+// 1/eps where the centred gradient is below eps.
+__device__ __forceinline__ double sum_four(const float (&x)[4], double sum)
 {
-    const uint32_t left = L - rem;                         // elements up to the row's end
-    double a = 0.0, b = 0.0;
-#pragma unroll
-    for (uint32_t j = 0; j < 4u; ++j) {
-        if (j < left) a += double(x[j]); else b += double(x[j]);
-    }
-    *lo = a;
-    *hi = b;
+    return sum + ((double(x[0]) + double(x[1])) + (double(x[2]) + double(x[3])));
 }
 
 // A row mean as an unevaluated sum of two floats (hi + lo carries ~48 bits).
@@ -145,172 +132,267 @@ __device__ __forceinline__ float2 split_mean(double sum, uint32_t L)
     return make_float2(hi, static_cast<float>(mu - double(hi)));
 }
 
-// Entries one CTA of the first kernel takes (consecutive in the table).  All
-// their table reads, then all their gradient loads, are issued together, so a
-// CTA pays the table -> record -> data latency chain once per 32 KB, not per 8 KB.
-#ifndef NOVAK_STATS_ROWS_ENTRIES
-#define NOVAK_STATS_ROWS_ENTRIES 1
-#endif
-constexpr int kStatsEntries = 4;                          // no tensor has rows
-constexpr int kStatsEntriesRows = NOVAK_STATS_ROWS_ENTRIES;   // row means: more registers per entry
+// Chunk-table entries one CTA of the plain path takes (consecutive in the
+// list).  All their table reads, then all their gradient loads, are issued
+// together, so a CTA pays the table -> record -> data latency chain once per
+// 32 KB, not per 8 KB.
+constexpr int kStatsEntries = 4;
 
-// Sums of one row piece [s0, s1) of `row`, to the row mean if the piece is the
-// whole row, else to the entry's first / last partial sum.
-__device__ __forceinline__ void store_row_piece(const TensorRec &rec, uint32_t row, uint32_t r0,
-                                                bool whole, double sum, uint32_t L,
-                                                double *seg_first, double *seg_last, int c)
+// Entries per CTA of the plain path: bf16 entries are half as many bytes, so a
+// CTA takes twice as many (with 128-bit loads) to keep the same bytes in
+// flight.  Where row units share the kernel the plain entries are the small
+// tensors only, and the lean generic path keeps the registers for the rows.
+template <int GT, bool ROWS>
+struct PlainEntries {
+    static constexpr bool wide = (GT == NOVAK_GRAD_BF16) && !ROWS;
+    static constexpr int value = wide ? 2 * kStatsEntries : kStatsEntries;
+};
+
+// Squares of 8 bf16 values packed in 16 bytes.
+__device__ __forceinline__ double sum_squares_bf16x8(const uint4 t, double sq)
 {
-    if (whole)
-        rec.mean[row] = split_mean(sum, L);   // whole row inside the entry
-    else if (row == r0)
-        seg_first[c] = sum;     // row began before this entry, or runs past it
-    else
-        seg_last[c] = sum;      // last row of the entry, continues in the next
+    const unsigned w[4] = {t.x, t.y, t.z, t.w};
+    float s = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float lo = __uint_as_float(w[j] << 16), hi = __uint_as_float(w[j] & 0xffff0000u);
+        s = fmaf(lo, lo, s);
+        s = fmaf(hi, hi, s);
+    }
+    return sq + double(s);
 }
 
-template <int GT, bool ROWS>
-__global__ void __launch_bounds__(kStatsBlock)
-novak_grad_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                        const TensorRec *__restrict__ recs,
-                        double *__restrict__ chunk_sq, double *__restrict__ seg_first,
-                        double *__restrict__ seg_last)
+// ---- tensors without rows, bf16 gradients: 8 consecutive entries, 128-bit loads
+__device__ __forceinline__ double plain_entries_bf16(const Chunk *__restrict__ plain, int n_plain,
+                                                     const TensorRec *__restrict__ recs, int c0)
 {
-    __shared__ double sh[kStatsWarps];
-    // per 4-element vector of an entry: the sum of the elements that belong to
-    // the row of its first element, and of those already in the next row
-    __shared__ double vec_lo[ROWS ? kStatsMaxVec : 1];
-    __shared__ double vec_hi[ROWS ? kStatsMaxVec : 1];
-    constexpr uint32_t kElemBytes = (GT == NOVAK_GRAD_BF16) ? 2u : 4u;
-    constexpr int K = ROWS ? kStatsEntriesRows : kStatsEntries;
-
-    grid_dependency_release();
-    const int c0 = blockIdx.x * K;
+    constexpr int K = PlainEntries<NOVAK_GRAD_BF16, false>::value;
     Chunk ch[K];
-    TensorRec rec[K];
+    const void *base[K];
 #pragma unroll
-    for (int k = 0; k < K; ++k) ch[k] = chunks[min(c0 + k, n_chunks - 1)];
+    for (int k = 0; k < K; ++k) ch[k] = plain[min(c0 + k, n_plain - 1)];
 #pragma unroll
-    for (int k = 0; k < K; ++k) rec[k] = recs[ch[k].tensor];
+    for (int k = 0; k < K; ++k) base[k] = recs[ch[k].tensor].g;
     grid_dependency_wait();          // the gradient may come from the previous kernel
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const void *g[K];
-    bool aligned[K], fast[K];
-    uint32_t ia[K], ib[K], na[K], nb[K];
-    float xa[K][4], xb[K][4];
-    // ---- every entry's first two vectors per thread, all loads in flight at once
+    const unsigned short *g[K];
+    bool wide[K];
+    uint4 x[K];
+    // one 16-byte vector (8 elements) per thread and entry, all loads in flight at once
 #pragma unroll
     for (int k = 0; k < K; ++k) {
-        const uintptr_t addr = reinterpret_cast<uintptr_t>(rec[k].g) +
-                               static_cast<uintptr_t>(ch[k].offset) * kElemBytes;
-        g[k] = reinterpret_cast<const void *>(addr);          // the entry's first element
-        aligned[k] = (addr & (4u * kElemBytes - 1u)) == 0;
-        const uint32_t len = static_cast<uint32_t>(ch[k].len);
-        const bool short_rows = ROWS && rec[k].mean != nullptr && rec[k].row_len < 4u;
-        fast[k] = (c0 + k < n_chunks) && !short_rows;
-        const uint32_t nvec = (len + 3u) >> 2;
-        const uint32_t va = threadIdx.x, vb = va + kStatsBlock;
-        ia[k] = va << 2;
-        ib[k] = vb << 2;
-        na[k] = (fast[k] && va < nvec) ? (len - ia[k] < 4u ? len - ia[k] : 4u) : 0u;
-        nb[k] = (fast[k] && vb < nvec) ? (len - ib[k] < 4u ? len - ib[k] : 4u) : 0u;
-        load_quad<GT>(g[k], aligned[k], ia[k], na[k], xa[k]);
-        load_quad<GT>(g[k], aligned[k], ib[k], nb[k], xb[k]);
+        g[k] = static_cast<const unsigned short *>(base[k]) + ch[k].offset;
+        const uint32_t len = (c0 + k < n_plain) ? static_cast<uint32_t>(ch[k].len) : 0u;
+        wide[k] = (reinterpret_cast<uintptr_t>(g[k]) & 15u) == 0;
+        x[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (wide[k] && (threadIdx.x + 1u) * 8u <= len)
+            x[k] = __ldg(reinterpret_cast<const uint4 *>(g[k]) + threadIdx.x);
     }
-
     double sq = 0.0;
 #pragma unroll
     for (int k = 0; k < K; ++k) {
-        if (c0 + k >= n_chunks) break;
-        const int c = c0 + k;
+        if (c0 + k >= n_plain) break;
+        sq = sum_squares_bf16x8(x[k], sq);
+        // what the one vector per thread did not cover: an unaligned entry, a ragged
+        // end, or an entry longer than 2048 elements
         const uint32_t len = static_cast<uint32_t>(ch[k].len);
-        const bool rows = ROWS && rec[k].mean != nullptr;
-        const uint32_t L = rec[k].row_len;
-        const uint32_t off = static_cast<uint32_t>(ch[k].offset);   // used with rows only (< 2^31)
-        const uint32_t end = off + len;
-
-        if (rows && L < 4u) {
-            // ---- rows of 1 to 3 elements: a thread per row, straight from global memory
-            const uint32_t r0 = off / L, r1 = (end - 1u) / L;
-            for (uint32_t row = r0 + threadIdx.x; row <= r1; row += kStatsBlock) {
-                const uint32_t row_begin = row * L, row_end = row_begin + L;
-                const uint32_t s0 = row_begin > off ? row_begin : off;
-                const uint32_t s1 = row_end < end ? row_end : end;
-                double sum = 0.0;
-                for (uint32_t e = s0; e < s1; ++e) {
-                    const float x = grad_at<GT>(rec[k].g, e);
-                    sum += double(x);
-                    sq = fma(double(x), double(x), sq);
-                }
-                store_row_piece(rec[k], row, r0, s0 == row_begin && s1 == row_end, sum, L,
-                                seg_first, seg_last, c);
-            }
-            continue;
+        const uint32_t done = wide[k] ? min(len & ~7u, 8u * kStatsBlock) : 0u;
+        for (uint32_t e = done + threadIdx.x; e < len; e += kStatsBlock) {
+            const float v = grad_at<NOVAK_GRAD_BF16>(g[k], e);
+            sq = fma(double(v), double(v), sq);
         }
+    }
+    return sq;
+}
 
-        // ---- pass 1: squares of the vectors already loaded and, for a tensor with
-        // rows, each vector's sum split at the row boundary
+// ---- tensors without rows: the sum of squares of 4 consecutive entries
+template <int GT, bool WIDE>
+__device__ __forceinline__ double plain_entries(const Chunk *__restrict__ plain, int n_plain,
+                                                const TensorRec *__restrict__ recs, int c0)
+{
+    if constexpr (WIDE) return plain_entries_bf16(plain, n_plain, recs, c0);
+    constexpr uint32_t kElemBytes = (GT == NOVAK_GRAD_BF16) ? 2u : 4u;
+    constexpr int K = kStatsEntries;
+    Chunk ch[K];
+    const void *base[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) ch[k] = plain[min(c0 + k, n_plain - 1)];
+#pragma unroll
+    for (int k = 0; k < K; ++k) base[k] = recs[ch[k].tensor].g;
+    grid_dependency_wait();          // the gradient may come from the previous kernel
+
+    const void *g[K];
+    bool aligned[K];
+    float xa[K][4], xb[K][4];
+    // every entry's first two vectors per thread, all loads in flight at once
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(base[k]) +
+                               static_cast<uintptr_t>(ch[k].offset) * kElemBytes;
+        g[k] = reinterpret_cast<const void *>(addr);          // the entry's first element
+        aligned[k] = (addr & (4u * kElemBytes - 1u)) == 0;
+        const uint32_t len = (c0 + k < n_plain) ? static_cast<uint32_t>(ch[k].len) : 0u;
+        const uint32_t nvec = (len + 3u) >> 2;
+        const uint32_t va = threadIdx.x, vb = va + kStatsBlock;
+        const uint32_t ia = va << 2, ib = vb << 2;
+        load_quad<GT>(g[k], aligned[k], ia, va < nvec ? (len - ia < 4u ? len - ia : 4u) : 0u, xa[k]);
+        load_quad<GT>(g[k], aligned[k], ib, vb < nvec ? (len - ib < 4u ? len - ib : 4u) : 0u, xb[k]);
+    }
+    double sq = 0.0;
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        if (c0 + k >= n_plain) break;
         sq = sum_squares(xa[k], sq);
         sq = sum_squares(xb[k], sq);
-        if (rows) {                     // entries of tensors with rows have at most 512 vectors
-            // where in its row each of this thread's two vectors starts: one division,
-            // the second vector lies 4 x 256 elements further on
-            const uint32_t ea = off + ia[k];
-            const uint32_t rem_a = ea - (ea / L) * L;
-            uint32_t rem_b = rem_a + 4u * kStatsBlock;
-            if (rem_b >= L) rem_b = (L >= 4u * kStatsBlock) ? rem_b - L : rem_b % L;
-            if (na[k]) split_at_row_end(xa[k], rem_a, L, &vec_lo[threadIdx.x], &vec_hi[threadIdx.x]);
-            if (nb[k]) split_at_row_end(xb[k], rem_b, L, &vec_lo[threadIdx.x + kStatsBlock],
-                                        &vec_hi[threadIdx.x + kStatsBlock]);
-        } else {
-            // entries longer than 2048 elements (no rows): the rest of the vectors
-            const uint32_t nvec = (len + 3u) >> 2;
-            for (uint32_t v = threadIdx.x + 2u * kStatsBlock; v < nvec; v += kStatsBlock) {
-                float x[4];
-                const uint32_t i = v << 2;
-                load_quad<GT>(g[k], aligned[k], i, len - i < 4u ? len - i : 4u, x);
-                sq = sum_squares(x, sq);
-            }
-        }
-        if (rows) {
-            // ---- pass 2: the pieces of rows inside this entry, summed in vector
-            // order.  Rows of 128 elements or more take a warp each, shorter ones
-            // a thread each.
-            __syncthreads();
-            const uint32_t r0 = off / L, r1 = (end - 1u) / L;
-            const bool by_warp = L >= 128u;
-            const uint32_t first = by_warp ? warp : threadIdx.x;
-            const uint32_t stride = by_warp ? kStatsWarps : kStatsBlock;
-            for (uint32_t row = r0 + first; row <= r1; row += stride) {
-                const uint32_t row_begin = row * L, row_end = row_begin + L;
-                const uint32_t s0 = row_begin > off ? row_begin : off;
-                const uint32_t s1 = row_end < end ? row_end : end;
-                const uint32_t vb = (s0 - off + 3u) >> 2, ve = (s1 - off + 3u) >> 2;
-                double sum = 0.0;
-                if (by_warp) {
-                    for (uint32_t v = vb + lane; v < ve; v += 32u) sum += vec_lo[v];
-                    sum = warp_sum(sum);
-                } else {
-                    for (uint32_t v = vb; v < ve; ++v) sum += vec_lo[v];
-                }
-                if (!by_warp || lane == 0) {
-                    if (((s0 - off) & 3u) != 0u) sum += vec_hi[vb - 1u];   // row starts mid-vector
-                    store_row_piece(rec[k], row, r0, s0 == row_begin && s1 == row_end, sum, L,
-                                    seg_first, seg_last, c);
-                }
-            }
-            __syncthreads();            // the slots are reused by the next entry
+        // entries longer than 2048 elements: the rest of the vectors
+        const uint32_t len = static_cast<uint32_t>(ch[k].len);
+        const uint32_t nvec = (len + 3u) >> 2;
+        for (uint32_t v = threadIdx.x + 2u * kStatsBlock; v < nvec; v += kStatsBlock) {
+            float x[4];
+            const uint32_t i = v << 2;
+            load_quad<GT>(g[k], aligned[k], i, len - i < 4u ? len - i : 4u, x);
+            sq = sum_squares(x, sq);
         }
     }
+    return sq;
+}
 
-    // one sum of squares per CTA, filed under its first entry
-    const double total = block_sum(sq, sh);
-    if (threadIdx.x == 0) {
-        chunk_sq[c0] = total;
-#pragma unroll
-        for (int k = 1; k < K; ++k)
-            if (c0 + k < n_chunks) chunk_sq[c0 + k] = 0.0;
+// One aligned vector of 4 gradient elements as fp32.
+template <int GT>
+__device__ __forceinline__ void load_vec(const void *g, uint32_t v, float (&x)[4])
+{
+    if constexpr (GT == NOVAK_GRAD_F32) {
+        const float4 t = __ldg(static_cast<const float4 *>(g) + v);
+        x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+    } else {
+        const uint2 t = __ldg(static_cast<const uint2 *>(g) + v);
+        x[0] = __uint_as_float(t.x << 16);
+        x[1] = __uint_as_float(t.x & 0xffff0000u);
+        x[2] = __uint_as_float(t.y << 16);
+        x[3] = __uint_as_float(t.y & 0xffff0000u);
     }
+}
+
+// Sum and sum of squares of elements [e0, e0 + n) of a tensor's gradient, the
+// calling threads (`nthreads` of them, this one being number `t`) striding over
+// 4-element vectors: 128-bit / 64-bit loads, four of them in flight per thread,
+// where the span is aligned; element by element otherwise.
+template <int GT>
+__device__ __forceinline__ void span_sums(const void *g_tensor, uint32_t e0, uint32_t n, uint32_t t,
+                                          uint32_t nthreads, double &sum, double &sq)
+{
+    constexpr uint32_t kElemBytes = (GT == NOVAK_GRAD_BF16) ? 2u : 4u;
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(g_tensor) + uintptr_t(e0) * kElemBytes;
+    const void *g = reinterpret_cast<const void *>(addr);
+    if ((addr & (4u * kElemBytes - 1u)) == 0) {
+        const uint32_t nfull = n >> 2;
+        uint32_t v = t;
+        for (; v + 3u * nthreads < nfull; v += 4u * nthreads) {
+            float x0[4], x1[4], x2[4], x3[4];
+            load_vec<GT>(g, v, x0);
+            load_vec<GT>(g, v + nthreads, x1);
+            load_vec<GT>(g, v + 2u * nthreads, x2);
+            load_vec<GT>(g, v + 3u * nthreads, x3);
+            sum = sum_four(x0, sum); sq = sum_squares(x0, sq);
+            sum = sum_four(x1, sum); sq = sum_squares(x1, sq);
+            sum = sum_four(x2, sum); sq = sum_squares(x2, sq);
+            sum = sum_four(x3, sum); sq = sum_squares(x3, sq);
+        }
+        if (v < nfull) {
+            // up to three more vectors, again loaded together
+            float x0[4] = {0.f, 0.f, 0.f, 0.f}, x1[4] = {0.f, 0.f, 0.f, 0.f}, x2[4] = {0.f, 0.f, 0.f, 0.f};
+            load_vec<GT>(g, v, x0);
+            if (v + nthreads < nfull) load_vec<GT>(g, v + nthreads, x1);
+            if (v + 2u * nthreads < nfull) load_vec<GT>(g, v + 2u * nthreads, x2);
+            sum = sum_four(x0, sum); sq = sum_squares(x0, sq);
+            sum = sum_four(x1, sum); sq = sum_squares(x1, sq);
+            sum = sum_four(x2, sum); sq = sum_squares(x2, sq);
+        }
+        const uint32_t e = (nfull << 2) + t;                  // ragged end: < 4 elements
+        if (e < n) {
+            const float x = grad_at<GT>(g, e);
+            sum += double(x);
+            sq = fma(double(x), double(x), sq);
+        }
+    } else {
+#pragma unroll 4
+        for (uint32_t e = t; e < n; e += nthreads) {
+            const float x = grad_at<GT>(g, e);
+            sum += double(x);
+            sq = fma(double(x), double(x), sq);
+        }
+    }
+}
+
+// ---- tensors with rows: one unit of the row table (see RowUnit)
+template <int GT>
+__device__ __forceinline__ double row_unit(const RowUnit u, const TensorRec rec,
+                                           double *__restrict__ part_sum, int unit_index,
+                                           double *sh)
+{
+    const uint32_t L = rec.row_len;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double sq = 0.0;
+    if (u.part_len != 0u) {
+        // a slice of one long row for the whole CTA: the whole row, or a piece whose
+        // sum the second kernel adds to its neighbours'
+        double sum = 0.0;
+        span_sums<GT>(rec.g, u.row0 * L + u.part_off, u.part_len, threadIdx.x, kStatsBlock, sum, sq);
+        const double total = block_sum(sum, sh);
+        if (threadIdx.x == 0) {
+            if (u.n_parts == 1u) rec.mean[u.row0] = split_mean(total, L);
+            else part_sum[unit_index] = total;
+        }
+    } else if (L >= 128u) {
+        // whole rows, a warp each
+        for (uint32_t r = u.row0 + warp; r < u.row0 + u.n_rows; r += kStatsWarps) {
+            double sum = 0.0;
+            span_sums<GT>(rec.g, r * L, L, lane, 32u, sum, sq);
+            sum = warp_sum(sum);
+            if (lane == 0) rec.mean[r] = split_mean(sum, L);
+        }
+    } else {
+        // short rows, a thread each
+        const uint32_t r = u.row0 + threadIdx.x;
+        if (threadIdx.x < u.n_rows) {
+            double sum = 0.0;
+            for (uint32_t e = r * L; e < (r + 1u) * L; ++e) {
+                const float x = grad_at<GT>(rec.g, e);
+                sum += double(x);
+                sq = fma(double(x), double(x), sq);
+            }
+            rec.mean[r] = split_mean(sum, L);
+        }
+    }
+    return sq;
+}
+
+// First kernel of the pass.  CTAs [0, ceil(n_plain / 4)) take 4 chunk-table
+// entries each of the tensors without rows; the following n_units CTAs take one
+// row unit each.  Every CTA leaves one sum of squares in part_sq[blockIdx.x].
+template <int GT, bool ROWS>
+__global__ void __launch_bounds__(kStatsBlock)
+novak_grad_stats_kernel(const Chunk *__restrict__ plain, int n_plain,
+                        const RowUnit *__restrict__ units, int n_units,
+                        const TensorRec *__restrict__ recs, double *__restrict__ part_sq,
+                        double *__restrict__ part_sum)
+{
+    __shared__ double sh[kStatsWarps];
+    grid_dependency_release();
+    using Per = PlainEntries<GT, ROWS>;
+    const int plain_ctas = (n_plain + Per::value - 1) / Per::value;
+    double sq;
+    if (!ROWS || static_cast<int>(blockIdx.x) < plain_ctas) {
+        sq = plain_entries<GT, Per::wide>(plain, n_plain, recs, blockIdx.x * Per::value);
+    } else {
+        const int ui = blockIdx.x - plain_ctas;
+        const RowUnit u = units[ui];
+        const TensorRec rec = recs[u.tensor];
+        grid_dependency_wait();      // the gradient may come from the previous kernel
+        sq = row_unit<GT>(u, rec, part_sum, ui, sh);
+    }
+    const double total = block_sum(sq, sh);
+    if (threadIdx.x == 0) part_sq[blockIdx.x] = total;
 }
 
 // Sum of squares of the parameters (for ||theta_t|| of Eq. 21): one CTA per 4
@@ -354,54 +436,36 @@ novak_param_sumsq_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
 }
 
-// Second kernel of the pass, one THREAD per chunk-table entry: puts together the
-// rows that entry boundaries cut (the thread of the entry in which such a row
-// BEGINS adds the pieces in entry order; the table lists a tensor's entries
-// consecutively, in element order), and sums the entries' sums of squares: per
-// CTA first, then the CTA that takes the last ticket adds the CTAs' sums in
-// index order and writes the norm and the clip factor.
-template <bool ROWS>
+// Second kernel of the pass, one THREAD per sum of the first: completes the
+// means of the long rows that were cut into slices (the thread of a row's first
+// slice adds the slices in order) and adds up the sums of squares: per CTA
+// first, then the CTA that takes the last ticket adds the CTAs' sums in index
+// order and writes the norm, the clip factor and, when asked, Eq. 20-22.
 __global__ void __launch_bounds__(kStatsBlock)
-novak_grad_stats_finish_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                               const TensorRec *__restrict__ recs, double c_clip,
-                               double auto_gamma, const double *__restrict__ chunk_sq,
-                               const double *__restrict__ chunk_psq,
-                               const double *__restrict__ seg_first,
-                               const double *__restrict__ seg_last,
-                               double *__restrict__ cta_sq, PrepOut *__restrict__ out)
+novak_grad_stats_finish_kernel(const RowUnit *__restrict__ units, int n_units,
+                               const TensorRec *__restrict__ recs, int n_work,
+                               const double *__restrict__ part_sq,
+                               const double *__restrict__ part_sum, int n_chunks,
+                               const double *__restrict__ chunk_psq, double c_clip,
+                               double auto_gamma, double *__restrict__ cta_sq,
+                               PrepOut *__restrict__ out)
 {
     __shared__ double sh[kStatsWarps];
     __shared__ unsigned sh_last;
 
     grid_dependency_release();
-    grid_dependency_wait();          // everything below is the first kernel's output
+    grid_dependency_wait();          // everything below is the earlier kernels' output
     const int i = blockIdx.x * kStatsBlock + threadIdx.x;
     double sq = 0.0, psq = 0.0;
-    if (i < n_chunks) {
-        sq = chunk_sq[i];
-        if (chunk_psq != nullptr) psq = chunk_psq[i];
-        if constexpr (ROWS) {
-            const Chunk ci = chunks[i];
-            const TensorRec ri = recs[ci.tensor];
-            if (ri.mean != nullptr) {
-                const uint32_t L = ri.row_len;
-                const uint32_t o = static_cast<uint32_t>(ci.offset);
-                const uint32_t e = o + static_cast<uint32_t>(ci.len);
-                const uint32_t row = (e - 1u) / L;
-                const uint32_t row_begin = row * L, row_end = row_begin + L;
-                // the entry's last row runs past it, and began inside it
-                if (row_end > e && row_begin >= o) {
-                    double sum = (row == o / L) ? seg_first[i] : seg_last[i];
-                    for (int j = i + 1; j < n_chunks; ++j) {
-                        const Chunk cj = chunks[j];
-                        if (cj.tensor != ci.tensor) break;
-                        sum += seg_first[j];
-                        if (static_cast<uint32_t>(cj.offset) + static_cast<uint32_t>(cj.len) >= row_end)
-                            break;
-                    }
-                    ri.mean[row] = split_mean(sum, L);
-                }
-            }
+    if (i < n_work) sq = part_sq[i];
+    if (chunk_psq != nullptr && i < n_chunks) psq = chunk_psq[i];
+    if (i < n_units) {
+        const RowUnit u = units[i];
+        if (u.n_parts > 1u && u.part_idx == 0u) {
+            double sum = 0.0;
+            for (uint32_t j = 0; j < u.n_parts; ++j) sum += part_sum[i + j];
+            const TensorRec r = recs[u.tensor];
+            r.mean[u.row0] = split_mean(sum, r.row_len);
         }
     }
     const double total = block_sum(sq, sh);
@@ -473,50 +537,59 @@ cudaError_t launch_pdl(const void *fn, unsigned grid, void **args, bool pdl, cud
 
 }  // namespace
 
-int grad_stats_ctas(int n_chunks) { return (n_chunks + kStatsBlock - 1) / kStatsBlock; }
-
-cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                              int grad_dtype, double c_clip, double auto_gamma, double *chunk_sq,
-                              double *chunk_psq, double *seg_first, double *seg_last,
-                              double *cta_sq, PrepOut *prep, bool any_rows, int pdl,
-                              cudaStream_t stream)
+int grad_stats_work(int n_plain, int n_units, int grad_dtype)
 {
-    if (auto_gamma > 0.0 && !chunk_psq) return cudaErrorInvalidValue;
-    if (n_chunks <= 0 || !d_chunks || !d_recs || !chunk_sq || !cta_sq || !prep)
-        return cudaErrorInvalidValue;
-    if (any_rows && (!seg_first || !seg_last)) return cudaErrorInvalidValue;
+    const int per = (grad_dtype == NOVAK_GRAD_BF16 && n_units == 0)
+                        ? PlainEntries<NOVAK_GRAD_BF16, false>::value : kStatsEntries;
+    return (n_plain + per - 1) / per + n_units;
+}
+
+int grad_stats_ctas(int n_work, int n_chunks)
+{
+    const int n = n_work > n_chunks ? n_work : n_chunks;
+    return (n + kStatsBlock - 1) / kStatsBlock;
+}
+
+cudaError_t launch_grad_stats(const StatsPlan &w, int grad_dtype, double c_clip, double auto_gamma,
+                              int pdl, cudaStream_t stream)
+{
+    const int n_work = grad_stats_work(w.n_plain, w.n_units, grad_dtype);
+    if (n_work <= 0 || !w.recs || !w.part_sq || !w.cta_sq || !w.prep) return cudaErrorInvalidValue;
+    if (w.n_plain > 0 && !w.plain) return cudaErrorInvalidValue;
+    if (w.n_units > 0 && (!w.units || !w.part_sum)) return cudaErrorInvalidValue;
+    if (auto_gamma > 0.0 && (!w.chunks || !w.chunk_psq || w.n_chunks <= 0)) return cudaErrorInvalidValue;
     const void *first = nullptr;
     switch (grad_dtype) {
     case NOVAK_GRAD_F32:
-        first = any_rows ? reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_F32, true>)
-                         : reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_F32, false>);
+        first = w.n_units > 0 ? reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_F32, true>)
+                              : reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_F32, false>);
         break;
     case NOVAK_GRAD_BF16:
-        first = any_rows ? reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_BF16, true>)
-                         : reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_BF16, false>);
+        first = w.n_units > 0 ? reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_BF16, true>)
+                              : reinterpret_cast<const void *>(novak_grad_stats_kernel<NOVAK_GRAD_BF16, false>);
         break;
     default: return cudaErrorInvalidValue;
     }
-    const void *second = any_rows ? reinterpret_cast<const void *>(novak_grad_stats_finish_kernel<true>)
-                                  : reinterpret_cast<const void *>(novak_grad_stats_finish_kernel<false>);
-    void *args1[] = {&d_chunks, &n_chunks, &d_recs, &chunk_sq, &seg_first, &seg_last};
-    const int per_cta = any_rows ? kStatsEntriesRows : kStatsEntries;
-    const unsigned grid1 = static_cast<unsigned>((n_chunks + per_cta - 1) / per_cta);
-    cudaError_t e = launch_pdl(first, grid1, args1, (pdl & 2) != 0, stream);
+    StatsPlan a = w;
+    void *args1[] = {&a.plain, &a.n_plain, &a.units, &a.n_units, &a.recs, &a.part_sq, &a.part_sum};
+    cudaError_t e = launch_pdl(first, static_cast<unsigned>(n_work), args1, (pdl & 2) != 0, stream);
     if (e != cudaSuccess) return e;
     const double *c_psq = nullptr;
     if (auto_gamma > 0.0) {
-        void *args_p[] = {&d_chunks, &n_chunks, &d_recs, &chunk_psq};
-        const unsigned grid_p = static_cast<unsigned>((n_chunks + kStatsEntries - 1) / kStatsEntries);
+        void *args_p[] = {&a.chunks, &a.n_chunks, &a.recs, &a.chunk_psq};
+        const unsigned grid_p = static_cast<unsigned>((a.n_chunks + kStatsEntries - 1) / kStatsEntries);
         e = launch_pdl(reinterpret_cast<const void *>(novak_param_sumsq_kernel), grid_p, args_p,
                        (pdl & 2) != 0, stream);
         if (e != cudaSuccess) return e;
-        c_psq = chunk_psq;
+        c_psq = a.chunk_psq;
     }
-    const double *c_sq = chunk_sq, *c_first = seg_first, *c_last = seg_last;
-    void *args2[] = {&d_chunks, &n_chunks, &d_recs, &c_clip, &auto_gamma, &c_sq, &c_psq,
-                     &c_first, &c_last, &cta_sq, &prep};
-    return launch_pdl(second, static_cast<unsigned>(grad_stats_ctas(n_chunks)), args2, (pdl & 4) != 0, stream);
+    int work = n_work;
+    const double *c_sq = a.part_sq, *c_sum = a.part_sum;
+    void *args2[] = {&a.units, &a.n_units, &a.recs, &work, &c_sq, &c_sum, &a.n_chunks, &c_psq,
+                     &c_clip, &auto_gamma, &a.cta_sq, &a.prep};
+    return launch_pdl(reinterpret_cast<const void *>(novak_grad_stats_finish_kernel),
+                      static_cast<unsigned>(grad_stats_ctas(n_work, c_psq ? a.n_chunks : 0)), args2,
+                      (pdl & 4) != 0, stream);
 }
 
 }  // namespace novak

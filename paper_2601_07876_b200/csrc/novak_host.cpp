@@ -16,6 +16,7 @@
 
 using novak::Chunk;
 using novak::PrepOut;
+using novak::RowUnit;
 using novak::StepScalars;
 using novak::TensorRec;
 
@@ -127,6 +128,35 @@ void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chu
     }
 }
 
+// Cuts the tensors that have rows into units of the statistics pass; see
+// novak_build_row_units in novak.h and RowUnit.
+void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out)
+{
+    out.clear();
+    for (int i = 0; i < n; ++i) {
+        if (rows[i] <= 0) continue;
+        const uint32_t R = static_cast<uint32_t>(rows[i]);
+        const uint32_t L = static_cast<uint32_t>(numel[i] / rows[i]);
+        if (L > novak::kRowWarpMax) {
+            // a CTA per slice of at most kRowUnitElems elements (one slice for most rows)
+            const uint32_t parts = (L + novak::kRowUnitElems - 1) / novak::kRowUnitElems;
+            for (uint32_t r = 0; r < R; ++r)
+                for (uint32_t p = 0; p < parts; ++p) {
+                    const uint32_t off = p * novak::kRowUnitElems;
+                    out.push_back(RowUnit{i, r, 1u, off, std::min(novak::kRowUnitElems, L - off),
+                                          parts, p, 0u});
+                }
+        } else {
+            // a warp per row from 128 elements on (at least one row for each of the
+            // CTA's 8 warps), else a thread per row
+            const uint32_t per = L >= 128u ? std::max(8u, novak::kRowUnitElems / L)
+                                           : novak::kRowUnitThreads;
+            for (uint32_t r = 0; r < R; r += per)
+                out.push_back(RowUnit{i, r, std::min(per, R - r), 0u, 0u, 1u, 0u, 0u});
+        }
+    }
+}
+
 }  // namespace
 
 struct novak_opt {
@@ -185,8 +215,12 @@ struct novak_opt {
     char *d_prep = nullptr;
     int64_t prep_rows = -1;             // total_rows the scratch was sized for
     PrepOut *prep_out = nullptr;
-    double *chunk_sq = nullptr, *seg_first = nullptr, *seg_last = nullptr, *cta_sq = nullptr;
-    double *chunk_psq = nullptr;
+    double *part_sq = nullptr, *part_sum = nullptr, *cta_sq = nullptr, *chunk_psq = nullptr;
+    Chunk *d_plain = nullptr;           // entries of the tensors without rows (NULL: all of them)
+    RowUnit *d_units = nullptr;
+    int n_plain = 0, n_units = 0;
+    int64_t rows_gen = 0;               // bumped whenever the row settings change
+    int64_t prep_key = -1;              // rows_gen and centring the scratch was laid out for
     // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
     bool ema_pending = false;
     double pending_g_bar = 0.0, pending_theta_bar = 0.0;
@@ -309,7 +343,11 @@ void release_device(novak_opt *o)
     o->d_prep = nullptr;
     o->prep_rows = -1;
     o->prep_out = nullptr;
-    o->chunk_sq = o->seg_first = o->seg_last = o->cta_sq = o->chunk_psq = nullptr;
+    o->part_sq = o->part_sum = o->cta_sq = o->chunk_psq = nullptr;
+    o->d_plain = nullptr;
+    o->d_units = nullptr;
+    o->n_plain = o->n_units = 0;
+    o->prep_key = -1;
     o->row_mean = nullptr;
     for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
     o->host_ev.clear();
@@ -386,10 +424,13 @@ void invalidate_tables(novak_opt *o)
     o->cur_table = -1;
 }
 
-// Scratch of the statistics pass, allocated when a step first needs it.
+// Scratch of the statistics pass, laid out when a step first needs it and
+// again when the row settings change.
 int prepare_prep(novak_opt *o, cudaStream_t stream)
 {
-    if (o->d_prep && o->prep_rows == o->total_rows) return NOVAK_OK;
+    const bool centre = o->h.centralize && o->total_rows > 0;
+    const int64_t key = o->rows_gen * 2 + (centre ? 1 : 0);
+    if (o->d_prep && o->prep_key == key) return NOVAK_OK;
     cudaError_t e;
     if (o->d_prep) {
         // sizes changed: keep the averages of Eq. 20-21 (the copy waits for the device)
@@ -405,14 +446,31 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
         o->d_prep = nullptr;
         invalidate_tables(o);
     }
+    // work of the pass: row units for the tensors with rows, chunk-table entries for the rest
+    std::vector<RowUnit> units;
+    std::vector<Chunk> plain;
+    if (centre) {
+        build_row_units(o->numel.data(), o->rows.data(), o->n, units);
+        for (const Chunk &c : o->h_chunks)
+            if (o->rows[c.tensor] <= 0) plain.push_back(c);
+    }
+    const size_t n_plain = centre ? plain.size() : static_cast<size_t>(o->n_chunks);
+    if (units.size() > static_cast<size_t>(INT32_MAX) / 2) return fail(o, NOVAK_EINVAL, "too many rows");
+    // sized for fp32 gradients; bf16 gradients take more entries per CTA and need less
+    const size_t n_work = static_cast<size_t>(novak::grad_stats_work(
+        static_cast<int>(n_plain), static_cast<int>(units.size()), NOVAK_GRAD_F32));
     const size_t nc = static_cast<size_t>(o->n_chunks);
-    const size_t off_sq = 256;
-    const size_t off_psq = off_sq + nc * sizeof(double);
-    const size_t off_first = off_psq + nc * sizeof(double);
-    const size_t off_last = off_first + nc * sizeof(double);
-    const size_t off_cta = off_last + nc * sizeof(double);
-    const size_t off_mean = off_cta + 2 * static_cast<size_t>(novak::grad_stats_ctas(o->n_chunks)) * sizeof(double);
-    const size_t bytes = off_mean + static_cast<size_t>(o->total_rows) * sizeof(float2) + 16;
+    const size_t ctas = static_cast<size_t>(novak::grad_stats_ctas(static_cast<int>(n_work), o->n_chunks));
+    size_t off = 256;
+    const size_t off_sq = off;      off += n_work * sizeof(double);
+    const size_t off_sum = off;     off += units.size() * sizeof(double);
+    const size_t off_psq = off;     off += nc * sizeof(double);
+    const size_t off_cta = off;     off += 2 * ctas * sizeof(double);
+    off = (off + 15) / 16 * 16;
+    const size_t off_plain = off;   off += plain.size() * sizeof(Chunk);
+    const size_t off_units = off;   off += units.size() * sizeof(RowUnit);
+    const size_t off_mean = off;    off += static_cast<size_t>(o->total_rows) * sizeof(float2);
+    const size_t bytes = off + 16;
     if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
         o->d_prep = nullptr;
         return fail(o, NOVAK_ENOMEM, "cudaMalloc(gradient statistics, %zu B): %s", bytes, cudaGetErrorString(e));
@@ -420,13 +478,27 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
     if ((e = cudaMemsetAsync(o->d_prep, 0, bytes, stream)) != cudaSuccess)
         return fail_cuda(o, e, "cudaMemsetAsync(gradient statistics)");
     o->prep_out = reinterpret_cast<PrepOut *>(o->d_prep);
-    o->chunk_sq = reinterpret_cast<double *>(o->d_prep + off_sq);
+    o->part_sq = reinterpret_cast<double *>(o->d_prep + off_sq);
+    o->part_sum = reinterpret_cast<double *>(o->d_prep + off_sum);
     o->chunk_psq = reinterpret_cast<double *>(o->d_prep + off_psq);
-    o->seg_first = reinterpret_cast<double *>(o->d_prep + off_first);
-    o->seg_last = reinterpret_cast<double *>(o->d_prep + off_last);
     o->cta_sq = reinterpret_cast<double *>(o->d_prep + off_cta);
+    o->d_plain = centre ? reinterpret_cast<Chunk *>(o->d_prep + off_plain) : nullptr;
+    o->d_units = reinterpret_cast<RowUnit *>(o->d_prep + off_units);
     o->row_mean = reinterpret_cast<float2 *>(o->d_prep + off_mean);
-    o->prep_rows = o->total_rows;
+    o->n_plain = static_cast<int>(n_plain);
+    o->n_units = static_cast<int>(units.size());
+    // The tables are built once per layout: blocking copies keep the host
+    // vectors' lifetime trivial.
+    if (!plain.empty() &&
+        (e = cudaMemcpyAsync(o->d_plain, plain.data(), plain.size() * sizeof(Chunk),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "statistics table upload");
+    if (!units.empty() &&
+        (e = cudaMemcpyAsync(o->d_units, units.data(), units.size() * sizeof(RowUnit),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "row unit upload");
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail_cuda(o, e, "statistics table upload");
+    o->prep_key = key;
     invalidate_tables(o);              // records carry pointers into this scratch
     return NOVAK_OK;
 }
@@ -852,9 +924,6 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     int rc;
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
     ctx->pre = pre_mode(o);
-    if (ctx->pre == novak::PRE_CENTER && o->chunk_elems > 2048)
-        return fail(o, NOVAK_ESTATE, "centralization needs chunk-table entries of at most 2048 "
-                    "elements (NOVAK_OPT_CHUNK_ELEMS is %lld)", static_cast<long long>(o->chunk_elems));
     if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
     if (o->ema_pending && o->prep_out) {
         // averages set by the caller (or saved over a reallocation) go into the scratch
@@ -906,10 +975,21 @@ cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stre
 // Phase 2's statistics pass over the whole group: global norm, clip factor, row means.
 cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream)
 {
-    return novak::launch_grad_stats(o->d_chunks, o->n_chunks, ctx.d_recs, ctx.grad_dtype,
-                                    o->h.clip, o->h.auto_lr ? o->h.auto_gamma : 0.0, o->chunk_sq,
-                                    o->chunk_psq, o->seg_first, o->seg_last,
-                                    o->cta_sq, o->prep_out, ctx.pre == novak::PRE_CENTER, o->pdl, stream);
+    novak::StatsPlan plan;
+    plan.plain = o->d_plain ? o->d_plain : o->d_chunks;
+    plan.n_plain = o->n_plain;
+    plan.units = o->d_units;
+    plan.n_units = o->n_units;
+    plan.recs = ctx.d_recs;
+    plan.chunks = o->d_chunks;
+    plan.n_chunks = o->n_chunks;
+    plan.part_sq = o->part_sq;
+    plan.part_sum = o->part_sum;
+    plan.chunk_psq = o->chunk_psq;
+    plan.cta_sq = o->cta_sq;
+    plan.prep = o->prep_out;
+    return novak::launch_grad_stats(plan, ctx.grad_dtype, o->h.clip,
+                                    o->h.auto_lr ? o->h.auto_gamma : 0.0, o->pdl, stream);
 }
 
 // One launch over chunk-table entries [c0, c1).
@@ -1260,6 +1340,7 @@ int novak_set_tensor_rows(novak_opt *o, const int64_t *rows, int n)
     int64_t off = 0;
     for (int i = 0; i < n; ++i) { o->row_off[i] = off; off += o->rows[i]; }
     o->total_rows = total;
+    o->rows_gen += 1;
     invalidate_tables(o);
     return NOVAK_OK;
 }
@@ -1429,6 +1510,28 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     o->warnings |= in->warnings;
     o->last_plan = make_plan(h, in->t > 0 ? in->t : 1);
     return NOVAK_OK;
+}
+
+int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
+                              int64_t *row0, int64_t *n_rows, int64_t *part_off,
+                              int64_t *part_len, int64_t cap)
+{
+    if (!numel || !rows || n <= 0 || cap < 0) return -1;
+    for (int i = 0; i < n; ++i)
+        if (numel[i] <= 0 || rows[i] < 0 || (rows[i] > 0 && (numel[i] % rows[i] != 0 ||
+                                                             numel[i] >= (int64_t(1) << 31))))
+            return -1;
+    std::vector<RowUnit> units;
+    build_row_units(numel, rows, n, units);
+    const int64_t count = static_cast<int64_t>(units.size());
+    for (int64_t i = 0; i < count && i < cap; ++i) {
+        if (tensor) tensor[i] = units[i].tensor;
+        if (row0) row0[i] = units[i].row0;
+        if (n_rows) n_rows[i] = units[i].n_rows;
+        if (part_off) part_off[i] = units[i].part_off;
+        if (part_len) part_len[i] = units[i].part_len;
+    }
+    return count;
 }
 
 int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,

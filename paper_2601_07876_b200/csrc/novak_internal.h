@@ -116,21 +116,55 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
                                double *chunk_u2, double *chunk_p2, float *trust, int pdl,
                                cudaStream_t stream);
 
-// Launches the gradient statistics pass over the whole chunk table (two
-// kernels): the global norm of the raw gradient and the clip factor into *prep,
-// and, where a tensor record has rows, the row means of Eq. 26.  Scratch:
-// chunk_sq, seg_first, seg_last of n_chunks doubles each (seg_* may be NULL
-// when no tensor has rows) and cta_sq of grad_stats_ctas(n_chunks) doubles.
-// With auto_gamma > 0 a third kernel sums the squares of the parameters into
-// chunk_psq (n_chunks doubles; cta_sq then holds 2 x grad_stats_ctas doubles)
-// and the pass also advances the averages of Eq. 20-21 in *prep and writes
-// Eq. 22's factor there; with auto_gamma = 0 that factor is written as 1.
-int grad_stats_ctas(int n_chunks);
-cudaError_t launch_grad_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                              int grad_dtype, double c_clip, double auto_gamma, double *chunk_sq,
-                              double *chunk_psq, double *seg_first, double *seg_last,
-                              double *cta_sq, PrepOut *prep, bool any_rows, int pdl,
-                              cudaStream_t stream);
+// One unit of work of the statistics pass for a tensor with rows (Eq. 26).
+// Rows of up to kRowWarpMax elements: n_rows whole rows starting at row0
+// (part_len = 0), a warp (or, below 128 elements, a thread) per row.  Longer
+// rows: one slice [part_off, part_off + part_len) of row row0 for the whole
+// CTA; the row is cut into n_parts slices of at most kRowUnitElems elements, of
+// which this is number part_idx (units of one row are consecutive in the table).
+struct __align__(16) RowUnit {
+    int32_t tensor;
+    uint32_t row0;
+    uint32_t n_rows;
+    uint32_t part_off;
+    uint32_t part_len;
+    uint32_t n_parts;
+    uint32_t part_idx;
+    uint32_t reserved;
+};
+
+// Elements a row unit aims at, and rows per unit where a thread takes a row.
+constexpr uint32_t kRowUnitElems = 8192;
+constexpr uint32_t kRowUnitThreads = 256;
+constexpr uint32_t kRowWarpMax = 1024;     // longest row a single warp streams
+
+// What the statistics pass works on, all in device memory.
+struct StatsPlan {
+    const Chunk *plain;      // chunk-table entries of the tensors without rows
+    int n_plain;
+    const RowUnit *units;    // row units of the tensors with rows
+    int n_units;
+    const TensorRec *recs;
+    const Chunk *chunks;     // the whole chunk table (parameter norm of Eq. 21)
+    int n_chunks;
+    double *part_sq;         // grad_stats_work(n_plain, n_units, fp32) doubles (bf16 needs fewer)
+    double *part_sum;        // n_units doubles
+    double *chunk_psq;       // n_chunks doubles, NULL without Eq. 20-22
+    double *cta_sq;          // 2 x grad_stats_ctas(...) doubles
+    PrepOut *prep;
+};
+
+// CTAs of the first kernel (= sums of squares it leaves), CTAs of the second.
+int grad_stats_work(int n_plain, int n_units, int grad_dtype);
+int grad_stats_ctas(int n_work, int n_chunks);
+
+// Launches the gradient statistics pass (two kernels; three with auto_gamma >
+// 0, which adds the sum of squares of the parameters): the global norm of the
+// raw gradient and the clip factor into *prep, the row means of Eq. 26 into
+// the tensor records' mean arrays, and Eq. 20-22's averages and factor into
+// *prep (the factor is written as 1 when auto_gamma = 0).
+cudaError_t launch_grad_stats(const StatsPlan &plan, int grad_dtype, double c_clip,
+                              double auto_gamma, int pdl, cudaStream_t stream);
 
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.

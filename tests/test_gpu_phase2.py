@@ -181,7 +181,8 @@ def test_step_host_with_phase2_matches_step():
                            B.NOVAK_GRAD_F32, stream)
         torch.cuda.synchronize()
         assert torch.equal(h_p, torch.cat([p.reshape(-1) for p in pa]).cpu())
-    assert a.grad_stats() == b.grad_stats()
+    # the two gradient buffers are aligned differently, so the sums run in another order
+    np.testing.assert_allclose(a.grad_stats(), b.grad_stats(), rtol=1e-7)
 
 
 def test_fullsize_resnet50_with_clipping_and_centralization():
