@@ -75,3 +75,43 @@ def test_partition_covers_every_element_once(world):
     assert max(sizes) - min(sizes) <= 64 + 63
     flat = [(t, a) for slices in parts for t, a, _ in slices]
     assert flat == sorted(flat)                            # contiguous, in order
+
+
+def _paper_constants():
+    path = os.path.join(os.path.dirname(__file__), "golden", "constants_sections_4_and_5.txt")
+    out = {}
+    for line in open(path):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            out[line[0]] = float(line[1])
+    return out
+
+
+def test_library_defaults_and_oracle_follow_the_constants_the_paper_prints():
+    import numpy as np
+    from oracle import novak_oracle as O
+    from paper_2601_07876_b200 import binding as B
+    c = _paper_constants()
+    h = B.Handle(beta1=c["beta1_default"], beta2=c["beta2_default"], eps=c["eps_default"])
+    assert h.get_option(B.NOVAK_OPT_BETA1_TAU) == c["tau1"]
+    assert h.get_option(B.NOVAK_OPT_BETA2_TAU) == c["tau2"]
+    assert h.get_option(B.NOVAK_OPT_AUTO_LR_GAMMA) == c["auto_lr_gamma"]
+    assert h.get_option(B.NOVAK_OPT_CLIP_THRESHOLD) == 0.0        # off unless asked for
+    # Eq. 6 and the threshold of Eq. 8, in the library's plan and in the oracle
+    o = O.Oracle(O.Config(beta1=c["beta1_default"], beta2=c["beta2_default"]), [np.zeros(1)])
+    assert abs(h.plan(1).rho_inf - c["rho_inf_beta2_0.999"]) < 1e-9
+    assert abs(o.scalars(1).rho_inf - c["rho_inf_beta2_0.999"]) < 1e-9
+    for t in range(1, 40):
+        for plan in (h.plan(t), o.scalars(t)):
+            assert plan.rect_branch == (1 if plan.rho_t >= c["rectification_threshold"] else 0)
+    assert [h.plan(t).rect_branch for t in (5, 6)] == [0, 1]
+    # the clip ranges of Eq. 19 and Eq. 22, in the oracle
+    for scale, lo_hi in ((1e-6, "low"), (1e6, "high")):
+        o = O.Oracle(O.Config(lookahead_k=0, layer_adaptation=True, auto_lr=True),
+                     [np.full(8, scale)])
+        o.step([np.full(8, 1.0 / scale)])
+        assert o.trust[0][0] == c[f"trust_clip_{lo_hi}"]
+        # the gradient scale runs the other way: tiny parameters, huge gradient -> upper bound
+        assert o.auto_scales[0] == c["auto_lr_clip_high" if lo_hi == "low" else "auto_lr_clip_low"]
+    assert O.Config().tau1 == c["tau1"] and O.Config().tau2 == c["tau2"]
+    assert O.Config().auto_lr_gamma == c["auto_lr_gamma"]
