@@ -10,7 +10,7 @@
 // Decomposition.  Tensors without rows: one CTA per 4 consecutive chunk-table
 // entries (the table of the step kernel), sum of squares only.  Tensors with
 // rows: a table of row units built on the host, aligned to ROWS, not to the
-// chunk table: a unit is a group of whole rows of up to 1024 elements (a warp
+// chunk table: a unit is a group of whole rows of up to 2048 elements (a warp
 // streams each row, or a thread for rows shorter than 128 elements), or a
 // slice of at most 8192 elements of a longer row (the whole CTA; usually the
 // whole row).  No shared-memory

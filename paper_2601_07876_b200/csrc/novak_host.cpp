@@ -149,7 +149,9 @@ void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vect
         } else {
             // a warp per row from 128 elements on (at least one row for each of the
             // CTA's 8 warps), else a thread per row
-            const uint32_t per = L >= 128u ? std::max(8u, novak::kRowUnitElems / L)
+            // (rows per unit a multiple of 8, so that no warp idles while others take a
+            // second row)
+            const uint32_t per = L >= 128u ? std::max(8u, novak::kRowUnitElems / L / 8u * 8u)
                                            : novak::kRowUnitThreads;
             for (uint32_t r = 0; r < R; r += per)
                 out.push_back(RowUnit{i, r, std::min(per, R - r), 0u, 0u, 1u, 0u, 0u});

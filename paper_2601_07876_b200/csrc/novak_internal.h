@@ -117,7 +117,8 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
                                cudaStream_t stream);
 
 // One unit of work of the statistics pass for a tensor with rows (Eq. 26).
-// Rows of up to kRowWarpMax elements: n_rows whole rows starting at row0
+// Rows of up to kRowWarpMax elements: n_rows (a multiple of 8 but for a tensor's
+// last unit) whole rows starting at row0
 // (part_len = 0), a warp (or, below 128 elements, a thread) per row.  Longer
 // rows: one slice [part_off, part_off + part_len) of row row0 for the whole
 // CTA; the row is cut into n_parts slices of at most kRowUnitElems elements, of
@@ -136,7 +137,7 @@ struct __align__(16) RowUnit {
 // Elements a row unit aims at, and rows per unit where a thread takes a row.
 constexpr uint32_t kRowUnitElems = 8192;
 constexpr uint32_t kRowUnitThreads = 256;
-constexpr uint32_t kRowWarpMax = 1024;     // longest row a single warp streams
+constexpr uint32_t kRowWarpMax = 2048;     // longest row a single warp streams
 
 // What the statistics pass works on, all in device memory.
 struct StatsPlan {
