@@ -246,6 +246,38 @@ int novak_step(novak_opt *opt, void *const *d_params,
                const void *const *d_grads, const int64_t *numel, int n,
                int grad_dtype, void *stream);
 
+/* One step in two halves, for a group that is cut across several processes
+ * (each owning a range of the flattened parameters and calling the library on
+ * its own range) AND uses gradient clipping or the automatic learning-rate
+ * scaling, whose norms run over the whole group (Section 5.8: with sharded
+ * state the step needs this one exchange):
+ *
+ *   novak_step_begin(...)          this process's statistics: sums of squares of
+ *                                  its gradients (and parameters)
+ *   novak_local_sums(opt, &d)      d[0..1]: those two sums, in device memory
+ *   <caller: all-reduce (sum) of the two doubles over the group's processes,
+ *    e.g. NCCL on the same stream, into any device buffer>
+ *   novak_step_finish(opt, d_total_sums, stream)
+ *                                  norm, clip factor, Eq. 20-22 from the totals,
+ *                                  then the update of this process's range
+ *
+ * Arguments of begin as novak_step.  d_total_sums: device pointer to the two
+ * all-reduced doubles; NULL takes the local ones (then the pair equals
+ * novak_step).  Between begin and finish no other step call is allowed on the
+ * handle (NOVAK_ESTATE), and the gradients must stay unchanged.  With neither
+ * clipping nor auto-LR on, begin enqueues nothing and finish is the plain step.
+ * Centralization and layer adaptation work on whole tensors and are refused
+ * here (NOVAK_ESTATE).  Both calls enqueue on `stream` and return without
+ * synchronising. */
+int novak_step_begin(novak_opt *opt, void *const *d_params, const void *const *d_grads,
+                     const int64_t *numel, int n, int grad_dtype, void *stream);
+int novak_local_sums(novak_opt *opt, double **d_sums);
+/* The same two sums copied (device to device, on `stream`) into a buffer of the
+ * caller's, e.g. the tensor its collective library reduces; zeros when the open
+ * step needed no statistics. */
+int novak_copy_local_sums(novak_opt *opt, double *d_dst, void *stream);
+int novak_step_finish(novak_opt *opt, const double *d_total_sums, void *stream);
+
 /* The same step for a caller whose gradients arrive in, and whose updated
  * parameters return to, HOST memory (pinned memory, or the copies do not
  * overlap anything).  The chunk table is cut into runs of about

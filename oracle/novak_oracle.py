@@ -228,6 +228,8 @@ class Oracle:
             numel = (ctypes.c_int64 * n)(*[g.size for g in gs])
             ptrs = (ctypes.POINTER(ctypes.c_double) * n)(*[_dptr(g) for g in gs])
             norm = self.lib.novak_oracle_global_norm(n, numel, ptrs)
+            if getattr(self, "_norms", None):
+                norm = self._norms[0]
             factor = self.lib.novak_oracle_clip_factor(norm, cfg.clip_threshold)
             self.grad_norms.append(norm)
             self.clip_factors.append(factor)
@@ -241,10 +243,20 @@ class Oracle:
                     self.lib.novak_oracle_centralize(r, g.size // r, _dptr(g))
         return gs
 
-    def step(self, grads, threads: int = 1):
+    def local_sums(self, grads):
+        """(sum of squares of these gradients, sum of squares of the parameters): what one
+        process of a sharded group contributes to the norms of the whole group."""
+        gs = [np.ascontiguousarray(np.asarray(g, dtype=np.float64)).reshape(-1) for g in grads]
+        return self._global_norm(gs) ** 2, self._global_norm(self.theta) ** 2
+
+    def step(self, grads, threads: int = 1, global_sums=None):
         """One step.  ``threads`` > 1 splits each tensor into disjoint element
-        ranges handled by separate host threads (elements are independent)."""
+        ranges handled by separate host threads (elements are independent).
+        ``global_sums``: (sum of g^2, sum of theta^2) over the WHOLE group when this
+        oracle holds only a shard of it; the norms then come from these."""
         assert len(grads) == len(self.theta)
+        self._norms = (None if global_sums is None
+                       else (float(np.sqrt(global_sums[0])), float(np.sqrt(global_sums[1]))))
         self.t += 1
         s = self.scalars(self.t)
         self.rect_flags.append(int(s.rect_branch))
@@ -257,7 +269,9 @@ class Oracle:
         auto = 1.0
         if self.cfg.auto_lr:
             auto = self.lib.novak_oracle_auto_lr(
-                self.cfg.auto_lr_gamma, self._global_norm(gs), self._global_norm(self.theta),
+                self.cfg.auto_lr_gamma,
+                self._norms[0] if self._norms else self._global_norm(gs),
+                self._norms[1] if self._norms else self._global_norm(self.theta),
                 ctypes.byref(self.g_bar), ctypes.byref(self.theta_bar))
             self.auto_scales.append(auto)
         gs = self.process_gradients(gs)

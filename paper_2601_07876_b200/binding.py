@@ -107,6 +107,10 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_attach_state": (c_int, [vp, vp, c_size_t, vpp, i64p, c_int, vp]),
         "novak_step": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_step_noalloc": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_step_begin": (c_int, [vp, vpp, vpp, i64p, c_int, c_int, vp]),
+        "novak_local_sums": (c_int, [vp, POINTER(c_void_p)]),
+        "novak_copy_local_sums": (c_int, [vp, vp, vp]),
+        "novak_step_finish": (c_int, [vp, vp, vp]),
         "novak_step_host": (c_int, [vp, vpp, vpp, vpp, vpp, i64p, c_int, c_int, vp]),
         "novak_set_tensor_rows": (c_int, [vp, i64p, c_int]),
         "novak_set_param_copies": (c_int, [vp, vpp, c_int]),
@@ -232,6 +236,26 @@ class Handle:
         st = self.lib.novak_step(self.h, params_arr, grads_arr, numel_arr, n, grad_dtype, stream)
         if st != NOVAK_OK:
             _check(self.lib, self.h, st, "novak_step")
+
+    def step_begin(self, params_arr, grads_arr, numel_arr, n: int, grad_dtype: int,
+                   stream: int = 0):
+        _check(self.lib, self.h,
+               self.lib.novak_step_begin(self.h, params_arr, grads_arr, numel_arr, n, grad_dtype,
+                                         stream), "novak_step_begin")
+
+    def local_sums(self) -> int:
+        """Device address of the two local sums of squares (0 when no statistics ran)."""
+        p = c_void_p()
+        _check(self.lib, self.h, self.lib.novak_local_sums(self.h, byref(p)), "novak_local_sums")
+        return p.value or 0
+
+    def copy_local_sums(self, d_dst: int, stream: int = 0):
+        _check(self.lib, self.h, self.lib.novak_copy_local_sums(self.h, d_dst, stream),
+               "novak_copy_local_sums")
+
+    def step_finish(self, d_total_sums: int = 0, stream: int = 0):
+        _check(self.lib, self.h, self.lib.novak_step_finish(self.h, d_total_sums or None, stream),
+               "novak_step_finish")
 
     def step_noalloc(self, params_arr, grads_arr, numel_arr, n: int, grad_dtype: int,
                      stream: int = 0):
@@ -460,6 +484,25 @@ class NovakOptimizer:
         self.handle.step(self._params_arr, gl.arr, self._numel_arr, self.n, gl.dtype,
                          self._stream())
         self._last_grads = gl
+
+    def step_begin(self, grads):
+        """First half of a step for a group cut across processes: local statistics.
+        Returns the device address of the two local sums of squares (0: none needed)."""
+        gl = grads if isinstance(grads, GradList) else self.prepare(grads)
+        self.handle.step_begin(self._params_arr, gl.arr, self._numel_arr, self.n, gl.dtype,
+                               self._stream())
+        self._last_grads = gl
+        return self.handle.local_sums()
+
+    def copy_local_sums(self, out):
+        """Copies the open step's two local sums into ``out`` (CUDA float64, 2 elements)."""
+        self.handle.copy_local_sums(out.data_ptr(), self._stream())
+
+    def step_finish(self, total_sums=None):
+        """Second half: ``total_sums`` is a CUDA float64 tensor of 2 elements holding the
+        all-reduced sums (None: the local ones)."""
+        ptr = total_sums.data_ptr() if total_sums is not None else 0
+        self.handle.step_finish(ptr, self._stream())
 
     def info(self) -> dict:
         return self.handle.get_info().as_dict()

@@ -436,6 +436,48 @@ novak_param_sumsq_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
 }
 
+// From the sums of squares to what the step kernel reads: the norm of the
+// gradient and the clip factor (Table 2: active when ||g|| > c_clip), and,
+// with has_p, the averages and the factor of Eq. 20-22 on the norm of the
+// gradient as given and of theta_t.  One thread.
+__device__ __forceinline__ void write_scalars(PrepOut *out, double sumsq, double psumsq,
+                                              double c_clip, double auto_gamma, bool has_p)
+{
+    const double norm = sqrt(sumsq);
+    const double factor = (c_clip > 0.0 && norm > c_clip) ? c_clip / norm : 1.0;
+    out->norm = norm;
+    out->factor = static_cast<float>(factor);
+    float scale = 1.0f;
+    if (has_p && auto_gamma > 0.0) {
+        const double pnorm = sqrt(psumsq);
+        const double g_bar = auto_gamma * norm + (1.0 - auto_gamma) * out->g_bar;
+        const double theta_bar = auto_gamma * pnorm + (1.0 - auto_gamma) * out->theta_bar;
+        double a = 1.0;              // 0/0: undefined, taken as 1
+        if (!(g_bar == 0.0 && theta_bar == 0.0)) {
+            a = g_bar / theta_bar;
+            a = a < 0.1 ? 0.1 : (a > 2.0 ? 2.0 : a);
+        }
+        out->pnorm = pnorm;
+        out->g_bar = g_bar;
+        out->theta_bar = theta_bar;
+        scale = static_cast<float>(a);
+    }
+    out->auto_scale = scale;
+}
+
+// For a group that is sharded over several processes: the sums of squares of
+// the WHOLE group (this process's local_sums, all-reduced by the caller) turned
+// into norm, clip factor and Eq. 20-22.  One thread.
+__global__ void novak_grad_norm_scalar_kernel(PrepOut *__restrict__ out,
+                                              const double *__restrict__ totals, double c_clip,
+                                              double auto_gamma, int has_p)
+{
+    grid_dependency_release();
+    grid_dependency_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        write_scalars(out, totals[0], totals[1], c_clip, auto_gamma, has_p != 0);
+}
+
 // Second kernel of the pass, one THREAD per sum of the first: completes the
 // means of the long rows that were cut into slices (the thread of a row's first
 // slice adds the slices in order) and adds up the sums of squares: per CTA
@@ -447,7 +489,7 @@ novak_grad_stats_finish_kernel(const RowUnit *__restrict__ units, int n_units,
                                const double *__restrict__ part_sq,
                                const double *__restrict__ part_sum, int n_chunks,
                                const double *__restrict__ chunk_psq, double c_clip,
-                               double auto_gamma, double *__restrict__ cta_sq,
+                               double auto_gamma, int finalize, double *__restrict__ cta_sq,
                                PrepOut *__restrict__ out)
 {
     __shared__ double sh[kStatsWarps];
@@ -491,28 +533,10 @@ novak_grad_stats_finish_kernel(const RowUnit *__restrict__ units, int n_units,
     const double sumsq = block_sum(t, sh);
     const double psumsq = chunk_psq != nullptr ? block_sum(tp, sh) : 0.0;
     if (threadIdx.x == 0) {
-        const double norm = sqrt(sumsq);
-        // Table 2: clipping is active when ||g|| > c_clip
-        const double factor = (c_clip > 0.0 && norm > c_clip) ? c_clip / norm : 1.0;
-        out->norm = norm;
-        out->factor = static_cast<float>(factor);
-        float scale = 1.0f;
-        if (chunk_psq != nullptr && auto_gamma > 0.0) {
-            // Eq. 20-22 on the norm of the gradient as given and of theta_t
-            const double pnorm = sqrt(psumsq);
-            const double g_bar = auto_gamma * norm + (1.0 - auto_gamma) * out->g_bar;
-            const double theta_bar = auto_gamma * pnorm + (1.0 - auto_gamma) * out->theta_bar;
-            double a = 1.0;              // 0/0: undefined, taken as 1
-            if (!(g_bar == 0.0 && theta_bar == 0.0)) {
-                a = g_bar / theta_bar;
-                a = a < 0.1 ? 0.1 : (a > 2.0 ? 2.0 : a);
-            }
-            out->pnorm = pnorm;
-            out->g_bar = g_bar;
-            out->theta_bar = theta_bar;
-            scale = static_cast<float>(a);
-        }
-        out->auto_scale = scale;
+        // what this process saw; a sharded group all-reduces these two before the scalars
+        out->local_sums[0] = sumsq;
+        out->local_sums[1] = psumsq;
+        if (finalize) write_scalars(out, sumsq, psumsq, c_clip, auto_gamma, chunk_psq != nullptr);
     }
 }
 
@@ -550,8 +574,26 @@ int grad_stats_ctas(int n_work, int n_chunks)
     return (n + kStatsBlock - 1) / kStatsBlock;
 }
 
+cudaError_t launch_grad_norm_scalars(PrepOut *prep, const double *d_totals, double c_clip,
+                                     double auto_gamma, int pdl, cudaStream_t stream)
+{
+    if (!prep || !d_totals) return cudaErrorInvalidValue;
+    int has_p = auto_gamma > 0.0 ? 1 : 0;
+    void *args[] = {&prep, &d_totals, &c_clip, &auto_gamma, &has_p};
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(1);
+    lc.blockDim = dim3(32);
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (pdl & 4) ? 1 : 0;
+    return cudaLaunchKernelExC(&lc, reinterpret_cast<const void *>(novak_grad_norm_scalar_kernel), args);
+}
+
 cudaError_t launch_grad_stats(const StatsPlan &w, int grad_dtype, double c_clip, double auto_gamma,
-                              int pdl, cudaStream_t stream)
+                              bool finalize, int pdl, cudaStream_t stream)
 {
     const int n_work = grad_stats_work(w.n_plain, w.n_units, grad_dtype);
     if (n_work <= 0 || !w.recs || !w.part_sq || !w.cta_sq || !w.prep) return cudaErrorInvalidValue;
@@ -584,9 +626,10 @@ cudaError_t launch_grad_stats(const StatsPlan &w, int grad_dtype, double c_clip,
         c_psq = a.chunk_psq;
     }
     int work = n_work;
+    int fin = finalize ? 1 : 0;
     const double *c_sq = a.part_sq, *c_sum = a.part_sum;
     void *args2[] = {&a.units, &a.n_units, &a.recs, &work, &c_sq, &c_sum, &a.n_chunks, &c_psq,
-                     &c_clip, &auto_gamma, &a.cta_sq, &a.prep};
+                     &c_clip, &auto_gamma, &fin, &a.cta_sq, &a.prep};
     return launch_pdl(reinterpret_cast<const void *>(novak_grad_stats_finish_kernel),
                       static_cast<unsigned>(grad_stats_ctas(n_work, c_psq ? a.n_chunks : 0)), args2,
                       (pdl & 4) != 0, stream);

@@ -224,6 +224,10 @@ struct novak_opt {
     int64_t rows_gen = 0;               // bumped whenever the row settings change
     int64_t prep_key = -1;              // rows_gen and centring the scratch was laid out for
     // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
+    // a step taken in two halves (novak_step_begin / novak_step_finish)
+    bool half_open = false;
+    int half_launches = 0;
+    alignas(8) unsigned char half_ctx[256] = {};   // the StepCtx of the open step
     bool ema_pending = false;
     double pending_g_bar = 0.0, pending_theta_bar = 0.0;
     float2 *row_mean = nullptr;
@@ -862,6 +866,7 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
     o->row_off.assign(n, 0);
     o->total_rows = 0;
     o->copies.clear();
+    o->half_open = false;
     o->ema_pending = false;
     o->t = 0; o->n_syncs = 0; o->last_sync = 0;
     o->attached = true;
@@ -911,6 +916,8 @@ int check_step_args(novak_opt *o, const char *who, void *const *d_params,
                     const void *const *d_grads, const int64_t *numel, int n, int grad_dtype)
 {
     if (!o->attached) return fail(o, NOVAK_ESTATE, "%s: no state attached", who);
+    if (o->half_open && std::strcmp(who, "step_begin") != 0)
+        return fail(o, NOVAK_ESTATE, "%s: a step begun with novak_step_begin is still open", who);
     if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "%s: NULL argument", who);
     if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16)
         return fail(o, NOVAK_EINVAL, "%s: unknown grad_dtype %d", who, grad_dtype);
@@ -953,16 +960,21 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
 // Everything that has to see the whole group before the first element is
 // updated: phase 2's statistics, then phase 7's trust ratios.  Returns the
 // number of kernels launched through *launches.
-cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream);
-cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, int *launches,
-                             const char **what)
+cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, bool finalize, cudaStream_t stream);
+cudaError_t launch_statistics(novak_opt *o, const StepCtx &ctx, bool finalize, cudaStream_t stream,
+                              int *launches, const char **what)
+{
+    if (ctx.pre == novak::PRE_NONE) return cudaSuccess;
+    *what = "gradient statistics kernel launch";
+    const cudaError_t e = launch_stats(o, ctx, finalize, stream);
+    if (e == cudaSuccess) *launches += o->h.auto_lr ? 3 : 2;
+    return e;
+}
+
+cudaError_t launch_trust(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, int *launches,
+                         const char **what)
 {
     cudaError_t e;
-    if (ctx.pre != novak::PRE_NONE) {
-        *what = "gradient statistics kernel launch";
-        if ((e = launch_stats(o, ctx, stream)) != cudaSuccess) return e;
-        *launches += o->h.auto_lr ? 3 : 2;
-    }
     if (ctx.trust) {
         *what = "layer adaptation kernel launch";
         e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
@@ -974,8 +986,15 @@ cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stre
     return cudaSuccess;
 }
 
+cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, int *launches,
+                             const char **what)
+{
+    const cudaError_t e = launch_statistics(o, ctx, true, stream, launches, what);
+    return e != cudaSuccess ? e : launch_trust(o, ctx, stream, launches, what);
+}
+
 // Phase 2's statistics pass over the whole group: global norm, clip factor, row means.
-cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream)
+cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, bool finalize, cudaStream_t stream)
 {
     novak::StatsPlan plan;
     plan.plain = o->d_plain ? o->d_plain : o->d_chunks;
@@ -991,7 +1010,7 @@ cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, cudaStream_t stream)
     plan.cta_sq = o->cta_sq;
     plan.prep = o->prep_out;
     return novak::launch_grad_stats(plan, ctx.grad_dtype, o->h.clip,
-                                    o->h.auto_lr ? o->h.auto_gamma : 0.0, o->pdl, stream);
+                                    o->h.auto_lr ? o->h.auto_gamma : 0.0, finalize, o->pdl, stream);
 }
 
 // One launch over chunk-table entries [c0, c1).
@@ -1115,6 +1134,76 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
         return fail_cuda(o, e, what);
     if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess)
         return fail_cuda(o, e, "step kernel launch");
+    commit_step(o, ctx, launches);
+    return NOVAK_OK;
+}
+
+int novak_step_begin(novak_opt *o, void *const *d_params, const void *const *d_grads,
+                     const int64_t *numel, int n, int grad_dtype, void *stream_)
+{
+    static_assert(sizeof(StepCtx) <= sizeof(o->half_ctx), "room for the open step");
+    if (!o) return NOVAK_EINVAL;
+    int rc = check_step_args(o, "step_begin", d_params, d_grads, numel, n, grad_dtype);
+    if (rc != NOVAK_OK) return rc;
+    if (o->half_open) return fail(o, NOVAK_ESTATE, "step_begin: the previous step was not finished");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    StepCtx ctx;
+    if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
+    if (ctx.pre == novak::PRE_CENTER || ctx.trust)
+        return fail(o, NOVAK_ESTATE, "step_begin: centralization and layer adaptation need whole "
+                    "tensors and are not available for a group cut across processes");
+    int launches = 0;
+    const char *what = "";
+    const cudaError_t e = launch_statistics(o, ctx, false, stream, &launches, &what);
+    if (e != cudaSuccess) return fail_cuda(o, e, what);
+    std::memcpy(o->half_ctx, &ctx, sizeof ctx);
+    o->half_launches = launches;
+    o->half_open = true;
+    return NOVAK_OK;
+}
+
+int novak_local_sums(novak_opt *o, double **d_sums)
+{
+    if (!o || !d_sums) return NOVAK_EINVAL;
+    if (!o->half_open) return fail(o, NOVAK_ESTATE, "local_sums: no step is open");
+    *d_sums = o->prep_out ? o->prep_out->local_sums : nullptr;
+    return NOVAK_OK;
+}
+
+int novak_copy_local_sums(novak_opt *o, double *d_dst, void *stream_)
+{
+    if (!o || !d_dst) return NOVAK_EINVAL;
+    if (!o->half_open) return fail(o, NOVAK_ESTATE, "copy_local_sums: no step is open");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    cudaError_t e;
+    if (o->prep_out)
+        e = cudaMemcpyAsync(d_dst, o->prep_out->local_sums, 2 * sizeof(double),
+                            cudaMemcpyDeviceToDevice, stream);
+    else
+        e = cudaMemsetAsync(d_dst, 0, 2 * sizeof(double), stream);   // no statistics: nothing to add
+    if (e != cudaSuccess) return fail_cuda(o, e, "copy_local_sums");
+    return NOVAK_OK;
+}
+
+int novak_step_finish(novak_opt *o, const double *d_total_sums, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    if (!o->half_open) return fail(o, NOVAK_ESTATE, "step_finish: no step is open");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    StepCtx ctx;
+    std::memcpy(&ctx, o->half_ctx, sizeof ctx);
+    int launches = o->half_launches + 1;
+    cudaError_t e;
+    if (ctx.pre != novak::PRE_NONE) {
+        const double *totals = d_total_sums ? d_total_sums : o->prep_out->local_sums;
+        e = novak::launch_grad_norm_scalars(o->prep_out, totals, o->h.clip,
+                                            o->h.auto_lr ? o->h.auto_gamma : 0.0, o->pdl, stream);
+        if (e != cudaSuccess) return fail_cuda(o, e, "gradient norm kernel launch");
+        ++launches;
+    }
+    if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "step kernel launch");
+    o->half_open = false;
     commit_step(o, ctx, launches);
     return NOVAK_OK;
 }

@@ -88,8 +88,13 @@ int grad_stats_ctas(int n_work, int n_chunks);
 // raw gradient and the clip factor into *prep, the row means of Eq. 26 into
 // the tensor records' mean arrays, and Eq. 20-22's averages and factor into
 // *prep (the factor is written as 1 when auto_gamma = 0).
+// With finalize = false the pass stops at prep->local_sums (this process's sums
+// of squares of gradients and parameters) and launch_grad_norm_scalars, given
+// the all-reduced sums of the whole group, forms norm and factors.
 cudaError_t launch_grad_stats(const StatsPlan &plan, int grad_dtype, double c_clip,
-                              double auto_gamma, int pdl, cudaStream_t stream);
+                              double auto_gamma, bool finalize, int pdl, cudaStream_t stream);
+cudaError_t launch_grad_norm_scalars(PrepOut *prep, const double *d_totals, double c_clip,
+                                     double auto_gamma, int pdl, cudaStream_t stream);
 
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.

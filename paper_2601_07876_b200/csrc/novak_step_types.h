@@ -81,6 +81,9 @@ struct __align__(16) PrepOut {
     double theta_bar;  // Eq. 21
     float auto_scale;  // Eq. 22, 1 when the scaling is off
     float reserved;
+    // sums of squares of this process's gradients and parameters; a group sharded over
+    // several processes all-reduces the two before norm and factors are formed
+    double local_sums[2];
 };
 
 }  // namespace novak

@@ -9,10 +9,12 @@ only 1/world of the optimizer state.  One step:
 The NOVAK step has no cross-element term, so the owned range may cut tensors
 anywhere; nothing is exchanged inside the step itself, and the ranks only have
 to take the same number of steps for their lookahead synchronisations to
-coincide.  Options that need a statistic of the WHOLE group (clipping,
-centralization, layer adaptation, automatic learning-rate scaling) would need
-an extra all-reduce between their statistics pass and the step; that is not
-built, and this class refuses them.
+coincide.  Two options need a norm over the WHOLE group, gradient clipping and
+the automatic learning-rate scaling: for them the step runs in two halves
+(novak_step_begin / novak_step_finish) with one all-reduce of two doubles (the
+ranks' sums of squares of gradients and parameters) in between.
+Centralization and layer adaptation work on whole tensors, which an arbitrary
+cut of the flat space does not keep together: this class refuses them.
 
 Only argument marshalling and collectives live here: the local step is
 whatever ``make_local`` returns (the CUDA optimizer on a GPU; the tests plug in
@@ -50,9 +52,10 @@ class ShardedNovak:
         self.total = sum(self.numel)
         if flat_params.dim() != 1 or flat_params.numel() != padded_numel(self.total, self.world):
             raise ValueError("flat_params must be a 1-d buffer of padded_numel(total, world) elements")
-        for key in ("clip_threshold", "centralize", "layer_adaptation", "auto_lr"):
+        for key in ("centralize", "layer_adaptation"):
             if hyper.get(key):
-                raise ValueError(f"{key} needs a statistic of the whole group: not available sharded")
+                raise ValueError(f"{key} works on whole tensors: not available for a flat-range shard")
+        self.two_halves = bool(hyper.get("clip_threshold") or hyper.get("auto_lr"))
         self.flat_params = flat_params
         self.shard = flat_params.numel() // self.world
         lo = self.rank * self.shard
@@ -65,6 +68,7 @@ class ShardedNovak:
             from .binding import NovakOptimizer
             make_local = lambda ps: NovakOptimizer(ps, **hyper) if ps else None
         self.local = make_local(pieces)
+        self.totals = torch.zeros(2, dtype=torch.float64, device=flat_params.device)
         self.steps = 0
 
     def _flat_ranges(self):
@@ -102,9 +106,20 @@ class ShardedNovak:
         else:
             dist.reduce_scatter_tensor(self.grad_shard, flat_grads, op=dist.ReduceOp.AVG,
                                        group=self.group)
-        if self.local is not None:
-            lo = self.lo
-            self.local.step([self.grad_shard[a - lo:b - lo] for a, b in self._flat_ranges()])
+        lo = self.lo
+        grads = [self.grad_shard[a - lo:b - lo] for a, b in self._flat_ranges()]
+        if not self.two_halves:
+            if self.local is not None:
+                self.local.step(grads)
+        else:
+            # local sums of squares -> all-reduce of two doubles -> norm, factors, update
+            self.totals.zero_()
+            if self.local is not None:
+                self.local.step_begin(grads)
+                self.local.copy_local_sums(self.totals)
+            dist.all_reduce(self.totals, op=dist.ReduceOp.SUM, group=self.group)
+            if self.local is not None:
+                self.local.step_finish(self.totals)
         self.steps += 1
         # every rank's updated range lands in every rank's own buffer
         dist.all_gather_into_tensor(self.flat_params, self.param_shard, group=self.group)

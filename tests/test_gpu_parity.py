@@ -427,8 +427,9 @@ def test_step_host_matches_step_and_returns_parameters(segment_elems, gdtype):
 
 def test_zero1_wrapper_drives_the_cuda_step_world_1():
     """One rank over NCCL: reduce-scatter and all-gather degenerate to copies, the local
-    CUDA step runs on views of the flat buffer and matches the oracle; options that need
-    a statistic of the whole group are refused."""
+    CUDA step runs on views of the flat buffer and matches the oracle, also with clipping
+    and auto-LR (two-half step, all-reduce of the sums of squares); options that need whole
+    tensors are refused."""
     import os
     import socket
     import torch.distributed as dist
@@ -458,7 +459,21 @@ def test_zero1_wrapper_drives_the_cuda_step_world_1():
         assert_close(flat_p[:total], oracle.theta[0], "zero1 theta")
         assert bool((flat_p[total:] == 0).all())
         assert opt.local.info()["t"] == 6 and opt.local.info()["n_syncs"] == 1
+        # clipping and auto-LR go through the two-half step with an all-reduce of two doubles
+        hyper = dict(BASE, clip_threshold=0.05, auto_lr=True)
+        flat_q = torch.zeros(n, device=DEV)
+        flat_q[:total].normal_(0.0, 0.05, generator=gen)
+        oracle = O.Oracle(oracle_config(dict(hyper)), [to_f64(flat_q[:total])])
+        opt = zero1.ShardedNovak(flat_q, numel, **hyper)
+        for _ in range(6):
+            flat_g = torch.zeros(n, device=DEV)
+            flat_g[:total].normal_(0.0, 1e-2, generator=gen)
+            oracle.step([to_f64(flat_g[:total])])
+            opt.step(flat_g)
+        torch.cuda.synchronize()
+        assert_close(flat_q[:total], oracle.theta[0], "zero1 clipped theta")
+        assert min(oracle.clip_factors) < 1.0
         with pytest.raises(ValueError):
-            zero1.ShardedNovak(flat_p, numel, clip_threshold=1.0, **BASE)
+            zero1.ShardedNovak(flat_p, numel, centralize=True, **BASE)
     finally:
         dist.destroy_process_group()

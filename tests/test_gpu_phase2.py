@@ -417,3 +417,69 @@ def test_auto_lr_state_survives_a_checkpoint_and_a_change_of_rows():
         c.handle.set_auto_lr_state(-1.0, 0.0)
     with pytest.raises(B.NovakError):
         c.handle.set_option(B.NOVAK_OPT_AUTO_LR_GAMMA, 0.0)
+
+
+# ---------------------------------------------------------------------------
+# A step in two halves (groups cut across processes)
+# ---------------------------------------------------------------------------
+def test_two_half_step_equals_the_one_call_and_two_shards_equal_the_whole():
+    numels = [70001, 33, 8192, 3000]
+    hyper = dict(BASE, clip_threshold=0.02, auto_lr=True)
+
+    def fresh(ns, seed):
+        _, views, _ = make_tensors(ns, DEV)
+        g = _gen(seed)
+        for p in views:
+            p.normal_(0.0, 0.05, generator=g)
+        return views
+
+    whole = fresh(numels, 5)
+    halves = fresh(numels, 5)
+    pair = Pair(whole, hyper)
+    two = B.NovakOptimizer(halves, **hyper)                 # begin + finish(NULL)
+    # the same group cut into two "ranks": tensors 0-1 and tensors 2-3
+    cut = fresh(numels, 5)
+    ranks = [B.NovakOptimizer(cut[:2], **hyper), B.NovakOptimizer(cut[2:], **hyper)]
+    totals = torch.zeros(2, dtype=torch.float64, device=DEV)
+    part = torch.zeros(2, dtype=torch.float64, device=DEV)
+    gen = _gen(6)
+    _, grads, _ = make_tensors(numels, DEV)
+    for _ in range(7):
+        _fill_grads(grads, gen, std=1e-3)
+        pair.step(grads)
+        assert two.step_begin(grads) != 0
+        with pytest.raises(B.NovakError) as e:              # nothing else while the step is open
+            two.step(grads)
+        assert e.value.status == B.NOVAK_ESTATE
+        two.step_finish(None)
+        totals.zero_()
+        for r, gs in zip(ranks, (grads[:2], grads[2:])):
+            r.step_begin(gs)
+            r.copy_local_sums(part)
+            totals += part                                   # what the all-reduce would do
+        for r in ranks:
+            r.step_finish(totals)
+    pair.check("whole group")
+    for a, b in zip(whole, halves):
+        assert torch.equal(a, b)                             # same kernels, same sums
+    for a, b in zip(whole, cut):                             # sums added in another order
+        assert torch.allclose(a, b, rtol=1e-6, atol=1e-9)
+    for r in ranks:
+        np.testing.assert_allclose(r.grad_stats(), pair.opt.grad_stats(), rtol=1e-12)
+        np.testing.assert_allclose(r.handle.get_auto_lr_state(), pair.opt.handle.get_auto_lr_state(),
+                                   rtol=1e-12)
+    assert two.info()["t"] == 7 and two.info()["launches"] == pair.opt.info()["launches"] + 7
+    with pytest.raises(B.NovakError) as e:
+        two.step_finish(None)                                # nothing open
+    assert e.value.status == B.NOVAK_ESTATE
+    _, shaped = _shaped([(6, 100)], [0])
+    gc = B.NovakOptimizer(shaped, **BASE, centralize=True)
+    _, sg = _shaped([(6, 100)], [0])
+    with pytest.raises(B.NovakError) as e:
+        gc.step_begin(sg)
+    assert e.value.status == B.NOVAK_ESTATE
+    plain = B.NovakOptimizer(fresh([100], 1), **BASE)        # no statistics: begin does nothing
+    _, pg, _ = make_tensors([100], DEV)
+    assert plain.step_begin(pg) == 0
+    plain.step_finish(None)
+    assert plain.info()["t"] == 1 and plain.info()["launches"] == 1
