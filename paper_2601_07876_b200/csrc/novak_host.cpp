@@ -215,7 +215,6 @@ struct novak_opt {
     // Scratch of the gradient statistics pass (one allocation): its result, one
     // sum of squares and two row-piece sums per chunk-table entry, the row means.
     char *d_prep = nullptr;
-    int64_t prep_rows = -1;             // total_rows the scratch was sized for
     PrepOut *prep_out = nullptr;
     double *part_sq = nullptr, *part_sum = nullptr, *cta_sq = nullptr, *chunk_psq = nullptr;
     Chunk *d_plain = nullptr;           // entries of the tensors without rows (NULL: all of them)
@@ -347,7 +346,6 @@ void release_device(novak_opt *o)
     o->trust = nullptr;
     if (o->d_prep) cudaFree(o->d_prep);
     o->d_prep = nullptr;
-    o->prep_rows = -1;
     o->prep_out = nullptr;
     o->part_sq = o->part_sum = o->cta_sq = o->chunk_psq = nullptr;
     o->d_plain = nullptr;

@@ -1,0 +1,77 @@
+"""Property tests (hypothesis) of the host-side table builders: whatever the tensor
+sizes, alignment phases, chunk lengths, row counts and world sizes, every element /
+row is covered exactly once and the documented bounds hold."""
+import numpy as np
+from hypothesis import given, settings
+from hypothesis import strategies as st
+
+from paper_2601_07876_b200 import binding as B
+from paper_2601_07876_b200 import sharding
+
+sizes = st.lists(st.integers(min_value=1, max_value=40_000), min_size=1, max_size=12)
+
+
+@settings(max_examples=60, deadline=None)
+@given(numel=sizes, data=st.data())
+def test_chunk_table_covers_every_element_once(numel, data):
+    phase = [data.draw(st.integers(0, 31)) for _ in numel]
+    chunk = data.draw(st.sampled_from([1024, 2048, 4096, 8192]))
+    t, off, ln = B.novak_build_chunks(numel, phase, chunk)
+    seen = [np.zeros(n, dtype=np.int8) for n in numel]
+    last = (-1, 0)
+    for ti, oi, li in zip(t, off, ln):
+        assert 0 < li <= chunk
+        assert (ti, oi) > last                      # tensor order, then element order
+        last = (ti, oi)
+        seen[ti][oi:oi + li] += 1
+        if oi > 0:                                  # after the head entry: 128-byte aligned
+            assert (phase[ti] + oi) % 32 == 0
+    assert all((s == 1).all() for s in seen)
+
+
+@settings(max_examples=60, deadline=None)
+@given(data=st.data())
+def test_row_units_cover_every_row_once(data):
+    n = data.draw(st.integers(1, 8))
+    numel, rows = [], []
+    for _ in range(n):
+        if data.draw(st.booleans()):
+            r = data.draw(st.integers(1, 600))
+            length = data.draw(st.sampled_from([1, 2, 3, 5, 27, 64, 127, 128, 129, 576, 1024, 2048,
+                                                2049, 4608, 8192, 8193, 20_000]))
+            numel.append(r * length)
+            rows.append(r)
+        else:
+            numel.append(data.draw(st.integers(1, 5000)))
+            rows.append(0)
+    units = B.novak_build_row_units(numel, rows)
+    seen = {i: np.zeros((r, numel[i] // r), dtype=np.int8) for i, r in enumerate(rows) if r}
+    for t, row0, n_rows, part_off, part_len in units:
+        L = numel[t] // rows[t]
+        if part_len:
+            assert L > 2048 and n_rows == 1 and part_len <= 8192
+            seen[t][row0, part_off:part_off + part_len] += 1
+        else:
+            assert L <= 2048
+            seen[t][row0:row0 + n_rows] += 1
+    assert all((s == 1).all() for s in seen.values())
+    assert {u[0] for u in units} == set(seen)
+
+
+@settings(max_examples=60, deadline=None)
+@given(numel=sizes, world=st.integers(1, 9), align=st.sampled_from([1, 4, 64]))
+def test_rank_partition_covers_every_element_once_and_is_balanced(numel, world, align):
+    parts = sharding.partition_flat(numel, world, align)
+    assert len(parts) == world
+    seen = [np.zeros(n, dtype=np.int8) for n in numel]
+    counts = []
+    for slices in parts:
+        c = 0
+        for t, a, b in slices:
+            assert 0 <= a < b <= numel[t]
+            seen[t][a:b] += 1
+            c += b - a
+        counts.append(c)
+    assert all((s == 1).all() for s in seen)
+    total = sum(numel)
+    assert max(counts) - min(counts) <= max(2 * align, total - (total // align) * align + align)
