@@ -1,0 +1,184 @@
+// The optimizer handle behind the C ABI and what the host translation units
+// (novak_host.cpp, novak_host_device.cpp, novak_host_step.cpp) share: the
+// hyperparameters, the per-step scalar plan and the helpers that cross files.
+// Private to the library.
+#pragma once
+
+#include "novak.h"
+#include "novak_internal.h"
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+namespace novak_host {
+
+using novak::Chunk;
+using novak::PrepOut;
+using novak::RowUnit;
+using novak::StepScalars;
+using novak::TensorRec;
+
+constexpr int kRing = 4;                       // pinned staging slots for tensor records
+constexpr int kRecTables = 8;                  // device record tables kept per handle
+constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763036ull;  // "NOVAKv06"
+constexpr int64_t kDefaultChunkElems = 2048;
+constexpr int kDefaultCtasPerSm = 0;
+constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
+constexpr int kMaxHostSegments = 32;
+
+struct Hyper {
+    double lr, beta1, beta2, eps, wd, beta_n, la_alpha;
+    double clip;            // c_clip of the global-norm clipping, 0: off
+    int nesterov, la_k, la_mode, rectified, bias1_power;
+    int centralize;         // Eq. 26 on tensors that were given rows
+    int layer_adapt;        // Eq. 19 / 25: one trust ratio per tensor
+    int adaptive_beta;      // Eq. 3-4
+    double tau1, tau2;      // warm-up time scales of beta1, beta2
+    double sparse_tau;      // tau of Eq. 27, 0: no mask
+    int auto_lr;            // Eq. 20-22
+    double auto_gamma;      // gamma of Eq. 20-21
+};
+
+struct Plan {
+    double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay;
+    double beta1_t, beta2_t;   // coefficients of Eq. 1-2 at this step (Eq. 3-4 when warmed up)
+    int rect_branch, is_sync;
+};
+
+struct Handle {
+    Hyper h{};
+    uint32_t warnings = 0;
+    int64_t chunk_elems = kDefaultChunkElems;
+    int ctas_per_sm = kDefaultCtasPerSm;
+    int serpentine = 0;
+    int pdl = 7;                       // bit 0: step kernel, 1: statistics, 2: its second kernel
+    int64_t host_segment_elems = kDefaultHostSegmentElems;
+
+    // state layout (fixed by novak_attach_state)
+    bool attached = false;
+    char *d_state = nullptr;
+    int n = 0;
+    int n_arrays = 0;
+    int64_t region_elems = 0;
+    int64_t total_numel = 0;
+    std::vector<int64_t> numel, slot_off;
+    std::vector<int32_t> phase;
+    std::vector<int64_t> rows, row_off;   // dimension 0 of each tensor (0: none), prefix sums
+    int64_t total_rows = 0;
+    std::vector<void *> copies;           // bf16 copies of the parameters the step also writes
+
+    // counters
+    int64_t t = 0, n_syncs = 0, last_sync = 0, launches = 0;
+    Plan last_plan{};
+    int last_grid = 0;
+
+    // device work table
+    Chunk *d_chunks = nullptr;
+    std::vector<Chunk> h_chunks;       // host copy of the device chunk table
+    int n_chunks = 0;
+    TensorRec *d_recs = nullptr;       // kRecTables tables of n records each
+    TensorRec *h_recs[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ring_ev[kRing] = {nullptr, nullptr, nullptr, nullptr};
+    int ring_pos = 0;
+    // Which (parameter, gradient) pointer lists the device tables hold.  A
+    // caller that rotates through a few gradient buffers finds its table
+    // already resident and the step enqueues nothing but the kernel.
+    struct RecTable {
+        std::vector<void *> p;
+        std::vector<const void *> g;
+        int gdtype = -1;
+        uint64_t hash = 0;
+        int64_t last_use = 0;
+    };
+    RecTable tables[kRecTables];
+    int cur_table = -1;
+    int64_t table_clock = 0;
+    int64_t record_uploads = 0;
+    int sms = 0;
+
+    // Scratch of the gradient statistics pass (one allocation): its result, one
+    // sum of squares and two row-piece sums per chunk-table entry, the row means.
+    char *d_prep = nullptr;
+    PrepOut *prep_out = nullptr;
+    double *part_sq = nullptr, *part_sum = nullptr, *cta_sq = nullptr, *chunk_psq = nullptr;
+    Chunk *d_plain = nullptr;           // entries of the tensors without rows (NULL: all of them)
+    RowUnit *d_units = nullptr;
+    int n_plain = 0, n_units = 0;
+    int64_t rows_gen = 0;               // bumped whenever the row settings change
+    int64_t prep_key = -1;              // rows_gen and centring the scratch was laid out for
+    // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
+    // a step taken in two halves (novak_step_begin / novak_step_finish)
+    bool half_open = false;
+    int half_launches = 0;
+    alignas(8) unsigned char half_ctx[256] = {};   // the StepCtx of the open step
+    bool ema_pending = false;
+    double pending_g_bar = 0.0, pending_theta_bar = 0.0;
+    float2 *row_mean = nullptr;
+
+    // Scratch of layer adaptation (one allocation): two sums of squares per
+    // chunk-table entry, where each tensor's entries start, the trust ratios.
+    char *d_trust = nullptr;
+    double *chunk_u2 = nullptr, *chunk_p2 = nullptr;
+    int *tensor_first = nullptr;
+    float *trust = nullptr;
+    std::vector<int> h_tensor_first;
+
+    // novak_step_host: the chunk table cut into segments, each with the element
+    // ranges it covers, two copy streams and the events that order them.
+    struct Range { int tensor; int64_t off, len; };
+    struct Segment { int c0, c1; std::vector<Range> ranges; };
+    std::vector<Segment> segments;
+    int64_t segments_for = -1;          // host_segment_elems the segments were cut for
+    cudaStream_t up_stream = nullptr, down_stream = nullptr;
+    std::vector<cudaEvent_t> host_ev;   // [0] start, [1] end, then (uploaded, stepped) per segment
+
+    // host copies of the work table for novak_step_noalloc (no device memory of ours)
+    std::vector<Chunk> na_chunks;
+    std::vector<TensorRec> na_recs;
+    std::vector<void *> na_p;
+    std::vector<const void *> na_g;
+    int na_gdtype = -1;
+    uint64_t na_token = 0;       // identifies this handle's upload in the shared table
+
+    std::string err;
+};
+
+}  // namespace novak_host
+
+struct novak_opt : novak_host::Handle {};
+
+namespace novak_host {
+
+// Planner (novak_host.cpp).  make_plan: Eq. 5-9 and 18 for the 1-based step t;
+// lookahead_action: the LA_* bits of step t (Eq. 28-31).
+Plan make_plan(const Hyper &h, int64_t t);
+int lookahead_action(const Hyper &h, int64_t t);
+int64_t round_up(int64_t x, int64_t a);
+void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chunk_elems,
+                  std::vector<Chunk> &out);
+void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out);
+int check_hyper(const Hyper &h, const char **why);
+
+// Error reporting: store the message in the handle, return the code.
+int fail(novak_opt *o, int code, const char *fmt, ...);
+int fail_cuda(novak_opt *o, cudaError_t e, const char *what);
+
+// State layout and mode helpers.
+int n_state_arrays(const Hyper &h);
+float *slice(const novak_opt *o, int array, int i);
+int pre_mode(const novak_opt *o);
+void fill_info(const novak_opt *o, const Plan &p, novak_info *out);
+
+// Device work tables (novak_host_device.cpp).
+void release_device(novak_opt *o);
+int prepare_device(novak_opt *o, cudaStream_t stream);
+void invalidate_tables(novak_opt *o);
+int prepare_prep(novak_opt *o, cudaStream_t stream);
+int prepare_trust(novak_opt *o, cudaStream_t stream);
+uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype);
+int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
+                    int grad_dtype, cudaStream_t stream);
+
+}  // namespace novak_host

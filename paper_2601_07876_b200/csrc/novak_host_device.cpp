@@ -1,0 +1,312 @@
+// Host side of the NOVAK step library, part 2: the device work tables of a
+// handle (chunk table, cached tensor-record tables with their pinned staging
+// ring, scratch of the statistics and layer-adaptation passes).
+#include "novak_handle.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+using namespace novak_host;
+
+namespace novak_host {
+
+void release_device(novak_opt *o)
+{
+    if (o->d_chunks) cudaFree(o->d_chunks);
+    if (o->d_recs) cudaFree(o->d_recs);
+    for (int i = 0; i < kRing; ++i) {
+        if (o->h_recs[i]) cudaFreeHost(o->h_recs[i]);
+        if (o->ring_ev[i]) cudaEventDestroy(o->ring_ev[i]);
+        o->h_recs[i] = nullptr;
+        o->ring_ev[i] = nullptr;
+    }
+    if (o->d_trust) cudaFree(o->d_trust);
+    o->d_trust = nullptr;
+    o->chunk_u2 = o->chunk_p2 = nullptr;
+    o->tensor_first = nullptr;
+    o->trust = nullptr;
+    if (o->d_prep) cudaFree(o->d_prep);
+    o->d_prep = nullptr;
+    o->prep_out = nullptr;
+    o->part_sq = o->part_sum = o->cta_sq = o->chunk_psq = nullptr;
+    o->d_plain = nullptr;
+    o->d_units = nullptr;
+    o->n_plain = o->n_units = 0;
+    o->prep_key = -1;
+    o->row_mean = nullptr;
+    for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
+    o->host_ev.clear();
+    if (o->up_stream) cudaStreamDestroy(o->up_stream);
+    if (o->down_stream) cudaStreamDestroy(o->down_stream);
+    o->up_stream = o->down_stream = nullptr;
+    o->segments.clear();
+    o->segments_for = -1;
+    o->h_chunks.clear();
+    o->d_chunks = nullptr;
+    o->d_recs = nullptr;
+    o->n_chunks = 0;
+    for (auto &tb : o->tables) {
+        tb.p.clear();
+        tb.g.clear();
+        tb.gdtype = -1;
+        tb.last_use = 0;
+    }
+    o->cur_table = -1;
+}
+
+// First step: chunk table and record buffers on the device.
+int prepare_device(novak_opt *o, cudaStream_t stream)
+{
+    cudaError_t e;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(o, e, "cudaGetDevice");
+    if ((e = cudaDeviceGetAttribute(&o->sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaDeviceGetAttribute");
+
+    std::vector<Chunk> chunks;
+    build_chunks(o->numel.data(), o->phase.data(), o->n, o->chunk_elems, chunks);
+    if (chunks.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
+
+    const size_t cbytes = chunks.size() * sizeof(Chunk);
+    const size_t rbytes = static_cast<size_t>(o->n) * sizeof(TensorRec);
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_chunks), cbytes)) != cudaSuccess) {
+        release_device(o);
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(chunk table, %zu B): %s", cbytes, cudaGetErrorString(e));
+    }
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_recs), rbytes * kRecTables)) != cudaSuccess) {
+        release_device(o);
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(tensor records, %zu B): %s", rbytes * kRecTables, cudaGetErrorString(e));
+    }
+    for (int i = 0; i < kRing; ++i) {
+        if ((e = cudaHostAlloc(reinterpret_cast<void **>(&o->h_recs[i]), rbytes, cudaHostAllocDefault)) != cudaSuccess ||
+            (e = cudaEventCreateWithFlags(&o->ring_ev[i], cudaEventDisableTiming)) != cudaSuccess) {
+            release_device(o);
+            return fail(o, NOVAK_ENOMEM, "pinned record ring: %s", cudaGetErrorString(e));
+        }
+    }
+    // The table is built once: a blocking copy keeps the host vector's
+    // lifetime trivial.  Ordered before the first launch by the stream sync.
+    if ((e = cudaMemcpyAsync(o->d_chunks, chunks.data(), cbytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess) {
+        release_device(o);
+        return fail_cuda(o, e, "chunk table upload");
+    }
+    o->n_chunks = static_cast<int>(chunks.size());
+    o->h_chunks.swap(chunks);
+    return NOVAK_OK;
+}
+
+// Forget which pointer lists the device record tables hold (their contents
+// depend on the centralization settings as well as on the pointers).
+void invalidate_tables(novak_opt *o)
+{
+    for (auto &tb : o->tables) {
+        tb.p.clear();
+        tb.g.clear();
+        tb.gdtype = -1;
+        tb.last_use = 0;
+    }
+    o->cur_table = -1;
+}
+
+// Scratch of the statistics pass, laid out when a step first needs it and
+// again when the row settings change.
+int prepare_prep(novak_opt *o, cudaStream_t stream)
+{
+    const bool centre = o->h.centralize && o->total_rows > 0;
+    const int64_t key = o->rows_gen * 2 + (centre ? 1 : 0);
+    if (o->d_prep && o->prep_key == key) return NOVAK_OK;
+    cudaError_t e;
+    if (o->d_prep) {
+        // sizes changed: keep the averages of Eq. 20-21 (the copy waits for the device)
+        if (!o->ema_pending) {
+            PrepOut old;
+            if ((e = cudaMemcpy(&old, o->prep_out, sizeof old, cudaMemcpyDeviceToHost)) != cudaSuccess)
+                return fail_cuda(o, e, "cudaMemcpy(gradient statistics)");
+            o->pending_g_bar = old.g_bar;
+            o->pending_theta_bar = old.theta_bar;
+            o->ema_pending = true;
+        }
+        cudaFree(o->d_prep);
+        o->d_prep = nullptr;
+        invalidate_tables(o);
+    }
+    // work of the pass: row units for the tensors with rows, chunk-table entries for the rest
+    std::vector<RowUnit> units;
+    std::vector<Chunk> plain;
+    if (centre) {
+        build_row_units(o->numel.data(), o->rows.data(), o->n, units);
+        for (const Chunk &c : o->h_chunks)
+            if (o->rows[c.tensor] <= 0) plain.push_back(c);
+    }
+    const size_t n_plain = centre ? plain.size() : static_cast<size_t>(o->n_chunks);
+    if (units.size() > static_cast<size_t>(INT32_MAX) / 2) return fail(o, NOVAK_EINVAL, "too many rows");
+    // sized for fp32 gradients; bf16 gradients take more entries per CTA and need less
+    const size_t n_work = static_cast<size_t>(novak::grad_stats_work(
+        static_cast<int>(n_plain), static_cast<int>(units.size()), NOVAK_GRAD_F32));
+    const size_t nc = static_cast<size_t>(o->n_chunks);
+    const size_t ctas = static_cast<size_t>(novak::grad_stats_ctas(static_cast<int>(n_work), o->n_chunks));
+    size_t off = 256;
+    const size_t off_sq = off;      off += n_work * sizeof(double);
+    const size_t off_sum = off;     off += units.size() * sizeof(double);
+    const size_t off_psq = off;     off += nc * sizeof(double);
+    const size_t off_cta = off;     off += 2 * ctas * sizeof(double);
+    off = (off + 15) / 16 * 16;
+    const size_t off_plain = off;   off += plain.size() * sizeof(Chunk);
+    const size_t off_units = off;   off += units.size() * sizeof(RowUnit);
+    const size_t off_mean = off;    off += static_cast<size_t>(o->total_rows) * sizeof(float2);
+    const size_t bytes = off + 16;
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
+        o->d_prep = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(gradient statistics, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    if ((e = cudaMemsetAsync(o->d_prep, 0, bytes, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaMemsetAsync(gradient statistics)");
+    o->prep_out = reinterpret_cast<PrepOut *>(o->d_prep);
+    o->part_sq = reinterpret_cast<double *>(o->d_prep + off_sq);
+    o->part_sum = reinterpret_cast<double *>(o->d_prep + off_sum);
+    o->chunk_psq = reinterpret_cast<double *>(o->d_prep + off_psq);
+    o->cta_sq = reinterpret_cast<double *>(o->d_prep + off_cta);
+    o->d_plain = centre ? reinterpret_cast<Chunk *>(o->d_prep + off_plain) : nullptr;
+    o->d_units = reinterpret_cast<RowUnit *>(o->d_prep + off_units);
+    o->row_mean = reinterpret_cast<float2 *>(o->d_prep + off_mean);
+    o->n_plain = static_cast<int>(n_plain);
+    o->n_units = static_cast<int>(units.size());
+    // The tables are built once per layout: blocking copies keep the host
+    // vectors' lifetime trivial.
+    if (!plain.empty() &&
+        (e = cudaMemcpyAsync(o->d_plain, plain.data(), plain.size() * sizeof(Chunk),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "statistics table upload");
+    if (!units.empty() &&
+        (e = cudaMemcpyAsync(o->d_units, units.data(), units.size() * sizeof(RowUnit),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "row unit upload");
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail_cuda(o, e, "statistics table upload");
+    o->prep_key = key;
+    invalidate_tables(o);              // records carry pointers into this scratch
+    return NOVAK_OK;
+}
+
+// Scratch of layer adaptation, allocated when a step first needs it.
+int prepare_trust(novak_opt *o, cudaStream_t stream)
+{
+    if (o->d_trust) return NOVAK_OK;
+    const size_t nc = static_cast<size_t>(o->n_chunks), n = static_cast<size_t>(o->n);
+    const size_t off_p2 = nc * sizeof(double);
+    const size_t off_first = 2 * nc * sizeof(double);
+    const size_t off_trust = off_first + (n + 1) * sizeof(int);
+    const size_t bytes = off_trust + n * sizeof(float) + 16;
+    cudaError_t e;
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_trust), bytes)) != cudaSuccess) {
+        o->d_trust = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(layer adaptation, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    o->chunk_u2 = reinterpret_cast<double *>(o->d_trust);
+    o->chunk_p2 = reinterpret_cast<double *>(o->d_trust + off_p2);
+    o->tensor_first = reinterpret_cast<int *>(o->d_trust + off_first);
+    o->trust = reinterpret_cast<float *>(o->d_trust + off_trust);
+    // the table lists a tensor's entries consecutively, tensors in order
+    o->h_tensor_first.assign(n + 1, o->n_chunks);
+    for (int c = o->n_chunks - 1; c >= 0; --c) o->h_tensor_first[o->h_chunks[c].tensor] = c;
+    if ((e = cudaMemcpyAsync(o->tensor_first, o->h_tensor_first.data(), (n + 1) * sizeof(int),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "layer adaptation table upload");
+    return NOVAK_OK;
+}
+
+uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype)
+{
+    uint64_t h = 0xcbf29ce484222325ull ^ static_cast<uint64_t>(grad_dtype);
+    for (int i = 0; i < n; ++i) {
+        h = (h ^ reinterpret_cast<uintptr_t>(d_params[i])) * 0x100000001b3ull;
+        h = (h ^ reinterpret_cast<uintptr_t>(d_grads[i])) * 0x100000001b3ull;
+    }
+    return h;
+}
+
+// Selects the device record table that holds the caller's pointer lists,
+// uploading them (in stream order, into the least recently used table) when
+// none does.
+int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
+                    int grad_dtype, cudaStream_t stream)
+{
+    const int n = o->n;
+    const uint64_t hash = hash_pointers(d_params, d_grads, n, grad_dtype);
+    int lru = 0;
+    for (int k = 0; k < kRecTables; ++k) {
+        novak_opt::RecTable &tb = o->tables[k];
+        if (tb.gdtype == grad_dtype && tb.hash == hash && !tb.p.empty() &&
+            std::memcmp(tb.p.data(), d_params, n * sizeof(void *)) == 0 &&
+            std::memcmp(tb.g.data(), d_grads, n * sizeof(void *)) == 0) {
+            tb.last_use = ++o->table_clock;
+            o->cur_table = k;
+            return NOVAK_OK;
+        }
+        if (tb.last_use < o->tables[lru].last_use) lru = k;
+    }
+
+    const uintptr_t gmask = grad_dtype == NOVAK_GRAD_BF16 ? 1u : 3u;
+    const uintptr_t gvec = grad_dtype == NOVAK_GRAD_BF16 ? 8u : 16u;
+    bool scalar_path = false;
+    for (int i = 0; i < n; ++i) {
+        const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
+        const uintptr_t g = reinterpret_cast<uintptr_t>(d_grads[i]);
+        if (!p || !g) return fail(o, NOVAK_EINVAL, "tensor %d: NULL pointer", i);
+        if ((p & 3u) || (g & gmask)) return fail(o, NOVAK_EINVAL, "tensor %d: pointer not aligned to its element size", i);
+        // 128-bit path needs parameter, state and gradient congruent mod 16 B.
+        const uintptr_t m = reinterpret_cast<uintptr_t>(slice(o, 0, i));
+        if (((p ^ m) & 15u) || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
+            scalar_path = true;
+        // the bf16 copy is stored 4 elements (8 bytes) at a time beside 16-byte parameters
+        if (!o->copies.empty() &&
+            ((p & 15u) >> 1) != (reinterpret_cast<uintptr_t>(o->copies[i]) & 7u))
+            scalar_path = true;
+    }
+    const int slot = o->ring_pos;
+    cudaError_t e;
+    if ((e = cudaEventSynchronize(o->ring_ev[slot])) != cudaSuccess)
+        return fail_cuda(o, e, "cudaEventSynchronize(record ring)");
+    TensorRec *h = o->h_recs[slot];
+    const bool la = o->h.la_k > 0;
+    const bool traj = la && o->h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN;
+    for (int i = 0; i < n; ++i) {
+        h[i].p = static_cast<float *>(d_params[i]);
+        h[i].g = d_grads[i];
+        h[i].m = slice(o, 0, i);
+        h[i].v = slice(o, 1, i);
+        h[i].slow = la ? slice(o, 2, i) : nullptr;
+        h[i].acc = traj ? slice(o, 3, i) : nullptr;
+        const bool rows = o->h.centralize && o->row_mean && !o->rows.empty() && o->rows[i] > 0;
+        h[i].mean = rows ? o->row_mean + o->row_off[i] : nullptr;
+        h[i].row_len = rows ? static_cast<uint32_t>(o->numel[i] / o->rows[i]) : 0u;
+        h[i].p16 = o->copies.empty() ? nullptr : static_cast<__nv_bfloat16 *>(o->copies[i]);
+        h[i].reserved = 0;
+    }
+    // Stream order puts this copy behind every earlier launch that read the
+    // table being replaced.
+    novak_opt::RecTable &tb = o->tables[lru];
+    tb.p.clear();
+    if ((e = cudaMemcpyAsync(o->d_recs + static_cast<size_t>(lru) * n, h, n * sizeof(TensorRec),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "tensor record upload");
+    if ((e = cudaEventRecord(o->ring_ev[slot], stream)) != cudaSuccess)
+        return fail_cuda(o, e, "cudaEventRecord(record ring)");
+    o->ring_pos = (slot + 1) % kRing;
+    tb.p.assign(d_params, d_params + n);
+    tb.g.assign(d_grads, d_grads + n);
+    tb.gdtype = grad_dtype;
+    tb.hash = hash;
+    tb.last_use = ++o->table_clock;
+    o->cur_table = lru;
+    o->record_uploads += 1;
+    if (scalar_path) o->warnings |= NOVAK_WARN_SCALAR_PATH;
+    return NOVAK_OK;
+}
+
+}  // namespace novak_host

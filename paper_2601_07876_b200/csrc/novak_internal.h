@@ -1,4 +1,4 @@
-// Internal types shared by the host planner (novak_host.cpp) and the device
+// Internal types shared by the host side (novak_host*.cpp) and the device
 // code (novak_*.cu) of the NOVAK step library.  Not part of the C ABI.
 #pragma once
 
