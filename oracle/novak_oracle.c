@@ -55,6 +55,16 @@
  *     uses), ||theta_t|| that of the parameters before the step, both over
  *     every tensor of the group; the averages start at 0.   [parity unpinned]
  *
+ *   - True Nesterov (Eq. 10-12, Section 5.8): the caller saves theta_{t-1},
+ *     sets the model to theta~ = theta_{t-1} + beta_N m_{t-1} (Eq. 10), obtains
+ *     g~ there (Eq. 11), restores theta_{t-1}, and g~ then stands where g_t
+ *     stands in every later phase: both moments, the direction and the update
+ *     (Section 5.8, point 5).  Eq. 12 prints only g~ over a v~ it does not
+ *     define and leaves m_t open; it is read as shorthand for that.  While
+ *     t <= N_taylor the step applies no Eq. 13 correction to g~; from step
+ *     N_taylor + 1 on the variant is the approximation of Eq. 13 (Section 5.2's
+ *     automatic fallback).                                 [parity unpinned]
+ *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
  */
@@ -69,7 +79,8 @@ typedef struct {
     double weight_decay;     /* lambda >= 0                                 */
     double nesterov_beta;    /* beta_N in [0,1)                             */
     double lookahead_alpha;  /* alpha_LA in (0,1), used when lookahead_k>0  */
-    int32_t nesterov_variant;/* 0 none, 1 approximation (Eq.13), 2 classical (Eq.16) */
+    int32_t nesterov_variant;/* 0 none, 1 approximation (Eq.13), 2 classical (Eq.16),
+                                3 true (Eq. 10-12) for the first true_steps steps   */
     int32_t lookahead_k;     /* 0 = lookahead off                           */
     int32_t lookahead_mode;  /* 0 LAST, 1 TRAJ_MEAN                         */
     int32_t rectified;       /* 1: Eq. 8-9, 0: r_t = 1 on every step        */
@@ -78,7 +89,34 @@ typedef struct {
     double tau1;             /* warm-up time scale of beta1 (paper: 1000)   */
     double tau2;             /* warm-up time scale of beta2 (paper: 5000)   */
     double sparse_threshold; /* tau of Eq. 27; 0 = no mask                  */
+    int32_t true_steps;      /* N_taylor: steps 1..N_taylor of variant 3 take g~ */
+    int32_t reserved;
 } novak_oracle_hparams;
+
+/* Whether step t applies the correction of Eq. 13 to the gradient it is given:
+ * always for the approximation variant; for the true variant only once the
+ * first N_taylor steps, whose gradient already is Eq. 11's g~, are over. */
+static int approximation_active(const novak_oracle_hparams *h, int64_t t)
+{
+    if (h->nesterov_variant == 3)
+        return t > (int64_t)h->true_steps;
+    return h->nesterov_variant == 1;
+}
+
+/* Eq. 10: the position the true variant evaluates the gradient at,
+ * theta~ = theta_{t-1} + beta_N m_{t-1}, element by element. */
+void novak_oracle_extrapolate(double beta_n, int64_t n, const double *theta,
+                              const double *m, double *theta_tilde)
+{
+    for (int64_t i = 0; i < n; ++i)
+        theta_tilde[i] = theta[i] + beta_n * m[i];
+}
+
+/* 1 when step t of these hyperparameters expects Eq. 11's gradient. */
+int32_t novak_oracle_wants_extrapolation(const novak_oracle_hparams *h, int64_t t)
+{
+    return (h->nesterov_variant == 3 && t <= (int64_t)h->true_steps) ? 1 : 0;
+}
 
 typedef struct {
     double bc1;       /* 1 - beta1^t                        (Eq. 5) */
@@ -142,7 +180,7 @@ double novak_oracle_trust_ratio(const novak_oracle_hparams *h, int64_t t, int64_
     double sum_theta = 0.0, sum_u = 0.0;
     for (int64_t i = 0; i < n; ++i) {
         double gt = g[i];
-        if (h->nesterov_variant == 1)
+        if (approximation_active(h, t))
             gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
         const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
         const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
@@ -176,7 +214,7 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
     for (int64_t i = 0; i < n; ++i) {
         /* Phase 2: Nesterov approximation, Eq. 13 (m[i] is m_{t-1}). */
         double gt = g[i];
-        if (h->nesterov_variant == 1)
+        if (approximation_active(h, t))
             gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
 
         /* Phase 4: Eq. 1-2 (with the coefficients of Eq. 3-4 when warmed up). */
@@ -281,7 +319,7 @@ void novak_oracle_direction(const novak_oracle_hparams *h, int64_t t, int64_t n,
     novak_oracle_scalars_at(h, t, &s);
     for (int64_t i = 0; i < n; ++i) {
         double gt = g[i];
-        if (h->nesterov_variant == 1)
+        if (approximation_active(h, t))
             gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
         const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
         const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;

@@ -23,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "novak_oracle.c")
 _LIB = os.path.join(_HERE, "libnovak_oracle.so")
 
-NESTEROV_NONE, NESTEROV_APPROX, NESTEROV_CLASSICAL = 0, 1, 2
+NESTEROV_NONE, NESTEROV_APPROX, NESTEROV_CLASSICAL, NESTEROV_TRUE = 0, 1, 2, 3
 LOOKAHEAD_LAST, LOOKAHEAD_TRAJ_MEAN = 0, 1
 
 
@@ -45,6 +45,8 @@ class HParams(ctypes.Structure):
         ("tau1", ctypes.c_double),
         ("tau2", ctypes.c_double),
         ("sparse_threshold", ctypes.c_double),
+        ("true_steps", ctypes.c_int32),
+        ("reserved", ctypes.c_int32),
     ]
 
 
@@ -106,6 +108,10 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.novak_oracle_scale.restype = None
     lib.novak_oracle_centralize.argtypes = [ctypes.c_int64, ctypes.c_int64, dp]
     lib.novak_oracle_centralize.restype = None
+    lib.novak_oracle_extrapolate.argtypes = [ctypes.c_double, ctypes.c_int64, dp, dp, dp]
+    lib.novak_oracle_extrapolate.restype = None
+    lib.novak_oracle_wants_extrapolation.argtypes = [ctypes.POINTER(HParams), ctypes.c_int64]
+    lib.novak_oracle_wants_extrapolation.restype = ctypes.c_int32
     return lib
 
 
@@ -145,6 +151,7 @@ class Config:
     sparse_threshold: float = 0.0        # tau of Eq. 27; 0 = off
     auto_lr: bool = False                # Eq. 20-22
     auto_lr_gamma: float = 0.1
+    true_steps: int = 0                  # N_taylor of the true variant (Section 5.2)
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -153,7 +160,7 @@ class Config:
                        self.nesterov_variant, self.lookahead_k,
                        self.lookahead_mode, int(self.rectified),
                        self.bias1_power, int(self.adaptive_beta), self.tau1, self.tau2,
-                       self.sparse_threshold)
+                       self.sparse_threshold, self.true_steps, 0)
 
 
 def _dptr(a: np.ndarray, offset: int = 0):
@@ -200,6 +207,23 @@ class Oracle:
         s = Scalars()
         self.lib.novak_oracle_scalars_at(ctypes.byref(self.h), t, ctypes.byref(s))
         return s
+
+    def wants_extrapolation(self) -> bool:
+        """Whether the NEXT step expects the gradient of Eq. 11 (true variant,
+        first N_taylor steps)."""
+        return bool(self.lib.novak_oracle_wants_extrapolation(ctypes.byref(self.h), self.t + 1))
+
+    def extrapolated(self):
+        """Eq. 10 for every tensor: theta + beta_N m, as new arrays (the oracle's
+        own parameters stay where they are, which is the save and restore of
+        Section 5.8 written out)."""
+        out = []
+        for th, m in zip(self.theta, self.m):
+            tt = np.empty_like(th)
+            self.lib.novak_oracle_extrapolate(self.h.nesterov_beta, th.size, _dptr(th),
+                                              _dptr(m), _dptr(tt))
+            out.append(tt)
+        return out
 
     def _run(self, i: int, g: np.ndarray, lo: int, hi: int, trust: float = 1.0):
         null = ctypes.POINTER(ctypes.c_double)()

@@ -755,6 +755,74 @@ def pin_auto_lr(lib):
                rtol=1e-9, atol=1e-15, what="alpha_auto times lambda_trust")
 
 
+# --------------------------------------------------------------------------
+# True Nesterov (Eq. 10-12, Section 5.8) and its fallback (Section 5.2)
+# --------------------------------------------------------------------------
+def pin_true_nesterov(lib):
+    """Eq. 10 in closed form (hand values; after one step from zero moments), the
+    closed loop on a quadratic against a scalar loop written here, the switch to
+    Eq. 13 after exactly N_taylor steps, and that looking ahead moves nothing."""
+    lr, b1, b2, eps, wd, bN = 1e-2, 0.9, 0.999, 0.5, 0.1, 0.8
+    kw = dict(lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd, lookahead_k=0,
+              rectified=False, nesterov_beta=bN)
+    # hand values of theta + beta_N m
+    out = np.empty(3)
+    th = np.array([1.0, -2.0, 0.5]); m = np.array([0.5, 0.25, -1.0])
+    lib.novak_oracle_extrapolate(bN, 3, O._dptr(th), O._dptr(m), O._dptr(out))
+    _close(out, np.array([1.4, -1.8, -0.3]), what="Eq. 10 by hand")
+    # after one step from zero moments: theta_1 = theta_0 d - lr g/(|g|+eps), m_1 = (1-b1) g
+    g = np.array([1.0, -0.25, 2.0])
+    o = _mk(lib, [th], nesterov_variant=O.NESTEROV_TRUE, true_steps=5, **kw)
+    assert o.wants_extrapolation()
+    _close(o.extrapolated()[0], th, what="m_0 = 0: the first look-ahead is the identity")
+    o.step([g])
+    before = o.theta[0].copy()
+    _close(o.extrapolated()[0],
+           th * (1 - lr * wd) - lr * g / (np.abs(g) + eps) + bN * (1 - b1) * g,
+           what="Eq. 10 at t = 2 (beta_N, not beta1)")
+    assert np.array_equal(o.theta[0], before), "looking ahead must not move theta"
+    # closed loop on L = a theta^2 / 2: g~ = a (theta + beta_N m), Adam with no correction
+    a, T = 3.0, 12
+    q = _mk(lib, [np.array([0.7])], nesterov_variant=O.NESTEROV_TRUE, true_steps=T, **kw)
+    x, mm, vv = 0.7, 0.0, 0.0
+    for t in range(1, T + 1):
+        q.step([a * q.extrapolated()[0]])
+        gt = a * (x + bN * mm)
+        mm = b1 * mm + (1 - b1) * gt
+        vv = b2 * vv + (1 - b2) * gt * gt
+        x = x * (1 - lr * wd) - lr * (mm / (1 - b1 ** t)) / (np.sqrt(vv / (1 - b2 ** t)) + eps)
+        _close(q.theta[0], np.array([x]), rtol=1e-11, what=f"quadratic, step {t}")
+    # N_taylor = 0: the approximation from the first step, bit for bit
+    rng = np.random.default_rng(7)
+    G = [rng.normal(0, 1, 5) for _ in range(8)]
+    th5 = rng.normal(0, 1, 5)
+    z = _mk(lib, [th5], nesterov_variant=O.NESTEROV_TRUE, true_steps=0, **kw)
+    ap = _mk(lib, [th5], nesterov_variant=O.NESTEROV_APPROX, **kw)
+    for gg in G:
+        assert not z.wants_extrapolation()
+        z.step([gg]); ap.step([gg])
+    assert np.array_equal(z.theta[0], ap.theta[0])
+    # N_taylor = 3: steps 1-3 as variant none, steps 4-8 as the approximation on that state
+    N = 3
+    tr = _mk(lib, [th5], nesterov_variant=O.NESTEROV_TRUE, true_steps=N, **kw)
+    no = _mk(lib, [th5], nesterov_variant=O.NESTEROV_NONE, **kw)
+    wants = []
+    for t, gg in enumerate(G, start=1):
+        wants.append(tr.wants_extrapolation())
+        tr.step([gg])
+        if t <= N:
+            no.step([gg])
+            assert np.array_equal(tr.theta[0], no.theta[0]), f"step {t}: no correction yet"
+        if t == N:
+            ap = _mk(lib, [no.theta[0]], nesterov_variant=O.NESTEROV_APPROX, **kw)
+            ap.m[0][:] = no.m[0]; ap.v[0][:] = no.v[0]; ap.t = N
+        if t > N:
+            ap.step([gg])
+            assert np.array_equal(tr.theta[0], ap.theta[0]), f"step {t}: Eq. 13 from N+1 on"
+    assert wants == [t <= N for t in range(1, len(G) + 1)]
+    assert not np.array_equal(tr.theta[0], z.theta[0])
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -778,4 +846,5 @@ ALL_PINS = [
     pin_trust_ratio,
     pin_sparse_mask,
     pin_auto_lr,
+    pin_true_nesterov,
 ]

@@ -55,6 +55,16 @@ MUTANTS = [
     ("warmup_in_classical_blend", "u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
      "u = s.beta1_t * m_hat + (1.0 - s.beta1_t) * u;"),
     ("warmup_flag_ignored", "if (h->adaptive_beta) {", "if (1) {"),
+    # true Nesterov (Eq. 10) and its fallback
+    ("extrapolate_sign", "theta_tilde[i] = theta[i] + beta_n * m[i];",
+     "theta_tilde[i] = theta[i] - beta_n * m[i];"),
+    ("extrapolate_drops_beta", "theta_tilde[i] = theta[i] + beta_n * m[i];",
+     "theta_tilde[i] = theta[i] + m[i];"),
+    ("fallback_off_by_one", "return t > (int64_t)h->true_steps;",
+     "return t >= (int64_t)h->true_steps;"),
+    ("fallback_never", "return t > (int64_t)h->true_steps;", "return 0;"),
+    ("true_corrected_from_the_start", "return t > (int64_t)h->true_steps;", "return 1;"),
+    ("wants_off_by_one", "t <= (int64_t)h->true_steps) ? 1 : 0", "t < (int64_t)h->true_steps) ? 1 : 0"),
     # phase 7: automatic learning-rate scaling
     ("auto_inverted", "double a = *g_bar / *theta_bar;", "double a = *theta_bar / *g_bar;"),
     ("auto_gamma_swapped", "*g_bar = gamma * grad_norm + (1.0 - gamma) * *g_bar;",
