@@ -50,9 +50,14 @@ enum {
     NOVAK_ENOMEM = 4   /* host or device allocation failed                   */
 };
 
-/* nesterov_variant (Section 4.4). TRUE needs a closure that re-evaluates the
- * gradient, which this path does not have: it is accepted and downgraded to
- * APPROX with NOVAK_WARN_TRUE_DOWNGRADED set (Section 7.3's downgrade rule). */
+/* nesterov_variant (Section 4.4).  TRUE needs a closure that re-evaluates the
+ * gradient at the look-ahead point, which stays with the caller: for the first
+ * N_taylor = NOVAK_OPT_TRUE_NESTEROV_STEPS steps the caller brackets its closure
+ * with novak_nesterov_extrapolate / novak_nesterov_restore and the step takes
+ * the gradient it is given as Eq. 11's; afterwards (Section 5.2's fallback), and
+ * from the first step while N_taylor = 0 (the default, with
+ * NOVAK_WARN_TRUE_DOWNGRADED set: Section 7.3's downgrade rule), the variant
+ * is APPROX. */
 enum {
     NOVAK_NESTEROV_NONE = 0,
     NOVAK_NESTEROV_APPROX = 1,
@@ -117,6 +122,13 @@ enum {
                                      the parameters once more (+4 B per element on top
                                      of clipping's +4).  0 (default)                  */
     NOVAK_OPT_AUTO_LR_GAMMA = 20, /* gamma in (0, 1] of Eq. 20-21 (default 0.1)        */
+    NOVAK_OPT_TRUE_NESTEROV_STEPS = 21, /* N_taylor >= 0 (Section 5.2; the paper uses
+                                     100-200): steps 1..N_taylor of a handle created
+                                     with NOVAK_NESTEROV_TRUE apply no correction of
+                                     Eq. 13 to the gradient, which the caller has
+                                     evaluated at Eq. 10's point; later steps run
+                                     APPROX.  0 (default): APPROX from the first step.
+                                     NOVAK_ESTATE for any other variant             */
     NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base
                                      directions with |u| <= tau are set to zero before
                                      the classical blend; 0 (default): no mask.  The
@@ -125,7 +137,8 @@ enum {
 
 /* Warning bits (novak_info.warnings). */
 enum {
-    NOVAK_WARN_TRUE_DOWNGRADED = 1u, /* nesterov_variant TRUE ran as APPROX           */
+    NOVAK_WARN_TRUE_DOWNGRADED = 1u, /* nesterov_variant TRUE runs as APPROX from the
+                                        first step (N_taylor = 0)                      */
     NOVAK_WARN_SCALAR_PATH = 2u      /* some tensor's pointers do not share 16-byte
                                         alignment; it runs on 4-byte accesses          */
 };
@@ -146,7 +159,8 @@ typedef struct novak_info {
     double decay;           /* 1 - alpha lambda                           (Eq. 18) */
     int32_t rect_branch;    /* 1: first case of Eq. 8 (rho_t >= 5) was taken       */
     int32_t is_sync;        /* 1: the last step synchronised                       */
-    int32_t nesterov_variant; /* effective variant (after the downgrade)           */
+    int32_t nesterov_variant; /* variant of that step: TRUE while t <= N_taylor, else
+                                 the configured one (APPROX after the fallback)    */
     int32_t lookahead_mode;
     int32_t lookahead_k;
     int32_t n_tensors;
@@ -181,7 +195,7 @@ typedef struct novak_meta {
     double sparse_threshold;
     double auto_lr_gamma;
     int32_t auto_lr;
-    int32_t reserved;
+    int32_t true_nesterov_steps; /* N_taylor; nesterov_variant is TRUE when requested */
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
@@ -388,6 +402,41 @@ int novak_get_grad_stats(novak_opt *opt, double *norm, double *factor, void *str
  * direction (Eq. 17); 1 where ||u_t|| = 0.  Copies n floats from the device and
  * SYNCHRONISES `stream`.  NOVAK_ESTATE when no such step has run. */
 int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
+
+/* True Nesterov momentum, Section 4.4 (Eq. 10-12) and Section 5.8 ("True
+ * Nesterov closure").  The gradient of Eq. 11 is the caller's to compute; these
+ * two calls do the parameter traffic around it for a handle created with
+ * NOVAK_NESTEROV_TRUE (NOVAK_ESTATE otherwise):
+ *
+ *   novak_nesterov_extrapolate   save <- theta_{t-1};
+ *                                theta <- theta_{t-1} + beta_N m_{t-1}   (Eq. 10)
+ *   ... the caller's forward and backward pass at theta~ (Eq. 11) ...
+ *   novak_nesterov_restore       theta <- save
+ *   novak_step(..., that gradient)      (no Eq. 13 correction while t <= N_taylor)
+ *
+ * One kernel each over the handle's chunk table, enqueued on `stream` (a
+ * cudaStream_t; NULL: the default stream); no host synchronisation.  In fp32:
+ * one fused multiply-add per element; the restored parameters are bit for bit
+ * the saved ones.
+ *
+ * d_params, numel, n: DEVICE pointers and sizes as in novak_step (fp32, the
+ * attached layout).  d_save: DEVICE buffer the CALLER owns, aligned to 16
+ * bytes, of at least novak_nesterov_save_bytes() bytes (0 before attach; the
+ * size of one state array), laid out like a state array; it must stay valid
+ * and unchanged until the restore, which takes the same d_params and d_save.
+ * Between the two calls every step entry point, novak_import_meta and
+ * NOVAK_OPT_TRUE_NESTEROV_STEPS return NOVAK_ESTATE.  m_{t-1} = 0 before the
+ * first step, so the first look-ahead leaves theta where it is.
+ * Errors: NOVAK_EINVAL (NULL, a misaligned or short buffer, restore with other
+ * buffers), NOVAK_ESTATE (not attached, wrong variant, a tensor list other
+ * than the attached one, extrapolate twice, restore without extrapolate),
+ * NOVAK_ENOMEM / NOVAK_ECUDA; the handle and the parameters are unchanged on
+ * error. */
+size_t novak_nesterov_save_bytes(const novak_opt *opt);
+int novak_nesterov_extrapolate(novak_opt *opt, void *const *d_params, void *d_save,
+                               size_t save_bytes, const int64_t *numel, int n, void *stream);
+int novak_nesterov_restore(novak_opt *opt, void *const *d_params, const void *d_save,
+                           size_t save_bytes, const int64_t *numel, int n, void *stream);
 
 /* Automatic learning-rate scaling (Eq. 20-22, NOVAK_OPT_AUTO_LR).  Its two
  * moving averages live in device memory.  get: copies them and the last step's

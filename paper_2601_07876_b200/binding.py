@@ -29,7 +29,7 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
  NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
- NOVAK_OPT_AUTO_LR_GAMMA) = range(1, 21)
+ NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS) = range(1, 22)
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -64,7 +64,7 @@ class novak_meta(Structure):
         ("warnings", c_uint32), ("centralize", c_int32), ("clip_threshold", c_double),
         ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
         ("layer_adaptation", c_int32), ("sparse_threshold", c_double),
-        ("auto_lr_gamma", c_double), ("auto_lr", c_int32), ("reserved", c_int32),
+        ("auto_lr_gamma", c_double), ("auto_lr", c_int32), ("true_nesterov_steps", c_int32),
     ]
 
 
@@ -119,6 +119,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
                                             POINTER(c_double), vp]),
         "novak_set_auto_lr_state": (c_int, [vp, c_double, c_double]),
         "novak_get_trust_ratios": (c_int, [vp, POINTER(ctypes.c_float), c_int, vp]),
+        "novak_nesterov_save_bytes": (c_size_t, [vp]),
+        "novak_nesterov_extrapolate": (c_int, [vp, vpp, vp, c_size_t, i64p, c_int, vp]),
+        "novak_nesterov_restore": (c_int, [vp, vpp, vp, c_size_t, i64p, c_int, vp]),
         "novak_get_info": (c_int, [vp, POINTER(novak_info)]),
         "novak_plan": (c_int, [vp, c_int64, POINTER(novak_info)]),
         "novak_state_ptrs": (c_int, [vp, c_int, vpp, vpp, vpp, vpp]),
@@ -311,6 +314,21 @@ class Handle:
                "novak_get_trust_ratios")
         return list(out)
 
+    def nesterov_save_bytes(self) -> int:
+        return int(self.lib.novak_nesterov_save_bytes(self.h))
+
+    def nesterov_extrapolate(self, params_arr, d_save: int, save_bytes: int, numel_arr, n: int,
+                             stream: int = 0):
+        _check(self.lib, self.h,
+               self.lib.novak_nesterov_extrapolate(self.h, params_arr, d_save, save_bytes, numel_arr,
+                                                   n, stream), "novak_nesterov_extrapolate")
+
+    def nesterov_restore(self, params_arr, d_save: int, save_bytes: int, numel_arr, n: int,
+                         stream: int = 0):
+        _check(self.lib, self.h,
+               self.lib.novak_nesterov_restore(self.h, params_arr, d_save, save_bytes, numel_arr,
+                                               n, stream), "novak_nesterov_restore")
+
     def get_info(self) -> novak_info:
         out = novak_info()
         _check(self.lib, self.h, self.lib.novak_get_info(self.h, byref(out)), "novak_get_info")
@@ -375,7 +393,7 @@ class NovakOptimizer:
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
-                 auto_lr=False, auto_lr_gamma=None,
+                 auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -442,6 +460,31 @@ class NovakOptimizer:
         self.param_copies = None
         if param_copies is not None:
             self.set_param_copies(param_copies)
+        self._save = None
+        if true_nesterov_steps:
+            h.set_option(NOVAK_OPT_TRUE_NESTEROV_STEPS, true_nesterov_steps)
+
+    def wants_extrapolation(self) -> bool:
+        """Whether the NEXT step is a true-Nesterov step (Section 5.2: the first
+        N_taylor steps), i.e. expects a gradient evaluated between extrapolate()
+        and restore()."""
+        t = self.handle.get_info().t + 1
+        return self.handle.plan(t).nesterov_variant == NOVAK_NESTEROV_TRUE
+
+    def extrapolate(self):
+        """Eq. 10: saves the parameters and moves them to theta + beta_N m, in place."""
+        import torch
+        if self._save is None:
+            self._save = torch.empty(self.handle.nesterov_save_bytes(), dtype=torch.uint8,
+                                     device=self.device)
+        self.handle.nesterov_extrapolate(self._params_arr, self._save.data_ptr(),
+                                         self._save.numel(), self._numel_arr, self.n,
+                                         self._stream())
+
+    def restore(self):
+        """Puts the parameters saved by extrapolate() back, bit for bit."""
+        self.handle.nesterov_restore(self._params_arr, self._save.data_ptr(), self._save.numel(),
+                                     self._numel_arr, self.n, self._stream())
 
     def set_param_copies(self, copies):
         """bf16 tensors (one per parameter) that every step fills with the updated

@@ -16,7 +16,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libnovak.so")
 SOURCES = [os.path.join(CSRC, f) for f in (
     "novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu",
-    "novak_grad_stats.cu", "novak_trust_stats.cu",
+    "novak_grad_stats.cu", "novak_trust_stats.cu", "novak_nesterov.cu",
     "novak_step_pre0.cu", "novak_step_pre1.cu", "novak_step_pre2.cu",
     "novak_step_pre0_copy.cu", "novak_step_pre1_copy.cu", "novak_step_pre2_copy.cu")]
 HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(CSRC, "novak_handle.h"),

@@ -22,7 +22,7 @@ using novak::TensorRec;
 constexpr int kRing = 4;                       // pinned staging slots for tensor records
 constexpr int kRecTables = 8;                  // device record tables kept per handle
 constexpr int64_t kSlotAlign = 32;             // elements: 128-byte slots
-constexpr uint64_t kMetaMagic = 0x4e4f56414b763036ull;  // "NOVAKv06"
+constexpr uint64_t kMetaMagic = 0x4e4f56414b763037ull;  // "NOVAKv07"
 constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
@@ -39,12 +39,15 @@ struct Hyper {
     double sparse_tau;      // tau of Eq. 27, 0: no mask
     int auto_lr;            // Eq. 20-22
     double auto_gamma;      // gamma of Eq. 20-21
+    int true_requested;     // the caller asked for the true variant (Eq. 10-12)
+    int true_steps;         // N_taylor: steps 1..N_taylor take Eq. 11's gradient as given
 };
 
 struct Plan {
     double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay;
     double beta1_t, beta2_t;   // coefficients of Eq. 1-2 at this step (Eq. 3-4 when warmed up)
     int rect_branch, is_sync;
+    int nesterov;              // variant of this step: TRUE while t <= N_taylor, else the configured one
 };
 
 struct Handle {
@@ -113,6 +116,12 @@ struct Handle {
     bool half_open = false;
     int half_launches = 0;
     alignas(8) unsigned char half_ctx[256] = {};   // the StepCtx of the open step
+    bool extrapolated = false;          // between novak_nesterov_extrapolate and _restore
+    novak::LookRec *d_look = nullptr;   // device records of the two look-ahead helpers
+    novak::LookRec *h_look = nullptr;   // pinned staging of those records
+    cudaEvent_t look_ev = nullptr;      // the staging buffer's last upload
+    std::vector<void *> look_p;         // the parameter list the device records hold
+    void *look_save = nullptr;          // save buffer of the open look-ahead
     bool ema_pending = false;
     double pending_g_bar = 0.0, pending_theta_bar = 0.0;
     float2 *row_mean = nullptr;
@@ -161,6 +170,13 @@ void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chu
 void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out);
 int check_hyper(const Hyper &h, const char **why);
 
+// The variant the kernels are instantiated for: a true step's gradient needs no
+// correction (Eq. 11's gradient is given), so it runs as variant none.
+inline int kernel_variant(const Plan &p)
+{
+    return p.nesterov == NOVAK_NESTEROV_TRUE ? NOVAK_NESTEROV_NONE : p.nesterov;
+}
+
 // Error reporting: store the message in the handle, return the code.
 int fail(novak_opt *o, int code, const char *fmt, ...);
 int fail_cuda(novak_opt *o, cudaError_t e, const char *what);
@@ -180,5 +196,8 @@ int prepare_trust(novak_opt *o, cudaStream_t stream);
 uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype);
 int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
                     int grad_dtype, cudaStream_t stream);
+// Device records of the look-ahead helpers for this parameter list (uploaded
+// only when the list differs from the one the device holds).
+int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream);
 
 }  // namespace novak_host

@@ -46,6 +46,9 @@ Plan make_plan(const Hyper &h, int64_t t)
         p.beta1_t = h.beta1 * -std::expm1(-td / h.tau1);
         p.beta2_t = h.beta2 * -std::expm1(-td / h.tau2);
     }
+    // Section 5.2: the true variant (the gradient is already Eq. 11's) for the
+    // first N_taylor steps, the approximation of Eq. 13 afterwards.
+    p.nesterov = (h.true_requested && t <= h.true_steps) ? NOVAK_NESTEROV_TRUE : h.nesterov;
     return p;
 }
 
@@ -179,7 +182,7 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->rho_inf = p.rho_inf; out->rho_t = p.rho_t;
     out->r_t = p.r_t; out->step_size = p.step_size; out->decay = p.decay;
     out->rect_branch = p.rect_branch; out->is_sync = p.is_sync;
-    out->nesterov_variant = o->h.nesterov;
+    out->nesterov_variant = p.nesterov;
     out->lookahead_mode = o->h.la_mode;
     out->lookahead_k = o->h.la_k;
     out->n_tensors = o->n;
@@ -247,8 +250,13 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.tau2 = 5000.0;
     uint32_t warn = 0;
     h.nesterov = nesterov_variant;
+    h.true_requested = 0;
+    h.true_steps = 0;
     if (nesterov_variant == NOVAK_NESTEROV_TRUE) {
-        h.nesterov = NOVAK_NESTEROV_APPROX;  // no closure on this path: downgrade, warn
+        // N_taylor = 0 until NOVAK_OPT_TRUE_NESTEROV_STEPS says otherwise: every
+        // step runs the approximation (Section 7.3's downgrade), with a warning
+        h.nesterov = NOVAK_NESTEROV_APPROX;
+        h.true_requested = 1;
         warn |= NOVAK_WARN_TRUE_DOWNGRADED;
     }
     const char *why;
@@ -297,6 +305,17 @@ int novak_set_option(novak_opt *o, int key, double value)
         h.auto_lr = static_cast<int>(value);
         break;
     case NOVAK_OPT_AUTO_LR_GAMMA: h.auto_gamma = value; break;
+    case NOVAK_OPT_TRUE_NESTEROV_STEPS:
+        if (!h.true_requested)
+            return fail(o, NOVAK_ESTATE, "true_nesterov_steps: the handle was not created with NOVAK_NESTEROV_TRUE");
+        if (o->extrapolated)
+            return fail(o, NOVAK_ESTATE, "true_nesterov_steps: parameters are extrapolated; restore them first");
+        if (!(value >= 0.0 && value <= 2147483647.0) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "true_nesterov_steps must be an integer >= 0");
+        h.true_steps = static_cast<int>(value);
+        if (h.true_steps > 0) o->warnings &= ~static_cast<uint32_t>(NOVAK_WARN_TRUE_DOWNGRADED);
+        else o->warnings |= NOVAK_WARN_TRUE_DOWNGRADED;
+        break;
     case NOVAK_OPT_LAYER_ADAPTATION:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "layer_adaptation must be 0 or 1");
         h.layer_adapt = static_cast<int>(value);
@@ -363,6 +382,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_SPARSE_THRESHOLD: *value = o->h.sparse_tau; break;
     case NOVAK_OPT_AUTO_LR: *value = o->h.auto_lr; break;
     case NOVAK_OPT_AUTO_LR_GAMMA: *value = o->h.auto_gamma; break;
+    case NOVAK_OPT_TRUE_NESTEROV_STEPS: *value = o->h.true_steps; break;
     case NOVAK_OPT_LAYER_ADAPTATION: *value = o->h.layer_adapt; break;
     case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
     case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
@@ -524,7 +544,9 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->lr = o->h.lr; out->beta1 = o->h.beta1; out->beta2 = o->h.beta2; out->eps = o->h.eps;
     out->weight_decay = o->h.wd; out->nesterov_beta = o->h.beta_n;
     out->lookahead_alpha = o->h.la_alpha;
-    out->nesterov_variant = o->h.nesterov; out->lookahead_k = o->h.la_k;
+    out->nesterov_variant = o->h.true_requested ? NOVAK_NESTEROV_TRUE : o->h.nesterov;
+    out->true_nesterov_steps = o->h.true_steps;
+    out->lookahead_k = o->h.la_k;
     out->lookahead_mode = o->h.la_mode; out->rectified = o->h.rectified;
     out->bias1_power = o->h.bias1_power;
     out->clip_threshold = o->h.clip;
@@ -546,6 +568,7 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     if (!o || !in) return NOVAK_EINVAL;
     if (in->magic != kMetaMagic) return fail(o, NOVAK_EINVAL, "import: not a NOVAK meta record");
     if (!o->attached) return fail(o, NOVAK_ESTATE, "import: attach the state first");
+    if (o->extrapolated) return fail(o, NOVAK_ESTATE, "import: parameters are extrapolated; restore them first");
     if (in->n_tensors != o->n || in->total_numel != o->total_numel ||
         in->lookahead_k != o->h.la_k || in->lookahead_mode != o->h.la_mode)
         return fail(o, NOVAK_ESTATE, "import: tensor list or lookahead layout differs");
@@ -554,6 +577,14 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     h.lr = in->lr; h.beta1 = in->beta1; h.beta2 = in->beta2; h.eps = in->eps;
     h.wd = in->weight_decay; h.beta_n = in->nesterov_beta; h.la_alpha = in->lookahead_alpha;
     h.nesterov = in->nesterov_variant; h.rectified = in->rectified;
+    h.true_requested = 0;
+    h.true_steps = 0;
+    if (in->nesterov_variant == NOVAK_NESTEROV_TRUE) {
+        if (in->true_nesterov_steps < 0) return fail(o, NOVAK_EINVAL, "import: negative true_nesterov_steps");
+        h.nesterov = NOVAK_NESTEROV_APPROX;
+        h.true_requested = 1;
+        h.true_steps = in->true_nesterov_steps;
+    }
     h.bias1_power = in->bias1_power;
     h.clip = in->clip_threshold;
     h.adaptive_beta = in->adaptive_beta;
@@ -570,6 +601,10 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     o->h = h;
     o->t = in->t; o->n_syncs = in->n_syncs; o->last_sync = in->last_sync_step;
     o->warnings |= in->warnings;
+    if (h.true_requested) {
+        if (h.true_steps > 0) o->warnings &= ~static_cast<uint32_t>(NOVAK_WARN_TRUE_DOWNGRADED);
+        else o->warnings |= NOVAK_WARN_TRUE_DOWNGRADED;
+    }
     o->last_plan = make_plan(h, in->t > 0 ? in->t : 1);
     return NOVAK_OK;
 }

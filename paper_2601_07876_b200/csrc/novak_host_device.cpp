@@ -24,6 +24,14 @@ void release_device(novak_opt *o)
         o->h_recs[i] = nullptr;
         o->ring_ev[i] = nullptr;
     }
+    if (o->d_look) cudaFree(o->d_look);
+    if (o->h_look) cudaFreeHost(o->h_look);
+    if (o->look_ev) cudaEventDestroy(o->look_ev);
+    o->d_look = o->h_look = nullptr;
+    o->look_ev = nullptr;
+    o->look_p.clear();
+    o->look_save = nullptr;
+    o->extrapolated = false;
     if (o->d_trust) cudaFree(o->d_trust);
     o->d_trust = nullptr;
     o->chunk_u2 = o->chunk_p2 = nullptr;
@@ -217,6 +225,50 @@ int prepare_trust(novak_opt *o, cudaStream_t stream)
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
         (e = cudaStreamSynchronize(stream)) != cudaSuccess)
         return fail_cuda(o, e, "layer adaptation table upload");
+    return NOVAK_OK;
+}
+
+// Records of the look-ahead helpers (Eq. 10): allocated on first use, uploaded
+// through one pinned buffer whenever the parameter list changes.
+int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream)
+{
+    const size_t n = static_cast<size_t>(o->n);
+    cudaError_t e;
+    if (!o->d_look) {
+        if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_look), n * sizeof(novak::LookRec))) != cudaSuccess) {
+            o->d_look = nullptr;
+            return fail(o, NOVAK_ENOMEM, "cudaMalloc(look-ahead records): %s", cudaGetErrorString(e));
+        }
+        if ((e = cudaMallocHost(reinterpret_cast<void **>(&o->h_look), n * sizeof(novak::LookRec))) != cudaSuccess) {
+            o->h_look = nullptr;
+            return fail(o, NOVAK_ENOMEM, "cudaMallocHost(look-ahead records): %s", cudaGetErrorString(e));
+        }
+        if ((e = cudaEventCreateWithFlags(&o->look_ev, cudaEventDisableTiming)) != cudaSuccess) {
+            o->look_ev = nullptr;
+            return fail_cuda(o, e, "cudaEventCreate(look-ahead records)");
+        }
+        o->look_p.clear();
+    }
+    if (o->look_p.size() == n && std::memcmp(o->look_p.data(), d_params, n * sizeof(void *)) == 0)
+        return NOVAK_OK;
+    for (size_t i = 0; i < n; ++i) {
+        const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
+        if (!p) return fail(o, NOVAK_EINVAL, "tensor %zu: NULL pointer", i);
+        if (p & 3u) return fail(o, NOVAK_EINVAL, "tensor %zu: pointer not aligned to its element size", i);
+    }
+    // the previous upload may still be reading the staging buffer
+    if (!o->look_p.empty() && (e = cudaEventSynchronize(o->look_ev)) != cudaSuccess)
+        return fail_cuda(o, e, "look-ahead record staging");
+    o->look_p.clear();
+    for (size_t i = 0; i < n; ++i) {
+        o->h_look[i].p = static_cast<float *>(d_params[i]);
+        o->h_look[i].state_off = o->slot_off[i] + o->phase[i];
+    }
+    if ((e = cudaMemcpyAsync(o->d_look, o->h_look, n * sizeof(novak::LookRec), cudaMemcpyHostToDevice,
+                             stream)) != cudaSuccess ||
+        (e = cudaEventRecord(o->look_ev, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "look-ahead record upload");
+    o->look_p.assign(d_params, d_params + n);
     return NOVAK_OK;
 }
 

@@ -52,6 +52,8 @@ int check_step_args(novak_opt *o, const char *who, void *const *d_params,
                     const void *const *d_grads, const int64_t *numel, int n, int grad_dtype)
 {
     if (!o->attached) return fail(o, NOVAK_ESTATE, "%s: no state attached", who);
+    if (o->extrapolated)
+        return fail(o, NOVAK_ESTATE, "%s: parameters are extrapolated (Eq. 10); call novak_nesterov_restore first", who);
     if (o->half_open && std::strcmp(who, "step_begin") != 0)
         return fail(o, NOVAK_ESTATE, "%s: a step begun with novak_step_begin is still open", who);
     if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "%s: NULL argument", who);
@@ -114,7 +116,7 @@ cudaError_t launch_trust(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, 
     if (ctx.trust) {
         *what = "layer adaptation kernel launch";
         e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
-                                      o->prep_out, ctx.s, o->h.nesterov, ctx.grad_dtype, ctx.pre,
+                                      o->prep_out, ctx.s, kernel_variant(ctx.plan), ctx.grad_dtype, ctx.pre,
                                       o->chunk_u2, o->chunk_p2, o->trust, o->pdl, stream);
         if (e != cudaSuccess) return e;
         *launches += 2;
@@ -161,7 +163,7 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16);
     o->last_grid = cfg.grid;
     return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.trust, ctx.s,
-                              o->h.nesterov, ctx.grad_dtype, ctx.la, cfg, stream);
+                              kernel_variant(ctx.plan), ctx.grad_dtype, ctx.la, cfg, stream);
 }
 
 void commit_step(novak_opt *o, const StepCtx &ctx, int launches)
@@ -535,7 +537,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
     cfg.pre = novak::PRE_NONE | (o->copies.empty() ? 0 : novak::PRE_COPY16);
-    e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, nullptr, s, o->h.nesterov, grad_dtype,
+    e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, nullptr, s, kernel_variant(p), grad_dtype,
                            la_action, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
 
@@ -544,6 +546,80 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     o->last_plan = p;
     o->last_grid = cfg.grid;
     if (p.is_sync) { o->n_syncs += 1; o->last_sync = t; }
+    return NOVAK_OK;
+}
+
+// ---- true Nesterov: the look-ahead around the caller's closure (Eq. 10-11) ----
+
+size_t novak_nesterov_save_bytes(const novak_opt *o)
+{
+    if (!o || !o->attached) return 0;
+    return static_cast<size_t>(o->region_elems) * sizeof(float);
+}
+
+namespace {
+
+int check_look_args(novak_opt *o, const char *who, void *const *d_params, const void *d_save,
+                    size_t save_bytes, const int64_t *numel, int n)
+{
+    if (!o->attached) return fail(o, NOVAK_ESTATE, "%s: no state attached", who);
+    if (o->half_open) return fail(o, NOVAK_ESTATE, "%s: a step begun with novak_step_begin is still open", who);
+    if (!o->h.true_requested)
+        return fail(o, NOVAK_ESTATE, "%s: the handle was not created with NOVAK_NESTEROV_TRUE", who);
+    if (!d_params || !d_save || !numel) return fail(o, NOVAK_EINVAL, "%s: NULL argument", who);
+    if (n != o->n || std::memcmp(numel, o->numel.data(), n * sizeof(int64_t)) != 0)
+        return fail(o, NOVAK_ESTATE, "%s: tensor list differs from the attached layout", who);
+    if (save_bytes < novak_nesterov_save_bytes(o))
+        return fail(o, NOVAK_EINVAL, "%s: save buffer holds %zu bytes, %zu needed", who, save_bytes,
+                    novak_nesterov_save_bytes(o));
+    if (reinterpret_cast<uintptr_t>(d_save) & 15u)
+        return fail(o, NOVAK_EINVAL, "%s: save buffer not aligned to 16 bytes", who);
+    return NOVAK_OK;
+}
+
+int look_grid(const novak_opt *o) { return std::min(o->n_chunks, o->sms * 8); }
+
+}  // namespace
+
+int novak_nesterov_extrapolate(novak_opt *o, void *const *d_params, void *d_save, size_t save_bytes,
+                               const int64_t *numel, int n, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    int rc = check_look_args(o, "nesterov_extrapolate", d_params, d_save, save_bytes, numel, n);
+    if (rc != NOVAK_OK) return rc;
+    if (o->extrapolated)
+        return fail(o, NOVAK_ESTATE, "nesterov_extrapolate: parameters are extrapolated already");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
+    if ((rc = prepare_look(o, d_params, stream)) != NOVAK_OK) return rc;
+    const cudaError_t e = novak::launch_extrapolate(
+        o->d_chunks, o->n_chunks, o->d_look, reinterpret_cast<const float *>(o->d_state),
+        static_cast<float *>(d_save), static_cast<float>(o->h.beta_n), look_grid(o), stream);
+    if (e != cudaSuccess) return fail_cuda(o, e, "look-ahead kernel launch");
+    o->extrapolated = true;
+    o->look_save = d_save;
+    o->launches += 1;
+    return NOVAK_OK;
+}
+
+int novak_nesterov_restore(novak_opt *o, void *const *d_params, const void *d_save, size_t save_bytes,
+                           const int64_t *numel, int n, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    int rc = check_look_args(o, "nesterov_restore", d_params, d_save, save_bytes, numel, n);
+    if (rc != NOVAK_OK) return rc;
+    if (!o->extrapolated)
+        return fail(o, NOVAK_ESTATE, "nesterov_restore: nothing to restore");
+    if (d_save != o->look_save ||
+        std::memcmp(o->look_p.data(), d_params, static_cast<size_t>(n) * sizeof(void *)) != 0)
+        return fail(o, NOVAK_EINVAL, "nesterov_restore: not the buffers novak_nesterov_extrapolate was given");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const cudaError_t e = novak::launch_restore(o->d_chunks, o->n_chunks, o->d_look,
+                                                static_cast<const float *>(d_save), look_grid(o), stream);
+    if (e != cudaSuccess) return fail_cuda(o, e, "restore kernel launch");
+    o->extrapolated = false;
+    o->look_save = nullptr;
+    o->launches += 1;
     return NOVAK_OK;
 }
 

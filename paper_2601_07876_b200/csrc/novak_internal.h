@@ -96,6 +96,22 @@ cudaError_t launch_grad_stats(const StatsPlan &plan, int grad_dtype, double c_cl
 cudaError_t launch_grad_norm_scalars(PrepOut *prep, const double *d_totals, double c_clip,
                                      double auto_gamma, int pdl, cudaStream_t stream);
 
+// ---- true Nesterov: the look-ahead of Eq. 10 and its undoing ----------------
+// Per-tensor record of the two helper kernels: the parameters, and where the
+// tensor sits inside a state region (first moment and save buffer share it).
+struct __align__(16) LookRec {
+    float *p;
+    int64_t state_off;   // elements from the start of a region
+};
+
+// save <- theta, theta <- theta + beta_N m (Eq. 10) over the chunk table.
+cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
+                               const float *m_region, float *save_region, float beta_n, int grid,
+                               cudaStream_t stream);
+// theta <- save (Section 5.8: restore the parameters after the closure).
+cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
+                           const float *save_region, int grid, cudaStream_t stream);
+
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.
 constexpr int kNoAllocMaxTensors = 4096;

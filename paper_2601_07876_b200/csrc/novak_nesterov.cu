@@ -1,0 +1,125 @@
+// True Nesterov momentum (Section 4.4, Eq. 10-12): the two passes around the
+// caller's closure.  novak_extrapolate_kernel saves theta_{t-1} and moves the
+// parameters to theta~ = theta_{t-1} + beta_N m_{t-1} (Eq. 10);
+// novak_restore_kernel puts theta_{t-1} back (Section 5.8's steps 1, 2 and 4).
+// Both walk the step kernel's chunk table, 128 bits per access where the
+// parameters, the first moment and the save buffer share 16-byte alignment.
+// HBM-bound: 16 B per element (theta and m read, save and theta written) and
+// 8 B per element (save read, theta written).
+#include "novak.h"
+#include "novak_internal.h"
+
+namespace novak {
+namespace {
+
+constexpr int kLookThreads = 256;
+
+__device__ __forceinline__ float4 ld_stream(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.cs.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream(float *p, float4 v)
+{
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// RESTORE = false: save <- theta, theta <- theta + beta_N m.
+// RESTORE = true:  theta <- save (m_region is not read).
+template <bool RESTORE>
+__global__ void __launch_bounds__(kLookThreads)
+novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec *__restrict__ recs,
+                  const float *__restrict__ m_region, float *__restrict__ save_region, float beta_n)
+{
+    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+        const Chunk ch = chunks[c];
+        const LookRec r = recs[ch.tensor];
+        float *p = r.p + ch.offset;
+        float *sv = save_region + r.state_off + ch.offset;
+        const float *m = RESTORE ? nullptr : m_region + r.state_off + ch.offset;
+        uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(sv);
+        if (!RESTORE) bits |= reinterpret_cast<uintptr_t>(m);
+        if ((bits & 15u) == 0) {
+            const int nvec = ch.len >> 2;
+            // two vectors per thread and pass: all loads first, then the stores
+            for (int i = threadIdx.x; i < nvec; i += 2 * kLookThreads) {
+                const int j = i + kLookThreads;
+                const bool two = j < nvec;
+                if (RESTORE) {
+                    const float4 a = ld_stream(sv + 4 * i);
+                    float4 b = a;
+                    if (two) b = ld_stream(sv + 4 * j);
+                    st_stream(p + 4 * i, a);
+                    if (two) st_stream(p + 4 * j, b);
+                } else {
+                    const float4 a = ld_stream(p + 4 * i);
+                    const float4 ma = ld_stream(m + 4 * i);
+                    float4 b = a, mb = ma;
+                    if (two) {
+                        b = ld_stream(p + 4 * j);
+                        mb = ld_stream(m + 4 * j);
+                    }
+                    st_stream(sv + 4 * i, a);
+                    st_stream(p + 4 * i, make_float4(fmaf(beta_n, ma.x, a.x), fmaf(beta_n, ma.y, a.y),
+                                                     fmaf(beta_n, ma.z, a.z), fmaf(beta_n, ma.w, a.w)));
+                    if (two) {
+                        st_stream(sv + 4 * j, b);
+                        st_stream(p + 4 * j, make_float4(fmaf(beta_n, mb.x, b.x), fmaf(beta_n, mb.y, b.y),
+                                                         fmaf(beta_n, mb.z, b.z), fmaf(beta_n, mb.w, b.w)));
+                    }
+                }
+            }
+            // ragged tail of a tensor: at most 3 elements
+            const int idx = (nvec << 2) + threadIdx.x;
+            if (idx < ch.len) {
+                if (RESTORE) {
+                    p[idx] = sv[idx];
+                } else {
+                    const float a = p[idx];
+                    sv[idx] = a;
+                    p[idx] = fmaf(beta_n, m[idx], a);
+                }
+            }
+        } else {
+            for (int i = threadIdx.x; i < ch.len; i += kLookThreads) {
+                if (RESTORE) {
+                    p[i] = sv[i];
+                } else {
+                    const float a = p[i];
+                    sv[i] = a;
+                    p[i] = fmaf(beta_n, m[i], a);
+                }
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
+                               const float *m_region, float *save_region, float beta_n, int grid,
+                               cudaStream_t stream)
+{
+    if (n_chunks <= 0) return cudaSuccess;
+    if (grid < 1 || grid > n_chunks) grid = n_chunks;
+    novak_look_kernel<false><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs, m_region,
+                                                                save_region, beta_n);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
+                           const float *save_region, int grid, cudaStream_t stream)
+{
+    if (n_chunks <= 0) return cudaSuccess;
+    if (grid < 1 || grid > n_chunks) grid = n_chunks;
+    // the kernel only reads the save buffer when restoring
+    novak_look_kernel<true><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs, nullptr,
+                                                               const_cast<float *>(save_region), 0.0f);
+    return cudaGetLastError();
+}
+
+}  // namespace novak

@@ -14,7 +14,7 @@ from paper_2601_07876_b200 import workloads as W
 RTOL, ATOL = 1e-5, 1e-7
 
 _NEST = {"none": O.NESTEROV_NONE, "approximation": O.NESTEROV_APPROX,
-         "classical": O.NESTEROV_CLASSICAL, "true": O.NESTEROV_APPROX}
+         "classical": O.NESTEROV_CLASSICAL, "true": O.NESTEROV_TRUE}
 _MODE = {"last": O.LOOKAHEAD_LAST, "traj_mean": O.LOOKAHEAD_TRAJ_MEAN}
 
 
@@ -34,7 +34,8 @@ def oracle_config(hyper: dict) -> O.Config:
         sparse_threshold=h.pop("sparse_threshold", 0.0),
         auto_lr=h.pop("auto_lr", False), auto_lr_gamma=h.pop("auto_lr_gamma", None) or 0.1,
         adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
-        tau2=h.pop("tau2", None) or 5000.0)
+        tau2=h.pop("tau2", None) or 5000.0,
+        true_steps=h.pop("true_nesterov_steps", 0))
 
 
 def tensor_rows(tensors):

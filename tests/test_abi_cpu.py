@@ -94,6 +94,40 @@ def test_true_nesterov_is_downgraded_with_warning():
     assert h2.get_info().warnings == 0
 
 
+def test_true_nesterov_steps_then_fallback_to_the_approximation():
+    """Section 5.2: with N_taylor > 0 the first N_taylor steps are true steps (no Eq. 13
+    correction to the gradient given), later ones the approximation; the warning goes."""
+    h = B.Handle(**{**GOOD, "nesterov_variant": B.NOVAK_NESTEROV_TRUE})
+    assert h.get_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS) == 0
+    h.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, 3)
+    assert h.get_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS) == 3
+    assert not (h.get_info().warnings & B.NOVAK_WARN_TRUE_DOWNGRADED)
+    got = [h.plan(t).nesterov_variant for t in range(1, 7)]
+    assert got == [B.NOVAK_NESTEROV_TRUE] * 3 + [B.NOVAK_NESTEROV_APPROX] * 3
+    # the oracle takes the same decision
+    from oracle import novak_oracle as O
+    olib = O.default_library()
+    hp = O.Config(nesterov_variant=O.NESTEROV_TRUE, true_steps=3).to_c()
+    import ctypes
+    assert [olib.novak_oracle_wants_extrapolation(ctypes.byref(hp), t) for t in range(1, 7)] == \
+        [int(v == B.NOVAK_NESTEROV_TRUE) for v in got]
+    h.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, 0)
+    assert h.get_info().warnings & B.NOVAK_WARN_TRUE_DOWNGRADED
+    assert h.plan(1).nesterov_variant == B.NOVAK_NESTEROV_APPROX
+    for bad in (-1, 2.5, float("nan"), 2.0 ** 31):
+        with pytest.raises(B.NovakError):
+            h.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, bad)
+    meta = h.export_meta()
+    assert meta.nesterov_variant == B.NOVAK_NESTEROV_TRUE and meta.true_nesterov_steps == 0
+    h.destroy()
+    # any other variant: the option is refused, the helpers too (nothing attached either)
+    g = B.Handle(**GOOD)
+    with pytest.raises(B.NovakError):
+        g.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, 5)
+    assert g.nesterov_save_bytes() == 0
+    g.destroy()
+
+
 def test_options_validate_and_roundtrip():
     h = B.Handle(**GOOD)
     assert h.get_option(B.NOVAK_OPT_NESTEROV_BETA) == 0.9   # default beta_N = beta1

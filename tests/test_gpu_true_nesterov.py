@@ -1,0 +1,150 @@
+"""True Nesterov momentum (Eq. 10-12) through the C ABI against the oracle: the
+look-ahead kernel, the bit-exact restore, the closed loop with a synthetic
+closure, the fallback after N_taylor steps and the state machine's refusals.
+
+The closure is a fixed seeded map of the look-ahead point, g~ = a * theta~ + b
+(a, b per element), evaluated ONCE per step in float64 from the oracle's theta~ and
+handed to both sides rounded to fp32, so that the two see the same gradient.
+"""
+import numpy as np
+import pytest
+import torch
+
+from harness import Pair, assert_close, make_tensors, to_f64
+from paper_2601_07876_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+RAGGED = [1, 2, 3, 5, 31, 33, 1023, 1025, 8191, 8193, 70001, 4096]
+BASE = dict(lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2, nesterov="true",
+            nesterov_beta=0.8, lookahead_k=5, lookahead_alpha=0.5)
+
+
+def _fresh(numels, offsets=None, seed=1, std=0.05):
+    flat, views, _ = make_tensors(numels, DEV, offsets)
+    g = torch.Generator(device=DEV).manual_seed(seed)
+    for v in views:
+        v.normal_(0.0, std, generator=g)
+    return flat, views
+
+
+def _closure(numels, seed=5):
+    rng = np.random.default_rng(seed)
+    a = [rng.uniform(0.5, 2.0, n) for n in numels]
+    b = [rng.normal(0.0, 1e-2, n) for n in numels]
+    return lambda points: [ai * x + bi for ai, bi, x in zip(a, b, points)]
+
+
+def _device_grads(gs64, offsets=None):
+    _, views, _ = make_tensors([g.size for g in gs64], DEV, offsets)
+    for v, g in zip(views, gs64):
+        v.copy_(torch.from_numpy(g.astype(np.float32)).to(DEV))
+    return views
+
+
+@pytest.mark.parametrize("offsets", [None, "phased"])
+def test_closed_loop_with_fallback(offsets):
+    """N_taylor = 4 of 9 steps: look ahead, compare theta~ with Eq. 10, restore bit for
+    bit, step on the closure's gradient; from step 5 on plain steps (Eq. 13)."""
+    offs = [(i % 4) if i % 3 == 2 else 0 for i in range(len(RAGGED))] if offsets else None
+    _, params = _fresh(RAGGED, offs)
+    pair = Pair(params, dict(BASE, true_nesterov_steps=4))
+    grad_of = _closure(RAGGED)
+    wanted = []
+    for t in range(1, 10):
+        want = pair.opt.wants_extrapolation()
+        assert want == pair.oracle.wants_extrapolation()
+        wanted.append(want)
+        if want:
+            before = [p.clone() for p in params]
+            pair.opt.extrapolate()
+            point = pair.oracle.extrapolated()
+            for i, p in enumerate(params):
+                assert_close(p, point[i], f"t={t} theta~[{i}]")
+            gs = grad_of(point)
+            pair.opt.restore()
+            for p, b in zip(params, before):
+                assert torch.equal(p, b), "restore must be bit-exact"
+        else:
+            gs = grad_of(pair.oracle.theta)
+        pair.step(_device_grads(gs, offs))
+        assert pair.opt.info()["nesterov_variant"] == (
+            B.NOVAK_NESTEROV_TRUE if want else B.NOVAK_NESTEROV_APPROX)
+        if t in (1, 4, 5):
+            pair.check(f"t={t}")
+    pair.check("end")
+    assert wanted == [True] * 4 + [False] * 5
+    assert not pair.opt.info()["warnings"] & B.NOVAK_WARN_TRUE_DOWNGRADED
+
+
+def test_first_look_ahead_is_the_identity_and_m_is_read_not_written():
+    _, params = _fresh([5000, 77])
+    opt = B.NovakOptimizer(params, **dict(BASE, true_nesterov_steps=10))
+    before = [p.clone() for p in params]
+    opt.extrapolate()
+    torch.cuda.synchronize()
+    for p, b in zip(params, before):
+        assert torch.equal(p, b)            # m_0 = 0
+    opt.restore()
+    g = [torch.full_like(p, 0.5) for p in params]
+    opt.step(g)
+    m = [opt.state(i)["m"].clone() for i in range(2)]
+    th = [p.clone() for p in params]
+    opt.extrapolate()
+    for i, p in enumerate(params):
+        assert torch.equal(opt.state(i)["m"], m[i])
+        # one fused multiply-add per element: theta + 0.8 m, rounded once
+        want = (th[i].double() + np.float32(0.8).astype(np.float64) * m[i].double()).float()
+        assert torch.equal(p, want)
+    opt.restore()
+    for p, b in zip(params, th):
+        assert torch.equal(p, b)
+
+
+def test_state_machine_refusals():
+    _, params = _fresh([4096, 100])
+    opt = B.NovakOptimizer(params, **dict(BASE, true_nesterov_steps=2))
+    g = [torch.zeros_like(p) for p in params]
+    with pytest.raises(B.NovakError):
+        opt.handle.nesterov_restore(opt._params_arr, params[0].data_ptr(), 1 << 30, opt._numel_arr,
+                                    opt.n, 0)                      # nothing to restore
+    opt.extrapolate()
+    with pytest.raises(B.NovakError):
+        opt.extrapolate()                                          # twice
+    with pytest.raises(B.NovakError):
+        opt.step(g)                                                # would step on theta~
+    with pytest.raises(B.NovakError):
+        opt.handle.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, 7)
+    other = torch.empty(opt.handle.nesterov_save_bytes(), dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.NovakError):
+        opt.handle.nesterov_restore(opt._params_arr, other.data_ptr(), other.numel(),
+                                    opt._numel_arr, opt.n, 0)      # another save buffer
+    opt.restore()
+    opt.step(g)
+    assert opt.info()["t"] == 1
+    # short and misaligned save buffers
+    need = opt.handle.nesterov_save_bytes()
+    buf = torch.empty(need + 64, dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.NovakError):
+        opt.handle.nesterov_extrapolate(opt._params_arr, buf.data_ptr(), need - 4, opt._numel_arr,
+                                        opt.n, 0)
+    with pytest.raises(B.NovakError):
+        opt.handle.nesterov_extrapolate(opt._params_arr, buf.data_ptr() + 4, need, opt._numel_arr,
+                                        opt.n, 0)
+    # a handle of another variant has no look-ahead
+    plain = B.NovakOptimizer(params, **dict(BASE, nesterov="approximation"))
+    with pytest.raises(B.NovakError):
+        plain.extrapolate()
+
+
+def test_checkpoint_carries_the_true_variant():
+    _, params = _fresh([3000])
+    a = B.NovakOptimizer(params, **dict(BASE, true_nesterov_steps=6))
+    a.step([torch.ones_like(params[0])])
+    sd = a.state_dict()
+    b = B.NovakOptimizer(params, **dict(BASE))          # N_taylor = 0 until the import
+    b.load_state_dict(sd)
+    assert b.handle.get_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS) == 6
+    assert b.wants_extrapolation() and b.info()["t"] == 1
+    assert not b.info()["warnings"] & B.NOVAK_WARN_TRUE_DOWNGRADED
