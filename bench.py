@@ -93,6 +93,10 @@ def parse_args():
                     help="Eq. 20-22: statistics pass plus one more read of the parameters")
     ap.add_argument("--bf16-copy", action="store_true",
                     help="the step also writes a bf16 copy of the parameters (+2 B per element)")
+    ap.add_argument("--true-nesterov", action="store_true",
+                    help="every step is a true-Nesterov step (Eq. 10-12): look-ahead kernel, "
+                         "restore kernel, step; the closure between the two is the caller's "
+                         "and not part of the step (+24 B per element)")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -110,7 +114,8 @@ def parse_args():
 
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
                                phase2: bool = False, trust: bool = False,
-                               copy16: bool = False, auto: bool = False) -> int:
+                               copy16: bool = False, auto: bool = False,
+                               true_nesterov: bool = False) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
     arrays on the steps that touch them, plus one more read of g when clipping or
@@ -122,6 +127,8 @@ def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
         b += 2
     if auto:
         b += 4                           # ||theta_t|| of Eq. 21
+    if true_nesterov:
+        b += 16 + 8                      # Eq. 10: theta, m read, save, theta written; restore
     if k <= 0:
         return b
     sync = t % k == 0
@@ -280,6 +287,8 @@ def cpu_baseline(wl, hyper, seconds):
     o.step([g], threads=cores)
     steps, t0 = 0, time.perf_counter()
     while time.perf_counter() - t0 < seconds and steps < 5000:
+        if o.wants_extrapolation():
+            o.extrapolated()             # Eq. 10 (the oracle's restore is a no-op)
         o.step([g], threads=cores)
         steps += 1
     dt = time.perf_counter() - t0
@@ -381,6 +390,8 @@ def main():
     lib = B.load_library(args.lib) if args.lib else None
     wl = W.get_workload(args.config)
     hyper = dict(wl.hyper, lookahead_mode=args.lookahead_mode)
+    if args.true_nesterov:
+        hyper.update(nesterov="true", true_nesterov_steps=2 ** 31 - 1)
     k = hyper["lookahead_k"]
     gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
 
@@ -411,6 +422,14 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    plain_step = opt.step
+    if args.true_nesterov:
+        def true_step(grads):
+            opt.extrapolate()
+            opt.restore()                # the caller's closure would run between the two
+            plain_step(grads)
+        opt.step = true_step
+
     # ---------------- resident timing: exactly K steps between two events
     for i in range(max(3, args.warmup)):
         opt.step(pool[i % pool_n])
@@ -435,13 +454,14 @@ def main():
     ms_per_step = ms / args.steps
     value = world * wl.total * args.steps / (ms * 1e-3)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
-                                         args.layer_adaptation, args.bf16_copy, args.auto_lr)
+                                         args.layer_adaptation, args.bf16_copy, args.auto_lr,
+                                         args.true_nesterov)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy or args.true_nesterov) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -522,6 +542,7 @@ def main():
                 "clip_threshold": args.clip, "centralize": bool(args.centralize),
                 "layer_adaptation": bool(args.layer_adaptation),
                 "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
+                "true_nesterov": bool(args.true_nesterov),
                 "auto_lr": bool(args.auto_lr),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
