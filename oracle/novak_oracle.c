@@ -65,6 +65,14 @@
  *     N_taylor + 1 on the variant is the approximation of Eq. 13 (Section 5.2's
  *     automatic fallback).                                 [parity unpinned]
  *
+ *   - Moments stored in bfloat16 (Section 10's "storing moments in bfloat16
+ *     while accumulating updates in float32", named as future work): m_{t-1}
+ *     and v_{t-1} are read back as stored, the step's own arithmetic (Eq. 1-2,
+ *     5, 17) runs on the unrounded m_t, v_t, and what is stored for the next
+ *     step is each of them rounded to the nearest bfloat16 (8 significant
+ *     bits, fp32's exponent range, ties to even).  The paper fixes neither the
+ *     rounding nor whether the step sees rounded values.   [parity unpinned]
+ *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
  * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
  */
@@ -90,8 +98,26 @@ typedef struct {
     double tau2;             /* warm-up time scale of beta2 (paper: 5000)   */
     double sparse_threshold; /* tau of Eq. 27; 0 = no mask                  */
     int32_t true_steps;      /* N_taylor: steps 1..N_taylor of variant 3 take g~ */
-    int32_t reserved;
+    int32_t moment_bf16;     /* 1: m and v are stored rounded to bfloat16        */
 } novak_oracle_hparams;
+
+/* Nearest bfloat16 to x, ties to even: 1 sign bit, 8 exponent bits (fp32's
+ * range: normal numbers from 2^-126, subnormals in steps of 2^-133, overflow
+ * to infinity) and 8 significant bits (7 stored). */
+double novak_oracle_round_bf16(double x)
+{
+    if (x == 0.0 || isnan(x) || isinf(x))
+        return x;
+    int e;
+    (void)frexp(x, &e);              /* |x| = f 2^e with f in [0.5, 1) */
+    int q = e - 8;                   /* quantum 2^q leaves 8 significant bits */
+    if (q < -133)
+        q = -133;                    /* subnormal range: fixed quantum */
+    const double r = ldexp(rint(ldexp(x, -q)), q);   /* rint: to nearest, ties to even */
+    if (fabs(r) >= ldexp(1.0, 128))
+        return x > 0.0 ? INFINITY : -INFINITY;
+    return r;
+}
 
 /* Whether step t applies the correction of Eq. 13 to the gradient it is given:
  * always for the approximation variant; for the true variant only once the
@@ -235,6 +261,13 @@ void novak_oracle_step(const novak_oracle_hparams *h, int64_t t, int64_t n,
         /* Phase 9: Eq. 18 then Eq. 24 (decay with the base rate alpha). */
         double theta_fast = theta[i] * s.decay - s.step_size * trust * u;
 
+        /* Reduced-precision storage: the step above used the unrounded moments;
+         * the next step reads back their bfloat16 roundings. */
+        if (h->moment_bf16) {
+            m[i] = novak_oracle_round_bf16(m[i]);
+            v[i] = novak_oracle_round_bf16(v[i]);
+        }
+
         /* Phase 10: lookahead. */
         if (k <= 0) {
             theta[i] = theta_fast;
@@ -324,6 +357,49 @@ void novak_oracle_direction(const novak_oracle_hparams *h, int64_t t, int64_t n,
         const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
         const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
         u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);
+    }
+}
+
+/* Distance from x to the nearest point where bfloat16 rounding changes its
+ * answer (the midpoint between two neighbouring bfloat16 values). */
+static double bf16_boundary_distance(double x)
+{
+    if (x == 0.0 || isnan(x) || isinf(x))
+        return INFINITY;
+    int e;
+    (void)frexp(x, &e);
+    int q = e - 8;
+    if (q < -133)
+        q = -133;
+    const double y = ldexp(fabs(x), -q);
+    return ldexp(fabs(y - floor(y) - 0.5), q);
+}
+
+/* For tests of the bfloat16 storage: how close the unrounded m_t and v_t that
+ * step t would produce come to a rounding boundary, relative to the size of
+ * the terms they are summed from (so that cancellation is accounted for), the
+ * smaller of the two per element.  An implementation in lower precision can
+ * round an element differently only where this is of the order of its own
+ * rounding error.  Nothing is written but margin_out. */
+void novak_oracle_rounding_margin(const novak_oracle_hparams *h, int64_t t, int64_t n,
+                                  const double *g, const double *m, const double *v,
+                                  double *margin_out)
+{
+    novak_oracle_scalars s;
+    novak_oracle_scalars_at(h, t, &s);
+    for (int64_t i = 0; i < n; ++i) {
+        double gt = g[i], g_scale = fabs(g[i]);
+        if (approximation_active(h, t)) {
+            gt = g[i] + h->nesterov_beta * (g[i] - m[i]);
+            g_scale = fabs(g[i]) + h->nesterov_beta * (fabs(g[i]) + fabs(m[i]));
+        }
+        const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;
+        const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;
+        const double m_scale = s.beta1_t * fabs(m[i]) + (1.0 - s.beta1_t) * g_scale;
+        const double v_scale = s.beta2_t * v[i] + (1.0 - s.beta2_t) * g_scale * g_scale;
+        double a = m_scale > 0.0 ? bf16_boundary_distance(m_new) / m_scale : INFINITY;
+        double b = v_scale > 0.0 ? bf16_boundary_distance(v_new) / v_scale : INFINITY;
+        margin_out[i] = a < b ? a : b;
     }
 }
 

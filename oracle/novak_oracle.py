@@ -46,7 +46,7 @@ class HParams(ctypes.Structure):
         ("tau2", ctypes.c_double),
         ("sparse_threshold", ctypes.c_double),
         ("true_steps", ctypes.c_int32),
-        ("reserved", ctypes.c_int32),
+        ("moment_bf16", ctypes.c_int32),
     ]
 
 
@@ -108,6 +108,11 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.novak_oracle_scale.restype = None
     lib.novak_oracle_centralize.argtypes = [ctypes.c_int64, ctypes.c_int64, dp]
     lib.novak_oracle_centralize.restype = None
+    lib.novak_oracle_round_bf16.argtypes = [ctypes.c_double]
+    lib.novak_oracle_round_bf16.restype = ctypes.c_double
+    lib.novak_oracle_rounding_margin.argtypes = [
+        ctypes.POINTER(HParams), ctypes.c_int64, ctypes.c_int64, dp, dp, dp, dp]
+    lib.novak_oracle_rounding_margin.restype = None
     lib.novak_oracle_extrapolate.argtypes = [ctypes.c_double, ctypes.c_int64, dp, dp, dp]
     lib.novak_oracle_extrapolate.restype = None
     lib.novak_oracle_wants_extrapolation.argtypes = [ctypes.POINTER(HParams), ctypes.c_int64]
@@ -152,6 +157,7 @@ class Config:
     auto_lr: bool = False                # Eq. 20-22
     auto_lr_gamma: float = 0.1
     true_steps: int = 0                  # N_taylor of the true variant (Section 5.2)
+    moment_bf16: bool = False            # m, v stored rounded to bfloat16
 
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
@@ -160,7 +166,7 @@ class Config:
                        self.nesterov_variant, self.lookahead_k,
                        self.lookahead_mode, int(self.rectified),
                        self.bias1_power, int(self.adaptive_beta), self.tau1, self.tau2,
-                       self.sparse_threshold, self.true_steps, 0)
+                       self.sparse_threshold, self.true_steps, int(self.moment_bf16))
 
 
 def _dptr(a: np.ndarray, offset: int = 0):
@@ -199,6 +205,8 @@ class Oracle:
                     else None)
         self.t = 0
         self.track_threshold_margin = False
+        self.track_rounding_margin = False
+        self.rounding_margin = [np.full(p.size, np.inf) for p in self.theta]
         self.threshold_margin = [np.full(p.size, np.inf) for p in self.theta]
         self.sync_steps: list[int] = []
         self.rect_flags: list[int] = []
@@ -308,6 +316,16 @@ class Oracle:
                                                 _dptr(self.m[i]), _dptr(self.v[i]), _dptr(u))
                 rel = np.abs(np.abs(u) / self.cfg.sparse_threshold - 1.0)
                 self.threshold_margin[i] = np.minimum(self.threshold_margin[i], rel)
+        if self.cfg.moment_bf16 and self.track_rounding_margin:
+            # how close the unrounded moments come to a bfloat16 rounding boundary, per
+            # element, over the whole run (for tests: fp32 arithmetic may round an
+            # element the other way right at a boundary)
+            for i, g in enumerate(gs):
+                mg = np.empty_like(g)
+                self.lib.novak_oracle_rounding_margin(ctypes.byref(self.h), self.t, g.size,
+                                                      _dptr(g), _dptr(self.m[i]),
+                                                      _dptr(self.v[i]), _dptr(mg))
+                self.rounding_margin[i] = np.minimum(self.rounding_margin[i], mg)
         trust = [1.0] * len(gs)
         if self.cfg.layer_adaptation:
             trust = [self.lib.novak_oracle_trust_ratio(

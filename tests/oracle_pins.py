@@ -13,6 +13,7 @@ in float64), worked examples and invariants (Prop. 6.3-6.5).
 """
 from __future__ import annotations
 
+import ctypes
 import math
 
 import numpy as np
@@ -767,7 +768,7 @@ def pin_true_nesterov(lib):
               rectified=False, nesterov_beta=bN)
     # hand values of theta + beta_N m
     out = np.empty(3)
-    th = np.array([1.0, -2.0, 0.5]); m = np.array([0.5, 0.25, -1.0])
+    th = np.array([1.0, -2.0, 0.5]); m = np.array([0.5, 0.25, -1.0])   # named: _dptr keeps no reference
     lib.novak_oracle_extrapolate(bN, 3, O._dptr(th), O._dptr(m), O._dptr(out))
     _close(out, np.array([1.4, -1.8, -0.3]), what="Eq. 10 by hand")
     # after one step from zero moments: theta_1 = theta_0 d - lr g/(|g|+eps), m_1 = (1-b1) g
@@ -823,6 +824,86 @@ def pin_true_nesterov(lib):
     assert not np.array_equal(tr.theta[0], z.theta[0])
 
 
+# --------------------------------------------------------------------------
+# Moments stored in bfloat16 (Section 10)
+# --------------------------------------------------------------------------
+def pin_bf16_moment_storage(lib):
+    """The rounding against torch's fp32 -> bfloat16 conversion (random values, exact
+    ties, subnormals, overflow); the stored moments are the roundings of what the plain
+    step computes; the step itself uses the unrounded values; a second moment that
+    cannot move under round-to-nearest (beta2 = 0.999 changes v by less than half a
+    step of its 8-bit grid) stays put."""
+    rnd = lambda a: np.array([lib.novak_oracle_round_bf16(float(x)) for x in a])
+    rng = np.random.default_rng(11)
+    x = (rng.normal(0, 1, 4000) * 10.0 ** rng.uniform(-30, 30, 4000)).astype(np.float32)
+    ties = (1.0 + np.arange(0, 64) * 2.0 ** -8).astype(np.float32)          # odd multiples: ties
+    sub = (np.arange(1, 300) * 2.0 ** -140).astype(np.float32)             # below 2^-126
+    big = np.array([3.38e38, 3.39e38, 3.4e38, -3.4e38, 2.0 ** 127, 1.5 * 2.0 ** 127], np.float32)
+    for arr in (x, ties, -ties, sub, -sub, big, np.array([0.0, -0.0], np.float32)):
+        want = torch.from_numpy(arr).to(torch.bfloat16).to(torch.float64).numpy()
+        got = rnd(arr.astype(np.float64))
+        assert np.array_equal(got, want), "round_bf16 differs from torch"
+    assert rnd([1.0 + 2.0 ** -8])[0] == 1.0 and rnd([1.0 + 3 * 2.0 ** -8])[0] == 1.0 + 2.0 ** -6
+    assert rnd([1.0 + 2.0 ** -8 + 2.0 ** -40])[0] == 1.0 + 2.0 ** -7      # just above a tie
+    # one step from a bf16-representable state: same theta as the plain step (the update
+    # sees the unrounded moments), stored moments = roundings of the plain step's moments
+    kw = dict(lr=1e-2, weight_decay=0.1, eps=1e-3, lookahead_k=0, rectified=False)
+    th = rng.normal(0, 1, 64)
+    g1, g2 = rng.normal(0, 1, 64), rng.normal(0, 1, 64)
+    a = _mk(lib, [th], moment_bf16=True, **kw)
+    b = _mk(lib, [th], **kw)
+    a.step([g1]); b.step([g1])
+    assert np.array_equal(a.theta[0], b.theta[0])
+    assert np.array_equal(a.m[0], rnd(b.m[0])) and np.array_equal(a.v[0], rnd(b.v[0]))
+    assert not np.array_equal(a.m[0], b.m[0])
+    # second step: reads the ROUNDED moments back (a plain run started from them agrees)
+    c = _mk(lib, [a.theta[0]], **kw)
+    c.m[0][:] = a.m[0]; c.v[0][:] = a.v[0]; c.t = 1
+    a.step([g2]); c.step([g2])
+    assert np.array_equal(a.theta[0], c.theta[0])
+    assert np.array_equal(a.m[0], rnd(c.m[0])) and np.array_equal(a.v[0], rnd(c.v[0]))
+    assert not np.array_equal(a.theta[0], _two_plain_steps(lib, th, g1, g2, kw))
+    # every stored value has at most 8 significant bits and lies within half a grid step
+    for arr, ref in ((a.m[0], c.m[0]), (a.v[0], c.v[0])):
+        mant, _ = np.frexp(arr)
+        assert np.array_equal(mant * 256, np.round(mant * 256))
+        assert np.all(np.abs(arr - ref) <= np.abs(ref) * 2.0 ** -8)
+    # stagnation: v = 1, g = 0: 0.999 rounds back to 1 (grid step 2^-8 below 1), m decays
+    z = _mk(lib, [np.ones(1)], moment_bf16=True, nesterov_variant=O.NESTEROV_NONE, **kw)
+    z.v[0][:] = 1.0; z.m[0][:] = 1.0
+    for _ in range(10):
+        z.step([np.zeros(1)])
+    assert z.v[0][0] == 1.0
+    mm = 1.0
+    for _ in range(10):
+        mm = lib.novak_oracle_round_bf16(0.9 * mm)
+    assert z.m[0][0] == mm and 0.3 < mm < 0.4
+    # the margin helper: distance to the nearest midpoint over the sum of the terms
+    mg = np.empty(1)
+    hp = O.Config(moment_bf16=True, nesterov_variant=O.NESTEROV_NONE, beta1=0.5, beta2=0.5).to_c()
+    # m_new = 0.5*1 + 0.5*(1 + 2^-6) = 1 + 2^-7: on the grid, 2^-8 from both midpoints
+    # v_new = 0.5*v + 0.5*g^2 with v chosen so that v_new = 1 + 2^-8 (a midpoint) -> margin 0
+    gq = 1.0 + 2.0 ** -6
+    vq = 2.0 * (1.0 + 2.0 ** -8) - gq * gq
+    ga, ma, va, vb = np.array([gq]), np.array([1.0]), np.array([vq]), np.array([gq * gq])
+    lib.novak_oracle_rounding_margin(ctypes.byref(hp), 1, 1, O._dptr(ga), O._dptr(ma), O._dptr(va),
+                                     O._dptr(mg))
+    assert mg[0] == 0.0
+    lib.novak_oracle_rounding_margin(ctypes.byref(hp), 1, 1, O._dptr(ga), O._dptr(ma), O._dptr(vb),
+                                     O._dptr(mg))
+    # m_new = 1 + 2^-7 sits 2^-8 from its midpoints; v_new = gq^2 = 1 + 2^-5 + 2^-12 sits
+    # 2^-8 - 2^-12 from one: the smaller ratio is reported
+    _close(mg, np.array([min(2.0 ** -8 / (1.0 + 2.0 ** -7), (2.0 ** -8 - 2.0 ** -12) / (gq * gq))]),
+           what="margin at step 1")
+    assert (2.0 ** -8 - 2.0 ** -12) / (gq * gq) < 2.0 ** -8 / (1.0 + 2.0 ** -7)
+
+
+def _two_plain_steps(lib, th, g1, g2, kw):
+    o = _mk(lib, [th], **kw)
+    o.step([g1]); o.step([g2])
+    return o.theta[0]
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -847,4 +928,5 @@ ALL_PINS = [
     pin_sparse_mask,
     pin_auto_lr,
     pin_true_nesterov,
+    pin_bf16_moment_storage,
 ]

@@ -65,6 +65,20 @@ MUTANTS = [
     ("fallback_never", "return t > (int64_t)h->true_steps;", "return 0;"),
     ("true_corrected_from_the_start", "return t > (int64_t)h->true_steps;", "return 1;"),
     ("wants_off_by_one", "t <= (int64_t)h->true_steps) ? 1 : 0", "t < (int64_t)h->true_steps) ? 1 : 0"),
+    # moments stored in bfloat16
+    ("bf16_truncates", "ldexp(rint(ldexp(x, -q)), q);", "ldexp(trunc(ldexp(x, -q)), q);"),
+    ("bf16_ties_away", "ldexp(rint(ldexp(x, -q)), q);", "ldexp(round(ldexp(x, -q)), q);"),
+    ("bf16_seven_bits", "int q = e - 8;                   /* quantum", "int q = e - 7;                   /* quantum"),
+    ("bf16_no_subnormals", "if (q < -133)\n        q = -133;                    /* subnormal", "if (0)\n        q = -133;                    /* subnormal"),
+    ("bf16_no_overflow", "if (fabs(r) >= ldexp(1.0, 128))", "if (0)"),
+    ("bf16_step_sees_rounded_m", "double m_hat = m[i] / s.bc1;",
+     "if (h->moment_bf16) m[i] = novak_oracle_round_bf16(m[i]); double m_hat = m[i] / s.bc1;"),
+    ("bf16_step_sees_rounded_v", "double v_hat = v[i] / s.bc2;",
+     "if (h->moment_bf16) v[i] = novak_oracle_round_bf16(v[i]); double v_hat = v[i] / s.bc2;"),
+    ("bf16_v_kept_exact", "            v[i] = novak_oracle_round_bf16(v[i]);\n", ""),
+    ("bf16_m_kept_exact", "            m[i] = novak_oracle_round_bf16(m[i]);\n", ""),
+    ("bf16_margin_to_grid_point", "ldexp(fabs(y - floor(y) - 0.5), q);", "ldexp(fabs(y - floor(y)), q);"),
+    ("bf16_margin_ignores_v", "margin_out[i] = a < b ? a : b;", "margin_out[i] = a;"),
     # phase 7: automatic learning-rate scaling
     ("auto_inverted", "double a = *g_bar / *theta_bar;", "double a = *theta_bar / *g_bar;"),
     ("auto_gamma_swapped", "*g_bar = gamma * grad_norm + (1.0 - gamma) * *g_bar;",
