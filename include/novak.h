@@ -67,6 +67,17 @@ enum {
 
 enum { NOVAK_GRAD_F32 = 0, NOVAK_GRAD_BF16 = 1 };
 
+/* Storage type of the moments m and v (NOVAK_OPT_MOMENT_DTYPE).  BF16 is
+ * Section 10's "moments in bfloat16, updates accumulated in float32": a step
+ * reads the stored values back, does all of its arithmetic (Eq. 1-2, 5, 17) in
+ * fp32 on the unrounded m_t, v_t, and stores each rounded to the nearest
+ * bfloat16, ties to even.  20 B per element and step instead of 28 (fp32
+ * gradients).  With beta2 = 0.999 a step changes v by about a quarter of the
+ * spacing of bfloat16 values, so round-to-nearest can hold v still for long
+ * stretches; the paper names that sensitivity and gives no remedy, and none is
+ * applied here. */
+enum { NOVAK_MOMENT_F32 = 0, NOVAK_MOMENT_BF16 = 1 };
+
 /* Lookahead rule applied on steps with t mod k == 0 (Section 4.7).
  * LAST:      slow += alpha_LA (theta_fast - slow); theta = slow.
  *            The slow weights are read and written on those steps only.
@@ -129,6 +140,8 @@ enum {
                                      evaluated at Eq. 10's point; later steps run
                                      APPROX.  0 (default): APPROX from the first step.
                                      NOVAK_ESTATE for any other variant             */
+    NOVAK_OPT_MOMENT_DTYPE = 22,  /* NOVAK_MOMENT_*: storage type of m and v; only
+                                     before attach (default NOVAK_MOMENT_F32)          */
     NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base
                                      directions with |u| <= tau are set to zero before
                                      the classical blend; 0 (default): no mask.  The
@@ -173,7 +186,7 @@ typedef struct novak_info {
     double beta1_t, beta2_t; /* coefficients the last step's Eq. 1-2 used: the base
                                 values, or Eq. 3-4 with NOVAK_OPT_ADAPTIVE_BETA     */
     int32_t layer_adaptation;
-    int32_t reserved2;
+    int32_t moment_dtype;    /* NOVAK_MOMENT_*                                      */
 } novak_info;
 
 /* Counters and hyperparameters for checkpoint / resume (Table 3: t and the
@@ -196,6 +209,8 @@ typedef struct novak_meta {
     double auto_lr_gamma;
     int32_t auto_lr;
     int32_t true_nesterov_steps; /* N_taylor; nesterov_variant is TRUE when requested */
+    int32_t moment_dtype;    /* NOVAK_MOMENT_*; must match the handle's on import   */
+    int32_t reserved;
 } novak_meta;
 
 /* Algorithm 1, Input / Section 5.8 "Hyperparameter validation".
@@ -215,13 +230,13 @@ void novak_destroy(novak_opt *opt);
 /* Options not in novak_create's list (Algorithm 1, Hyperparameters).  Values
  * are validated like novak_create's (NOVAK_EINVAL); keys that change the
  * state layout or the chunk table return NOVAK_ESTATE once state is attached
- * (LOOKAHEAD_MODE) or a step was taken (CHUNK_ELEMS). */
+ * (LOOKAHEAD_MODE, MOMENT_DTYPE) or a step was taken (CHUNK_ELEMS). */
 int novak_set_option(novak_opt *opt, int key, double value);
 int novak_get_option(const novak_opt *opt, int key, double *value);
 
 /* Table 3: bytes of optimizer state for n tensors of numel[i] fp32 elements:
- * m and v always, the slow weights when lookahead_k > 0, the running sum in
- * TRAJ_MEAN mode.  Includes per-tensor padding (each tensor's slice may start
+ * m and v always (fp32, or 2 bytes each under NOVAK_MOMENT_BF16), the slow
+ * weights when lookahead_k > 0, the running sum in TRAJ_MEAN mode (both fp32).  Includes per-tensor padding (each tensor's slice may start
  * up to 31 elements into a 128-byte aligned slot so that it shares the
  * parameter's alignment).  Returns 0 on bad arguments. */
 size_t novak_state_bytes(const novak_opt *opt, const int64_t *numel, int n);
@@ -459,7 +474,9 @@ int novak_get_info(const novak_opt *opt, novak_info *out);
 int novak_plan(const novak_opt *opt, int64_t t, novak_info *out);
 
 /* Device pointers of tensor i's state slices (NULL for arrays the mode does
- * not keep).  For checkpointing and for tests; valid after attach. */
+ * not keep): numel[i] elements each, fp32 but for m and v under
+ * NOVAK_MOMENT_BF16 (bfloat16).  For checkpointing and for tests; valid after
+ * attach. */
 int novak_state_ptrs(const novak_opt *opt, int tensor, void **d_m, void **d_v,
                      void **d_slow, void **d_acc);
 

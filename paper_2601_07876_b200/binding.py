@@ -29,7 +29,8 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
  NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
- NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS) = range(1, 22)
+ NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS, NOVAK_OPT_MOMENT_DTYPE) = range(1, 23)
+NOVAK_MOMENT_F32, NOVAK_MOMENT_BF16 = 0, 1
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
@@ -46,7 +47,7 @@ class novak_info(Structure):
         ("n_chunks", c_int32), ("grid", c_int32), ("block", c_int32), ("warnings", c_uint32),
         ("grad_processing", c_int32), ("reserved", c_int32),
         ("beta1_t", c_double), ("beta2_t", c_double),
-        ("layer_adaptation", c_int32), ("reserved2", c_int32),
+        ("layer_adaptation", c_int32), ("moment_dtype", c_int32),
     ]
 
     def as_dict(self) -> dict:
@@ -65,6 +66,7 @@ class novak_meta(Structure):
         ("beta1_tau", c_double), ("beta2_tau", c_double), ("adaptive_beta", c_int32),
         ("layer_adaptation", c_int32), ("sparse_threshold", c_double),
         ("auto_lr_gamma", c_double), ("auto_lr", c_int32), ("true_nesterov_steps", c_int32),
+        ("moment_dtype", c_int32), ("reserved", c_int32),
     ]
 
 
@@ -393,7 +395,7 @@ class NovakOptimizer:
                  nesterov_beta=None, lookahead_mode="last", rectified=True, bias1_power=1,
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
-                 auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0,
+                 auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0, moment_dtype="f32",
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -412,6 +414,10 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_NESTEROV_BETA, nesterov_beta)
         mode = _LA_MODE[lookahead_mode] if isinstance(lookahead_mode, str) else int(lookahead_mode)
         h.set_option(NOVAK_OPT_LOOKAHEAD_MODE, mode)
+        self.moment_bf16 = moment_dtype in ("bf16", NOVAK_MOMENT_BF16)
+        if not self.moment_bf16 and moment_dtype not in ("f32", NOVAK_MOMENT_F32):
+            raise ValueError("moment_dtype must be 'f32' or 'bf16'")
+        h.set_option(NOVAK_OPT_MOMENT_DTYPE, NOVAK_MOMENT_BF16 if self.moment_bf16 else NOVAK_MOMENT_F32)
         h.set_option(NOVAK_OPT_RECTIFIED, 1 if rectified else 0)
         h.set_option(NOVAK_OPT_BIAS1_POWER, bias1_power)
         if chunk_elems is not None:
@@ -553,17 +559,21 @@ class NovakOptimizer:
     def plan(self, t: int) -> dict:
         return self.handle.plan(t).as_dict()
 
-    def _view(self, ptr, numel):
+    def _view(self, ptr, numel, bf16=False):
+        import torch
         if not ptr:
             return None
         off = ptr - self.state_buffer.data_ptr()
+        if bf16:
+            return self.state_buffer[off: off + 2 * numel].view(torch.bfloat16)
         return self.state_buffer[off: off + 4 * numel].view(self.params[0].dtype)
 
     def state(self, i: int) -> dict:
         """Views (no copies) of tensor i's state slices inside the state buffer."""
         m, v, s, a = self.handle.state_ptrs(i)
         n = self.numel[i]
-        return {"m": self._view(m, n), "v": self._view(v, n), "slow": self._view(s, n),
+        b = self.moment_bf16
+        return {"m": self._view(m, n, b), "v": self._view(v, n, b), "slow": self._view(s, n),
                 "acc": self._view(a, n)}
 
     def state_dict(self) -> dict:

@@ -18,7 +18,10 @@ SOURCES = [os.path.join(CSRC, f) for f in (
     "novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu",
     "novak_grad_stats.cu", "novak_trust_stats.cu", "novak_nesterov.cu",
     "novak_step_pre0.cu", "novak_step_pre1.cu", "novak_step_pre2.cu",
-    "novak_step_pre0_copy.cu", "novak_step_pre1_copy.cu", "novak_step_pre2_copy.cu")]
+    "novak_step_pre0_copy.cu", "novak_step_pre1_copy.cu", "novak_step_pre2_copy.cu",
+    "novak_step_pre0_mom16.cu", "novak_step_pre1_mom16.cu", "novak_step_pre2_mom16.cu",
+    "novak_step_pre0_copy_mom16.cu", "novak_step_pre1_copy_mom16.cu",
+    "novak_step_pre2_copy_mom16.cu")]
 HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(CSRC, "novak_handle.h"),
            os.path.join(CSRC, "novak_step_types.h"),
            os.path.join(CSRC, "novak_step_kernel.cuh"),

@@ -41,6 +41,7 @@ struct Hyper {
     double auto_gamma;      // gamma of Eq. 20-21
     int true_requested;     // the caller asked for the true variant (Eq. 10-12)
     int true_steps;         // N_taylor: steps 1..N_taylor take Eq. 11's gradient as given
+    int mom16;              // m and v stored as bf16 (fixed at attach: it sets the layout)
 };
 
 struct Plan {
@@ -183,7 +184,12 @@ int fail_cuda(novak_opt *o, cudaError_t e, const char *what);
 
 // State layout and mode helpers.
 int n_state_arrays(const Hyper &h);
-float *slice(const novak_opt *o, int array, int i);
+// Start of tensor i inside state array `array` (0 m, 1 v, 2 slow, 3 running
+// sum): m and v hold fp32 or bf16 elements, the lookahead arrays fp32.
+void *slice(const novak_opt *o, int array, int i);
+inline int moment_bytes(const Hyper &h) { return h.mom16 ? 2 : 4; }
+// Bytes of the whole state for a region of `region_elems` padded elements.
+size_t state_bytes_for(const Hyper &h, int64_t region_elems);
 int pre_mode(const novak_opt *o);
 void fill_info(const novak_opt *o, const Plan &p, novak_info *out);
 

@@ -156,10 +156,18 @@ int n_state_arrays(const Hyper &h)
     return a;
 }
 
-float *slice(const novak_opt *o, int array, int i)
+void *slice(const novak_opt *o, int array, int i)
 {
-    return reinterpret_cast<float *>(o->d_state) + array * o->region_elems + o->slot_off[i] +
-           o->phase[i];
+    const int64_t mb = moment_bytes(o->h);
+    const int64_t elem = o->slot_off[i] + o->phase[i];
+    if (array < 2) return o->d_state + (array * o->region_elems + elem) * mb;
+    return o->d_state + 2 * o->region_elems * mb + ((array - 2) * o->region_elems + elem) * 4;
+}
+
+size_t state_bytes_for(const Hyper &h, int64_t region_elems)
+{
+    return static_cast<size_t>(region_elems) *
+           (2 * moment_bytes(h) + sizeof(float) * (n_state_arrays(h) - 2));
 }
 
 int pre_mode(const novak_opt *o)
@@ -192,6 +200,7 @@ void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
     out->warnings = o->warnings;
     out->grad_processing = pre_mode(o);
     out->layer_adaptation = o->h.layer_adapt;
+    out->moment_dtype = o->h.mom16 ? NOVAK_MOMENT_BF16 : NOVAK_MOMENT_F32;
     out->beta1_t = p.beta1_t;
     out->beta2_t = p.beta2_t;
 }
@@ -252,6 +261,7 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
     h.nesterov = nesterov_variant;
     h.true_requested = 0;
     h.true_steps = 0;
+    h.mom16 = 0;
     if (nesterov_variant == NOVAK_NESTEROV_TRUE) {
         // N_taylor = 0 until NOVAK_OPT_TRUE_NESTEROV_STEPS says otherwise: every
         // step runs the approximation (Section 7.3's downgrade), with a warning
@@ -305,6 +315,12 @@ int novak_set_option(novak_opt *o, int key, double value)
         h.auto_lr = static_cast<int>(value);
         break;
     case NOVAK_OPT_AUTO_LR_GAMMA: h.auto_gamma = value; break;
+    case NOVAK_OPT_MOMENT_DTYPE:
+        if (o->attached) return fail(o, NOVAK_ESTATE, "moment dtype changes the state layout: set it before attach");
+        if (value != NOVAK_MOMENT_F32 && value != NOVAK_MOMENT_BF16)
+            return fail(o, NOVAK_EINVAL, "unknown moment dtype");
+        h.mom16 = value == NOVAK_MOMENT_BF16 ? 1 : 0;
+        break;
     case NOVAK_OPT_TRUE_NESTEROV_STEPS:
         if (!h.true_requested)
             return fail(o, NOVAK_ESTATE, "true_nesterov_steps: the handle was not created with NOVAK_NESTEROV_TRUE");
@@ -383,6 +399,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_AUTO_LR: *value = o->h.auto_lr; break;
     case NOVAK_OPT_AUTO_LR_GAMMA: *value = o->h.auto_gamma; break;
     case NOVAK_OPT_TRUE_NESTEROV_STEPS: *value = o->h.true_steps; break;
+    case NOVAK_OPT_MOMENT_DTYPE: *value = o->h.mom16 ? NOVAK_MOMENT_BF16 : NOVAK_MOMENT_F32; break;
     case NOVAK_OPT_LAYER_ADAPTATION: *value = o->h.layer_adapt; break;
     case NOVAK_OPT_ADAPTIVE_BETA: *value = o->h.adaptive_beta; break;
     case NOVAK_OPT_BETA1_TAU: *value = o->h.tau1; break;
@@ -407,7 +424,7 @@ size_t novak_state_bytes(const novak_opt *o, const int64_t *numel, int n)
         if (numel[i] <= 0) return 0;
         region += round_up(numel[i] + kSlotAlign - 1, kSlotAlign);
     }
-    return static_cast<size_t>(region) * sizeof(float) * n_state_arrays(o->h);
+    return state_bytes_for(o->h, region);
 }
 
 int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d_params,
@@ -546,6 +563,7 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     out->lookahead_alpha = o->h.la_alpha;
     out->nesterov_variant = o->h.true_requested ? NOVAK_NESTEROV_TRUE : o->h.nesterov;
     out->true_nesterov_steps = o->h.true_steps;
+    out->moment_dtype = o->h.mom16 ? NOVAK_MOMENT_BF16 : NOVAK_MOMENT_F32;
     out->lookahead_k = o->h.la_k;
     out->lookahead_mode = o->h.la_mode; out->rectified = o->h.rectified;
     out->bias1_power = o->h.bias1_power;
@@ -570,8 +588,9 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     if (!o->attached) return fail(o, NOVAK_ESTATE, "import: attach the state first");
     if (o->extrapolated) return fail(o, NOVAK_ESTATE, "import: parameters are extrapolated; restore them first");
     if (in->n_tensors != o->n || in->total_numel != o->total_numel ||
-        in->lookahead_k != o->h.la_k || in->lookahead_mode != o->h.la_mode)
-        return fail(o, NOVAK_ESTATE, "import: tensor list or lookahead layout differs");
+        in->lookahead_k != o->h.la_k || in->lookahead_mode != o->h.la_mode ||
+        (in->moment_dtype == NOVAK_MOMENT_BF16) != (o->h.mom16 != 0))
+        return fail(o, NOVAK_ESTATE, "import: tensor list, lookahead layout or moment dtype differs");
     if (in->t < 0 || in->n_syncs < 0) return fail(o, NOVAK_EINVAL, "import: negative counter");
     Hyper h = o->h;
     h.lr = in->lr; h.beta1 = in->beta1; h.beta2 = in->beta2; h.eps = in->eps;

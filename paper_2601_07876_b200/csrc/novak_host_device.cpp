@@ -311,9 +311,11 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         const uintptr_t g = reinterpret_cast<uintptr_t>(d_grads[i]);
         if (!p || !g) return fail(o, NOVAK_EINVAL, "tensor %d: NULL pointer", i);
         if ((p & 3u) || (g & gmask)) return fail(o, NOVAK_EINVAL, "tensor %d: pointer not aligned to its element size", i);
-        // 128-bit path needs parameter, state and gradient congruent mod 16 B.
+        // 128-bit path needs parameter, state and gradient congruent mod 16 B
+        // (bf16 moments: 8-byte accesses at half the parameter's offset).
         const uintptr_t m = reinterpret_cast<uintptr_t>(slice(o, 0, i));
-        if (((p ^ m) & 15u) || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
+        const bool m_ok = o->h.mom16 ? ((p & 15u) >> 1) == (m & 7u) : ((p ^ m) & 15u) == 0;
+        if (!m_ok || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
             scalar_path = true;
         // the bf16 copy is stored 4 elements (8 bytes) at a time beside 16-byte parameters
         if (!o->copies.empty() &&
@@ -332,8 +334,8 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
         h[i].g = d_grads[i];
         h[i].m = slice(o, 0, i);
         h[i].v = slice(o, 1, i);
-        h[i].slow = la ? slice(o, 2, i) : nullptr;
-        h[i].acc = traj ? slice(o, 3, i) : nullptr;
+        h[i].slow = la ? static_cast<float *>(slice(o, 2, i)) : nullptr;
+        h[i].acc = traj ? static_cast<float *>(slice(o, 3, i)) : nullptr;
         const bool rows = o->h.centralize && o->row_mean && !o->rows.empty() && o->rows[i] > 0;
         h[i].mean = rows ? o->row_mean + o->row_off[i] : nullptr;
         h[i].row_len = rows ? static_cast<uint32_t>(o->numel[i] / o->rows[i]) : 0u;

@@ -116,7 +116,8 @@ cudaError_t launch_trust(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, 
     if (ctx.trust) {
         *what = "layer adaptation kernel launch";
         e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
-                                      o->prep_out, ctx.s, kernel_variant(ctx.plan), ctx.grad_dtype, ctx.pre,
+                                      o->prep_out, ctx.s, kernel_variant(ctx.plan), ctx.grad_dtype,
+                                      ctx.pre | (o->h.mom16 ? novak::PRE_MOM16 : 0),
                                       o->chunk_u2, o->chunk_p2, o->trust, o->pdl, stream);
         if (e != cudaSuccess) return e;
         *launches += 2;
@@ -160,7 +161,8 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     if (o->ctas_per_sm > 0) cfg.grid = std::min(count, o->sms * o->ctas_per_sm);
     cfg.reverse = ctx.reverse;
     cfg.pdl = o->pdl;
-    cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16);
+    cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16) |
+              (o->h.mom16 ? novak::PRE_MOM16 : 0);
     o->last_grid = cfg.grid;
     return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.trust, ctx.s,
                               kernel_variant(ctx.plan), ctx.grad_dtype, ctx.la, cfg, stream);
@@ -489,8 +491,8 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
             r.g = d_grads[i];
             r.m = slice(o, 0, i);
             r.v = slice(o, 1, i);
-            r.slow = la ? slice(o, 2, i) : nullptr;
-            r.acc = traj ? slice(o, 3, i) : nullptr;
+            r.slow = la ? static_cast<float *>(slice(o, 2, i)) : nullptr;
+            r.acc = traj ? static_cast<float *>(slice(o, 3, i)) : nullptr;
             r.mean = nullptr;
             r.p16 = o->copies.empty() ? nullptr : static_cast<__nv_bfloat16 *>(o->copies[i]);
             r.row_len = 0;
@@ -536,7 +538,8 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     cfg.grid = n_chunks;
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
-    cfg.pre = novak::PRE_NONE | (o->copies.empty() ? 0 : novak::PRE_COPY16);
+    cfg.pre = novak::PRE_NONE | (o->copies.empty() ? 0 : novak::PRE_COPY16) |
+              (o->h.mom16 ? novak::PRE_MOM16 : 0);
     e = novak::launch_step(d_chunks, n_chunks, d_recs, nullptr, nullptr, s, kernel_variant(p), grad_dtype,
                            la_action, cfg, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "step kernel launch");
@@ -593,8 +596,7 @@ int novak_nesterov_extrapolate(novak_opt *o, void *const *d_params, void *d_save
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
     if ((rc = prepare_look(o, d_params, stream)) != NOVAK_OK) return rc;
     const cudaError_t e = novak::launch_extrapolate(
-        o->d_chunks, o->n_chunks, o->d_look, reinterpret_cast<const float *>(o->d_state),
-        static_cast<float *>(d_save), static_cast<float>(o->h.beta_n), look_grid(o), stream);
+        o->d_chunks, o->n_chunks, o->d_look, o->d_state, o->h.mom16, static_cast<float *>(d_save), static_cast<float>(o->h.beta_n), look_grid(o), stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "look-ahead kernel launch");
     o->extrapolated = true;
     o->look_save = d_save;

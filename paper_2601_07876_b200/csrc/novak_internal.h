@@ -104,10 +104,11 @@ struct __align__(16) LookRec {
     int64_t state_off;   // elements from the start of a region
 };
 
-// save <- theta, theta <- theta + beta_N m (Eq. 10) over the chunk table.
+// save <- theta, theta <- theta + beta_N m (Eq. 10) over the chunk table; the
+// first-moment region holds fp32, or bf16 when moments_bf16 is set.
 cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
-                               const float *m_region, float *save_region, float beta_n, int grid,
-                               cudaStream_t stream);
+                               const void *m_region, int moments_bf16, float *save_region,
+                               float beta_n, int grid, cudaStream_t stream);
 // theta <- save (Section 5.8: restore the parameters after the closure).
 cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
                            const float *save_region, int grid, cudaStream_t stream);

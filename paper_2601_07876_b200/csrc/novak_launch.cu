@@ -18,6 +18,12 @@ void *step_kernel_pre2(int nesterov, int grad_dtype, int la);
 void *step_kernel_pre0_copy(int nesterov, int grad_dtype, int la);
 void *step_kernel_pre1_copy(int nesterov, int grad_dtype, int la);
 void *step_kernel_pre2_copy(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre0_mom16(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre1_mom16(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre2_mom16(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre0_copy_mom16(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre1_copy_mom16(int nesterov, int grad_dtype, int la);
+void *step_kernel_pre2_copy_mom16(int nesterov, int grad_dtype, int la);
 
 namespace {
 
@@ -36,6 +42,12 @@ StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
     case PRE_NONE | PRE_COPY16: fn = step_kernel_pre0_copy(nesterov, grad_dtype, la); break;
     case PRE_SCALE | PRE_COPY16: fn = step_kernel_pre1_copy(nesterov, grad_dtype, la); break;
     case PRE_CENTER | PRE_COPY16: fn = step_kernel_pre2_copy(nesterov, grad_dtype, la); break;
+    case PRE_NONE | PRE_MOM16: fn = step_kernel_pre0_mom16(nesterov, grad_dtype, la); break;
+    case PRE_SCALE | PRE_MOM16: fn = step_kernel_pre1_mom16(nesterov, grad_dtype, la); break;
+    case PRE_CENTER | PRE_MOM16: fn = step_kernel_pre2_mom16(nesterov, grad_dtype, la); break;
+    case PRE_NONE | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre0_copy_mom16(nesterov, grad_dtype, la); break;
+    case PRE_SCALE | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre1_copy_mom16(nesterov, grad_dtype, la); break;
+    case PRE_CENTER | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre2_copy_mom16(nesterov, grad_dtype, la); break;
     default: break;
     }
     return reinterpret_cast<StepKernelFn>(fn);

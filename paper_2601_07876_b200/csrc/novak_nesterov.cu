@@ -28,21 +28,48 @@ __device__ __forceinline__ void st_stream(float *p, float4 v)
                  :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
+// Four first moments as stored: fp32, or bf16 widened exactly.
+template <bool M16>
+__device__ __forceinline__ float4 ld_moment4(const void *m, int vec)
+{
+    if constexpr (M16) {
+        uint2 t;
+        asm volatile("ld.global.cs.v2.u32 {%0,%1}, [%2];"
+                     : "=r"(t.x), "=r"(t.y) : "l"(static_cast<const uint2 *>(m) + vec));
+        return make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+                           __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+    } else {
+        return ld_stream(static_cast<const float *>(m) + 4 * vec);
+    }
+}
+
+template <bool M16>
+__device__ __forceinline__ float ld_moment1(const void *m, int idx)
+{
+    if constexpr (M16)
+        return __uint_as_float(static_cast<unsigned>(static_cast<const unsigned short *>(m)[idx]) << 16);
+    else
+        return static_cast<const float *>(m)[idx];
+}
+
 // RESTORE = false: save <- theta, theta <- theta + beta_N m.
 // RESTORE = true:  theta <- save (m_region is not read).
-template <bool RESTORE>
+// M16: the first moment is stored as bf16.
+template <bool RESTORE, bool M16>
 __global__ void __launch_bounds__(kLookThreads)
 novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec *__restrict__ recs,
-                  const float *__restrict__ m_region, float *__restrict__ save_region, float beta_n)
+                  const void *__restrict__ m_region, float *__restrict__ save_region, float beta_n)
 {
+    constexpr int kMomBytes = M16 ? 2 : 4;
     for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
         const Chunk ch = chunks[c];
         const LookRec r = recs[ch.tensor];
         float *p = r.p + ch.offset;
         float *sv = save_region + r.state_off + ch.offset;
-        const float *m = RESTORE ? nullptr : m_region + r.state_off + ch.offset;
+        const void *m = RESTORE ? nullptr
+                                : static_cast<const char *>(m_region) + (r.state_off + ch.offset) * kMomBytes;
         uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(sv);
-        if (!RESTORE) bits |= reinterpret_cast<uintptr_t>(m);
+        if (!RESTORE) bits |= reinterpret_cast<uintptr_t>(m) << (M16 ? 1 : 0);
         if ((bits & 15u) == 0) {
             const int nvec = ch.len >> 2;
             // two vectors per thread and pass: all loads first, then the stores
@@ -57,11 +84,11 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
                     if (two) st_stream(p + 4 * j, b);
                 } else {
                     const float4 a = ld_stream(p + 4 * i);
-                    const float4 ma = ld_stream(m + 4 * i);
+                    const float4 ma = ld_moment4<M16>(m, i);
                     float4 b = a, mb = ma;
                     if (two) {
                         b = ld_stream(p + 4 * j);
-                        mb = ld_stream(m + 4 * j);
+                        mb = ld_moment4<M16>(m, j);
                     }
                     st_stream(sv + 4 * i, a);
                     st_stream(p + 4 * i, make_float4(fmaf(beta_n, ma.x, a.x), fmaf(beta_n, ma.y, a.y),
@@ -81,7 +108,7 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
                 } else {
                     const float a = p[idx];
                     sv[idx] = a;
-                    p[idx] = fmaf(beta_n, m[idx], a);
+                    p[idx] = fmaf(beta_n, ld_moment1<M16>(m, idx), a);
                 }
             }
         } else {
@@ -91,7 +118,7 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
                 } else {
                     const float a = p[i];
                     sv[i] = a;
-                    p[i] = fmaf(beta_n, m[i], a);
+                    p[i] = fmaf(beta_n, ld_moment1<M16>(m, i), a);
                 }
             }
         }
@@ -101,13 +128,17 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
 }  // namespace
 
 cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
-                               const float *m_region, float *save_region, float beta_n, int grid,
-                               cudaStream_t stream)
+                               const void *m_region, int moments_bf16, float *save_region,
+                               float beta_n, int grid, cudaStream_t stream)
 {
     if (n_chunks <= 0) return cudaSuccess;
     if (grid < 1 || grid > n_chunks) grid = n_chunks;
-    novak_look_kernel<false><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs, m_region,
-                                                                save_region, beta_n);
+    if (moments_bf16)
+        novak_look_kernel<false, true><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs,
+                                                                          m_region, save_region, beta_n);
+    else
+        novak_look_kernel<false, false><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs,
+                                                                           m_region, save_region, beta_n);
     return cudaGetLastError();
 }
 
@@ -117,8 +148,8 @@ cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d
     if (n_chunks <= 0) return cudaSuccess;
     if (grid < 1 || grid > n_chunks) grid = n_chunks;
     // the kernel only reads the save buffer when restoring
-    novak_look_kernel<true><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs, nullptr,
-                                                               const_cast<float *>(save_region), 0.0f);
+    novak_look_kernel<true, false><<<grid, kLookThreads, 0, stream>>>(
+        d_chunks, n_chunks, d_recs, nullptr, const_cast<float *>(save_region), 0.0f);
     return cudaGetLastError();
 }
 

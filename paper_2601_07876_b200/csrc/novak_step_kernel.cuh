@@ -118,6 +118,22 @@ __device__ __forceinline__ Vec<N> load_grad(const void *base, int idx)
     }
 }
 
+// Moments as stored: fp32, or bf16 (M16) widened exactly on load and rounded to
+// nearest even on store.
+template <int N, bool M16>
+__device__ __forceinline__ Vec<N> load_moment(const void *base, int idx)
+{
+    if constexpr (M16) return load_grad<N, NOVAK_GRAD_BF16>(base, idx);
+    else return load_f32<N>(static_cast<const float *>(base), idx);
+}
+
+template <int N, bool M16>
+__device__ __forceinline__ void store_moment(void *base, int idx, const Vec<N> &x)
+{
+    if constexpr (M16) store_bf16<N>(static_cast<__nv_bfloat16 *>(base), idx, x);
+    else store_f32<N>(static_cast<float *>(base), idx, x);
+}
+
 // ---- phase 2 before the Nesterov approximation: clip factor and centralization
 struct PreArgs {
     __nv_bfloat16 *copy; // bf16 copy of the chunk's parameters (PRE_COPY16), else unused
@@ -224,10 +240,11 @@ __device__ __forceinline__ void update_element(float &p, float g, float &m, floa
 // One full tile: U vectors per thread and per stream, every load issued
 // before the first use so that U x (4..6) 16-byte requests are in flight.
 template <int N, int U, int NEST, int GT, int LA, int PRE>
-__device__ __forceinline__ void run_tile(float *p, const void *g, float *m, float *v,
+__device__ __forceinline__ void run_tile(float *p, const void *g, void *m, void *v,
                                          float *slow, float *acc, int first,
                                          const StepScalars &s, const PreArgs &pre)
 {
+    constexpr bool kMom16 = (PRE & PRE_MOM16) != 0;
     constexpr bool kReadS = (LA & LA_S_READ) != 0;
     constexpr bool kWriteS = (LA & LA_S_WRITE) != 0;
     constexpr bool kReadA = (LA & LA_A_READ) != 0;
@@ -238,8 +255,8 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
         const int idx = first + j * kBlock;
         P[j] = load_f32<N>(p, idx);
         G[j] = load_grad<N, GT>(g, idx);
-        M[j] = load_f32<N>(m, idx);
-        V[j] = load_f32<N>(v, idx);
+        M[j] = load_moment<N, kMom16>(m, idx);
+        V[j] = load_moment<N, kMom16>(v, idx);
         if constexpr (kReadS) S[j] = load_f32<N>(slow, idx);
         if constexpr (kReadA) A[j] = load_f32<N>(acc, idx);
     }
@@ -253,8 +270,8 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
                                      S[j].a[e], A[j].a[e], s, pre.step);
         store_f32<N>(p, idx, P[j]);
         if constexpr ((PRE & PRE_COPY16) != 0) store_bf16<N>(pre.copy, idx, P[j]);
-        store_f32<N>(m, idx, M[j]);
-        store_f32<N>(v, idx, V[j]);
+        store_moment<N, kMom16>(m, idx, M[j]);
+        store_moment<N, kMom16>(v, idx, V[j]);
         if constexpr (kWriteS) store_f32<N>(slow, idx, S[j]);
         if constexpr (kWriteA) store_f32<N>(acc, idx, A[j]);
     }
@@ -263,7 +280,7 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, float *m, floa
 // nvec vectors of N elements: full tiles of U vectors per thread, then the
 // remainder one vector per thread at a time.
 template <int N, int U, int NEST, int GT, int LA, int PRE>
-__device__ __forceinline__ void run_span(float *p, const void *g, float *m, float *v,
+__device__ __forceinline__ void run_span(float *p, const void *g, void *m, void *v,
                                          float *slow, float *acc, int nvec,
                                          const StepScalars &s, const PreArgs &pre)
 {
@@ -297,6 +314,7 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                   const float *__restrict__ trust, const StepScalars s, int reverse)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
     constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
 
@@ -327,14 +345,16 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
         pre.elem0 = static_cast<uint32_t>(ch.offset);
         pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
         float *p = r.p + ch.offset;
-        float *m = r.m + ch.offset;
-        float *v = r.v + ch.offset;
+        void *m = static_cast<char *>(r.m) + ch.offset * kMomBytes;
+        void *v = static_cast<char *>(r.v) + ch.offset * kMomBytes;
         float *slow = kUseS ? r.slow + ch.offset : nullptr;
         float *acc = kUseA ? r.acc + ch.offset : nullptr;
         const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
 
-        uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(m) |
-                         reinterpret_cast<uintptr_t>(v);
+        // four bf16 moments are one 64-bit access: half the parameters' alignment
+        uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
+                         ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
+                          << (kMomBytes == 2 ? 1 : 0));
         if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
         if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
         // the 64-bit stores of the bf16 copy need half the parameters' alignment

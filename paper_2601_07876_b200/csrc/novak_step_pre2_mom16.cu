@@ -1,0 +1,12 @@
+// Step kernel instantiations for the gradient centralized (Eq. 26) and scaled by the clip factor, with
+// the moments stored as bf16.
+#include "novak_step_kernel.cuh"
+
+namespace novak {
+
+void *step_kernel_pre2_mom16(int nesterov, int grad_dtype, int la)
+{
+    return reinterpret_cast<void *>(pick_step_kernel<PRE_CENTER | PRE_MOM16>(nesterov, grad_dtype, la));
+}
+
+}  // namespace novak

@@ -13,8 +13,8 @@ namespace novak {
 struct __align__(16) TensorRec {
     float *p;          // parameters theta, fp32, updated in place
     const void *g;     // gradient, fp32 or bf16, read only
-    float *m;          // first moment   (Eq. 1)
-    float *v;          // second moment  (Eq. 2)
+    void *m;           // first moment   (Eq. 1), fp32, or bf16 under PRE_MOM16
+    void *v;           // second moment  (Eq. 2), same type as m
     float *slow;       // slow weights   (Eq. 28), NULL when lookahead is off
     float *acc;        // running sum of the window's fast iterates (TRAJ_MEAN)
     float2 *mean;      // row means of the raw gradient (Eq. 26) as hi + lo, NULL: not centralized
@@ -66,7 +66,10 @@ enum : int {
     PRE_CENTER = 2,  // g <- factor (g - row mean) for tensors that have rows (Eq. 26)
     PRE_MASK = 3,
     // OR-ed onto the above: the step also stores a bf16 copy of the new parameters
-    PRE_COPY16 = 4
+    PRE_COPY16 = 4,
+    // OR-ed onto the above: m and v are stored as bf16 (read back as stored, advanced
+    // in fp32, the step uses the unrounded values, stored rounded to nearest even)
+    PRE_MOM16 = 8
 };
 
 // Result of the gradient statistics pass, in device memory; the step kernel

@@ -43,14 +43,14 @@ __device__ __forceinline__ double trust_block_sum(double x, double *sh)
 // Squares of N parameters and of the N base directions their gradients give.
 // Each group of N squares is added in fp32, groups in double.
 template <int N, int NEST, int GT, int PRE>
-__device__ __forceinline__ void accumulate(const float *p, const void *g, const float *m,
-                                           const float *v, int idx, const StepScalars &s,
+__device__ __forceinline__ void accumulate(const float *p, const void *g, const void *m,
+                                           const void *v, int idx, const StepScalars &s,
                                            const PreArgs &pre, double &sum_p, double &sum_u)
 {
     const Vec<N> P = load_f32<N>(p, idx);
     Vec<N> G = load_grad<N, GT>(g, idx);
-    const Vec<N> M = load_f32<N>(m, idx);
-    const Vec<N> V = load_f32<N>(v, idx);
+    const Vec<N> M = load_moment<N, (PRE & PRE_MOM16) != 0>(m, idx);
+    const Vec<N> V = load_moment<N, (PRE & PRE_MOM16) != 0>(v, idx);
     preprocess<N, PRE>(G, pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
     float sp = 0.0f, su = 0.0f;
 #pragma unroll
@@ -73,6 +73,7 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 {
     __shared__ double sh[kTrustWarps];
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
 
     grid_dependency_release();
     const int c = blockIdx.x;            // the grid has exactly n_chunks CTAs
@@ -85,17 +86,18 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     pre.copy = nullptr;
     pre.step = 0.0f;
     pre.factor = 1.0f;
-    if constexpr (PRE != PRE_NONE) pre.factor = prep->factor;
-    pre.mean = (PRE == PRE_CENTER) ? r.mean : nullptr;
+    if constexpr ((PRE & PRE_MASK) != PRE_NONE) pre.factor = prep->factor;
+    pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
     pre.row_len = r.row_len;
     pre.elem0 = static_cast<uint32_t>(ch.offset);
 
     const float *p = r.p + ch.offset;
-    const float *m = r.m + ch.offset;
-    const float *v = r.v + ch.offset;
+    const void *m = static_cast<const char *>(r.m) + ch.offset * kMomBytes;
+    const void *v = static_cast<const char *>(r.v) + ch.offset * kMomBytes;
     const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
-    const uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(m) |
-                           reinterpret_cast<uintptr_t>(v);
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
+                           ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
+                            << (kMomBytes == 2 ? 1 : 0));
     const bool aligned = (bits & 15u) == 0 &&
                          (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
     double sum_p = 0.0, sum_u = 0.0;
@@ -157,6 +159,9 @@ TrustFn pick_pre(int pre)
     case PRE_NONE: return novak_trust_stats_kernel<NEST, GT, PRE_NONE>;
     case PRE_SCALE: return novak_trust_stats_kernel<NEST, GT, PRE_SCALE>;
     case PRE_CENTER: return novak_trust_stats_kernel<NEST, GT, PRE_CENTER>;
+    case PRE_NONE | PRE_MOM16: return novak_trust_stats_kernel<NEST, GT, PRE_NONE | PRE_MOM16>;
+    case PRE_SCALE | PRE_MOM16: return novak_trust_stats_kernel<NEST, GT, PRE_SCALE | PRE_MOM16>;
+    case PRE_CENTER | PRE_MOM16: return novak_trust_stats_kernel<NEST, GT, PRE_CENTER | PRE_MOM16>;
     default: return nullptr;
     }
 }
@@ -207,7 +212,7 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
     TrustFn fn = pick_trust(nesterov, grad_dtype, pre);
     if (!fn || n_chunks <= 0 || n_tensors <= 0 || !tensor_first || !chunk_u2 || !chunk_p2 || !trust)
         return cudaErrorInvalidValue;
-    if (pre != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
+    if ((pre & PRE_MASK) != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[1];
     fill_config(&lc, attr, static_cast<unsigned>(n_chunks), (pdl & 2) != 0, stream);

@@ -35,7 +35,8 @@ def oracle_config(hyper: dict) -> O.Config:
         auto_lr=h.pop("auto_lr", False), auto_lr_gamma=h.pop("auto_lr_gamma", None) or 0.1,
         adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
         tau2=h.pop("tau2", None) or 5000.0,
-        true_steps=h.pop("true_nesterov_steps", 0))
+        true_steps=h.pop("true_nesterov_steps", 0),
+        moment_bf16=h.pop("moment_dtype", "f32") == "bf16")
 
 
 def tensor_rows(tensors):
