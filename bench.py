@@ -45,9 +45,9 @@ FALLBACK_HBM_GBS = 6650.0
 # = null) as soon as the kernel sources differ from what was profiled.
 NCU_TRAFFIC = {
     ("resnet50", "last"): {
-        "plain": 660.03e6, "sync": 866.12e6,
-        "sources": {"novak_step_kernel.cuh": "f51d40a775747adf",
-                    "novak_step_types.h": "ce28e09724aa5348", "novak_launch.cu": "23a36fb136f5917e"},
+        "plain": 660.34e6, "sync": 866.01e6,
+        "sources": {"novak_step_kernel.cuh": "56a6c2d56fecf4fd",
+                    "novak_step_types.h": "75b76d99858631ba", "novak_launch.cu": "4a258ea7b5f62c16"},
         "summary": "profiles/novak_step_kernel_resnet50.md",
     },
 }
@@ -97,6 +97,8 @@ def parse_args():
                     help="every step is a true-Nesterov step (Eq. 10-12): look-ahead kernel, "
                          "restore kernel, step; the closure between the two is the caller's "
                          "and not part of the step (+24 B per element)")
+    ap.add_argument("--moment-dtype", default="f32", choices=["f32", "bf16"],
+                    help="storage type of m and v (bf16: 20 B per element instead of 28)")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -115,20 +117,21 @@ def parse_args():
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
                                phase2: bool = False, trust: bool = False,
                                copy16: bool = False, auto: bool = False,
-                               true_nesterov: bool = False) -> int:
+                               true_nesterov: bool = False, moment_bytes: int = 4) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
     arrays on the steps that touch them, plus one more read of g when clipping or
     centralization is on (the norm and the row means are needed before the update)."""
-    b = 12 + grad_bytes + 12 + (grad_bytes if phase2 else 0)
+    mb = moment_bytes
+    b = 4 + 2 * mb + grad_bytes + 4 + 2 * mb + (grad_bytes if phase2 else 0)
     if trust:
-        b += 12 + grad_bytes             # theta, g, m, v read once more for the norms of Eq. 19
+        b += 4 + 2 * mb + grad_bytes     # theta, g, m, v read once more for the norms of Eq. 19
     if copy16:
         b += 2
     if auto:
         b += 4                           # ||theta_t|| of Eq. 21
     if true_nesterov:
-        b += 16 + 8                      # Eq. 10: theta, m read, save, theta written; restore
+        b += 12 + mb + 8                 # Eq. 10: theta, m read, save, theta written; restore
     if k <= 0:
         return b
     sync = t % k == 0
@@ -392,6 +395,9 @@ def main():
     hyper = dict(wl.hyper, lookahead_mode=args.lookahead_mode)
     if args.true_nesterov:
         hyper.update(nesterov="true", true_nesterov_steps=2 ** 31 - 1)
+    if args.moment_dtype == "bf16":
+        hyper.update(moment_dtype="bf16")
+    mbytes = 2 if args.moment_dtype == "bf16" else 4
     k = hyper["lookahead_k"]
     gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
 
@@ -455,13 +461,13 @@ def main():
     value = world * wl.total * args.steps / (ms * 1e-3)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
                                          args.layer_adaptation, args.bf16_copy, args.auto_lr,
-                                         args.true_nesterov)
+                                         args.true_nesterov, mbytes)
               for t in range(t_first, t_first + args.steps)) / args.steps
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
     n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy or args.true_nesterov) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy or args.true_nesterov or mbytes == 2) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -543,6 +549,7 @@ def main():
                 "layer_adaptation": bool(args.layer_adaptation),
                 "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
                 "true_nesterov": bool(args.true_nesterov),
+                "moment_dtype": args.moment_dtype,
                 "auto_lr": bool(args.auto_lr),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "

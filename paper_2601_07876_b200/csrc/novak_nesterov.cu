@@ -1,11 +1,11 @@
 // True Nesterov momentum (Section 4.4, Eq. 10-12): the two passes around the
-// caller's closure.  novak_extrapolate_kernel saves theta_{t-1} and moves the
+// caller's closure.  novak_look_kernel<false, .> saves theta_{t-1} and moves the
 // parameters to theta~ = theta_{t-1} + beta_N m_{t-1} (Eq. 10);
-// novak_restore_kernel puts theta_{t-1} back (Section 5.8's steps 1, 2 and 4).
-// Both walk the step kernel's chunk table, 128 bits per access where the
+// novak_look_kernel<true, .> puts theta_{t-1} back (Section 5.8's steps 1, 2 and
+// 4).  Both walk the step kernel's chunk table, 128 bits per access where the
 // parameters, the first moment and the save buffer share 16-byte alignment.
-// HBM-bound: 16 B per element (theta and m read, save and theta written) and
-// 8 B per element (save read, theta written).
+// HBM-bound: 16 B per element (theta and m read, save and theta written; 14 B
+// with bf16 moments) and 8 B per element (save read, theta written).
 #include "novak.h"
 #include "novak_internal.h"
 
