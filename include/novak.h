@@ -384,7 +384,7 @@ int novak_step_noalloc(novak_opt *opt, void *const *d_params,
  * gradient, before any other processing (Section 7.3).  Three launches per
  * step, no host synchronisation, no floating-point atomics (results are
  * bit-identical from run to run); the scratch (about 16 B per chunk-table entry
- * + 8 B per row + 48 B per 8192 elements of tensors with rows) is allocated by
+ * + 8 B per row + 48 B per 16384 elements of tensors with rows) is allocated by
  * the first such step and again when the rows change.
  * novak_step_noalloc refuses to run in this mode (NOVAK_ESTATE). */
 int novak_set_tensor_rows(novak_opt *opt, const int64_t *rows, int n);
@@ -498,8 +498,8 @@ int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
 
 /* Host-only helper exposing how the statistics pass of the centralization cuts
  * tensors with rows into units: groups of whole rows of up to 2048 elements,
- * about 8192 elements per group (part_len = 0), or, for longer rows, slices
- * [part_off, part_off + part_len) of at most 8192 elements of one row
+ * about 16384 elements per group (part_len = 0), or, for longer rows, slices
+ * [part_off, part_off + part_len) of at most 16384 elements of one row
  * (n_rows = 1), consecutive in the table.  rows[i] as in novak_set_tensor_rows.  Writes up to cap entries and
  * returns the number the table needs (negative on bad arguments). */
 int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,

@@ -11,9 +11,9 @@
 // entries (the table of the step kernel), sum of squares only.  Tensors with
 // rows: a table of row units built on the host, aligned to ROWS, not to the
 // chunk table: a unit is a group of whole rows of up to 2048 elements (a warp
-// streams each row, or a thread for rows shorter than 128 elements), or a
-// slice of at most 8192 elements of a longer row (the whole CTA; usually the
-// whole row).  No shared-memory
+// streams each row; eight lanes for rows shorter than 128 elements, a thread
+// below 32), or a slice of at most 16384 elements of a longer row (the whole
+// CTA; usually the whole row).  No shared-memory
 // staging, no per-vector row arithmetic: a lane only ever adds along one row.
 // All sums are carried in double precision and combined in a fixed order (per
 // lane, warp shuffle tree, warps in index order, CTAs in index order), so the
@@ -28,6 +28,11 @@
 
 namespace novak {
 namespace {
+
+// Resident CTAs per SM the first kernel of the pass is compiled for.
+#ifndef NOVAK_STATS_MIN_CTAS
+#define NOVAK_STATS_MIN_CTAS 6
+#endif
 
 constexpr int kStatsBlock = 256;
 constexpr int kStatsWarps = kStatsBlock / 32;
@@ -351,11 +356,27 @@ __device__ __forceinline__ double row_unit(const RowUnit u, const TensorRec rec,
             sum = warp_sum(sum);
             if (lane == 0) rec.mean[r] = split_mean(sum, L);
         }
+    } else if (L >= 32u) {
+        // short rows: eight lanes each, a warp takes four rows at a time (a thread
+        // per row would read its row as a chain of dependent scalar loads)
+        const uint32_t sub = lane >> 3, l8 = lane & 7u;
+        const uint32_t end = u.row0 + u.n_rows;
+        for (uint32_t r0 = u.row0 + warp * 4u; r0 < end; r0 += kStatsWarps * 4u) {
+            const uint32_t r = r0 + sub;
+            const bool live = r < end;
+            double sum = 0.0;
+            span_sums<GT>(rec.g, live ? r * L : 0u, live ? L : 0u, l8, 8u, sum, sq);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+            if (live && l8 == 0u) rec.mean[r] = split_mean(sum, L);
+        }
     } else {
-        // short rows, a thread each
+        // very short rows, a thread each
         const uint32_t r = u.row0 + threadIdx.x;
         if (threadIdx.x < u.n_rows) {
             double sum = 0.0;
+#pragma unroll 4
             for (uint32_t e = r * L; e < (r + 1u) * L; ++e) {
                 const float x = grad_at<GT>(rec.g, e);
                 sum += double(x);
@@ -371,7 +392,7 @@ __device__ __forceinline__ double row_unit(const RowUnit u, const TensorRec rec,
 // entries each of the tensors without rows; the following n_units CTAs take one
 // row unit each.  Every CTA leaves one sum of squares in part_sq[blockIdx.x].
 template <int GT, bool ROWS>
-__global__ void __launch_bounds__(kStatsBlock)
+__global__ void __launch_bounds__(kStatsBlock, NOVAK_STATS_MIN_CTAS)
 novak_grad_stats_kernel(const Chunk *__restrict__ plain, int n_plain,
                         const RowUnit *__restrict__ units, int n_units,
                         const TensorRec *__restrict__ recs, double *__restrict__ part_sq,

@@ -116,7 +116,8 @@ void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vect
                 }
         } else {
             // a warp per row from 128 elements on (at least one row for each of the
-            // CTA's 8 warps), else a thread per row
+            // CTA's 8 warps), else up to 256 rows per unit (eight lanes per row from 32
+            // elements on, a thread per row below)
             // (rows per unit a multiple of 8, so that no warp idles while others take a
             // second row)
             const uint32_t per = L >= 128u ? std::max(8u, novak::kRowUnitElems / L / 8u * 8u)

@@ -228,10 +228,11 @@ def test_planner_adaptive_beta_agrees_with_oracle():
 
 def test_row_units_cover_every_row_once():
     """The statistics pass's row table: rows of up to 2048 elements whole, in groups of about
-    8192 elements; longer rows in consecutive slices of at most 8192 elements; tensors
+    16384 elements; longer rows in consecutive slices of at most 16384 elements; tensors
     without rows left out."""
     shapes = [(8, 27), (33,), (10, 257), (3, 5000), (4097, 2), (1, 7), (5, 1), (2048,), (6, 2048),
-              (7, 3000), (2, 12300), (1, 100000), (3, 8192), (2, 8193), (300, 127), (300, 128)]
+              (7, 3000), (2, 12300), (1, 100000), (3, 8192), (2, 8193), (3, 16384), (2, 16385),
+              (2, 40000), (300, 127), (300, 128)]
     numel = [int(np.prod(sh)) for sh in shapes]
     rows = [sh[0] if len(sh) > 1 else 0 for sh in shapes]
     units = B.novak_build_row_units(numel, rows)
@@ -241,14 +242,14 @@ def test_row_units_cover_every_row_once():
         L = numel[t] // rows[t]
         assert rows[t] > 0 and n_rows >= 1 and row0 + n_rows <= rows[t]
         if part_len:
-            assert L > 2048 and n_rows == 1 and 0 < part_len <= 8192 and part_off % 8192 == 0
+            assert L > 2048 and n_rows == 1 and 0 < part_len <= 16384 and part_off % 16384 == 0
             assert part_off + part_len <= L
             if part_off:          # slices of a row are consecutive, in order
                 assert prev[:2] == (t, row0) and prev[3] + prev[4] == part_off
             seen[t][row0, part_off:part_off + part_len] += 1
         else:
             assert L <= 2048
-            assert n_rows * L <= max(8192, 8 * L) if L >= 128 else n_rows <= 256
+            assert n_rows * L <= max(16384, 8 * L) if L >= 128 else n_rows <= 256
             seen[t][row0:row0 + n_rows, :] += 1
         prev = (t, row0, n_rows, part_off, part_len)
     for i, sarr in enumerate(seen):

@@ -38,7 +38,7 @@ def test_row_units_cover_every_row_once(data):
         if data.draw(st.booleans()):
             r = data.draw(st.integers(1, 600))
             length = data.draw(st.sampled_from([1, 2, 3, 5, 27, 64, 127, 128, 129, 576, 1024, 2048,
-                                                2049, 4608, 8192, 8193, 20_000]))
+                                                2049, 4608, 8192, 8193, 16384, 16385, 40_000]))
             numel.append(r * length)
             rows.append(r)
         else:
@@ -49,7 +49,7 @@ def test_row_units_cover_every_row_once(data):
     for t, row0, n_rows, part_off, part_len in units:
         L = numel[t] // rows[t]
         if part_len:
-            assert L > 2048 and n_rows == 1 and part_len <= 8192
+            assert L > 2048 and n_rows == 1 and part_len <= 16384
             seen[t][row0, part_off:part_off + part_len] += 1
         else:
             assert L <= 2048
