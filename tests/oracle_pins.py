@@ -904,6 +904,68 @@ def _two_plain_steps(lib, th, g1, g2, kw):
     return o.theta[0]
 
 
+# --------------------------------------------------------------------------
+# Everything at once against 40-digit arithmetic
+# --------------------------------------------------------------------------
+def pin_high_precision_all_variants(lib):
+    """Every Nesterov variant x lookahead mode x rectification on/off, 30 steps on 12
+    elements, against a reference in 40-digit arithmetic (mpmath) that forms the moments
+    as explicit sums over the gradient history and the step scalars from Eq. 5-9 as
+    printed.  Agreement to 1e-11 also bounds the oracle's own rounding (the
+    cancellation in rho_t, the long powers)."""
+    import mpmath as mp
+    mp.mp.dps = 40
+    rng = np.random.default_rng(23)
+    T, n = 30, 12
+    G = rng.normal(0, 1e-2, size=(T, n)); G[4, 1] = 0.0
+    th0 = rng.normal(0, 0.05, size=n)
+    lr, b1, b2, eps, wd, bN, aLA = 2e-3, 0.9, 0.999, 1e-8, 0.03, 0.7, 0.4
+    F = mp.mpf
+    for variant in (O.NESTEROV_NONE, O.NESTEROV_APPROX, O.NESTEROV_CLASSICAL):
+        for k, mode in ((0, O.LOOKAHEAD_LAST), (4, O.LOOKAHEAD_LAST), (4, O.LOOKAHEAD_TRAJ_MEAN),
+                        (1, O.LOOKAHEAD_TRAJ_MEAN)):
+            for rect in (True, False):
+                o = _mk(lib, [th0], lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd,
+                        nesterov_variant=variant, nesterov_beta=bN, lookahead_k=k,
+                        lookahead_alpha=aLA, lookahead_mode=mode, rectified=rect)
+                for t in range(T):
+                    o.step([G[t]])
+                for e in range(n):
+                    g = [F(float(G[t, e])) for t in range(T)]
+                    theta = F(float(th0[e])); slow = theta; acc = F(0)
+                    gt = []                      # the gradients the moments see
+                    for t in range(1, T + 1):
+                        m_prev = sum((1 - F(b1)) * F(b1) ** (t - 1 - i) * gt[i - 1]
+                                     for i in range(1, t)) if t > 1 else F(0)
+                        cur = g[t - 1]
+                        if variant == O.NESTEROV_APPROX:
+                            cur = cur + F(bN) * (cur - m_prev)
+                        gt.append(cur)
+                        m = sum((1 - F(b1)) * F(b1) ** (t - i) * gt[i - 1] for i in range(1, t + 1))
+                        v = sum((1 - F(b2)) * F(b2) ** (t - i) * gt[i - 1] ** 2 for i in range(1, t + 1))
+                        mh = m / (1 - F(b1) ** t); vh = v / (1 - F(b2) ** t)
+                        u = mh / (mp.sqrt(vh) + F(eps))
+                        if variant == O.NESTEROV_CLASSICAL:
+                            u = F(b1) * mh + (1 - F(b1)) * u
+                        rho_inf = 2 / (1 - F(b2)) - 1
+                        rho = rho_inf - 2 * t * F(b2) ** t / (1 - F(b2) ** t)
+                        r = F(1)
+                        if rect and rho >= 5:
+                            r = mp.sqrt((rho - 4) * (rho - 2) * rho_inf / ((rho_inf - 4) * (rho_inf - 2) * rho))
+                        fast = theta * (1 - F(lr) * F(wd)) - F(lr) * r * u
+                        theta = fast
+                        if k > 0:
+                            acc += fast
+                            if t % k == 0:
+                                target = acc / k if mode == O.LOOKAHEAD_TRAJ_MEAN else fast
+                                theta = slow + F(aLA) * (target - slow)
+                                slow = theta
+                                acc = F(0)
+                    ref = float(theta)
+                    assert abs(o.theta[0][e] - ref) <= 1e-11 * abs(ref) + 1e-15, \
+                        (variant, k, mode, rect, e, o.theta[0][e], ref)
+
+
 ALL_PINS = [
     pin_constant_grad_none,
     pin_constant_grad_approx,
@@ -929,4 +991,5 @@ ALL_PINS = [
     pin_auto_lr,
     pin_true_nesterov,
     pin_bf16_moment_storage,
+    pin_high_precision_all_variants,
 ]
