@@ -203,3 +203,32 @@ def test_checkpoint_round_trip_and_dtype_mismatch():
     c = B.NovakOptimizer(params, **dict(BASE, moment_dtype="f32"))
     with pytest.raises(B.NovakError):
         c.load_state_dict(sd)
+
+
+@pytest.mark.parametrize("index", [1, 3])
+def test_fullsize_launch_configuration(index):
+    """The ResNet-50-shaped (fp32 gradients) and ViT-B/16-shaped (bf16 gradients) sets at
+    full size, 12 steps; the oracle follows the usual sample of elements."""
+    from harness import SampledPair
+    from paper_2601_07876_b200 import workloads as W
+    wl = W.get_workload(index)
+    pair = SampledPair(wl, DEV, dict(moment_dtype="bf16"))
+    o = pair.oracle
+    o.track_rounding_margin = True
+    for _ in range(12):
+        pair.step(threads=8)
+    torch.cuda.synchronize()
+    assert pair.opt.info()["t"] == o.t and pair.sync_steps == o.sync_steps
+    near = o.rounding_margin[0] < MARGIN
+    ok = ~near
+    frac = float(near.mean())
+    assert frac <= (0.12 if wl.grad_dtype == torch.float32 else 0.5), frac
+    gm, gv = to_f64(pair._gather_state("m")), to_f64(pair._gather_state("v"))
+    assert np.array_equal(gm[ok], o.m[0][ok]) and np.array_equal(gv[ok], o.v[0][ok])
+    assert_close(to_f64(pair.flat_p[pair.idx])[ok], o.theta[0][ok], f"{wl.name} theta")
+    assert_close(to_f64(pair._gather_state("slow"))[ok], o.slow[0][ok], f"{wl.name} slow")
+    print(f"\nBF16 MOMENTS {wl.name}: {ok.sum()} of {ok.size} sampled elements compared bit for bit, "
+          f"{frac:.4f} set aside")
+    assert pair.opt.info()["launches"] == 12
+    del pair
+    torch.cuda.empty_cache()

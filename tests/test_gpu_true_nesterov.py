@@ -148,3 +148,30 @@ def test_checkpoint_carries_the_true_variant():
     assert b.handle.get_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS) == 6
     assert b.wants_extrapolation() and b.info()["t"] == 1
     assert not b.info()["warnings"] & B.NOVAK_WARN_TRUE_DOWNGRADED
+
+
+def test_fullsize_resnet50_launch_configuration():
+    """The ResNet-50-shaped set at full size: five true steps, then the fallback; the
+    oracle follows the usual sample of elements (gradients are the workload's seeded
+    random ones: the kernels do not care where a gradient was evaluated)."""
+    from harness import SampledPair
+    from paper_2601_07876_b200 import workloads as W
+    wl = W.get_workload(1)
+    pair = SampledPair(wl, DEV, dict(nesterov="true", nesterov_beta=0.8, true_nesterov_steps=5))
+    for t in range(1, 9):
+        want = pair.opt.wants_extrapolation()
+        assert want == pair.oracle.wants_extrapolation() == (t <= 5)
+        if want:
+            before = pair.flat_p.clone()
+            pair.opt.extrapolate()
+            assert_close(pair.flat_p[pair.idx], pair.oracle.extrapolated()[0], f"t={t} theta~")
+            if t > 1:
+                assert not torch.equal(pair.flat_p, before)
+            pair.opt.restore()
+            assert torch.equal(pair.flat_p, before)
+            del before
+        pair.step(threads=8)
+    pair.check()
+    assert pair.opt.info()["launches"] == 8 + 2 * 5
+    del pair
+    torch.cuda.empty_cache()
