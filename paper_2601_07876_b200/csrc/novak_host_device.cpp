@@ -234,20 +234,23 @@ int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream)
 {
     const size_t n = static_cast<size_t>(o->n);
     cudaError_t e;
+    // each of the three is created once; a call that failed half-way is completed here
     if (!o->d_look) {
         if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_look), n * sizeof(novak::LookRec))) != cudaSuccess) {
             o->d_look = nullptr;
             return fail(o, NOVAK_ENOMEM, "cudaMalloc(look-ahead records): %s", cudaGetErrorString(e));
         }
-        if ((e = cudaMallocHost(reinterpret_cast<void **>(&o->h_look), n * sizeof(novak::LookRec))) != cudaSuccess) {
-            o->h_look = nullptr;
-            return fail(o, NOVAK_ENOMEM, "cudaMallocHost(look-ahead records): %s", cudaGetErrorString(e));
-        }
-        if ((e = cudaEventCreateWithFlags(&o->look_ev, cudaEventDisableTiming)) != cudaSuccess) {
-            o->look_ev = nullptr;
-            return fail_cuda(o, e, "cudaEventCreate(look-ahead records)");
-        }
         o->look_p.clear();
+    }
+    if (!o->h_look &&
+        (e = cudaMallocHost(reinterpret_cast<void **>(&o->h_look), n * sizeof(novak::LookRec))) != cudaSuccess) {
+        o->h_look = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMallocHost(look-ahead records): %s", cudaGetErrorString(e));
+    }
+    if (!o->look_ev &&
+        (e = cudaEventCreateWithFlags(&o->look_ev, cudaEventDisableTiming)) != cudaSuccess) {
+        o->look_ev = nullptr;
+        return fail_cuda(o, e, "cudaEventCreate(look-ahead records)");
     }
     if (o->look_p.size() == n && std::memcmp(o->look_p.data(), d_params, n * sizeof(void *)) == 0)
         return NOVAK_OK;

@@ -446,6 +446,10 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
 {
     if (!o) return NOVAK_EINVAL;
     if (!o->attached) return fail(o, NOVAK_ESTATE, "step_noalloc: no state attached");
+    if (o->extrapolated)
+        return fail(o, NOVAK_ESTATE, "step_noalloc: parameters are extrapolated (Eq. 10); call novak_nesterov_restore first");
+    if (o->half_open)
+        return fail(o, NOVAK_ESTATE, "step_noalloc: a step begun with novak_step_begin is still open");
     if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step_noalloc: NULL argument");
     if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16)
         return fail(o, NOVAK_EINVAL, "step_noalloc: unknown grad_dtype %d", grad_dtype);

@@ -114,6 +114,9 @@ def test_state_machine_refusals():
         opt.extrapolate()                                          # twice
     with pytest.raises(B.NovakError):
         opt.step(g)                                                # would step on theta~
+    gl = opt.prepare(g)
+    with pytest.raises(B.NovakError):
+        opt.handle.step_noalloc(opt._params_arr, gl.arr, opt._numel_arr, opt.n, gl.dtype, 0)
     with pytest.raises(B.NovakError):
         opt.handle.set_option(B.NOVAK_OPT_TRUE_NESTEROV_STEPS, 7)
     other = torch.empty(opt.handle.nesterov_save_bytes(), dtype=torch.uint8, device=DEV)
