@@ -295,9 +295,19 @@ def cpu_baseline(wl, hyper, seconds):
         o.step([g], threads=cores)
         steps += 1
     dt = time.perf_counter() - t0
+    # the same on one thread, a quarter of the time
+    steps1, t1 = 0, time.perf_counter()
+    while time.perf_counter() - t1 < seconds / 4 and steps1 < 5000:
+        if o.wants_extrapolation():
+            o.extrapolated()
+        o.step([g], threads=1)
+        steps1 += 1
+    dt1 = time.perf_counter() - t1
     return {"value": n * steps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "single_thread_value": n * steps1 / dt1,
             "sample": f"{n} elements of {wl.name} as one tensor x {steps} steps "
-                      f"({dt:.1f} s), threads over disjoint element ranges"}
+                      f"({dt:.1f} s), threads over disjoint element ranges; one thread: "
+                      f"{steps1} steps ({dt1:.1f} s)"}
 
 
 def run_zero1(args, rank, world, local):
