@@ -406,6 +406,7 @@ class NovakOptimizer:
             if p.dtype != torch.float32 or not p.is_cuda or not p.is_contiguous():
                 raise ValueError("parameters must be contiguous float32 CUDA tensors")
         self.device = self.params[0].device
+        self._raw_stream = None
         variant = _NESTEROV[nesterov] if isinstance(nesterov, str) else int(nesterov)
         self.handle = Handle(lr, betas[0], betas[1], eps, weight_decay, variant, lookahead_k,
                              lookahead_alpha, lib=lib)
@@ -518,6 +519,21 @@ class NovakOptimizer:
         return self.handle.get_grad_stats(self._stream())
 
     def _stream(self) -> int:
+        """Handle of torch's current stream on the parameters' device (the raw lookup
+        where torch has it: the Stream object costs 2 us per step)."""
+        raw = self._raw_stream
+        if raw is None:
+            import torch
+            raw = getattr(torch._C, "_cuda_getCurrentRawStream", False)
+            if raw:
+                index = self.device.index
+                if index is None:
+                    index = torch.cuda.current_device()
+                self._raw_stream = raw = (raw, index)
+            else:
+                self._raw_stream = raw = False
+        if raw:
+            return raw[0](raw[1])
         import torch
         return torch.cuda.current_stream(self.device).cuda_stream
 
@@ -530,8 +546,11 @@ class NovakOptimizer:
     def step(self, grads):
         """One step.  ``grads``: list of tensors, or a ``GradList`` from prepare()."""
         gl = grads if isinstance(grads, GradList) else self.prepare(grads)
-        self.handle.step(self._params_arr, gl.arr, self._numel_arr, self.n, gl.dtype,
-                         self._stream())
+        h = self.handle
+        st = h.lib.novak_step(h.h, self._params_arr, gl.arr, self._numel_arr, self.n, gl.dtype,
+                              self._stream())
+        if st != NOVAK_OK:
+            _check(h.lib, h.h, st, "novak_step")
         self._last_grads = gl
 
     def step_begin(self, grads):
