@@ -232,3 +232,44 @@ def test_fullsize_launch_configuration(index):
     assert pair.opt.info()["launches"] == 12
     del pair
     torch.cuda.empty_cache()
+
+
+def test_other_entry_points_and_chunk_sizes_give_the_same_bits():
+    """novak_step_noalloc, novak_step_host and entries of 1024 / 4096 elements run the same
+    kernels on bf16 moments: bit-identical parameters and state to novak_step."""
+    numels = [70001, 33, 2048, 1, 9000]
+    offs = [0, 1, 0, 3, 2]
+    hyper = dict(BASE, lookahead_k=2)
+
+    def fresh(**kw):
+        ps = _fresh(numels, offs, seed=4)
+        return ps, B.NovakOptimizer(ps, **hyper, **kw)
+
+    (pa, a), (pb, b), (pc, c), (pd, d), (pe, e) = (fresh(), fresh(), fresh(),
+                                                   fresh(chunk_elems=1024), fresh(chunk_elems=4096))
+    gen = _gen(8)
+    total = sum(numels)
+    h_g = torch.empty(total, dtype=torch.float32).pin_memory()
+    h_p = torch.empty(total, dtype=torch.float32).pin_memory()
+    d_g = torch.empty(total, dtype=torch.float32, device=DEV)
+    starts = np.concatenate([[0], np.cumsum(numels)])[:-1]
+    hg = B.ptr_array([h_g.data_ptr() + 4 * int(o) for o in starts])
+    hp = B.ptr_array([h_p.data_ptr() + 4 * int(o) for o in starts])
+    dg = B.ptr_array([d_g.data_ptr() + 4 * int(o) for o in starts])
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(5):
+        grads = _grads(numels, gen, offsets=offs)
+        a.step(grads)
+        gl = b.prepare(grads)
+        b.handle.step_noalloc(b._params_arr, gl.arr, b._numel_arr, b.n, gl.dtype, stream)
+        h_g.copy_(torch.cat([g.reshape(-1) for g in grads]).cpu())
+        c.handle.step_host(hp, hg, c._params_arr, dg, c._numel_arr, c.n, B.NOVAK_GRAD_F32, stream)
+        d.step(grads)
+        e.step(grads)
+    torch.cuda.synchronize()
+    for other, ps in ((b, pb), (c, pc), (d, pd), (e, pe)):
+        for i in range(len(numels)):
+            assert torch.equal(ps[i], pa[i])
+            for k in ("m", "v", "slow"):
+                assert torch.equal(other.state(i)[k], a.state(i)[k])
+    assert torch.equal(h_p.to(DEV), torch.cat([p.reshape(-1) for p in pc]))

@@ -102,6 +102,30 @@ def test_first_look_ahead_is_the_identity_and_m_is_read_not_written():
         assert torch.equal(p, b)
 
 
+@pytest.mark.parametrize("chunk", [1024, 4096, 8192])
+def test_look_ahead_with_other_entry_sizes(chunk):
+    """Entries of 1024 ... 8192 elements: the look-ahead kernels loop over more than one
+    pair of vectors per thread; same bits as with the default entries."""
+    numels = [70001, 33, 9000, 5]
+    offs = [0, 2, 0, 1]
+    _, pa = _fresh(numels, offs)
+    _, pb = _fresh(numels, offs)
+    hyper = dict(BASE, true_nesterov_steps=3)
+    a = B.NovakOptimizer(pa, **hyper)
+    b = B.NovakOptimizer(pb, **hyper, chunk_elems=chunk)
+    for t in range(3):
+        g = _device_grads([np.full(n, 0.01 * (t + 1)) for n in numels], offs)
+        for o in (a, b):
+            o.extrapolate()
+        for x, y in zip(pa, pb):
+            assert torch.equal(x, y)
+        for o in (a, b):
+            o.restore()
+            o.step(g)
+    for x, y in zip(pa, pb):
+        assert torch.equal(x, y)
+
+
 def test_state_machine_refusals():
     _, params = _fresh([4096, 100])
     opt = B.NovakOptimizer(params, **dict(BASE, true_nesterov_steps=2))
