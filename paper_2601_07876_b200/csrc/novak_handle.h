@@ -6,6 +6,7 @@
 
 #include "novak.h"
 #include "novak_internal.h"
+#include "novak_plan.h"
 
 #include <cstdint>
 #include <string>
@@ -27,29 +28,6 @@ constexpr int64_t kDefaultChunkElems = 2048;
 constexpr int kDefaultCtasPerSm = 0;
 constexpr int64_t kDefaultHostSegmentElems = 4 << 20;  // elements per pipelined segment
 constexpr int kMaxHostSegments = 32;
-
-struct Hyper {
-    double lr, beta1, beta2, eps, wd, beta_n, la_alpha;
-    double clip;            // c_clip of the global-norm clipping, 0: off
-    int nesterov, la_k, la_mode, rectified, bias1_power;
-    int centralize;         // Eq. 26 on tensors that were given rows
-    int layer_adapt;        // Eq. 19 / 25: one trust ratio per tensor
-    int adaptive_beta;      // Eq. 3-4
-    double tau1, tau2;      // warm-up time scales of beta1, beta2
-    double sparse_tau;      // tau of Eq. 27, 0: no mask
-    int auto_lr;            // Eq. 20-22
-    double auto_gamma;      // gamma of Eq. 20-21
-    int true_requested;     // the caller asked for the true variant (Eq. 10-12)
-    int true_steps;         // N_taylor: steps 1..N_taylor take Eq. 11's gradient as given
-    int mom16;              // m and v stored as bf16 (fixed at attach: it sets the layout)
-};
-
-struct Plan {
-    double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay;
-    double beta1_t, beta2_t;   // coefficients of Eq. 1-2 at this step (Eq. 3-4 when warmed up)
-    int rect_branch, is_sync;
-    int nesterov;              // variant of this step: TRUE while t <= N_taylor, else the configured one
-};
 
 struct Handle {
     Hyper h{};
@@ -161,10 +139,7 @@ struct novak_opt : novak_host::Handle {};
 
 namespace novak_host {
 
-// Planner (novak_host.cpp).  make_plan: Eq. 5-9 and 18 for the 1-based step t;
-// lookahead_action: the LA_* bits of step t (Eq. 28-31).
-Plan make_plan(const Hyper &h, int64_t t);
-int lookahead_action(const Hyper &h, int64_t t);
+// Planner helpers (novak_host.cpp); the scalar plan itself is in novak_plan.h.
 int64_t round_up(int64_t x, int64_t a);
 void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chunk_elems,
                   std::vector<Chunk> &out);

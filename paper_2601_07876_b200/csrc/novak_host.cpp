@@ -15,64 +15,6 @@ using namespace novak_host;
 
 namespace novak_host {
 
-// Eq. 5-9 and 18 for the 1-based step index t.  1 - beta^t is evaluated as
-// -expm1(t log beta) for every t (Section 5.8 gives the log form for large t).
-Plan make_plan(const Hyper &h, int64_t t)
-{
-    Plan p;
-    const double td = static_cast<double>(t);
-    const double l1 = h.beta1 > 0.0 ? td * std::log(h.beta1) : -INFINITY;
-    const double l2 = h.beta2 > 0.0 ? td * std::log(h.beta2) : -INFINITY;
-    p.bc1 = -std::expm1(l1);
-    p.bc2 = -std::expm1(l2);
-    const double b2t = std::exp(l2);
-    p.rho_inf = 2.0 / (1.0 - h.beta2) - 1.0;
-    p.rho_t = p.rho_inf - 2.0 * td * b2t / p.bc2;
-    p.rect_branch = (h.rectified && p.rho_t >= 5.0) ? 1 : 0;
-    p.r_t = 1.0;
-    if (p.rect_branch) {
-        const double a = (p.rho_t - 4.0) / (p.rho_inf - 4.0);
-        const double b = (p.rho_t - 2.0) / (p.rho_inf - 2.0);
-        p.r_t = std::sqrt(a * b * (p.rho_inf / p.rho_t));
-    }
-    p.step_size = h.lr * p.r_t;
-    if (h.bias1_power == 2) p.step_size /= p.bc1;
-    p.decay = 1.0 - h.lr * h.wd;
-    p.is_sync = (h.la_k > 0 && t % h.la_k == 0) ? 1 : 0;
-    // Phase 3, Eq. 3-4: only the moment updates see the warmed-up coefficients.
-    p.beta1_t = h.beta1;
-    p.beta2_t = h.beta2;
-    if (h.adaptive_beta) {
-        p.beta1_t = h.beta1 * -std::expm1(-td / h.tau1);
-        p.beta2_t = h.beta2 * -std::expm1(-td / h.tau2);
-    }
-    // Section 5.2: the true variant (the gradient is already Eq. 11's) for the
-    // first N_taylor steps, the approximation of Eq. 13 afterwards.
-    p.nesterov = (h.true_requested && t <= h.true_steps) ? NOVAK_NESTEROV_TRUE : h.nesterov;
-    return p;
-}
-
-int lookahead_action(const Hyper &h, int64_t t)
-{
-    using namespace novak;
-    if (h.la_k <= 0) return LA_NONE;
-    const bool first_step = (t == 1);
-    const bool sync = (t % h.la_k == 0);
-    const bool first_of_window = ((t - 1) % h.la_k == 0);
-    const bool traj = (h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN && h.la_k > 1);
-    int la = 0;
-    if (first_step) la |= LA_S_INIT | LA_S_WRITE;
-    if (sync) {
-        la |= LA_SYNC | LA_S_WRITE;
-        if (!first_step) la |= LA_S_READ;
-    }
-    if (traj) {
-        if (!first_of_window) la |= LA_A_READ;
-        if (sync) la |= LA_TRAJ; else la |= LA_A_WRITE;
-    }
-    return la;
-}
-
 int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
 // Splits tensors into chunk-table entries; see novak_build_chunks in novak.h.

@@ -14,27 +14,6 @@ using namespace novak_host;
 
 namespace {
 
-StepScalars make_scalars(const Hyper &h, const Plan &p)
-{
-    StepScalars s;
-    s.beta1 = static_cast<float>(p.beta1_t);
-    s.omb1 = static_cast<float>(1.0 - p.beta1_t);
-    s.beta2 = static_cast<float>(p.beta2_t);
-    s.omb2 = static_cast<float>(1.0 - p.beta2_t);
-    s.blend_b1 = static_cast<float>(h.beta1);
-    s.blend_omb1 = static_cast<float>(1.0 - h.beta1);
-    s.beta_n = static_cast<float>(h.beta_n);
-    s.inv_bc1 = static_cast<float>(1.0 / p.bc1);
-    s.inv_bc2 = static_cast<float>(1.0 / p.bc2);
-    s.eps = static_cast<float>(h.eps);
-    s.decay = static_cast<float>(p.decay);
-    s.step = static_cast<float>(p.step_size);
-    s.la_alpha = static_cast<float>(h.la_alpha);
-    s.k = static_cast<float>(h.la_k > 0 ? h.la_k : 1);
-    s.sparse_tau = h.sparse_tau > 0.0 ? static_cast<float>(h.sparse_tau) : -1.0f;
-    return s;
-}
-
 // Everything one step needs, fixed before anything is enqueued.
 struct StepCtx {
     int64_t t;
