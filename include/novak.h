@@ -142,6 +142,26 @@ enum {
                                      NOVAK_ESTATE for any other variant             */
     NOVAK_OPT_MOMENT_DTYPE = 22,  /* NOVAK_MOMENT_*: storage type of m and v; only
                                      before attach (default NOVAK_MOMENT_F32)          */
+    NOVAK_OPT_GRAPH_CAPTURABLE = 23, /* 1: novak_step may be captured into a CUDA graph
+                                     (stream capture) and replayed: the step counter,
+                                     the scalars of Eq. 3-9 / 18 and the lookahead
+                                     action then live in device memory, advanced by a
+                                     one-thread kernel in front of the step kernel
+                                     (one launch more per step), so that every replay
+                                     is the NEXT step.  Take one step outside the
+                                     capture first (it allocates and uploads the work
+                                     table), keep the captured pointer lists alive,
+                                     and change options or import checkpoints outside
+                                     a capture only: LR and WEIGHT_DECAY reach the
+                                     device at the next novak_step CALL, the other
+                                     hyperparameters are part of a captured launch.
+                                     novak_get_info and novak_export_meta read the
+                                     counters back and SYNCHRONISE the device in this
+                                     mode.  Not covered (NOVAK_ESTATE): layer
+                                     adaptation, bf16 parameter copies, bf16 moments,
+                                     true Nesterov steps, novak_step_begin / _host /
+                                     _noalloc; NOVAK_OPT_SERPENTINE is ignored.  Only
+                                     before the first step.  0 (default)              */
     NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base
                                      directions with |u| <= tau are set to zero before
                                      the classical blend; 0 (default): no mask.  The

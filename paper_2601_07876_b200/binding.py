@@ -29,7 +29,8 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_WEIGHT_DECAY, NOVAK_OPT_DEPENDENT_LAUNCH, NOVAK_OPT_HOST_SEGMENT_ELEMS,
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
  NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
- NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS, NOVAK_OPT_MOMENT_DTYPE) = range(1, 23)
+ NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS, NOVAK_OPT_MOMENT_DTYPE,
+ NOVAK_OPT_GRAPH_CAPTURABLE) = range(1, 24)
 NOVAK_MOMENT_F32, NOVAK_MOMENT_BF16 = 0, 1
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
 
@@ -396,6 +397,7 @@ class NovakOptimizer:
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
                  auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0, moment_dtype="f32",
+                 graph_capturable=False,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -421,6 +423,8 @@ class NovakOptimizer:
         h.set_option(NOVAK_OPT_MOMENT_DTYPE, NOVAK_MOMENT_BF16 if self.moment_bf16 else NOVAK_MOMENT_F32)
         h.set_option(NOVAK_OPT_RECTIFIED, 1 if rectified else 0)
         h.set_option(NOVAK_OPT_BIAS1_POWER, bias1_power)
+        if graph_capturable:
+            h.set_option(NOVAK_OPT_GRAPH_CAPTURABLE, 1)
         if chunk_elems is not None:
             h.set_option(NOVAK_OPT_CHUNK_ELEMS, chunk_elems)
         if ctas_per_sm is not None:

@@ -95,6 +95,10 @@ struct Handle {
     bool half_open = false;
     int half_launches = 0;
     alignas(8) unsigned char half_ctx[256] = {};   // the StepCtx of the open step
+    // graph-capturable step: the counters and the plan in device memory
+    int dyn = 0;
+    novak::DevPlan *d_plan = nullptr;
+    bool dyn_upload_counters = true, dyn_upload_rates = true;
     bool extrapolated = false;          // between novak_nesterov_extrapolate and _restore
     novak::LookRec *d_look = nullptr;   // device records of the two look-ahead helpers
     novak::LookRec *h_look = nullptr;   // pinned staging of those records
@@ -180,5 +184,10 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
 // Device records of the look-ahead helpers for this parameter list (uploaded
 // only when the list differs from the one the device holds).
 int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream);
+// Device-resident plan of the graph-capturable step: allocated on first use;
+// counters and rates are uploaded when the host has changed them.
+int prepare_dyn(novak_opt *o, cudaStream_t stream);
+// The device-resident plan copied to the host (synchronises the device).
+int read_dyn(const novak_opt *o, novak::DevPlan *out);
 
 }  // namespace novak_host

@@ -246,8 +246,8 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "rectified must be 0 or 1");
         h.rectified = static_cast<int>(value);
         break;
-    case NOVAK_OPT_LR: h.lr = value; break;
-    case NOVAK_OPT_WEIGHT_DECAY: h.wd = value; break;
+    case NOVAK_OPT_LR: h.lr = value; o->dyn_upload_rates = true; break;
+    case NOVAK_OPT_WEIGHT_DECAY: h.wd = value; o->dyn_upload_rates = true; break;
     case NOVAK_OPT_BIAS1_POWER:
         if (value != 1.0 && value != 2.0) return fail(o, NOVAK_EINVAL, "bias1_power must be 1 or 2");
         h.bias1_power = static_cast<int>(value);
@@ -291,6 +291,11 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (h.centralize != static_cast<int>(value)) invalidate_tables(o);
         h.centralize = static_cast<int>(value);
         break;
+    case NOVAK_OPT_GRAPH_CAPTURABLE:
+        if (o->t > 0) return fail(o, NOVAK_ESTATE, "graph_capturable is fixed once a step was taken");
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "graph_capturable must be 0 or 1");
+        o->dyn = static_cast<int>(value);
+        return NOVAK_OK;
     case NOVAK_OPT_CHUNK_ELEMS: {
         if (o->d_chunks || !o->na_chunks.empty())
             return fail(o, NOVAK_ESTATE, "chunk size is fixed once a step was taken");
@@ -349,6 +354,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_BETA2_TAU: *value = o->h.tau2; break;
     case NOVAK_OPT_CLIP_THRESHOLD: *value = o->h.clip; break;
     case NOVAK_OPT_CENTRALIZE: *value = o->h.centralize; break;
+    case NOVAK_OPT_GRAPH_CAPTURABLE: *value = o->dyn; break;
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
@@ -473,6 +479,19 @@ int novak_get_info(const novak_opt *o, novak_info *out)
 {
     if (!o || !out) return NOVAK_EINVAL;
     fill_info(o, o->last_plan, out);
+    if (o->dyn && o->d_plan) {
+        // replays of a captured step advance only the device's counters
+        novak::DevPlan dp;
+        if (read_dyn(o, &dp) != NOVAK_OK) return NOVAK_ECUDA;
+        out->t = dp.t; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
+        if (dp.t > 0) {
+            out->bc1 = dp.bc1; out->bc2 = dp.bc2; out->rho_inf = dp.rho_inf; out->rho_t = dp.rho_t;
+            out->r_t = dp.r_t; out->step_size = dp.step_size; out->decay = dp.decay;
+            out->rect_branch = dp.rect_branch; out->is_sync = dp.is_sync;
+            out->nesterov_variant = dp.nesterov;
+            out->beta1_t = dp.beta1_t; out->beta2_t = dp.beta2_t;
+        }
+    }
     return NOVAK_OK;
 }
 
@@ -500,6 +519,11 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     std::memset(out, 0, sizeof *out);
     out->magic = kMetaMagic;
     out->t = o->t; out->n_syncs = o->n_syncs; out->last_sync_step = o->last_sync;
+    if (o->dyn && o->d_plan) {
+        novak::DevPlan dp;
+        if (read_dyn(o, &dp) != NOVAK_OK) return NOVAK_ECUDA;
+        out->t = dp.t; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
+    }
     out->total_numel = o->total_numel;
     out->lr = o->h.lr; out->beta1 = o->h.beta1; out->beta2 = o->h.beta2; out->eps = o->h.eps;
     out->weight_decay = o->h.wd; out->nesterov_beta = o->h.beta_n;
@@ -562,6 +586,7 @@ int novak_import_meta(novak_opt *o, const novak_meta *in)
     if (!check_hyper(h, &why)) return fail(o, NOVAK_EINVAL, "import: %s", why);
     o->h = h;
     o->t = in->t; o->n_syncs = in->n_syncs; o->last_sync = in->last_sync_step;
+    o->dyn_upload_counters = o->dyn_upload_rates = true;
     o->warnings |= in->warnings;
     if (h.true_requested) {
         if (h.true_steps > 0) o->warnings &= ~static_cast<uint32_t>(NOVAK_WARN_TRUE_DOWNGRADED);

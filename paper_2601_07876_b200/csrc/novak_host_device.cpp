@@ -24,6 +24,9 @@ void release_device(novak_opt *o)
         o->h_recs[i] = nullptr;
         o->ring_ev[i] = nullptr;
     }
+    if (o->d_plan) cudaFree(o->d_plan);
+    o->d_plan = nullptr;
+    o->dyn_upload_counters = o->dyn_upload_rates = true;
     if (o->d_look) cudaFree(o->d_look);
     if (o->h_look) cudaFreeHost(o->h_look);
     if (o->look_ev) cudaEventDestroy(o->look_ev);
@@ -272,6 +275,44 @@ int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream)
         (e = cudaEventRecord(o->look_ev, stream)) != cudaSuccess)
         return fail_cuda(o, e, "look-ahead record upload");
     o->look_p.assign(d_params, d_params + n);
+    return NOVAK_OK;
+}
+
+int prepare_dyn(novak_opt *o, cudaStream_t stream)
+{
+    cudaError_t e;
+    if (!o->d_plan) {
+        if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_plan), sizeof(novak::DevPlan))) != cudaSuccess) {
+            o->d_plan = nullptr;
+            return fail(o, NOVAK_ENOMEM, "cudaMalloc(device plan): %s", cudaGetErrorString(e));
+        }
+        if ((e = cudaMemsetAsync(o->d_plan, 0, sizeof(novak::DevPlan), stream)) != cudaSuccess)
+            return fail_cuda(o, e, "cudaMemsetAsync(device plan)");
+        o->dyn_upload_counters = o->dyn_upload_rates = true;
+    }
+    // Copies from the stack: staged by the driver before the call returns (not
+    // possible while the stream is being captured: change options and import
+    // checkpoints outside a capture).
+    if (o->dyn_upload_counters) {
+        const long long c[3] = {o->t, o->n_syncs, o->last_sync};
+        if ((e = cudaMemcpyAsync(&o->d_plan->t, c, sizeof c, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "upload of the step counters");
+        o->dyn_upload_counters = false;
+    }
+    if (o->dyn_upload_rates) {
+        const double r[2] = {o->h.lr, o->h.wd};
+        if ((e = cudaMemcpyAsync(&o->d_plan->lr, r, sizeof r, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "upload of learning rate and weight decay");
+        o->dyn_upload_rates = false;
+    }
+    return NOVAK_OK;
+}
+
+int read_dyn(const novak_opt *o, novak::DevPlan *out)
+{
+    if (!o->d_plan) return NOVAK_ESTATE;
+    if (cudaDeviceSynchronize() != cudaSuccess) return NOVAK_ECUDA;
+    if (cudaMemcpy(out, o->d_plan, sizeof *out, cudaMemcpyDeviceToHost) != cudaSuccess) return NOVAK_ECUDA;
     return NOVAK_OK;
 }
 

@@ -43,6 +43,15 @@ int check_step_args(novak_opt *o, const char *who, void *const *d_params,
     return NOVAK_OK;
 }
 
+// What the graph-capturable step does not cover.
+int check_dyn(novak_opt *o, const char *who)
+{
+    if (o->h.layer_adapt || !o->copies.empty() || o->h.mom16 || (o->h.true_requested && o->h.true_steps > 0))
+        return fail(o, NOVAK_ESTATE, "%s: the graph-capturable step has no layer adaptation, bf16 parameter "
+                    "copies, bf16 moments or true Nesterov steps", who);
+    return NOVAK_OK;
+}
+
 // Work table on the device, records for these pointers, the scalar plan of step t+1.
 int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, int grad_dtype,
                cudaStream_t stream, StepCtx *ctx)
@@ -244,15 +253,34 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     int rc = check_step_args(o, "step", d_params, d_grads, numel, n, grad_dtype);
     if (rc != NOVAK_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (o->dyn && (rc = check_dyn(o, "step")) != NOVAK_OK) return rc;
     StepCtx ctx;
     if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
     cudaError_t e;
     int launches = 1;
     const char *what = "";
+    if (o->dyn && (rc = prepare_dyn(o, stream)) != NOVAK_OK) return rc;
     if ((e = launch_prepasses(o, ctx, stream, &launches, &what)) != cudaSuccess)
         return fail_cuda(o, e, what);
-    if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess)
+    if (o->dyn) {
+        // the step counter and the scalars live on the device: a captured launch
+        // replays as the next step
+        if ((e = novak::launch_plan(o->d_plan, &o->h, sizeof o->h, o->pdl, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "plan kernel launch");
+        novak::LaunchCfg cfg;
+        cfg.grid = o->n_chunks;
+        if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
+        cfg.reverse = ctx.pre != novak::PRE_NONE ? 1 : 0;      // serpentine needs t: not here
+        cfg.pdl = o->pdl;
+        cfg.pre = ctx.pre;
+        o->last_grid = cfg.grid;
+        if ((e = novak::launch_step_dyn(o->d_chunks, o->n_chunks, ctx.d_recs, o->prep_out, o->d_plan,
+                                        o->h.nesterov, grad_dtype, cfg, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "step kernel launch");
+        launches += 1;
+    } else if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess) {
         return fail_cuda(o, e, "step kernel launch");
+    }
     commit_step(o, ctx, launches);
     return NOVAK_OK;
 }
@@ -264,6 +292,7 @@ int novak_step_begin(novak_opt *o, void *const *d_params, const void *const *d_g
     if (!o) return NOVAK_EINVAL;
     int rc = check_step_args(o, "step_begin", d_params, d_grads, numel, n, grad_dtype);
     if (rc != NOVAK_OK) return rc;
+    if (o->dyn) return fail(o, NOVAK_ESTATE, "step_begin: not available with NOVAK_OPT_GRAPH_CAPTURABLE");
     if (o->half_open) return fail(o, NOVAK_ESTATE, "step_begin: the previous step was not finished");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     StepCtx ctx;
@@ -336,6 +365,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
     int rc = check_step_args(o, "step_host", d_params, const_cast<const void *const *>(d_grads),
                              numel, n, grad_dtype);
     if (rc != NOVAK_OK) return rc;
+    if (o->dyn) return fail(o, NOVAK_ESTATE, "step_host: not available with NOVAK_OPT_GRAPH_CAPTURABLE");
     for (int i = 0; i < n; ++i)
         if (!h_params[i] || !h_grads[i] || !d_params[i] || !d_grads[i])
             return fail(o, NOVAK_EINVAL, "step_host: tensor %d has a NULL pointer", i);
@@ -429,6 +459,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
         return fail(o, NOVAK_ESTATE, "step_noalloc: parameters are extrapolated (Eq. 10); call novak_nesterov_restore first");
     if (o->half_open)
         return fail(o, NOVAK_ESTATE, "step_noalloc: a step begun with novak_step_begin is still open");
+    if (o->dyn) return fail(o, NOVAK_ESTATE, "step_noalloc: not available with NOVAK_OPT_GRAPH_CAPTURABLE");
     if (!d_params || !d_grads || !numel) return fail(o, NOVAK_EINVAL, "step_noalloc: NULL argument");
     if (grad_dtype != NOVAK_GRAD_F32 && grad_dtype != NOVAK_GRAD_BF16)
         return fail(o, NOVAK_EINVAL, "step_noalloc: unknown grad_dtype %d", grad_dtype);

@@ -114,6 +114,30 @@ cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRe
 cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
                            const float *save_region, int grid, cudaStream_t stream);
 
+// ---- graph-capturable step: the step counter and the scalar plan in device memory
+// What novak_plan_kernel writes and novak_step_dyn_kernel reads.  t, n_syncs and
+// last_sync persist from step to step; lr and weight_decay are the values the
+// next plan uses (uploaded by the host when an option changes them).
+struct __align__(16) DevPlan {
+    long long t, n_syncs, last_sync;
+    double lr, weight_decay;
+    StepScalars s;
+    int la;                  // LA_* bits of step t
+    int nesterov;            // variant of step t
+    int rect_branch, is_sync;
+    double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay, beta1_t, beta2_t;
+};
+
+// Advances DevPlan by one step (one thread; Eq. 3-9, 18 in double on the device).
+// `hyper` is a novak_host::Hyper passed by value (opaque here).
+cudaError_t launch_plan(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
+                        cudaStream_t stream);
+// The step kernel that takes its scalars and lookahead action from *d_plan.
+// cfg.pre: PRE_NONE, PRE_SCALE or PRE_CENTER.  cudaErrorInvalidValue otherwise.
+cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
+                            const PrepOut *prep, const DevPlan *d_plan, int nesterov,
+                            int grad_dtype, const LaunchCfg &cfg, cudaStream_t stream);
+
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.
 constexpr int kNoAllocMaxTensors = 4096;

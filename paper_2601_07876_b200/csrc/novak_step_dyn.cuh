@@ -1,0 +1,124 @@
+// Graph-capturable form of the step kernel (template; instantiated by
+// novak_step_dyn_pre*.cu).  Same arithmetic, same access pattern and the same
+// building blocks as novak_step_kernel, but the per-step scalars and the
+// lookahead action are read from device memory (DevPlan, written by
+// novak_plan_kernel just before), so that a captured launch replays as the
+// NEXT step rather than as the captured one.  The lookahead action, a
+// template parameter of the plain kernel, is a uniform run-time switch here.
+#pragma once
+
+#include "novak_step_kernel.cuh"
+
+namespace novak {
+namespace {
+
+// The plain kernel's loop over chunk-table entries for one lookahead action.
+template <int NEST, int GT, int LA, int PRE>
+__device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, int n_chunks,
+                                            const TensorRec *__restrict__ recs, const PreArgs &pre0,
+                                            const StepScalars &s, int reverse, int c, Chunk ch,
+                                            TensorRec r)
+{
+    constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
+    constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
+    PreArgs pre = pre0;
+#pragma unroll 1
+    for (;;) {
+        pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
+        pre.row_len = r.row_len;
+        pre.elem0 = static_cast<uint32_t>(ch.offset);
+        float *p = r.p + ch.offset;
+        void *m = static_cast<char *>(r.m) + ch.offset * 4;
+        void *v = static_cast<char *>(r.v) + ch.offset * 4;
+        float *slow = kUseS ? r.slow + ch.offset : nullptr;
+        float *acc = kUseA ? r.acc + ch.offset : nullptr;
+        const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
+        uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(m) |
+                         reinterpret_cast<uintptr_t>(v);
+        if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
+        if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
+        const bool aligned = (bits & 15u) == 0 &&
+                             (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
+        if (aligned) {
+            const int nvec = ch.len >> 2;
+            run_span<4, kUnroll, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, nvec, s, pre);
+            const int idx = (nvec << 2) + threadIdx.x;      // ragged tail: at most 3 elements
+            if (idx < ch.len)
+                run_tile<1, 1, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, idx, s, pre);
+        } else {
+            run_span<1, 4, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, ch.len, s, pre);
+        }
+        c += gridDim.x;
+        if (c >= n_chunks) break;
+        ch = chunks[reverse ? n_chunks - 1 - c : c];
+        r = recs[ch.tensor];
+    }
+}
+
+// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER (fp32 moments, no bf16 copy).  Three
+// resident CTAs per SM (85 registers): the kernel holds every lookahead action's
+// code, and the plain kernel runs as fast at 3 CTAs per SM as at 4.
+template <int NEST, int GT, int PRE>
+__global__ void __launch_bounds__(NOVAK_BLOCK, 3)
+novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
+                      const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
+                      const DevPlan *__restrict__ plan, int reverse)
+{
+    grid_dependency_release();
+    const int c = blockIdx.x;
+    if (c >= n_chunks) return;
+    const Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
+    const TensorRec r = recs[ch.tensor];
+    grid_dependency_wait();              // the plan kernel's (and the statistics pass's) output
+
+    const StepScalars s = plan->s;
+    const int la = plan->la;
+    PreArgs pre;
+    pre.copy = nullptr;
+    pre.factor = 1.0f;
+    pre.step = s.step;
+    if constexpr ((PRE & PRE_MASK) != PRE_NONE) {
+        pre.factor = prep->factor;
+        pre.step *= prep->auto_scale;
+    }
+    switch (la) {
+#define NOVAK_DYN_CASE(X) \
+    case (X): dyn_entries<NEST, GT, (X), PRE>(chunks, n_chunks, recs, pre, s, reverse, c, ch, r); break;
+        NOVAK_DYN_CASE(LA_NONE)
+        NOVAK_DYN_CASE(LA_S_INIT | LA_S_WRITE)
+        NOVAK_DYN_CASE(LA_S_INIT | LA_S_WRITE | LA_SYNC)
+        NOVAK_DYN_CASE(LA_S_READ | LA_S_WRITE | LA_SYNC)
+        NOVAK_DYN_CASE(LA_A_WRITE)
+        NOVAK_DYN_CASE(LA_A_WRITE | LA_S_INIT | LA_S_WRITE)
+        NOVAK_DYN_CASE(LA_A_READ | LA_A_WRITE)
+        NOVAK_DYN_CASE(LA_A_READ | LA_S_READ | LA_S_WRITE | LA_SYNC | LA_TRAJ)
+#undef NOVAK_DYN_CASE
+    default: break;                      // not a lookahead action: leave everything untouched
+    }
+}
+
+using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const DevPlan *,
+                           int);
+
+template <int PRE>
+StepDynFn pick_step_dyn_kernel(int nesterov, int grad_dtype)
+{
+    const bool bf = grad_dtype == NOVAK_GRAD_BF16;
+    if (grad_dtype != NOVAK_GRAD_F32 && !bf) return nullptr;
+    switch (nesterov) {
+    case NOVAK_NESTEROV_NONE:
+        return bf ? novak_step_dyn_kernel<NOVAK_NESTEROV_NONE, NOVAK_GRAD_BF16, PRE>
+                  : novak_step_dyn_kernel<NOVAK_NESTEROV_NONE, NOVAK_GRAD_F32, PRE>;
+    case NOVAK_NESTEROV_APPROX:
+        return bf ? novak_step_dyn_kernel<NOVAK_NESTEROV_APPROX, NOVAK_GRAD_BF16, PRE>
+                  : novak_step_dyn_kernel<NOVAK_NESTEROV_APPROX, NOVAK_GRAD_F32, PRE>;
+    case NOVAK_NESTEROV_CLASSICAL:
+        return bf ? novak_step_dyn_kernel<NOVAK_NESTEROV_CLASSICAL, NOVAK_GRAD_BF16, PRE>
+                  : novak_step_dyn_kernel<NOVAK_NESTEROV_CLASSICAL, NOVAK_GRAD_F32, PRE>;
+    default: return nullptr;
+    }
+}
+
+}  // namespace
+}  // namespace novak
