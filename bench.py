@@ -99,6 +99,10 @@ def parse_args():
                          "and not part of the step (+24 B per element)")
     ap.add_argument("--moment-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of m and v (bf16: 20 B per element instead of 28)")
+    ap.add_argument("--graph", type=int, default=0, metavar="G",
+                    help="graph-capturable step: G consecutive steps are captured into one CUDA "
+                         "graph (stream capture) and the timed region replays it; steps is "
+                         "rounded down to a multiple of G")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
@@ -424,7 +428,7 @@ def main():
     del scratch
     opt = B.NovakOptimizer(params, **hyper, clip_threshold=args.clip, centralize=args.centralize,
                            layer_adaptation=args.layer_adaptation, adaptive_beta=args.adaptive_beta,
-                           auto_lr=args.auto_lr,
+                           auto_lr=args.auto_lr, graph_capturable=args.graph > 0,
                            chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
@@ -449,6 +453,22 @@ def main():
     # ---------------- resident timing: exactly K steps between two events
     for i in range(max(3, args.warmup)):
         opt.step(pool[i % pool_n])
+    graph = None
+    if args.graph > 0:
+        args.no_e2e = True                 # novak_step_host has no graph-capturable form
+        # every pointer list of the pool is resident after the warm-up; capture G steps
+        for i in range(pool_n):
+            opt.step(pool[i])
+        args.steps = max(args.graph, args.steps // args.graph * args.graph)
+        torch.cuda.synchronize()
+        l0 = opt.info()["launches"]
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(args.graph):
+                opt.step(pool[i % pool_n])
+        launches_per_graph = opt.info()["launches"] - l0
+        for _ in range(3):
+            graph.replay()
     t_first = opt.info()["t"] + 1
     launches0 = opt.info()["launches"]
     uploads0 = opt.info()["record_uploads"]
@@ -456,12 +476,19 @@ def main():
     barrier()
     with ClockSampler(local) as clocks:
         ev0.record()
-        for i in range(args.steps):
-            opt.step(pool[i % pool_n])
+        if graph is not None:
+            for _ in range(args.steps // args.graph):
+                graph.replay()
+        else:
+            for i in range(args.steps):
+                opt.step(pool[i % pool_n])
         ev1.record()
         barrier()
     ms = ev0.elapsed_time(ev1)
     launches = opt.info()["launches"] - launches0
+    if graph is not None:
+        launches = launches_per_graph * (args.steps // args.graph)
+        assert opt.info()["t"] == t_first - 1 + args.steps     # every replayed step counted
     uploads = opt.info()["record_uploads"] - uploads0
     if world > 1:
         t = torch.tensor([ms], device=dev)
@@ -481,7 +508,7 @@ def main():
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
-    if rank == 0:
+    if rank == 0 and graph is None:
         n_ps = min(args.steps, 300)
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_ps + 1)]
         t_ps = opt.info()["t"] + 1
@@ -560,6 +587,7 @@ def main():
                 "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
                 "true_nesterov": bool(args.true_nesterov),
                 "moment_dtype": args.moment_dtype,
+                "cuda_graph_steps": args.graph,
                 "auto_lr": bool(args.auto_lr),
                 "grad_pool": pool_n,
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "

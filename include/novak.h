@@ -146,9 +146,10 @@ enum {
                                      (stream capture) and replayed: the step counter,
                                      the scalars of Eq. 3-9 / 18 and the lookahead
                                      action then live in device memory, advanced by a
-                                     one-thread kernel in front of the step kernel
-                                     (one launch more per step), so that every replay
-                                     is the NEXT step.  Take one step outside the
+                                     one-thread kernel behind the step kernel (one
+                                     launch more per step; it computes the next plan
+                                     while the step runs), so that every replay is
+                                     the NEXT step.  Take one step outside the
                                      capture first (it allocates and uploads the work
                                      table), keep the captured pointer lists alive,
                                      and change options or import checkpoints outside

@@ -1,6 +1,6 @@
-// Launch side of the graph-capturable step: the one-thread kernel that advances
-// the device-resident step counter and scalar plan, and the selection of the
-// step kernel that reads them.
+// Launch side of the graph-capturable step: the one-thread kernels that keep the
+// device-resident step counter and scalar plan, and the selection of the step
+// kernel that reads them.
 #include "novak_plan.h"
 
 #include "novak_internal.h"
@@ -17,32 +17,52 @@ void *step_dyn_kernel_pre2(int nesterov, int grad_dtype);
 
 namespace {
 
-// t <- t + 1 and everything the host planner would compute for that step, from
-// the hyperparameters given by value and the learning rate and weight decay
-// kept in device memory.
-__global__ void novak_plan_kernel(DevPlan *__restrict__ dp, novak_host::Hyper h)
+// Everything the host planner would compute for step t, from the
+// hyperparameters given by value.
+__device__ void fill_slot(PlanSlot *out, const novak_host::Hyper &h, long long t)
 {
-    asm volatile("griddepcontrol.launch_dependents;");
-    asm volatile("griddepcontrol.wait;" ::: "memory");    // the previous step reads *dp
+    const novak_host::Plan p = novak_host::make_plan(h, t);
+    out->s = novak_host::make_scalars(h, p);
+    out->la = novak_host::lookahead_action(h, t);
+    out->nesterov = p.nesterov;
+    out->rect_branch = p.rect_branch;
+    out->is_sync = p.is_sync;
+    out->bc1 = p.bc1; out->bc2 = p.bc2;
+    out->rho_inf = p.rho_inf; out->rho_t = p.rho_t;
+    out->r_t = p.r_t; out->step_size = p.step_size; out->decay = p.decay;
+    out->beta1_t = p.beta1_t; out->beta2_t = p.beta2_t;
+}
+
+// After the host has uploaded counters or rates: the plan of the next step.
+__global__ void novak_plan_arm_kernel(DevPlan *__restrict__ dp, novak_host::Hyper h)
+{
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
-    const long long t = dp->t + 1;
     h.lr = dp->lr;
     h.wd = dp->weight_decay;
-    const novak_host::Plan p = novak_host::make_plan(h, t);
-    dp->t = t;
-    dp->s = novak_host::make_scalars(h, p);
-    dp->la = novak_host::lookahead_action(h, t);
-    dp->nesterov = p.nesterov;
-    dp->rect_branch = p.rect_branch;
-    dp->is_sync = p.is_sync;
-    if (p.is_sync) {
+    fill_slot(&dp->slot[dp->t & 1], h, dp->t);
+}
+
+// Launched behind the step kernel of step t.  That kernel releases its
+// dependents only after its own wait, so the plan kernel in front of it has
+// completed and dp->t is stable: the plan of step t + 1 is computed while step
+// t runs and published, together with step t's synchronisation counters, once
+// step t has completed.
+__global__ void novak_plan_next_kernel(DevPlan *__restrict__ dp, novak_host::Hyper h)
+{
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    const long long t = dp->t;
+    h.lr = dp->lr;
+    h.wd = dp->weight_decay;
+    PlanSlot next;
+    fill_slot(&next, h, t + 1);
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // step t has read slot[t & 1]
+    dp->slot[(t + 1) & 1] = next;
+    if (dp->slot[t & 1].is_sync) {
         dp->n_syncs += 1;
         dp->last_sync = t;
     }
-    dp->bc1 = p.bc1; dp->bc2 = p.bc2;
-    dp->rho_inf = p.rho_inf; dp->rho_t = p.rho_t;
-    dp->r_t = p.r_t; dp->step_size = p.step_size; dp->decay = p.decay;
-    dp->beta1_t = p.beta1_t; dp->beta2_t = p.beta2_t;
+    dp->t = t + 1;
 }
 
 using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const DevPlan *,
@@ -50,8 +70,17 @@ using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut 
 
 }  // namespace
 
-cudaError_t launch_plan(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
-                        cudaStream_t stream)
+cudaError_t launch_plan_arm(DevPlan *d_plan, const void *hyper, size_t hyper_bytes,
+                            cudaStream_t stream)
+{
+    if (!d_plan || !hyper || hyper_bytes != sizeof(novak_host::Hyper)) return cudaErrorInvalidValue;
+    const novak_host::Hyper h = *static_cast<const novak_host::Hyper *>(hyper);
+    novak_plan_arm_kernel<<<1, 32, 0, stream>>>(d_plan, h);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_plan_next(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
+                             cudaStream_t stream)
 {
     if (!d_plan || !hyper || hyper_bytes != sizeof(novak_host::Hyper)) return cudaErrorInvalidValue;
     novak_host::Hyper h = *static_cast<const novak_host::Hyper *>(hyper);
@@ -64,7 +93,7 @@ cudaError_t launch_plan(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = (pdl & 1) ? 1 : 0;
-    return cudaLaunchKernelEx(&lc, novak_plan_kernel, d_plan, h);
+    return cudaLaunchKernelEx(&lc, novak_plan_next_kernel, d_plan, h);
 }
 
 cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,

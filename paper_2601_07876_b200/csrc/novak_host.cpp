@@ -483,13 +483,15 @@ int novak_get_info(const novak_opt *o, novak_info *out)
         // replays of a captured step advance only the device's counters
         novak::DevPlan dp;
         if (read_dyn(o, &dp) != NOVAK_OK) return NOVAK_ECUDA;
-        out->t = dp.t; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
-        if (dp.t > 0) {
-            out->bc1 = dp.bc1; out->bc2 = dp.bc2; out->rho_inf = dp.rho_inf; out->rho_t = dp.rho_t;
-            out->r_t = dp.r_t; out->step_size = dp.step_size; out->decay = dp.decay;
-            out->rect_branch = dp.rect_branch; out->is_sync = dp.is_sync;
-            out->nesterov_variant = dp.nesterov;
-            out->beta1_t = dp.beta1_t; out->beta2_t = dp.beta2_t;
+        // dp.t is the step that runs next; the last one's plan is in the other slot
+        out->t = dp.t - 1; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
+        if (dp.t > 1) {
+            const novak::PlanSlot &s = dp.slot[(dp.t - 1) & 1];
+            out->bc1 = s.bc1; out->bc2 = s.bc2; out->rho_inf = s.rho_inf; out->rho_t = s.rho_t;
+            out->r_t = s.r_t; out->step_size = s.step_size; out->decay = s.decay;
+            out->rect_branch = s.rect_branch; out->is_sync = s.is_sync;
+            out->nesterov_variant = s.nesterov;
+            out->beta1_t = s.beta1_t; out->beta2_t = s.beta2_t;
         }
     }
     return NOVAK_OK;
@@ -522,7 +524,7 @@ int novak_export_meta(const novak_opt *o, novak_meta *out)
     if (o->dyn && o->d_plan) {
         novak::DevPlan dp;
         if (read_dyn(o, &dp) != NOVAK_OK) return NOVAK_ECUDA;
-        out->t = dp.t; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
+        out->t = dp.t - 1; out->n_syncs = dp.n_syncs; out->last_sync_step = dp.last_sync;
     }
     out->total_numel = o->total_numel;
     out->lr = o->h.lr; out->beta1 = o->h.beta1; out->beta2 = o->h.beta2; out->eps = o->h.eps;

@@ -293,8 +293,10 @@ int prepare_dyn(novak_opt *o, cudaStream_t stream)
     // Copies from the stack: staged by the driver before the call returns (not
     // possible while the stream is being captured: change options and import
     // checkpoints outside a capture).
+    const bool arm = o->dyn_upload_counters || o->dyn_upload_rates;
     if (o->dyn_upload_counters) {
-        const long long c[3] = {o->t, o->n_syncs, o->last_sync};
+        // the device counts the step that runs next
+        const long long c[3] = {o->t + 1, o->n_syncs, o->last_sync};
         if ((e = cudaMemcpyAsync(&o->d_plan->t, c, sizeof c, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
             return fail_cuda(o, e, "upload of the step counters");
         o->dyn_upload_counters = false;
@@ -305,6 +307,9 @@ int prepare_dyn(novak_opt *o, cudaStream_t stream)
             return fail_cuda(o, e, "upload of learning rate and weight decay");
         o->dyn_upload_rates = false;
     }
+    if (arm && (e = novak::launch_plan_arm(o->d_plan, &o->h, sizeof o->h, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "plan kernel launch");
+    if (arm) o->launches += 1;
     return NOVAK_OK;
 }
 

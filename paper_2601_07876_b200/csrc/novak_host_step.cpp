@@ -265,8 +265,6 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     if (o->dyn) {
         // the step counter and the scalars live on the device: a captured launch
         // replays as the next step
-        if ((e = novak::launch_plan(o->d_plan, &o->h, sizeof o->h, o->pdl, stream)) != cudaSuccess)
-            return fail_cuda(o, e, "plan kernel launch");
         novak::LaunchCfg cfg;
         cfg.grid = o->n_chunks;
         if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
@@ -277,6 +275,9 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
         if ((e = novak::launch_step_dyn(o->d_chunks, o->n_chunks, ctx.d_recs, o->prep_out, o->d_plan,
                                         o->h.nesterov, grad_dtype, cfg, stream)) != cudaSuccess)
             return fail_cuda(o, e, "step kernel launch");
+        // behind it: the next step's plan, computed while this step runs
+        if ((e = novak::launch_plan_next(o->d_plan, &o->h, sizeof o->h, o->pdl, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "plan kernel launch");
         launches += 1;
     } else if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess) {
         return fail_cuda(o, e, "step kernel launch");

@@ -115,24 +115,37 @@ cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d
                            const float *save_region, int grid, cudaStream_t stream);
 
 // ---- graph-capturable step: the step counter and the scalar plan in device memory
-// What novak_plan_kernel writes and novak_step_dyn_kernel reads.  t, n_syncs and
-// last_sync persist from step to step; lr and weight_decay are the values the
-// next plan uses (uploaded by the host when an option changes them).
-struct __align__(16) DevPlan {
-    long long t, n_syncs, last_sync;
-    double lr, weight_decay;
+// One step's plan as the kernels and novak_get_info need it.
+struct __align__(16) PlanSlot {
     StepScalars s;
-    int la;                  // LA_* bits of step t
-    int nesterov;            // variant of step t
+    int la;                  // LA_* bits
+    int nesterov;            // variant
     int rect_branch, is_sync;
     double bc1, bc2, rho_inf, rho_t, r_t, step_size, decay, beta1_t, beta2_t;
 };
 
-// Advances DevPlan by one step (one thread; Eq. 3-9, 18 in double on the device).
-// `hyper` is a novak_host::Hyper passed by value (opaque here).
-cudaError_t launch_plan(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
-                        cudaStream_t stream);
-// The step kernel that takes its scalars and lookahead action from *d_plan.
+// t is the index of the step that runs NEXT; its plan is armed in slot[t & 1]
+// and the plan of the step that ran last is still in slot[(t - 1) & 1].  The
+// step kernel only reads; novak_plan_next_kernel, launched behind it, computes
+// the plan of step t + 1 while the step runs and publishes it (and t + 1, and
+// the synchronisation counters of step t) once the step has completed.  lr and
+// weight_decay are what the next plan uses (uploaded by the host when an
+// option changes them, followed by novak_plan_arm_kernel).
+struct __align__(16) DevPlan {
+    long long t, n_syncs, last_sync;
+    double lr, weight_decay;
+    PlanSlot slot[2];
+};
+
+// (Re)computes the armed plan slot[t & 1] from dp->t and the rates in *dp (after
+// the host has uploaded counters or rates).  `hyper` is a novak_host::Hyper
+// passed by value (opaque here).  Plain launch.
+cudaError_t launch_plan_arm(DevPlan *d_plan, const void *hyper, size_t hyper_bytes,
+                            cudaStream_t stream);
+// Behind the step kernel: the plan of step t + 1, published when the step is done.
+cudaError_t launch_plan_next(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
+                             cudaStream_t stream);
+// The step kernel that takes its scalars and lookahead action from the armed slot.
 // cfg.pre: PRE_NONE, PRE_SCALE or PRE_CENTER.  cudaErrorInvalidValue otherwise.
 cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
                             const PrepOut *prep, const DevPlan *d_plan, int nesterov,

@@ -1,13 +1,18 @@
 // Graph-capturable form of the step kernel (template; instantiated by
 // novak_step_dyn_pre*.cu).  Same arithmetic, same access pattern and the same
 // building blocks as novak_step_kernel, but the per-step scalars and the
-// lookahead action are read from device memory (DevPlan, written by
-// novak_plan_kernel just before), so that a captured launch replays as the
-// NEXT step rather than as the captured one.  The lookahead action, a
+// lookahead action are read from device memory (the armed slot of DevPlan),
+// so that a captured launch replays as the NEXT step rather than as the
+// captured one.  The kernel only reads the plan; novak_plan_next_kernel,
+// launched behind it, advances it.  The lookahead action, a
 // template parameter of the plain kernel, is a uniform run-time switch here.
 #pragma once
 
 #include "novak_step_kernel.cuh"
+
+#ifndef NOVAK_DYN_MIN_CTAS
+#define NOVAK_DYN_MIN_CTAS 4
+#endif
 
 namespace novak {
 namespace {
@@ -56,24 +61,28 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
     }
 }
 
-// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER (fp32 moments, no bf16 copy).  Three
-// resident CTAs per SM (85 registers): the kernel holds every lookahead action's
-// code, and the plain kernel runs as fast at 3 CTAs per SM as at 4.
+// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER (fp32 moments, no bf16 copy).  The
+// kernel holds every lookahead action's code; at four resident CTAs per SM (64
+// registers) it spills a little on the heavier actions, which costs less than
+// the lost CTA of the 80-register build when the gradient is pre-processed.
 template <int NEST, int GT, int PRE>
-__global__ void __launch_bounds__(NOVAK_BLOCK, 3)
+__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_DYN_MIN_CTAS)
 novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                       const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
                       const DevPlan *__restrict__ plan, int reverse)
 {
-    grid_dependency_release();
     const int c = blockIdx.x;
     if (c >= n_chunks) return;
     const Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
     const TensorRec r = recs[ch.tensor];
-    grid_dependency_wait();              // the plan kernel's (and the statistics pass's) output
+    grid_dependency_wait();              // the previous plan kernel's (and the statistics pass's) output
+    // Only now may the plan kernel behind this one start: it reads the step
+    // counter, which the plan kernel in front has just finished writing.
+    grid_dependency_release();
 
-    const StepScalars s = plan->s;
-    const int la = plan->la;
+    const PlanSlot *slot = &plan->slot[plan->t & 1];
+    const StepScalars s = slot->s;
+    const int la = slot->la;
     PreArgs pre;
     pre.copy = nullptr;
     pre.factor = 1.0f;

@@ -18,7 +18,7 @@ from . import binding as B
 _GROUP_KEYS = ("lr", "betas", "eps", "weight_decay", "nesterov", "lookahead_k", "lookahead_alpha",
                "nesterov_beta", "lookahead_mode", "rectified", "clip_threshold", "centralize",
                "adaptive_beta", "layer_adaptation", "sparse_threshold", "auto_lr",
-               "true_nesterov_steps", "moment_dtype")
+               "true_nesterov_steps", "moment_dtype", "graph_capturable")
 
 
 class Novak(torch.optim.Optimizer):
@@ -28,21 +28,25 @@ class Novak(torch.optim.Optimizer):
     have a gradient (float32 or bfloat16, one dtype per group) when ``step`` is
     called.  ``lr`` and ``weight_decay`` of a group may be changed between steps
     (learning-rate schedulers); the other entries are fixed once the group has
-    taken its first step.
+    taken its first step.  With ``graph_capturable=True`` the step counter and the
+    per-step scalars live on the device, so that ``step()`` may be captured into a
+    CUDA graph (``torch.cuda.graph``) after one eager step and replayed.
     """
 
     def __init__(self, params, lr=1e-3, betas=(0.9, 0.999), eps=1e-8, weight_decay=1e-2,
                  nesterov="approximation", lookahead_k=5, lookahead_alpha=0.5, *,
                  nesterov_beta=None, lookahead_mode="last", rectified=True, clip_threshold=0.0,
                  centralize=False, adaptive_beta=False, layer_adaptation=False,
-                 sparse_threshold=0.0, auto_lr=False, true_nesterov_steps=0, moment_dtype="f32"):
+                 sparse_threshold=0.0, auto_lr=False, true_nesterov_steps=0, moment_dtype="f32",
+                 graph_capturable=False):
         defaults = dict(lr=lr, betas=betas, eps=eps, weight_decay=weight_decay, nesterov=nesterov,
                         lookahead_k=lookahead_k, lookahead_alpha=lookahead_alpha,
                         nesterov_beta=nesterov_beta, lookahead_mode=lookahead_mode,
                         rectified=rectified, clip_threshold=clip_threshold, centralize=centralize,
                         adaptive_beta=adaptive_beta, layer_adaptation=layer_adaptation,
                         sparse_threshold=sparse_threshold, auto_lr=auto_lr,
-                        true_nesterov_steps=true_nesterov_steps, moment_dtype=moment_dtype)
+                        true_nesterov_steps=true_nesterov_steps, moment_dtype=moment_dtype,
+                        graph_capturable=graph_capturable)
         super().__init__(params, defaults)
         self._engines: list[B.NovakOptimizer | None] = [None] * len(self.param_groups)
         self._applied: list[tuple] = [()] * len(self.param_groups)

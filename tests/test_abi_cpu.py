@@ -128,6 +128,18 @@ def test_true_nesterov_steps_then_fallback_to_the_approximation():
     g.destroy()
 
 
+def test_graph_capturable_option():
+    h = B.Handle(**GOOD)
+    assert h.get_option(B.NOVAK_OPT_GRAPH_CAPTURABLE) == 0
+    h.set_option(B.NOVAK_OPT_GRAPH_CAPTURABLE, 1)
+    assert h.get_option(B.NOVAK_OPT_GRAPH_CAPTURABLE) == 1
+    for bad in (2, -1, 0.5, float("nan")):
+        with pytest.raises(B.NovakError):
+            h.set_option(B.NOVAK_OPT_GRAPH_CAPTURABLE, bad)
+    assert h.get_info().t == 0          # nothing on the device yet: no read-back, no CUDA call
+    h.destroy()
+
+
 def test_options_validate_and_roundtrip():
     h = B.Handle(**GOOD)
     assert h.get_option(B.NOVAK_OPT_NESTEROV_BETA) == 0.9   # default beta_N = beta1

@@ -123,3 +123,41 @@ def test_closure_is_evaluated_at_the_look_ahead_point():
     eng = opt._engines[0]
     assert_close(eng.state(0)["m"], oracle.m[0], "m")
     assert eng.info()["t"] == 7 and eng.info()["launches"] == 7 + 2 * 4
+
+
+def test_whole_iteration_captured_into_a_cuda_graph():
+    """Forward, backward and the optimizer step captured once (static input buffer) and
+    replayed: the same parameters as the eager loop of a twin model."""
+    a, b = _model(3), _model(3)
+    kw = dict(HYPER, clip_threshold=0.5)
+    eager = Novak(a.parameters(), **kw)
+    graphed = Novak(b.parameters(), **kw, graph_capturable=True)
+    xs = [torch.randn(16, 37, device=DEV) for _ in range(9)]
+    static_x = torch.empty(16, 37, device=DEV)
+
+    def iteration(model, opt, x):
+        opt.zero_grad(set_to_none=False)         # gradients stay where they are: static buffers
+        model(x).square().mean().backward()
+        opt.step()
+
+    for x in xs[:2]:                             # warm-up outside the capture, on a side stream
+        iteration(a, eager, x)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for x in xs[:2]:
+            static_x.copy_(x)
+            iteration(b, graphed, static_x)
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    static_x.copy_(xs[2])
+    with torch.cuda.graph(graph):
+        iteration(b, graphed, static_x)
+    for x in xs[2:]:
+        iteration(a, eager, x)
+        static_x.copy_(x)
+        graph.replay()
+    torch.cuda.synchronize()
+    assert graphed._engines[0].info()["t"] == 9 == eager._engines[0].info()["t"]
+    for pa, pb in zip(a.parameters(), b.parameters()):
+        torch.testing.assert_close(pb, pa, rtol=1e-5, atol=1e-7)
