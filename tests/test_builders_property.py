@@ -75,3 +75,38 @@ def test_rank_partition_covers_every_element_once_and_is_balanced(numel, world, 
     assert all((s == 1).all() for s in seen)
     total = sum(numel)
     assert max(counts) - min(counts) <= max(2 * align, total - (total // align) * align + align)
+
+
+@settings(max_examples=150, deadline=None)
+@given(beta1=st.floats(0.0, 0.9999), beta2=st.floats(0.0, 0.99999),
+       lr=st.floats(1e-6, 1.0), wd=st.floats(0.0, 1.0), k=st.integers(0, 12),
+       t=st.one_of(st.integers(1, 200), st.integers(200, 10 ** 7)),
+       adaptive=st.booleans(), rectified=st.booleans())
+def test_planner_agrees_with_the_oracle_for_any_hyperparameters(beta1, beta2, lr, wd, k, t,
+                                                                adaptive, rectified):
+    """The library's host plan (double, -expm1(t log beta)) against the oracle's scalars
+    (long double powers): Eq. 3-9, 18, the branch of Eq. 8 and the sync schedule.  Where
+    rho_t comes within 1e-6 of 5 the branch may legitimately differ and the case is skipped."""
+    from oracle import novak_oracle as O
+    h = B.Handle(lr=lr, beta1=beta1, beta2=beta2, eps=1e-8, weight_decay=wd,
+                 nesterov_variant=B.NOVAK_NESTEROV_APPROX, lookahead_k=k, lookahead_alpha=0.5)
+    h.set_option(B.NOVAK_OPT_RECTIFIED, 1 if rectified else 0)
+    h.set_option(B.NOVAK_OPT_ADAPTIVE_BETA, 1 if adaptive else 0)
+    o = O.Oracle(O.Config(lr=lr, beta1=beta1, beta2=beta2, weight_decay=wd, lookahead_k=k,
+                          rectified=rectified, adaptive_beta=adaptive), [np.zeros(1)])
+    a, b = h.plan(t), o.scalars(t)
+    h.destroy()
+    if abs(b.rho_t - 5.0) < 1e-6:
+        return
+    assert a.rect_branch == b.rect_branch and a.is_sync == b.is_sync
+    for name in ("bc1", "bc2", "rho_inf", "decay", "beta1_t", "beta2_t"):
+        x, y = getattr(a, name), getattr(b, name)
+        assert abs(x - y) <= 1e-11 * abs(y) + 1e-300, (name, x, y)
+    # rho_t = rho_inf - 2 t beta2^t / (1 - beta2^t) cancels: compare at the scale of rho_inf
+    assert abs(a.rho_t - b.rho_t) <= 1e-9 * max(1.0, b.rho_inf)
+    if a.rect_branch:
+        # r_t is well conditioned away from rho_t = 4 (the branch needs rho_t >= 5)
+        assert abs(a.r_t - b.r_t) <= 1e-7 * b.r_t
+        assert abs(a.step_size - b.step_size) <= 1e-7 * b.step_size
+    else:
+        assert a.r_t == 1.0 == b.r_t and abs(a.step_size - b.step_size) <= 1e-12 * b.step_size
