@@ -125,3 +125,33 @@ def test_what_the_mode_does_not_cover_is_refused():
     with pytest.raises(B.NovakError):                     # fixed once a step was taken
         opt.handle.set_option(B.NOVAK_OPT_GRAPH_CAPTURABLE, 0)
     assert opt.info()["t"] == 1
+
+
+def test_fullsize_resnet50_replayed():
+    """The ResNet-50-shaped set at full size: one eager step, one captured step, 18 replays
+    (gradients refilled in the captured buffer between replays); the oracle follows the
+    usual sample of elements."""
+    from harness import SampledPair
+    from paper_2601_07876_b200 import workloads as W
+    wl = W.get_workload(1)
+    pair = SampledPair(wl, DEV, opt_kwargs=dict(graph_capturable=True))
+    pair.step(threads=8)                                  # eager: t = 1
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    pair.src.fill(pair.flat_g, pair.scratch)
+    with torch.cuda.graph(graph):
+        pair.opt.step(pair.glist)
+    for t in range(2, 21):
+        if t > 2:
+            pair.src.fill(pair.flat_g, pair.scratch)
+        graph.replay()
+        pair.oracle.step([to_f64(pair.flat_g[pair.idx])], threads=8)
+    torch.cuda.synchronize()
+    info = pair.opt.info()
+    assert info["t"] == 20 == pair.oracle.t and info["n_syncs"] == 4 and info["last_sync_step"] == 20
+    assert_close(pair.flat_p[pair.idx], pair.oracle.theta[0], "resnet50 replayed theta")
+    assert_close(pair._gather_state("m"), pair.oracle.m[0], "resnet50 replayed m")
+    assert_close(pair._gather_state("v"), pair.oracle.v[0], "resnet50 replayed v")
+    assert_close(pair._gather_state("slow"), pair.oracle.slow[0], "resnet50 replayed slow")
+    del pair
+    torch.cuda.empty_cache()
