@@ -270,6 +270,10 @@ size_t novak_state_bytes(const novak_opt *opt, const int64_t *numel, int n);
  * 16-byte alignment; with NULL, slices start at their slot's base.  The whole
  * buffer is zero-filled asynchronously on `stream` (a cudaStream_t); the slow
  * weights are set to theta_0 by the first step's kernel (Eq. 28).
+ * The device d_state lives on becomes the handle's device: every later call
+ * that touches CUDA makes it current for its own duration and puts the
+ * caller's device back, so one process may hold handles on several GPUs (a
+ * stream passed to a call must belong to the handle's device).
  * Errors: NOVAK_EINVAL (NULL, n <= 0, numel[i] <= 0, misaligned or short
  * buffer, parameter pointer not 4-byte aligned), NOVAK_ECUDA. */
 int novak_attach_state(novak_opt *opt, void *d_state, size_t bytes,

@@ -95,6 +95,8 @@ struct Handle {
     bool half_open = false;
     int half_launches = 0;
     alignas(8) unsigned char half_ctx[256] = {};   // the StepCtx of the open step
+    int device = -1;                    // CUDA device of the attached state buffer (-1: unknown)
+
     // graph-capturable step: the counters and the plan in device memory
     int dyn = 0;
     novak::DevPlan *d_plan = nullptr;
@@ -156,6 +158,24 @@ inline int kernel_variant(const Plan &p)
 {
     return p.nesterov == NOVAK_NESTEROV_TRUE ? NOVAK_NESTEROV_NONE : p.nesterov;
 }
+
+// Makes the handle's device current for the lifetime of the object when it is
+// not (a process that drives several GPUs); restores the caller's device.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int want)
+    {
+        if (want < 0 || cudaGetDevice(&prev) != cudaSuccess || prev == want) return;
+        switched = cudaSetDevice(want) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+    DeviceGuard(const DeviceGuard &) = delete;
+    DeviceGuard &operator=(const DeviceGuard &) = delete;
+};
 
 // Error reporting: store the message in the handle, return the code.
 int fail(novak_opt *o, int code, const char *fmt, ...);

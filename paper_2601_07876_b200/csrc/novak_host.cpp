@@ -226,6 +226,7 @@ int novak_create(novak_opt **out, double lr, double beta1, double beta2, double 
 void novak_destroy(novak_opt *opt)
 {
     if (!opt) return;
+    DeviceGuard on_device(opt->device);
     release_device(opt);
     delete opt;
 }
@@ -393,10 +394,24 @@ int novak_attach_state(novak_opt *o, void *d_state, size_t bytes, void *const *d
             phase[i] = static_cast<int32_t>((p % (kSlotAlign * 4)) / 4);
         }
     }
-    cudaError_t e = cudaMemsetAsync(d_state, 0, need, static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) return fail_cuda(o, e, "cudaMemsetAsync(state)");
+    // the device the buffer lives on becomes the handle's device
+    int device = -1;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, d_state) == cudaSuccess && attr.type == cudaMemoryTypeDevice)
+        device = attr.device;
+    else
+        (void)cudaGetLastError();       // not a device pointer the runtime knows: no guard
+    {
+        DeviceGuard on_device(device);
+        cudaError_t e = cudaMemsetAsync(d_state, 0, need, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return fail_cuda(o, e, "cudaMemsetAsync(state)");
+    }
+    {
+        DeviceGuard old_device(o->device);   // a previous attachment's tables are freed where they live
+        release_device(o);
+    }
+    o->device = device;
 
-    release_device(o);
     o->na_chunks.clear();
     o->na_p.clear();
     o->na_token = 0;
@@ -478,6 +493,7 @@ int novak_set_param_copies(novak_opt *o, void *const *d_copies, int n)
 int novak_get_info(const novak_opt *o, novak_info *out)
 {
     if (!o || !out) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     fill_info(o, o->last_plan, out);
     if (o->dyn && o->d_plan) {
         // replays of a captured step advance only the device's counters
@@ -518,6 +534,7 @@ int novak_state_ptrs(const novak_opt *o, int tensor, void **d_m, void **d_v, voi
 int novak_export_meta(const novak_opt *o, novak_meta *out)
 {
     if (!o || !out) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     std::memset(out, 0, sizeof *out);
     out->magic = kMetaMagic;
     out->t = o->t; out->n_syncs = o->n_syncs; out->last_sync_step = o->last_sync;

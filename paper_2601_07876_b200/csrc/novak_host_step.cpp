@@ -250,6 +250,7 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
                const int64_t *numel, int n, int grad_dtype, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     int rc = check_step_args(o, "step", d_params, d_grads, numel, n, grad_dtype);
     if (rc != NOVAK_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -314,6 +315,7 @@ int novak_step_begin(novak_opt *o, void *const *d_params, const void *const *d_g
 int novak_local_sums(novak_opt *o, double **d_sums)
 {
     if (!o || !d_sums) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!o->half_open) return fail(o, NOVAK_ESTATE, "local_sums: no step is open");
     *d_sums = o->prep_out ? o->prep_out->local_sums : nullptr;
     return NOVAK_OK;
@@ -322,6 +324,7 @@ int novak_local_sums(novak_opt *o, double **d_sums)
 int novak_copy_local_sums(novak_opt *o, double *d_dst, void *stream_)
 {
     if (!o || !d_dst) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!o->half_open) return fail(o, NOVAK_ESTATE, "copy_local_sums: no step is open");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     cudaError_t e;
@@ -337,6 +340,7 @@ int novak_copy_local_sums(novak_opt *o, double *d_dst, void *stream_)
 int novak_step_finish(novak_opt *o, const double *d_total_sums, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!o->half_open) return fail(o, NOVAK_ESTATE, "step_finish: no step is open");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     StepCtx ctx;
@@ -362,6 +366,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
                     int grad_dtype, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!h_params || !h_grads) return fail(o, NOVAK_EINVAL, "step_host: NULL argument");
     int rc = check_step_args(o, "step_host", d_params, const_cast<const void *const *>(d_grads),
                              numel, n, grad_dtype);
@@ -455,6 +460,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
                        const int64_t *numel, int n, int grad_dtype, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!o->attached) return fail(o, NOVAK_ESTATE, "step_noalloc: no state attached");
     if (o->extrapolated)
         return fail(o, NOVAK_ESTATE, "step_noalloc: parameters are extrapolated (Eq. 10); call novak_nesterov_restore first");
@@ -603,6 +609,7 @@ int novak_nesterov_extrapolate(novak_opt *o, void *const *d_params, void *d_save
                                const int64_t *numel, int n, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     int rc = check_look_args(o, "nesterov_extrapolate", d_params, d_save, save_bytes, numel, n);
     if (rc != NOVAK_OK) return rc;
     if (o->extrapolated)
@@ -623,6 +630,7 @@ int novak_nesterov_restore(novak_opt *o, void *const *d_params, const void *d_sa
                            const int64_t *numel, int n, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     int rc = check_look_args(o, "nesterov_restore", d_params, d_save, save_bytes, numel, n);
     if (rc != NOVAK_OK) return rc;
     if (!o->extrapolated)
@@ -643,6 +651,7 @@ int novak_nesterov_restore(novak_opt *o, void *const *d_params, const void *d_sa
 int novak_get_grad_stats(novak_opt *o, double *norm, double *factor, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!o->prep_out) return fail(o, NOVAK_ESTATE, "get_grad_stats: no step with clipping or centralization yet");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     PrepOut h;
@@ -659,6 +668,7 @@ int novak_get_auto_lr_state(novak_opt *o, double *g_bar, double *theta_bar, doub
                             void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (o->ema_pending || !o->prep_out) {
         // nothing on the device yet: what a resume put in, or the initial zeros
         if (g_bar) *g_bar = o->ema_pending ? o->pending_g_bar : 0.0;
@@ -692,6 +702,7 @@ int novak_set_auto_lr_state(novak_opt *o, double g_bar, double theta_bar)
 int novak_get_trust_ratios(novak_opt *o, float *h_out, int n, void *stream_)
 {
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     if (!h_out || n != o->n) return fail(o, NOVAK_EINVAL, "get_trust_ratios: NULL or wrong tensor count");
     if (!o->trust || o->t == 0) return fail(o, NOVAK_ESTATE, "get_trust_ratios: no step with layer adaptation yet");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
