@@ -522,7 +522,7 @@ int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
                            int32_t *len, int64_t cap);
 
 /* Host-only helper exposing how the statistics pass of the centralization cuts
- * tensors with rows into units: groups of whole rows of up to 2048 elements,
+ * tensors with rows into units: groups of whole rows of up to 8192 elements,
  * about 16384 elements per group (part_len = 0), or, for longer rows, slices
  * [part_off, part_off + part_len) of at most 16384 elements of one row
  * (n_rows = 1), consecutive in the table.  rows[i] as in novak_set_tensor_rows.  Writes up to cap entries and

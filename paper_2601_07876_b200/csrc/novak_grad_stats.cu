@@ -10,10 +10,10 @@
 // Decomposition.  Tensors without rows: one CTA per 4 consecutive chunk-table
 // entries (the table of the step kernel), sum of squares only.  Tensors with
 // rows: a table of row units built on the host, aligned to ROWS, not to the
-// chunk table: a unit is a group of whole rows of up to 2048 elements (a warp
-// streams each row; eight lanes for rows shorter than 128 elements, a thread
-// below 32), or a slice of at most 16384 elements of a longer row (the whole
-// CTA; usually the whole row).  No shared-memory
+// chunk table: a unit is a group of whole rows of up to 8192 elements (a warp
+// streams each row; half a warp for rows of up to 1024 elements, eight lanes
+// below 128, a thread below 32), or a slice of at most 16384 elements of a
+// longer row (the whole CTA).  No shared-memory
 // staging, no per-vector row arithmetic: a lane only ever adds along one row.
 // All sums are carried in double precision and combined in a fixed order (per
 // lane, warp shuffle tree, warps in index order, CTAs in index order), so the
@@ -329,6 +329,29 @@ __device__ __forceinline__ void span_sums(const void *g_tensor, uint32_t e0, uin
     }
 }
 
+// Whole rows [row0, row0 + n_rows) of length L, LANES lanes per row (8, 16 or
+// 32), so that a warp works on 32 / LANES rows at a time: the loads of several
+// rows are in flight together and a lane's share of a short row still fills a
+// batch of four loads.  Row means are written; the squares go into sq.
+template <int GT, int LANES>
+__device__ __forceinline__ void rows_by_lane_group(const TensorRec &rec, uint32_t row0, uint32_t n_rows,
+                                                   uint32_t L, double &sq)
+{
+    constexpr uint32_t kPerWarp = 32u / LANES;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    const uint32_t sub = lane / LANES, l = lane % LANES;
+    const uint32_t end = row0 + n_rows;
+    for (uint32_t r0 = row0 + warp * kPerWarp; r0 < end; r0 += kStatsWarps * kPerWarp) {
+        const uint32_t r = r0 + sub;
+        const bool live = r < end;
+        double sum = 0.0;
+        span_sums<GT>(rec.g, live ? r * L : 0u, live ? L : 0u, l, LANES, sum, sq);
+#pragma unroll
+        for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (live && l == 0u) rec.mean[r] = split_mean(sum, L);
+    }
+}
+
 // ---- tensors with rows: one unit of the row table (see RowUnit)
 template <int GT>
 __device__ __forceinline__ double row_unit(const RowUnit u, const TensorRec rec,
@@ -348,29 +371,13 @@ __device__ __forceinline__ double row_unit(const RowUnit u, const TensorRec rec,
             if (u.n_parts == 1u) rec.mean[u.row0] = split_mean(total, L);
             else part_sum[unit_index] = total;
         }
+    } else if (L > kRowHalfWarpMax) {
+        rows_by_lane_group<GT, 32>(rec, u.row0, u.n_rows, L, sq);     // a warp per row
     } else if (L >= 128u) {
-        // whole rows, a warp each
-        for (uint32_t r = u.row0 + warp; r < u.row0 + u.n_rows; r += kStatsWarps) {
-            double sum = 0.0;
-            span_sums<GT>(rec.g, r * L, L, lane, 32u, sum, sq);
-            sum = warp_sum(sum);
-            if (lane == 0) rec.mean[r] = split_mean(sum, L);
-        }
+        rows_by_lane_group<GT, 16>(rec, u.row0, u.n_rows, L, sq);     // two rows per warp
     } else if (L >= 32u) {
-        // short rows: eight lanes each, a warp takes four rows at a time (a thread
-        // per row would read its row as a chain of dependent scalar loads)
-        const uint32_t sub = lane >> 3, l8 = lane & 7u;
-        const uint32_t end = u.row0 + u.n_rows;
-        for (uint32_t r0 = u.row0 + warp * 4u; r0 < end; r0 += kStatsWarps * 4u) {
-            const uint32_t r = r0 + sub;
-            const bool live = r < end;
-            double sum = 0.0;
-            span_sums<GT>(rec.g, live ? r * L : 0u, live ? L : 0u, l8, 8u, sum, sq);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-            if (live && l8 == 0u) rec.mean[r] = split_mean(sum, L);
-        }
+        // (a thread per row would read its row as a chain of dependent scalar loads)
+        rows_by_lane_group<GT, 8>(rec, u.row0, u.n_rows, L, sq);      // four rows per warp
     } else {
         // very short rows, a thread each
         const uint32_t r = u.row0 + threadIdx.x;

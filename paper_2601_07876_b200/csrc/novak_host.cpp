@@ -62,7 +62,9 @@ void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vect
             // elements on, a thread per row below)
             // (rows per unit a multiple of 8, so that no warp idles while others take a
             // second row)
-            const uint32_t per = L >= 128u ? std::max(8u, novak::kRowUnitElems / L / 8u * 8u)
+            // (16 where two rows share a warp)
+            const uint32_t step = L <= novak::kRowHalfWarpMax ? 16u : 8u;
+            const uint32_t per = L >= 128u ? std::max(step, novak::kRowUnitElems / L / step * step)
                                            : novak::kRowUnitThreads;
             for (uint32_t r = 0; r < R; r += per)
                 out.push_back(RowUnit{i, r, std::min(per, R - r), 0u, 0u, 1u, 0u, 0u});

@@ -43,8 +43,8 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
 // One unit of work of the statistics pass for a tensor with rows (Eq. 26).
 // Rows of up to kRowWarpMax elements: n_rows (a multiple of 8 but for a tensor's
 // last unit) whole rows starting at row0
-// (part_len = 0), a warp per row (below 128 elements eight lanes, below 32 a
-// thread).  Longer
+// (part_len = 0), a warp per row (half a warp up to kRowHalfWarpMax elements,
+// eight lanes below 128, a thread below 32).  Longer
 // rows: one slice [part_off, part_off + part_len) of row row0 for the whole
 // CTA; the row is cut into n_parts slices of at most kRowUnitElems elements, of
 // which this is number part_idx (units of one row are consecutive in the table).
@@ -62,7 +62,8 @@ struct __align__(16) RowUnit {
 // Elements a row unit aims at, and rows per unit where a thread takes a row.
 constexpr uint32_t kRowUnitElems = 16384;
 constexpr uint32_t kRowUnitThreads = 256;
-constexpr uint32_t kRowWarpMax = 2048;     // longest row a single warp streams
+constexpr uint32_t kRowWarpMax = 8192;     // longest row a single warp streams
+constexpr uint32_t kRowHalfWarpMax = 1024; // longest row that gets half a warp (two rows per warp)
 
 // What the statistics pass works on, all in device memory.
 struct StatsPlan {

@@ -239,7 +239,7 @@ def test_planner_adaptive_beta_agrees_with_oracle():
 
 
 def test_row_units_cover_every_row_once():
-    """The statistics pass's row table: rows of up to 2048 elements whole, in groups of about
+    """The statistics pass's row table: rows of up to 8192 elements whole, in groups of about
     16384 elements; longer rows in consecutive slices of at most 16384 elements; tensors
     without rows left out."""
     shapes = [(8, 27), (33,), (10, 257), (3, 5000), (4097, 2), (1, 7), (5, 1), (2048,), (6, 2048),
@@ -254,13 +254,13 @@ def test_row_units_cover_every_row_once():
         L = numel[t] // rows[t]
         assert rows[t] > 0 and n_rows >= 1 and row0 + n_rows <= rows[t]
         if part_len:
-            assert L > 2048 and n_rows == 1 and 0 < part_len <= 16384 and part_off % 16384 == 0
+            assert L > 8192 and n_rows == 1 and 0 < part_len <= 16384 and part_off % 16384 == 0
             assert part_off + part_len <= L
             if part_off:          # slices of a row are consecutive, in order
                 assert prev[:2] == (t, row0) and prev[3] + prev[4] == part_off
             seen[t][row0, part_off:part_off + part_len] += 1
         else:
-            assert L <= 2048
+            assert L <= 8192
             assert n_rows * L <= max(16384, 8 * L) if L >= 128 else n_rows <= 256
             seen[t][row0:row0 + n_rows, :] += 1
         prev = (t, row0, n_rows, part_off, part_len)

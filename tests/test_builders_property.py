@@ -49,10 +49,10 @@ def test_row_units_cover_every_row_once(data):
     for t, row0, n_rows, part_off, part_len in units:
         L = numel[t] // rows[t]
         if part_len:
-            assert L > 2048 and n_rows == 1 and part_len <= 16384
+            assert L > 8192 and n_rows == 1 and part_len <= 16384
             seen[t][row0, part_off:part_off + part_len] += 1
         else:
-            assert L <= 2048
+            assert L <= 8192
             seen[t][row0:row0 + n_rows] += 1
     assert all((s == 1).all() for s in seen.values())
     assert {u[0] for u in units} == set(seen)
