@@ -150,14 +150,35 @@ struct PreArgs {
 // crosses into the next one.  The mean comes as hi + lo: where g and the mean
 // nearly cancel, g - hi is exact and lo supplies the mean's remaining bits, so
 // the centred gradient carries a relative rounding error only.
+// Where a vector starts inside its tensor's rows, with that row's mean.
+struct RowPos {
+    uint32_t row, rem;
+    float2 mu;
+};
+
+template <int PRE>
+__device__ __forceinline__ RowPos row_position(uint32_t e, const PreArgs &a)
+{
+    RowPos r;
+    r.row = 0u; r.rem = 0u; r.mu = make_float2(0.0f, 0.0f);
+    if constexpr ((PRE & PRE_MASK) == PRE_CENTER) {
+        if (a.mean != nullptr) {
+            r.row = e / a.row_len;
+            r.rem = e - r.row * a.row_len;
+            r.mu = __ldg(a.mean + r.row);
+        }
+    }
+    return r;
+}
+
 template <int N, int PRE>
-__device__ __forceinline__ void preprocess(Vec<N> &G, uint32_t e, const PreArgs &a)
+__device__ __forceinline__ void preprocess(Vec<N> &G, const RowPos &pos, const PreArgs &a)
 {
     if constexpr ((PRE & PRE_MASK) == PRE_CENTER) {
         if (a.mean != nullptr) {
-            uint32_t row = e / a.row_len;
-            uint32_t rem = e - row * a.row_len;
-            float2 mu = __ldg(a.mean + row);
+            uint32_t row = pos.row;
+            uint32_t rem = pos.rem;
+            float2 mu = pos.mu;
 #pragma unroll
             for (int j = 0; j < N; ++j) {
                 if (rem == a.row_len) {     // stepped over the end of the row
@@ -249,10 +270,16 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, void *m, void 
     constexpr bool kWriteS = (LA & LA_S_WRITE) != 0;
     constexpr bool kReadA = (LA & LA_A_READ) != 0;
     constexpr bool kWriteA = (LA & LA_A_WRITE) != 0;
+    // On steps without a synchronisation (fewer live registers) the row means
+    // are fetched together with the streams, so that their latency overlaps.
+    constexpr bool kEarlyMean = (LA & LA_SYNC) == 0 && (PRE & PRE_MASK) == PRE_CENTER;
     Vec<N> P[U], G[U], M[U], V[U], S[U], A[U];
+    RowPos R[U];
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const int idx = first + j * kBlock;
+        if constexpr (kEarlyMean)
+            R[j] = row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
         P[j] = load_f32<N>(p, idx);
         G[j] = load_grad<N, GT>(g, idx);
         M[j] = load_moment<N, kMom16>(m, idx);
@@ -263,7 +290,9 @@ __device__ __forceinline__ void run_tile(float *p, const void *g, void *m, void 
 #pragma unroll
     for (int j = 0; j < U; ++j) {
         const int idx = first + j * kBlock;
-        preprocess<N, PRE>(G[j], pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
+        if constexpr (!kEarlyMean)
+            R[j] = row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
+        preprocess<N, PRE>(G[j], R[j], pre);
 #pragma unroll
         for (int e = 0; e < N; ++e)
             update_element<NEST, LA>(P[j].a[e], G[j].a[e], M[j].a[e], V[j].a[e],

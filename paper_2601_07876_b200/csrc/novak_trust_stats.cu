@@ -51,7 +51,7 @@ __device__ __forceinline__ void accumulate(const float *p, const void *g, const 
     Vec<N> G = load_grad<N, GT>(g, idx);
     const Vec<N> M = load_moment<N, (PRE & PRE_MOM16) != 0>(m, idx);
     const Vec<N> V = load_moment<N, (PRE & PRE_MOM16) != 0>(v, idx);
-    preprocess<N, PRE>(G, pre.elem0 + static_cast<uint32_t>(idx) * N, pre);
+    preprocess<N, PRE>(G, row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre), pre);
     float sp = 0.0f, su = 0.0f;
 #pragma unroll
     for (int e = 0; e < N; ++e) {
