@@ -485,6 +485,7 @@ def main():
         ev1.record()
         barrier()
     ms = ev0.elapsed_time(ev1)
+    grid_timed = opt.info()["grid"]          # before the end-to-end leg launches its runs
     launches = opt.info()["launches"] - launches0
     if graph is not None:
         launches = launches_per_graph * (args.steps // args.graph)
@@ -597,7 +598,7 @@ def main():
                 "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
                 "dependent_launch": int(opt.handle.get_option(B.NOVAK_OPT_DEPENDENT_LAUNCH)),
                 "record_uploads_in_timed_region": uploads,
-                "grid": info["grid"], "block": info["block"], "n_chunks": info["n_chunks"],
+                "grid": grid_timed, "block": info["block"], "n_chunks": info["n_chunks"],
                 "replicas": "each rank steps its own replica; no data-path collective",
             },
             "hbm_gbs": achieved,
