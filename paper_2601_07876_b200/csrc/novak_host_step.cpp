@@ -618,7 +618,7 @@ int novak_nesterov_extrapolate(novak_opt *o, void *const *d_params, void *d_save
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
     if ((rc = prepare_look(o, d_params, stream)) != NOVAK_OK) return rc;
     const cudaError_t e = novak::launch_extrapolate(
-        o->d_chunks, o->n_chunks, o->d_look, o->d_state, o->h.mom16, static_cast<float *>(d_save), static_cast<float>(o->h.beta_n), look_grid(o), stream);
+        o->d_chunks, o->n_chunks, o->d_look, o->d_state, o->h.mom16, static_cast<float *>(d_save), static_cast<float>(o->h.beta_n), look_grid(o), o->pdl, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "look-ahead kernel launch");
     o->extrapolated = true;
     o->look_save = d_save;
@@ -640,7 +640,7 @@ int novak_nesterov_restore(novak_opt *o, void *const *d_params, const void *d_sa
         return fail(o, NOVAK_EINVAL, "nesterov_restore: not the buffers novak_nesterov_extrapolate was given");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const cudaError_t e = novak::launch_restore(o->d_chunks, o->n_chunks, o->d_look,
-                                                static_cast<const float *>(d_save), look_grid(o), stream);
+                                                static_cast<const float *>(d_save), look_grid(o), o->pdl, stream);
     if (e != cudaSuccess) return fail_cuda(o, e, "restore kernel launch");
     o->extrapolated = false;
     o->look_save = nullptr;

@@ -110,10 +110,10 @@ struct __align__(16) LookRec {
 // first-moment region holds fp32, or bf16 when moments_bf16 is set.
 cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
                                const void *m_region, int moments_bf16, float *save_region,
-                               float beta_n, int grid, cudaStream_t stream);
+                               float beta_n, int grid, int pdl, cudaStream_t stream);
 // theta <- save (Section 5.8: restore the parameters after the closure).
 cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
-                           const float *save_region, int grid, cudaStream_t stream);
+                           const float *save_region, int grid, int pdl, cudaStream_t stream);
 
 // ---- graph-capturable step: the step counter and the scalar plan in device memory
 // One step's plan as the kernels and novak_get_info need it.

@@ -61,9 +61,16 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
                   const void *__restrict__ m_region, float *__restrict__ save_region, float beta_n)
 {
     constexpr int kMomBytes = M16 ? 2 : 4;
-    for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-        const Chunk ch = chunks[c];
-        const LookRec r = recs[ch.tensor];
+    // Programmatic dependent launch: CTAs become resident and read their first
+    // work-table entry (written by copies only) while the previous kernel on
+    // the stream drains; no tensor is touched before it has completed.
+    asm volatile("griddepcontrol.launch_dependents;");
+    int c = blockIdx.x;
+    if (c >= n_chunks) return;
+    Chunk ch = chunks[c];
+    LookRec r = recs[ch.tensor];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (;;) {
         float *p = r.p + ch.offset;
         float *sv = save_region + r.state_off + ch.offset;
         const void *m = RESTORE ? nullptr
@@ -122,35 +129,52 @@ novak_look_kernel(const Chunk *__restrict__ chunks, int n_chunks, const LookRec 
                 }
             }
         }
+        c += gridDim.x;
+        if (c >= n_chunks) break;
+        ch = chunks[c];
+        r = recs[ch.tensor];
     }
+}
+
+template <typename Kernel, typename... Args>
+cudaError_t launch_look(Kernel kernel, int grid, int pdl, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(grid));
+    lc.blockDim = dim3(kLookThreads);
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (pdl & 1) ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, kernel, args...);
 }
 
 }  // namespace
 
 cudaError_t launch_extrapolate(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
                                const void *m_region, int moments_bf16, float *save_region,
-                               float beta_n, int grid, cudaStream_t stream)
+                               float beta_n, int grid, int pdl, cudaStream_t stream)
 {
     if (n_chunks <= 0) return cudaSuccess;
     if (grid < 1 || grid > n_chunks) grid = n_chunks;
     if (moments_bf16)
-        novak_look_kernel<false, true><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs,
-                                                                          m_region, save_region, beta_n);
-    else
-        novak_look_kernel<false, false><<<grid, kLookThreads, 0, stream>>>(d_chunks, n_chunks, d_recs,
-                                                                           m_region, save_region, beta_n);
-    return cudaGetLastError();
+        return launch_look(novak_look_kernel<false, true>, grid, pdl, stream, d_chunks, n_chunks, d_recs,
+                           m_region, save_region, beta_n);
+    return launch_look(novak_look_kernel<false, false>, grid, pdl, stream, d_chunks, n_chunks, d_recs,
+                       m_region, save_region, beta_n);
 }
 
 cudaError_t launch_restore(const Chunk *d_chunks, int n_chunks, const LookRec *d_recs,
-                           const float *save_region, int grid, cudaStream_t stream)
+                           const float *save_region, int grid, int pdl, cudaStream_t stream)
 {
     if (n_chunks <= 0) return cudaSuccess;
     if (grid < 1 || grid > n_chunks) grid = n_chunks;
     // the kernel only reads the save buffer when restoring
-    novak_look_kernel<true, false><<<grid, kLookThreads, 0, stream>>>(
-        d_chunks, n_chunks, d_recs, nullptr, const_cast<float *>(save_region), 0.0f);
-    return cudaGetLastError();
+    const void *no_moments = nullptr;
+    return launch_look(novak_look_kernel<true, false>, grid, pdl, stream, d_chunks, n_chunks, d_recs,
+                       no_moments, const_cast<float *>(save_region), 0.0f);
 }
 
 }  // namespace novak
