@@ -142,7 +142,10 @@ enum {
                                      NOVAK_ESTATE for any other variant             */
     NOVAK_OPT_MOMENT_DTYPE = 22,  /* NOVAK_MOMENT_*: storage type of m and v; only
                                      before attach (default NOVAK_MOMENT_F32)          */
-    NOVAK_OPT_GRAPH_CAPTURABLE = 23, /* 1: novak_step may be captured into a CUDA graph
+    NOVAK_OPT_GRAPH_CAPTURABLE = 23, /* Without it every step entry point returns
+                                     NOVAK_ESTATE while its stream is being captured (a
+                                     replay would repeat ONE step's scalars).
+                                     1: novak_step may be captured into a CUDA graph
                                      (stream capture) and replayed: the step counter,
                                      the scalars of Eq. 3-9 / 18 and the lookahead
                                      action then live in device memory, advanced by a

@@ -43,6 +43,21 @@ int check_step_args(novak_opt *o, const char *who, void *const *d_params,
     return NOVAK_OK;
 }
 
+// The plain step passes the scalars of ONE step by value: captured into a CUDA
+// graph it would replay that step's scalars for ever.  Refuse instead.
+int refuse_capture(novak_opt *o, const char *who, cudaStream_t stream)
+{
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return NOVAK_OK;
+    }
+    if (st != cudaStreamCaptureStatusNone)
+        return fail(o, NOVAK_ESTATE, "%s: the stream is being captured; only a handle with "
+                    "NOVAK_OPT_GRAPH_CAPTURABLE may be captured into a CUDA graph", who);
+    return NOVAK_OK;
+}
+
 // What the graph-capturable step does not cover.
 int check_dyn(novak_opt *o, const char *who)
 {
@@ -255,6 +270,7 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     if (rc != NOVAK_OK) return rc;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (o->dyn && (rc = check_dyn(o, "step")) != NOVAK_OK) return rc;
+    if (!o->dyn && (rc = refuse_capture(o, "step", stream)) != NOVAK_OK) return rc;
     StepCtx ctx;
     if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
     cudaError_t e;
@@ -297,6 +313,7 @@ int novak_step_begin(novak_opt *o, void *const *d_params, const void *const *d_g
     if (o->dyn) return fail(o, NOVAK_ESTATE, "step_begin: not available with NOVAK_OPT_GRAPH_CAPTURABLE");
     if (o->half_open) return fail(o, NOVAK_ESTATE, "step_begin: the previous step was not finished");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if ((rc = refuse_capture(o, "step_begin", stream)) != NOVAK_OK) return rc;
     StepCtx ctx;
     if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
     if (ctx.pre == novak::PRE_CENTER || ctx.trust)
@@ -376,6 +393,7 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
         if (!h_params[i] || !h_grads[i] || !d_params[i] || !d_grads[i])
             return fail(o, NOVAK_EINVAL, "step_host: tensor %d has a NULL pointer", i);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if ((rc = refuse_capture(o, "step_host", stream)) != NOVAK_OK) return rc;
     const size_t gsz = grad_dtype == NOVAK_GRAD_BF16 ? 2 : 4;
 
     StepCtx ctx;
@@ -479,6 +497,10 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
         return fail(o, NOVAK_EINVAL, "step_noalloc: %d tensors exceed the static table's %d; "
                     "split the group or use novak_step", n, novak::kNoAllocMaxTensors);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    {
+        const int rc = refuse_capture(o, "step_noalloc", stream);
+        if (rc != NOVAK_OK) return rc;
+    }
 
     if (o->na_chunks.empty())
         build_chunks(o->numel.data(), o->phase.data(), o->n, o->chunk_elems, o->na_chunks);

@@ -106,6 +106,23 @@ def test_captured_once_and_replayed(extra):
         assert_close(p, oracle.theta[i], f"after the rate change theta[{i}]")
 
 
+def test_the_plain_step_refuses_to_be_captured():
+    """Its scalars are launch parameters: a replay would repeat one step for ever."""
+    params = _fresh([4096, 100])
+    g = [torch.zeros_like(p) for p in params]
+    opt = B.NovakOptimizer(params, **BASE)
+    opt.step(g)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with pytest.raises(B.NovakError) as e:
+        with torch.cuda.graph(graph):
+            opt.step(g)
+    assert e.value.status == B.NOVAK_ESTATE and "captured" in str(e.value)
+    torch.cuda.synchronize()
+    opt.step(g)                                  # the handle and the context are fine
+    assert opt.info()["t"] == 2
+
+
 def test_what_the_mode_does_not_cover_is_refused():
     params = _fresh([4096, 100])
     g = [torch.zeros_like(p) for p in params]
