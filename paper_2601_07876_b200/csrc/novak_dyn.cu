@@ -14,6 +14,9 @@ namespace novak {
 void *step_dyn_kernel_pre0(int nesterov, int grad_dtype);
 void *step_dyn_kernel_pre1(int nesterov, int grad_dtype);
 void *step_dyn_kernel_pre2(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre0_copy(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre1_copy(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre2_copy(int nesterov, int grad_dtype);
 
 namespace {
 
@@ -105,11 +108,14 @@ cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec
     case PRE_NONE: raw = step_dyn_kernel_pre0(nesterov, grad_dtype); break;
     case PRE_SCALE: raw = step_dyn_kernel_pre1(nesterov, grad_dtype); break;
     case PRE_CENTER: raw = step_dyn_kernel_pre2(nesterov, grad_dtype); break;
+    case PRE_NONE | PRE_COPY16: raw = step_dyn_kernel_pre0_copy(nesterov, grad_dtype); break;
+    case PRE_SCALE | PRE_COPY16: raw = step_dyn_kernel_pre1_copy(nesterov, grad_dtype); break;
+    case PRE_CENTER | PRE_COPY16: raw = step_dyn_kernel_pre2_copy(nesterov, grad_dtype); break;
     default: break;
     }
     StepDynFn fn = reinterpret_cast<StepDynFn>(raw);
     if (!fn || !d_plan || n_chunks <= 0 || cfg.grid <= 0) return cudaErrorInvalidValue;
-    if (cfg.pre != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
+    if ((cfg.pre & PRE_MASK) != PRE_NONE && prep == nullptr) return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(cfg.grid));
     lc.blockDim = dim3(NOVAK_BLOCK);

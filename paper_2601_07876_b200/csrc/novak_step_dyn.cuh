@@ -33,6 +33,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
         pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
+        pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
         float *p = r.p + ch.offset;
         void *m = static_cast<char *>(r.m) + ch.offset * 4;
         void *v = static_cast<char *>(r.v) + ch.offset * 4;
@@ -43,6 +44,8 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
                          reinterpret_cast<uintptr_t>(v);
         if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
         if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
+        // the 64-bit stores of the bf16 copy need half the parameters' alignment
+        if ((PRE & PRE_COPY16) != 0) bits |= reinterpret_cast<uintptr_t>(pre.copy) << 1;
         const bool aligned = (bits & 15u) == 0 &&
                              (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
         if (aligned) {
@@ -61,7 +64,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
     }
 }
 
-// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER (fp32 moments, no bf16 copy).  The
+// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16 (fp32 moments).  The
 // kernel holds every lookahead action's code; at four resident CTAs per SM (64
 // registers) it spills a little on the heavier actions, which costs less than
 // the lost CTA of the 80-register build when the gradient is pre-processed.

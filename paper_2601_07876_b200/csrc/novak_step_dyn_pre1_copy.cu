@@ -1,0 +1,12 @@
+// Graph-capturable step kernel instantiations, gradient pre-processing mode PRE_SCALE, storing a
+// bf16 copy of the updated parameters beside the fp32 ones.
+#include "novak_step_dyn.cuh"
+
+namespace novak {
+
+void *step_dyn_kernel_pre1_copy(int nesterov, int grad_dtype)
+{
+    return reinterpret_cast<void *>(pick_step_dyn_kernel<PRE_SCALE | PRE_COPY16>(nesterov, grad_dtype));
+}
+
+}  // namespace novak

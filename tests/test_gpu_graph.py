@@ -50,8 +50,11 @@ def test_eager_steps_match_the_oracle(nesterov, la, gdtype):
 
 
 @pytest.mark.parametrize("extra", [dict(), dict(clip_threshold=0.05, centralize=True),
-                                   dict(adaptive_beta=True, lookahead_mode="traj_mean")])
+                                   dict(adaptive_beta=True, lookahead_mode="traj_mean"),
+                                   dict(clip_threshold=0.05, copies=True)])
 def test_captured_once_and_replayed(extra):
+    extra = dict(extra)
+    with_copies = extra.pop("copies", False)
     shapes = [(64, 33), (1000,), (16, 3, 5, 5), (7,), (300, 40)]
     numels = [int(np.prod(s)) for s in shapes]
     params = _fresh(numels, shapes=shapes)
@@ -59,6 +62,10 @@ def test_captured_once_and_replayed(extra):
     rows = [s[0] if len(s) > 1 else 0 for s in shapes]
     oracle = O.Oracle(oracle_config(hyper), [to_f64(p) for p in params], rows=rows)
     opt = B.NovakOptimizer(params, **hyper, graph_capturable=True)
+    copies = None
+    if with_copies:                        # bf16 model copies written by the replayed steps
+        copies = make_tensors(numels, DEV, dtype=torch.bfloat16)[1]
+        opt.set_param_copies(copies)
     _, gviews, _ = make_tensors(numels, DEV)
     static = [v.view(s) for v, s in zip(gviews, shapes)]       # the captured gradient buffers
     gen = _gen(17)
@@ -90,6 +97,9 @@ def test_captured_once_and_replayed(extra):
         assert_close(st["m"], oracle.m[i], f"replayed m[{i}]")
         assert_close(st["v"], oracle.v[i], f"replayed v[{i}]")
         assert_close(st["slow"], oracle.slow[i], f"replayed slow[{i}]")
+    if copies is not None:
+        for p, c in zip(params, copies):
+            assert torch.equal(c.view(p.shape), p.to(torch.bfloat16))
     # a checkpoint taken now carries the device's counters
     assert opt.handle.export_meta().t == 13
     # the learning rate reaches the device at the next CALL; replays keep what they find
