@@ -68,8 +68,8 @@ __global__ void novak_plan_next_kernel(DevPlan *__restrict__ dp, novak_host::Hyp
     dp->t = t + 1;
 }
 
-using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const DevPlan *,
-                           int);
+using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const float *,
+                           const DevPlan *, int);
 
 }  // namespace
 
@@ -100,8 +100,9 @@ cudaError_t launch_plan_next(DevPlan *d_plan, const void *hyper, size_t hyper_by
 }
 
 cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                            const PrepOut *prep, const DevPlan *d_plan, int nesterov,
-                            int grad_dtype, const LaunchCfg &cfg, cudaStream_t stream)
+                            const PrepOut *prep, const float *trust, const DevPlan *d_plan,
+                            int nesterov, int grad_dtype, const LaunchCfg &cfg,
+                            cudaStream_t stream)
 {
     void *raw = nullptr;
     switch (cfg.pre) {
@@ -125,7 +126,7 @@ cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
-    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, d_plan, cfg.reverse);
+    return cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, trust, d_plan, cfg.reverse);
 }
 
 }  // namespace novak

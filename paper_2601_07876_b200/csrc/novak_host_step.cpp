@@ -61,9 +61,9 @@ int refuse_capture(novak_opt *o, const char *who, cudaStream_t stream)
 // What the graph-capturable step does not cover.
 int check_dyn(novak_opt *o, const char *who)
 {
-    if (o->h.layer_adapt || o->h.mom16 || (o->h.true_requested && o->h.true_steps > 0))
-        return fail(o, NOVAK_ESTATE, "%s: the graph-capturable step has no layer adaptation, bf16 moments "
-                    "or true Nesterov steps", who);
+    if (o->h.mom16 || (o->h.true_requested && o->h.true_steps > 0))
+        return fail(o, NOVAK_ESTATE, "%s: the graph-capturable step has no bf16 moments and no true "
+                    "Nesterov steps", who);
     return NOVAK_OK;
 }
 
@@ -119,7 +119,8 @@ cudaError_t launch_trust(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, 
     if (ctx.trust) {
         *what = "layer adaptation kernel launch";
         e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
-                                      o->prep_out, ctx.s, kernel_variant(ctx.plan), ctx.grad_dtype,
+                                      o->prep_out, ctx.s, o->dyn ? o->d_plan : nullptr,
+                                      kernel_variant(ctx.plan), ctx.grad_dtype,
                                       ctx.pre | (o->h.mom16 ? novak::PRE_MOM16 : 0),
                                       o->chunk_u2, o->chunk_p2, o->trust, o->pdl, stream);
         if (e != cudaSuccess) return e;
@@ -285,11 +286,11 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
         novak::LaunchCfg cfg;
         cfg.grid = o->n_chunks;
         if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
-        cfg.reverse = ctx.pre != novak::PRE_NONE ? 1 : 0;      // serpentine needs t: not here
+        cfg.reverse = (ctx.pre != novak::PRE_NONE || ctx.trust) ? 1 : 0;   // serpentine needs t: not here
         cfg.pdl = o->pdl;
         cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16);
         o->last_grid = cfg.grid;
-        if ((e = novak::launch_step_dyn(o->d_chunks, o->n_chunks, ctx.d_recs, o->prep_out, o->d_plan,
+        if ((e = novak::launch_step_dyn(o->d_chunks, o->n_chunks, ctx.d_recs, o->prep_out, ctx.trust, o->d_plan,
                                         o->h.nesterov, grad_dtype, cfg, stream)) != cudaSuccess)
             return fail_cuda(o, e, "step kernel launch");
         // behind it: the next step's plan, computed while this step runs

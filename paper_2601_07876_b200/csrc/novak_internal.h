@@ -28,17 +28,20 @@ cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_
                         const PrepOut *prep, const float *trust, const StepScalars &s, int nesterov,
                         int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream);
 
+struct DevPlan;
+
 // Layer-wise adaptation (Eq. 19 / 25), two kernels over the whole chunk table:
 // per entry the sums of squares of theta_t and of this step's base direction
 // u_t (moments advanced in registers, nothing stored) into chunk_p2 / chunk_u2
 // (n_chunks doubles each), then one CTA per tensor adds its entries
 // [tensor_first[i], tensor_first[i+1]) in order and writes
-// trust[i] = clip(||theta|| / ||u||, 0.1, 10), 1 where ||u|| = 0.
+// trust[i] = clip(||theta|| / ||u||, 0.1, 10), 1 where ||u|| = 0.  With d_plan
+// (graph-capturable step) the scalars come from its armed slot instead of s.
 cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
                                int n_tensors, const int *tensor_first, const PrepOut *prep,
-                               const StepScalars &s, int nesterov, int grad_dtype, int pre,
-                               double *chunk_u2, double *chunk_p2, float *trust, int pdl,
-                               cudaStream_t stream);
+                               const StepScalars &s, const DevPlan *d_plan, int nesterov,
+                               int grad_dtype, int pre, double *chunk_u2, double *chunk_p2,
+                               float *trust, int pdl, cudaStream_t stream);
 
 // One unit of work of the statistics pass for a tensor with rows (Eq. 26).
 // Rows of up to kRowWarpMax elements: n_rows (a multiple of 8 but for a tensor's
@@ -150,8 +153,9 @@ cudaError_t launch_plan_next(DevPlan *d_plan, const void *hyper, size_t hyper_by
 // cfg.pre: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16;
 // cudaErrorInvalidValue otherwise.
 cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
-                            const PrepOut *prep, const DevPlan *d_plan, int nesterov,
-                            int grad_dtype, const LaunchCfg &cfg, cudaStream_t stream);
+                            const PrepOut *prep, const float *trust, const DevPlan *d_plan,
+                            int nesterov, int grad_dtype, const LaunchCfg &cfg,
+                            cudaStream_t stream);
 
 // ---- work table for callers that cannot allocate device memory --------------
 // Capacity of the statically allocated table behind novak_step_noalloc.

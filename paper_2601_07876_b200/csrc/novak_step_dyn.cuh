@@ -21,6 +21,7 @@ namespace {
 template <int NEST, int GT, int LA, int PRE>
 __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, int n_chunks,
                                             const TensorRec *__restrict__ recs, const PreArgs &pre0,
+                                            const float *__restrict__ trust,
                                             const StepScalars &s, int reverse, int c, Chunk ch,
                                             TensorRec r)
 {
@@ -30,6 +31,8 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
     PreArgs pre = pre0;
 #pragma unroll 1
     for (;;) {
+        // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
+        pre.step = trust != nullptr ? pre0.step * __ldg(trust + ch.tensor) : pre0.step;
         pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
@@ -72,7 +75,7 @@ template <int NEST, int GT, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_DYN_MIN_CTAS)
 novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                       const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                      const DevPlan *__restrict__ plan, int reverse)
+                      const float *__restrict__ trust, const DevPlan *__restrict__ plan, int reverse)
 {
     const int c = blockIdx.x;
     if (c >= n_chunks) return;
@@ -96,7 +99,7 @@ novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
     switch (la) {
 #define NOVAK_DYN_CASE(X) \
-    case (X): dyn_entries<NEST, GT, (X), PRE>(chunks, n_chunks, recs, pre, s, reverse, c, ch, r); break;
+    case (X): dyn_entries<NEST, GT, (X), PRE>(chunks, n_chunks, recs, pre, trust, s, reverse, c, ch, r); break;
         NOVAK_DYN_CASE(LA_NONE)
         NOVAK_DYN_CASE(LA_S_INIT | LA_S_WRITE)
         NOVAK_DYN_CASE(LA_S_INIT | LA_S_WRITE | LA_SYNC)
@@ -110,8 +113,8 @@ novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     }
 }
 
-using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const DevPlan *,
-                           int);
+using StepDynFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, const float *,
+                           const DevPlan *, int);
 
 template <int PRE>
 StepDynFn pick_step_dyn_kernel(int nesterov, int grad_dtype)

@@ -68,8 +68,8 @@ template <int NEST, int GT, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK)
 novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                          const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                         const StepScalars s, double *__restrict__ chunk_u2,
-                         double *__restrict__ chunk_p2)
+                         const StepScalars s_host, const DevPlan *__restrict__ plan,
+                         double *__restrict__ chunk_u2, double *__restrict__ chunk_p2)
 {
     __shared__ double sh[kTrustWarps];
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
@@ -81,6 +81,8 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     const Chunk ch = chunks[c];
     const TensorRec r = recs[ch.tensor];
     grid_dependency_wait();              // parameters, moments, clip factor, row means
+    // the graph-capturable step keeps this step's scalars in device memory
+    const StepScalars s = plan != nullptr ? plan->slot[plan->t & 1].s : s_host;
 
     PreArgs pre;
     pre.copy = nullptr;
@@ -150,7 +152,7 @@ novak_trust_finish_kernel(const int *__restrict__ tensor_first,
 }
 
 using TrustFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, StepScalars,
-                         double *, double *);
+                         const DevPlan *, double *, double *);
 
 template <int NEST, int GT>
 TrustFn pick_pre(int pre)
@@ -205,9 +207,9 @@ void fill_config(cudaLaunchConfig_t *lc, cudaLaunchAttribute *attr, unsigned gri
 
 cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
                                int n_tensors, const int *tensor_first, const PrepOut *prep,
-                               const StepScalars &s, int nesterov, int grad_dtype, int pre,
-                               double *chunk_u2, double *chunk_p2, float *trust, int pdl,
-                               cudaStream_t stream)
+                               const StepScalars &s, const DevPlan *d_plan, int nesterov,
+                               int grad_dtype, int pre, double *chunk_u2, double *chunk_p2,
+                               float *trust, int pdl, cudaStream_t stream)
 {
     TrustFn fn = pick_trust(nesterov, grad_dtype, pre);
     if (!fn || n_chunks <= 0 || n_tensors <= 0 || !tensor_first || !chunk_u2 || !chunk_p2 || !trust)
@@ -216,7 +218,7 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[1];
     fill_config(&lc, attr, static_cast<unsigned>(n_chunks), (pdl & 2) != 0, stream);
-    cudaError_t e = cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, s, chunk_u2, chunk_p2);
+    cudaError_t e = cudaLaunchKernelEx(&lc, fn, d_chunks, n_chunks, d_recs, prep, s, d_plan, chunk_u2, chunk_p2);
     if (e != cudaSuccess) return e;
     fill_config(&lc, attr, static_cast<unsigned>(n_tensors), (pdl & 4) != 0, stream);
     const double *u2 = chunk_u2, *p2 = chunk_p2;

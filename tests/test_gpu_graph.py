@@ -51,7 +51,8 @@ def test_eager_steps_match_the_oracle(nesterov, la, gdtype):
 
 @pytest.mark.parametrize("extra", [dict(), dict(clip_threshold=0.05, centralize=True),
                                    dict(adaptive_beta=True, lookahead_mode="traj_mean"),
-                                   dict(clip_threshold=0.05, copies=True)])
+                                   dict(clip_threshold=0.05, copies=True),
+                                   dict(layer_adaptation=True, clip_threshold=0.05, centralize=True)])
 def test_captured_once_and_replayed(extra):
     extra = dict(extra)
     with_copies = extra.pop("copies", False)
@@ -136,7 +137,7 @@ def test_the_plain_step_refuses_to_be_captured():
 def test_what_the_mode_does_not_cover_is_refused():
     params = _fresh([4096, 100])
     g = [torch.zeros_like(p) for p in params]
-    for kw in (dict(layer_adaptation=True), dict(moment_dtype="bf16"),
+    for kw in (dict(moment_dtype="bf16"),
                dict(nesterov="true", true_nesterov_steps=3)):
         opt = B.NovakOptimizer(params, **dict(BASE, **kw), graph_capturable=True)
         with pytest.raises(B.NovakError) as e:
