@@ -20,12 +20,19 @@
  *     lookahead on steps with t mod k == 0                 (Eq. 28-31)
  * The per-step scalars (1-beta^t, rho_t, the branch of Eq. 8, r_t, the decay
  * factor, the sync flag) are computed once per step on the host in double
- * precision and passed to the kernel by value.
+ * precision and passed to the kernel by value (with NOVAK_OPT_GRAPH_CAPTURABLE:
+ * by the same code in a one-thread kernel, from a counter in device memory).
+ * Around that step, each behind an option and off by default: gradient clipping
+ * and centralization (phase 2), adaptive beta (phase 3), layer adaptation and
+ * automatic learning-rate scaling (phase 7), the sparse mask (phase 8), bf16
+ * parameter copies, bf16 moment storage, the two parameter passes of true
+ * Nesterov momentum, a step in two halves for sharded groups.
  *
  * Threading: a handle is not thread safe; use one handle per host thread.
  * Streams: all work of a handle must be issued on one stream (or on streams
  * the caller orders itself): the device work table is updated in stream order.
- * No call synchronises the device.  Pointers named d_* are device pointers,
+ * No call synchronises the device unless its description says so (the calls
+ * that read a result back).  Pointers named d_* are device pointers,
  * h_* host pointers; "host array of device pointers" means the array lives in
  * host memory and its entries point to device memory.
  */
