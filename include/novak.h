@@ -168,8 +168,8 @@ enum {
                                      hyperparameters are part of a captured launch.
                                      novak_get_info and novak_export_meta read the
                                      counters back and SYNCHRONISE the device in this
-                                     mode.  Not covered (NOVAK_ESTATE): bf16
-                                     moments, true Nesterov steps, novak_step_begin / _host /
+                                     mode.  Not covered (NOVAK_ESTATE): true
+                                     Nesterov steps, novak_step_begin / _host /
                                      _noalloc; NOVAK_OPT_SERPENTINE is ignored.  Only
                                      before the first step.  0 (default)              */
     NOVAK_OPT_SPARSE_THRESHOLD = 18 /* tau >= 0 of the sparse updates (Eq. 27): base

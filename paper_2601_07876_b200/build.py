@@ -23,7 +23,10 @@ SOURCES = [os.path.join(CSRC, f) for f in (
     "novak_step_pre0_copy_mom16.cu", "novak_step_pre1_copy_mom16.cu",
     "novak_step_pre2_copy_mom16.cu",
     "novak_dyn.cu", "novak_step_dyn_pre0.cu", "novak_step_dyn_pre1.cu", "novak_step_dyn_pre2.cu",
-    "novak_step_dyn_pre0_copy.cu", "novak_step_dyn_pre1_copy.cu", "novak_step_dyn_pre2_copy.cu")]
+    "novak_step_dyn_pre0_copy.cu", "novak_step_dyn_pre1_copy.cu", "novak_step_dyn_pre2_copy.cu",
+    "novak_step_dyn_pre0_mom16.cu", "novak_step_dyn_pre1_mom16.cu", "novak_step_dyn_pre2_mom16.cu",
+    "novak_step_dyn_pre0_copy_mom16.cu", "novak_step_dyn_pre1_copy_mom16.cu",
+    "novak_step_dyn_pre2_copy_mom16.cu")]
 HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(CSRC, "novak_handle.h"), os.path.join(CSRC, "novak_plan.h"),
            os.path.join(CSRC, "novak_step_types.h"),
            os.path.join(CSRC, "novak_step_kernel.cuh"), os.path.join(CSRC, "novak_step_dyn.cuh"),

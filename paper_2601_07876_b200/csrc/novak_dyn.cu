@@ -17,6 +17,12 @@ void *step_dyn_kernel_pre2(int nesterov, int grad_dtype);
 void *step_dyn_kernel_pre0_copy(int nesterov, int grad_dtype);
 void *step_dyn_kernel_pre1_copy(int nesterov, int grad_dtype);
 void *step_dyn_kernel_pre2_copy(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre0_mom16(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre0_copy_mom16(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre1_mom16(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre1_copy_mom16(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre2_mom16(int nesterov, int grad_dtype);
+void *step_dyn_kernel_pre2_copy_mom16(int nesterov, int grad_dtype);
 
 namespace {
 
@@ -112,6 +118,12 @@ cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec
     case PRE_NONE | PRE_COPY16: raw = step_dyn_kernel_pre0_copy(nesterov, grad_dtype); break;
     case PRE_SCALE | PRE_COPY16: raw = step_dyn_kernel_pre1_copy(nesterov, grad_dtype); break;
     case PRE_CENTER | PRE_COPY16: raw = step_dyn_kernel_pre2_copy(nesterov, grad_dtype); break;
+    case PRE_NONE | PRE_MOM16: raw = step_dyn_kernel_pre0_mom16(nesterov, grad_dtype); break;
+    case PRE_NONE | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre0_copy_mom16(nesterov, grad_dtype); break;
+    case PRE_SCALE | PRE_MOM16: raw = step_dyn_kernel_pre1_mom16(nesterov, grad_dtype); break;
+    case PRE_SCALE | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre1_copy_mom16(nesterov, grad_dtype); break;
+    case PRE_CENTER | PRE_MOM16: raw = step_dyn_kernel_pre2_mom16(nesterov, grad_dtype); break;
+    case PRE_CENTER | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre2_copy_mom16(nesterov, grad_dtype); break;
     default: break;
     }
     StepDynFn fn = reinterpret_cast<StepDynFn>(raw);

@@ -61,9 +61,9 @@ int refuse_capture(novak_opt *o, const char *who, cudaStream_t stream)
 // What the graph-capturable step does not cover.
 int check_dyn(novak_opt *o, const char *who)
 {
-    if (o->h.mom16 || (o->h.true_requested && o->h.true_steps > 0))
-        return fail(o, NOVAK_ESTATE, "%s: the graph-capturable step has no bf16 moments and no true "
-                    "Nesterov steps", who);
+    if (o->h.true_requested && o->h.true_steps > 0)
+        return fail(o, NOVAK_ESTATE, "%s: the graph-capturable step has no true Nesterov steps (the "
+                    "closure is the caller's)", who);
     return NOVAK_OK;
 }
 
@@ -288,7 +288,8 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
         if (o->ctas_per_sm > 0) cfg.grid = std::min(o->n_chunks, o->sms * o->ctas_per_sm);
         cfg.reverse = (ctx.pre != novak::PRE_NONE || ctx.trust) ? 1 : 0;   // serpentine needs t: not here
         cfg.pdl = o->pdl;
-        cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16);
+        cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16) |
+                  (o->h.mom16 ? novak::PRE_MOM16 : 0);
         o->last_grid = cfg.grid;
         if ((e = novak::launch_step_dyn(o->d_chunks, o->n_chunks, ctx.d_recs, o->prep_out, ctx.trust, o->d_plan,
                                         o->h.nesterov, grad_dtype, cfg, stream)) != cudaSuccess)

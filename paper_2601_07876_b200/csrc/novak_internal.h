@@ -150,8 +150,8 @@ cudaError_t launch_plan_arm(DevPlan *d_plan, const void *hyper, size_t hyper_byt
 cudaError_t launch_plan_next(DevPlan *d_plan, const void *hyper, size_t hyper_bytes, int pdl,
                              cudaStream_t stream);
 // The step kernel that takes its scalars and lookahead action from the armed slot.
-// cfg.pre: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16;
-// cudaErrorInvalidValue otherwise.
+// cfg.pre: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16 and
+// PRE_MOM16; cudaErrorInvalidValue otherwise.
 cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,
                             const PrepOut *prep, const float *trust, const DevPlan *d_plan,
                             int nesterov, int grad_dtype, const LaunchCfg &cfg,

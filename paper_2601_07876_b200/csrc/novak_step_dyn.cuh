@@ -26,6 +26,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
                                             TensorRec r)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
     constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
     PreArgs pre = pre0;
@@ -38,13 +39,15 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
         pre.elem0 = static_cast<uint32_t>(ch.offset);
         pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
         float *p = r.p + ch.offset;
-        void *m = static_cast<char *>(r.m) + ch.offset * 4;
-        void *v = static_cast<char *>(r.v) + ch.offset * 4;
+        void *m = static_cast<char *>(r.m) + ch.offset * kMomBytes;
+        void *v = static_cast<char *>(r.v) + ch.offset * kMomBytes;
         float *slow = kUseS ? r.slow + ch.offset : nullptr;
         float *acc = kUseA ? r.acc + ch.offset : nullptr;
         const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
-        uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(m) |
-                         reinterpret_cast<uintptr_t>(v);
+        // four bf16 moments are one 64-bit access: half the parameters' alignment
+        uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
+                         ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
+                          << (kMomBytes == 2 ? 1 : 0));
         if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
         if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
         // the 64-bit stores of the bf16 copy need half the parameters' alignment
@@ -67,7 +70,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
     }
 }
 
-// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16 (fp32 moments).  The
+// PRE: PRE_NONE, PRE_SCALE or PRE_CENTER, with or without PRE_COPY16 and PRE_MOM16.  The
 // kernel holds every lookahead action's code; at four resident CTAs per SM (64
 // registers) it spills a little on the heavier actions, which costs less than
 // the lost CTA of the 80-register build when the gradient is pre-processed.
