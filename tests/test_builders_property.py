@@ -110,3 +110,20 @@ def test_planner_agrees_with_the_oracle_for_any_hyperparameters(beta1, beta2, lr
         assert abs(a.step_size - b.step_size) <= 1e-7 * b.step_size
     else:
         assert a.r_t == 1.0 == b.r_t and abs(a.step_size - b.step_size) <= 1e-12 * b.step_size
+
+
+@settings(max_examples=300, deadline=None)
+@given(bits=st.lists(st.integers(0, 2 ** 32 - 1), min_size=1, max_size=64))
+def test_oracle_bf16_rounding_equals_the_library_conversion_on_any_bit_pattern(bits):
+    """Every finite fp32 bit pattern (subnormals, ties, values next to overflow): the
+    oracle's nearest-even bfloat16 rounding against torch's fp32 -> bfloat16 conversion."""
+    import torch
+    from oracle import novak_oracle as O
+    lib = O.default_library()
+    x = np.array(bits, dtype=np.uint32).view(np.float32)
+    x = x[np.isfinite(x)]
+    if x.size == 0:
+        return
+    want = torch.from_numpy(x.copy()).to(torch.bfloat16).to(torch.float64).numpy()
+    got = np.array([lib.novak_oracle_round_bf16(float(v)) for v in x])
+    assert np.array_equal(got, want) and np.array_equal(np.signbit(got), np.signbit(want))
