@@ -234,8 +234,6 @@ def run_reference(args, rank):
     import torch
     from oracle import novak_oracle as O
     from paper_2601_07876_b200 import workloads as W
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from harness import oracle_config
 
     wl = W.get_workload(args.config)
     hyper = dict(wl.hyper, lookahead_mode=args.lookahead_mode)
@@ -243,7 +241,7 @@ def run_reference(args, rank):
     rng = np.random.default_rng(W.MASTER_SEED)
 
     def make(n):
-        o = O.Oracle(oracle_config(hyper), [rng.normal(0, 0.05, n)])
+        o = O.Oracle(O.Config.from_hyper(hyper), [rng.normal(0, 0.05, n)])
         g = rng.normal(0, 1e-3, n).astype(np.float32).astype(np.float64)
         return o, g
 
@@ -284,12 +282,10 @@ def cpu_baseline(wl, hyper, seconds):
     """Oracle on the host cores for about `seconds` of work on a bounded sample."""
     import numpy as np
     from oracle import novak_oracle as O
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
-    from harness import oracle_config
     cores = len(os.sched_getaffinity(0))
     n = min(wl.total, 1 << 24)
     rng = np.random.default_rng(1)
-    o = O.Oracle(oracle_config(hyper), [rng.normal(0, 0.05, n)])
+    o = O.Oracle(O.Config.from_hyper(hyper), [rng.normal(0, 0.05, n)])
     g = rng.normal(0, 1e-3, n).astype(np.float32).astype(np.float64)
     o.step([g], threads=cores)
     steps, t0 = 0, time.perf_counter()

@@ -388,7 +388,11 @@ int novak_step_host(novak_opt *opt, void *const *h_params,
  * reads whenever another handle used the table in between or this handle's
  * pointers changed (nothing in it needs to start from zero).  Two calls that
  * may overlap on the GPU (different streams, no ordering between them) race on
- * the table: order them yourself.
+ * the table: order them yourself.  On the HOST the call may be made from several
+ * threads at once, each with a handle of its own: the library keeps track of
+ * whose records the table holds under one process-wide lock that covers the
+ * upload and the launch, so a kernel is always enqueued behind its own handle's
+ * records.  NOVAK_OPT_CTAS_PER_SM caps the grid as in novak_step.
  *
  * The first call on each device looks up the array's device address (with that
  * device current); make that first call outside any stream capture.

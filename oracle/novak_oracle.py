@@ -159,6 +159,34 @@ class Config:
     true_steps: int = 0                  # N_taylor of the true variant (Section 5.2)
     moment_bf16: bool = False            # m, v stored rounded to bfloat16
 
+    @classmethod
+    def from_hyper(cls, hyper: dict) -> "Config":
+        """From the keyword spelling the workloads and tests use (``betas=(b1, b2)``,
+        ``nesterov="approximation"``, ``lookahead_mode="last"``, ``moment_dtype="bf16"`` ...);
+        absent keys take the defaults of the benchmark configurations; keys that only
+        concern an implementation's launch (chunk sizes and the like) are ignored."""
+        h = dict(hyper)
+        b1, b2 = h.pop("betas", (0.9, 0.999))
+        nest = {"none": NESTEROV_NONE, "approximation": NESTEROV_APPROX,
+                "classical": NESTEROV_CLASSICAL, "true": NESTEROV_TRUE}
+        mode = {"last": LOOKAHEAD_LAST, "traj_mean": LOOKAHEAD_TRAJ_MEAN}
+        return cls(
+            lr=h.pop("lr", 1e-3), beta1=b1, beta2=b2, eps=h.pop("eps", 1e-8),
+            weight_decay=h.pop("weight_decay", 1e-2),
+            nesterov_variant=nest[h.pop("nesterov", "approximation")],
+            lookahead_k=h.pop("lookahead_k", 5), lookahead_alpha=h.pop("lookahead_alpha", 0.5),
+            nesterov_beta=h.pop("nesterov_beta", None),
+            lookahead_mode=mode[h.pop("lookahead_mode", "last")],
+            rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1),
+            clip_threshold=h.pop("clip_threshold", 0.0), centralize=h.pop("centralize", False),
+            layer_adaptation=h.pop("layer_adaptation", False),
+            sparse_threshold=h.pop("sparse_threshold", 0.0),
+            auto_lr=h.pop("auto_lr", False), auto_lr_gamma=h.pop("auto_lr_gamma", None) or 0.1,
+            adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
+            tau2=h.pop("tau2", None) or 5000.0,
+            true_steps=h.pop("true_nesterov_steps", 0),
+            moment_bf16=h.pop("moment_dtype", "f32") == "bf16")
+
     def to_c(self) -> HParams:
         nb = self.beta1 if self.nesterov_beta is None else self.nesterov_beta
         return HParams(self.lr, self.beta1, self.beta2, self.eps,

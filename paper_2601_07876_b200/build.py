@@ -14,19 +14,19 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libnovak.so")
-SOURCES = [os.path.join(CSRC, f) for f in (
-    "novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu",
-    "novak_grad_stats.cu", "novak_trust_stats.cu", "novak_nesterov.cu",
-    "novak_step_pre0.cu", "novak_step_pre1.cu", "novak_step_pre2.cu",
-    "novak_step_pre0_copy.cu", "novak_step_pre1_copy.cu", "novak_step_pre2_copy.cu",
-    "novak_step_pre0_mom16.cu", "novak_step_pre1_mom16.cu", "novak_step_pre2_mom16.cu",
-    "novak_step_pre0_copy_mom16.cu", "novak_step_pre1_copy_mom16.cu",
-    "novak_step_pre2_copy_mom16.cu",
-    "novak_dyn.cu", "novak_step_dyn_pre0.cu", "novak_step_dyn_pre1.cu", "novak_step_dyn_pre2.cu",
-    "novak_step_dyn_pre0_copy.cu", "novak_step_dyn_pre1_copy.cu", "novak_step_dyn_pre2_copy.cu",
-    "novak_step_dyn_pre0_mom16.cu", "novak_step_dyn_pre1_mom16.cu", "novak_step_dyn_pre2_mom16.cu",
-    "novak_step_dyn_pre0_copy_mom16.cu", "novak_step_dyn_pre1_copy_mom16.cu",
-    "novak_step_dyn_pre2_copy_mom16.cu")]
+# Gradient pre-processing modes of the step kernel (PRE_NONE / PRE_SCALE / PRE_CENTER,
+# | 4 with a bf16 parameter copy, | 8 with bf16 moments): novak_step_inst.cu is compiled
+# once per mode, and once more per mode for the graph-capturable kernel.
+PRE_MODES = (0, 1, 2, 4, 5, 6, 8, 9, 10, 12, 13, 14)
+PLAIN_SOURCES = ("novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu",
+                 "novak_grad_stats.cu", "novak_trust_stats.cu", "novak_nesterov.cu", "novak_dyn.cu")
+# (source, object name, extra flags)
+UNITS = [(os.path.join(CSRC, f), f + ".o", []) for f in PLAIN_SOURCES]
+UNITS += [(os.path.join(CSRC, "novak_step_inst.cu"), f"novak_step_mode{m}.o",
+           [f"-DNOVAK_PRE_MODE={m}"]) for m in PRE_MODES]
+UNITS += [(os.path.join(CSRC, "novak_step_inst.cu"), f"novak_step_dyn_mode{m}.o",
+           [f"-DNOVAK_PRE_MODE={m}", "-DNOVAK_INST_DYN"]) for m in PRE_MODES]
+SOURCES = sorted({u[0] for u in UNITS})
 HEADERS = [os.path.join(CSRC, "novak_internal.h"), os.path.join(CSRC, "novak_handle.h"), os.path.join(CSRC, "novak_plan.h"),
            os.path.join(CSRC, "novak_step_types.h"),
            os.path.join(CSRC, "novak_step_kernel.cuh"), os.path.join(CSRC, "novak_step_dyn.cuh"),
@@ -70,14 +70,15 @@ def build(force: bool = False, verbose: bool = False, extra: list[str] | None = 
         return LIB
     flags = (["-Xptxas", "-v"] if verbose else []) + (extra or [])
     with tempfile.TemporaryDirectory(prefix="novak_build_") as tmpdir:
-        objs = [os.path.join(tmpdir, os.path.basename(s) + ".o") for s in SOURCES]
+        objs = [os.path.join(tmpdir, u[1]) for u in UNITS]
 
         def one(pair):
-            return subprocess.run(compile_command(pair[0], pair[1], flags),
+            unit, obj = pair
+            return subprocess.run(compile_command(unit[0], obj, flags + unit[2]),
                                   capture_output=True, text=True)
 
-        with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
-            results = list(pool.map(one, zip(SOURCES, objs)))
+        with ThreadPoolExecutor(max_workers=len(UNITS)) as pool:
+            results = list(pool.map(one, zip(UNITS, objs)))
         failed = [r for r in results if r.returncode != 0]
         if verbose or failed:
             for r in results:

@@ -11,18 +11,12 @@
 
 namespace novak {
 
-void *step_dyn_kernel_pre0(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre1(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre2(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre0_copy(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre1_copy(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre2_copy(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre0_mom16(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre0_copy_mom16(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre1_mom16(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre1_copy_mom16(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre2_mom16(int nesterov, int grad_dtype);
-void *step_dyn_kernel_pre2_copy_mom16(int nesterov, int grad_dtype);
+// novak_step_inst.cu, compiled once per gradient pre-processing mode with
+// -DNOVAK_INST_DYN, holds the kernels; mode N exports step_dyn_kernel_mode<N>.
+#define NOVAK_FOR_EACH_PRE_MODE(X) X(0) X(1) X(2) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(13) X(14)
+#define NOVAK_DECLARE(N) void *step_dyn_kernel_mode##N(int nesterov, int grad_dtype);
+NOVAK_FOR_EACH_PRE_MODE(NOVAK_DECLARE)
+#undef NOVAK_DECLARE
 
 namespace {
 
@@ -112,18 +106,9 @@ cudaError_t launch_step_dyn(const Chunk *d_chunks, int n_chunks, const TensorRec
 {
     void *raw = nullptr;
     switch (cfg.pre) {
-    case PRE_NONE: raw = step_dyn_kernel_pre0(nesterov, grad_dtype); break;
-    case PRE_SCALE: raw = step_dyn_kernel_pre1(nesterov, grad_dtype); break;
-    case PRE_CENTER: raw = step_dyn_kernel_pre2(nesterov, grad_dtype); break;
-    case PRE_NONE | PRE_COPY16: raw = step_dyn_kernel_pre0_copy(nesterov, grad_dtype); break;
-    case PRE_SCALE | PRE_COPY16: raw = step_dyn_kernel_pre1_copy(nesterov, grad_dtype); break;
-    case PRE_CENTER | PRE_COPY16: raw = step_dyn_kernel_pre2_copy(nesterov, grad_dtype); break;
-    case PRE_NONE | PRE_MOM16: raw = step_dyn_kernel_pre0_mom16(nesterov, grad_dtype); break;
-    case PRE_NONE | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre0_copy_mom16(nesterov, grad_dtype); break;
-    case PRE_SCALE | PRE_MOM16: raw = step_dyn_kernel_pre1_mom16(nesterov, grad_dtype); break;
-    case PRE_SCALE | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre1_copy_mom16(nesterov, grad_dtype); break;
-    case PRE_CENTER | PRE_MOM16: raw = step_dyn_kernel_pre2_mom16(nesterov, grad_dtype); break;
-    case PRE_CENTER | PRE_COPY16 | PRE_MOM16: raw = step_dyn_kernel_pre2_copy_mom16(nesterov, grad_dtype); break;
+#define NOVAK_CASE(N) case N: raw = step_dyn_kernel_mode##N(nesterov, grad_dtype); break;
+        NOVAK_FOR_EACH_PRE_MODE(NOVAK_CASE)
+#undef NOVAK_CASE
     default: break;
     }
     StepDynFn fn = reinterpret_cast<StepDynFn>(raw);

@@ -496,8 +496,7 @@ __device__ __forceinline__ void write_scalars(PrepOut *out, double sumsq, double
 // For a group that is sharded over several processes: the sums of squares of
 // the WHOLE group (this process's local_sums, all-reduced by the caller) turned
 // into norm, clip factor and Eq. 20-22.  One thread.
-__global__ void novak_grad_norm_scalar_kernel(PrepOut *__restrict__ out,
-                                              const double *__restrict__ totals, double c_clip,
+__global__ void novak_grad_norm_scalar_kernel(PrepOut *out, const double *totals, double c_clip,
                                               double auto_gamma, int has_p)
 {
     grid_dependency_release();
@@ -511,14 +510,14 @@ __global__ void novak_grad_norm_scalar_kernel(PrepOut *__restrict__ out,
 // slice adds the slices in order) and adds up the sums of squares: per CTA
 // first, then the CTA that takes the last ticket adds the CTAs' sums in index
 // order and writes the norm, the clip factor and, when asked, Eq. 20-22.
+// The sums it reads are written by kernels that may still run while this grid
+// is resident (dependent launch): they are not declared read-only.
 __global__ void __launch_bounds__(kStatsBlock)
 novak_grad_stats_finish_kernel(const RowUnit *__restrict__ units, int n_units,
                                const TensorRec *__restrict__ recs, int n_work,
-                               const double *__restrict__ part_sq,
-                               const double *__restrict__ part_sum, int n_chunks,
-                               const double *__restrict__ chunk_psq, double c_clip,
-                               double auto_gamma, int finalize, double *__restrict__ cta_sq,
-                               PrepOut *__restrict__ out)
+                               const double *part_sq, const double *part_sum, int n_chunks,
+                               const double *chunk_psq, double c_clip,
+                               double auto_gamma, int finalize, double *cta_sq, PrepOut *out)
 {
     __shared__ double sh[kStatsWarps];
     __shared__ unsigned sh_last;

@@ -8,6 +8,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 using namespace novak_host;
@@ -310,6 +311,7 @@ int novak_step_begin(novak_opt *o, void *const *d_params, const void *const *d_g
 {
     static_assert(sizeof(StepCtx) <= sizeof(o->half_ctx), "room for the open step");
     if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
     int rc = check_step_args(o, "step_begin", d_params, d_grads, numel, n, grad_dtype);
     if (rc != NOVAK_OK) return rc;
     if (o->dyn) return fail(o, NOVAK_ESTATE, "step_begin: not available with NOVAK_OPT_GRAPH_CAPTURABLE");
@@ -472,6 +474,12 @@ int novak_step_host(novak_opt *o, void *const *h_params, const void *const *h_gr
 // ---------------------------------------------------------------------------
 namespace {
 // Which upload the shared table of each device currently holds (0 = none).
+// Every handle of the process shares the table, so the bookkeeping and the
+// sequence "compare owner -> upload -> take token -> launch" run under one
+// lock: host threads with a handle each may call at the same time, and a
+// launch then always finds the records its own handle uploaded last (given
+// that the caller orders the GPU work, e.g. by using one stream).
+std::mutex g_noalloc_mutex;
 uint64_t g_noalloc_owner[64] = {};
 uint64_t g_noalloc_next_token = 1;
 }  // namespace
@@ -556,6 +564,11 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     int dev = 0;
     cudaError_t e;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return fail_cuda(o, e, "cudaGetDevice");
+    if (dev < 0 || dev >= 64) return fail(o, NOVAK_EINVAL, "step_noalloc: device index %d out of range", dev);
+    // From the owner check to the launch nothing of another handle's call may
+    // come in between: the table would hold one handle's records while the
+    // other handle's kernel reads it.
+    std::lock_guard<std::mutex> table_lock(g_noalloc_mutex);
     if ((e = novak::noalloc_table(&d_recs, &d_chunks)) != cudaSuccess)
         return fail_cuda(o, e, "cudaGetSymbolAddress(static work table)");
     if (o->na_token == 0 || g_noalloc_owner[dev] != o->na_token) {
@@ -581,6 +594,14 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
     const int n_chunks = static_cast<int>(o->na_chunks.size());
     novak::LaunchCfg cfg;
     cfg.grid = n_chunks;
+    if (o->ctas_per_sm > 0) {
+        // NOVAK_OPT_CTAS_PER_SM as in novak_step; the SM count is a device
+        // attribute query, not an allocation
+        if (o->sms <= 0 &&
+            (e = cudaDeviceGetAttribute(&o->sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return fail_cuda(o, e, "cudaDeviceGetAttribute(SM count)");
+        cfg.grid = std::min(n_chunks, o->sms * o->ctas_per_sm);
+    }
     cfg.reverse = (o->serpentine && (t % 2 == 0)) ? 1 : 0;
     cfg.pdl = o->pdl;
     cfg.pre = novak::PRE_NONE | (o->copies.empty() ? 0 : novak::PRE_COPY16) |

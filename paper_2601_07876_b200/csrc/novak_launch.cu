@@ -5,25 +5,20 @@
 
 #include "novak.h"
 
+#include <mutex>
+
 #ifndef NOVAK_BLOCK
 #define NOVAK_BLOCK 256
 #endif
 
 namespace novak {
 
-// One translation unit per gradient pre-processing mode holds the kernels.
-void *step_kernel_pre0(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre1(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre2(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre0_copy(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre1_copy(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre2_copy(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre0_mom16(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre1_mom16(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre2_mom16(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre0_copy_mom16(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre1_copy_mom16(int nesterov, int grad_dtype, int la);
-void *step_kernel_pre2_copy_mom16(int nesterov, int grad_dtype, int la);
+// novak_step_inst.cu, compiled once per gradient pre-processing mode, holds the
+// kernels; mode N (the PRE_* bits as a number) exports step_kernel_mode<N>.
+#define NOVAK_FOR_EACH_PRE_MODE(X) X(0) X(1) X(2) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(13) X(14)
+#define NOVAK_DECLARE(N) void *step_kernel_mode##N(int nesterov, int grad_dtype, int la);
+NOVAK_FOR_EACH_PRE_MODE(NOVAK_DECLARE)
+#undef NOVAK_DECLARE
 
 namespace {
 
@@ -36,18 +31,9 @@ StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
 {
     void *fn = nullptr;
     switch (pre) {
-    case PRE_NONE: fn = step_kernel_pre0(nesterov, grad_dtype, la); break;
-    case PRE_SCALE: fn = step_kernel_pre1(nesterov, grad_dtype, la); break;
-    case PRE_CENTER: fn = step_kernel_pre2(nesterov, grad_dtype, la); break;
-    case PRE_NONE | PRE_COPY16: fn = step_kernel_pre0_copy(nesterov, grad_dtype, la); break;
-    case PRE_SCALE | PRE_COPY16: fn = step_kernel_pre1_copy(nesterov, grad_dtype, la); break;
-    case PRE_CENTER | PRE_COPY16: fn = step_kernel_pre2_copy(nesterov, grad_dtype, la); break;
-    case PRE_NONE | PRE_MOM16: fn = step_kernel_pre0_mom16(nesterov, grad_dtype, la); break;
-    case PRE_SCALE | PRE_MOM16: fn = step_kernel_pre1_mom16(nesterov, grad_dtype, la); break;
-    case PRE_CENTER | PRE_MOM16: fn = step_kernel_pre2_mom16(nesterov, grad_dtype, la); break;
-    case PRE_NONE | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre0_copy_mom16(nesterov, grad_dtype, la); break;
-    case PRE_SCALE | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre1_copy_mom16(nesterov, grad_dtype, la); break;
-    case PRE_CENTER | PRE_COPY16 | PRE_MOM16: fn = step_kernel_pre2_copy_mom16(nesterov, grad_dtype, la); break;
+#define NOVAK_CASE(N) case N: fn = step_kernel_mode##N(nesterov, grad_dtype, la); break;
+        NOVAK_FOR_EACH_PRE_MODE(NOVAK_CASE)
+#undef NOVAK_CASE
     default: break;
     }
     return reinterpret_cast<StepKernelFn>(fn);
@@ -69,6 +55,8 @@ cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks)
 {
     constexpr int kMaxDevices = 64;
     static void *resolved[kMaxDevices] = {};
+    static std::mutex resolved_mutex;   // host threads may make their first call together
+    std::lock_guard<std::mutex> lock(resolved_mutex);
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;

@@ -21,7 +21,7 @@ namespace {
 template <int NEST, int GT, int LA, int PRE>
 __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, int n_chunks,
                                             const TensorRec *__restrict__ recs, const PreArgs &pre0,
-                                            const float *__restrict__ trust,
+                                            const float *trust,
                                             const StepScalars &s, int reverse, int c, Chunk ch,
                                             TensorRec r)
 {
@@ -33,7 +33,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
 #pragma unroll 1
     for (;;) {
         // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
-        pre.step = trust != nullptr ? pre0.step * __ldg(trust + ch.tensor) : pre0.step;
+        pre.step = trust != nullptr ? pre0.step * trust[ch.tensor] : pre0.step;
         pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
@@ -77,8 +77,8 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
 template <int NEST, int GT, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_DYN_MIN_CTAS)
 novak_step_dyn_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                      const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                      const float *__restrict__ trust, const DevPlan *__restrict__ plan, int reverse)
+                      const TensorRec *__restrict__ recs, const PrepOut *prep,
+                      const float *trust, const DevPlan *plan, int reverse)
 {
     const int c = blockIdx.x;
     if (c >= n_chunks) return;

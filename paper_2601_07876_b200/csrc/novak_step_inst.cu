@@ -1,0 +1,37 @@
+// Every instantiation of the step kernel for ONE gradient pre-processing mode.
+// The build compiles this file once per mode, in parallel:
+//   -DNOVAK_PRE_MODE=<PRE_NONE|PRE_SCALE|PRE_CENTER, optionally | PRE_COPY16 | PRE_MOM16,
+//                     as a number>
+//   -DNOVAK_INST_DYN   for the graph-capturable kernel (scalars and lookahead
+//                      action read from device memory) instead of the plain one.
+// Each object exports one selector, step_kernel_mode<N> or step_dyn_kernel_mode<N>.
+#ifndef NOVAK_PRE_MODE
+#error "compile with -DNOVAK_PRE_MODE=<mode bits>"
+#endif
+
+#define NOVAK_PASTE2(a, b) a##b
+#define NOVAK_PASTE(a, b) NOVAK_PASTE2(a, b)
+
+#ifdef NOVAK_INST_DYN
+#include "novak_step_dyn.cuh"
+
+namespace novak {
+
+void *NOVAK_PASTE(step_dyn_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad_dtype)
+{
+    return reinterpret_cast<void *>(pick_step_dyn_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype));
+}
+
+}  // namespace novak
+#else
+#include "novak_step_kernel.cuh"
+
+namespace novak {
+
+void *NOVAK_PASTE(step_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad_dtype, int la)
+{
+    return reinterpret_cast<void *>(pick_step_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype, la));
+}
+
+}  // namespace novak
+#endif

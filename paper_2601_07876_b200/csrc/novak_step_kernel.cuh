@@ -165,7 +165,7 @@ __device__ __forceinline__ RowPos row_position(uint32_t e, const PreArgs &a)
         if (a.mean != nullptr) {
             r.row = e / a.row_len;
             r.rem = e - r.row * a.row_len;
-            r.mu = __ldg(a.mean + r.row);
+            r.mu = a.mean[r.row];
         }
     }
     return r;
@@ -184,7 +184,7 @@ __device__ __forceinline__ void preprocess(Vec<N> &G, const RowPos &pos, const P
                 if (rem == a.row_len) {     // stepped over the end of the row
                     rem = 0;
                     ++row;
-                    mu = __ldg(a.mean + row);
+                    mu = a.mean[row];
                 }
                 G.a[j] = (G.a[j] - mu.x) - mu.y;
                 ++rem;
@@ -339,8 +339,8 @@ __device__ __forceinline__ void grid_dependency_wait()
 template <int NEST, int GT, int LA, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS)
 novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                  const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                  const float *__restrict__ trust, const StepScalars s, int reverse)
+                  const TensorRec *__restrict__ recs, const PrepOut *prep,
+                  const float *trust, const StepScalars s, int reverse)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
     constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
@@ -351,7 +351,10 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     int c = blockIdx.x;
     if (c >= n_chunks) return;
     // The work table is written by copies only, never by a kernel, so it may be
-    // read before the previous kernel on the stream has finished.
+    // read before the previous kernel on the stream has finished.  prep, trust
+    // and the row means ARE the previous kernels' output and this grid may be
+    // resident while they are written: they are not declared read-only
+    // (no __restrict__, no non-coherent loads) and are read after the wait.
     Chunk ch = chunks[reverse ? n_chunks - 1 - c : c];
     TensorRec r = recs[ch.tensor];
     grid_dependency_wait();
@@ -368,7 +371,7 @@ novak_step_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 #pragma unroll 1
     for (;;) {
         // Eq. 24a: the tensor's trust ratio stretches the step (layer adaptation)
-        pre.step = trust != nullptr ? step * __ldg(trust + ch.tensor) : step;
+        pre.step = trust != nullptr ? step * trust[ch.tensor] : step;
         pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);

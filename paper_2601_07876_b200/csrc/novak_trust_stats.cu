@@ -67,8 +67,8 @@ __device__ __forceinline__ void accumulate(const float *p, const void *g, const 
 template <int NEST, int GT, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK)
 novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
-                         const TensorRec *__restrict__ recs, const PrepOut *__restrict__ prep,
-                         const StepScalars s_host, const DevPlan *__restrict__ plan,
+                         const TensorRec *__restrict__ recs, const PrepOut *prep,
+                         const StepScalars s_host, const DevPlan *plan,
                          double *__restrict__ chunk_u2, double *__restrict__ chunk_p2)
 {
     __shared__ double sh[kTrustWarps];
@@ -126,8 +126,8 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 // One CTA per tensor: its entries' sums in table order, then Eq. 19's ratio.
 __global__ void __launch_bounds__(NOVAK_BLOCK)
 novak_trust_finish_kernel(const int *__restrict__ tensor_first,
-                          const double *__restrict__ chunk_u2,
-                          const double *__restrict__ chunk_p2, float *__restrict__ trust)
+                          const double *chunk_u2,
+                          const double *chunk_p2, float *__restrict__ trust)
 {
     __shared__ double sh[kTrustWarps];
     grid_dependency_release();

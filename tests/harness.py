@@ -13,30 +13,8 @@ from paper_2601_07876_b200 import workloads as W
 # |gpu - oracle| <= ATOL + RTOL * |oracle| for theta, m, v, slow, acc.
 RTOL, ATOL = 1e-5, 1e-7
 
-_NEST = {"none": O.NESTEROV_NONE, "approximation": O.NESTEROV_APPROX,
-         "classical": O.NESTEROV_CLASSICAL, "true": O.NESTEROV_TRUE}
-_MODE = {"last": O.LOOKAHEAD_LAST, "traj_mean": O.LOOKAHEAD_TRAJ_MEAN}
-
-
 def oracle_config(hyper: dict) -> O.Config:
-    h = dict(hyper)
-    b1, b2 = h.pop("betas", (0.9, 0.999))
-    return O.Config(
-        lr=h.pop("lr", 1e-3), beta1=b1, beta2=b2, eps=h.pop("eps", 1e-8),
-        weight_decay=h.pop("weight_decay", 1e-2),
-        nesterov_variant=_NEST[h.pop("nesterov", "approximation")],
-        lookahead_k=h.pop("lookahead_k", 5), lookahead_alpha=h.pop("lookahead_alpha", 0.5),
-        nesterov_beta=h.pop("nesterov_beta", None),
-        lookahead_mode=_MODE[h.pop("lookahead_mode", "last")],
-        rectified=h.pop("rectified", True), bias1_power=h.pop("bias1_power", 1),
-        clip_threshold=h.pop("clip_threshold", 0.0), centralize=h.pop("centralize", False),
-        layer_adaptation=h.pop("layer_adaptation", False),
-        sparse_threshold=h.pop("sparse_threshold", 0.0),
-        auto_lr=h.pop("auto_lr", False), auto_lr_gamma=h.pop("auto_lr_gamma", None) or 0.1,
-        adaptive_beta=h.pop("adaptive_beta", False), tau1=h.pop("tau1", None) or 1000.0,
-        tau2=h.pop("tau2", None) or 5000.0,
-        true_steps=h.pop("true_nesterov_steps", 0),
-        moment_bf16=h.pop("moment_dtype", "f32") == "bf16")
+    return O.Config.from_hyper(hyper)
 
 
 def tensor_rows(tensors):
@@ -174,6 +152,67 @@ def gaps_mask(total, starts, numels, device):
     for s, n in zip(starts, numels):
         m[s:s + n] = False
     return m
+
+
+class FullPair:
+    """Full-size workload on the GPU and the oracle on EVERY element of it.
+
+    The oracle sees the workload's flat buffer as one tensor (the step has no
+    cross-element term; the padding between tensors holds zero parameters and zero
+    gradients and stays zero on both sides), so its arrays line up with the flat
+    parameter and gradient buffers; the library's own state layout is compared tensor
+    by tensor through novak_state_ptrs."""
+
+    def __init__(self, wl: W.Workload, device, hyper_override: dict | None = None,
+                 opt_kwargs: dict | None = None):
+        self.wl = wl
+        self.hyper = dict(wl.hyper, **(hyper_override or {}))
+        self.flat_p = W.alloc_flat(wl, torch.float32, device)
+        W.init_params(wl, self.flat_p)
+        self.flat_g = W.alloc_flat(wl, wl.grad_dtype, device)
+        self.scratch = (W.alloc_flat(wl, torch.float32, device)
+                        if wl.grad_dtype != torch.float32 else None)
+        self.params = W.views(self.flat_p, wl)
+        self.grads = W.views(self.flat_g, wl)
+        self.offs, _ = W.element_offsets(wl)
+        self.src = W.GradSource(wl, device)
+        self.oracle = O.Oracle(oracle_config(self.hyper), [to_f64(self.flat_p)])
+        self.opt = B.NovakOptimizer(self.params, **self.hyper, **(opt_kwargs or {}))
+        self.glist = self.opt.prepare(self.grads)
+        self.sync_steps, self.rect_flags = [], []
+        self.compared = 0
+
+    def step(self, threads=1):
+        self.src.fill(self.flat_g, self.scratch)
+        self.opt.step(self.glist)
+        info = self.opt.info()
+        if info["is_sync"]:
+            self.sync_steps.append(info["t"])
+        self.rect_flags.append(info["rect_branch"])
+        self.oracle.step([to_f64(self.flat_g)], threads=threads)
+
+    def check(self):
+        torch.cuda.synchronize()
+        o, info = self.oracle, self.opt.info()
+        assert info["t"] == o.t and self.sync_steps == o.sync_steps
+        assert self.rect_flags == o.rect_flags
+        assert info["n_syncs"] == len(o.sync_steps)
+        name = self.wl.name
+        # parameters: the whole flat buffer, padding included (nothing may be written there)
+        assert_close(self.flat_p, o.theta[0], f"{name} theta")
+        with_acc = o.acc is not None and o.cfg.lookahead_k > 1 and o.t % o.cfg.lookahead_k != 0
+        for i, (off, n) in enumerate(zip(self.offs, self.wl.numel)):
+            st = self.opt.state(i)
+            assert_close(st["m"], o.m[0][off:off + n], f"{name} m")
+            assert_close(st["v"], o.v[0][off:off + n], f"{name} v")
+            if n >= 1024:     # a root mean square needs a population
+                assert_close_scaled(st["m"], o.m[0][off:off + n], f"{name} m")
+                assert_close_scaled(st["v"], o.v[0][off:off + n], f"{name} v")
+            if o.slow is not None:
+                assert_close(st["slow"], o.slow[0][off:off + n], f"{name} slow")
+            if with_acc:
+                assert_close(st["acc"], o.acc[0][off:off + n], f"{name} acc")
+            self.compared += n
 
 
 class SampledPair:

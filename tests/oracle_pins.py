@@ -702,6 +702,57 @@ def pin_sparse_mask(lib):
     assert t1.trust[0][0] == t0.trust[0][0]
 
 
+def _direction(lib, o, g):
+    """novak_oracle_direction for the step the oracle object `o` would take next."""
+    u = np.empty_like(g)
+    lib.novak_oracle_direction(ctypes.byref(o.h), o.t + 1, g.size, O._dptr(g), O._dptr(o.m[0]),
+                               O._dptr(o.v[0]), O._dptr(u))
+    return u
+
+
+def pin_direction(lib):
+    """novak_oracle_direction (the base direction of Eq. 17 that the next step would
+    produce, used to see how close |u| comes to Eq. 27's threshold) against the step itself,
+    which the pins above fix: with no weight decay, rectification off and alpha = 1 the step
+    of Eq. 24 moves every parameter by exactly -u, so theta_before - theta_after = u.  Runs
+    from non-zero moments, for the plain and the approximation variant and under the warm-up
+    of Eq. 3-4; at t = 1 from zero moments u is known in closed form."""
+    rng = np.random.default_rng(77)
+    n = 64
+    for kw in (dict(nesterov_variant=O.NESTEROV_NONE),
+               dict(nesterov_variant=O.NESTEROV_APPROX, nesterov_beta=0.7),
+               dict(nesterov_variant=O.NESTEROV_APPROX, adaptive_beta=True, tau1=3.0, tau2=11.0),
+               dict(nesterov_variant=O.NESTEROV_TRUE, true_steps=2, nesterov_beta=0.6)):
+        o = _mk(lib, [rng.normal(0, 0.5, n)], lr=1.0, weight_decay=0.0, rectified=False,
+                lookahead_k=0, eps=1e-3, **kw)
+        for t in range(1, 7):
+            g = rng.normal(0, 1.0, n) * 10.0 ** rng.integers(-4, 1, n)
+            m0, v0 = o.m[0].copy(), o.v[0].copy()
+            u = _direction(lib, o, g)
+            assert np.array_equal(o.m[0], m0) and np.array_equal(o.v[0], v0), "nothing is written"
+            before = o.theta[0].copy()
+            o.step([g])
+            # theta_after = theta_before - u: recover u to the rounding of that subtraction
+            _close(u, before - o.theta[0], rtol=1e-9, atol=4e-16 * np.abs(before).max(),
+                   what=f"direction against the step, t={t} {kw}")
+    # closed forms at t = 1 from zero moments: m_hat = g~, v_hat = g~^2, u = g~/(|g~|+eps)
+    g = np.array([0.3, -0.02, 1e-4, -7.0, 0.0, 2.5e-3])
+    eps = 1e-2
+    o = _mk(lib, [np.zeros(g.size)], eps=eps, nesterov_variant=O.NESTEROV_NONE)
+    _close(_direction(lib, o, g), g / (np.abs(g) + eps), what="u_1, variant none")
+    bn = 0.5
+    o = _mk(lib, [np.zeros(g.size)], eps=eps, nesterov_variant=O.NESTEROV_APPROX, nesterov_beta=bn)
+    gt = g * (1 + bn)                                        # Eq. 13 with m_0 = 0
+    _close(_direction(lib, o, g), gt / (np.abs(gt) + eps), what="u_1, approximation")
+    # eps sits outside the root: with v_hat = g^2 = 1e-12 and eps = 1e-3, u = g/(1e-6+1e-3)
+    o = _mk(lib, [np.zeros(1)], eps=1e-3, nesterov_variant=O.NESTEROV_NONE)
+    _close(_direction(lib, o, np.array([1e-6])), [1e-6 / (1e-6 + 1e-3)], what="eps outside the root")
+    # the classical blend and the mask come after Eq. 17: the base direction ignores both
+    a = _mk(lib, [np.zeros(g.size)], eps=eps, nesterov_variant=O.NESTEROV_CLASSICAL,
+            sparse_threshold=0.4)
+    _close(_direction(lib, a, g), g / (np.abs(g) + eps), what="before blend and mask")
+
+
 # --------------------------------------------------------------------------
 # Phase 7: automatic learning-rate scaling (Eq. 20-22)
 # --------------------------------------------------------------------------
@@ -988,6 +1039,7 @@ ALL_PINS = [
     pin_adaptive_beta,
     pin_trust_ratio,
     pin_sparse_mask,
+    pin_direction,
     pin_auto_lr,
     pin_true_nesterov,
     pin_bf16_moment_storage,

@@ -1,34 +1,25 @@
 """Parity at the benchmark's full sizes, in the launch configuration bench.py
-times.  The oracle runs on a fixed sample of elements (small tensors whole,
-both ends of every tensor, a stride-997 comb); that is exact for the sampled
-elements because the step has no cross-element term."""
+times.  The ResNet-50-, VGG-16- and ViT-B/16-shaped sets are compared on EVERY
+element in both lookahead modes (the oracle runs on all host cores).  For the
+1 B-parameter set the oracle follows a fixed sample of elements (small tensors
+whole, both ends of every tensor, a stride-997 comb); that is exact for the
+sampled elements because the step has no cross-element term."""
+import os
+
 import pytest
 import torch
 
 import harness
-from harness import SampledPair
+from harness import FullPair, SampledPair
 from paper_2601_07876_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
+CORES = max(1, len(os.sched_getaffinity(0)))
 
 
-@pytest.mark.parametrize("index,mode", [(1, "last"), (1, "traj_mean"), (2, "last"),
-                                        (3, "last"), (3, "traj_mean"), (4, "last"),
-                                        (4, "traj_mean")])
-def test_fullsize_workload(index, mode):
-    wl = W.get_workload(index)
-    free, _ = torch.cuda.mem_get_info()
-    need = wl.total * 4 * 8
-    if free < need:
-        pytest.skip(f"needs {need >> 30} GiB of device memory")
-    harness.MARGINS.clear()
-    harness.SCALED.clear()
-    pair = SampledPair(wl, DEV, dict(lookahead_mode=mode))
-    for _ in range(wl.steps):
-        pair.step(threads=8)
-    pair.check()
-    print(f"\nPARITY {wl.name} {mode} steps={wl.steps} sampled={pair.idx.numel()} worst |err|/tol: "
+def _report(pair, wl, mode, compared):
+    print(f"\nPARITY {wl.name} {mode} steps={wl.steps} compared={compared} worst |err|/tol: "
           + ", ".join(f"{k.split()[-1]} {v:.3f}" for k, v in harness.MARGINS.items())
           + "; moments relative to their rms: "
           + ", ".join(f"{k.split()[-1]} {v:.2e}" for k, v in harness.SCALED.items()))
@@ -39,6 +30,42 @@ def test_fullsize_workload(index, mode):
     assert info["launches"] == wl.steps and info["total_numel"] == wl.total
     misaligned = bool(info["warnings"] & 2)
     assert not misaligned, "every tensor should run on 128-bit accesses"
+
+
+@pytest.mark.parametrize("index,mode", [(1, "last"), (1, "traj_mean"), (2, "last"),
+                                        (2, "traj_mean"), (3, "last"), (3, "traj_mean")])
+def test_fullsize_workload_every_element(index, mode):
+    wl = W.get_workload(index)
+    free, _ = torch.cuda.mem_get_info()
+    need = wl.total * 4 * 8
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory")
+    harness.MARGINS.clear()
+    harness.SCALED.clear()
+    pair = FullPair(wl, DEV, dict(lookahead_mode=mode))
+    for _ in range(wl.steps):
+        pair.step(threads=CORES)
+    pair.check()
+    assert pair.compared == wl.total
+    _report(pair, wl, mode, pair.compared)
+    del pair
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("mode", ["last", "traj_mean"])
+def test_fullsize_1b_set_on_a_sample(mode):
+    wl = W.get_workload(4)
+    free, _ = torch.cuda.mem_get_info()
+    need = wl.total * 4 * 8
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory")
+    harness.MARGINS.clear()
+    harness.SCALED.clear()
+    pair = SampledPair(wl, DEV, dict(lookahead_mode=mode))
+    for _ in range(wl.steps):
+        pair.step(threads=min(8, CORES))
+    pair.check()
+    _report(pair, wl, mode, pair.idx.numel())
     del pair
     torch.cuda.empty_cache()
 

@@ -67,20 +67,22 @@ def test_variants_ragged_multi_tensor(nesterov, la, gdtype):
     assert not pair.opt.info()["warnings"] & B.NOVAK_WARN_SCALAR_PATH
 
 
-def test_config0_flat_1m_every_element():
-    """First benchmark configuration: one flat tensor of 1,048,576, 20 steps."""
+@pytest.mark.parametrize("mode", ["last", "traj_mean"])
+def test_config0_flat_1m_every_element(mode):
+    """First benchmark configuration: one flat tensor of 1,048,576, 20 steps, in both
+    lookahead modes."""
     from paper_2601_07876_b200 import workloads as W
     wl = W.get_workload(0)
     flat = W.alloc_flat(wl, torch.float32, DEV)
     W.init_params(wl, flat)
     params = W.views(flat, wl)
-    pair = Pair(params, wl.hyper)
+    pair = Pair(params, dict(wl.hyper, lookahead_mode=mode))
     src = W.GradSource(wl, DEV)
     gflat = W.alloc_flat(wl, torch.float32, DEV)
     for _ in range(wl.steps):
         src.fill(gflat)
         pair.step(W.views(gflat, wl), threads=4)
-    pair.check("flat-1M")
+    pair.check(f"flat-1M {mode}")
     assert pair.sync_steps == [5, 10, 15, 20]
     assert pair.rect_flags == [0] * 5 + [1] * 15
     info = pair.opt.info()

@@ -94,6 +94,16 @@ MUTANTS = [
     ("mask_after_blend", "if (h->sparse_threshold > 0.0 && !(fabs(u) > h->sparse_threshold))\n            u = 0.0;\n        if (h->nesterov_variant == 2)\n            u = h->beta1 * m_hat + (1.0 - h->beta1) * u;",
      "if (h->nesterov_variant == 2)\n            u = h->beta1 * m_hat + (1.0 - h->beta1) * u;\n        if (h->sparse_threshold > 0.0 && !(fabs(u) > h->sparse_threshold))\n            u = 0.0;"),
     ("mask_on_gradient", "!(fabs(u) > h->sparse_threshold))", "!(fabs(gt) > h->sparse_threshold))"),
+    # the base direction on its own (novak_oracle_direction)
+    ("direction_stale_moments", "u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);",
+     "u_out[i] = (m[i] / s.bc1) / (sqrt(v[i] / s.bc2) + h->eps);"),
+    ("direction_eps_inside_root", "u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);",
+     "u_out[i] = (m_new / s.bc1) / sqrt(v_new / s.bc2 + h->eps);"),
+    ("direction_without_nesterov_term",
+     "gt = g[i] + h->nesterov_beta * (g[i] - m[i]);\n        const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;\n        const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;\n        u_out",
+     "gt = g[i];\n        const double m_new = s.beta1_t * m[i] + (1.0 - s.beta1_t) * gt;\n        const double v_new = s.beta2_t * v[i] + (1.0 - s.beta2_t) * gt * gt;\n        u_out"),
+    ("direction_uncorrected_second_moment", "u_out[i] = (m_new / s.bc1) / (sqrt(v_new / s.bc2) + h->eps);",
+     "u_out[i] = (m_new / s.bc1) / (sqrt(v_new) + h->eps);"),
     # phase 7: layer-wise adaptation
     ("trust_inverted", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sqrt(sum_u) / sqrt(sum_theta);"),
     ("trust_of_squared_norms", "double eta = sqrt(sum_theta) / sqrt(sum_u);", "double eta = sum_theta / sum_u;"),

@@ -111,3 +111,78 @@ def test_noalloc_rejects_sizes_beyond_the_static_table():
     assert e.value.status == B.NOVAK_EINVAL and "4096" in str(e.value)
     assert opt.info()["t"] == 0
     torch.cuda.synchronize()
+
+
+def test_noalloc_against_the_oracle():
+    """The entry point on its own merits: 12 steps of novak_step_noalloc against the CPU
+    oracle on every element (rectification switch at t = 6, six lookahead syncs), rather
+    than only through its agreement with novak_step."""
+    from harness import Pair
+    _, params, _ = make_tensors(NUMELS, DEV, OFFSETS)
+    gen = torch.Generator(device=DEV).manual_seed(9)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    for mode in ("last", "traj_mean"):
+        pair = Pair([p.clone() for p in params], dict(HYPER, lookahead_mode=mode))
+        keep = []
+        pair.opt.step = lambda grads: keep.append(_step_noalloc(pair.opt, grads))
+        for _ in range(12):
+            pair.step(_grads(gen))
+        pair.check(f"noalloc {mode}")
+        assert pair.sync_steps == [2, 4, 6, 8, 10, 12]
+        assert pair.rect_flags == [0] * 5 + [1] * 7
+        info = pair.opt.info()
+        assert info["launches"] == 12 and info["n_chunks"] == 0   # nothing was allocated for it
+
+
+def test_noalloc_two_host_threads_on_one_stream():
+    """Two host threads, a handle each, call novak_step_noalloc at the same time.  Both
+    enqueue on ONE stream, so the GPU side is ordered and only the host side interleaves:
+    the table must always hold the calling handle's own records when its kernel is
+    enqueued.  Each result has to equal, bit for bit, what novak_step gives that handle's
+    twin from the same gradients."""
+    import threading
+    steps = 150
+    pa, a = _setup(21)                     # thread 1, noalloc
+    pb, b = _setup(22, mode="traj_mean")   # thread 2, noalloc
+    ra, ta = _setup(21)                    # their twins on novak_step
+    rb, tb = _setup(22, mode="traj_mean")
+    gen = torch.Generator(device=DEV).manual_seed(23)
+    ga = [_grads(gen) for _ in range(3)]
+    gb = [_grads(gen) for _ in range(3)]
+    la, lb = [a.prepare(g) for g in ga], [b.prepare(g) for g in gb]
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    raw = stream.cuda_stream
+    start = threading.Barrier(2)
+    errors = []
+
+    def run(opt, lists):
+        try:
+            start.wait()
+            for i in range(steps):
+                gl = lists[i % 3]
+                opt.handle.step_noalloc(opt._params_arr, gl.arr, opt._numel_arr, opt.n, gl.dtype, raw)
+        except Exception as exc:            # pragma: no cover
+            errors.append(exc)
+
+    threads = [threading.Thread(target=run, args=(a, la)), threading.Thread(target=run, args=(b, lb))]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    stream.synchronize()
+    assert not errors, errors
+    for i in range(steps):
+        ta.step(ga[i % 3])
+        tb.step(gb[i % 3])
+    torch.cuda.synchronize()
+    assert a.info()["t"] == b.info()["t"] == steps
+    for x, y in zip(ra, pa):
+        assert torch.equal(x, y)
+    for x, y in zip(rb, pb):
+        assert torch.equal(x, y)
+    for i in range(len(NUMELS)):
+        for k in ("m", "v", "slow"):
+            assert torch.equal(ta.state(i)[k], a.state(i)[k])
+            assert torch.equal(tb.state(i)[k], b.state(i)[k])
