@@ -83,8 +83,16 @@ def parse_args():
                     help="c_clip of the global-norm clipping (0: off, the headline path)")
     ap.add_argument("--centralize", action="store_true",
                     help="gradient centralization on tensors with more than one dimension")
+    ap.add_argument("--centralize-in-step", type=int, default=None, choices=[0, 1],
+                    help="0: centralization always through the statistics pass (default 1: "
+                         "inside the step kernel when nothing else needs the whole gradient)")
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
+    ap.add_argument("--layer-adaptation-in-step", type=int, default=None, choices=[0, 1],
+                    help="0: layer adaptation as two statistics kernels and the step (default 1: "
+                         "one persistent kernel whose update items find their tensor in L2)")
+    ap.add_argument("--layer-adaptation-lead", type=int, default=None,
+                    help="elements by which that kernel's statistics run ahead of its updates")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
     ap.add_argument("--zero1", action="store_true",
                     help="one group sharded over the ranks (reduce-scatter, step on the owned "
@@ -94,9 +102,13 @@ def parse_args():
     ap.add_argument("--bf16-copy", action="store_true",
                     help="the step also writes a bf16 copy of the parameters (+2 B per element)")
     ap.add_argument("--true-nesterov", action="store_true",
-                    help="every step is a true-Nesterov step (Eq. 10-12): look-ahead kernel, "
-                         "restore kernel, step; the closure between the two is the caller's "
-                         "and not part of the step (+24 B per element)")
+                    help="every step is a true-Nesterov step (Eq. 10-12): look-ahead kernel, then "
+                         "the step, which reads theta_{t-1} from the save buffer; the closure "
+                         "between the two is the caller's and not part of the step (+16 B per "
+                         "element)")
+    ap.add_argument("--restore-pass", action="store_true",
+                    help="with --true-nesterov: a separate restore kernel between look-ahead "
+                         "and step (+8 B per element more)")
     ap.add_argument("--moment-dtype", default="f32", choices=["f32", "bf16"],
                     help="storage type of m and v (bf16: 20 B per element instead of 28)")
     ap.add_argument("--graph", type=int, default=0, metavar="G",
@@ -104,6 +116,9 @@ def parse_args():
                          "graph (stream capture) and the timed region replays it; steps is "
                          "rounded down to a multiple of G")
     ap.add_argument("--pool", type=int, default=4, help="gradient sets rotated through")
+    ap.add_argument("--grad-offset", type=int, default=0, metavar="E",
+                    help="start every gradient buffer E elements off the parameters' 16-byte "
+                         "phase (E = 1..3: the gradient alone is then fetched element by element)")
     ap.add_argument("--chunk-elems", type=int, default=None)
     ap.add_argument("--ctas-per-sm", type=int, default=None)
     ap.add_argument("--serpentine", type=int, default=None)
@@ -115,27 +130,42 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--min-timed-seconds", type=float, default=0.5,
+                    help="the K-step timed region is repeated until the repeats total at least "
+                         "this long; ms_per_step is the median over the repeats")
+    ap.add_argument("--max-repeats", type=int, default=2000)
+    ap.add_argument("--per-step-steps", type=int, default=300,
+                    help="steps of the separate pass that times every step on its own (0: skip)")
+    ap.add_argument("--no-per-workload", action="store_true",
+                    help="skip the other workloads / lookahead modes (key per_workload)")
     return ap.parse_args()
 
 
 def algorithmic_bytes_per_elem(grad_bytes: int, k: int, mode: str, t: int,
-                               phase2: bool = False, trust: bool = False,
+                               phase2: bool = False, trust: float = 0.0,
                                copy16: bool = False, auto: bool = False,
                                true_nesterov: bool = False, moment_bytes: int = 4) -> int:
     """Bytes the method itself has to move for one element on step t: theta, g, m, v
     read, theta, m, v written (Section 5.5: 4 reads + 3 writes), plus the lookahead
-    arrays on the steps that touch them, plus one more read of g when clipping or
-    centralization is on (the norm and the row means are needed before the update)."""
+    arrays on the steps that touch them, plus one more read of g (`phase2`) when the
+    global norm is needed before the first update (clipping, automatic learning-rate
+    scaling).  Centralization alone adds nothing: a row mean is a statistic of one row,
+    which fits on chip, so every byte still has to move only once."""
     mb = moment_bytes
     b = 4 + 2 * mb + grad_bytes + 4 + 2 * mb + (grad_bytes if phase2 else 0)
     if trust:
-        b += 4 + 2 * mb + grad_bytes     # theta, g, m, v read once more for the norms of Eq. 19
+        # theta, g, m, v are needed twice (the norms of Eq. 19, then the update).  A tensor
+        # that fits in L2 has to come from DRAM only once; `trust` is the share of the
+        # group's elements in tensors too large for that (1.0: every tensor read twice).
+        b += float(trust) * (4 + 2 * mb + grad_bytes)
     if copy16:
         b += 2
     if auto:
         b += 4                           # ||theta_t|| of Eq. 21
     if true_nesterov:
-        b += 12 + mb + 8                 # Eq. 10: theta, m read, save, theta written; restore
+        b += 12 + mb                     # Eq. 10: theta, m read, save, theta written
+    if true_nesterov == "restore":
+        b += 8                           # the separate restore pass: save read, theta written
     if k <= 0:
         return b
     sync = t % k == 0
@@ -204,7 +234,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.01)
 
     def __enter__(self):
         if self._h is not None:
@@ -376,6 +406,77 @@ def run_zero1(args, rank, world, local):
     dist.destroy_process_group()
 
 
+def quantile(sorted_vals, f):
+    return sorted_vals[min(len(sorted_vals) - 1, int(f * len(sorted_vals)))] if sorted_vals else None
+
+
+def timed_repeats(torch, step_fn, steps, repeats, barrier):
+    """`repeats` back-to-back regions of exactly `steps` steps, each between two CUDA events
+    on the launching stream, a barrier + synchronize before the first and after the last.
+    Returns the regions' durations in ms."""
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    barrier()
+    evs[0].record()
+    i = 0
+    for r in range(repeats):
+        for _ in range(steps):
+            step_fn(i)
+            i += 1
+        evs[r + 1].record()
+    barrier()
+    return [evs[r].elapsed_time(evs[r + 1]) for r in range(repeats)]
+
+
+def repeats_for(ms_per_step_estimate, steps, min_seconds, max_repeats):
+    region = max(1e-6, ms_per_step_estimate * steps * 1e-3)
+    return int(max(1, min(max_repeats, -(-min_seconds // region))))
+
+
+def time_one_workload(torch, B, W, dev, index, mode, steps, warmup, min_seconds, max_repeats,
+                      pool_want, lib, barrier):
+    """One workload in one lookahead mode, everything resident: median ms per step over
+    repeated `steps`-step regions, with the algorithmic bytes of exactly those steps."""
+    wl = W.get_workload(index)
+    hyper = dict(wl.hyper, lookahead_mode=mode)
+    k = hyper["lookahead_k"]
+    gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
+    flat_p = W.alloc_flat(wl, torch.float32, dev)
+    W.init_params(wl, flat_p)
+    params = W.views(flat_p, wl)
+    pool_n = max(1, min(pool_want, int(8e9 // (wl.total * gbytes)) or 1))
+    src = W.GradSource(wl, dev)
+    scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
+    pool_flat = [W.alloc_flat(wl, wl.grad_dtype, dev) for _ in range(pool_n)]
+    for gf in pool_flat:
+        src.fill(gf, scratch)
+    del scratch
+    opt = B.NovakOptimizer(params, **hyper, lib=lib)
+    pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
+    for i in range(max(3, warmup)):
+        opt.step(pool[i % pool_n])
+    # a short probe sizes the number of repeats
+    probe = timed_repeats(torch, lambda i: opt.step(pool[i % pool_n]), steps, 1, barrier)[0] / steps
+    repeats = repeats_for(probe, steps, min_seconds, max_repeats)
+    t_first = opt.info()["t"] + 1
+    times = timed_repeats(torch, lambda i: opt.step(pool[i % pool_n]), steps, repeats, barrier)
+    per = sorted(x / steps for x in times)
+    ms = quantile(per, 0.5)
+    alg = sum(algorithmic_bytes_per_elem(gbytes, k, mode, t)
+              for t in range(t_first, t_first + steps * repeats)) / (steps * repeats)
+    gbs = alg * wl.total / (ms * 1e-3) / 1e9
+    peak, _ = measured_peak()
+    out = {"workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
+           "grad_dtype": "bf16" if gbytes == 2 else "f32", "lookahead_mode": mode,
+           "lookahead_k": k, "steps": steps, "repeats": repeats, "ms_per_step": ms,
+           "p10": quantile(per, 0.1), "p90": quantile(per, 0.9),
+           "updates_per_s": wl.total / (ms * 1e-3), "algorithmic_bytes_per_elem": alg,
+           "hbm_gbs": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0,
+           "grad_pool": pool_n, "launches": opt.info()["launches"]}
+    del opt, pool, pool_flat, params, flat_p
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -414,17 +515,23 @@ def main():
     flat_p = W.alloc_flat(wl, torch.float32, dev)
     W.init_params(wl, flat_p)
     params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
-    phase2 = args.clip > 0 or args.centralize or args.auto_lr
+    phase2 = args.clip > 0 or args.auto_lr        # the whole gradient is read twice
+    prepass = phase2 or args.centralize
     pool_n = max(1, min(args.pool, int(8e9 // (wl.total * gbytes)) or 1))
     src = W.GradSource(wl, dev, seed_offset=rank)
     scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
-    pool_flat = [W.alloc_flat(wl, wl.grad_dtype, dev) for _ in range(pool_n)]
+    pool_base = [torch.zeros(W.element_offsets(wl)[1] + 64, dtype=wl.grad_dtype, device=dev)
+                 for _ in range(pool_n)]
+    pool_flat = [b[args.grad_offset:args.grad_offset + W.element_offsets(wl)[1]] for b in pool_base]
     for gf in pool_flat:
         src.fill(gf, scratch)
     del scratch
     opt = B.NovakOptimizer(params, **hyper, clip_threshold=args.clip, centralize=args.centralize,
                            layer_adaptation=args.layer_adaptation, adaptive_beta=args.adaptive_beta,
                            auto_lr=args.auto_lr, graph_capturable=args.graph > 0,
+                           centralize_in_step=args.centralize_in_step,
+                           layer_adaptation_in_step=args.layer_adaptation_in_step,
+                           layer_adaptation_lead=args.layer_adaptation_lead,
                            chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)
@@ -441,8 +548,9 @@ def main():
     plain_step = opt.step
     if args.true_nesterov:
         def true_step(grads):
-            opt.extrapolate()
-            opt.restore()                # the caller's closure would run between the two
+            opt.extrapolate()            # the caller's closure would run behind this
+            if args.restore_pass:
+                opt.restore()
             plain_step(grads)
         opt.step = true_step
 
@@ -465,48 +573,59 @@ def main():
         launches_per_graph = opt.info()["launches"] - l0
         for _ in range(3):
             graph.replay()
+    if graph is not None:
+        step_units = args.steps // args.graph          # one unit = one replay of G steps
+        step_fn = lambda i: graph.replay()
+    else:
+        step_units = args.steps
+        step_fn = lambda i: opt.step(pool[i % pool_n])
+    # a probe region sizes the number of repeats of the K-step region
+    probe_ms = timed_repeats(torch, step_fn, step_units, 1, barrier)[0]
+    repeats = repeats_for(probe_ms / args.steps, args.steps, args.min_timed_seconds, args.max_repeats)
+    if world > 1:
+        r = torch.tensor([repeats], device=dev)
+        dist.all_reduce(r, op=dist.ReduceOp.MAX)
+        repeats = int(r.item())
     t_first = opt.info()["t"] + 1
     launches0 = opt.info()["launches"]
     uploads0 = opt.info()["record_uploads"]
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     with ClockSampler(local) as clocks:
-        ev0.record()
-        if graph is not None:
-            for _ in range(args.steps // args.graph):
-                graph.replay()
-        else:
-            for i in range(args.steps):
-                opt.step(pool[i % pool_n])
-        ev1.record()
-        barrier()
-    ms = ev0.elapsed_time(ev1)
+        region_ms = timed_repeats(torch, step_fn, step_units, repeats, barrier)
     grid_timed = opt.info()["grid"]          # before the end-to-end leg launches its runs
-    launches = opt.info()["launches"] - launches0
+    launches = (opt.info()["launches"] - launches0) // repeats
     if graph is not None:
         launches = launches_per_graph * (args.steps // args.graph)
-        assert opt.info()["t"] == t_first - 1 + args.steps     # every replayed step counted
+        assert opt.info()["t"] == t_first - 1 + args.steps * repeats   # every replayed step counted
     uploads = opt.info()["record_uploads"] - uploads0
     if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    ms_per_step = ms / args.steps
-    value = world * wl.total * args.steps / (ms * 1e-3)
+        t = torch.tensor(region_ms, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)         # per region, the slowest rank
+        region_ms = [float(x) for x in t.tolist()]
+    per_region = sorted(x / args.steps for x in region_ms)
+    ms_per_step = quantile(per_region, 0.5)
+    value = world * wl.total / (ms_per_step * 1e-3)
+    n_timed = args.steps * repeats
+    # layer adaptation: tensors whose theta, g, m, v exceed 48 MB cannot wait in the 126 MB L2
+    # between their statistics and their update
+    per_elem_twice = 4 + 2 * mbytes + gbytes
+    big = sum(n for n in wl.numel if n * per_elem_twice > 48e6) / wl.total
+    trust_share = 0.0 if not args.layer_adaptation else (
+        big if (args.layer_adaptation_in_step != 0 and not prepass) else 1.0)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
-                                         args.layer_adaptation, args.bf16_copy, args.auto_lr,
-                                         args.true_nesterov, mbytes)
-              for t in range(t_first, t_first + args.steps)) / args.steps
+                                         trust_share, args.bf16_copy, args.auto_lr,
+                                         ("restore" if args.restore_pass else True) if args.true_nesterov else False,
+                                         mbytes)
+              for t in range(t_first, t_first + n_timed)) / n_timed
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
-    n_sync = sum(1 for t in range(t_first, t_first + args.steps) if k > 0 and t % k == 0)
-    traffic = None if (phase2 or args.layer_adaptation or args.bf16_copy or args.true_nesterov or mbytes == 2) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / args.steps)
+    n_sync = sum(1 for t in range(t_first, t_first + n_timed) if k > 0 and t % k == 0)
+    traffic = None if (prepass or args.layer_adaptation or args.bf16_copy or args.true_nesterov or mbytes == 2) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / n_timed)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
-    if rank == 0 and graph is None:
-        n_ps = min(args.steps, 300)
+    if rank == 0 and graph is None and args.per_step_steps > 0:
+        n_ps = args.per_step_steps
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_ps + 1)]
         t_ps = opt.info()["t"] + 1
         evs[0].record()
@@ -517,7 +636,7 @@ def main():
         times = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_ps)]
         sync = sorted(x for i, x in enumerate(times) if k > 0 and (t_ps + i) % k == 0)
         plain = sorted(x for i, x in enumerate(times) if not (k > 0 and (t_ps + i) % k == 0))
-        q = lambda s, f: s[min(len(s) - 1, int(f * len(s)))] if s else None
+        q = quantile
         per = {"non_sync_ms": {"p10": q(plain, .1), "p50": q(plain, .5), "p90": q(plain, .9)},
                "sync_ms": {"p10": q(sync, .1), "p50": q(sync, .5), "p90": q(sync, .9)},
                "steps": n_ps}
@@ -569,11 +688,49 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(wl, hyper, args.cpu_seconds)
 
+    info = opt.info() if rank == 0 else None
+    headline_key = (wl.index, args.lookahead_mode)
+    plain_headline = not (prepass or args.layer_adaptation or args.bf16_copy or args.true_nesterov
+                          or args.adaptive_beta or mbytes == 2 or graph is not None)
+    per_workload = None
+    if rank == 0 and world == 1 and plain_headline and not args.no_per_workload:
+        # every other workload and lookahead mode, one after the other, each freed before the next
+        opt_cfg = {"chunk_elems": int(opt.handle.get_option(B.NOVAK_OPT_CHUNK_ELEMS)),
+                   "ctas_per_sm": int(opt.handle.get_option(B.NOVAK_OPT_CTAS_PER_SM)),
+                   "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
+                   "dependent_launch": int(opt.handle.get_option(B.NOVAK_OPT_DEPENDENT_LAUNCH))}
+        del opt, pool, pool_flat, pool_base, params, flat_p
+        torch.cuda.empty_cache()
+        per_workload = [{
+            "workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
+            "grad_dtype": "bf16" if gbytes == 2 else "f32", "lookahead_mode": args.lookahead_mode,
+            "lookahead_k": k, "steps": args.steps, "repeats": repeats, "ms_per_step": ms_per_step,
+            "p10": quantile(per_region, 0.1), "p90": quantile(per_region, 0.9),
+            "updates_per_s": value, "algorithmic_bytes_per_elem": alg, "hbm_gbs": achieved,
+            "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
+            "grad_pool": pool_n, "headline": True}]
+        free_bytes, _ = torch.cuda.mem_get_info()
+        for index in range(5):
+            for mode in ("last", "traj_mean"):
+                if (index, mode) == headline_key:
+                    continue
+                wl_i = W.get_workload(index)
+                if wl_i.total * 4 * 8 > free_bytes:
+                    per_workload.append({"workload": wl_i.name, "lookahead_mode": mode,
+                                         "skipped": "not enough free device memory"})
+                    continue
+                # large sets take fewer steps per region: a region of the 1 B set is 0.1 s
+                steps_i = args.steps if wl_i.total < 5e8 else min(args.steps, 20)
+                per_workload.append(time_one_workload(
+                    torch, B, W, dev, index, mode, steps_i, args.warmup, args.min_timed_seconds,
+                    args.max_repeats, args.pool, lib, barrier))
+
     if rank == 0:
-        info = opt.info()
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "repeats": repeats, "p10": quantile(per_region, 0.1), "p90": quantile(per_region, 0.9),
+            "timed_seconds": sum(region_ms) * 1e-3,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": wl.name, "params": wl.total, "tensors": len(wl.numel),
@@ -581,18 +738,21 @@ def main():
                 "lookahead_k": k, "lookahead_mode": args.lookahead_mode,
                 "clip_threshold": args.clip, "centralize": bool(args.centralize),
                 "layer_adaptation": bool(args.layer_adaptation),
+                "layer_adaptation_elements_read_twice": trust_share,
                 "adaptive_beta": bool(args.adaptive_beta), "bf16_copy": bool(args.bf16_copy),
-                "true_nesterov": bool(args.true_nesterov),
+                "true_nesterov": bool(args.true_nesterov), "restore_pass": bool(args.restore_pass),
                 "moment_dtype": args.moment_dtype,
                 "cuda_graph_steps": args.graph,
                 "auto_lr": bool(args.auto_lr),
-                "grad_pool": pool_n,
+                "grad_pool": pool_n, "grad_offset_elems": args.grad_offset,
+                "warnings": info["warnings"],
                 "l2": "no flush: working set %.2f GB per step rotates through %d gradient sets, "
                       "larger than the 126 MB L2" % (bytes_per_launch / 1e9, pool_n),
-                "chunk_elems": int(opt.handle.get_option(B.NOVAK_OPT_CHUNK_ELEMS)),
-                "ctas_per_sm": int(opt.handle.get_option(B.NOVAK_OPT_CTAS_PER_SM)),
-                "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
-                "dependent_launch": int(opt.handle.get_option(B.NOVAK_OPT_DEPENDENT_LAUNCH)),
+                **(opt_cfg if per_workload is not None else {
+                    "chunk_elems": int(opt.handle.get_option(B.NOVAK_OPT_CHUNK_ELEMS)),
+                    "ctas_per_sm": int(opt.handle.get_option(B.NOVAK_OPT_CTAS_PER_SM)),
+                    "serpentine": int(opt.handle.get_option(B.NOVAK_OPT_SERPENTINE)),
+                    "dependent_launch": int(opt.handle.get_option(B.NOVAK_OPT_DEPENDENT_LAUNCH))}),
                 "record_uploads_in_timed_region": uploads,
                 "grid": grid_timed, "block": info["block"], "n_chunks": info["n_chunks"],
                 "replicas": "each rank steps its own replica; no data-path collective",
@@ -604,6 +764,7 @@ def main():
                          "traffic": traffic,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "per_step": per,
+            "per_workload": per_workload,
             "e2e": e2e,
             "cpu_baseline": cpu,
             "gpu_launches": launches,

@@ -149,6 +149,26 @@ enum {
                                      NOVAK_ESTATE for any other variant             */
     NOVAK_OPT_MOMENT_DTYPE = 22,  /* NOVAK_MOMENT_*: storage type of m and v; only
                                      before attach (default NOVAK_MOMENT_F32)          */
+    NOVAK_OPT_CENTRALIZE_IN_STEP = 24, /* 1 (default): with centralization on and nothing
+                                     else that needs the whole gradient first (no
+                                     clipping, no automatic learning-rate scaling, no
+                                     layer adaptation), novak_step forms the row means
+                                     of Eq. 26 inside the step kernel, whose CTAs then
+                                     own whole rows (rows of up to 32768 elements;
+                                     longer ones keep the statistics pass): one launch
+                                     and 28 B per element instead of three launches and
+                                     32 B.  0: always the statistics pass              */
+    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1 (default): with layer adaptation on and no
+                                     clipping, centralization or automatic learning-
+                                     rate scaling, novak_step runs statistics and
+                                     update as ONE kernel in which a tensor's update
+                                     follows its statistics closely enough to find its
+                                     theta, g, m, v still in L2 (about 28 B per
+                                     element from DRAM instead of 44).  0: two
+                                     statistics kernels, then the step                */
+    NOVAK_OPT_LAYER_ADAPTATION_LEAD = 26, /* how far, in elements, that kernel's statistics
+                                     run ahead of its updates (default 2^21: 32 MB of
+                                     theta, g, m, v); only before the first such step */
     NOVAK_OPT_GRAPH_CAPTURABLE = 23, /* Without it every step entry point returns
                                      NOVAK_ESTATE while its stream is being captured (a
                                      replay would repeat ONE step's scalars).
@@ -182,8 +202,13 @@ enum {
 enum {
     NOVAK_WARN_TRUE_DOWNGRADED = 1u, /* nesterov_variant TRUE runs as APPROX from the
                                         first step (N_taylor = 0)                      */
-    NOVAK_WARN_SCALAR_PATH = 2u      /* some tensor's pointers do not share 16-byte
-                                        alignment; it runs on 4-byte accesses          */
+    NOVAK_WARN_SCALAR_PATH = 2u,     /* some tensor's parameter, state (or bf16 copy)
+                                        pointers do not share 16-byte alignment; it
+                                        runs on 4-byte accesses                        */
+    NOVAK_WARN_NARROW_GRADIENT = 4u  /* some tensor's gradient sits at another offset
+                                        from a 16-byte boundary than its parameter; its
+                                        gradient is fetched element by element while
+                                        parameter and state keep 128-bit accesses      */
 };
 
 /* Read-only view of the handle after the last successful step. */
@@ -300,8 +325,10 @@ int novak_attach_state(novak_opt *opt, void *d_state, size_t bytes,
  * of the 8 most recently used (params, grads) pointer lists, so a caller that
  * cycles through a few gradient buffers enqueues nothing but the kernel; a list
  * it does not hold is uploaded in stream order (novak_info.record_uploads).  Tensors whose parameter, gradient and state
- * addresses are congruent modulo 16 bytes run on 128-bit accesses; others on
- * 4-byte accesses (NOVAK_WARN_SCALAR_PATH).
+ * addresses are congruent modulo 16 bytes run on 128-bit accesses; where only
+ * the gradient is off, it alone is fetched element by element
+ * (NOVAK_WARN_NARROW_GRADIENT); where parameter and state disagree the tensor
+ * runs on 4-byte accesses (NOVAK_WARN_SCALAR_PATH).
  * Errors: NOVAK_EINVAL (NULL, n mismatch, bad dtype, misaligned pointer),
  * NOVAK_ESTATE (no state attached), NOVAK_ENOMEM, NOVAK_ECUDA.  On any error
  * nothing is enqueued and t is unchanged. */
@@ -467,6 +494,17 @@ int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
  *   novak_nesterov_restore       theta <- save
  *   novak_step(..., that gradient)      (no Eq. 13 correction while t <= N_taylor)
  *
+ * or, one pass and 8 bytes per element less, without the restore:
+ *
+ *   novak_nesterov_extrapolate
+ *   ... the caller's forward and backward pass at theta~ ...
+ *   novak_step(..., that gradient)      reads theta_{t-1} from the save buffer and
+ *                                       writes theta_t over theta~ in the parameters
+ *
+ * (novak_step only, with the d_params of the extrapolate call; the result is bit
+ * for bit that of the three-call form.  novak_nesterov_restore stays for callers
+ * that abandon the step.)
+ *
  * One kernel each over the handle's chunk table, enqueued on `stream` (a
  * cudaStream_t; NULL: the default stream); no host synchronisation.  In fp32:
  * one fused multiply-add per element; the restored parameters are bit for bit
@@ -477,8 +515,9 @@ int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
  * bytes, of at least novak_nesterov_save_bytes() bytes (0 before attach; the
  * size of one state array), laid out like a state array; it must stay valid
  * and unchanged until the restore, which takes the same d_params and d_save.
- * Between the two calls every step entry point, novak_import_meta and
- * NOVAK_OPT_TRUE_NESTEROV_STEPS return NOVAK_ESTATE.  m_{t-1} = 0 before the
+ * Between extrapolate and restore novak_import_meta,
+ * NOVAK_OPT_TRUE_NESTEROV_STEPS and every step entry point other than
+ * novak_step return NOVAK_ESTATE.  m_{t-1} = 0 before the
  * first step, so the first look-ahead leaves theta where it is.
  * Errors: NOVAK_EINVAL (NULL, a misaligned or short buffer, restore with other
  * buffers), NOVAK_ESTATE (not attached, wrong variant, a tensor list other
@@ -543,6 +582,27 @@ int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,
 int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
                               int64_t *row0, int64_t *n_rows, int64_t *part_off,
                               int64_t *part_len, int64_t cap);
+
+/* Host-only helper exposing the units of the step kernel that centralizes by
+ * itself (NOVAK_OPT_CENTRALIZE_IN_STEP): whole rows [row0, row0 + n_rows) of the
+ * tensors whose rows have at most 32768 elements, as many rows as fit in 4096
+ * elements (at least one, at most 256) per unit; tensors with longer rows get
+ * no unit (they keep the statistics pass).  Arguments and result as in
+ * novak_build_row_units. */
+int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
+                              int64_t *row0, int64_t *n_rows, int64_t cap);
+
+/* Host-only helper exposing the order in which the one-launch form of layer
+ * adaptation (NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) takes its items.  The group's
+ * chunk table lists tensor i's entries at [tensor_first[i], tensor_first[i+1])
+ * (n + 1 values, non-decreasing, tensor_first[0] = 0).  out[k] is the k-th item:
+ * a chunk-table index for a statistics item, the index | 0x80000000 for an
+ * update item.  Tensor after tensor emits its statistics items; a tensor's
+ * update items follow once at least lead_items further items stand behind its
+ * last statistics item.  Writes up to cap items and returns the number of items
+ * (2 x tensor_first[n]; negative on bad arguments). */
+int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_items,
+                                int32_t *out, int64_t cap);
 
 /* Text of the last error on this handle ("" if none).  Owned by the handle. */
 const char *novak_last_error(const novak_opt *opt);

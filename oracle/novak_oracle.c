@@ -65,8 +65,8 @@
  *     N_taylor + 1 on the variant is the approximation of Eq. 13 (Section 5.2's
  *     automatic fallback).                                 [parity unpinned]
  *
- *   - Moments stored in bfloat16 (Section 10's "storing moments in bfloat16
- *     while accumulating updates in float32", named as future work): m_{t-1}
+ *   - Moments stored in bfloat16 (Section 10 names bfloat16 storage of the
+ *     moments, with the arithmetic kept in float32, as future work): m_{t-1}
  *     and v_{t-1} are read back as stored, the step's own arithmetic (Eq. 1-2,
  *     5, 17) runs on the unrounded m_t, v_t, and what is stored for the next
  *     step is each of them rounded to the nearest bfloat16 (8 significant
@@ -74,7 +74,10 @@
  *     rounding nor whether the step sees rounded values.   [parity unpinned]
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, torch.optim.AdamW/RAdam
- * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5).
+ * special cases, unrolled-sum brute force, invariants of Prop. 6.3-6.5); every
+ * function of this file has a pin, novak_oracle_direction included (against the
+ * pinned step: with alpha = 1, no decay and no rectification the step moves
+ * every parameter by exactly -u).
  */
 #include <math.h>
 #include <stdint.h>

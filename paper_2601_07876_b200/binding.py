@@ -30,9 +30,10 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_CLIP_THRESHOLD, NOVAK_OPT_CENTRALIZE, NOVAK_OPT_ADAPTIVE_BETA, NOVAK_OPT_BETA1_TAU,
  NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
  NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS, NOVAK_OPT_MOMENT_DTYPE,
- NOVAK_OPT_GRAPH_CAPTURABLE) = range(1, 24)
+ NOVAK_OPT_GRAPH_CAPTURABLE, NOVAK_OPT_CENTRALIZE_IN_STEP, NOVAK_OPT_LAYER_ADAPTATION_IN_STEP,
+ NOVAK_OPT_LAYER_ADAPTATION_LEAD) = range(1, 27)
 NOVAK_MOMENT_F32, NOVAK_MOMENT_BF16 = 0, 1
-NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH = 1, 2
+NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH, NOVAK_WARN_NARROW_GRADIENT = 1, 2, 4
 
 _STATUS = {0: "NOVAK_OK", 1: "NOVAK_EINVAL", 2: "NOVAK_ESTATE", 3: "NOVAK_ECUDA", 4: "NOVAK_ENOMEM"}
 
@@ -132,6 +133,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_import_meta": (c_int, [vp, POINTER(novak_meta)]),
         "novak_build_chunks": (c_int64, [i64p, POINTER(c_int32), c_int, c_int64,
                                          POINTER(c_int32), i64p, POINTER(c_int32), c_int64]),
+        "novak_build_own_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, c_int64]),
+        "novak_build_adapt_order": (c_int64, [POINTER(c_int32), c_int, c_int64, POINTER(c_int32),
+                                              c_int64]),
         "novak_build_row_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, i64p,
                                             i64p, c_int64]),
         "novak_last_error": (c_char_p, [vp]),
@@ -187,6 +191,35 @@ def novak_build_row_units(numel, rows, lib=None):
     cols = [(c_int64 * need)() for _ in range(4)]
     lib.novak_build_row_units(num, rw, n, t, *cols, need)
     return list(zip(list(t), *[list(c) for c in cols]))
+
+
+def novak_build_own_units(numel, rows, lib=None):
+    """Host-only: the units of the step kernel that centralizes by itself, as a list of
+    (tensor, row0, n_rows)."""
+    lib = lib or load_library()
+    n = len(numel)
+    num, rw = i64_array(numel), i64_array(rows)
+    need = lib.novak_build_own_units(num, rw, n, None, None, None, 0)
+    if need < 0:
+        raise NovakError(NOVAK_EINVAL, "novak_build_own_units")
+    t = (c_int32 * need)()
+    cols = [(c_int64 * need)() for _ in range(2)]
+    lib.novak_build_own_units(num, rw, n, t, *cols, need)
+    return list(zip(list(t), *[list(c) for c in cols]))
+
+
+def novak_build_adapt_order(tensor_first, lead_items, lib=None):
+    """Host-only: the item order of the one-launch layer adaptation, as a list of
+    (chunk index, is_update)."""
+    lib = lib or load_library()
+    n = len(tensor_first) - 1
+    first = (c_int32 * (n + 1))(*tensor_first)
+    need = lib.novak_build_adapt_order(first, n, lead_items, None, 0)
+    if need < 0:
+        raise NovakError(NOVAK_EINVAL, "novak_build_adapt_order")
+    out = (c_int32 * need)()
+    lib.novak_build_adapt_order(first, n, lead_items, out, need)
+    return [(v & 0x7fffffff, v < 0) for v in out]
 
 
 _NESTEROV = {"none": NOVAK_NESTEROV_NONE, "approximation": NOVAK_NESTEROV_APPROX,
@@ -397,7 +430,8 @@ class NovakOptimizer:
                  clip_threshold=0.0, centralize=False, adaptive_beta=False, tau1=None, tau2=None,
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
                  auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0, moment_dtype="f32",
-                 graph_capturable=False,
+                 graph_capturable=False, centralize_in_step=None, layer_adaptation_in_step=None,
+                 layer_adaptation_lead=None,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -425,6 +459,12 @@ class NovakOptimizer:
         h.set_option(NOVAK_OPT_BIAS1_POWER, bias1_power)
         if graph_capturable:
             h.set_option(NOVAK_OPT_GRAPH_CAPTURABLE, 1)
+        if layer_adaptation_in_step is not None:
+            h.set_option(NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 1 if layer_adaptation_in_step else 0)
+        if layer_adaptation_lead is not None:
+            h.set_option(NOVAK_OPT_LAYER_ADAPTATION_LEAD, layer_adaptation_lead)
+        if centralize_in_step is not None:
+            h.set_option(NOVAK_OPT_CENTRALIZE_IN_STEP, 1 if centralize_in_step else 0)
         if chunk_elems is not None:
             h.set_option(NOVAK_OPT_CHUNK_ELEMS, chunk_elems)
         if ctas_per_sm is not None:
@@ -493,7 +533,9 @@ class NovakOptimizer:
                                          self._stream())
 
     def restore(self):
-        """Puts the parameters saved by extrapolate() back, bit for bit."""
+        """Puts the parameters saved by extrapolate() back, bit for bit.  Only needed when
+        the step is abandoned: step() called directly after extrapolate() reads the saved
+        parameters itself."""
         self.handle.nesterov_restore(self._params_arr, self._save.data_ptr(), self._save.numel(),
                                      self._numel_arr, self.n, self._stream())
 
@@ -540,6 +582,21 @@ class NovakOptimizer:
             return raw[0](raw[1])
         import torch
         return torch.cuda.current_stream(self.device).cuda_stream
+
+    def rebind_params(self, params):
+        """The same parameters at new addresses (tensors that were moved or re-created):
+        later steps take these pointers; the attached state stays as it is.  State
+        slices keep the alignment phase of the tensors given at construction, so
+        tensors at another offset from a 16-byte boundary run on narrow accesses."""
+        params = list(params)
+        if [p.numel() for p in params] != self.numel:
+            raise ValueError("parameter shapes do not match the attached layout")
+        for p in params:
+            if p.dtype != self.params[0].dtype or not p.is_cuda or not p.is_contiguous():
+                raise ValueError("parameters must be contiguous float32 CUDA tensors")
+        self.params = params
+        self._param_ptrs = [p.data_ptr() for p in params]
+        self._params_arr = ptr_array(self._param_ptrs)
 
     def prepare(self, grads) -> GradList:
         gl = GradList(grads)

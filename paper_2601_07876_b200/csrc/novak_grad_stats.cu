@@ -439,7 +439,7 @@ novak_param_sumsq_kernel(const Chunk *__restrict__ chunks, int n_chunks,
 #pragma unroll
     for (int k = 0; k < K; ++k) ch[k] = chunks[min(c0 + k, n_chunks - 1)];
 #pragma unroll
-    for (int k = 0; k < K; ++k) p[k] = recs[ch[k].tensor].p + ch[k].offset;
+    for (int k = 0; k < K; ++k) p[k] = recs[ch[k].tensor].p_in + ch[k].offset;
     grid_dependency_wait();          // the parameters come from the previous step
     double sq = 0.0;
 #pragma unroll

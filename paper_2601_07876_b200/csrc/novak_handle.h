@@ -70,6 +70,7 @@ struct Handle {
     struct RecTable {
         std::vector<void *> p;
         std::vector<const void *> g;
+        const void *save = nullptr;   // save buffer theta_{t-1} is read from (NULL: the parameters)
         int gdtype = -1;
         uint64_t hash = 0;
         int64_t last_use = 0;
@@ -88,6 +89,13 @@ struct Handle {
     Chunk *d_plain = nullptr;           // entries of the tensors without rows (NULL: all of them)
     RowUnit *d_units = nullptr;
     int n_plain = 0, n_units = 0;
+    // step kernel that forms the row means itself (PRE_CENTER_ROWS): the chunk-table
+    // entries of the tensors it does not own rows of, and its units of whole rows
+    int center_in_step = 1;             // NOVAK_OPT_CENTRALIZE_IN_STEP
+    bool prep_rows_layout = false;      // the scratch is laid out for that kernel
+    Chunk *d_rest = nullptr;
+    RowUnit *d_own = nullptr;
+    int n_rest = 0, n_own = 0;
     int64_t rows_gen = 0;               // bumped whenever the row settings change
     int64_t prep_key = -1;              // rows_gen and centring the scratch was laid out for
     // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
@@ -118,6 +126,20 @@ struct Handle {
     int *tensor_first = nullptr;
     float *trust = nullptr;
     std::vector<int> h_tensor_first;
+    // layer adaptation and step in one launch: the claim-ordered item list, the
+    // kernel's counters and per-tensor flags (one allocation), a host-mapped error word
+    int adapt_in_step = 1;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
+    int64_t adapt_lead_elems = 1 << 21;    // NOVAK_OPT_LAYER_ADAPTATION_LEAD
+    char *d_adapt = nullptr;
+    int *d_item_code = nullptr;
+    Chunk *d_item_chunk = nullptr;
+    int n_items = 0;
+    novak::AdaptCtl *adapt_ctl = nullptr;
+    unsigned *adapt_arrived = nullptr;
+    unsigned long long *adapt_ready = nullptr;
+    unsigned *h_adapt_error = nullptr;  // pinned, mapped; written by the kernel
+    unsigned *d_adapt_error = nullptr;  // its device address
+    unsigned adapt_epoch = 0;
 
     // novak_step_host: the chunk table cut into segments, each with the element
     // ranges it covers, two copy streams and the events that order them.
@@ -150,6 +172,10 @@ int64_t round_up(int64_t x, int64_t a);
 void build_chunks(const int64_t *numel, const int32_t *phase, int n, int64_t chunk_elems,
                   std::vector<Chunk> &out);
 void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out);
+// Units of the step kernel that owns rows: whole rows of the tensors whose rows
+// have at most novak::kOwnRowMax elements, about novak::kOwnUnitElems elements
+// and at most novak::kOwnUnitRows rows per unit.
+void build_own_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out);
 int check_hyper(const Hyper &h, const char **why);
 
 // The variant the kernels are instantiated for: a true step's gradient needs no
@@ -190,17 +216,32 @@ inline int moment_bytes(const Hyper &h) { return h.mom16 ? 2 : 4; }
 // Bytes of the whole state for a region of `region_elems` padded elements.
 size_t state_bytes_for(const Hyper &h, int64_t region_elems);
 int pre_mode(const novak_opt *o);
+// The mode a step actually runs in: pre_mode, or PRE_CENTER_ROWS where the step
+// kernel can centralize by itself (whole_table: the step is one launch over the
+// whole group, as in novak_step).
+int step_pre_mode(const novak_opt *o, bool whole_table);
+int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream);
 void fill_info(const novak_opt *o, const Plan &p, novak_info *out);
 
 // Device work tables (novak_host_device.cpp).
 void release_device(novak_opt *o);
 int prepare_device(novak_opt *o, cudaStream_t stream);
 void invalidate_tables(novak_opt *o);
-int prepare_prep(novak_opt *o, cudaStream_t stream);
 int prepare_trust(novak_opt *o, cudaStream_t stream);
-uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype);
+// The item list and counters of the one-launch form of layer adaptation.
+int prepare_adapt(novak_opt *o, cudaStream_t stream);
+// Claim order of that kernel.  Tensor after tensor emits its S items (chunk-
+// table index); a tensor's U items (index | 0x80000000) follow once at least
+// `lead_items` further items have been emitted behind its last S item, tensors
+// in order; what is still pending at the end follows in order.
+void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_items,
+                       std::vector<int32_t> &items);
+uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype,
+                       const void *save);
+// `save`: NULL, or the save buffer of an open look-ahead, from which the step
+// then reads theta_{t-1} (the parameter tensors hold Eq. 10's point).
 int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
-                    int grad_dtype, cudaStream_t stream);
+                    int grad_dtype, const void *save, cudaStream_t stream);
 // Device records of the look-ahead helpers for this parameter list (uploaded
 // only when the list differs from the one the device holds).
 int prepare_look(novak_opt *o, void *const *d_params, cudaStream_t stream);

@@ -73,6 +73,41 @@ void build_row_units(const int64_t *numel, const int64_t *rows, int n, std::vect
 }
 
 
+void build_own_units(const int64_t *numel, const int64_t *rows, int n, std::vector<RowUnit> &out)
+{
+    out.clear();
+    for (int i = 0; i < n; ++i) {
+        if (rows[i] <= 0) continue;
+        const uint32_t R = static_cast<uint32_t>(rows[i]);
+        const uint32_t L = static_cast<uint32_t>(numel[i] / rows[i]);
+        if (L == 0 || L > novak::kOwnRowMax) continue;
+        const uint32_t per = std::max(1u, std::min(novak::kOwnUnitRows, novak::kOwnUnitElems / L));
+        for (uint32_t r = 0; r < R; r += per)
+            out.push_back(RowUnit{i, r, std::min(per, R - r), 0u, 0u, 1u, 0u, 0u});
+    }
+}
+
+void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_items,
+                       std::vector<int32_t> &items)
+{
+    items.clear();
+    if (n <= 0) return;
+    items.reserve(2 * static_cast<size_t>(tensor_first[n]));
+    const int32_t kUpdate = static_cast<int32_t>(0x80000000u);
+    std::vector<int64_t> s_end(n, 0);   // items emitted when tensor i's last S item was
+    int pending = 0;                    // first tensor whose U items are still to come
+    auto emit_updates = [&](int i) {
+        for (int c = tensor_first[i]; c < tensor_first[i + 1]; ++c) items.push_back(c | kUpdate);
+    };
+    for (int i = 0; i < n; ++i) {
+        for (int c = tensor_first[i]; c < tensor_first[i + 1]; ++c) items.push_back(c);
+        s_end[i] = static_cast<int64_t>(items.size());
+        while (pending <= i && static_cast<int64_t>(items.size()) - s_end[pending] >= lead_items)
+            emit_updates(pending++);
+    }
+    while (pending < n) emit_updates(pending++);
+}
+
 int fail(novak_opt *o, int code, const char *fmt, ...)
 {
     if (o) {
@@ -120,6 +155,15 @@ int pre_mode(const novak_opt *o)
     if (o->h.centralize && o->total_rows > 0) return novak::PRE_CENTER;
     if (o->h.clip > 0.0 || o->h.auto_lr) return novak::PRE_SCALE;
     return novak::PRE_NONE;
+}
+
+int step_pre_mode(const novak_opt *o, bool whole_table)
+{
+    const int pre = pre_mode(o);
+    if (pre == novak::PRE_CENTER && whole_table && o->center_in_step && !o->dyn &&
+        !(o->h.clip > 0.0) && !o->h.auto_lr && !o->h.layer_adapt)
+        return novak::PRE_CENTER_ROWS;
+    return pre;
 }
 
 void fill_info(const novak_opt *o, const Plan &p, novak_info *out)
@@ -294,6 +338,20 @@ int novak_set_option(novak_opt *o, int key, double value)
         if (h.centralize != static_cast<int>(value)) invalidate_tables(o);
         h.centralize = static_cast<int>(value);
         break;
+    case NOVAK_OPT_LAYER_ADAPTATION_IN_STEP:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "layer_adaptation_in_step must be 0 or 1");
+        o->adapt_in_step = static_cast<int>(value);
+        return NOVAK_OK;
+    case NOVAK_OPT_LAYER_ADAPTATION_LEAD:
+        if (o->d_adapt) return fail(o, NOVAK_ESTATE, "the lead is fixed once a step with layer adaptation was taken");
+        if (!(value >= 0.0 && value <= 1073741824.0) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "layer_adaptation_lead must be an integer in [0, 2^30]");
+        o->adapt_lead_elems = static_cast<int64_t>(value);
+        return NOVAK_OK;
+    case NOVAK_OPT_CENTRALIZE_IN_STEP:
+        if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "centralize_in_step must be 0 or 1");
+        o->center_in_step = static_cast<int>(value);
+        return NOVAK_OK;
     case NOVAK_OPT_GRAPH_CAPTURABLE:
         if (o->t > 0) return fail(o, NOVAK_ESTATE, "graph_capturable is fixed once a step was taken");
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "graph_capturable must be 0 or 1");
@@ -358,6 +416,9 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_CLIP_THRESHOLD: *value = o->h.clip; break;
     case NOVAK_OPT_CENTRALIZE: *value = o->h.centralize; break;
     case NOVAK_OPT_GRAPH_CAPTURABLE: *value = o->dyn; break;
+    case NOVAK_OPT_CENTRALIZE_IN_STEP: *value = o->center_in_step; break;
+    case NOVAK_OPT_LAYER_ADAPTATION_IN_STEP: *value = o->adapt_in_step; break;
+    case NOVAK_OPT_LAYER_ADAPTATION_LEAD: *value = static_cast<double>(o->adapt_lead_elems); break;
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
@@ -636,6 +697,40 @@ int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, 
         if (part_off) part_off[i] = units[i].part_off;
         if (part_len) part_len[i] = units[i].part_len;
     }
+    return count;
+}
+
+int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
+                              int64_t *row0, int64_t *n_rows, int64_t cap)
+{
+    if (!numel || !rows || n <= 0 || cap < 0) return -1;
+    for (int i = 0; i < n; ++i)
+        if (numel[i] <= 0 || rows[i] < 0 || (rows[i] > 0 && (numel[i] % rows[i] != 0 ||
+                                                             numel[i] >= (int64_t(1) << 31))))
+            return -1;
+    std::vector<RowUnit> units;
+    build_own_units(numel, rows, n, units);
+    const int64_t count = static_cast<int64_t>(units.size());
+    for (int64_t i = 0; i < count && i < cap; ++i) {
+        if (tensor) tensor[i] = units[i].tensor;
+        if (row0) row0[i] = units[i].row0;
+        if (n_rows) n_rows[i] = units[i].n_rows;
+    }
+    return count;
+}
+
+int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_items,
+                                int32_t *out, int64_t cap)
+{
+    if (!tensor_first || n <= 0 || lead_items < 0 || cap < 0 || tensor_first[0] != 0) return -1;
+    for (int i = 0; i < n; ++i)
+        if (tensor_first[i + 1] < tensor_first[i]) return -1;
+    std::vector<int> first(tensor_first, tensor_first + n + 1);
+    std::vector<int32_t> items;
+    build_adapt_items(first, n, lead_items, items);
+    const int64_t count = static_cast<int64_t>(items.size());
+    for (int64_t i = 0; i < count && i < cap; ++i)
+        if (out) out[i] = items[i];
     return count;
 }
 

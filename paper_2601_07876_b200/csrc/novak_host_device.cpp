@@ -35,6 +35,16 @@ void release_device(novak_opt *o)
     o->look_p.clear();
     o->look_save = nullptr;
     o->extrapolated = false;
+    if (o->d_adapt) cudaFree(o->d_adapt);
+    if (o->h_adapt_error) cudaFreeHost(o->h_adapt_error);
+    o->d_adapt = nullptr;
+    o->d_item_code = nullptr;
+    o->d_item_chunk = nullptr;
+    o->n_items = 0;
+    o->adapt_ctl = nullptr;
+    o->adapt_arrived = nullptr;
+    o->adapt_ready = nullptr;
+    o->h_adapt_error = o->d_adapt_error = nullptr;
     if (o->d_trust) cudaFree(o->d_trust);
     o->d_trust = nullptr;
     o->chunk_u2 = o->chunk_p2 = nullptr;
@@ -126,10 +136,10 @@ void invalidate_tables(novak_opt *o)
 
 // Scratch of the statistics pass, laid out when a step first needs it and
 // again when the row settings change.
-int prepare_prep(novak_opt *o, cudaStream_t stream)
+int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream)
 {
     const bool centre = o->h.centralize && o->total_rows > 0;
-    const int64_t key = o->rows_gen * 2 + (centre ? 1 : 0);
+    const int64_t key = o->rows_gen * 4 + (centre ? 1 : 0) + (rows_layout ? 2 : 0);
     if (o->d_prep && o->prep_key == key) return NOVAK_OK;
     cudaError_t e;
     if (o->d_prep) {
@@ -147,15 +157,29 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
         invalidate_tables(o);
     }
     // work of the pass: row units for the tensors with rows, chunk-table entries for the rest
-    std::vector<RowUnit> units;
-    std::vector<Chunk> plain;
-    if (centre) {
+    std::vector<RowUnit> units, own;
+    std::vector<Chunk> plain, rest;
+    if (centre && rows_layout) {
+        // The step kernel owns the rows of up to kOwnRowMax elements.  The statistics
+        // pass shrinks to the tensors with longer rows (no norm is needed: nothing for
+        // its plain part); the step kernel takes those tensors, and the ones without
+        // rows, by chunk-table entries.
+        build_own_units(o->numel.data(), o->rows.data(), o->n, own);
+        std::vector<int64_t> long_rows(o->rows.size(), 0);
+        for (int i = 0; i < o->n; ++i)
+            if (o->rows[i] > 0 && o->numel[i] / o->rows[i] > static_cast<int64_t>(novak::kOwnRowMax))
+                long_rows[i] = o->rows[i];
+        build_row_units(o->numel.data(), long_rows.data(), o->n, units);
+        for (const Chunk &c : o->h_chunks)
+            if (o->rows[c.tensor] <= 0 || long_rows[c.tensor] > 0) rest.push_back(c);
+    } else if (centre) {
         build_row_units(o->numel.data(), o->rows.data(), o->n, units);
         for (const Chunk &c : o->h_chunks)
             if (o->rows[c.tensor] <= 0) plain.push_back(c);
     }
     const size_t n_plain = centre ? plain.size() : static_cast<size_t>(o->n_chunks);
-    if (units.size() > static_cast<size_t>(INT32_MAX) / 2) return fail(o, NOVAK_EINVAL, "too many rows");
+    if (units.size() > static_cast<size_t>(INT32_MAX) / 2 || own.size() > static_cast<size_t>(INT32_MAX) / 2)
+        return fail(o, NOVAK_EINVAL, "too many rows");
     // sized for fp32 gradients; bf16 gradients take more entries per CTA and need less
     const size_t n_work = static_cast<size_t>(novak::grad_stats_work(
         static_cast<int>(n_plain), static_cast<int>(units.size()), NOVAK_GRAD_F32));
@@ -168,7 +192,9 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
     const size_t off_cta = off;     off += 2 * ctas * sizeof(double);
     off = (off + 15) / 16 * 16;
     const size_t off_plain = off;   off += plain.size() * sizeof(Chunk);
+    const size_t off_rest = off;    off += rest.size() * sizeof(Chunk);
     const size_t off_units = off;   off += units.size() * sizeof(RowUnit);
+    const size_t off_own = off;     off += own.size() * sizeof(RowUnit);
     const size_t off_mean = off;    off += static_cast<size_t>(o->total_rows) * sizeof(float2);
     const size_t bytes = off + 16;
     if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
@@ -183,18 +209,31 @@ int prepare_prep(novak_opt *o, cudaStream_t stream)
     o->chunk_psq = reinterpret_cast<double *>(o->d_prep + off_psq);
     o->cta_sq = reinterpret_cast<double *>(o->d_prep + off_cta);
     o->d_plain = centre ? reinterpret_cast<Chunk *>(o->d_prep + off_plain) : nullptr;
+    o->d_rest = reinterpret_cast<Chunk *>(o->d_prep + off_rest);
     o->d_units = reinterpret_cast<RowUnit *>(o->d_prep + off_units);
+    o->d_own = reinterpret_cast<RowUnit *>(o->d_prep + off_own);
     o->row_mean = reinterpret_cast<float2 *>(o->d_prep + off_mean);
-    o->n_plain = static_cast<int>(n_plain);
+    o->n_plain = (centre && rows_layout) ? 0 : static_cast<int>(n_plain);
     o->n_units = static_cast<int>(units.size());
+    o->n_rest = static_cast<int>(rest.size());
+    o->n_own = static_cast<int>(own.size());
+    o->prep_rows_layout = centre && rows_layout;
     // The tables are built once per layout: blocking copies keep the host
     // vectors' lifetime trivial.
     if (!plain.empty() &&
         (e = cudaMemcpyAsync(o->d_plain, plain.data(), plain.size() * sizeof(Chunk),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return fail_cuda(o, e, "statistics table upload");
+    if (!rest.empty() &&
+        (e = cudaMemcpyAsync(o->d_rest, rest.data(), rest.size() * sizeof(Chunk),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "step table upload");
     if (!units.empty() &&
         (e = cudaMemcpyAsync(o->d_units, units.data(), units.size() * sizeof(RowUnit),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+        return fail_cuda(o, e, "row unit upload");
+    if (!own.empty() &&
+        (e = cudaMemcpyAsync(o->d_own, own.data(), own.size() * sizeof(RowUnit),
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess)
         return fail_cuda(o, e, "row unit upload");
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail_cuda(o, e, "statistics table upload");
@@ -228,6 +267,56 @@ int prepare_trust(novak_opt *o, cudaStream_t stream)
                              cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
         (e = cudaStreamSynchronize(stream)) != cudaSuccess)
         return fail_cuda(o, e, "layer adaptation table upload");
+    return NOVAK_OK;
+}
+
+// Item list, counters and flags of the kernel that adapts and steps in one
+// launch; allocated when a step first needs them (after prepare_trust).
+int prepare_adapt(novak_opt *o, cudaStream_t stream)
+{
+    if (o->d_adapt) return NOVAK_OK;
+    std::vector<int32_t> codes;
+    const int64_t lead_items = (o->adapt_lead_elems + o->chunk_elems - 1) / o->chunk_elems;
+    build_adapt_items(o->h_tensor_first, o->n, lead_items, codes);
+    if (codes.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
+    std::vector<Chunk> entries(codes.size());
+    for (size_t k = 0; k < codes.size(); ++k) entries[k] = o->h_chunks[codes[k] & 0x7fffffff];
+    const size_t n = static_cast<size_t>(o->n);
+    const size_t off_ready = 256;
+    const size_t off_arrived = off_ready + n * sizeof(unsigned long long);
+    const size_t off_chunk = (off_arrived + n * sizeof(unsigned) + 15) / 16 * 16;
+    const size_t off_code = off_chunk + entries.size() * sizeof(Chunk);
+    const size_t bytes = off_code + codes.size() * sizeof(int32_t) + 16;
+    cudaError_t e;
+    if (!o->h_adapt_error) {
+        if ((e = cudaHostAlloc(reinterpret_cast<void **>(&o->h_adapt_error), sizeof(unsigned),
+                               cudaHostAllocMapped)) != cudaSuccess) {
+            o->h_adapt_error = nullptr;
+            return fail(o, NOVAK_ENOMEM, "cudaHostAlloc(error word): %s", cudaGetErrorString(e));
+        }
+        *o->h_adapt_error = 0u;
+        if ((e = cudaHostGetDevicePointer(reinterpret_cast<void **>(&o->d_adapt_error),
+                                          o->h_adapt_error, 0)) != cudaSuccess)
+            return fail_cuda(o, e, "cudaHostGetDevicePointer(error word)");
+    }
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_adapt), bytes)) != cudaSuccess) {
+        o->d_adapt = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(layer adaptation items, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    o->adapt_ctl = reinterpret_cast<novak::AdaptCtl *>(o->d_adapt);
+    o->adapt_arrived = reinterpret_cast<unsigned *>(o->d_adapt + off_arrived);
+    o->adapt_ready = reinterpret_cast<unsigned long long *>(o->d_adapt + off_ready);
+    o->d_item_chunk = reinterpret_cast<Chunk *>(o->d_adapt + off_chunk);
+    o->d_item_code = reinterpret_cast<int *>(o->d_adapt + off_code);
+    o->n_items = static_cast<int>(codes.size());
+    // built once: blocking copies keep the host vectors' lifetime trivial
+    if ((e = cudaMemsetAsync(o->d_adapt, 0, off_chunk, stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(o->d_item_chunk, entries.data(), entries.size() * sizeof(Chunk),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(o->d_item_code, codes.data(), codes.size() * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(stream)) != cudaSuccess)
+        return fail_cuda(o, e, "layer adaptation item upload");
     return NOVAK_OK;
 }
 
@@ -321,9 +410,11 @@ int read_dyn(const novak_opt *o, novak::DevPlan *out)
     return NOVAK_OK;
 }
 
-uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype)
+uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype,
+                       const void *save)
 {
     uint64_t h = 0xcbf29ce484222325ull ^ static_cast<uint64_t>(grad_dtype);
+    h = (h ^ reinterpret_cast<uintptr_t>(save)) * 0x100000001b3ull;
     for (int i = 0; i < n; ++i) {
         h = (h ^ reinterpret_cast<uintptr_t>(d_params[i])) * 0x100000001b3ull;
         h = (h ^ reinterpret_cast<uintptr_t>(d_grads[i])) * 0x100000001b3ull;
@@ -335,14 +426,14 @@ uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n,
 // uploading them (in stream order, into the least recently used table) when
 // none does.
 int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_grads,
-                    int grad_dtype, cudaStream_t stream)
+                    int grad_dtype, const void *save, cudaStream_t stream)
 {
     const int n = o->n;
-    const uint64_t hash = hash_pointers(d_params, d_grads, n, grad_dtype);
+    const uint64_t hash = hash_pointers(d_params, d_grads, n, grad_dtype, save);
     int lru = 0;
     for (int k = 0; k < kRecTables; ++k) {
         novak_opt::RecTable &tb = o->tables[k];
-        if (tb.gdtype == grad_dtype && tb.hash == hash && !tb.p.empty() &&
+        if (tb.gdtype == grad_dtype && tb.hash == hash && tb.save == save && !tb.p.empty() &&
             std::memcmp(tb.p.data(), d_params, n * sizeof(void *)) == 0 &&
             std::memcmp(tb.g.data(), d_grads, n * sizeof(void *)) == 0) {
             tb.last_use = ++o->table_clock;
@@ -354,18 +445,21 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
 
     const uintptr_t gmask = grad_dtype == NOVAK_GRAD_BF16 ? 1u : 3u;
     const uintptr_t gvec = grad_dtype == NOVAK_GRAD_BF16 ? 8u : 16u;
-    bool scalar_path = false;
+    bool scalar_path = false, narrow_grad = false;
     for (int i = 0; i < n; ++i) {
         const uintptr_t p = reinterpret_cast<uintptr_t>(d_params[i]);
         const uintptr_t g = reinterpret_cast<uintptr_t>(d_grads[i]);
         if (!p || !g) return fail(o, NOVAK_EINVAL, "tensor %d: NULL pointer", i);
         if ((p & 3u) || (g & gmask)) return fail(o, NOVAK_EINVAL, "tensor %d: pointer not aligned to its element size", i);
-        // 128-bit path needs parameter, state and gradient congruent mod 16 B
-        // (bf16 moments: 8-byte accesses at half the parameter's offset).
+        // 128-bit path needs parameter and state congruent mod 16 B (bf16 moments:
+        // 8-byte accesses at half the parameter's offset); the state slices (and the
+        // save buffer's) share the phase the parameters had at attach.
         const uintptr_t m = reinterpret_cast<uintptr_t>(slice(o, 0, i));
         const bool m_ok = o->h.mom16 ? ((p & 15u) >> 1) == (m & 7u) : ((p ^ m) & 15u) == 0;
-        if (!m_ok || (((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
-            scalar_path = true;
+        if (!m_ok) scalar_path = true;
+        // a gradient at another offset is fetched element by element, the rest stays wide
+        if ((((p & 15u) / 4u) != ((g % gvec) / (gvec / 4u))) || (g % (gvec / 4u)))
+            narrow_grad = true;
         // the bf16 copy is stored 4 elements (8 bytes) at a time beside 16-byte parameters
         if (!o->copies.empty() &&
             ((p & 15u) >> 1) != (reinterpret_cast<uintptr_t>(o->copies[i]) & 7u))
@@ -380,6 +474,8 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
     const bool traj = la && o->h.la_mode == NOVAK_LOOKAHEAD_TRAJ_MEAN;
     for (int i = 0; i < n; ++i) {
         h[i].p = static_cast<float *>(d_params[i]);
+        // the save buffer is laid out like a state array: same slot, same phase
+        h[i].p_in = save ? static_cast<const float *>(save) + o->slot_off[i] + o->phase[i] : h[i].p;
         h[i].g = d_grads[i];
         h[i].m = slice(o, 0, i);
         h[i].v = slice(o, 1, i);
@@ -403,12 +499,14 @@ int refresh_records(novak_opt *o, void *const *d_params, const void *const *d_gr
     o->ring_pos = (slot + 1) % kRing;
     tb.p.assign(d_params, d_params + n);
     tb.g.assign(d_grads, d_grads + n);
+    tb.save = save;
     tb.gdtype = grad_dtype;
     tb.hash = hash;
     tb.last_use = ++o->table_clock;
     o->cur_table = lru;
     o->record_uploads += 1;
     if (scalar_path) o->warnings |= NOVAK_WARN_SCALAR_PATH;
+    if (narrow_grad) o->warnings |= NOVAK_WARN_NARROW_GRADIENT;
     return NOVAK_OK;
 }
 

@@ -17,6 +17,7 @@ namespace {
 
 // Everything one step needs, fixed before anything is enqueued.
 struct StepCtx {
+    bool adapt_in_step;      // layer adaptation and update as one persistent kernel
     int64_t t;
     Plan plan;
     int la;
@@ -32,7 +33,9 @@ int check_step_args(novak_opt *o, const char *who, void *const *d_params,
                     const void *const *d_grads, const int64_t *numel, int n, int grad_dtype)
 {
     if (!o->attached) return fail(o, NOVAK_ESTATE, "%s: no state attached", who);
-    if (o->extrapolated)
+    // novak_step itself may follow the look-ahead directly: it then reads
+    // theta_{t-1} from the save buffer and needs no restore pass
+    if (o->extrapolated && std::strcmp(who, "step") != 0)
         return fail(o, NOVAK_ESTATE, "%s: parameters are extrapolated (Eq. 10); call novak_nesterov_restore first", who);
     if (o->half_open && std::strcmp(who, "step_begin") != 0)
         return fail(o, NOVAK_ESTATE, "%s: a step begun with novak_step_begin is still open", who);
@@ -69,13 +72,19 @@ int check_dyn(novak_opt *o, const char *who)
 }
 
 // Work table on the device, records for these pointers, the scalar plan of step t+1.
+// `save`: NULL, or the save buffer of the open look-ahead (theta_{t-1} is read there).
+// whole_table: the step is one launch over the whole group (novak_step), so the
+// step kernel may own rows (PRE_CENTER_ROWS).
 int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, int grad_dtype,
-               cudaStream_t stream, StepCtx *ctx)
+               cudaStream_t stream, StepCtx *ctx, const void *save = nullptr,
+               bool whole_table = false)
 {
     int rc;
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
-    ctx->pre = pre_mode(o);
-    if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
+    ctx->pre = step_pre_mode(o, whole_table);
+    if (ctx->pre != novak::PRE_NONE &&
+        (rc = prepare_prep(o, ctx->pre == novak::PRE_CENTER_ROWS, stream)) != NOVAK_OK)
+        return rc;
     if (o->ema_pending && o->prep_out) {
         // averages set by the caller (or saved over a reallocation) go into the scratch
         const double ema[2] = {o->pending_g_bar, o->pending_theta_bar};
@@ -85,7 +94,13 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     }
     if (o->h.layer_adapt && (rc = prepare_trust(o, stream)) != NOVAK_OK) return rc;
     ctx->trust = o->h.layer_adapt ? o->trust : nullptr;
-    if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, stream)) != NOVAK_OK) return rc;
+    ctx->adapt_in_step = o->h.layer_adapt && whole_table && o->adapt_in_step && !o->dyn &&
+                         ctx->pre == novak::PRE_NONE;
+    if (ctx->adapt_in_step && (rc = prepare_adapt(o, stream)) != NOVAK_OK) return rc;
+    if (o->h_adapt_error && *o->h_adapt_error)
+        return fail(o, NOVAK_ECUDA, "an earlier step's layer-adaptation kernel gave up waiting for a "
+                    "tensor's trust ratio and left entries un-updated; the optimizer state is not usable");
+    if ((rc = refresh_records(o, d_params, d_grads, grad_dtype, save, stream)) != NOVAK_OK) return rc;
     ctx->t = o->t + 1;
     ctx->plan = make_plan(o->h, ctx->t);
     ctx->la = lookahead_action(o->h, ctx->t);
@@ -95,7 +110,9 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     ctx->reverse = (o->serpentine && (ctx->t % 2 == 0)) ? 1 : 0;
     // After a statistics pass the END of the gradient is what L2 still holds:
     // the step kernel then walks the table from the end.
-    if (ctx->pre != novak::PRE_NONE || ctx->trust) ctx->reverse = 1;
+    if ((ctx->pre != novak::PRE_NONE && ctx->pre != novak::PRE_CENTER_ROWS) ||
+        (ctx->trust && !ctx->adapt_in_step))
+        ctx->reverse = 1;
     return NOVAK_OK;
 }
 
@@ -107,6 +124,8 @@ cudaError_t launch_statistics(novak_opt *o, const StepCtx &ctx, bool finalize, c
                               int *launches, const char **what)
 {
     if (ctx.pre == novak::PRE_NONE) return cudaSuccess;
+    // the step kernel owns its rows: only tensors with longer rows need the pass
+    if (ctx.pre == novak::PRE_CENTER_ROWS && o->n_units == 0) return cudaSuccess;
     *what = "gradient statistics kernel launch";
     const cudaError_t e = launch_stats(o, ctx, finalize, stream);
     if (e == cudaSuccess) *launches += o->h.auto_lr ? 3 : 2;
@@ -117,7 +136,7 @@ cudaError_t launch_trust(novak_opt *o, const StepCtx &ctx, cudaStream_t stream, 
                          const char **what)
 {
     cudaError_t e;
-    if (ctx.trust) {
+    if (ctx.trust && !ctx.adapt_in_step) {
         *what = "layer adaptation kernel launch";
         e = novak::launch_trust_stats(o->d_chunks, o->n_chunks, ctx.d_recs, o->n, o->tensor_first,
                                       o->prep_out, ctx.s, o->dyn ? o->d_plan : nullptr,
@@ -168,6 +187,25 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
     cfg.pdl = o->pdl;
     cfg.pre = ctx.pre | (o->copies.empty() ? 0 : novak::PRE_COPY16) |
               (o->h.mom16 ? novak::PRE_MOM16 : 0);
+    if (ctx.adapt_in_step) {
+        // statistics and update of the whole group as items of one grid
+        cfg.grid = o->n_items;
+        o->last_grid = cfg.grid;
+        const unsigned epoch = o->adapt_epoch == 0xffffffffu ? 1u : o->adapt_epoch + 1u;
+        const cudaError_t e = novak::launch_step_adapt(
+            o->d_item_code, o->d_item_chunk, o->n_items, ctx.d_recs,
+            o->tensor_first, o->chunk_u2, o->chunk_p2, o->trust, o->adapt_ctl, o->adapt_arrived,
+            o->adapt_ready, o->d_adapt_error, ctx.s, epoch, kernel_variant(ctx.plan), ctx.grad_dtype,
+            ctx.la, cfg, stream);
+        if (e == cudaSuccess) o->adapt_epoch = epoch;
+        return e;
+    }
+    if (ctx.pre == novak::PRE_CENTER_ROWS) {
+        // always the whole group (begin_step chose the mode for a one-launch step)
+        o->last_grid = o->n_rest + o->n_own;
+        return novak::launch_step_rows(o->d_rest, o->n_rest, o->d_own, o->n_own, ctx.d_recs, ctx.s,
+                                       kernel_variant(ctx.plan), ctx.grad_dtype, ctx.la, cfg, stream);
+    }
     o->last_grid = cfg.grid;
     return novak::launch_step(o->d_chunks + c0, count, ctx.d_recs, o->prep_out, ctx.trust, ctx.s,
                               kernel_variant(ctx.plan), ctx.grad_dtype, ctx.la, cfg, stream);
@@ -273,8 +311,18 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (o->dyn && (rc = check_dyn(o, "step")) != NOVAK_OK) return rc;
     if (!o->dyn && (rc = refuse_capture(o, "step", stream)) != NOVAK_OK) return rc;
+    // Directly behind novak_nesterov_extrapolate (no restore in between) the step
+    // reads theta_{t-1} from the save buffer and writes theta_t over Eq. 10's
+    // point in the parameter tensors: the restore pass is folded into the step.
+    const void *save = nullptr;
+    if (o->extrapolated) {
+        if (o->dyn) return fail(o, NOVAK_ESTATE, "step: parameters are extrapolated (Eq. 10)");
+        if (std::memcmp(o->look_p.data(), d_params, static_cast<size_t>(n) * sizeof(void *)) != 0)
+            return fail(o, NOVAK_EINVAL, "step: not the parameter tensors novak_nesterov_extrapolate was given");
+        save = o->look_save;
+    }
     StepCtx ctx;
-    if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx)) != NOVAK_OK) return rc;
+    if ((rc = begin_step(o, d_params, d_grads, grad_dtype, stream, &ctx, save, true)) != NOVAK_OK) return rc;
     cudaError_t e;
     int launches = 1;
     const char *what = "";
@@ -301,6 +349,11 @@ int novak_step(novak_opt *o, void *const *d_params, const void *const *d_grads,
         launches += 1;
     } else if ((e = launch_range(o, ctx, 0, o->n_chunks, stream)) != cudaSuccess) {
         return fail_cuda(o, e, "step kernel launch");
+    }
+    if (save) {
+        // the parameter tensors hold theta_t now; the save buffer is the caller's again
+        o->extrapolated = false;
+        o->look_save = nullptr;
     }
     commit_step(o, ctx, launches);
     return NOVAK_OK;
@@ -541,6 +594,7 @@ int novak_step_noalloc(novak_opt *o, void *const *d_params, const void *const *d
         for (int i = 0; i < n; ++i) {
             TensorRec &r = o->na_recs[i];
             r.p = static_cast<float *>(d_params[i]);
+            r.p_in = r.p;
             r.g = d_grads[i];
             r.m = slice(o, 0, i);
             r.v = slice(o, 1, i);

@@ -43,6 +43,29 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
                                int grad_dtype, int pre, double *chunk_u2, double *chunk_p2,
                                float *trust, int pdl, cudaStream_t stream);
 
+// ---- layer adaptation and step in one launch (novak_step_adapt.cuh) ---------
+// State of the kernel in device memory, zero before the first launch.
+struct __align__(16) AdaptCtl {
+    unsigned error;       // a bounded wait gave up (sticky)
+    unsigned reserved[3];
+};
+
+// item_code: n_items codes in block order, a chunk-table index for an S item,
+// the index | 0x80000000 for a U item, every entry once as each, a tensor's S
+// items all before any of its U items; item_chunk: the entry itself, item by
+// item.  arrived: one counter per tensor; ready: one 64-bit word per tensor
+// (launch number in the high half, the ratio's bits in the low half); both
+// zero before the first launch.  epoch: a launch number no earlier launch on
+// these buffers used (never 0).  host_error: device address of a host-mapped
+// word, set to 1 if a wait gives up.  cfg.pre: PRE_NONE with or without
+// PRE_COPY16 and PRE_MOM16.  The grid is n_items CTAs.
+cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int n_items,
+                              const TensorRec *d_recs, const int *tensor_first,
+                              double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
+                              unsigned *arrived, unsigned long long *ready, unsigned *host_error,
+                              const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
+                              int la, const LaunchCfg &cfg, cudaStream_t stream);
+
 // One unit of work of the statistics pass for a tensor with rows (Eq. 26).
 // Rows of up to kRowWarpMax elements: n_rows (a multiple of 8 but for a tensor's
 // last unit) whole rows starting at row0
@@ -61,6 +84,25 @@ struct __align__(16) RowUnit {
     uint32_t part_idx;
     uint32_t reserved;
 };
+
+// Step kernel that centralizes by itself (PRE_CENTER_ROWS): rows of up to
+// kOwnRowMax elements are owned by one CTA, in units of whole rows: as many as
+// fit in kOwnUnitElems elements (at most kOwnUnitRows), or one longer row;
+// rows beyond kOwnRowMax keep the statistics pass.
+constexpr uint32_t kOwnRowMax = 32768;
+constexpr uint32_t kOwnUnitElems = 4096;
+constexpr uint32_t kOwnUnitRows = 256;
+// Units of up to this many elements pass their gradient through shared memory.
+constexpr uint32_t kOwnStageElems = 8192;
+
+// Launches it: CTAs [0, n_rest) take one chunk-table entry each of `rest` (the
+// tensors without rows, and those with longer rows, whose means the statistics
+// pass has left in their records); the next n_units CTAs one unit of whole rows
+// each (RowUnit with part_len = 0).  cfg.pre: PRE_CENTER_ROWS with or without
+// PRE_COPY16 and PRE_MOM16; cfg.grid and cfg.reverse are ignored.
+cudaError_t launch_step_rows(const Chunk *d_rest, int n_rest, const RowUnit *d_units, int n_units,
+                             const TensorRec *d_recs, const StepScalars &s, int nesterov,
+                             int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream);
 
 // Elements a row unit aims at, and rows per unit where a thread takes a row.
 constexpr uint32_t kRowUnitElems = 16384;

@@ -15,9 +15,16 @@ namespace novak {
 
 // novak_step_inst.cu, compiled once per gradient pre-processing mode, holds the
 // kernels; mode N (the PRE_* bits as a number) exports step_kernel_mode<N>.
-#define NOVAK_FOR_EACH_PRE_MODE(X) X(0) X(1) X(2) X(4) X(5) X(6) X(8) X(9) X(10) X(12) X(13) X(14)
+#define NOVAK_FOR_EACH_PRE_MODE(X) \
+    X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15)
 #define NOVAK_DECLARE(N) void *step_kernel_mode##N(int nesterov, int grad_dtype, int la);
 NOVAK_FOR_EACH_PRE_MODE(NOVAK_DECLARE)
+#undef NOVAK_DECLARE
+
+// The kernels that adapt and step in one launch: the four PRE_NONE modes.
+#define NOVAK_FOR_EACH_ADAPT_MODE(X) X(0) X(4) X(8) X(12)
+#define NOVAK_DECLARE(N) void *step_adapt_kernel_mode##N(int nesterov, int grad_dtype, int la);
+NOVAK_FOR_EACH_ADAPT_MODE(NOVAK_DECLARE)
 #undef NOVAK_DECLARE
 
 namespace {
@@ -27,7 +34,10 @@ constexpr int kBlock = NOVAK_BLOCK;
 using StepKernelFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *,
                               const float *, StepScalars, int);
 
-StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
+using StepRowsKernelFn = void (*)(const Chunk *, int, const RowUnit *, int, const TensorRec *,
+                                  StepScalars);
+
+void *pick_kernel_raw(int nesterov, int grad_dtype, int la, int pre)
 {
     void *fn = nullptr;
     switch (pre) {
@@ -36,7 +46,13 @@ StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
 #undef NOVAK_CASE
     default: break;
     }
-    return reinterpret_cast<StepKernelFn>(fn);
+    return fn;
+}
+
+StepKernelFn pick_kernel(int nesterov, int grad_dtype, int la, int pre)
+{
+    if ((pre & PRE_MASK) == PRE_CENTER_ROWS) return nullptr;     // another signature
+    return reinterpret_cast<StepKernelFn>(pick_kernel_raw(nesterov, grad_dtype, la, pre));
 }
 
 }  // namespace
@@ -75,11 +91,67 @@ cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks)
 
 int step_block_threads() { return kBlock; }
 
+cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int n_items,
+                              const TensorRec *d_recs, const int *tensor_first,
+                              double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
+                              unsigned *arrived, unsigned long long *ready, unsigned *host_error,
+                              const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
+                              int la, const LaunchCfg &cfg, cudaStream_t stream)
+{
+    using Fn = void (*)(const int *, const Chunk *, int, const TensorRec *, const int *, double *,
+                        double *, float *, AdaptCtl *, unsigned *, unsigned long long *, unsigned *,
+                        StepScalars, unsigned);
+    void *raw = nullptr;
+    switch (cfg.pre) {
+#define NOVAK_CASE(N) case N: raw = step_adapt_kernel_mode##N(nesterov, grad_dtype, la); break;
+        NOVAK_FOR_EACH_ADAPT_MODE(NOVAK_CASE)
+#undef NOVAK_CASE
+    default: break;
+    }
+    Fn fn = reinterpret_cast<Fn>(raw);
+    if (!fn || !item_code || !item_chunk || n_items <= 0 || epoch == 0u || !ctl || !arrived || !ready ||
+        !host_error || !tensor_first || !chunk_u2 || !chunk_p2 || !trust)
+        return cudaErrorInvalidValue;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(n_items));
+    lc.blockDim = dim3(kBlock);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, fn, item_code, item_chunk, n_items, d_recs, tensor_first,
+                              chunk_u2, chunk_p2, trust, ctl, arrived, ready, host_error, s, epoch);
+}
+
 cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int pre, int *ctas_per_sm)
 {
-    StepKernelFn fn = pick_kernel(nesterov, grad_dtype, la, pre);
+    void *fn = pick_kernel_raw(nesterov, grad_dtype, la, pre);
     if (!fn) return cudaErrorInvalidValue;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, fn, kBlock, 0);
+}
+
+cudaError_t launch_step_rows(const Chunk *d_rest, int n_rest, const RowUnit *d_units, int n_units,
+                             const TensorRec *d_recs, const StepScalars &s, int nesterov,
+                             int grad_dtype, int la, const LaunchCfg &cfg, cudaStream_t stream)
+{
+    if ((cfg.pre & PRE_MASK) != PRE_CENTER_ROWS || n_rest < 0 || n_units < 0 || n_rest + n_units <= 0)
+        return cudaErrorInvalidValue;
+    StepRowsKernelFn fn = reinterpret_cast<StepRowsKernelFn>(pick_kernel_raw(nesterov, grad_dtype, la, cfg.pre));
+    if (!fn) return cudaErrorInvalidValue;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(static_cast<unsigned>(n_rest + n_units));
+    lc.blockDim = dim3(kBlock);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
+    return cudaLaunchKernelEx(&lc, fn, d_rest, n_rest, d_units, n_units, d_recs, s);
 }
 
 cudaError_t launch_step(const Chunk *d_chunks, int n_chunks, const TensorRec *d_recs,

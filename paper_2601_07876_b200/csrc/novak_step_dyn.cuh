@@ -25,10 +25,6 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
                                             const StepScalars &s, int reverse, int c, Chunk ch,
                                             TensorRec r)
 {
-    constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
-    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
-    constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
-    constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
     PreArgs pre = pre0;
 #pragma unroll 1
     for (;;) {
@@ -38,31 +34,7 @@ __device__ __forceinline__ void dyn_entries(const Chunk *__restrict__ chunks, in
         pre.row_len = r.row_len;
         pre.elem0 = static_cast<uint32_t>(ch.offset);
         pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
-        float *p = r.p + ch.offset;
-        void *m = static_cast<char *>(r.m) + ch.offset * kMomBytes;
-        void *v = static_cast<char *>(r.v) + ch.offset * kMomBytes;
-        float *slow = kUseS ? r.slow + ch.offset : nullptr;
-        float *acc = kUseA ? r.acc + ch.offset : nullptr;
-        const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
-        // four bf16 moments are one 64-bit access: half the parameters' alignment
-        uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
-                         ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
-                          << (kMomBytes == 2 ? 1 : 0));
-        if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
-        if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
-        // the 64-bit stores of the bf16 copy need half the parameters' alignment
-        if ((PRE & PRE_COPY16) != 0) bits |= reinterpret_cast<uintptr_t>(pre.copy) << 1;
-        const bool aligned = (bits & 15u) == 0 &&
-                             (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
-        if (aligned) {
-            const int nvec = ch.len >> 2;
-            run_span<4, kUnroll, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, nvec, s, pre);
-            const int idx = (nvec << 2) + threadIdx.x;      // ragged tail: at most 3 elements
-            if (idx < ch.len)
-                run_tile<1, 1, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, idx, s, pre);
-        } else {
-            run_span<1, 4, NEST, GT, LA, PRE>(p, g, m, v, slow, acc, ch.len, s, pre);
-        }
+        run_entry<NEST, GT, LA, PRE>(ch, r, s, pre);
         c += gridDim.x;
         if (c >= n_chunks) break;
         ch = chunks[reverse ? n_chunks - 1 - c : c];

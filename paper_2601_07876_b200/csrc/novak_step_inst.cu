@@ -4,7 +4,10 @@
 //                     as a number>
 //   -DNOVAK_INST_DYN   for the graph-capturable kernel (scalars and lookahead
 //                      action read from device memory) instead of the plain one.
-// Each object exports one selector, step_kernel_mode<N> or step_dyn_kernel_mode<N>.
+//   -DNOVAK_INST_ADAPT for the kernel that runs layer adaptation and the update
+//                      as one persistent launch (PRE_NONE modes only).
+// Each object exports one selector: step_kernel_mode<N>, step_dyn_kernel_mode<N>
+// or step_adapt_kernel_mode<N>.
 #ifndef NOVAK_PRE_MODE
 #error "compile with -DNOVAK_PRE_MODE=<mode bits>"
 #endif
@@ -23,6 +26,17 @@ void *NOVAK_PASTE(step_dyn_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad_d
 }
 
 }  // namespace novak
+#elif defined(NOVAK_INST_ADAPT)
+#include "novak_step_adapt.cuh"
+
+namespace novak {
+
+void *NOVAK_PASTE(step_adapt_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad_dtype, int la)
+{
+    return pick_step_adapt_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype, la);
+}
+
+}  // namespace novak
 #else
 #include "novak_step_kernel.cuh"
 
@@ -30,7 +44,7 @@ namespace novak {
 
 void *NOVAK_PASTE(step_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad_dtype, int la)
 {
-    return reinterpret_cast<void *>(pick_step_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype, la));
+    return pick_step_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype, la);
 }
 
 }  // namespace novak

@@ -11,7 +11,7 @@ namespace novak {
 
 // Per-tensor record in device memory: where the tensor's streams start.
 struct __align__(16) TensorRec {
-    float *p;          // parameters theta, fp32, updated in place
+    float *p;          // parameters theta, fp32: where theta_t is written
     const void *g;     // gradient, fp32 or bf16, read only
     void *m;           // first moment   (Eq. 1), fp32, or bf16 under PRE_MOM16
     void *v;           // second moment  (Eq. 2), same type as m
@@ -19,9 +19,13 @@ struct __align__(16) TensorRec {
     float *acc;        // running sum of the window's fast iterates (TRAJ_MEAN)
     float2 *mean;      // row means of the raw gradient (Eq. 26) as hi + lo, NULL: not centralized
     __nv_bfloat16 *p16; // bf16 copy of theta written by the step, NULL: none
+    const float *p_in; // where theta_{t-1} is read: p itself, or the tensor's slice of the
+                       // save buffer on the step behind a true-Nesterov look-ahead (the
+                       // parameter tensor then still holds Eq. 10's extrapolated point)
     uint32_t row_len;  // elements per row (product of dimensions 1..d), 0: not centralized
     uint32_t reserved;
 };
+static_assert(sizeof(TensorRec) == 80, "TensorRec is 80 bytes");
 
 // One unit of work: `len` consecutive elements of one tensor.
 struct __align__(16) Chunk {
@@ -64,6 +68,8 @@ enum : int {
     PRE_NONE = 0,    // g as given
     PRE_SCALE = 1,   // g <- factor g, the clip factor read from device memory
     PRE_CENTER = 2,  // g <- factor (g - row mean) for tensors that have rows (Eq. 26)
+    PRE_CENTER_ROWS = 3,  // Eq. 26 without a pass of its own: the step kernel's CTAs own whole
+                          // rows and form the means themselves (no clipping, no factor)
     PRE_MASK = 3,
     // OR-ed onto the above: the step also stores a bf16 copy of the new parameters
     PRE_COPY16 = 4,

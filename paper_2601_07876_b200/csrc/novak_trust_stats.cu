@@ -9,60 +9,10 @@
 // kernel, one CTA per tensor, adds a tensor's entries in table order.  All
 // sums are in double in a fixed order: bit-identical from run to run, no
 // atomics, nothing spins.
-#include "novak_step_kernel.cuh"
+#include "novak_trust.cuh"
 
 namespace novak {
 namespace {
-
-constexpr int kTrustBlock = NOVAK_BLOCK;
-constexpr int kTrustWarps = kTrustBlock / 32;
-
-__device__ __forceinline__ double trust_warp_sum(double x)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_down_sync(0xffffffffu, x, o);
-    return x;
-}
-
-// Sum over the CTA, warps in index order; thread 0 holds the total.
-__device__ __forceinline__ double trust_block_sum(double x, double *sh)
-{
-    x = trust_warp_sum(x);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    __syncthreads();
-    if (lane == 0) sh[warp] = x;
-    __syncthreads();
-    double t = 0.0;
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int w = 0; w < kTrustWarps; ++w) t += sh[w];
-    }
-    return t;
-}
-
-// Squares of N parameters and of the N base directions their gradients give.
-// Each group of N squares is added in fp32, groups in double.
-template <int N, int NEST, int GT, int PRE>
-__device__ __forceinline__ void accumulate(const float *p, const void *g, const void *m,
-                                           const void *v, int idx, const StepScalars &s,
-                                           const PreArgs &pre, double &sum_p, double &sum_u)
-{
-    const Vec<N> P = load_f32<N>(p, idx);
-    Vec<N> G = load_grad<N, GT>(g, idx);
-    const Vec<N> M = load_moment<N, (PRE & PRE_MOM16) != 0>(m, idx);
-    const Vec<N> V = load_moment<N, (PRE & PRE_MOM16) != 0>(v, idx);
-    preprocess<N, PRE>(G, row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre), pre);
-    float sp = 0.0f, su = 0.0f;
-#pragma unroll
-    for (int e = 0; e < N; ++e) {
-        float mm = M.a[e], vv = V.a[e], m_hat;
-        const float u = base_direction<NEST>(G.a[e], mm, vv, m_hat, s);
-        sp = fmaf(P.a[e], P.a[e], sp);
-        su = fmaf(u, u, su);
-    }
-    sum_p += double(sp);
-    sum_u += double(su);
-}
 
 template <int NEST, int GT, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK)
@@ -72,8 +22,6 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
                          double *__restrict__ chunk_u2, double *__restrict__ chunk_p2)
 {
     __shared__ double sh[kTrustWarps];
-    constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
-    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
 
     grid_dependency_release();
     const int c = blockIdx.x;            // the grid has exactly n_chunks CTAs
@@ -93,30 +41,8 @@ novak_trust_stats_kernel(const Chunk *__restrict__ chunks, int n_chunks,
     pre.row_len = r.row_len;
     pre.elem0 = static_cast<uint32_t>(ch.offset);
 
-    const float *p = r.p + ch.offset;
-    const void *m = static_cast<const char *>(r.m) + ch.offset * kMomBytes;
-    const void *v = static_cast<const char *>(r.v) + ch.offset * kMomBytes;
-    const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
-    const uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
-                           ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
-                            << (kMomBytes == 2 ? 1 : 0));
-    const bool aligned = (bits & 15u) == 0 &&
-                         (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
-    double sum_p = 0.0, sum_u = 0.0;
-    if (aligned) {
-        const int nvec = ch.len >> 2;
-#pragma unroll 2
-        for (int i = threadIdx.x; i < nvec; i += kTrustBlock)
-            accumulate<4, NEST, GT, PRE>(p, g, m, v, i, s, pre, sum_p, sum_u);
-        const int idx = (nvec << 2) + threadIdx.x;          // ragged tail: < 4 elements
-        if (idx < ch.len) accumulate<1, NEST, GT, PRE>(p, g, m, v, idx, s, pre, sum_p, sum_u);
-    } else {
-#pragma unroll 4
-        for (int i = threadIdx.x; i < ch.len; i += kTrustBlock)
-            accumulate<1, NEST, GT, PRE>(p, g, m, v, i, s, pre, sum_p, sum_u);
-    }
-    const double tp = trust_block_sum(sum_p, sh);
-    const double tu = trust_block_sum(sum_u, sh);
+    double tp, tu;
+    entry_trust_sums<NEST, GT, PRE>(ch, r, s, pre, sh, tp, tu);
     if (threadIdx.x == 0) {
         chunk_p2[c] = tp;
         chunk_u2[c] = tu;
@@ -134,21 +60,8 @@ novak_trust_finish_kernel(const int *__restrict__ tensor_first,
     const int t = blockIdx.x;
     const int c0 = tensor_first[t], c1 = tensor_first[t + 1];
     grid_dependency_wait();              // the first kernel's sums
-    double sp = 0.0, su = 0.0;
-    for (int c = c0 + threadIdx.x; c < c1; c += kTrustBlock) {
-        sp += chunk_p2[c];
-        su += chunk_u2[c];
-    }
-    const double tp = trust_block_sum(sp, sh);
-    const double tu = trust_block_sum(su, sh);
-    if (threadIdx.x == 0) {
-        double eta = 1.0;                // ||u|| = 0: the ratio is undefined, the update zero
-        if (tu > 0.0) {
-            eta = sqrt(tp) / sqrt(tu);
-            eta = eta < 0.1 ? 0.1 : (eta > 10.0 ? 10.0 : eta);
-        }
-        trust[t] = static_cast<float>(eta);
-    }
+    const float eta = tensor_trust_ratio(chunk_p2, chunk_u2, c0, c1, sh);
+    if (threadIdx.x == 0) trust[t] = eta;
 }
 
 using TrustFn = void (*)(const Chunk *, int, const TensorRec *, const PrepOut *, StepScalars,

@@ -6,8 +6,8 @@ variant).  This class only collects pointers and forwards: every parameter
 group is one handle of the C-ABI library (one fused multi-tensor step per
 group), ``p.grad`` supplies the gradients, and a closure passed to ``step``
 is evaluated at Eq. 10's look-ahead point while the group is in its first
-N_taylor steps (Section 5.8: save, extrapolate, evaluate, restore).  No
-arithmetic of the method happens here.
+N_taylor steps (Section 5.8: save, extrapolate, evaluate; the step then reads the
+saved parameters, which is the restore).  No arithmetic of the method happens here.
 """
 from __future__ import annotations
 
@@ -109,9 +109,10 @@ class Novak(torch.optim.Optimizer):
             try:
                 with torch.enable_grad():
                     loss = closure()
-            finally:
+            except BaseException:
                 for e in ahead:
-                    e.restore()
+                    e.restore()          # the step is abandoned: put theta_{t-1} back
+                raise
         for gi, e in enumerate(engines):
             e.step(self._grads(gi, e))
         return loss

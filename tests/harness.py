@@ -158,10 +158,10 @@ class FullPair:
     """Full-size workload on the GPU and the oracle on EVERY element of it.
 
     The oracle sees the workload's flat buffer as one tensor (the step has no
-    cross-element term; the padding between tensors holds zero parameters and zero
-    gradients and stays zero on both sides), so its arrays line up with the flat
-    parameter and gradient buffers; the library's own state layout is compared tensor
-    by tensor through novak_state_ptrs."""
+    cross-element term), so its arrays line up with the flat parameter and gradient
+    buffers; every tensor's elements are compared, the padding between tensors is left
+    out (and must still be zero on the GPU).  The library's own state layout is
+    compared tensor by tensor through novak_state_ptrs."""
 
     def __init__(self, wl: W.Workload, device, hyper_override: dict | None = None,
                  opt_kwargs: dict | None = None):
@@ -198,11 +198,18 @@ class FullPair:
         assert self.rect_flags == o.rect_flags
         assert info["n_syncs"] == len(o.sync_steps)
         name = self.wl.name
-        # parameters: the whole flat buffer, padding included (nothing may be written there)
-        assert_close(self.flat_p, o.theta[0], f"{name} theta")
+        # the padding between tensors is not the library's to write: still zero (the
+        # gradient generator may have put numbers there, which the oracle then followed)
+        pad = torch.ones(self.flat_p.numel(), dtype=torch.bool, device=self.flat_p.device)
+        for off, n in zip(self.offs, self.wl.numel):
+            pad[off:off + n] = False
+        assert not bool(self.flat_p[pad].any()), f"{name}: padding between tensors was written"
+        del pad
+        theta_gpu = to_f64(self.flat_p)
         with_acc = o.acc is not None and o.cfg.lookahead_k > 1 and o.t % o.cfg.lookahead_k != 0
         for i, (off, n) in enumerate(zip(self.offs, self.wl.numel)):
             st = self.opt.state(i)
+            assert_close(theta_gpu[off:off + n], o.theta[0][off:off + n], f"{name} theta")
             assert_close(st["m"], o.m[0][off:off + n], f"{name} m")
             assert_close(st["v"], o.v[0][off:off + n], f"{name} v")
             if n >= 1024:     # a root mean square needs a population

@@ -59,6 +59,67 @@ def test_row_units_cover_every_row_once(data):
 
 
 @settings(max_examples=60, deadline=None)
+@given(data=st.data())
+def test_own_units_cover_the_rows_of_owned_tensors_once(data):
+    """Units of the step kernel that forms its row means itself: every row of every tensor
+    whose rows have at most 32768 elements exactly once, whole rows only, at most 256 rows
+    and (beyond one row) at most 4096 elements per unit; nothing for longer rows."""
+    n = data.draw(st.integers(1, 8))
+    numel, rows = [], []
+    for _ in range(n):
+        if data.draw(st.booleans()):
+            r = data.draw(st.integers(1, 600))
+            length = data.draw(st.sampled_from([1, 2, 3, 5, 15, 16, 17, 27, 64, 147, 576, 2048, 2049,
+                                                4096, 4097, 4608, 32768, 32769, 40_000]))
+            numel.append(r * length)
+            rows.append(r)
+        else:
+            numel.append(data.draw(st.integers(1, 5000)))
+            rows.append(0)
+    units = B.novak_build_own_units(numel, rows)
+    owned = {i for i, r in enumerate(rows) if r and numel[i] // r <= 32768}
+    seen = {i: np.zeros(rows[i], dtype=np.int8) for i in owned}
+    for t, row0, n_rows in units:
+        assert t in owned and 1 <= n_rows <= 256
+        L = numel[t] // rows[t]
+        assert n_rows == 1 or n_rows * L <= 4096
+        seen[t][row0:row0 + n_rows] += 1
+    assert all((s == 1).all() for s in seen.values())
+    # consecutive units of a tensor are adjacent and in order
+    for (t0, r0, n0), (t1, r1, _) in zip(units, units[1:]):
+        assert (t1 == t0 and r1 == r0 + n0) or (t1 > t0 and r1 == 0)
+
+
+@settings(max_examples=80, deadline=None)
+@given(counts=st.lists(st.integers(1, 40), min_size=1, max_size=30), lead=st.integers(0, 120))
+def test_adapt_order_puts_statistics_first_and_keeps_the_lead(counts, lead):
+    """Item order of the one-launch layer adaptation: every chunk-table entry once as a
+    statistics item and once as an update item; all statistics items of a tensor before
+    any of its update items (what the kernel's freedom from deadlock rests on); tensors in
+    order within each kind; at least `lead` items between a tensor's last statistics item
+    and its first update item, except for what is flushed at the end."""
+    first = np.concatenate([[0], np.cumsum(counts)]).tolist()
+    order = B.novak_build_adapt_order(first, lead)
+    total = first[-1]
+    assert len(order) == 2 * total
+    tensor_of = np.repeat(np.arange(len(counts)), counts)
+    stats = [c for c, upd in order if not upd]
+    upds = [c for c, upd in order if upd]
+    assert stats == list(range(total)) and upds == list(range(total))
+    pos_s = {c: k for k, (c, upd) in enumerate(order) if not upd}
+    pos_u = {c: k for k, (c, upd) in enumerate(order) if upd}
+    last_stats_item = max(pos_s.values())
+    for t in range(len(counts)):
+        cs = range(first[t], first[t + 1])
+        s_last = max(pos_s[c] for c in cs)
+        u_first = min(pos_u[c] for c in cs)
+        assert s_last < u_first
+        if u_first < last_stats_item:          # not part of the final flush
+            assert u_first - s_last - 1 >= lead
+    assert (np.diff(tensor_of[stats]) >= 0).all()
+
+
+@settings(max_examples=60, deadline=None)
 @given(numel=sizes, world=st.integers(1, 9), align=st.sampled_from([1, 4, 64]))
 def test_rank_partition_covers_every_element_once_and_is_balanced(numel, world, align):
     parts = sharding.partition_flat(numel, world, align)

@@ -103,15 +103,37 @@ def test_true_nesterov_runs_as_approximation():
     assert a.info()["warnings"] & B.NOVAK_WARN_TRUE_DOWNGRADED
 
 
-def test_mismatched_gradient_alignment_takes_scalar_path():
-    """Gradients whose offset from a 16-byte boundary differs from the
-    parameters' cannot use 128-bit accesses: same result, warning bit set."""
+def test_mismatched_gradient_alignment_narrows_the_gradient_loads_only():
+    """Gradients whose offset from a 16-byte boundary differs from the parameters' are
+    fetched element by element while parameters and state keep their 128-bit accesses:
+    same result, its own warning bit set."""
     numels = [3000, 9001, 17]
     _, params, _ = _fresh(numels, [0, 1, 2])
     pair = Pair(params, dict(BASE, lookahead_mode="traj_mean", lookahead_k=3))
     gen = _gen(5)
     for _ in range(7):
         pair.step(_grads(numels, gen, offsets=[1, 3, 0]))
+    pair.check("narrow gradient loads")
+    assert pair.opt.info()["warnings"] & B.NOVAK_WARN_NARROW_GRADIENT
+    assert not pair.opt.info()["warnings"] & B.NOVAK_WARN_SCALAR_PATH
+
+
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_parameters_off_their_state_phase_take_the_scalar_path(gdtype):
+    """State attached for one set of parameter addresses, then stepped with tensors at
+    another offset from a 16-byte boundary: parameter and state no longer share
+    alignment and everything runs on 4-byte (2-byte) accesses."""
+    numels = [3000, 9001, 17, 1]
+    _, params, _ = _fresh(numels, [0, 1, 2, 3])
+    pair = Pair(params, dict(BASE, lookahead_k=2))
+    _, moved, _ = _fresh(numels, [1, 3, 0, 1])
+    for src, dst in zip(params, moved):
+        dst.copy_(src)
+    pair.params = moved
+    pair.opt.rebind_params(moved)
+    gen = _gen(6)
+    for _ in range(5):
+        pair.step(_grads(numels, gen, gdtype, offsets=[0, 1, 2, 3]))
     pair.check("scalar path")
     assert pair.opt.info()["warnings"] & B.NOVAK_WARN_SCALAR_PATH
 

@@ -66,11 +66,94 @@ def test_clip_and_centralize_every_element(gdtype, phase2, variant):
     pair.check(f"phase2 {phase2}")
     info = pair.opt.info()
     assert info["grad_processing"] == (2 if phase2.get("centralize") else 1)
-    assert info["launches"] == 3 * 7          # two statistics kernels + the step kernel
+    if phase2 == dict(centralize=True):
+        assert info["launches"] == 7          # the step kernel forms the row means itself
+    else:
+        assert info["launches"] == 3 * 7      # two statistics kernels + the step kernel
     if phase2.get("clip_threshold") == 0.05:
         assert all(f < 1.0 for f in pair.clip_factors)
     if phase2.get("clip_threshold") == 1e3:
         assert all(f == 1.0 for f in pair.clip_factors)
+
+
+# rows of every kind the row-owning step kernel distinguishes: shorter than a warp's
+# vector pass, odd lengths that start off a 16-byte boundary, a row for every warp and
+# fewer rows than warps, one row per unit, rows at the largest owned length, and rows
+# beyond it (2 x 40000, 1 x 70001) that keep the statistics pass
+OWN_SHAPES = SHAPES + [(64, 147), (16, 64), (40, 27), (300, 40), (9, 576), (3, 4608), (2, 32768),
+                       (2, 40000), (1, 70001), (5, 32769)]
+OWN_OFFSETS = OFFSETS + [0, 0, 1, 0, 2, 0, 0, 3, 0, 1]
+
+
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("long_rows", [False, True])
+@pytest.mark.parametrize("variant", [("approximation", "last", 5), ("classical", "traj_mean", 2),
+                                     ("none", "last", 0)])
+@pytest.mark.parametrize("in_step", [1, 0])
+def test_centralization_alone_inside_the_step_kernel(in_step, variant, long_rows, gdtype):
+    """Eq. 26 with nothing else that needs the whole gradient: the step kernel's CTAs own
+    whole rows and form the means themselves (one launch per step); tensors with rows
+    beyond the owned length still get theirs from the statistics pass.  Same oracle,
+    same tolerance, in both forms."""
+    nesterov, mode, k = variant
+    n = len(OWN_SHAPES) if long_rows else len(OWN_SHAPES) - 3
+    shapes, offsets = OWN_SHAPES[:n], OWN_OFFSETS[:n]
+    _, params = _shaped(shapes, offsets)
+    gen = _gen(15)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    copies = make_tensors([math.prod(s) for s in shapes], DEV, offsets, dtype=torch.bfloat16)[1]
+    hyper = dict(BASE, nesterov=nesterov, lookahead_mode=mode, lookahead_k=k, centralize=True)
+    pair = Pair(params, hyper, opt_kwargs=dict(centralize_in_step=in_step, param_copies=copies))
+    _, grads = _shaped(shapes, offsets, dtype=gdtype)
+    steps = 7
+    for t in range(steps):
+        _fill_grads(grads, gen, std=1e-3, mean=5e-4 * (1 + t % 3))
+        pair.step(grads)
+    pair.check(f"centralize, in step {in_step}")
+    for p, c in zip(params, copies):
+        assert torch.equal(c.view(p.shape), p.to(torch.bfloat16))
+    info = pair.opt.info()
+    assert info["grad_processing"] == 2
+    own = bool(in_step) and not long_rows
+    assert info["launches"] == (steps if own else 3 * steps)
+    assert not info["warnings"] & (B.NOVAK_WARN_SCALAR_PATH | B.NOVAK_WARN_NARROW_GRADIENT)
+
+
+def test_row_owning_step_is_bit_identical_from_run_to_run_and_takes_misphased_gradients():
+    """Two runs of the row-owning kernel give the same bits (fixed summation order, no
+    atomics); a gradient at another 16-byte phase than its parameter only narrows the
+    gradient loads."""
+    shapes, offsets = OWN_SHAPES[:-3], OWN_OFFSETS[:-3]
+    runs = []
+    for rep in range(2):
+        _, params = _shaped(shapes, offsets)
+        gen = _gen(17)
+        for p in params:
+            p.normal_(0.0, 0.05, generator=gen)
+        opt = B.NovakOptimizer(params, **BASE, centralize=True)
+        _, grads = _shaped(shapes, offsets)
+        for t in range(4):
+            _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+            opt.step(grads)
+        torch.cuda.synchronize()
+        assert opt.info()["launches"] == 4
+        runs.append([p.clone() for p in params] + [opt.state(i)["v"].clone() for i in range(len(shapes))])
+    for a, b in zip(*runs):
+        assert torch.equal(a, b)
+    _, params = _shaped(shapes, offsets)
+    gen = _gen(18)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    pair = Pair(params, dict(BASE, centralize=True, lookahead_k=2))
+    goffs = [(o + 1 + i % 3) % 4 for i, o in enumerate(offsets)]
+    _, grads = _shaped(shapes, goffs)
+    for t in range(5):
+        _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+        pair.step(grads)
+    pair.check("row-owning kernel, gradients off the parameters' phase")
+    assert pair.opt.info()["warnings"] & B.NOVAK_WARN_NARROW_GRADIENT
+    assert pair.opt.info()["launches"] == 5
 
 
 def test_phase2_is_bit_identical_from_run_to_run_and_across_launch_options():
@@ -185,9 +268,12 @@ def test_step_host_with_phase2_matches_step():
     np.testing.assert_allclose(a.grad_stats(), b.grad_stats(), rtol=1e-7)
 
 
-def test_fullsize_resnet50_with_clipping_and_centralization():
+@pytest.mark.parametrize("clip", [1.0, 0.0])
+def test_fullsize_resnet50_with_clipping_and_centralization(clip):
     """The benchmark's ResNet-50-shaped set with its real tensor shapes (53 conv / fc
-    weights with rows, 108 one-dimensional tensors), every element against the oracle."""
+    weights with rows, 108 one-dimensional tensors), every element against the oracle:
+    clipping + centralization (statistics pass), and centralization alone (formed inside
+    the step kernel, one launch per step)."""
     wl = W.get_workload(1)
     flat_p = W.alloc_flat(wl, torch.float32, DEV)
     W.init_params(wl, flat_p)
@@ -196,19 +282,22 @@ def test_fullsize_resnet50_with_clipping_and_centralization():
     grads = [v.view(s) for v, s in zip(W.views(flat_g, wl), wl.shapes)]
     src = W.GradSource(wl, DEV)
     harness.MARGINS.clear()
-    pair = Pair(params, dict(wl.hyper, clip_threshold=1.0, centralize=True))
+    pair = Pair(params, dict(wl.hyper, clip_threshold=clip, centralize=True))
     for _ in range(12):
         src.fill(flat_g)
         pair.step(grads, threads=8)
-        pair.record_grad_stats()
+        if clip:
+            pair.record_grad_stats()
     pair.check("resnet50 phase2")
-    assert all(f < 1.0 for f in pair.clip_factors)     # norm ~ 5: the clipping is active
+    if clip:
+        assert all(f < 1.0 for f in pair.clip_factors)     # norm ~ 5: the clipping is active
+    assert pair.opt.info()["launches"] == (36 if clip else 12)
     top = sorted(harness.MARGINS.items(), key=lambda kv: -kv[1])[:4]
     print("\nworst tensors:", [(k, round(v, 3), wl.shapes[int(k.split("[")[1][:-1])]) for k, v in top])
     worst = {}
     for k, v in harness.MARGINS.items():
         worst[k.split()[-1].split("[")[0]] = max(worst.get(k.split()[-1].split("[")[0], 0.0), v)
-    print("\nPARITY resnet50 clip+centralize steps=12 every element worst |err|/tol: "
+    print(f"\nPARITY resnet50 clip={clip}+centralize steps=12 every element worst |err|/tol: "
           + ", ".join(f"{k} {v:.3f}" for k, v in worst.items()))
 
 
@@ -238,9 +327,58 @@ def test_layer_adaptation_every_element(gdtype, extra, variant):
     pair.check(f"layer adaptation {extra}")
     seen = np.array(pair.oracle.trust)
     assert (seen == 0.1).any() and (seen == 10.0).any() and ((seen > 0.1) & (seen < 10.0)).any()
-    n_pre = 2 if extra.get("centralize") or extra.get("clip_threshold") else 0
-    assert pair.opt.info()["launches"] == 7 * (3 + n_pre)
+    if extra.get("centralize") or extra.get("clip_threshold"):
+        assert pair.opt.info()["launches"] == 7 * 5     # statistics x 2, ratios x 2, the step
+    else:
+        assert pair.opt.info()["launches"] == 7         # statistics and update in one launch
     assert pair.opt.info()["layer_adaptation"] == 1
+
+
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("lead", [0, 20000, None])
+@pytest.mark.parametrize("variant", [("approximation", "last", 5), ("classical", "traj_mean", 2),
+                                     ("none", "last", 0)])
+def test_layer_adaptation_in_one_launch_equals_the_three_launch_form(gdtype, lead, variant):
+    """Statistics and update as items of one grid (the statistics `lead` elements ahead of
+    the updates: none at all, so that updates wait for their ratio, a few entries, the
+    default) against the two statistics kernels followed by the step: the same sums in the same order, so ratios, parameters
+    and state agree bit for bit, over 8 steps with bf16 parameter copies switched on; the
+    one-launch form is also held against the oracle."""
+    nesterov, mode, k = variant
+    shapes = SHAPES + [(70001,), (3, 30000)]
+    offsets = OFFSETS + [2, 0]
+    hyper = dict(BASE, nesterov=nesterov, lookahead_mode=mode, lookahead_k=k, layer_adaptation=True)
+    numels = [math.prod(s) for s in shapes]
+    sets = []
+    for in_step in (1, 0):
+        _, params = _shaped(shapes, offsets)
+        gen = _gen(72)
+        for i, p in enumerate(params):
+            p.normal_(0.0, 10.0 ** (-4 + 5.5 * i / (len(params) - 1)), generator=gen)
+        copies = make_tensors(numels, DEV, offsets, dtype=torch.bfloat16)[1]
+        kw = dict(layer_adaptation_in_step=in_step, param_copies=copies)
+        if lead is not None:
+            kw["layer_adaptation_lead"] = lead
+        sets.append((params, copies, kw))
+    pair = Pair(sets[0][0], hyper, opt_kwargs=sets[0][2])
+    twin = B.NovakOptimizer(sets[1][0], **hyper, **sets[1][2])
+    gen = _gen(73)
+    _, grads = _shaped(shapes, offsets, dtype=gdtype)
+    for t in range(8):
+        _fill_grads(grads, gen, std=1e-3, mean=5e-4)
+        pair.step(grads)
+        twin.step(grads)
+        assert pair.opt.trust_ratios() == twin.trust_ratios()
+        np.testing.assert_allclose(pair.opt.trust_ratios(), pair.oracle.trust[-1], rtol=2e-6)
+    pair.check("layer adaptation in one launch")
+    for i, (x, y) in enumerate(zip(sets[0][0], sets[1][0])):
+        assert torch.equal(x, y)
+        assert torch.equal(sets[0][1][i], sets[1][1][i])
+        assert torch.equal(sets[0][1][i].view(x.shape), x.to(torch.bfloat16))
+        sa, sb = pair.opt.state(i), twin.state(i)
+        for key in ("m", "v", "slow", "acc"):
+            assert (sa[key] is None and sb[key] is None) or torch.equal(sa[key], sb[key])
+    assert pair.opt.info()["launches"] == 8 and twin.info()["launches"] == 24
 
 
 def test_layer_adaptation_zero_gradient_and_reruns():

@@ -43,10 +43,13 @@ def _device_grads(gs64, offsets=None):
     return views
 
 
+@pytest.mark.parametrize("route", ["restore", "fused"])
 @pytest.mark.parametrize("offsets", [None, "phased"])
-def test_closed_loop_with_fallback(offsets):
+def test_closed_loop_with_fallback(offsets, route):
     """N_taylor = 4 of 9 steps: look ahead, compare theta~ with Eq. 10, restore bit for
-    bit, step on the closure's gradient; from step 5 on plain steps (Eq. 13)."""
+    bit (route "restore") or let the step read theta_{t-1} from the save buffer (route
+    "fused": no restore pass), step on the closure's gradient; from step 5 on plain steps
+    (Eq. 13)."""
     offs = [(i % 4) if i % 3 == 2 else 0 for i in range(len(RAGGED))] if offsets else None
     _, params = _fresh(RAGGED, offs)
     pair = Pair(params, dict(BASE, true_nesterov_steps=4))
@@ -63,9 +66,10 @@ def test_closed_loop_with_fallback(offsets):
             for i, p in enumerate(params):
                 assert_close(p, point[i], f"t={t} theta~[{i}]")
             gs = grad_of(point)
-            pair.opt.restore()
-            for p, b in zip(params, before):
-                assert torch.equal(p, b), "restore must be bit-exact"
+            if route == "restore":
+                pair.opt.restore()
+                for p, b in zip(params, before):
+                    assert torch.equal(p, b), "restore must be bit-exact"
         else:
             gs = grad_of(pair.oracle.theta)
         pair.step(_device_grads(gs, offs))
@@ -76,6 +80,45 @@ def test_closed_loop_with_fallback(offsets):
     pair.check("end")
     assert wanted == [True] * 4 + [False] * 5
     assert not pair.opt.info()["warnings"] & B.NOVAK_WARN_TRUE_DOWNGRADED
+    assert pair.opt.info()["launches"] == 9 + (8 if route == "restore" else 4)
+
+
+@pytest.mark.parametrize("extra", [dict(), dict(lookahead_mode="traj_mean", lookahead_k=2),
+                                   dict(layer_adaptation=True),
+                                   dict(auto_lr=True, clip_threshold=0.05),
+                                   dict(moment_dtype="bf16"), dict(lookahead_k=0)])
+def test_step_behind_the_look_ahead_equals_restore_then_step(extra):
+    """The two routes, side by side on twin handles: extrapolate, restore, step against
+    extrapolate, step.  Parameters and every state array bit for bit the same after each
+    of 6 steps (4 of them true steps), also where another kernel reads theta_{t-1} first
+    (the norms of layer adaptation and of the automatic learning-rate scaling)."""
+    offs = [(i % 4) if i % 3 == 2 else 0 for i in range(len(RAGGED))]
+    _, pa = _fresh(RAGGED, offs)
+    _, pb = _fresh(RAGGED, offs)
+    hyper = dict(BASE, true_nesterov_steps=4, **extra)
+    a = B.NovakOptimizer(pa, **hyper)
+    b = B.NovakOptimizer(pb, **hyper)
+    gen = torch.Generator(device=DEV).manual_seed(12)
+    for t in range(1, 7):
+        _, grads, _ = make_tensors(RAGGED, DEV, offs)
+        for g in grads:
+            g.normal_(0.0, 1e-2, generator=gen)
+        if a.wants_extrapolation():
+            a.extrapolate()
+            a.restore()
+            b.extrapolate()
+            if t > 1:
+                assert not torch.equal(pb[-2], pa[-2])      # b's parameters still sit at theta~
+        a.step(grads)
+        b.step(grads)
+        torch.cuda.synchronize()
+        for x, y in zip(pa, pb):
+            assert torch.equal(x, y), f"t={t}"
+        for i in range(len(RAGGED)):
+            sa, sb = a.state(i), b.state(i)
+            for k in ("m", "v", "slow", "acc"):
+                assert (sa[k] is None and sb[k] is None) or torch.equal(sa[k], sb[k]), (t, i, k)
+    assert a.info()["launches"] - b.info()["launches"] == 4
 
 
 def test_first_look_ahead_is_the_identity_and_m_is_read_not_written():
@@ -136,8 +179,6 @@ def test_state_machine_refusals():
     opt.extrapolate()
     with pytest.raises(B.NovakError):
         opt.extrapolate()                                          # twice
-    with pytest.raises(B.NovakError):
-        opt.step(g)                                                # would step on theta~
     gl = opt.prepare(g)
     with pytest.raises(B.NovakError):
         opt.handle.step_noalloc(opt._params_arr, gl.arr, opt._numel_arr, opt.n, gl.dtype, 0)
@@ -150,6 +191,12 @@ def test_state_machine_refusals():
     opt.restore()
     opt.step(g)
     assert opt.info()["t"] == 1
+    # novak_step may follow the look-ahead directly; there is nothing to restore afterwards
+    opt.extrapolate()
+    opt.step(g)
+    assert opt.info()["t"] == 2
+    with pytest.raises(B.NovakError):
+        opt.restore()
     # short and misaligned save buffers
     need = opt.handle.nesterov_save_bytes()
     buf = torch.empty(need + 64, dtype=torch.uint8, device=DEV)
@@ -194,11 +241,12 @@ def test_fullsize_resnet50_launch_configuration():
             assert_close(pair.flat_p[pair.idx], pair.oracle.extrapolated()[0], f"t={t} theta~")
             if t > 1:
                 assert not torch.equal(pair.flat_p, before)
-            pair.opt.restore()
-            assert torch.equal(pair.flat_p, before)
-            del before
+            if t % 2 == 0:
+                pair.opt.restore()
+                assert torch.equal(pair.flat_p, before)
+            del before                   # odd steps: the step reads the save buffer itself
         pair.step(threads=8)
     pair.check()
-    assert pair.opt.info()["launches"] == 8 + 2 * 5
+    assert pair.opt.info()["launches"] == 8 + 2 * 2 + 3
     del pair
     torch.cuda.empty_cache()
