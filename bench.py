@@ -89,8 +89,8 @@ def parse_args():
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
     ap.add_argument("--layer-adaptation-in-step", type=int, default=None, choices=[0, 1],
-                    help="0: layer adaptation as two statistics kernels and the step (default 1: "
-                         "one persistent kernel whose update items find their tensor in L2)")
+                    help="1: layer adaptation and update as one kernel whose update items find "
+                         "their tensor in L2 (default 0: two statistics kernels, then the step)")
     ap.add_argument("--layer-adaptation-lead", type=int, default=None,
                     help="elements by which that kernel's statistics run ahead of its updates")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
@@ -610,7 +610,7 @@ def main():
     per_elem_twice = 4 + 2 * mbytes + gbytes
     big = sum(n for n in wl.numel if n * per_elem_twice > 48e6) / wl.total
     trust_share = 0.0 if not args.layer_adaptation else (
-        big if (args.layer_adaptation_in_step != 0 and not prepass) else 1.0)
+        big if (args.layer_adaptation_in_step == 1 and not prepass) else 1.0)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
                                          trust_share, args.bf16_copy, args.auto_lr,
                                          ("restore" if args.restore_pass else True) if args.true_nesterov else False,

@@ -154,18 +154,22 @@ enum {
                                      clipping, no automatic learning-rate scaling, no
                                      layer adaptation), novak_step forms the row means
                                      of Eq. 26 inside the step kernel, whose CTAs then
-                                     own whole rows (rows of up to 32768 elements;
-                                     longer ones keep the statistics pass): one launch
-                                     and 28 B per element instead of three launches and
-                                     32 B.  0: always the statistics pass              */
-    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1 (default): with layer adaptation on and no
-                                     clipping, centralization or automatic learning-
-                                     rate scaling, novak_step runs statistics and
-                                     update as ONE kernel in which a tensor's update
-                                     follows its statistics closely enough to find its
-                                     theta, g, m, v still in L2 (about 28 B per
-                                     element from DRAM instead of 44).  0: two
-                                     statistics kernels, then the step                */
+                                     own whole rows (units of 8192 elements or one
+                                     row of up to 32768; longer rows keep the
+                                     statistics pass): one launch and 28 B per element
+                                     instead of three launches and 32 B.  0: always
+                                     the statistics pass                               */
+    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1: with layer adaptation on and no clipping,
+                                     centralization or automatic learning-rate
+                                     scaling, novak_step runs statistics and update as
+                                     ONE kernel in which a tensor's update follows its
+                                     statistics closely enough to find its theta, g,
+                                     m, v still in L2 (about 28 B per element from
+                                     DRAM instead of 44; measured slower all the same,
+                                     the kernel being bound by instruction issue and
+                                     latency, not by DRAM).  0 (default): two
+                                     statistics kernels, then the step.  Same results
+                                     bit for bit                                      */
     NOVAK_OPT_LAYER_ADAPTATION_LEAD = 26, /* how far, in elements, that kernel's statistics
                                      run ahead of its updates (default 2^21: 32 MB of
                                      theta, g, m, v); only before the first such step */
@@ -585,7 +589,7 @@ int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, 
 
 /* Host-only helper exposing the units of the step kernel that centralizes by
  * itself (NOVAK_OPT_CENTRALIZE_IN_STEP): whole rows [row0, row0 + n_rows) of the
- * tensors whose rows have at most 32768 elements, as many rows as fit in 4096
+ * tensors whose rows have at most 32768 elements, as many rows as fit in 8192
  * elements (at least one, at most 256) per unit; tensors with longer rows get
  * no unit (they keep the statistics pass).  Arguments and result as in
  * novak_build_row_units. */

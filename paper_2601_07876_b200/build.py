@@ -7,6 +7,8 @@ import os
 import shutil
 import subprocess
 import sys
+import tempfile
+import zlib
 from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
@@ -67,7 +69,9 @@ def up_to_date(out: str = LIB) -> bool:
     return all(os.path.getmtime(f) <= t for f in SOURCES + HEADERS + [os.path.abspath(__file__)])
 
 
-OBJ_CACHE = os.path.join(PKG, "_build")     # objects and their dependency lists, kept between builds
+# objects and their dependency lists, kept between builds (outside the source tree: the
+# tree is what gets copied around, and the objects are as large as the library)
+OBJ_CACHE = os.path.join(tempfile.gettempdir(), "novak_build_%08x" % (zlib.crc32(PKG.encode()) & 0xffffffff))
 
 
 def _object_is_current(obj: str, flags_key: str) -> bool:
@@ -87,7 +91,7 @@ def _object_is_current(obj: str, flags_key: str) -> bool:
 def build(force: bool = False, verbose: bool = False, extra: list[str] | None = None,
           out: str = LIB) -> str:
     """Compiles the library if a source is newer than the built file.  Objects are kept
-    under _build/ with nvcc's dependency lists, so that a later build recompiles only the
+    in a cache directory under the system's temporary directory with nvcc's dependency lists, so that a later build recompiles only the
     units whose sources changed; force=True recompiles everything."""
     if not force and not extra and out == LIB and up_to_date():
         return LIB

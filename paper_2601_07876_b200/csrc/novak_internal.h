@@ -90,7 +90,7 @@ struct __align__(16) RowUnit {
 // fit in kOwnUnitElems elements (at most kOwnUnitRows), or one longer row;
 // rows beyond kOwnRowMax keep the statistics pass.
 constexpr uint32_t kOwnRowMax = 32768;
-constexpr uint32_t kOwnUnitElems = 4096;
+constexpr uint32_t kOwnUnitElems = 8192;
 constexpr uint32_t kOwnUnitRows = 256;
 // Units of up to this many elements pass their gradient through shared memory.
 constexpr uint32_t kOwnStageElems = 8192;

@@ -88,7 +88,10 @@ __device__ __forceinline__ unsigned long long wait_for_ratio(const unsigned long
 // Three resident CTAs per SM (85 registers) at every lookahead action: the
 // kernel holds the statistics and the update path.
 template <int NEST, int GT, int LA, int PRE>
-__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS_WIDE)
+#ifndef NOVAK_ADAPT_MIN_CTAS
+#define NOVAK_ADAPT_MIN_CTAS step_min_ctas(LA)
+#endif
+__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_ADAPT_MIN_CTAS)
 novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restrict__ item_chunk,
                         int n_items, const TensorRec *__restrict__ recs,
                         const int *__restrict__ tensor_first, double *chunk_u2, double *chunk_p2,

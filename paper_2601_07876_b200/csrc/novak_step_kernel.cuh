@@ -727,15 +727,22 @@ __device__ __forceinline__ void unit_tile_finish(TileRegs<U> &t, const UnitBody 
     }
 }
 
-// Vectors per thread and stream of the row-owning kernel's tiles: four (a tile
-// is then a whole unit of 4096 elements, every load of the unit in flight at
-// once) where the lookahead arrays are not read, two where they are.  Three
-// resident CTAs per SM (85 registers) either way.
+// Vectors per thread and stream of the row-owning kernel's tiles, and its
+// resident CTAs per SM: as the plain kernel's.  (Measured on the ResNet-50-
+// shaped set, ms per step: two vectors at four CTAs 0.138; four vectors at
+// three CTAs, a whole unit in flight at once, 0.158; one vector at six CTAs
+// 0.182.)
+#ifndef NOVAK_ROWS_U
+#define NOVAK_ROWS_U 2
+#endif
 template <int LA>
-constexpr int kRowsUnroll = (LA & (LA_S_READ | LA_A_READ)) != 0 ? 2 : 4;
+constexpr int kRowsUnroll = (LA & (LA_S_READ | LA_A_READ)) != 0 ? 2 : NOVAK_ROWS_U;
+#ifndef NOVAK_ROWS_MIN_CTAS
+#define NOVAK_ROWS_MIN_CTAS step_min_ctas(LA)
+#endif
 
 template <int NEST, int GT, int LA, int PRE>
-__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_MIN_CTAS_WIDE)
+__global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_ROWS_MIN_CTAS)
 novak_step_rows_kernel(const Chunk *__restrict__ rest, int n_rest,
                        const RowUnit *__restrict__ units, int n_units,
                        const TensorRec *__restrict__ recs, const StepScalars s)

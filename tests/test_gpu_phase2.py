@@ -327,10 +327,8 @@ def test_layer_adaptation_every_element(gdtype, extra, variant):
     pair.check(f"layer adaptation {extra}")
     seen = np.array(pair.oracle.trust)
     assert (seen == 0.1).any() and (seen == 10.0).any() and ((seen > 0.1) & (seen < 10.0)).any()
-    if extra.get("centralize") or extra.get("clip_threshold"):
-        assert pair.opt.info()["launches"] == 7 * 5     # statistics x 2, ratios x 2, the step
-    else:
-        assert pair.opt.info()["launches"] == 7         # statistics and update in one launch
+    n_pre = 2 if extra.get("centralize") or extra.get("clip_threshold") else 0
+    assert pair.opt.info()["launches"] == 7 * (3 + n_pre)
     assert pair.opt.info()["layer_adaptation"] == 1
 
 
