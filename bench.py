@@ -39,28 +39,33 @@ METRIC = "parameter updates/sec per novak_step"
 UNIT = "param-updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the step kernel from the
-# ncu captures summarised under profiles/: bytes of a non-sync and of a sync launch, and
-# the hashes of the kernel sources at capture time.  A capture stops counting (traffic
-# = null) as soon as the kernel sources differ from what was profiled.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the step kernel, by the
+# lookahead action of the launch, from the ncu captures summarised under profiles/
+# (novak_step_kernel_traffic.md): LAST: a step without / with a synchronisation;
+# TRAJ_MEAN: first step of a window, a middle step, the synchronisation step.  A capture
+# stops counting (traffic = null) as soon as the kernel sources differ from what was
+# profiled (hashes below).
+NCU_SOURCES = {"novak_step_kernel.cuh": "3d9d93c97c875874", "novak_step_types.h": "42992d0d45a7d8b6",
+               "novak_launch.cu": "2166a9fd78239db0"}
 NCU_TRAFFIC = {
-    ("resnet50", "last"): {
-        "plain": 660.21e6, "sync": 866.28e6,
-        "sources": {"novak_step_kernel.cuh": "eaa24ecab255bf4a",
-                    "novak_step_types.h": "75b76d99858631ba", "novak_launch.cu": "4a258ea7b5f62c16"},
-        "summary": "profiles/novak_step_kernel_resnet50.md",
-    },
+    ("resnet50", "last"): {"plain": 656.86e6, "sync": 861.35e6},
+    ("resnet50", "traj_mean"): {"first": 759.37e6, "middle": 860.62e6, "sync": 965.29e6},
+    ("vgg16", "last"): {"plain": 3815.71e6, "sync": 4921.80e6},
+    ("vgg16", "traj_mean"): {"first": 4372.40e6, "middle": 4921.85e6, "sync": 5481.21e6},
+    ("vit-b16", "last"): {"plain": 2190.60e6, "sync": 2882.43e6},
+    ("vit-b16", "traj_mean"): {"first": 2537.18e6, "middle": 2884.01e6, "sync": 3233.32e6},
 }
 
 
-def ncu_traffic(workload: str, mode: str, sync_fraction: float):
-    """Per-launch DRAM traffic from the committed ncu capture, averaged over the sync
-    schedule of the timed steps, or None when no capture matches the built kernel."""
+def ncu_traffic(workload: str, mode: str, k: int, t_first: int, n_steps: int):
+    """Per-launch DRAM traffic from the committed ncu captures, averaged over the lookahead
+    schedule of the timed steps [t_first, t_first + n_steps), or None when no capture
+    matches the workload or the built kernel."""
     import hashlib
     rec = NCU_TRAFFIC.get((workload, mode))
-    if rec is None:
+    if rec is None or k <= 1 or t_first <= 1:
         return None
-    for name, want in rec["sources"].items():
+    for name, want in NCU_SOURCES.items():
         path = os.path.join(ROOT, "paper_2601_07876_b200", "csrc", name)
         try:
             with open(path, "rb") as f:
@@ -68,7 +73,15 @@ def ncu_traffic(workload: str, mode: str, sync_fraction: float):
                     return None
         except OSError:
             return None
-    return (1.0 - sync_fraction) * rec["plain"] + sync_fraction * rec["sync"]
+    total = 0.0
+    for t in range(t_first, t_first + n_steps):
+        if t % k == 0:
+            total += rec["sync"]
+        elif mode == "last":
+            total += rec["plain"]
+        else:
+            total += rec["first"] if (t - 1) % k == 0 else rec["middle"]
+    return total / n_steps
 
 
 def parse_args():
@@ -471,6 +484,7 @@ def time_one_workload(torch, B, W, dev, index, mode, steps, warmup, min_seconds,
            "p10": quantile(per, 0.1), "p90": quantile(per, 0.9),
            "updates_per_s": wl.total / (ms * 1e-3), "algorithmic_bytes_per_elem": alg,
            "hbm_gbs": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0,
+           "traffic": ncu_traffic(wl.name, mode, k, t_first, steps * repeats),
            "grad_pool": pool_n, "launches": opt.info()["launches"]}
     del opt, pool, pool_flat, params, flat_p
     torch.cuda.empty_cache()
@@ -619,8 +633,9 @@ def main():
     bytes_per_launch = alg * wl.total
     achieved = bytes_per_launch / (ms_per_step * 1e-3) / 1e9
     peak, peak_src = measured_peak()
-    n_sync = sum(1 for t in range(t_first, t_first + n_timed) if k > 0 and t % k == 0)
-    traffic = None if (prepass or args.layer_adaptation or args.bf16_copy or args.true_nesterov or mbytes == 2) else ncu_traffic(wl.name, args.lookahead_mode, n_sync / n_timed)
+    traffic = None if (prepass or args.layer_adaptation or args.bf16_copy or args.true_nesterov
+                       or mbytes == 2 or args.grad_offset) else \
+        ncu_traffic(wl.name, args.lookahead_mode, k, t_first, n_timed)
 
     # ---------------- per-step distribution (separate short pass, event per step)
     per = {}
@@ -708,7 +723,7 @@ def main():
             "p10": quantile(per_region, 0.1), "p90": quantile(per_region, 0.9),
             "updates_per_s": value, "algorithmic_bytes_per_elem": alg, "hbm_gbs": achieved,
             "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
-            "grad_pool": pool_n, "headline": True}]
+            "traffic": traffic, "grad_pool": pool_n, "headline": True}]
         free_bytes, _ = torch.cuda.mem_get_info()
         for index in range(5):
             for mode in ("last", "traj_mean"):
