@@ -141,7 +141,14 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_last_error": (c_char_p, [vp]),
     }
     for name, (res, args) in sigs.items():
-        fn = getattr(lib, name)
+        try:
+            fn = getattr(lib, name)
+        except AttributeError:
+            # an alternative build given by path (tuning, A/B against an older build) may
+            # lack the host-only table-builder hooks; the library proper must have everything
+            if path != _build.LIB and name.startswith("novak_build_"):
+                continue
+            raise
         fn.restype = res
         fn.argtypes = args
     if path == _build.LIB:
