@@ -154,7 +154,7 @@ enum {
                                      clipping, no automatic learning-rate scaling, no
                                      layer adaptation), novak_step forms the row means
                                      of Eq. 26 inside the step kernel, whose CTAs then
-                                     own whole rows (units of 8192 elements or one
+                                     own whole rows (units of 4096 elements or one
                                      row of up to 32768; longer rows keep the
                                      statistics pass): one launch and 28 B per element
                                      instead of three launches and 32 B.  0: always
@@ -589,7 +589,7 @@ int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, 
 
 /* Host-only helper exposing the units of the step kernel that centralizes by
  * itself (NOVAK_OPT_CENTRALIZE_IN_STEP): whole rows [row0, row0 + n_rows) of the
- * tensors whose rows have at most 32768 elements, as many rows as fit in 8192
+ * tensors whose rows have at most 32768 elements, as many rows as fit in 4096
  * elements (at least one, at most 256) per unit; tensors with longer rows get
  * no unit (they keep the statistics pass).  Arguments and result as in
  * novak_build_row_units. */

@@ -143,7 +143,7 @@ cudaError_t launch_step_rows(const Chunk *d_rest, int n_rest, const RowUnit *d_u
     if (!fn) return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(n_rest + n_units));
-    lc.blockDim = dim3(kBlock);
+    lc.blockDim = dim3(kOwnBlockThreads);
     lc.dynamicSmemBytes = 0;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];

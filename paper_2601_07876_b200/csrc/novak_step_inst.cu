@@ -12,6 +12,14 @@
 #error "compile with -DNOVAK_PRE_MODE=<mode bits>"
 #endif
 
+// The row-owning kernel (PRE_CENTER_ROWS modes) runs in CTAs of 128 threads, eight
+// resident per SM (six where lookahead arrays are read): see kOwnBlockThreads.
+#if ((NOVAK_PRE_MODE) & 3) == 3 && !defined(NOVAK_INST_DYN) && !defined(NOVAK_INST_ADAPT)
+#define NOVAK_BLOCK 128
+#define NOVAK_MIN_CTAS 8
+#define NOVAK_MIN_CTAS_WIDE 6
+#endif
+
 #define NOVAK_PASTE2(a, b) a##b
 #define NOVAK_PASTE(a, b) NOVAK_PASTE2(a, b)
 

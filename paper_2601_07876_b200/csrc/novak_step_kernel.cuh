@@ -731,10 +731,10 @@ __device__ __forceinline__ void unit_tile_finish(TileRegs<U> &t, const UnitBody 
 }
 
 // Vectors per thread and stream of the row-owning kernel's tiles, and its
-// resident CTAs per SM: as the plain kernel's.  (Measured on the ResNet-50-
-// shaped set, ms per step: two vectors at four CTAs 0.138; four vectors at
-// three CTAs, a whole unit in flight at once, 0.158; one vector at six CTAs
-// 0.182.)
+// registers per thread: as the plain kernel's.  (Measured on the ResNet-50-
+// shaped set with CTAs of 256 threads, ms per step: two vectors at four CTAs
+// 0.138; four vectors at three CTAs, a whole unit in flight at once, 0.158; one
+// vector at six CTAs 0.182.)
 #ifndef NOVAK_ROWS_U
 #define NOVAK_ROWS_U 2
 #endif
@@ -751,6 +751,8 @@ novak_step_rows_kernel(const Chunk *__restrict__ rest, int n_rest,
                        const TensorRec *__restrict__ recs, const StepScalars s)
 {
     static_assert((PRE & PRE_MASK) == PRE_CENTER_ROWS, "the row-owning kernel is its own mode");
+    static_assert((PRE & PRE_MASK) != PRE_CENTER_ROWS || kBlock == kOwnBlockThreads,
+                  "compiled for the block size it is launched with");
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
     constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
     constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;

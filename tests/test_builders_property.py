@@ -63,7 +63,7 @@ def test_row_units_cover_every_row_once(data):
 def test_own_units_cover_the_rows_of_owned_tensors_once(data):
     """Units of the step kernel that forms its row means itself: every row of every tensor
     whose rows have at most 32768 elements exactly once, whole rows only, at most 256 rows
-    and (beyond one row) at most 8192 elements per unit; nothing for longer rows."""
+    and (beyond one row) at most 4096 elements per unit; nothing for longer rows."""
     n = data.draw(st.integers(1, 8))
     numel, rows = [], []
     for _ in range(n):
@@ -82,7 +82,7 @@ def test_own_units_cover_the_rows_of_owned_tensors_once(data):
     for t, row0, n_rows in units:
         assert t in owned and 1 <= n_rows <= 256
         L = numel[t] // rows[t]
-        assert n_rows == 1 or n_rows * L <= 8192
+        assert n_rows == 1 or n_rows * L <= 4096
         seen[t][row0:row0 + n_rows] += 1
     assert all((s == 1).all() for s in seen.values())
     # consecutive units of a tensor are adjacent and in order
