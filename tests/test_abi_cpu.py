@@ -140,6 +140,28 @@ def test_graph_capturable_option():
     h.destroy()
 
 
+def test_in_step_options_roundtrip_and_defaults():
+    """Centralization inside the step kernel is on by default, the one-launch layer
+    adaptation off; its lead is an element count."""
+    h = B.Handle(**GOOD)
+    assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 1
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 0
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 2 ** 21
+    h.set_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP, 0)
+    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 1)
+    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0)
+    assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 0
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 1
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 0
+    for key, bad in ((B.NOVAK_OPT_CENTRALIZE_IN_STEP, 2), (B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, -1),
+                     (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, -1), (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0.5),
+                     (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 2.0 ** 31)):
+        with pytest.raises(B.NovakError) as e:
+            h.set_option(key, bad)
+        assert e.value.status == B.NOVAK_EINVAL
+    h.destroy()
+
+
 def test_options_validate_and_roundtrip():
     h = B.Handle(**GOOD)
     assert h.get_option(B.NOVAK_OPT_NESTEROV_BETA) == 0.9   # default beta_N = beta1
