@@ -92,10 +92,10 @@ struct Handle {
     // step kernel that forms the row means itself (PRE_CENTER_ROWS): the chunk-table
     // entries of the tensors it does not own rows of, and its units of whole rows
     int center_in_step = 1;             // NOVAK_OPT_CENTRALIZE_IN_STEP
-    bool prep_rows_layout = false;      // the scratch is laid out for that kernel
     Chunk *d_rest = nullptr;
     RowUnit *d_own = nullptr;
-    int n_rest = 0, n_own = 0;
+    RowUnit *d_long_units = nullptr;    // statistics units of the tensors with rows too long to own
+    int n_rest = 0, n_own = 0, n_long_units = 0;
     int64_t rows_gen = 0;               // bumped whenever the row settings change
     int64_t prep_key = -1;              // rows_gen and centring the scratch was laid out for
     // the averages of Eq. 20-21 live in the scratch; values waiting to be written there
@@ -220,7 +220,7 @@ int pre_mode(const novak_opt *o);
 // kernel can centralize by itself (whole_table: the step is one launch over the
 // whole group, as in novak_step).
 int step_pre_mode(const novak_opt *o, bool whole_table);
-int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream);
+int prepare_prep(novak_opt *o, cudaStream_t stream);
 void fill_info(const novak_opt *o, const Plan &p, novak_info *out);
 
 // Device work tables (novak_host_device.cpp).

@@ -57,6 +57,9 @@ void release_device(novak_opt *o)
     o->d_plain = nullptr;
     o->d_units = nullptr;
     o->n_plain = o->n_units = 0;
+    o->d_rest = nullptr;
+    o->d_own = o->d_long_units = nullptr;
+    o->n_rest = o->n_own = o->n_long_units = 0;
     o->prep_key = -1;
     o->row_mean = nullptr;
     for (cudaEvent_t ev : o->host_ev) cudaEventDestroy(ev);
@@ -136,10 +139,10 @@ void invalidate_tables(novak_opt *o)
 
 // Scratch of the statistics pass, laid out when a step first needs it and
 // again when the row settings change.
-int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream)
+int prepare_prep(novak_opt *o, cudaStream_t stream)
 {
     const bool centre = o->h.centralize && o->total_rows > 0;
-    const int64_t key = o->rows_gen * 4 + (centre ? 1 : 0) + (rows_layout ? 2 : 0);
+    const int64_t key = o->rows_gen * 2 + (centre ? 1 : 0);
     if (o->d_prep && o->prep_key == key) return NOVAK_OK;
     cudaError_t e;
     if (o->d_prep) {
@@ -156,31 +159,34 @@ int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream)
         o->d_prep = nullptr;
         invalidate_tables(o);
     }
-    // work of the pass: row units for the tensors with rows, chunk-table entries for the rest
-    std::vector<RowUnit> units, own;
+    // Work of the statistics pass: row units for the tensors with rows, chunk-table
+    // entries for the rest.  With centralization the same allocation also holds the
+    // tables of the step kernel that owns rows (used by steps that need no statistic
+    // of the whole gradient): its units of whole rows, the chunk-table entries of the
+    // tensors it does not own (those without rows, and those with rows too long to
+    // own), and the statistics units of the latter, which is all the pass then has to
+    // do.  Both sets are built together, so a caller may alternate between entry points
+    // that use one or the other without any reallocation.
+    std::vector<RowUnit> units, own, long_units;
     std::vector<Chunk> plain, rest;
-    if (centre && rows_layout) {
-        // The step kernel owns the rows of up to kOwnRowMax elements.  The statistics
-        // pass shrinks to the tensors with longer rows (no norm is needed: nothing for
-        // its plain part); the step kernel takes those tensors, and the ones without
-        // rows, by chunk-table entries.
+    if (centre) {
+        build_row_units(o->numel.data(), o->rows.data(), o->n, units);
+        for (const Chunk &c : o->h_chunks)
+            if (o->rows[c.tensor] <= 0) plain.push_back(c);
         build_own_units(o->numel.data(), o->rows.data(), o->n, own);
         std::vector<int64_t> long_rows(o->rows.size(), 0);
         for (int i = 0; i < o->n; ++i)
             if (o->rows[i] > 0 && o->numel[i] / o->rows[i] > static_cast<int64_t>(novak::kOwnRowMax))
                 long_rows[i] = o->rows[i];
-        build_row_units(o->numel.data(), long_rows.data(), o->n, units);
+        build_row_units(o->numel.data(), long_rows.data(), o->n, long_units);
         for (const Chunk &c : o->h_chunks)
             if (o->rows[c.tensor] <= 0 || long_rows[c.tensor] > 0) rest.push_back(c);
-    } else if (centre) {
-        build_row_units(o->numel.data(), o->rows.data(), o->n, units);
-        for (const Chunk &c : o->h_chunks)
-            if (o->rows[c.tensor] <= 0) plain.push_back(c);
     }
     const size_t n_plain = centre ? plain.size() : static_cast<size_t>(o->n_chunks);
     if (units.size() > static_cast<size_t>(INT32_MAX) / 2 || own.size() > static_cast<size_t>(INT32_MAX) / 2)
         return fail(o, NOVAK_EINVAL, "too many rows");
     // sized for fp32 gradients; bf16 gradients take more entries per CTA and need less
+    // (the pass over the long rows alone needs fewer sums than the pass over everything)
     const size_t n_work = static_cast<size_t>(novak::grad_stats_work(
         static_cast<int>(n_plain), static_cast<int>(units.size()), NOVAK_GRAD_F32));
     const size_t nc = static_cast<size_t>(o->n_chunks);
@@ -195,6 +201,7 @@ int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream)
     const size_t off_rest = off;    off += rest.size() * sizeof(Chunk);
     const size_t off_units = off;   off += units.size() * sizeof(RowUnit);
     const size_t off_own = off;     off += own.size() * sizeof(RowUnit);
+    const size_t off_long = off;    off += long_units.size() * sizeof(RowUnit);
     const size_t off_mean = off;    off += static_cast<size_t>(o->total_rows) * sizeof(float2);
     const size_t bytes = off + 16;
     if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_prep), bytes)) != cudaSuccess) {
@@ -212,30 +219,26 @@ int prepare_prep(novak_opt *o, bool rows_layout, cudaStream_t stream)
     o->d_rest = reinterpret_cast<Chunk *>(o->d_prep + off_rest);
     o->d_units = reinterpret_cast<RowUnit *>(o->d_prep + off_units);
     o->d_own = reinterpret_cast<RowUnit *>(o->d_prep + off_own);
+    o->d_long_units = reinterpret_cast<RowUnit *>(o->d_prep + off_long);
     o->row_mean = reinterpret_cast<float2 *>(o->d_prep + off_mean);
-    o->n_plain = (centre && rows_layout) ? 0 : static_cast<int>(n_plain);
+    o->n_plain = static_cast<int>(n_plain);
     o->n_units = static_cast<int>(units.size());
     o->n_rest = static_cast<int>(rest.size());
     o->n_own = static_cast<int>(own.size());
-    o->prep_rows_layout = centre && rows_layout;
+    o->n_long_units = static_cast<int>(long_units.size());
     // The tables are built once per layout: blocking copies keep the host
     // vectors' lifetime trivial.
-    if (!plain.empty() &&
-        (e = cudaMemcpyAsync(o->d_plain, plain.data(), plain.size() * sizeof(Chunk),
-                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-        return fail_cuda(o, e, "statistics table upload");
-    if (!rest.empty() &&
-        (e = cudaMemcpyAsync(o->d_rest, rest.data(), rest.size() * sizeof(Chunk),
-                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-        return fail_cuda(o, e, "step table upload");
-    if (!units.empty() &&
-        (e = cudaMemcpyAsync(o->d_units, units.data(), units.size() * sizeof(RowUnit),
-                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-        return fail_cuda(o, e, "row unit upload");
-    if (!own.empty() &&
-        (e = cudaMemcpyAsync(o->d_own, own.data(), own.size() * sizeof(RowUnit),
-                             cudaMemcpyHostToDevice, stream)) != cudaSuccess)
-        return fail_cuda(o, e, "row unit upload");
+    const struct { void *dst; const void *src; size_t bytes; } uploads[] = {
+        {o->d_plain, plain.data(), plain.size() * sizeof(Chunk)},
+        {o->d_rest, rest.data(), rest.size() * sizeof(Chunk)},
+        {o->d_units, units.data(), units.size() * sizeof(RowUnit)},
+        {o->d_own, own.data(), own.size() * sizeof(RowUnit)},
+        {o->d_long_units, long_units.data(), long_units.size() * sizeof(RowUnit)},
+    };
+    for (const auto &u : uploads)
+        if (u.bytes != 0 &&
+            (e = cudaMemcpyAsync(u.dst, u.src, u.bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return fail_cuda(o, e, "statistics table upload");
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return fail_cuda(o, e, "statistics table upload");
     o->prep_key = key;
     invalidate_tables(o);              // records carry pointers into this scratch

@@ -82,9 +82,7 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     int rc;
     if (!o->d_chunks && (rc = prepare_device(o, stream)) != NOVAK_OK) return rc;
     ctx->pre = step_pre_mode(o, whole_table);
-    if (ctx->pre != novak::PRE_NONE &&
-        (rc = prepare_prep(o, ctx->pre == novak::PRE_CENTER_ROWS, stream)) != NOVAK_OK)
-        return rc;
+    if (ctx->pre != novak::PRE_NONE && (rc = prepare_prep(o, stream)) != NOVAK_OK) return rc;
     if (o->ema_pending && o->prep_out) {
         // averages set by the caller (or saved over a reallocation) go into the scratch
         const double ema[2] = {o->pending_g_bar, o->pending_theta_bar};
@@ -125,7 +123,7 @@ cudaError_t launch_statistics(novak_opt *o, const StepCtx &ctx, bool finalize, c
 {
     if (ctx.pre == novak::PRE_NONE) return cudaSuccess;
     // the step kernel owns its rows: only tensors with longer rows need the pass
-    if (ctx.pre == novak::PRE_CENTER_ROWS && o->n_units == 0) return cudaSuccess;
+    if (ctx.pre == novak::PRE_CENTER_ROWS && o->n_long_units == 0) return cudaSuccess;
     *what = "gradient statistics kernel launch";
     const cudaError_t e = launch_stats(o, ctx, finalize, stream);
     if (e == cudaSuccess) *launches += o->h.auto_lr ? 3 : 2;
@@ -160,10 +158,18 @@ cudaError_t launch_prepasses(novak_opt *o, const StepCtx &ctx, cudaStream_t stre
 cudaError_t launch_stats(novak_opt *o, const StepCtx &ctx, bool finalize, cudaStream_t stream)
 {
     novak::StatsPlan plan;
-    plan.plain = o->d_plain ? o->d_plain : o->d_chunks;
-    plan.n_plain = o->n_plain;
-    plan.units = o->d_units;
-    plan.n_units = o->n_units;
+    if (ctx.pre == novak::PRE_CENTER_ROWS) {
+        // no norm is needed: only the means of the rows too long for the step kernel to own
+        plan.plain = nullptr;
+        plan.n_plain = 0;
+        plan.units = o->d_long_units;
+        plan.n_units = o->n_long_units;
+    } else {
+        plan.plain = o->d_plain ? o->d_plain : o->d_chunks;
+        plan.n_plain = o->n_plain;
+        plan.units = o->d_units;
+        plan.n_units = o->n_units;
+    }
     plan.recs = ctx.d_recs;
     plan.chunks = o->d_chunks;
     plan.n_chunks = o->n_chunks;

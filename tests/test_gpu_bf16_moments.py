@@ -162,6 +162,20 @@ def test_with_clipping_centralization_and_layer_adaptation():
     np.testing.assert_allclose(tr, pair.oracle.trust[-1], rtol=2e-3)
 
 
+def test_centralization_inside_the_step_kernel_with_bf16_moments():
+    """The row-owning step kernel (centralization alone) in its bf16-moment instantiation."""
+    shapes = [(64, 33), (1000,), (16, 3, 5, 5), (7,), (300, 40), (3, 4608)]
+    numels = [int(np.prod(s)) for s in shapes]
+    params = _fresh(numels, shapes=shapes)
+    pair = Pair(params, dict(BASE, centralize=True))
+    pair.oracle.track_rounding_margin = True
+    gen = _gen(22)
+    for _ in range(8):
+        pair.step(_grads(numels, gen, shapes=shapes))
+    _check(pair, max_fraction=0.1)
+    assert pair.opt.info()["launches"] == 8
+
+
 def test_true_nesterov_reads_bf16_first_moments():
     numels = [5000, 77, 2048]
     params = _fresh(numels)

@@ -156,6 +156,47 @@ def test_row_owning_step_is_bit_identical_from_run_to_run_and_takes_misphased_gr
     assert pair.opt.info()["launches"] == 5
 
 
+def test_row_owning_step_and_host_step_alternate_on_one_handle():
+    """novak_step (row-owning kernel) and novak_step_host (statistics pass, the step in
+    runs) take turns on one handle with centralization alone: both routes against the
+    oracle, and no reallocation of the scratch in between (one layout serves both)."""
+    shapes = [(20, 300), (31,), (9, 1000), (3,), (2, 40000)]
+    numels = [math.prod(s) for s in shapes]
+    _, params = _shaped(shapes, [0] * 5)
+    gen = _gen(29)
+    for p in params:
+        p.normal_(0.0, 0.05, generator=gen)
+    pair = Pair(params, dict(BASE, lookahead_k=2, centralize=True))
+    opt = pair.opt
+    opt.handle.set_option(B.NOVAK_OPT_HOST_SEGMENT_ELEMS, 8192)
+    total = sum(numels)
+    h_g = torch.empty(total, dtype=torch.float32).pin_memory()
+    h_p = torch.empty(total, dtype=torch.float32).pin_memory()
+    d_g = torch.empty(total, dtype=torch.float32, device=DEV)
+    offs = np.concatenate([[0], np.cumsum(numels)])[:-1]
+    hg = B.ptr_array([h_g.data_ptr() + 4 * int(o) for o in offs])
+    hp = B.ptr_array([h_p.data_ptr() + 4 * int(o) for o in offs])
+    dg = B.ptr_array([d_g.data_ptr() + 4 * int(o) for o in offs])
+    stream = torch.cuda.current_stream().cuda_stream
+    _, grads = _shaped(shapes, [0] * 5)
+    for t in range(6):
+        _fill_grads(grads, gen, std=1e-3, mean=1e-3)
+        if t % 2 == 0:
+            pair.step(grads)
+        else:
+            h_g.copy_(torch.cat([g.reshape(-1) for g in grads]).cpu())
+            opt.handle.step_host(hp, hg, opt._params_arr, dg, opt._numel_arr, len(numels),
+                                 B.NOVAK_GRAD_F32, stream)
+            info = opt.info()
+            if info["is_sync"]:
+                pair.sync_steps.append(info["t"])
+            pair.rect_flags.append(info["rect_branch"])
+            pair.oracle.step([to_f64(g) for g in grads])
+            torch.cuda.synchronize()
+            assert torch.equal(h_p, torch.cat([p.reshape(-1) for p in params]).cpu())
+    pair.check("row-owning step and host step in turns")
+
+
 def test_phase2_is_bit_identical_from_run_to_run_and_across_launch_options():
     results = []
     for kw in (dict(), dict(), dict(dependent_launch=False), dict(chunk_elems=1024)):
