@@ -106,6 +106,8 @@ def parse_args():
                          "their tensor in L2 (default 0: two statistics kernels, then the step)")
     ap.add_argument("--layer-adaptation-lead", type=int, default=None,
                     help="elements by which that kernel's statistics run ahead of its updates")
+    ap.add_argument("--layer-adaptation-group", type=int, default=None,
+                    help="chunk-table entries per CTA of that kernel (1..8)")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")
     ap.add_argument("--zero1", action="store_true",
                     help="one group sharded over the ranks (reduce-scatter, step on the owned "
@@ -546,6 +548,7 @@ def main():
                            centralize_in_step=args.centralize_in_step,
                            layer_adaptation_in_step=args.layer_adaptation_in_step,
                            layer_adaptation_lead=args.layer_adaptation_lead,
+                           layer_adaptation_group=args.layer_adaptation_group,
                            chunk_elems=args.chunk_elems,
                            ctas_per_sm=args.ctas_per_sm, serpentine=args.serpentine,
                            dependent_launch=args.dependent_launch, lib=lib)

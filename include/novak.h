@@ -171,8 +171,11 @@ enum {
                                      statistics kernels, then the step.  Same results
                                      bit for bit                                      */
     NOVAK_OPT_LAYER_ADAPTATION_LEAD = 26, /* how far, in elements, that kernel's statistics
-                                     run ahead of its updates (default 2^21: 32 MB of
-                                     theta, g, m, v); only before the first such step */
+                                     run ahead of its updates (default 2^22); only
+                                     before the first such step                        */
+    NOVAK_OPT_LAYER_ADAPTATION_GROUP = 27, /* chunk-table entries one CTA of that kernel
+                                     takes, 1..8 (default 4); only before the first
+                                     such step                                         */
     NOVAK_OPT_GRAPH_CAPTURABLE = 23, /* Without it every step entry point returns
                                      NOVAK_ESTATE while its stream is being captured (a
                                      replay would repeat ONE step's scalars).
@@ -599,14 +602,16 @@ int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, 
 /* Host-only helper exposing the order in which the one-launch form of layer
  * adaptation (NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) takes its items.  The group's
  * chunk table lists tensor i's entries at [tensor_first[i], tensor_first[i+1])
- * (n + 1 values, non-decreasing, tensor_first[0] = 0).  out[k] is the k-th item:
- * a chunk-table index for a statistics item, the index | 0x80000000 for an
- * update item.  Tensor after tensor emits its statistics items; a tensor's
- * update items follow once at least lead_items further items stand behind its
- * last statistics item.  Writes up to cap items and returns the number of items
- * (2 x tensor_first[n]; negative on bad arguments). */
-int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_items,
-                                int32_t *out, int64_t cap);
+ * (n + 1 values, non-decreasing, tensor_first[0] = 0).  An item is a run of
+ * consecutive entries of one tensor: the tensor's first entry alone, the others
+ * in runs of `group` (1..8).  out[k] is the k-th item's first chunk-table index
+ * (| 0x80000000 for an update item, plain for a statistics item), count[k] its
+ * number of entries (either array may be NULL).  Tensor after tensor emits its
+ * statistics items; a tensor's update items follow once items of at least
+ * lead_entries further entries stand behind its last statistics item.  Writes
+ * up to cap items and returns the number of items (negative on bad arguments). */
+int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_entries, int group,
+                                int32_t *out, int32_t *count, int64_t cap);
 
 /* Text of the last error on this handle ("" if none).  Owned by the handle. */
 const char *novak_last_error(const novak_opt *opt);

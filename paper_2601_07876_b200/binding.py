@@ -31,7 +31,7 @@ NOVAK_LOOKAHEAD_LAST, NOVAK_LOOKAHEAD_TRAJ_MEAN = 0, 1
  NOVAK_OPT_BETA2_TAU, NOVAK_OPT_LAYER_ADAPTATION, NOVAK_OPT_SPARSE_THRESHOLD, NOVAK_OPT_AUTO_LR,
  NOVAK_OPT_AUTO_LR_GAMMA, NOVAK_OPT_TRUE_NESTEROV_STEPS, NOVAK_OPT_MOMENT_DTYPE,
  NOVAK_OPT_GRAPH_CAPTURABLE, NOVAK_OPT_CENTRALIZE_IN_STEP, NOVAK_OPT_LAYER_ADAPTATION_IN_STEP,
- NOVAK_OPT_LAYER_ADAPTATION_LEAD) = range(1, 27)
+ NOVAK_OPT_LAYER_ADAPTATION_LEAD, NOVAK_OPT_LAYER_ADAPTATION_GROUP) = range(1, 28)
 NOVAK_MOMENT_F32, NOVAK_MOMENT_BF16 = 0, 1
 NOVAK_WARN_TRUE_DOWNGRADED, NOVAK_WARN_SCALAR_PATH, NOVAK_WARN_NARROW_GRADIENT = 1, 2, 4
 
@@ -134,8 +134,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
         "novak_build_chunks": (c_int64, [i64p, POINTER(c_int32), c_int, c_int64,
                                          POINTER(c_int32), i64p, POINTER(c_int32), c_int64]),
         "novak_build_own_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, c_int64]),
-        "novak_build_adapt_order": (c_int64, [POINTER(c_int32), c_int, c_int64, POINTER(c_int32),
-                                              c_int64]),
+        "novak_build_adapt_order": (c_int64, [POINTER(c_int32), c_int, c_int64, c_int,
+                                              POINTER(c_int32), POINTER(c_int32), c_int64]),
         "novak_build_row_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, i64p,
                                             i64p, c_int64]),
         "novak_last_error": (c_char_p, [vp]),
@@ -215,18 +215,19 @@ def novak_build_own_units(numel, rows, lib=None):
     return list(zip(list(t), *[list(c) for c in cols]))
 
 
-def novak_build_adapt_order(tensor_first, lead_items, lib=None):
+def novak_build_adapt_order(tensor_first, lead_entries, group=1, lib=None):
     """Host-only: the item order of the one-launch layer adaptation, as a list of
-    (chunk index, is_update)."""
+    (first chunk index, number of entries, is_update)."""
     lib = lib or load_library()
     n = len(tensor_first) - 1
     first = (c_int32 * (n + 1))(*tensor_first)
-    need = lib.novak_build_adapt_order(first, n, lead_items, None, 0)
+    need = lib.novak_build_adapt_order(first, n, lead_entries, group, None, None, 0)
     if need < 0:
         raise NovakError(NOVAK_EINVAL, "novak_build_adapt_order")
     out = (c_int32 * need)()
-    lib.novak_build_adapt_order(first, n, lead_items, out, need)
-    return [(v & 0x7fffffff, v < 0) for v in out]
+    cnt = (c_int32 * need)()
+    lib.novak_build_adapt_order(first, n, lead_entries, group, out, cnt, need)
+    return [(v & 0x7fffffff, k, v < 0) for v, k in zip(out, cnt)]
 
 
 _NESTEROV = {"none": NOVAK_NESTEROV_NONE, "approximation": NOVAK_NESTEROV_APPROX,
@@ -438,7 +439,7 @@ class NovakOptimizer:
                  layer_adaptation=False, sparse_threshold=0.0, param_copies=None,
                  auto_lr=False, auto_lr_gamma=None, true_nesterov_steps=0, moment_dtype="f32",
                  graph_capturable=False, centralize_in_step=None, layer_adaptation_in_step=None,
-                 layer_adaptation_lead=None,
+                 layer_adaptation_lead=None, layer_adaptation_group=None,
                  chunk_elems=None, ctas_per_sm=None, serpentine=None, dependent_launch=None,
                  lib=None):
         import torch
@@ -470,6 +471,8 @@ class NovakOptimizer:
             h.set_option(NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 1 if layer_adaptation_in_step else 0)
         if layer_adaptation_lead is not None:
             h.set_option(NOVAK_OPT_LAYER_ADAPTATION_LEAD, layer_adaptation_lead)
+        if layer_adaptation_group is not None:
+            h.set_option(NOVAK_OPT_LAYER_ADAPTATION_GROUP, layer_adaptation_group)
         if centralize_in_step is not None:
             h.set_option(NOVAK_OPT_CENTRALIZE_IN_STEP, 1 if centralize_in_step else 0)
         if chunk_elems is not None:

@@ -129,7 +129,8 @@ struct Handle {
     // layer adaptation and step in one launch: the claim-ordered item list, the
     // kernel's counters and per-tensor flags (one allocation), a host-mapped error word
     int adapt_in_step = 0;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
-    int64_t adapt_lead_elems = 1 << 21;    // NOVAK_OPT_LAYER_ADAPTATION_LEAD
+    int64_t adapt_lead_elems = 1 << 22;    // NOVAK_OPT_LAYER_ADAPTATION_LEAD
+    int adapt_group = 4;                   // NOVAK_OPT_LAYER_ADAPTATION_GROUP
     char *d_adapt = nullptr;
     int *d_item_code = nullptr;
     Chunk *d_item_chunk = nullptr;
@@ -140,6 +141,8 @@ struct Handle {
     unsigned *h_adapt_error = nullptr;  // pinned, mapped; written by the kernel
     unsigned *d_adapt_error = nullptr;  // its device address
     unsigned adapt_epoch = 0;
+    float *adapt_direction = nullptr;   // one slot of adapt_slot_elems floats per chunk-table entry
+    int adapt_slot_elems = 0;
 
     // novak_step_host: the chunk table cut into segments, each with the element
     // ranges it covers, two copy streams and the events that order them.
@@ -230,12 +233,15 @@ void invalidate_tables(novak_opt *o);
 int prepare_trust(novak_opt *o, cudaStream_t stream);
 // The item list and counters of the one-launch form of layer adaptation.
 int prepare_adapt(novak_opt *o, cudaStream_t stream);
-// Claim order of that kernel.  Tensor after tensor emits its S items (chunk-
-// table index); a tensor's U items (index | 0x80000000) follow once at least
-// `lead_items` further items have been emitted behind its last S item, tensors
-// in order; what is still pending at the end follows in order.
-void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_items,
-                       std::vector<int32_t> &items);
+// Item order of that kernel.  An item is a run of consecutive chunk-table entries
+// of one tensor: the tensor's first entry alone, the others in runs of `group`.
+// items[k] is the item's first entry (| 0x80000000 for a U item), counts[k] its
+// number of entries.  Tensor after tensor emits its S items; a tensor's U items
+// follow once items of at least `lead_entries` further entries have been emitted
+// behind its last S item, tensors in order; what is still pending at the end
+// follows in order.
+void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
+                       std::vector<int32_t> &items, std::vector<int32_t> &counts);
 uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype,
                        const void *save);
 // `save`: NULL, or the save buffer of an open look-ahead, from which the step

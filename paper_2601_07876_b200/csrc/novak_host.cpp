@@ -87,25 +87,35 @@ void build_own_units(const int64_t *numel, const int64_t *rows, int n, std::vect
     }
 }
 
-void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_items,
-                       std::vector<int32_t> &items)
+void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
+                       std::vector<int32_t> &items, std::vector<int32_t> &counts)
 {
     items.clear();
+    counts.clear();
     if (n <= 0) return;
-    items.reserve(2 * static_cast<size_t>(tensor_first[n]));
     const int32_t kUpdate = static_cast<int32_t>(0x80000000u);
-    std::vector<int64_t> s_end(n, 0);   // items emitted when tensor i's last S item was
+    std::vector<int64_t> s_end(n, 0);   // entries emitted when tensor i's last S item was
+    int64_t emitted = 0;                // entries of all items so far, both kinds
     int pending = 0;                    // first tensor whose U items are still to come
-    auto emit_updates = [&](int i) {
-        for (int c = tensor_first[i]; c < tensor_first[i + 1]; ++c) items.push_back(c | kUpdate);
+    // A tensor's first entry (the only one besides its last that may be short) stands
+    // alone; the others go in runs of `group`.
+    auto emit = [&](int i, int32_t flag) {
+        int c = tensor_first[i];
+        const int c1 = tensor_first[i + 1];
+        while (c < c1) {
+            const int cnt = (c == tensor_first[i]) ? 1 : std::min(group, c1 - c);
+            items.push_back(c | flag);
+            counts.push_back(cnt);
+            emitted += cnt;
+            c += cnt;
+        }
     };
     for (int i = 0; i < n; ++i) {
-        for (int c = tensor_first[i]; c < tensor_first[i + 1]; ++c) items.push_back(c);
-        s_end[i] = static_cast<int64_t>(items.size());
-        while (pending <= i && static_cast<int64_t>(items.size()) - s_end[pending] >= lead_items)
-            emit_updates(pending++);
+        emit(i, 0);
+        s_end[i] = emitted;
+        while (pending <= i && emitted - s_end[pending] >= lead_entries) emit(pending++, kUpdate);
     }
-    while (pending < n) emit_updates(pending++);
+    while (pending < n) emit(pending++, kUpdate);
 }
 
 int fail(novak_opt *o, int code, const char *fmt, ...)
@@ -348,6 +358,12 @@ int novak_set_option(novak_opt *o, int key, double value)
             return fail(o, NOVAK_EINVAL, "layer_adaptation_lead must be an integer in [0, 2^30]");
         o->adapt_lead_elems = static_cast<int64_t>(value);
         return NOVAK_OK;
+    case NOVAK_OPT_LAYER_ADAPTATION_GROUP:
+        if (o->d_adapt) return fail(o, NOVAK_ESTATE, "the group is fixed once a step with layer adaptation was taken");
+        if (!(value >= 1.0 && value <= double(novak::kAdaptGroupMax)) || value != std::floor(value))
+            return fail(o, NOVAK_EINVAL, "layer_adaptation_group must be an integer in [1, %d]", novak::kAdaptGroupMax);
+        o->adapt_group = static_cast<int>(value);
+        return NOVAK_OK;
     case NOVAK_OPT_CENTRALIZE_IN_STEP:
         if (value != 0.0 && value != 1.0) return fail(o, NOVAK_EINVAL, "centralize_in_step must be 0 or 1");
         o->center_in_step = static_cast<int>(value);
@@ -419,6 +435,7 @@ int novak_get_option(const novak_opt *o, int key, double *value)
     case NOVAK_OPT_CENTRALIZE_IN_STEP: *value = o->center_in_step; break;
     case NOVAK_OPT_LAYER_ADAPTATION_IN_STEP: *value = o->adapt_in_step; break;
     case NOVAK_OPT_LAYER_ADAPTATION_LEAD: *value = static_cast<double>(o->adapt_lead_elems); break;
+    case NOVAK_OPT_LAYER_ADAPTATION_GROUP: *value = o->adapt_group; break;
     case NOVAK_OPT_CHUNK_ELEMS: *value = static_cast<double>(o->chunk_elems); break;
     case NOVAK_OPT_CTAS_PER_SM: *value = o->ctas_per_sm; break;
     case NOVAK_OPT_SERPENTINE: *value = o->serpentine; break;
@@ -719,19 +736,23 @@ int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, 
     return count;
 }
 
-int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_items,
-                                int32_t *out, int64_t cap)
+int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_entries, int group,
+                                int32_t *out, int32_t *count, int64_t cap)
 {
-    if (!tensor_first || n <= 0 || lead_items < 0 || cap < 0 || tensor_first[0] != 0) return -1;
+    if (!tensor_first || n <= 0 || lead_entries < 0 || cap < 0 || tensor_first[0] != 0 ||
+        group < 1 || group > novak::kAdaptGroupMax)
+        return -1;
     for (int i = 0; i < n; ++i)
         if (tensor_first[i + 1] < tensor_first[i]) return -1;
     std::vector<int> first(tensor_first, tensor_first + n + 1);
-    std::vector<int32_t> items;
-    build_adapt_items(first, n, lead_items, items);
-    const int64_t count = static_cast<int64_t>(items.size());
-    for (int64_t i = 0; i < count && i < cap; ++i)
+    std::vector<int32_t> items, counts;
+    build_adapt_items(first, n, lead_entries, group, items, counts);
+    const int64_t total = static_cast<int64_t>(items.size());
+    for (int64_t i = 0; i < total && i < cap; ++i) {
         if (out) out[i] = items[i];
-    return count;
+        if (count) count[i] = counts[i];
+    }
+    return total;
 }
 
 int64_t novak_build_chunks(const int64_t *numel, const int32_t *phase, int n,

@@ -36,6 +36,8 @@ void release_device(novak_opt *o)
     o->look_save = nullptr;
     o->extrapolated = false;
     if (o->d_adapt) cudaFree(o->d_adapt);
+    if (o->adapt_direction) cudaFree(o->adapt_direction);
+    o->adapt_direction = nullptr;
     if (o->h_adapt_error) cudaFreeHost(o->h_adapt_error);
     o->d_adapt = nullptr;
     o->d_item_code = nullptr;
@@ -278,12 +280,22 @@ int prepare_trust(novak_opt *o, cudaStream_t stream)
 int prepare_adapt(novak_opt *o, cudaStream_t stream)
 {
     if (o->d_adapt) return NOVAK_OK;
-    std::vector<int32_t> codes;
-    const int64_t lead_items = (o->adapt_lead_elems + o->chunk_elems - 1) / o->chunk_elems;
-    build_adapt_items(o->h_tensor_first, o->n, lead_items, codes);
+    std::vector<int32_t> codes, counts;
+    const int64_t lead_entries = (o->adapt_lead_elems + o->chunk_elems - 1) / o->chunk_elems;
+    build_adapt_items(o->h_tensor_first, o->n, lead_entries, o->adapt_group, codes, counts);
     if (codes.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
+    // an item's entries as one span: consecutive in their tensor, all but the last full
     std::vector<Chunk> entries(codes.size());
-    for (size_t k = 0; k < codes.size(); ++k) entries[k] = o->h_chunks[codes[k] & 0x7fffffff];
+    for (size_t k = 0; k < codes.size(); ++k) {
+        const int c = codes[k] & 0x7fffffff;
+        Chunk span = o->h_chunks[c];
+        for (int j = 1; j < counts[k]; ++j) {
+            if (o->h_chunks[c + j - 1].len != o->chunk_elems || o->h_chunks[c + j].tensor != span.tensor)
+                return fail(o, NOVAK_EINVAL, "layer adaptation items: a short entry inside a tensor");
+            span.len += o->h_chunks[c + j].len;
+        }
+        entries[k] = span;
+    }
     const size_t n = static_cast<size_t>(o->n);
     const size_t off_ready = 256;
     const size_t off_arrived = off_ready + n * sizeof(unsigned long long);
@@ -305,6 +317,17 @@ int prepare_adapt(novak_opt *o, cudaStream_t stream)
     if ((e = cudaMalloc(reinterpret_cast<void **>(&o->d_adapt), bytes)) != cudaSuccess) {
         o->d_adapt = nullptr;
         return fail(o, NOVAK_ENOMEM, "cudaMalloc(layer adaptation items, %zu B): %s", bytes, cudaGetErrorString(e));
+    }
+    // the directions of one step, 4 B per element of the group: written by the S items,
+    // read by the U items a few MB of traffic later
+    o->adapt_slot_elems = static_cast<int>((o->chunk_elems + 3) / 4 * 4);
+    const size_t dir_bytes = static_cast<size_t>(o->n_chunks) * o->adapt_slot_elems * sizeof(float);
+    if ((e = cudaMalloc(reinterpret_cast<void **>(&o->adapt_direction), dir_bytes)) != cudaSuccess) {
+        o->adapt_direction = nullptr;
+        cudaFree(o->d_adapt);
+        o->d_adapt = nullptr;
+        return fail(o, NOVAK_ENOMEM, "cudaMalloc(layer adaptation directions, %zu B): %s", dir_bytes,
+                    cudaGetErrorString(e));
     }
     o->adapt_ctl = reinterpret_cast<novak::AdaptCtl *>(o->d_adapt);
     o->adapt_arrived = reinterpret_cast<unsigned *>(o->d_adapt + off_arrived);

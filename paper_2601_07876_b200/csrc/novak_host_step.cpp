@@ -201,7 +201,7 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
         const cudaError_t e = novak::launch_step_adapt(
             o->d_item_code, o->d_item_chunk, o->n_items, ctx.d_recs,
             o->tensor_first, o->chunk_u2, o->chunk_p2, o->trust, o->adapt_ctl, o->adapt_arrived,
-            o->adapt_ready, o->d_adapt_error, ctx.s, epoch, kernel_variant(ctx.plan), ctx.grad_dtype,
+            o->adapt_ready, o->d_adapt_error, o->adapt_direction, o->adapt_slot_elems, ctx.s, epoch, kernel_variant(ctx.plan), ctx.grad_dtype,
             ctx.la, cfg, stream);
         if (e == cudaSuccess) o->adapt_epoch = epoch;
         return e;

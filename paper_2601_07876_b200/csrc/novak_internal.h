@@ -45,24 +45,31 @@ cudaError_t launch_trust_stats(const Chunk *d_chunks, int n_chunks, const Tensor
 
 // ---- layer adaptation and step in one launch (novak_step_adapt.cuh) ---------
 // State of the kernel in device memory, zero before the first launch.
+constexpr int kAdaptGroupMax = 8;      // chunk-table entries per item at most
 struct __align__(16) AdaptCtl {
     unsigned error;       // a bounded wait gave up (sticky)
     unsigned reserved[3];
 };
 
-// item_code: n_items codes in block order, a chunk-table index for an S item,
-// the index | 0x80000000 for a U item, every entry once as each, a tensor's S
-// items all before any of its U items; item_chunk: the entry itself, item by
-// item.  arrived: one counter per tensor; ready: one 64-bit word per tensor
+// An item is up to kAdaptGroupMax consecutive chunk-table entries of one tensor,
+// all but the last slot_elems long.  item_code: n_items codes in block order,
+// the item's first chunk-table index for an S item, the index | 0x80000000 for
+// a U item, every entry in one item of each kind, a tensor's S items all before
+// any of its U items; item_chunk: the item's entries as one span (tensor,
+// offset of the first, total length).  arrived: one counter per tensor; ready: one 64-bit word per tensor
 // (launch number in the high half, the ratio's bits in the low half); both
 // zero before the first launch.  epoch: a launch number no earlier launch on
 // these buffers used (never 0).  host_error: device address of a host-mapped
-// word, set to 1 if a wait gives up.  cfg.pre: PRE_NONE with or without
+// word, set to 1 if a wait gives up.  direction: scratch of slot_elems floats
+// per chunk-table entry (entry c at c * slot_elems; slot_elems a multiple of 4
+// and at least the longest entry, the array 16-byte aligned), written and read
+// within the launch.  cfg.pre: PRE_NONE with or without
 // PRE_COPY16 and PRE_MOM16.  The grid is n_items CTAs.
 cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int n_items,
                               const TensorRec *d_recs, const int *tensor_first,
                               double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
                               unsigned *arrived, unsigned long long *ready, unsigned *host_error,
+                              float *direction, int slot_elems,
                               const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
                               int la, const LaunchCfg &cfg, cudaStream_t stream);
 

@@ -95,12 +95,13 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
                               const TensorRec *d_recs, const int *tensor_first,
                               double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
                               unsigned *arrived, unsigned long long *ready, unsigned *host_error,
+                              float *direction, int slot_elems,
                               const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
                               int la, const LaunchCfg &cfg, cudaStream_t stream)
 {
     using Fn = void (*)(const int *, const Chunk *, int, const TensorRec *, const int *, double *,
                         double *, float *, AdaptCtl *, unsigned *, unsigned long long *, unsigned *,
-                        StepScalars, unsigned);
+                        float *, int, StepScalars, unsigned);
     void *raw = nullptr;
     switch (cfg.pre) {
 #define NOVAK_CASE(N) case N: raw = step_adapt_kernel_mode##N(nesterov, grad_dtype, la); break;
@@ -110,7 +111,8 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
     }
     Fn fn = reinterpret_cast<Fn>(raw);
     if (!fn || !item_code || !item_chunk || n_items <= 0 || epoch == 0u || !ctl || !arrived || !ready ||
-        !host_error || !tensor_first || !chunk_u2 || !chunk_p2 || !trust)
+        !host_error || !tensor_first || !chunk_u2 || !chunk_p2 || !trust || !direction ||
+        slot_elems <= 0 || (slot_elems & 3) != 0)
         return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(static_cast<unsigned>(n_items));
@@ -123,7 +125,8 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
     lc.attrs = attr;
     lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
     return cudaLaunchKernelEx(&lc, fn, item_code, item_chunk, n_items, d_recs, tensor_first,
-                              chunk_u2, chunk_p2, trust, ctl, arrived, ready, host_error, s, epoch);
+                              chunk_u2, chunk_p2, trust, ctl, arrived, ready, host_error, direction,
+                              slot_elems, s, epoch);
 }
 
 cudaError_t step_occupancy(int nesterov, int grad_dtype, int la, int pre, int *ctas_per_sm)

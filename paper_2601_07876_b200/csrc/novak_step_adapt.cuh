@@ -85,6 +85,193 @@ __device__ __forceinline__ unsigned long long wait_for_ratio(const unsigned long
     return 0ull;
 }
 
+// ---- the direction a step applies, formed once -------------------------------
+// An S item advances the moments for good and leaves, element by element, the
+// direction the update multiplies by the step (Eq. 17 after the mask of Eq. 27
+// and the blend of Eq. 16) in a scratch array; the U item reads it back from L2.
+// The operations and their order are those of update_element(), cut in two
+// after the direction: results are bit-identical to the two-pass route.
+
+// Phases 2, 4, 5, 8 for U vectors of N elements per thread (vectors beyond nvec
+// are skipped): every load issued before the first use; moments advanced and
+// stored, direction stored, the squares of theta and of the base direction
+// added up vector by vector in index order.
+template <int N, int U, int NEST, int GT, int PRE>
+__device__ __forceinline__ void direction_tile(const float *p, const void *g, void *m, void *v,
+                                               float *d, int first, int nvec, const StepScalars &s,
+                                               double &sum_p, double &sum_u)
+{
+    constexpr bool kMom16 = (PRE & PRE_MOM16) != 0;
+    Vec<N> P[U], G[U], M[U], V[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+        if (idx < nvec) {
+            P[j] = load_f32<N, LD_KEEP>(p, idx);        // the U item reads theta again
+            G[j] = load_grad<N, GT>(g, idx);
+            M[j] = load_moment<N, kMom16>(m, idx);
+            V[j] = load_moment<N, kMom16>(v, idx);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+        if (idx < nvec) {
+            Vec<N> D;
+            float sp = 0.0f, su = 0.0f;
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                float m_hat;
+                float u = base_direction<NEST>(G[j].a[e], M[j].a[e], V[j].a[e], m_hat, s);
+                sp = fmaf(P[j].a[e], P[j].a[e], sp);
+                su = fmaf(u, u, su);                            // Eq. 19: the unmasked base direction
+                u = (fabsf(u) <= s.sparse_tau) ? 0.0f : u;      // Eq. 27
+                if constexpr (NEST == NOVAK_NESTEROV_CLASSICAL)
+                    u = fmaf(s.blend_b1, m_hat, s.blend_omb1 * u);      // Eq. 16
+                D.a[e] = u;
+            }
+            sum_p += double(sp);
+            sum_u += double(su);
+            store_moment<N, kMom16>(m, idx, M[j]);
+            store_moment<N, kMom16>(v, idx, V[j]);
+            // default policy: the line stays in L2 for the U item
+            if constexpr (N == 4)
+                reinterpret_cast<float4 *>(d)[idx] = make_float4(D.a[0], D.a[1], D.a[2], D.a[3]);
+            else
+                d[idx] = D.a[0];
+        }
+    }
+}
+
+// One chunk-table entry of an S item; every thread returns its share of the
+// two sums (the vectors it took, in index order).
+template <int NEST, int GT, int PRE>
+__device__ __forceinline__ void entry_direction(const Chunk &ch, const TensorRec &r, float *d,
+                                                const StepScalars &s, double &sum_p, double &sum_u)
+{
+    constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
+    constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
+    const float *p = r.p_in + ch.offset;     // theta_{t-1}
+    void *m = static_cast<char *>(r.m) + ch.offset * kMomBytes;
+    void *v = static_cast<char *>(r.v) + ch.offset * kMomBytes;
+    const void *g = static_cast<const char *>(r.g) + ch.offset * kGradBytes;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(p) |
+                           ((reinterpret_cast<uintptr_t>(m) | reinterpret_cast<uintptr_t>(v))
+                            << (kMomBytes == 2 ? 1 : 0));
+    const bool aligned = (bits & 15u) == 0 &&
+                         (reinterpret_cast<uintptr_t>(g) & (4u * kGradBytes - 1u)) == 0;
+    sum_p = 0.0;
+    sum_u = 0.0;
+    if (aligned) {
+        const int nvec = ch.len >> 2;
+#pragma unroll 1
+        for (int base = 0; base < nvec; base += kBlock * 2)
+            direction_tile<4, 2, NEST, GT, PRE>(p, g, m, v, d, base + threadIdx.x, nvec, s, sum_p, sum_u);
+        // ragged tail: < 4 elements
+        direction_tile<1, 1, NEST, GT, PRE>(p, g, m, v, d, (nvec << 2) + threadIdx.x, ch.len, s,
+                                            sum_p, sum_u);
+    } else {
+#pragma unroll 1
+        for (int base = 0; base < ch.len; base += kBlock * 4)
+            direction_tile<1, 4, NEST, GT, PRE>(p, g, m, v, d, base + threadIdx.x, ch.len, s,
+                                                sum_p, sum_u);
+    }
+}
+
+// Phases 9 and 10 (Eq. 18, 24, 28-31) for one element from its stored direction.
+template <int LA>
+__device__ __forceinline__ void apply_direction(float &p, float u, float &slow, float &acc,
+                                                const StepScalars &s, float step)
+{
+    const float theta_in = p;
+    const float theta_fast = fmaf(theta_in, s.decay, -(step * u));
+    float out = theta_fast;
+    float sum = theta_fast;
+    if constexpr ((LA & LA_A_READ) != 0)
+        sum = acc + theta_fast;
+    if constexpr ((LA & LA_A_WRITE) != 0)
+        acc = sum;
+    if constexpr ((LA & LA_SYNC) != 0) {
+        const float slow_in = (LA & LA_S_INIT) ? theta_in : slow;
+        const float target = (LA & LA_TRAJ) ? __fdiv_rn(sum, s.k) : theta_fast;
+        out = fmaf(s.la_alpha, target - slow_in, slow_in);
+        slow = out;
+    } else if constexpr ((LA & LA_S_INIT) != 0) {
+        slow = theta_in;
+    }
+    p = out;
+}
+
+// U vectors of N elements per thread, every load issued before the first use.
+// The direction was written by another CTA of this grid: L2 loads.
+template <int N, int U, int LA, int PRE>
+__device__ __forceinline__ void apply_tile(float *p, const float *pin, const float *d, float *slow,
+                                           float *acc, __nv_bfloat16 *copy, int first, int nvec,
+                                           const StepScalars &s, float step)
+{
+    constexpr bool kReadS = (LA & LA_S_READ) != 0;
+    constexpr bool kWriteS = (LA & LA_S_WRITE) != 0;
+    constexpr bool kReadA = (LA & LA_A_READ) != 0;
+    constexpr bool kWriteA = (LA & LA_A_WRITE) != 0;
+    Vec<N> P[U], D[U], S[U], A[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+        if (idx < nvec) {
+            P[j] = load_f32<N>(pin, idx);
+            D[j] = load_f32<N, LD_KEEP>(d, idx);
+            if constexpr (kReadS) S[j] = load_f32<N>(slow, idx);
+            if constexpr (kReadA) A[j] = load_f32<N>(acc, idx);
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+        const int idx = first + j * kBlock;
+        if (idx < nvec) {
+#pragma unroll
+            for (int e = 0; e < N; ++e)
+                apply_direction<LA>(P[j].a[e], D[j].a[e], S[j].a[e], A[j].a[e], s, step);
+            store_f32<N>(p, idx, P[j]);
+            if constexpr ((PRE & PRE_COPY16) != 0) store_bf16<N>(copy, idx, P[j]);
+            if constexpr (kWriteS) store_f32<N>(slow, idx, S[j]);
+            if constexpr (kWriteA) store_f32<N>(acc, idx, A[j]);
+        }
+    }
+}
+
+// A U item: its entries are consecutive in their tensor and in the direction
+// scratch (every entry but a tensor's first and last is slot_elems long), one span.
+template <int LA, int PRE>
+__device__ __forceinline__ void entry_apply(const Chunk &ch, const TensorRec &r, const float *d,
+                                            const StepScalars &s, float step)
+{
+    constexpr bool kUseS = (LA & (LA_S_READ | LA_S_WRITE)) != 0;
+    constexpr bool kUseA = (LA & (LA_A_READ | LA_A_WRITE)) != 0;
+    // an item is a few entries long: four vectors per thread where the registers allow
+    constexpr int kU = (LA & (LA_S_READ | LA_A_READ)) != 0 ? 2 : 4;
+    float *p = r.p + ch.offset;
+    const float *pin = r.p_in + ch.offset;
+    float *slow = kUseS ? r.slow + ch.offset : nullptr;
+    float *acc = kUseA ? r.acc + ch.offset : nullptr;
+    __nv_bfloat16 *copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
+    uintptr_t bits = reinterpret_cast<uintptr_t>(p) | reinterpret_cast<uintptr_t>(pin);
+    if (kUseS) bits |= reinterpret_cast<uintptr_t>(slow);
+    if (kUseA) bits |= reinterpret_cast<uintptr_t>(acc);
+    if ((PRE & PRE_COPY16) != 0) bits |= reinterpret_cast<uintptr_t>(copy) << 1;
+    if ((bits & 15u) == 0) {
+        const int nvec = ch.len >> 2;
+#pragma unroll 1
+        for (int base = 0; base < nvec; base += kBlock * kU)
+            apply_tile<4, kU, LA, PRE>(p, pin, d, slow, acc, copy, base + threadIdx.x, nvec, s, step);
+        // ragged tail of a tensor: at most 3 elements
+        apply_tile<1, 1, LA, PRE>(p, pin, d, slow, acc, copy, (nvec << 2) + threadIdx.x, ch.len, s, step);
+    } else {
+#pragma unroll 1
+        for (int base = 0; base < ch.len; base += kBlock * 4)
+            apply_tile<1, 4, LA, PRE>(p, pin, d, slow, acc, copy, base + threadIdx.x, ch.len, s, step);
+    }
+}
+
 // Resident CTAs per SM as for the plain step kernel's instantiation of the same
 // lookahead action (three for every action measured 0.233 against 0.220 ms per
 // step on the ResNet-50-shaped set).
@@ -97,13 +284,12 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
                         int n_items, const TensorRec *__restrict__ recs,
                         const int *__restrict__ tensor_first, double *chunk_u2, double *chunk_p2,
                         float *trust, AdaptCtl *ctl, unsigned *arrived, unsigned long long *ready,
-                        unsigned *host_error, const StepScalars s, unsigned epoch)
+                        unsigned *host_error, float *direction, int slot_elems,
+                        const StepScalars s, unsigned epoch)
 {
     static_assert((PRE & PRE_MASK) == PRE_NONE, "gradient pre-processing keeps the two-pass route");
-    // the classical blend (Eq. 16) comes after the base direction
-    constexpr int kStatNest = (NEST == NOVAK_NESTEROV_APPROX) ? NOVAK_NESTEROV_APPROX
-                                                              : NOVAK_NESTEROV_NONE;
     __shared__ double sh[kTrustWarps];
+    __shared__ double sh_part[kAdaptGroupMax][2][kTrustWarps];
     __shared__ int sh_flag;
 
     grid_dependency_release();
@@ -112,35 +298,58 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
     // The item tables and the records are written by copies only, never by a
     // kernel: read before the previous kernel on the stream has finished.
     const int code = item_code[it];
-    const Chunk ch = item_chunk[it];
-    const int c = code & 0x7fffffff;                    // the entry's index in the chunk table
+    const Chunk ch = item_chunk[it];                    // the item's entries as one span
+    const int c = code & 0x7fffffff;                    // its first entry's index in the chunk table
     const TensorRec r = recs[ch.tensor];
     grid_dependency_wait();
 
-    PreArgs pre;
-    pre.factor = 1.0f;
-    pre.mean = nullptr;
-    pre.row_len = 0u;
-    pre.elem0 = static_cast<uint32_t>(ch.offset);
+    // entry c + j of the item keeps element e at d[j * slot_elems + e]
+    float *d = direction + static_cast<size_t>(c) * static_cast<size_t>(slot_elems);
 
     if (code >= 0) {
-        // ---- S item: this entry's two sums of squares
+        // ---- S item: moments, direction and the two sums of squares of each entry
         const int c0 = tensor_first[ch.tensor], c1 = tensor_first[ch.tensor + 1];
-        pre.step = 0.0f;
-        pre.copy = nullptr;
-        double tp, tu;
-        entry_trust_sums<kStatNest, GT, PRE, LD_KEEP>(ch, r, s, pre, sh, tp, tu);
+        const int cnt = (ch.len + slot_elems - 1) / slot_elems;        // <= kAdaptGroupMax
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll 1
+        for (int j = 0; j < cnt; ++j) {
+            Chunk sub;
+            sub.tensor = ch.tensor;
+            sub.offset = ch.offset + static_cast<int64_t>(j) * slot_elems;
+            sub.len = min(slot_elems, ch.len - j * slot_elems);
+            double sp, su;
+            entry_direction<NEST, GT, PRE>(sub, r, d + static_cast<size_t>(j) * slot_elems, s, sp, su);
+            sp = trust_warp_sum(sp);
+            su = trust_warp_sum(su);
+            if (lane == 0) {
+                sh_part[j][0][warp] = sp;
+                sh_part[j][1][warp] = su;
+            }
+        }
+        __syncthreads();
+        if (static_cast<int>(threadIdx.x) < cnt) {
+            // warps in index order, as the two-pass route adds them
+            double tp = 0.0, tu = 0.0;
+#pragma unroll
+            for (int w = 0; w < kTrustWarps; ++w) {
+                tp += sh_part[threadIdx.x][0][w];
+                tu += sh_part[threadIdx.x][1][w];
+            }
+            chunk_p2[c + threadIdx.x] = tp;
+            chunk_u2[c + threadIdx.x] = tu;
+        }
+        __syncthreads();
         if (threadIdx.x == 0) {
-            chunk_p2[c] = tp;
-            chunk_u2[c] = tu;
-            __threadfence();                 // the sums before the arrival
-            const unsigned last = static_cast<unsigned>(c1 - c0) - 1u;
-            // wraps to 0 with the tensor's last entry, ready for the next launch
-            sh_flag = atomicInc(&arrived[ch.tensor], last) == last ? 1 : 0;
+            __threadfence();                 // the CTA's sums and directions before the arrival
+            const unsigned total = static_cast<unsigned>(c1 - c0);
+            const unsigned before = atomicAdd(&arrived[ch.tensor], static_cast<unsigned>(cnt));
+            sh_flag = (before + static_cast<unsigned>(cnt) == total) ? 1 : 0;
+            // the tensor's last item leaves the counter at 0 for the next launch
+            if (sh_flag) atomicExch(&arrived[ch.tensor], 0u);
         }
         __syncthreads();
         if (sh_flag == 0) return;
-        // the tensor's last entry: every sum is there
+        // the tensor's last item: every sum is there
         __threadfence();
         const float eta = tensor_trust_ratio(chunk_p2, chunk_u2, c0, c1, sh);
         if (threadIdx.x == 0) {
@@ -160,11 +369,11 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
             *reinterpret_cast<volatile unsigned *>(host_error) = 1u;
         }
     }
+    __syncwarp();                        // lane 0's acquire orders the whole warp's loads below
     word = __shfl_sync(0xffffffffu, word, 0);
     if (word == 0ull) return;            // (the update below has no CTA-wide barrier)
-    pre.step = s.step * __uint_as_float(static_cast<unsigned>(word));      // Eq. 24a
-    pre.copy = ((PRE & PRE_COPY16) != 0) ? r.p16 + ch.offset : nullptr;
-    run_entry<NEST, GT, LA, PRE>(ch, r, s, pre);
+    const float step = s.step * __uint_as_float(static_cast<unsigned>(word));      // Eq. 24a
+    entry_apply<LA, PRE>(ch, r, d, s, step);
 }
 
 template <int NEST, int GT, int PRE>

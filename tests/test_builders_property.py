@@ -91,32 +91,45 @@ def test_own_units_cover_the_rows_of_owned_tensors_once(data):
 
 
 @settings(max_examples=80, deadline=None)
-@given(counts=st.lists(st.integers(1, 40), min_size=1, max_size=30), lead=st.integers(0, 120))
-def test_adapt_order_puts_statistics_first_and_keeps_the_lead(counts, lead):
-    """Item order of the one-launch layer adaptation: every chunk-table entry once as a
-    statistics item and once as an update item; all statistics items of a tensor before
-    any of its update items (what the kernel's freedom from deadlock rests on); tensors in
-    order within each kind; at least `lead` items between a tensor's last statistics item
-    and its first update item, except for what is flushed at the end."""
+@given(counts=st.lists(st.integers(1, 40), min_size=1, max_size=30), lead=st.integers(0, 120),
+       group=st.integers(1, 8))
+def test_adapt_order_puts_statistics_first_and_keeps_the_lead(counts, lead, group):
+    """Item order of the one-launch layer adaptation: every chunk-table entry in exactly one
+    statistics item and one update item; an item is a run of at most `group` entries of one
+    tensor, the tensor's first entry (the only one but its last that may be short) alone;
+    all statistics items of a tensor before any of its update items (what the kernel's
+    freedom from deadlock rests on); tensors in order within each kind; items of at least
+    `lead` entries between a tensor's last statistics item and its first update item,
+    except for what is flushed at the end."""
     first = np.concatenate([[0], np.cumsum(counts)]).tolist()
-    order = B.novak_build_adapt_order(first, lead)
+    order = B.novak_build_adapt_order(first, lead, group)
     total = first[-1]
-    assert len(order) == 2 * total
     tensor_of = np.repeat(np.arange(len(counts)), counts)
-    stats = [c for c, upd in order if not upd]
-    upds = [c for c, upd in order if upd]
-    assert stats == list(range(total)) and upds == list(range(total))
-    pos_s = {c: k for k, (c, upd) in enumerate(order) if not upd}
-    pos_u = {c: k for k, (c, upd) in enumerate(order) if upd}
-    last_stats_item = max(pos_s.values())
+    for kind in (False, True):
+        covered = []
+        for c, k, upd in order:
+            if upd != kind:
+                continue
+            assert 1 <= k <= group
+            assert len(set(tensor_of[c:c + k])) == 1            # one tensor
+            if c == first[tensor_of[c]]:
+                assert k == 1                                       # its first entry stands alone
+            covered.extend(range(c, c + k))
+        assert covered == list(range(total))                       # once each, tensors in order
+    # position of every item measured in entries emitted before it
+    before, pos_s, pos_u = 0, {}, {}
+    for c, k, upd in order:
+        for e in range(c, c + k):
+            (pos_u if upd else pos_s)[e] = (before, before + k)
+        before += k
+    last_stats_end = max(end for _, end in pos_s.values())
     for t in range(len(counts)):
         cs = range(first[t], first[t + 1])
-        s_last = max(pos_s[c] for c in cs)
-        u_first = min(pos_u[c] for c in cs)
-        assert s_last < u_first
-        if u_first < last_stats_item:          # not part of the final flush
-            assert u_first - s_last - 1 >= lead
-    assert (np.diff(tensor_of[stats]) >= 0).all()
+        s_end = max(pos_s[c][1] for c in cs)
+        u_start = min(pos_u[c][0] for c in cs)
+        assert s_end <= u_start
+        if u_start < last_stats_end:           # not part of the final flush
+            assert u_start - s_end >= lead
 
 
 @settings(max_examples=60, deadline=None)
