@@ -599,19 +599,19 @@ int64_t novak_build_row_units(const int64_t *numel, const int64_t *rows, int n, 
 int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, int32_t *tensor,
                               int64_t *row0, int64_t *n_rows, int64_t cap);
 
-/* Host-only helper exposing the order in which the one-launch form of layer
- * adaptation (NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) takes its items.  The group's
- * chunk table lists tensor i's entries at [tensor_first[i], tensor_first[i+1])
- * (n + 1 values, non-decreasing, tensor_first[0] = 0).  An item is a run of
- * consecutive entries of one tensor: the tensor's first entry alone, the others
- * in runs of `group` (1..8).  out[k] is the k-th item's first chunk-table index
- * (| 0x80000000 for an update item, plain for a statistics item), count[k] its
- * number of entries (either array may be NULL).  Tensor after tensor emits its
- * statistics items; a tensor's update items follow once items of at least
- * lead_entries further entries stand behind its last statistics item.  Writes
- * up to cap items and returns the number of items (negative on bad arguments). */
+/* Host-only helper exposing the work list of the one-launch form of layer
+ * adaptation (NOVAK_OPT_LAYER_ADAPTATION_IN_STEP).  The group's chunk table lists
+ * tensor i's entries at [tensor_first[i], tensor_first[i+1]) (n + 1 values,
+ * non-decreasing, tensor_first[0] = 0).  An item is a run of consecutive entries
+ * of one tensor: the tensor's first entry alone, the others in runs of `group`
+ * (1..8); items come in tensor order.  out[k] is the k-th item's first chunk-
+ * table index, count[k] its number of entries (either array may be NULL).  CTA b
+ * of the kernel takes the statistics of item b and the update of item b - *lag:
+ * *lag (may be NULL) is the number of items of the tensor that has most, minus
+ * one, plus ceil(lead_entries / group).  Writes up to cap items and returns the
+ * number of items (negative on bad arguments). */
 int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_entries, int group,
-                                int32_t *out, int32_t *count, int64_t cap);
+                                int32_t *out, int32_t *count, int64_t cap, int64_t *lag);
 
 /* Text of the last error on this handle ("" if none).  Owned by the handle. */
 const char *novak_last_error(const novak_opt *opt);

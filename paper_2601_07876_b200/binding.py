@@ -135,7 +135,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
                                          POINTER(c_int32), i64p, POINTER(c_int32), c_int64]),
         "novak_build_own_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, c_int64]),
         "novak_build_adapt_order": (c_int64, [POINTER(c_int32), c_int, c_int64, c_int,
-                                              POINTER(c_int32), POINTER(c_int32), c_int64]),
+                                              POINTER(c_int32), POINTER(c_int32), c_int64, i64p]),
         "novak_build_row_units": (c_int64, [i64p, i64p, c_int, POINTER(c_int32), i64p, i64p, i64p,
                                             i64p, c_int64]),
         "novak_last_error": (c_char_p, [vp]),
@@ -216,18 +216,20 @@ def novak_build_own_units(numel, rows, lib=None):
 
 
 def novak_build_adapt_order(tensor_first, lead_entries, group=1, lib=None):
-    """Host-only: the item order of the one-launch layer adaptation, as a list of
-    (first chunk index, number of entries, is_update)."""
+    """Host-only: the work list of the one-launch layer adaptation, as a list of
+    (first chunk index, number of entries), and the lag between a CTA's statistics
+    item and its update item."""
     lib = lib or load_library()
     n = len(tensor_first) - 1
     first = (c_int32 * (n + 1))(*tensor_first)
-    need = lib.novak_build_adapt_order(first, n, lead_entries, group, None, None, 0)
+    need = lib.novak_build_adapt_order(first, n, lead_entries, group, None, None, 0, None)
     if need < 0:
         raise NovakError(NOVAK_EINVAL, "novak_build_adapt_order")
     out = (c_int32 * need)()
     cnt = (c_int32 * need)()
-    lib.novak_build_adapt_order(first, n, lead_entries, group, out, cnt, need)
-    return [(v & 0x7fffffff, k, v < 0) for v, k in zip(out, cnt)]
+    lag = c_int64(0)
+    lib.novak_build_adapt_order(first, n, lead_entries, group, out, cnt, need, ctypes.byref(lag))
+    return list(zip(out, cnt)), lag.value
 
 
 _NESTEROV = {"none": NOVAK_NESTEROV_NONE, "approximation": NOVAK_NESTEROV_APPROX,

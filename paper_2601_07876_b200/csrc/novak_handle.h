@@ -135,6 +135,7 @@ struct Handle {
     int *d_item_code = nullptr;
     Chunk *d_item_chunk = nullptr;
     int n_items = 0;
+    int adapt_lag = 0;                  // CTA b updates item b - adapt_lag
     novak::AdaptCtl *adapt_ctl = nullptr;
     unsigned *adapt_arrived = nullptr;
     unsigned long long *adapt_ready = nullptr;
@@ -233,15 +234,14 @@ void invalidate_tables(novak_opt *o);
 int prepare_trust(novak_opt *o, cudaStream_t stream);
 // The item list and counters of the one-launch form of layer adaptation.
 int prepare_adapt(novak_opt *o, cudaStream_t stream);
-// Item order of that kernel.  An item is a run of consecutive chunk-table entries
-// of one tensor: the tensor's first entry alone, the others in runs of `group`.
-// items[k] is the item's first entry (| 0x80000000 for a U item), counts[k] its
-// number of entries.  Tensor after tensor emits its S items; a tensor's U items
-// follow once items of at least `lead_entries` further entries have been emitted
-// behind its last S item, tensors in order; what is still pending at the end
-// follows in order.
-void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
-                       std::vector<int32_t> &items, std::vector<int32_t> &counts);
+// Items of that kernel, in tensor order.  An item is a run of consecutive chunk-
+// table entries of one tensor: the tensor's first entry alone, the others in
+// runs of `group`.  items[k] is the item's first entry, counts[k] its number of
+// entries.  Returns the lag: CTA b takes the statistics of item b and the update
+// of item b - lag; the longest tensor's items minus one (so that an update only
+// ever waits for CTAs with a lower index) plus lead_entries / group.
+int64_t build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
+                          std::vector<int32_t> &items, std::vector<int32_t> &counts);
 uint64_t hash_pointers(void *const *d_params, const void *const *d_grads, int n, int grad_dtype,
                        const void *save);
 // `save`: NULL, or the save buffer of an open look-ahead, from which the step

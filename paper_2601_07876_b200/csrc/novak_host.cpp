@@ -87,35 +87,29 @@ void build_own_units(const int64_t *numel, const int64_t *rows, int n, std::vect
     }
 }
 
-void build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
-                       std::vector<int32_t> &items, std::vector<int32_t> &counts)
+int64_t build_adapt_items(const std::vector<int> &tensor_first, int n, int64_t lead_entries, int group,
+                          std::vector<int32_t> &items, std::vector<int32_t> &counts)
 {
     items.clear();
     counts.clear();
-    if (n <= 0) return;
-    const int32_t kUpdate = static_cast<int32_t>(0x80000000u);
-    std::vector<int64_t> s_end(n, 0);   // entries emitted when tensor i's last S item was
-    int64_t emitted = 0;                // entries of all items so far, both kinds
-    int pending = 0;                    // first tensor whose U items are still to come
+    if (n <= 0) return 0;
     // A tensor's first entry (the only one besides its last that may be short) stands
     // alone; the others go in runs of `group`.
-    auto emit = [&](int i, int32_t flag) {
+    int64_t longest = 0;                // items of the tensor that has most
+    for (int i = 0; i < n; ++i) {
+        const size_t before = items.size();
         int c = tensor_first[i];
         const int c1 = tensor_first[i + 1];
         while (c < c1) {
             const int cnt = (c == tensor_first[i]) ? 1 : std::min(group, c1 - c);
-            items.push_back(c | flag);
+            items.push_back(c);
             counts.push_back(cnt);
-            emitted += cnt;
             c += cnt;
         }
-    };
-    for (int i = 0; i < n; ++i) {
-        emit(i, 0);
-        s_end[i] = emitted;
-        while (pending <= i && emitted - s_end[pending] >= lead_entries) emit(pending++, kUpdate);
+        longest = std::max<int64_t>(longest, static_cast<int64_t>(items.size() - before));
     }
-    while (pending < n) emit(pending++, kUpdate);
+    // every S part a U part waits for has a lower block index, or is the CTA's own
+    return std::max<int64_t>(longest - 1, 0) + (lead_entries + group - 1) / group;
 }
 
 int fail(novak_opt *o, int code, const char *fmt, ...)
@@ -737,7 +731,7 @@ int64_t novak_build_own_units(const int64_t *numel, const int64_t *rows, int n, 
 }
 
 int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead_entries, int group,
-                                int32_t *out, int32_t *count, int64_t cap)
+                                int32_t *out, int32_t *count, int64_t cap, int64_t *lag)
 {
     if (!tensor_first || n <= 0 || lead_entries < 0 || cap < 0 || tensor_first[0] != 0 ||
         group < 1 || group > novak::kAdaptGroupMax)
@@ -746,7 +740,8 @@ int64_t novak_build_adapt_order(const int32_t *tensor_first, int n, int64_t lead
         if (tensor_first[i + 1] < tensor_first[i]) return -1;
     std::vector<int> first(tensor_first, tensor_first + n + 1);
     std::vector<int32_t> items, counts;
-    build_adapt_items(first, n, lead_entries, group, items, counts);
+    const int64_t l = build_adapt_items(first, n, lead_entries, group, items, counts);
+    if (lag) *lag = l;
     const int64_t total = static_cast<int64_t>(items.size());
     for (int64_t i = 0; i < total && i < cap; ++i) {
         if (out) out[i] = items[i];

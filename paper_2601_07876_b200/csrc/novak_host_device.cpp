@@ -282,12 +282,13 @@ int prepare_adapt(novak_opt *o, cudaStream_t stream)
     if (o->d_adapt) return NOVAK_OK;
     std::vector<int32_t> codes, counts;
     const int64_t lead_entries = (o->adapt_lead_elems + o->chunk_elems - 1) / o->chunk_elems;
-    build_adapt_items(o->h_tensor_first, o->n, lead_entries, o->adapt_group, codes, counts);
-    if (codes.size() > static_cast<size_t>(INT32_MAX)) return fail(o, NOVAK_EINVAL, "too many chunks");
+    const int64_t lag = build_adapt_items(o->h_tensor_first, o->n, lead_entries, o->adapt_group, codes, counts);
+    if (codes.size() + static_cast<size_t>(lag) > static_cast<size_t>(INT32_MAX))
+        return fail(o, NOVAK_EINVAL, "too many chunks");
     // an item's entries as one span: consecutive in their tensor, all but the last full
     std::vector<Chunk> entries(codes.size());
     for (size_t k = 0; k < codes.size(); ++k) {
-        const int c = codes[k] & 0x7fffffff;
+        const int c = codes[k];
         Chunk span = o->h_chunks[c];
         for (int j = 1; j < counts[k]; ++j) {
             if (o->h_chunks[c + j - 1].len != o->chunk_elems || o->h_chunks[c + j].tensor != span.tensor)
@@ -335,6 +336,7 @@ int prepare_adapt(novak_opt *o, cudaStream_t stream)
     o->d_item_chunk = reinterpret_cast<Chunk *>(o->d_adapt + off_chunk);
     o->d_item_code = reinterpret_cast<int *>(o->d_adapt + off_code);
     o->n_items = static_cast<int>(codes.size());
+    o->adapt_lag = static_cast<int>(lag);
     // built once: blocking copies keep the host vectors' lifetime trivial
     if ((e = cudaMemsetAsync(o->d_adapt, 0, off_chunk, stream)) != cudaSuccess ||
         (e = cudaMemcpyAsync(o->d_item_chunk, entries.data(), entries.size() * sizeof(Chunk),

@@ -195,11 +195,11 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
               (o->h.mom16 ? novak::PRE_MOM16 : 0);
     if (ctx.adapt_in_step) {
         // statistics and update of the whole group as items of one grid
-        cfg.grid = o->n_items;
+        cfg.grid = o->n_items + o->adapt_lag;
         o->last_grid = cfg.grid;
         const unsigned epoch = o->adapt_epoch == 0xffffffffu ? 1u : o->adapt_epoch + 1u;
         const cudaError_t e = novak::launch_step_adapt(
-            o->d_item_code, o->d_item_chunk, o->n_items, ctx.d_recs,
+            o->d_item_code, o->d_item_chunk, o->n_items, o->adapt_lag, ctx.d_recs,
             o->tensor_first, o->chunk_u2, o->chunk_p2, o->trust, o->adapt_ctl, o->adapt_arrived,
             o->adapt_ready, o->d_adapt_error, o->adapt_direction, o->adapt_slot_elems, ctx.s, epoch, kernel_variant(ctx.plan), ctx.grad_dtype,
             ctx.la, cfg, stream);

@@ -52,20 +52,20 @@ struct __align__(16) AdaptCtl {
 };
 
 // An item is up to kAdaptGroupMax consecutive chunk-table entries of one tensor,
-// all but the last slot_elems long.  item_code: n_items codes in block order,
-// the item's first chunk-table index for an S item, the index | 0x80000000 for
-// a U item, every entry in one item of each kind, a tensor's S items all before
-// any of its U items; item_chunk: the item's entries as one span (tensor,
-// offset of the first, total length).  arrived: one counter per tensor; ready: one 64-bit word per tensor
-// (launch number in the high half, the ratio's bits in the low half); both
-// zero before the first launch.  epoch: a launch number no earlier launch on
-// these buffers used (never 0).  host_error: device address of a host-mapped
-// word, set to 1 if a wait gives up.  direction: scratch of slot_elems floats
-// per chunk-table entry (entry c at c * slot_elems; slot_elems a multiple of 4
-// and at least the longest entry, the array 16-byte aligned), written and read
-// within the launch.  cfg.pre: PRE_NONE with or without
-// PRE_COPY16 and PRE_MOM16.  The grid is n_items CTAs.
-cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int n_items,
+// all but the last slot_elems long.  item_first: the n_items items' first chunk-
+// table indices, tensors in order, every entry in one item; item_chunk: the
+// item's entries as one span (tensor, offset of the first, total length).  CTA b
+// takes the statistics of item b and the update of item b - lag; lag is at least
+// the longest tensor's number of items minus one.  arrived: one counter per
+// tensor; ready: one 64-bit word per tensor (launch number in the high half, the
+// ratio's bits in the low half); both zero before the first launch.  epoch: a
+// launch number no earlier launch on these buffers used (never 0).  host_error:
+// device address of a host-mapped word, set to 1 if a wait gives up.  direction:
+// scratch of slot_elems floats per chunk-table entry (entry c at c * slot_elems;
+// slot_elems a multiple of 4 and at least the longest entry, the array 16-byte
+// aligned), written and read within the launch.  cfg.pre: PRE_NONE with or
+// without PRE_COPY16 and PRE_MOM16.  The grid is n_items + lag CTAs.
+cudaError_t launch_step_adapt(const int *item_first, const Chunk *item_chunk, int n_items, int lag,
                               const TensorRec *d_recs, const int *tensor_first,
                               double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
                               unsigned *arrived, unsigned long long *ready, unsigned *host_error,

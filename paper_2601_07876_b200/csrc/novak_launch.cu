@@ -91,7 +91,7 @@ cudaError_t noalloc_table(TensorRec **d_recs, Chunk **d_chunks)
 
 int step_block_threads() { return kBlock; }
 
-cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int n_items,
+cudaError_t launch_step_adapt(const int *item_first, const Chunk *item_chunk, int n_items, int lag,
                               const TensorRec *d_recs, const int *tensor_first,
                               double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
                               unsigned *arrived, unsigned long long *ready, unsigned *host_error,
@@ -99,7 +99,7 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
                               const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
                               int la, const LaunchCfg &cfg, cudaStream_t stream)
 {
-    using Fn = void (*)(const int *, const Chunk *, int, const TensorRec *, const int *, double *,
+    using Fn = void (*)(const int *, const Chunk *, int, int, const TensorRec *, const int *, double *,
                         double *, float *, AdaptCtl *, unsigned *, unsigned long long *, unsigned *,
                         float *, int, StepScalars, unsigned);
     void *raw = nullptr;
@@ -110,12 +110,12 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
     default: break;
     }
     Fn fn = reinterpret_cast<Fn>(raw);
-    if (!fn || !item_code || !item_chunk || n_items <= 0 || epoch == 0u || !ctl || !arrived || !ready ||
+    if (!fn || !item_first || !item_chunk || n_items <= 0 || lag < 0 || epoch == 0u || !ctl || !arrived || !ready ||
         !host_error || !tensor_first || !chunk_u2 || !chunk_p2 || !trust || !direction ||
         slot_elems <= 0 || (slot_elems & 3) != 0)
         return cudaErrorInvalidValue;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(static_cast<unsigned>(n_items));
+    lc.gridDim = dim3(static_cast<unsigned>(n_items) + static_cast<unsigned>(lag));
     lc.blockDim = dim3(kBlock);
     lc.dynamicSmemBytes = 0;
     lc.stream = stream;
@@ -124,7 +124,7 @@ cudaError_t launch_step_adapt(const int *item_code, const Chunk *item_chunk, int
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = (cfg.pdl & 1) ? 1 : 0;
-    return cudaLaunchKernelEx(&lc, fn, item_code, item_chunk, n_items, d_recs, tensor_first,
+    return cudaLaunchKernelEx(&lc, fn, item_first, item_chunk, n_items, lag, d_recs, tensor_first,
                               chunk_u2, chunk_p2, trust, ctl, arrived, ready, host_error, direction,
                               slot_elems, s, epoch);
 }

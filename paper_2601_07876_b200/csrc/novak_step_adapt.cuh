@@ -1,34 +1,42 @@
 // Layer-wise adaptation (Eq. 19 / 25) and the step in ONE launch for sm_100a.
 //
 // The trust ratio of a tensor needs ||u_t|| over the whole tensor before any of
-// its elements moves, so theta, g, m, v of a tensor are needed twice.  Run as
-// two passes over the whole group (novak_trust_stats.cu, then the step kernel)
-// the second pass finds nothing of the first in L2: 16 + 28 B per element from
-// DRAM.  Here both passes are ITEMS of one grid, one item per CTA: S items (the
-// two sums of squares of one chunk-table entry, loads that stay in L2) and U
-// items (the ordinary step over one entry, streaming loads), in an order in
-// which the statistics run a fixed number of items ahead of the updates:
+// its elements moves.  Run as two passes over the whole group
+// (novak_trust_stats.cu, then the step kernel) theta, g, m, v are read twice,
+// and the second pass finds nothing of the first in L2: 16 + 28 B per element
+// from DRAM.  Here the work is cut differently.  The group is a list of ITEMS (a
+// few consecutive chunk-table entries of one tensor each), and CTA number b does
+// two things:
 //
-//     S(T0) S(T1) ... | U(T0) S(Tk) U(T1) S(Tk+1) ...        (whole tensors)
+//   S part, item b: the whole of phases 2-8 for the item's elements - moments
+//       advanced and stored for good, the direction the update will multiply by
+//       the step (Eq. 17 after Eq. 27 and Eq. 16) left in a scratch array, the
+//       squares of theta and of the base direction added up.  The CTA that
+//       completes a tensor's last S part adds the tensor's sums in table order
+//       (fixed order: bit-identical from run to run) and publishes the ratio as
+//       one 64-bit word (launch number, ratio).
+//   U part, item b - lag: phases 9-10 from theta and the stored direction, both
+//       of which the S part of that item touched a few tens of MB of traffic
+//       ago and which are still in the 126 MB L2.
 //
-// so that a tensor's update follows its statistics by a few tens of MB of
-// traffic, while its 16 B per element are still in the 126 MB L2.  CTA number b
-// takes item number b.  The CTA that completes a tensor's last S item adds the
-// tensor's sums in table order (fixed order: bit-identical from run to run) and
-// publishes the ratio as one 64-bit word (launch number, ratio); a U item waits
-// for its tensor's word, every warp polling for itself (no CTA-wide barrier on
-// the way to the first load).
+// DRAM sees theta, g, m, v once and m, v, theta written once: about 30 B per
+// element instead of 44.  The operations and their order are those of
+// update_element(), cut in two after the direction: results are bit-identical
+// to the two-pass route.
 //
-// The wait and forward progress: a U item waits only for S items that stand
-// earlier in the order.  The hardware hands out the CTAs of a grid in
-// increasing block index as slots become free (the behaviour single-pass scans
-// with look-back rely on as well), so those S items belong to CTAs that are
-// running or have finished, and S items never wait; with the lead between S
-// and U the ratio is normally there long before it is asked for.  Nothing in
-// the programming model promises that order, so the wait is bounded: after
-// about two seconds (at once, when another CTA has already given up) a warp
-// gives up, raises an error flag in host-mapped memory, leaves its part of the
-// entry untouched and returns; the next call on the handle reports it, and
+// The wait and forward progress: the U part waits for its tensor's word.  lag
+// is at least the number of items of the longest tensor minus one, so the S
+// parts it waits for belong to CTAs with a lower block index (or to this CTA,
+// which has finished its own S part by then), and an S part never waits.  The
+// hardware hands out the CTAs of a grid in increasing block index as slots
+// become free (the behaviour single-pass scans with look-back rely on as well),
+// so those CTAs are running or have finished; with a lag beyond the number of
+// resident CTAs the word is normally there long before it is asked for.
+// Nothing in the programming model promises that order, so the wait is
+// bounded: after about two seconds (at once, when another CTA has already given
+// up) a warp gives up, raises an error flag in host-mapped memory, leaves its
+// share of the item's parameters untouched (the moments HAVE advanced) and
+// returns; the next call on the handle reports it, and
 // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 0 selects the three-launch form.
 #pragma once
 
@@ -280,8 +288,8 @@ __device__ __forceinline__ void entry_apply(const Chunk &ch, const TensorRec &r,
 #endif
 template <int NEST, int GT, int LA, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_ADAPT_MIN_CTAS)
-novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restrict__ item_chunk,
-                        int n_items, const TensorRec *__restrict__ recs,
+novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restrict__ item_chunk,
+                        int n_items, int lag, const TensorRec *__restrict__ recs,
                         const int *__restrict__ tensor_first, double *chunk_u2, double *chunk_p2,
                         float *trust, AdaptCtl *ctl, unsigned *arrived, unsigned long long *ready,
                         unsigned *host_error, float *direction, int slot_elems,
@@ -293,30 +301,32 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
     __shared__ int sh_flag;
 
     grid_dependency_release();
-    const int it = blockIdx.x;
-    if (it >= n_items) return;
-    // The item tables and the records are written by copies only, never by a
+    const int bs = blockIdx.x;               // item of the S part
+    const int bu = bs - lag;                 // item of the U part
+    const bool has_s = bs < n_items;
+    const bool has_u = bu >= 0 && bu < n_items;
+    // The item table and the records are written by copies only, never by a
     // kernel: read before the previous kernel on the stream has finished.
-    const int code = item_code[it];
-    const Chunk ch = item_chunk[it];                    // the item's entries as one span
-    const int c = code & 0x7fffffff;                    // its first entry's index in the chunk table
-    const TensorRec r = recs[ch.tensor];
+    int c_s = 0, c_u = 0;
+    Chunk ch_s = {}, ch_u = {};
+    if (has_s) { c_s = item_first[bs]; ch_s = item_chunk[bs]; }
+    if (has_u) { c_u = item_first[bu]; ch_u = item_chunk[bu]; }
     grid_dependency_wait();
 
-    // entry c + j of the item keeps element e at d[j * slot_elems + e]
-    float *d = direction + static_cast<size_t>(c) * static_cast<size_t>(slot_elems);
-
-    if (code >= 0) {
-        // ---- S item: moments, direction and the two sums of squares of each entry
-        const int c0 = tensor_first[ch.tensor], c1 = tensor_first[ch.tensor + 1];
-        const int cnt = (ch.len + slot_elems - 1) / slot_elems;        // <= kAdaptGroupMax
+    if (has_s) {
+        // ---- S part: moments, direction and the two sums of squares of each entry;
+        // entry c_s + j keeps element e at d[j * slot_elems + e]
+        const TensorRec r = recs[ch_s.tensor];
+        float *d = direction + static_cast<size_t>(c_s) * static_cast<size_t>(slot_elems);
+        const int c0 = tensor_first[ch_s.tensor], c1 = tensor_first[ch_s.tensor + 1];
+        const int cnt = (ch_s.len + slot_elems - 1) / slot_elems;      // <= kAdaptGroupMax
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll 1
         for (int j = 0; j < cnt; ++j) {
             Chunk sub;
-            sub.tensor = ch.tensor;
-            sub.offset = ch.offset + static_cast<int64_t>(j) * slot_elems;
-            sub.len = min(slot_elems, ch.len - j * slot_elems);
+            sub.tensor = ch_s.tensor;
+            sub.offset = ch_s.offset + static_cast<int64_t>(j) * slot_elems;
+            sub.len = min(slot_elems, ch_s.len - j * slot_elems);
             double sp, su;
             entry_direction<NEST, GT, PRE>(sub, r, d + static_cast<size_t>(j) * slot_elems, s, sp, su);
             sp = trust_warp_sum(sp);
@@ -335,35 +345,37 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
                 tp += sh_part[threadIdx.x][0][w];
                 tu += sh_part[threadIdx.x][1][w];
             }
-            chunk_p2[c + threadIdx.x] = tp;
-            chunk_u2[c + threadIdx.x] = tu;
+            chunk_p2[c_s + threadIdx.x] = tp;
+            chunk_u2[c_s + threadIdx.x] = tu;
         }
         __syncthreads();
         if (threadIdx.x == 0) {
             __threadfence();                 // the CTA's sums and directions before the arrival
             const unsigned total = static_cast<unsigned>(c1 - c0);
-            const unsigned before = atomicAdd(&arrived[ch.tensor], static_cast<unsigned>(cnt));
+            const unsigned before = atomicAdd(&arrived[ch_s.tensor], static_cast<unsigned>(cnt));
             sh_flag = (before + static_cast<unsigned>(cnt) == total) ? 1 : 0;
             // the tensor's last item leaves the counter at 0 for the next launch
-            if (sh_flag) atomicExch(&arrived[ch.tensor], 0u);
+            if (sh_flag) atomicExch(&arrived[ch_s.tensor], 0u);
         }
         __syncthreads();
-        if (sh_flag == 0) return;
-        // the tensor's last item: every sum is there
-        __threadfence();
-        const float eta = tensor_trust_ratio(chunk_p2, chunk_u2, c0, c1, sh);
-        if (threadIdx.x == 0) {
-            trust[ch.tensor] = eta;          // for novak_get_trust_ratios
-            store_release(&ready[ch.tensor], pack_ratio(epoch, eta));
+        if (sh_flag != 0) {                  // (uniform over the CTA)
+            // the tensor's last item: every sum is there
+            __threadfence();
+            const float eta = tensor_trust_ratio(chunk_p2, chunk_u2, c0, c1, sh);
+            if (threadIdx.x == 0) {
+                trust[ch_s.tensor] = eta;    // for novak_get_trust_ratios
+                store_release(&ready[ch_s.tensor], pack_ratio(epoch, eta));
+            }
         }
-        return;
     }
+    if (!has_u) return;
 
-    // ---- U item: the ordinary step over this entry, stretched by the tensor's ratio.
+    // ---- U part: phases 9-10 over an earlier item, stretched by its tensor's ratio.
     // Lane 0 of every warp polls; the warp goes on as soon as it has the ratio.
+    const TensorRec r = recs[ch_u.tensor];
     unsigned long long word = 0ull;
     if ((threadIdx.x & 31u) == 0u) {
-        word = wait_for_ratio(&ready[ch.tensor], epoch, &ctl->error);
+        word = wait_for_ratio(&ready[ch_u.tensor], epoch, &ctl->error);
         if (word == 0ull) {
             atomicExch(&ctl->error, 1u);
             *reinterpret_cast<volatile unsigned *>(host_error) = 1u;
@@ -373,7 +385,8 @@ novak_step_adapt_kernel(const int *__restrict__ item_code, const Chunk *__restri
     word = __shfl_sync(0xffffffffu, word, 0);
     if (word == 0ull) return;            // (the update below has no CTA-wide barrier)
     const float step = s.step * __uint_as_float(static_cast<unsigned>(word));      // Eq. 24a
-    entry_apply<LA, PRE>(ch, r, d, s, step);
+    entry_apply<LA, PRE>(ch_u, r, direction + static_cast<size_t>(c_u) * static_cast<size_t>(slot_elems),
+                         s, step);
 }
 
 template <int NEST, int GT, int PRE>

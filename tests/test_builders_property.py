@@ -93,43 +93,32 @@ def test_own_units_cover_the_rows_of_owned_tensors_once(data):
 @settings(max_examples=80, deadline=None)
 @given(counts=st.lists(st.integers(1, 40), min_size=1, max_size=30), lead=st.integers(0, 120),
        group=st.integers(1, 8))
-def test_adapt_order_puts_statistics_first_and_keeps_the_lead(counts, lead, group):
-    """Item order of the one-launch layer adaptation: every chunk-table entry in exactly one
-    statistics item and one update item; an item is a run of at most `group` entries of one
-    tensor, the tensor's first entry (the only one but its last that may be short) alone;
-    all statistics items of a tensor before any of its update items (what the kernel's
-    freedom from deadlock rests on); tensors in order within each kind; items of at least
-    `lead` entries between a tensor's last statistics item and its first update item,
-    except for what is flushed at the end."""
+def test_adapt_items_cover_the_table_and_the_lag_orders_statistics_before_updates(counts, lead, group):
+    """Work list of the one-launch layer adaptation: every chunk-table entry in exactly one
+    item, items in tensor order; an item is a run of at most `group` entries of one tensor,
+    the tensor's first entry (the only one but its last that may be short) alone.  CTA b
+    takes the statistics of item b and the update of item b - lag: every statistics part
+    an update waits for belongs to a CTA with a lower index or to the CTA itself (what the
+    kernel's freedom from deadlock rests on), and the lag is no shorter than the lead asks."""
     first = np.concatenate([[0], np.cumsum(counts)]).tolist()
-    order = B.novak_build_adapt_order(first, lead, group)
+    items, lag = B.novak_build_adapt_order(first, lead, group)
     total = first[-1]
     tensor_of = np.repeat(np.arange(len(counts)), counts)
-    for kind in (False, True):
-        covered = []
-        for c, k, upd in order:
-            if upd != kind:
-                continue
-            assert 1 <= k <= group
-            assert len(set(tensor_of[c:c + k])) == 1            # one tensor
-            if c == first[tensor_of[c]]:
-                assert k == 1                                       # its first entry stands alone
-            covered.extend(range(c, c + k))
-        assert covered == list(range(total))                       # once each, tensors in order
-    # position of every item measured in entries emitted before it
-    before, pos_s, pos_u = 0, {}, {}
-    for c, k, upd in order:
-        for e in range(c, c + k):
-            (pos_u if upd else pos_s)[e] = (before, before + k)
-        before += k
-    last_stats_end = max(end for _, end in pos_s.values())
-    for t in range(len(counts)):
-        cs = range(first[t], first[t + 1])
-        s_end = max(pos_s[c][1] for c in cs)
-        u_start = min(pos_u[c][0] for c in cs)
-        assert s_end <= u_start
-        if u_start < last_stats_end:           # not part of the final flush
-            assert u_start - s_end >= lead
+    covered = []
+    for c, k in items:
+        assert 1 <= k <= group
+        assert len(set(tensor_of[c:c + k])) == 1            # one tensor
+        if c == first[tensor_of[c]]:
+            assert k == 1                                       # its first entry stands alone
+        covered.extend(range(c, c + k))
+    assert covered == list(range(total))                       # once each, tensors in order
+    item_tensor = [int(tensor_of[c]) for c, _ in items]
+    last_item = {t: i for i, t in enumerate(item_tensor)}
+    for u, t in enumerate(item_tensor):
+        cta = u + lag                                           # the CTA that updates item u
+        assert last_item[t] <= cta                              # statistics of the whole tensor: earlier CTAs or its own
+    longest = max(np.bincount(item_tensor))
+    assert lag == longest - 1 + -(-lead // group)
 
 
 @settings(max_examples=60, deadline=None)
