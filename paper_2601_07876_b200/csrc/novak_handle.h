@@ -128,7 +128,7 @@ struct Handle {
     std::vector<int> h_tensor_first;
     // layer adaptation and step in one launch: the claim-ordered item list, the
     // kernel's counters and per-tensor flags (one allocation), a host-mapped error word
-    int adapt_in_step = 0;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
+    int adapt_in_step = 1;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
     int64_t adapt_lead_elems = 1 << 22;    // NOVAK_OPT_LAYER_ADAPTATION_LEAD
     int adapt_group = 4;                   // NOVAK_OPT_LAYER_ADAPTATION_GROUP
     char *d_adapt = nullptr;

@@ -313,6 +313,8 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
     if (has_u) { c_u = item_first[bu]; ch_u = item_chunk[bu]; }
     grid_dependency_wait();
 
+    TensorRec r_u = {};
+    unsigned long long word = 0ull;          // lane 0: the U part's tensor's word, once it is this launch's
     if (has_s) {
         // ---- S part: moments, direction and the two sums of squares of each entry;
         // entry c_s + j keeps element e at d[j * slot_elems + e]
@@ -335,6 +337,11 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
                 sh_part[j][0][warp] = sp;
                 sh_part[j][1][warp] = su;
             }
+        }
+        // the U part's record and its tensor's word: on their way during the reduction below
+        if (has_u) {
+            r_u = recs[ch_u.tensor];
+            if (lane == 0) word = load_acquire(&ready[ch_u.tensor]);
         }
         __syncthreads();
         if (static_cast<int>(threadIdx.x) < cnt) {
@@ -372,10 +379,10 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
 
     // ---- U part: phases 9-10 over an earlier item, stretched by its tensor's ratio.
     // Lane 0 of every warp polls; the warp goes on as soon as it has the ratio.
-    const TensorRec r = recs[ch_u.tensor];
-    unsigned long long word = 0ull;
+    if (!has_s) r_u = recs[ch_u.tensor];
     if ((threadIdx.x & 31u) == 0u) {
-        word = wait_for_ratio(&ready[ch_u.tensor], epoch, &ctl->error);
+        if (static_cast<unsigned>(word >> 32) != epoch)
+            word = wait_for_ratio(&ready[ch_u.tensor], epoch, &ctl->error);
         if (word == 0ull) {
             atomicExch(&ctl->error, 1u);
             *reinterpret_cast<volatile unsigned *>(host_error) = 1u;
@@ -385,7 +392,7 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
     word = __shfl_sync(0xffffffffu, word, 0);
     if (word == 0ull) return;            // (the update below has no CTA-wide barrier)
     const float step = s.step * __uint_as_float(static_cast<unsigned>(word));      // Eq. 24a
-    entry_apply<LA, PRE>(ch_u, r, direction + static_cast<size_t>(c_u) * static_cast<size_t>(slot_elems),
+    entry_apply<LA, PRE>(ch_u, r_u, direction + static_cast<size_t>(c_u) * static_cast<size_t>(slot_elems),
                          s, step);
 }
 

@@ -141,20 +141,20 @@ def test_graph_capturable_option():
 
 
 def test_in_step_options_roundtrip_and_defaults():
-    """Centralization inside the step kernel is on by default, the one-launch layer
-    adaptation off; its lead is an element count, its group a number of entries."""
+    """Centralization inside the step kernel and the one-launch layer adaptation are on
+    by default; its lead is an element count, its group a number of entries."""
     h = B.Handle(**GOOD)
     assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 1
-    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 0
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 1
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 2 ** 22
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP) == 4
     h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP, 8)
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP) == 8
     h.set_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP, 0)
-    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 1)
+    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 0)
     h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0)
     assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 0
-    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 1
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 0
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 0
     for key, bad in ((B.NOVAK_OPT_CENTRALIZE_IN_STEP, 2), (B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, -1),
                      (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, -1), (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0.5),
