@@ -102,10 +102,11 @@ def parse_args():
     ap.add_argument("--layer-adaptation", action="store_true",
                     help="layer-wise trust ratios (Eq. 19): theta, g, m, v are read once more")
     ap.add_argument("--layer-adaptation-in-step", type=int, default=None, choices=[0, 1],
-                    help="1: layer adaptation and update as one kernel whose update items find "
-                         "their tensor in L2 (default 0: two statistics kernels, then the step)")
+                    help="0: two statistics kernels, then the step (default 1: layer adaptation and "
+                         "update as one kernel whose updates find theta and the direction in L2)")
     ap.add_argument("--layer-adaptation-lead", type=int, default=None,
-                    help="elements by which that kernel's statistics run ahead of its updates")
+                    help="elements by which that kernel's updates trail its statistics beyond what "
+                         "the longest tensor needs")
     ap.add_argument("--layer-adaptation-group", type=int, default=None,
                     help="chunk-table entries per CTA of that kernel (1..8)")
     ap.add_argument("--adaptive-beta", action="store_true", help="Eq. 3-4 (host scalars only)")

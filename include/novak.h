@@ -159,20 +159,23 @@ enum {
                                      statistics pass): one launch and 28 B per element
                                      instead of three launches and 32 B.  0: always
                                      the statistics pass                               */
-    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1: with layer adaptation on and no clipping,
-                                     centralization or automatic learning-rate
+    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1 (default): with layer adaptation on and no
+                                     clipping, centralization or automatic learning-rate
                                      scaling, novak_step runs statistics and update as
-                                     ONE kernel in which a tensor's update follows its
-                                     statistics closely enough to find its theta, g,
-                                     m, v still in L2 (about 28 B per element from
-                                     DRAM instead of 44; measured slower all the same,
-                                     the kernel being bound by instruction issue and
-                                     latency, not by DRAM).  0 (default): two
+                                     ONE kernel: a CTA advances the moments of one run
+                                     of chunk-table entries, leaves the direction of
+                                     the update in a scratch array (4 B per element of
+                                     the group, allocated at the first such step) and
+                                     adds up the norms, then applies the update of an
+                                     earlier run whose tensor's ratio is known, from
+                                     theta and the direction still in L2: about 30 B
+                                     per element from DRAM instead of 44.  0: two
                                      statistics kernels, then the step.  Same results
                                      bit for bit                                      */
-    NOVAK_OPT_LAYER_ADAPTATION_LEAD = 26, /* how far, in elements, that kernel's statistics
-                                     run ahead of its updates (default 2^22); only
-                                     before the first such step                        */
+    NOVAK_OPT_LAYER_ADAPTATION_LEAD = 26, /* elements by which that kernel's updates trail
+                                     the statistics beyond what the longest tensor
+                                     needs (default 0); only before the first such
+                                     step                                              */
     NOVAK_OPT_LAYER_ADAPTATION_GROUP = 27, /* chunk-table entries one CTA of that kernel
                                      takes, 1..8 (default 4); only before the first
                                      such step                                         */

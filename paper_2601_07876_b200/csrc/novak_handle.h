@@ -129,7 +129,7 @@ struct Handle {
     // layer adaptation and step in one launch: the claim-ordered item list, the
     // kernel's counters and per-tensor flags (one allocation), a host-mapped error word
     int adapt_in_step = 1;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
-    int64_t adapt_lead_elems = 1 << 22;    // NOVAK_OPT_LAYER_ADAPTATION_LEAD
+    int64_t adapt_lead_elems = 0;          // NOVAK_OPT_LAYER_ADAPTATION_LEAD
     int adapt_group = 4;                   // NOVAK_OPT_LAYER_ADAPTATION_GROUP
     char *d_adapt = nullptr;
     int *d_item_code = nullptr;

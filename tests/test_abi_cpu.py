@@ -146,16 +146,16 @@ def test_in_step_options_roundtrip_and_defaults():
     h = B.Handle(**GOOD)
     assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 1
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 1
-    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 2 ** 22
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 0
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP) == 4
     h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP, 8)
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_GROUP) == 8
     h.set_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP, 0)
     h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, 0)
-    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0)
+    h.set_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 2 ** 20)
     assert h.get_option(B.NOVAK_OPT_CENTRALIZE_IN_STEP) == 0
     assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP) == 0
-    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 0
+    assert h.get_option(B.NOVAK_OPT_LAYER_ADAPTATION_LEAD) == 2 ** 20
     for key, bad in ((B.NOVAK_OPT_CENTRALIZE_IN_STEP, 2), (B.NOVAK_OPT_LAYER_ADAPTATION_IN_STEP, -1),
                      (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, -1), (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 0.5),
                      (B.NOVAK_OPT_LAYER_ADAPTATION_LEAD, 2.0 ** 31),
