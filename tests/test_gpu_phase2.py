@@ -342,6 +342,41 @@ def test_fullsize_resnet50_with_clipping_and_centralization(clip):
           + ", ".join(f"{k} {v:.3f}" for k, v in worst.items()))
 
 
+def test_fullsize_resnet50_with_layer_adaptation():
+    """The benchmark's ResNet-50-shaped set, layer adaptation in one launch (items of four
+    chunk-table entries, updates trailing the statistics by the longest tensor's 287 items)
+    for 12 steps: every element and every trust ratio against the oracle, and parameters bit
+    for bit against a twin that takes the three-launch form."""
+    wl = W.get_workload(1)
+    flats, sets = [], []
+    for _ in range(2):
+        flat_p = W.alloc_flat(wl, torch.float32, DEV)
+        W.init_params(wl, flat_p)
+        flats.append(flat_p)
+        sets.append([v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)])
+    flat_g = W.alloc_flat(wl, torch.float32, DEV)
+    grads = [v.view(s) for v, s in zip(W.views(flat_g, wl), wl.shapes)]
+    src = W.GradSource(wl, DEV)
+    harness.MARGINS.clear()
+    hyper = dict(wl.hyper, layer_adaptation=True)
+    pair = Pair(sets[0], hyper)
+    twin = B.NovakOptimizer(sets[1], **hyper, layer_adaptation_in_step=0)
+    for _ in range(12):
+        src.fill(flat_g)
+        pair.step(grads, threads=8)
+        twin.step(grads)
+        np.testing.assert_allclose(pair.opt.trust_ratios(), pair.oracle.trust[-1], rtol=2e-6)
+    pair.check("resnet50 layer adaptation")
+    assert torch.equal(flats[0], flats[1])
+    assert pair.opt.trust_ratios() == twin.trust_ratios()
+    assert pair.opt.info()["launches"] == 12 and twin.info()["launches"] == 36
+    worst = {}
+    for k, v in harness.MARGINS.items():
+        worst[k.split()[-1].split("[")[0]] = max(worst.get(k.split()[-1].split("[")[0], 0.0), v)
+    print("\nPARITY resnet50 layer adaptation (one launch) steps=12 every element worst |err|/tol: "
+          + ", ".join(f"{k} {v:.3f}" for k, v in worst.items()))
+
+
 # ---------------------------------------------------------------------------
 # Phase 7: layer-wise adaptation (Eq. 19 / 25)
 # ---------------------------------------------------------------------------
