@@ -485,25 +485,6 @@ def test_layer_adaptation_zero_gradient_and_reruns():
         assert torch.equal(a, b)
 
 
-def test_fullsize_resnet50_with_layer_adaptation():
-    wl = W.get_workload(1)
-    flat_p = W.alloc_flat(wl, torch.float32, DEV)
-    W.init_params(wl, flat_p)
-    params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
-    flat_g = W.alloc_flat(wl, torch.float32, DEV)
-    grads = [v.view(s) for v, s in zip(W.views(flat_g, wl), wl.shapes)]
-    src = W.GradSource(wl, DEV)
-    harness.MARGINS.clear()
-    pair = Pair(params, dict(wl.hyper, layer_adaptation=True))
-    for _ in range(12):
-        src.fill(flat_g)
-        pair.step(grads, threads=8)
-        np.testing.assert_allclose(pair.opt.trust_ratios(), pair.oracle.trust[-1], rtol=2e-6)
-    pair.check("resnet50 layer adaptation")
-    worst = max(harness.MARGINS.values())
-    print(f"\nPARITY resnet50 layer adaptation steps=12 every element worst |err|/tol: {worst:.3f}")
-
-
 # ---------------------------------------------------------------------------
 # Phase 8: sparse updates (Eq. 27)
 # ---------------------------------------------------------------------------
