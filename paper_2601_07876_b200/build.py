@@ -20,7 +20,7 @@ LIB = os.path.join(PKG, "libnovak.so")
 # once per mode, and once more per mode for the graph-capturable kernel.
 PRE_MODES = tuple(range(16))
 DYN_PRE_MODES = (0, 1, 2, 4, 5, 6, 8, 9, 10, 12, 13, 14)   # no row-owning form (mode 3)
-PLAIN_SOURCES = ("novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu",
+PLAIN_SOURCES = ("novak_host.cpp", "novak_host_device.cpp", "novak_host_step.cpp", "novak_launch.cu", "novak_launch_adapt.cu",
                  "novak_grad_stats.cu", "novak_trust_stats.cu", "novak_nesterov.cu", "novak_dyn.cu")
 # (source, object name, extra flags)
 UNITS = [(os.path.join(CSRC, f), f + ".o", []) for f in PLAIN_SOURCES]
