@@ -152,6 +152,8 @@ def parse_args():
     ap.add_argument("--max-repeats", type=int, default=2000)
     ap.add_argument("--per-step-steps", type=int, default=300,
                     help="steps of the separate pass that times every step on its own (0: skip)")
+    ap.add_argument("--no-per-feature", action="store_true",
+                    help="skip the paths around the plain step on the headline workload (key per_feature)")
     ap.add_argument("--no-per-workload", action="store_true",
                     help="skip the other workloads / lookahead modes (key per_workload)")
     return ap.parse_args()
@@ -494,6 +496,75 @@ def time_one_workload(torch, B, W, dev, index, mode, steps, warmup, min_seconds,
     return out
 
 
+# The paths around the plain step, each timed on the headline workload (key per_feature).
+# (name, optimizer keywords, bf16 parameter copies, algorithmic-byte keywords)
+FEATURES = (
+    ("clip", dict(clip_threshold=1.0), False, dict(phase2=True)),
+    ("centralize", dict(centralize=True), False, dict()),
+    ("clip+centralize", dict(clip_threshold=1.0, centralize=True), False, dict(phase2=True)),
+    ("layer_adaptation", dict(layer_adaptation=True), False, dict(trust="fits")),
+    ("layer_adaptation, three launches", dict(layer_adaptation=True, layer_adaptation_in_step=0),
+     False, dict(trust=1.0)),
+    ("bf16 moments", dict(moment_dtype="bf16"), False, dict(moment_bytes=2)),
+    ("bf16 parameter copies", dict(), True, dict(copy16=True)),
+)
+
+
+def time_one_feature(torch, B, W, dev, index, mode, feature, steps, warmup, min_seconds,
+                     max_repeats, pool_want, lib, barrier):
+    """One of FEATURES on one workload, everything resident: median ms per step over
+    repeated `steps`-step regions, against the bytes that path has to move."""
+    name, kw, copies, alg_kw = feature
+    wl = W.get_workload(index)
+    hyper = dict(wl.hyper, lookahead_mode=mode)
+    k = hyper["lookahead_k"]
+    gbytes = 2 if wl.grad_dtype == torch.bfloat16 else 4
+    flat_p = W.alloc_flat(wl, torch.float32, dev)
+    W.init_params(wl, flat_p)
+    params = [v.view(s) for v, s in zip(W.views(flat_p, wl), wl.shapes)]
+    pool_n = max(1, min(pool_want, int(8e9 // (wl.total * gbytes)) or 1))
+    src = W.GradSource(wl, dev)
+    scratch = W.alloc_flat(wl, torch.float32, dev) if gbytes == 2 else None
+    pool_flat = [W.alloc_flat(wl, wl.grad_dtype, dev) for _ in range(pool_n)]
+    for gf in pool_flat:
+        src.fill(gf, scratch)
+    del scratch
+    opt = B.NovakOptimizer(params, **hyper, **kw, lib=lib)
+    pool = [opt.prepare(W.views(gf, wl)) for gf in pool_flat]
+    copy_flat = None
+    if copies:
+        copy_flat = W.alloc_flat(wl, torch.bfloat16, dev)
+        opt.set_param_copies(W.views(copy_flat, wl))
+    for i in range(max(3, warmup)):
+        opt.step(pool[i % pool_n])
+    probe = timed_repeats(torch, lambda i: opt.step(pool[i % pool_n]), steps, 1, barrier)[0] / steps
+    repeats = repeats_for(probe, steps, min_seconds, max_repeats)
+    t_first = opt.info()["t"] + 1
+    l0 = opt.info()["launches"]
+    times = timed_repeats(torch, lambda i: opt.step(pool[i % pool_n]), steps, repeats, barrier)
+    launches = (opt.info()["launches"] - l0) / (steps * repeats)
+    per = sorted(x / steps for x in times)
+    ms = quantile(per, 0.5)
+    alg_kw = dict(alg_kw)
+    mbytes = alg_kw.get("moment_bytes", 4)
+    if alg_kw.get("trust") == "fits":
+        # one launch: only tensors too large to wait in L2 (theta, g, m, v beyond 48 MB) count twice
+        per_elem_twice = 4 + 2 * mbytes + gbytes
+        alg_kw["trust"] = sum(n for n in wl.numel if n * per_elem_twice > 48e6) / wl.total
+    alg = sum(algorithmic_bytes_per_elem(gbytes, k, mode, t, **alg_kw)
+              for t in range(t_first, t_first + steps * repeats)) / (steps * repeats)
+    gbs = alg * wl.total / (ms * 1e-3) / 1e9
+    peak, _ = measured_peak()
+    out = {"feature": name, "workload": wl.name, "lookahead_mode": mode, "steps": steps,
+           "repeats": repeats, "ms_per_step": ms, "p10": quantile(per, 0.1), "p90": quantile(per, 0.9),
+           "updates_per_s": wl.total / (ms * 1e-3), "algorithmic_bytes_per_elem": alg,
+           "hbm_gbs": gbs, "frac": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0,
+           "launches_per_step": launches, "warnings": opt.info()["warnings"]}
+    del opt, pool, pool_flat, params, flat_p, copy_flat
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -744,6 +815,13 @@ def main():
                     torch, B, W, dev, index, mode, steps_i, args.warmup, args.min_timed_seconds,
                     args.max_repeats, args.pool, lib, barrier))
 
+    per_feature = None
+    if per_workload is not None and not args.no_per_feature:
+        per_feature = [time_one_feature(torch, B, W, dev, wl.index, args.lookahead_mode, feat,
+                                        args.steps, args.warmup, args.min_timed_seconds / 2,
+                                        args.max_repeats, args.pool, lib, barrier)
+                       for feat in FEATURES]
+
     if rank == 0:
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -784,6 +862,7 @@ def main():
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "per_step": per,
             "per_workload": per_workload,
+            "per_feature": per_feature,
             "e2e": e2e,
             "cpu_baseline": cpu,
             "gpu_launches": launches,
