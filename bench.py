@@ -505,6 +505,8 @@ FEATURES = (
     ("layer_adaptation", dict(layer_adaptation=True), False, dict(trust="fits")),
     ("layer_adaptation, three launches", dict(layer_adaptation=True, layer_adaptation_in_step=0),
      False, dict(trust=1.0)),
+    ("clip+centralize+layer_adaptation", dict(clip_threshold=1.0, centralize=True, layer_adaptation=True),
+     False, dict(phase2=True, trust="fits")),
     ("bf16 moments", dict(moment_dtype="bf16"), False, dict(moment_bytes=2)),
     ("bf16 parameter copies", dict(), True, dict(copy16=True)),
 )
@@ -699,7 +701,7 @@ def main():
     per_elem_twice = 4 + 2 * mbytes + gbytes
     big = sum(n for n in wl.numel if n * per_elem_twice > 48e6) / wl.total
     trust_share = 0.0 if not args.layer_adaptation else (
-        big if (args.layer_adaptation_in_step != 0 and not prepass) else 1.0)
+        big if args.layer_adaptation_in_step != 0 else 1.0)
     alg = sum(algorithmic_bytes_per_elem(gbytes, k, args.lookahead_mode, t, phase2,
                                          trust_share, args.bf16_copy, args.auto_lr,
                                          ("restore" if args.restore_pass else True) if args.true_nesterov else False,

@@ -159,10 +159,11 @@ enum {
                                      statistics pass): one launch and 28 B per element
                                      instead of three launches and 32 B.  0: always
                                      the statistics pass                               */
-    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1 (default): with layer adaptation on and no
-                                     clipping, centralization or automatic learning-rate
-                                     scaling, novak_step runs statistics and update as
-                                     ONE kernel: a CTA advances the moments of one run
+    NOVAK_OPT_LAYER_ADAPTATION_IN_STEP = 25, /* 1 (default): with layer adaptation on,
+                                     novak_step runs its statistics and the update as
+                                     ONE kernel (behind the gradient's own statistics
+                                     pass where clipping, centralization or automatic
+                                     learning-rate scaling are on): a CTA advances the moments of one run
                                      of chunk-table entries, leaves the direction of
                                      the update in a scratch array (4 B per element of
                                      the group, allocated at the first such step) and

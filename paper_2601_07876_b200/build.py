@@ -28,7 +28,7 @@ UNITS += [(os.path.join(CSRC, "novak_step_inst.cu"), f"novak_step_mode{m}.o",
            [f"-DNOVAK_PRE_MODE={m}"]) for m in PRE_MODES]
 UNITS += [(os.path.join(CSRC, "novak_step_inst.cu"), f"novak_step_dyn_mode{m}.o",
            [f"-DNOVAK_PRE_MODE={m}", "-DNOVAK_INST_DYN"]) for m in DYN_PRE_MODES]
-ADAPT_PRE_MODES = (0, 4, 8, 12)     # layer adaptation and update in one launch: PRE_NONE modes
+ADAPT_PRE_MODES = DYN_PRE_MODES     # layer adaptation and update in one launch: no row-owning form either
 UNITS += [(os.path.join(CSRC, "novak_step_inst.cu"), f"novak_step_adapt_mode{m}.o",
            [f"-DNOVAK_PRE_MODE={m}", "-DNOVAK_INST_ADAPT"]) for m in ADAPT_PRE_MODES]
 SOURCES = sorted({u[0] for u in UNITS})

@@ -92,8 +92,7 @@ int begin_step(novak_opt *o, void *const *d_params, const void *const *d_grads, 
     }
     if (o->h.layer_adapt && (rc = prepare_trust(o, stream)) != NOVAK_OK) return rc;
     ctx->trust = o->h.layer_adapt ? o->trust : nullptr;
-    ctx->adapt_in_step = o->h.layer_adapt && whole_table && o->adapt_in_step && !o->dyn &&
-                         ctx->pre == novak::PRE_NONE;
+    ctx->adapt_in_step = o->h.layer_adapt && whole_table && o->adapt_in_step && !o->dyn;
     if (ctx->adapt_in_step && (rc = prepare_adapt(o, stream)) != NOVAK_OK) return rc;
     if (o->h_adapt_error && *o->h_adapt_error)
         return fail(o, NOVAK_ECUDA, "an earlier step's layer-adaptation kernel gave up waiting for a "
@@ -199,7 +198,7 @@ cudaError_t launch_range(novak_opt *o, const StepCtx &ctx, int c0, int c1, cudaS
         o->last_grid = cfg.grid;
         const unsigned epoch = o->adapt_epoch == 0xffffffffu ? 1u : o->adapt_epoch + 1u;
         const cudaError_t e = novak::launch_step_adapt(
-            o->d_item_code, o->d_item_chunk, o->n_items, o->adapt_lag, ctx.d_recs,
+            o->d_item_code, o->d_item_chunk, o->n_items, o->adapt_lag, ctx.d_recs, o->prep_out,
             o->tensor_first, o->chunk_u2, o->chunk_p2, o->trust, o->adapt_ctl, o->adapt_arrived,
             o->adapt_ready, o->d_adapt_error, o->adapt_direction, o->adapt_slot_elems, ctx.s, epoch, kernel_variant(ctx.plan), ctx.grad_dtype,
             ctx.la, cfg, stream);

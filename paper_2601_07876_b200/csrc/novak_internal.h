@@ -63,10 +63,11 @@ struct __align__(16) AdaptCtl {
 // device address of a host-mapped word, set to 1 if a wait gives up.  direction:
 // scratch of slot_elems floats per chunk-table entry (entry c at c * slot_elems;
 // slot_elems a multiple of 4 and at least the longest entry, the array 16-byte
-// aligned), written and read within the launch.  cfg.pre: PRE_NONE with or
-// without PRE_COPY16 and PRE_MOM16.  The grid is n_items + lag CTAs.
+// aligned), written and read within the launch.  prep: the statistics pass's
+// output (clip factor, Eq. 22), needed unless cfg.pre is a PRE_NONE mode.  cfg.pre:
+// any mode but the row-owning ones.  The grid is n_items + lag CTAs.
 cudaError_t launch_step_adapt(const int *item_first, const Chunk *item_chunk, int n_items, int lag,
-                              const TensorRec *d_recs, const int *tensor_first,
+                              const TensorRec *d_recs, const PrepOut *prep, const int *tensor_first,
                               double *chunk_u2, double *chunk_p2, float *trust, AdaptCtl *ctl,
                               unsigned *arrived, unsigned long long *ready, unsigned *host_error,
                               float *direction, int slot_elems,

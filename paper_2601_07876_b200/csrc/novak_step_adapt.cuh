@@ -107,7 +107,7 @@ __device__ __forceinline__ unsigned long long wait_for_ratio(const unsigned long
 template <int N, int U, int NEST, int GT, int PRE>
 __device__ __forceinline__ void direction_tile(const float *p, const void *g, void *m, void *v,
                                                float *d, int first, int nvec, const StepScalars &s,
-                                               double &sum_p, double &sum_u)
+                                               const PreArgs &pre, double &sum_p, double &sum_u)
 {
     constexpr bool kMom16 = (PRE & PRE_MOM16) != 0;
     Vec<N> P[U], G[U], M[U], V[U];
@@ -126,6 +126,8 @@ __device__ __forceinline__ void direction_tile(const float *p, const void *g, vo
         const int idx = first + j * kBlock;
         if (idx < nvec) {
             Vec<N> D;
+            // phase 2 on the gradient first: clip factor and row means, the statistics pass's output
+            preprocess<N, PRE>(G[j], row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre), pre);
             float sp = 0.0f, su = 0.0f;
 #pragma unroll
             for (int e = 0; e < N; ++e) {
@@ -155,7 +157,8 @@ __device__ __forceinline__ void direction_tile(const float *p, const void *g, vo
 // two sums (the vectors it took, in index order).
 template <int NEST, int GT, int PRE>
 __device__ __forceinline__ void entry_direction(const Chunk &ch, const TensorRec &r, float *d,
-                                                const StepScalars &s, double &sum_p, double &sum_u)
+                                                const StepScalars &s, const PreArgs &pre,
+                                                double &sum_p, double &sum_u)
 {
     constexpr int kGradBytes = (GT == NOVAK_GRAD_BF16) ? 2 : 4;
     constexpr int kMomBytes = (PRE & PRE_MOM16) ? 2 : 4;
@@ -174,15 +177,15 @@ __device__ __forceinline__ void entry_direction(const Chunk &ch, const TensorRec
         const int nvec = ch.len >> 2;
 #pragma unroll 1
         for (int base = 0; base < nvec; base += kBlock * 2)
-            direction_tile<4, 2, NEST, GT, PRE>(p, g, m, v, d, base + threadIdx.x, nvec, s, sum_p, sum_u);
+            direction_tile<4, 2, NEST, GT, PRE>(p, g, m, v, d, base + threadIdx.x, nvec, s, pre, sum_p, sum_u);
         // ragged tail: < 4 elements
         direction_tile<1, 1, NEST, GT, PRE>(p, g, m, v, d, (nvec << 2) + threadIdx.x, ch.len, s,
-                                            sum_p, sum_u);
+                                            pre, sum_p, sum_u);
     } else {
 #pragma unroll 1
         for (int base = 0; base < ch.len; base += kBlock * 4)
             direction_tile<1, 4, NEST, GT, PRE>(p, g, m, v, d, base + threadIdx.x, ch.len, s,
-                                                sum_p, sum_u);
+                                                pre, sum_p, sum_u);
     }
 }
 
@@ -289,13 +292,13 @@ __device__ __forceinline__ void entry_apply(const Chunk &ch, const TensorRec &r,
 template <int NEST, int GT, int LA, int PRE>
 __global__ void __launch_bounds__(NOVAK_BLOCK, NOVAK_ADAPT_MIN_CTAS)
 novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restrict__ item_chunk,
-                        int n_items, int lag, const TensorRec *__restrict__ recs,
+                        int n_items, int lag, const TensorRec *__restrict__ recs, const PrepOut *prep,
                         const int *__restrict__ tensor_first, double *chunk_u2, double *chunk_p2,
                         float *trust, AdaptCtl *ctl, unsigned *arrived, unsigned long long *ready,
                         unsigned *host_error, float *direction, int slot_elems,
                         const StepScalars s, unsigned epoch)
 {
-    static_assert((PRE & PRE_MASK) == PRE_NONE, "gradient pre-processing keeps the two-pass route");
+    static_assert((PRE & PRE_MASK) != PRE_CENTER_ROWS, "the row-owning kernel is a form of its own");
     __shared__ double sh[kTrustWarps];
     __shared__ double sh_part[kAdaptGroupMax][2][kTrustWarps];
     __shared__ int sh_flag;
@@ -313,6 +316,14 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
     if (has_u) { c_u = item_first[bu]; ch_u = item_chunk[bu]; }
     grid_dependency_wait();
 
+    // The clip factor and Eq. 22 are the statistics pass's output (it may still have been
+    // running while this grid became resident): plain loads, only now.
+    float factor = 1.0f, step_all = s.step;
+    if constexpr ((PRE & PRE_MASK) == PRE_SCALE || (PRE & PRE_MASK) == PRE_CENTER) {
+        factor = prep->factor;
+        step_all *= prep->auto_scale;        // 1 when the scaling is off; Eq. 24a
+    }
+
     TensorRec r_u = {};
     unsigned long long word = 0ull;          // lane 0: the U part's tensor's word, once it is this launch's
     if (has_s) {
@@ -329,8 +340,15 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
             sub.tensor = ch_s.tensor;
             sub.offset = ch_s.offset + static_cast<int64_t>(j) * slot_elems;
             sub.len = min(slot_elems, ch_s.len - j * slot_elems);
+            PreArgs pre;
+            pre.copy = nullptr;
+            pre.step = 0.0f;
+            pre.factor = factor;
+            pre.mean = ((PRE & PRE_MASK) == PRE_CENTER) ? r.mean : nullptr;
+            pre.row_len = r.row_len;
+            pre.elem0 = static_cast<uint32_t>(sub.offset);
             double sp, su;
-            entry_direction<NEST, GT, PRE>(sub, r, d + static_cast<size_t>(j) * slot_elems, s, sp, su);
+            entry_direction<NEST, GT, PRE>(sub, r, d + static_cast<size_t>(j) * slot_elems, s, pre, sp, su);
             sp = trust_warp_sum(sp);
             su = trust_warp_sum(su);
             if (lane == 0) {
@@ -391,7 +409,7 @@ novak_step_adapt_kernel(const int *__restrict__ item_first, const Chunk *__restr
     __syncwarp();                        // lane 0's acquire orders the whole warp's loads below
     word = __shfl_sync(0xffffffffu, word, 0);
     if (word == 0ull) return;            // (the update below has no CTA-wide barrier)
-    const float step = s.step * __uint_as_float(static_cast<unsigned>(word));      // Eq. 24a
+    const float step = step_all * __uint_as_float(static_cast<unsigned>(word));    // Eq. 24a
     entry_apply<LA, PRE>(ch_u, r_u, direction + static_cast<size_t>(c_u) * static_cast<size_t>(slot_elems),
                          s, step);
 }
@@ -424,7 +442,8 @@ void *pick_adapt_gt(int grad_dtype, int la)
     }
 }
 
-// Every instantiation for one mode (PRE_NONE with or without PRE_COPY16 and PRE_MOM16).
+// Every instantiation for one mode (PRE_NONE, PRE_SCALE or PRE_CENTER, with or without
+// PRE_COPY16 and PRE_MOM16).
 template <int PRE>
 void *pick_step_adapt_kernel(int nesterov, int grad_dtype, int la)
 {

@@ -5,7 +5,7 @@
 //   -DNOVAK_INST_DYN   for the graph-capturable kernel (scalars and lookahead
 //                      action read from device memory) instead of the plain one.
 //   -DNOVAK_INST_ADAPT for the kernel that runs layer adaptation and the update
-//                      as one persistent launch (PRE_NONE modes only).
+//                      in one launch (every mode but the row-owning ones).
 // Each object exports one selector: step_kernel_mode<N>, step_dyn_kernel_mode<N>
 // or step_adapt_kernel_mode<N>.
 #ifndef NOVAK_PRE_MODE

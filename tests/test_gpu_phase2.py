@@ -403,26 +403,31 @@ def test_layer_adaptation_every_element(gdtype, extra, variant):
     pair.check(f"layer adaptation {extra}")
     seen = np.array(pair.oracle.trust)
     assert (seen == 0.1).any() and (seen == 10.0).any() and ((seen > 0.1) & (seen < 10.0)).any()
-    # statistics and update in one launch unless the gradient is pre-processed as well
-    per_step = 5 if extra.get("centralize") or extra.get("clip_threshold") else 1
+    # statistics and update in one launch, behind the two kernels of the gradient's own statistics
+    per_step = 3 if extra.get("centralize") or extra.get("clip_threshold") else 1
     assert pair.opt.info()["launches"] == 7 * per_step
     assert pair.opt.info()["layer_adaptation"] == 1
 
 
 @pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("lead", [0, 20000, None])
+@pytest.mark.parametrize("lead,extra", [(0, {}), (20000, {}), (None, {}),
+                                        (None, dict(clip_threshold=0.05)),
+                                        (0, dict(clip_threshold=0.05, centralize=True)),
+                                        (None, dict(auto_lr=True, centralize=True))])
 @pytest.mark.parametrize("variant", [("approximation", "last", 5), ("classical", "traj_mean", 2),
                                      ("none", "last", 0)])
-def test_layer_adaptation_in_one_launch_equals_the_three_launch_form(gdtype, lead, variant):
-    """Statistics and update as items of one grid (the statistics `lead` elements ahead of
-    the updates: none at all, so that updates wait for their ratio, a few entries, the
-    default) against the two statistics kernels followed by the step: the same sums in the same order, so ratios, parameters
-    and state agree bit for bit, over 8 steps with bf16 parameter copies switched on; the
-    one-launch form is also held against the oracle."""
+def test_layer_adaptation_in_one_launch_equals_the_three_launch_form(gdtype, lead, extra, variant):
+    """Statistics and update in one grid (the updates trailing the statistics by what the
+    longest tensor needs plus `lead` elements) against the two statistics kernels followed
+    by the step: the same sums in the same order, so ratios, parameters and state agree bit
+    for bit, over 8 steps with bf16 parameter copies switched on, also behind clipping,
+    centralization and the automatic learning-rate scaling; the one-launch form is also
+    held against the oracle."""
     nesterov, mode, k = variant
     shapes = SHAPES + [(70001,), (3, 30000)]
     offsets = OFFSETS + [2, 0]
-    hyper = dict(BASE, nesterov=nesterov, lookahead_mode=mode, lookahead_k=k, layer_adaptation=True)
+    hyper = dict(BASE, nesterov=nesterov, lookahead_mode=mode, lookahead_k=k, layer_adaptation=True,
+                 **extra)
     numels = [math.prod(s) for s in shapes]
     sets = []
     for in_step in (1, 0):
@@ -453,7 +458,9 @@ def test_layer_adaptation_in_one_launch_equals_the_three_launch_form(gdtype, lea
         sa, sb = pair.opt.state(i), twin.state(i)
         for key in ("m", "v", "slow", "acc"):
             assert (sa[key] is None and sb[key] is None) or torch.equal(sa[key], sb[key])
-    assert pair.opt.info()["launches"] == 8 and twin.info()["launches"] == 24
+    # in front of both: the kernels of the gradient's own statistics where phase 2 is on
+    n_pre = 0 if not extra else (3 if extra.get("auto_lr") else 2)
+    assert pair.opt.info()["launches"] == 8 * (1 + n_pre) and twin.info()["launches"] == 8 * (3 + n_pre)
 
 
 def test_layer_adaptation_zero_gradient_and_reruns():
@@ -559,8 +566,8 @@ def test_auto_lr_every_element(gdtype, extra):
     pair.check(f"auto lr {extra}")
     seen = pair.oracle.auto_scales
     assert min(seen) == 0.1 and max(seen) == 2.0 and any(0.1 < s < 2.0 for s in seen)
-    per_step = 1 + 3 + (2 if extra.get("layer_adaptation") else 0)
-    assert pair.opt.info()["launches"] == 8 * per_step
+    # three statistics kernels, then the step (with layer adaptation: its one-launch form)
+    assert pair.opt.info()["launches"] == 8 * (1 + 3)
 
 
 def test_auto_lr_state_survives_a_checkpoint_and_a_change_of_rows():
