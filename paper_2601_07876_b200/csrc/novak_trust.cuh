@@ -1,7 +1,8 @@
 // Layer-wise adaptation (Eq. 19 / 25), device side shared by the two-kernel
-// pass (novak_trust_stats.cu) and by the step kernel that adapts in one launch
-// (novak_step_adapt.cuh): the sums of squares of theta_t and of this step's
-// base direction u_t over one chunk-table entry, and the ratio of a tensor.
+// pass (novak_trust_stats.cu: the sums of squares of theta_t and of this step's
+// base direction u_t over one chunk-table entry) and by the kernel that adapts
+// and steps in one launch (novak_step_adapt.cuh: the same block and warp sums,
+// the ratio of a tensor).
 //
 // u_t is the direction THIS step produces, so the moments are advanced exactly
 // as the step kernel will advance them (same device functions, same fp32
@@ -41,18 +42,16 @@ __device__ __forceinline__ double trust_block_sum(double x, double *sh)
 }
 
 // Squares of N parameters and of the N base directions their gradients give.
-// Each group of N squares is added in fp32, groups in double.  POL: cache
-// policy of the loads (LD_KEEP where the step kernel reads the same bytes
-// again shortly and should find them in L2).
-template <int N, int NEST, int GT, int PRE, int POL = LD_STREAM>
+// Each group of N squares is added in fp32, groups in double.
+template <int N, int NEST, int GT, int PRE>
 __device__ __forceinline__ void accumulate(const float *p, const void *g, const void *m,
                                            const void *v, int idx, const StepScalars &s,
                                            const PreArgs &pre, double &sum_p, double &sum_u)
 {
-    const Vec<N> P = load_f32<N, POL>(p, idx);
-    Vec<N> G = load_grad<N, GT, POL>(g, idx);
-    const Vec<N> M = load_moment<N, (PRE & PRE_MOM16) != 0, POL>(m, idx);
-    const Vec<N> V = load_moment<N, (PRE & PRE_MOM16) != 0, POL>(v, idx);
+    const Vec<N> P = load_f32<N>(p, idx);
+    Vec<N> G = load_grad<N, GT>(g, idx);
+    const Vec<N> M = load_moment<N, (PRE & PRE_MOM16) != 0>(m, idx);
+    const Vec<N> V = load_moment<N, (PRE & PRE_MOM16) != 0>(v, idx);
     preprocess<N, PRE>(G, row_position<PRE>(pre.elem0 + static_cast<uint32_t>(idx) * N, pre), pre);
     float sp = 0.0f, su = 0.0f;
 #pragma unroll
@@ -67,7 +66,7 @@ __device__ __forceinline__ void accumulate(const float *p, const void *g, const 
 }
 
 // The two sums over one chunk-table entry; thread 0 returns them in tp, tu.
-template <int NEST, int GT, int PRE, int POL = LD_STREAM>
+template <int NEST, int GT, int PRE>
 __device__ __forceinline__ void entry_trust_sums(const Chunk &ch, const TensorRec &r,
                                                  const StepScalars &s, const PreArgs &pre,
                                                  double *sh, double &tp, double &tu)
@@ -88,13 +87,13 @@ __device__ __forceinline__ void entry_trust_sums(const Chunk &ch, const TensorRe
         const int nvec = ch.len >> 2;
 #pragma unroll 2
         for (int i = threadIdx.x; i < nvec; i += kTrustBlock)
-            accumulate<4, NEST, GT, PRE, POL>(p, g, m, v, i, s, pre, sum_p, sum_u);
+            accumulate<4, NEST, GT, PRE>(p, g, m, v, i, s, pre, sum_p, sum_u);
         const int idx = (nvec << 2) + threadIdx.x;          // ragged tail: < 4 elements
-        if (idx < ch.len) accumulate<1, NEST, GT, PRE, POL>(p, g, m, v, idx, s, pre, sum_p, sum_u);
+        if (idx < ch.len) accumulate<1, NEST, GT, PRE>(p, g, m, v, idx, s, pre, sum_p, sum_u);
     } else {
 #pragma unroll 4
         for (int i = threadIdx.x; i < ch.len; i += kTrustBlock)
-            accumulate<1, NEST, GT, PRE, POL>(p, g, m, v, i, s, pre, sum_p, sum_u);
+            accumulate<1, NEST, GT, PRE>(p, g, m, v, i, s, pre, sum_p, sum_u);
     }
     tp = trust_block_sum(sum_p, sh);
     tu = trust_block_sum(sum_u, sh);
