@@ -126,13 +126,14 @@ struct Handle {
     int *tensor_first = nullptr;
     float *trust = nullptr;
     std::vector<int> h_tensor_first;
-    // layer adaptation and step in one launch: the claim-ordered item list, the
-    // kernel's counters and per-tensor flags (one allocation), a host-mapped error word
+    // layer adaptation and step in one launch: the item list, the kernel's counters
+    // and per-tensor words (one allocation), the directions of one step (another), a
+    // host-mapped error word
     int adapt_in_step = 1;              // NOVAK_OPT_LAYER_ADAPTATION_IN_STEP
     int64_t adapt_lead_elems = 0;          // NOVAK_OPT_LAYER_ADAPTATION_LEAD
     int adapt_group = 4;                   // NOVAK_OPT_LAYER_ADAPTATION_GROUP
     char *d_adapt = nullptr;
-    int *d_item_code = nullptr;
+    int *d_item_code = nullptr;         // every item's first chunk-table entry
     Chunk *d_item_chunk = nullptr;
     int n_items = 0;
     int adapt_lag = 0;                  // CTA b updates item b - adapt_lag

@@ -30,8 +30,12 @@
 // which has finished its own S part by then), and an S part never waits.  The
 // hardware hands out the CTAs of a grid in increasing block index as slots
 // become free (the behaviour single-pass scans with look-back rely on as well),
-// so those CTAs are running or have finished; with a lag beyond the number of
-// resident CTAs the word is normally there long before it is asked for.
+// so those CTAs are running or have finished, and the word is there when it is
+// asked for or shortly after (a longer lag makes the wait rarer but lets theta
+// and the direction leave L2 before the U part comes for them; measured, the
+// shortest lag is the fastest).  With gradient pre-processing on, the clip
+// factor, the row means and Eq. 22 come from the statistics pass in front of
+// this launch and the S part applies them to g first.
 // Nothing in the programming model promises that order, so the wait is
 // bounded: after about two seconds (at once, when another CTA has already given
 // up) a warp gives up, raises an error flag in host-mapped memory, leaves its
