@@ -494,6 +494,16 @@ int novak_get_grad_stats(novak_opt *opt, double *norm, double *factor, void *str
  * SYNCHRONISES `stream`.  NOVAK_ESTATE when no such step has run. */
 int novak_get_trust_ratios(novak_opt *opt, float *h_out, int n, void *stream);
 
+/* Test hook for the one place where a kernel of this library waits for another
+ * CTA (the update part of the one-launch layer adaptation waits for its tensor's
+ * ratio; see NOVAK_OPT_LAYER_ADAPTATION_IN_STEP).  Runs that wait, on `stream`, on
+ * a word that nothing publishes, and SYNCHRONISES: *gave_up = 1 when the wait
+ * returned empty-handed, *seconds = how long it waited on the device (about two
+ * seconds: the bound).  Allocates and frees 32 bytes of device memory.  Nothing
+ * else on the device is touched; the handle only supplies the device and the
+ * error text.  The paper has no counterpart. */
+int novak_selftest_bounded_wait(novak_opt *opt, int *gave_up, double *seconds, void *stream);
+
 /* True Nesterov momentum, Section 4.4 (Eq. 10-12) and Section 5.8 ("True
  * Nesterov closure").  The gradient of Eq. 11 is the caller's to compute; these
  * two calls do the parameter traffic around it for a handle created with

@@ -123,6 +123,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
                                             POINTER(c_double), vp]),
         "novak_set_auto_lr_state": (c_int, [vp, c_double, c_double]),
         "novak_get_trust_ratios": (c_int, [vp, POINTER(ctypes.c_float), c_int, vp]),
+        "novak_selftest_bounded_wait": (c_int, [vp, POINTER(c_int), POINTER(c_double), vp]),
         "novak_nesterov_save_bytes": (c_size_t, [vp]),
         "novak_nesterov_extrapolate": (c_int, [vp, vpp, vp, c_size_t, i64p, c_int, vp]),
         "novak_nesterov_restore": (c_int, [vp, vpp, vp, c_size_t, i64p, c_int, vp]),
@@ -359,6 +360,15 @@ class Handle:
         _check(self.lib, self.h, self.lib.novak_get_trust_ratios(self.h, out, n, stream),
                "novak_get_trust_ratios")
         return list(out)
+
+    def selftest_bounded_wait(self, stream: int = 0):
+        """Runs the one-launch layer adaptation's wait on a word nobody publishes:
+        (gave_up, seconds waited on the device).  Takes about two seconds."""
+        gave_up, seconds = c_int(-1), c_double(0.0)
+        _check(self.lib, self.h,
+               self.lib.novak_selftest_bounded_wait(self.h, byref(gave_up), byref(seconds), stream),
+               "novak_selftest_bounded_wait")
+        return bool(gave_up.value), float(seconds.value)
 
     def nesterov_save_bytes(self) -> int:
         return int(self.lib.novak_nesterov_save_bytes(self.h))

@@ -817,4 +817,27 @@ int novak_get_trust_ratios(novak_opt *o, float *h_out, int n, void *stream_)
     return NOVAK_OK;
 }
 
+int novak_selftest_bounded_wait(novak_opt *o, int *gave_up, double *seconds, void *stream_)
+{
+    if (!o) return NOVAK_EINVAL;
+    DeviceGuard on_device(o->device);
+    if (!gave_up || !seconds) return fail(o, NOVAK_EINVAL, "selftest_bounded_wait: NULL output");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // [0]: the word nobody publishes, [1]: the error word, [2..3]: the kernel's report
+    unsigned long long *d = nullptr;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&d), 4 * sizeof(unsigned long long));
+    if (e != cudaSuccess) return fail(o, NOVAK_ENOMEM, "selftest_bounded_wait: %s", cudaGetErrorString(e));
+    unsigned long long h[2] = {~0ull, 0ull};
+    if ((e = cudaMemsetAsync(d, 0, 4 * sizeof(unsigned long long), stream)) == cudaSuccess &&
+        (e = novak::launch_adapt_wait_probe(d, 1u, reinterpret_cast<const unsigned *>(d + 1), d + 2,
+                                            stream)) == cudaSuccess &&
+        (e = cudaMemcpyAsync(h, d + 2, sizeof h, cudaMemcpyDeviceToHost, stream)) == cudaSuccess)
+        e = cudaStreamSynchronize(stream);
+    cudaFree(d);
+    if (e != cudaSuccess) return fail_cuda(o, e, "selftest_bounded_wait");
+    *gave_up = h[0] == 0ull ? 1 : 0;
+    *seconds = static_cast<double>(h[1]) * 1e-9;
+    return NOVAK_OK;
+}
+
 }  // extern "C"

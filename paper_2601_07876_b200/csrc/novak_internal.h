@@ -74,6 +74,12 @@ cudaError_t launch_step_adapt(const int *item_first, const Chunk *item_chunk, in
                               const StepScalars &s, unsigned epoch, int nesterov, int grad_dtype,
                               int la, const LaunchCfg &cfg, cudaStream_t stream);
 
+// Runs that kernel's bounded wait on a word that nothing publishes (all zero, epoch
+// non-zero): out[0] receives what the wait returned (0: it gave up), out[1] the
+// nanoseconds it took.  error: a zero word in device memory.
+cudaError_t launch_adapt_wait_probe(const unsigned long long *word, unsigned epoch,
+                                    const unsigned *error, unsigned long long *out, cudaStream_t stream);
+
 // One unit of work of the statistics pass for a tensor with rows (Eq. 26).
 // Rows of up to kRowWarpMax elements: n_rows (a multiple of 8 but for a tensor's
 // last unit) whole rows starting at row0

@@ -97,6 +97,17 @@ __device__ __forceinline__ unsigned long long wait_for_ratio(const unsigned long
     return 0ull;
 }
 
+// The bound of that wait, on its own: one thread waits for a word that nothing
+// publishes and reports what it got (0: gave up) and how long it waited.
+__global__ void novak_adapt_wait_probe_kernel(const unsigned long long *word, unsigned epoch,
+                                              const unsigned *error, unsigned long long *out)
+{
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    const unsigned long long t0 = global_timer_ns();
+    out[0] = wait_for_ratio(word, epoch, error);
+    out[1] = global_timer_ns() - t0;
+}
+
 // ---- the direction a step applies, formed once -------------------------------
 // An S item advances the moments for good and leaves, element by element, the
 // direction the update multiplies by the step (Eq. 17 after the mask of Eq. 27

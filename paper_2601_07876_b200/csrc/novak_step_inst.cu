@@ -44,6 +44,16 @@ void *NOVAK_PASTE(step_adapt_kernel_mode, NOVAK_PRE_MODE)(int nesterov, int grad
     return pick_step_adapt_kernel<NOVAK_PRE_MODE>(nesterov, grad_dtype, la);
 }
 
+#if (NOVAK_PRE_MODE) == 0
+// The wait of the kernel's update part on its own (once in the library: this object).
+cudaError_t launch_adapt_wait_probe(const unsigned long long *word, unsigned epoch,
+                                    const unsigned *error, unsigned long long *out, cudaStream_t stream)
+{
+    novak_adapt_wait_probe_kernel<<<1, 32, 0, stream>>>(word, epoch, error, out);
+    return cudaGetLastError();
+}
+#endif
+
 }  // namespace novak
 #else
 #include "novak_step_kernel.cuh"

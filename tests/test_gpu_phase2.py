@@ -492,6 +492,25 @@ def test_layer_adaptation_zero_gradient_and_reruns():
         assert torch.equal(a, b)
 
 
+def test_the_update_part_gives_up_waiting_after_its_bound_and_the_device_stays_usable():
+    """The only wait on another CTA in the library (the update part of the one-launch layer
+    adaptation waits for its tensor's ratio) run on a word that nothing publishes: it returns
+    empty-handed after about two seconds instead of spinning on, and the same handle then
+    steps as usual."""
+    _, params = _shaped([(300, 40), (5000,)], [0, 0])
+    gen = _gen(5)
+    for p in params:
+        p.normal_(0.0, 0.1, generator=gen)
+    pair = Pair(params, dict(BASE, layer_adaptation=True))
+    gave_up, seconds = pair.opt.handle.selftest_bounded_wait(pair.opt._stream())
+    assert gave_up and 1.5 < seconds < 6.0
+    _, grads = _shaped([(300, 40), (5000,)], [0, 0])
+    for _ in range(3):
+        _fill_grads(grads, gen, std=1e-2)
+        pair.step(grads)
+    pair.check("after the bounded wait")
+
+
 # ---------------------------------------------------------------------------
 # Phase 8: sparse updates (Eq. 27)
 # ---------------------------------------------------------------------------
